@@ -1,0 +1,191 @@
+/*
+ * lopro.h -- C ABI of the LoPRo quantized-linear forward for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, for a linear layer W in R^{m x n} (m = d_out, n = d_in) that was
+ * quantized with LoPRo, the forward of Eq. 8 of the paper,
+ *
+ *        y = W_r x + Qz(R') Q^T P^T x ,        W_r = A B ,   R' = (W - W_r) P Q ,
+ *
+ * where P is the column permutation built from the index vector `perm` (Eq. 5), Q the partial
+ * block-wise Walsh-Hadamard matrix diag(I_{b_I}, H_wal, ..., H_wal) with blocks of size b_H
+ * (Eq. 6, Hadamard recursion of Eq. 2), Qz(R') the group-quantized residual stored as d_q-bit
+ * codes with one fp16 scale and one fp16 zero-point per group of g consecutive rotated columns
+ * (Appendix A.2), and A = U Sigma [m][r], B = V alpha^-1 [r][n] the folded rank-r factors
+ * (Eq. 4).  The steps are those of Appendix A.3: permutation, fast Walsh-Hadamard transform,
+ * dequantize-and-multiply, the two skinny low-rank products, and the sum.
+ *
+ * Conventions
+ *   - Activations hold one token per row: x[T][ldx] bf16 (the paper writes tokens as the
+ *     columns of X in R^{n x b}).  Outputs y[T][ldy], bf16 or fp32.
+ *   - Permutation is a gather: (P^T x)[k] = x[perm[k]].
+ *   - Dequantization: W^[i][k] = scale[i][k / g] * (code[i][k] - zero[i][k / g]); column k
+ *     is a column of the permuted and rotated basis.
+ *   - 16-bit floats cross the ABI as their bit patterns (uint16_t).
+ *   - Unless a parameter says "host", every array pointer is a DEVICE pointer that the caller
+ *     owns.  The library allocates no memory, frees nothing and never synchronises the
+ *     stream, except where an entry point says so.  `stream` is a cudaStream_t passed as
+ *     void* (NULL = the default stream).  All work is enqueued on the current device.
+ *   - Every entry point validates its arguments on the host and returns a status; none
+ *     aborts, exits or traps the GPU.  Asynchronous device-side conditions are reported
+ *     through the status word at the start of the workspace (see lopro_linear_fwd).
+ *   - There is no CPU fallback: without a usable CUDA device the calls return
+ *     LOPRO_ERR_CUDA.
+ */
+#ifndef LOPRO_H_
+#define LOPRO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define LOPRO_API __attribute__((visibility("default")))
+#else
+#define LOPRO_API
+#endif
+
+typedef enum {
+    LOPRO_OK = 0,
+    LOPRO_ERR_INVALID_ARG = 1,      /* null pointer, bad size, misaligned pointer, bad descriptor  */
+    LOPRO_ERR_UNSUPPORTED = 2,      /* legal by the method but outside what the kernels cover     */
+    LOPRO_ERR_BUFFER_TOO_SMALL = 3, /* packed blob or workspace smaller than required             */
+    LOPRO_ERR_CUDA = 4,             /* a CUDA runtime call failed (no device, launch failure ...)  */
+    LOPRO_ERR_TIMEOUT = 5,          /* a bounded device-side wait expired (status word only)      */
+    LOPRO_ERR_INVALID_DATA = 6      /* lopro_pack: perm is no permutation, code out of range,
+                                       non-finite or zero scale, non-finite zero-point           */
+} lopro_status;
+
+/* Output element types of lopro_linear_fwd. */
+enum { LOPRO_OUT_BF16 = 0, LOPRO_OUT_F32 = 1 };
+
+/* Code layouts inside the packed blob. */
+enum {
+    LOPRO_LAYOUT_CANONICAL = 0, /* per row, code k occupies bits [k q, (k+1) q) of a little-endian
+                                   bit stream stored as uint32 words (4-bit: 8 codes per word, low
+                                   nibble first); interchange format, not accepted by the forward */
+    LOPRO_LAYOUT_FRAGMENT = 1   /* tensor-core fragment order read by the forward kernels         */
+};
+
+/* Descriptor of one quantized layer (plain data, host memory).
+ *   d_in  = n, multiple of 64;  d_out = m, multiple of 16;
+ *   bits  = d_q in {2, 3, 4};   group_size = g = 64 * 2^k (64, 128, 256, ...) dividing d_in;
+ *   block_size = b_H, a power of two in [2, 1024];
+ *   identity_cols = b_I >= 0 with (d_in - b_I) a multiple of b_H (Eq. 6); b_I = d_in disables
+ *   the rotation;  rank = r in [0, 512] (stored padded with zeros to a multiple of 16). */
+typedef struct {
+    int32_t d_in;
+    int32_t d_out;
+    int32_t bits;
+    int32_t group_size;
+    int32_t block_size;
+    int32_t identity_cols;
+    int32_t rank;
+    int32_t layout;
+} lopro_desc;
+
+/* Sections of the packed blob, for lopro_packed_section. */
+enum {
+    LOPRO_SEC_HEADER = 0,
+    LOPRO_SEC_CODES = 1,  /* packed codes in the descriptor's layout                               */
+    LOPRO_SEC_SCALEZERO = 2, /* (scale, zero) fp16 pairs: canonical [m][n/g]; fragment layout
+                                [m/16][n/g][16]                                                    */
+    LOPRO_SEC_PERM = 3,   /* int32 [n]                                                             */
+    LOPRO_SEC_A = 4,      /* fp16 [m][r_pad]                                                       */
+    LOPRO_SEC_B = 5,      /* fp16 [r_pad][n]                                                       */
+    LOPRO_SEC_COUNT = 6
+};
+
+/* Library version (major * 10000 + minor * 100 + patch). */
+LOPRO_API int lopro_version(void);
+
+/* Static, human-readable name of a status code. */
+LOPRO_API const char* lopro_status_str(lopro_status s);
+
+/* LOPRO_OK if the descriptor is inside the domain stated above, else the reason class. */
+LOPRO_API lopro_status lopro_check_desc(const lopro_desc* desc);
+
+/* Size in bytes of the packed blob of a layer (0 for an invalid descriptor).  The blob is a
+ * flat, relocatable byte buffer: a 256-byte header followed by 256-byte aligned sections;
+ * copying it (device to device, to the host, to a file) copies the layer.  Its size follows
+ * the storage accounting of Eq. 13 with this library's widths: d_q bits per code, 2 x 16 bits
+ * per group (scale and zero-point), 16 bits per factor entry, 32 bits per permutation entry. */
+LOPRO_API size_t lopro_packed_bytes(const lopro_desc* desc);
+
+/* Offset and size in bytes of one section of the blob.  Returns LOPRO_ERR_INVALID_ARG for a
+ * bad descriptor or section id. */
+LOPRO_API lopro_status lopro_packed_section(const lopro_desc* desc, int32_t section, size_t* offset, size_t* bytes);
+
+/* Bytes of device workspace lopro_linear_fwd needs for up to T tokens (0 on bad arguments).
+ * Monotone in T. */
+LOPRO_API size_t lopro_workspace_bytes(const lopro_desc* desc, int32_t T);
+
+/* Build the packed blob from plain arrays -- the record (W_q, U, V, Sigma, p, s) that
+ * Algorithm 1 saves, with U Sigma and V diag(s)^-1 folded into A and B (Eq. 4).
+ *   codes      uint8 [m][n], one code per byte, columns in permuted-and-rotated order
+ *   scales_f16 fp16  [m][n/g]        zeros_f16  fp16 [m][n/g] (code units, any finite value)
+ *   perm       int32 [n]             A_f16 fp16 [m][r]        B_f16 fp16 [r][n]  (NULL if r = 0)
+ *   packed     output blob of packed_bytes >= lopro_packed_bytes(desc), 256-byte aligned
+ * The inputs are validated on the device: perm must be a bijection of [0, n), every code
+ * < 2^bits, every scale finite and non-zero, every zero-point finite; otherwise
+ * LOPRO_ERR_INVALID_DATA is returned and the blob content is unspecified.  This entry point
+ * SYNCHRONISES the stream once (to read the validation result); it is a one-time set-up step. */
+LOPRO_API lopro_status lopro_pack(const lopro_desc* desc, const uint8_t* codes, const uint16_t* scales_f16,
+                        const uint16_t* zeros_f16, const int32_t* perm, const uint16_t* A_f16,
+                        const uint16_t* B_f16, void* packed, size_t packed_bytes, void* stream);
+
+/* Exact inverse of lopro_pack for either layout: writes the arrays lopro_pack was given, bit
+ * for bit.  Any output pointer may be NULL to skip that array.  `words` (optional) receives
+ * the codes as the canonical uint32 bit stream [m][n*bits/32] regardless of the blob's layout.
+ * Checks the blob header against `desc` (one small synchronous device-to-host copy) and returns
+ * LOPRO_ERR_INVALID_DATA on a mismatch. */
+LOPRO_API lopro_status lopro_unpack(const lopro_desc* desc, const void* packed, uint8_t* codes, uint32_t* words,
+                          uint16_t* scales_f16, uint16_t* zeros_f16, int32_t* perm, uint16_t* A_f16,
+                          uint16_t* B_f16, void* stream);
+
+/* Activation-side transform of Eq. 8: xrot[t] = Q^T P^T x[t] for T token rows (Appendix A.3:
+ * O(n) gather, then log2(b_H) butterfly stages per Hadamard block; Hadamard matrix in the
+ * natural order of the recursion of Eq. 2, normalised by 1/sqrt(b_H); the first b_I entries
+ * are only permuted).  Butterflies run in fp32, the result is rounded once to bf16.
+ *   perm int32 [n] (a section of the blob or any other device array);
+ *   x bf16 [T][ldx], xrot bf16 [T][ldo], ldx, ldo >= n; x and xrot 16-byte aligned with ldx
+ *   and ldo multiples of 8; x and xrot must not overlap.  Uses d_in, block_size and
+ *   identity_cols of the descriptor only.  T = 0 is a no-op. */
+LOPRO_API lopro_status lopro_rotate(const lopro_desc* desc, const int32_t* perm, const uint16_t* x_bf16, int64_t ldx,
+                          uint16_t* xrot_bf16, int64_t ldo, int32_t T, void* stream);
+
+/* Forward of the quantized layer (Eq. 8; steps of Appendix A.3):
+ *        y[t] = A (B x[t]) + W^ (Q^T P^T x[t])           for t in [0, T).
+ *   packed    blob written by lopro_pack with LOPRO_LAYOUT_FRAGMENT, 256-byte aligned
+ *   x         bf16 [T][ldx], 16-byte aligned, ldx >= n and a multiple of 8
+ *   y         bf16 or fp32 [T][ldy] per out_dtype, ldy >= m; must not overlap x
+ *   workspace at least lopro_workspace_bytes(desc, T) bytes, 256-byte aligned; scratch for the
+ *             rotated activations, the low-rank intermediate and split-K partial sums.  Its
+ *             first 4 bytes are a status word: it is set to LOPRO_OK when the call starts and a
+ *             kernel that gives up on a bounded wait stores LOPRO_ERR_TIMEOUT there (read it
+ *             after synchronising).  Calls that share a workspace must be ordered on one stream.
+ * Arithmetic: rotated activations rounded to bf16; the code-times-activation products are
+ * accumulated in fp32 (tensor cores), scales and zero-points applied in fp32; B x accumulated in
+ * fp32 and rounded to fp16; A times that accumulated in fp32 into the same sum; one final
+ * rounding to the output type.  T = 0 is a no-op. */
+LOPRO_API lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const uint16_t* x_bf16, int64_t ldx,
+                              void* y, int64_t ldy, int32_t out_dtype, int32_t T, void* workspace,
+                              size_t workspace_bytes, void* stream);
+
+/* The same forward for callers whose activations live in HOST memory (Eq. 8 end to end):
+ * copies x_host [T][n] (dense, bf16; pinned memory makes the copy asynchronous) to the device,
+ * runs lopro_linear_fwd and copies y [T][m] back to y_host.  `workspace` must hold
+ * lopro_workspace_bytes(desc, T) + lopro_host_staging_bytes(desc, T, out_dtype) bytes.  The call
+ * enqueues everything on `stream` and does not synchronise; y_host is valid after the caller
+ * synchronises the stream. */
+LOPRO_API size_t lopro_host_staging_bytes(const lopro_desc* desc, int32_t T, int32_t out_dtype);
+LOPRO_API lopro_status lopro_linear_fwd_host(const lopro_desc* desc, const void* packed, const uint16_t* x_host,
+                                   void* y_host, int32_t out_dtype, int32_t T, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOPRO_H_ */

@@ -1,0 +1,296 @@
+// Host side of the C ABI: argument validation, blob and workspace layout, dispatch.
+#include <stdlib.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace lopro {
+
+lopro_status check_desc(const lopro_desc& d) {
+    if (d.d_in <= 0 || d.d_out <= 0) return LOPRO_ERR_INVALID_ARG;
+    if (d.bits != 2 && d.bits != 3 && d.bits != 4) return LOPRO_ERR_INVALID_ARG;
+    if (d.group_size <= 0 || d.d_in % d.group_size != 0) return LOPRO_ERR_INVALID_ARG;
+    if (d.block_size < 2 || d.block_size > 1024 || (d.block_size & (d.block_size - 1))) return LOPRO_ERR_INVALID_ARG;
+    if (d.identity_cols < 0 || d.identity_cols > d.d_in) return LOPRO_ERR_INVALID_ARG;
+    if ((d.d_in - d.identity_cols) % d.block_size != 0) return LOPRO_ERR_INVALID_ARG;
+    if (d.rank < 0 || d.rank > 512) return LOPRO_ERR_INVALID_ARG;
+    if (d.layout != LOPRO_LAYOUT_CANONICAL && d.layout != LOPRO_LAYOUT_FRAGMENT) return LOPRO_ERR_INVALID_ARG;
+    // Kernel coverage: 64-column steps, 16-row tiles, rows short enough for one CTA's shared memory.
+    if (d.d_in % 64 != 0 || d.d_out % 16 != 0 || d.group_size % 64 != 0) return LOPRO_ERR_UNSUPPORTED;
+    if ((d.group_size / 64) & (d.group_size / 64 - 1)) return LOPRO_ERR_UNSUPPORTED;  // g = 64 * 2^k
+    if (d.d_in > 32768 || d.d_out > (1 << 20)) return LOPRO_ERR_UNSUPPORTED;
+    return LOPRO_OK;
+}
+
+lopro_status blob_layout(const lopro_desc& d, BlobLayout* out) {
+    lopro_status st = check_desc(d);
+    if (st != LOPRO_OK) return st;
+    const size_t m = d.d_out, n = d.d_in, ng = d.d_in / d.group_size;
+    const int r_pad = round_up_int(d.rank, 16);
+    size_t bytes[LOPRO_SEC_COUNT];
+    bytes[LOPRO_SEC_HEADER] = kHeaderBytes;
+    bytes[LOPRO_SEC_CODES] = m * n * (size_t)d.bits / 8;
+    bytes[LOPRO_SEC_SCALEZERO] = m * ng * 4;
+    bytes[LOPRO_SEC_PERM] = n * 4;
+    bytes[LOPRO_SEC_A] = m * (size_t)r_pad * 2;
+    bytes[LOPRO_SEC_B] = (size_t)r_pad * n * 2;
+    size_t off = 0;
+    for (int s = 0; s < LOPRO_SEC_COUNT; ++s) {
+        out->off[s] = off;
+        out->bytes[s] = bytes[s];
+        off = round_up_size(off + bytes[s], kSectionAlign);
+    }
+    out->total = off;
+    out->r_pad = r_pad;
+    return LOPRO_OK;
+}
+
+// Split-K factor of the small-batch kernel: enough CTAs to cover the SMs about twice, K slices
+// that are whole groups and at least 256 columns long.
+int decode_split(const lopro_desc& d, int T) {
+    static int forced = -1;
+    if (forced < 0) {
+        const char* e = getenv("LOPRO_DECODE_SPLIT");
+        forced = e ? atoi(e) : 0;
+    }
+    const int mt = (d.d_out + 127) / 128;
+    const int zc = (T + kDecodeMaxT - 1) / kDecodeMaxT;
+    int split = 1;
+    if (forced > 0) {
+        split = forced;
+    } else {
+        while (split < kDecodeMaxSplit && mt * zc * split < 2 * 148) split *= 2;
+    }
+    const int unit = d.group_size > 512 ? d.group_size : 512;
+    while (split > 1 && (d.d_in % (split * unit) != 0)) split /= 2;
+    if (split > kDecodeMaxSplit) split = kDecodeMaxSplit;
+    while (split > 1 && (d.d_in % (split * d.group_size) != 0)) split /= 2;
+    if (zc > 1) split = 1;  // many tokens: the token chunks already fill the machine
+    return split;
+}
+
+lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
+    lopro_status st = check_desc(d);
+    if (st != LOPRO_OK) return st;
+    if (T < 0) return LOPRO_ERR_INVALID_ARG;
+    const int t_pad = round_up_int(T > 0 ? T : 1, 8);
+    const int r_pad = round_up_int(d.rank, 16);
+    size_t off = 0;
+    W->t_pad = t_pad;
+    W->off_status = off;
+    off += 256;
+    W->max_tickets = kMaxTickets;
+    W->off_tickets = off;
+    off += round_up_size((size_t)kMaxTickets * 4, 256);
+    W->off_xrot = off;
+    off += round_up_size((size_t)t_pad * d.d_in * 2, 256);
+    W->off_s64 = off;
+    off += round_up_size((size_t)t_pad * (d.d_in / 64) * 4, 256);
+    W->off_t = off;
+    off += round_up_size((size_t)t_pad * (r_pad > 0 ? r_pad : 16) * 2, 256);
+    W->off_partial = off;
+    // Partial sums exist only while one launch covers all tokens (T <= 32); sized for the
+    // largest split so that the size does not depend on tuning.
+    const int tp = t_pad < kDecodeMaxT ? t_pad : kDecodeMaxT;
+    W->partial_bytes = (size_t)kDecodeMaxSplit * tp * d.d_out * 4;
+    off += round_up_size(W->partial_bytes, 256);
+    W->total = off;
+    return LOPRO_OK;
+}
+
+static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+}  // namespace lopro
+
+using namespace lopro;
+
+extern "C" {
+
+int lopro_version(void) { return 100; }
+
+const char* lopro_status_str(lopro_status s) {
+    switch (s) {
+        case LOPRO_OK: return "ok";
+        case LOPRO_ERR_INVALID_ARG: return "invalid argument";
+        case LOPRO_ERR_UNSUPPORTED: return "unsupported configuration";
+        case LOPRO_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case LOPRO_ERR_CUDA: return "CUDA error";
+        case LOPRO_ERR_TIMEOUT: return "device-side wait timed out";
+        case LOPRO_ERR_INVALID_DATA: return "invalid layer data";
+    }
+    return "unknown status";
+}
+
+lopro_status lopro_check_desc(const lopro_desc* desc) {
+    if (!desc) return LOPRO_ERR_INVALID_ARG;
+    return check_desc(*desc);
+}
+
+size_t lopro_packed_bytes(const lopro_desc* desc) {
+    BlobLayout L;
+    if (!desc || blob_layout(*desc, &L) != LOPRO_OK) return 0;
+    return L.total;
+}
+
+lopro_status lopro_packed_section(const lopro_desc* desc, int32_t section, size_t* offset, size_t* bytes) {
+    BlobLayout L;
+    if (!desc || section < 0 || section >= LOPRO_SEC_COUNT) return LOPRO_ERR_INVALID_ARG;
+    lopro_status st = blob_layout(*desc, &L);
+    if (st != LOPRO_OK) return st;
+    if (offset) *offset = L.off[section];
+    if (bytes) *bytes = L.bytes[section];
+    return LOPRO_OK;
+}
+
+size_t lopro_workspace_bytes(const lopro_desc* desc, int32_t T) {
+    WorkspaceLayout W;
+    if (!desc || workspace_layout(*desc, T, &W) != LOPRO_OK) return 0;
+    return W.total;
+}
+
+lopro_status lopro_pack(const lopro_desc* desc, const uint8_t* codes, const uint16_t* scales_f16,
+                        const uint16_t* zeros_f16, const int32_t* perm, const uint16_t* A_f16,
+                        const uint16_t* B_f16, void* packed, size_t packed_bytes, void* stream) {
+    if (!desc) return LOPRO_ERR_INVALID_ARG;
+    BlobLayout L;
+    lopro_status st = blob_layout(*desc, &L);
+    if (st != LOPRO_OK) return st;
+    if (!codes || !scales_f16 || !zeros_f16 || !perm || !packed) return LOPRO_ERR_INVALID_ARG;
+    if (desc->rank > 0 && (!A_f16 || !B_f16)) return LOPRO_ERR_INVALID_ARG;
+    if (!aligned(packed, 256)) return LOPRO_ERR_INVALID_ARG;
+    if (packed_bytes < L.total) return LOPRO_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t s = (cudaStream_t)stream;
+
+    BlobHeader h;
+    memset(&h, 0, sizeof(h));
+    h.magic = kBlobMagic;
+    h.version = kBlobVersion;
+    h.desc = *desc;
+    h.total_bytes = L.total;
+    for (int i = 0; i < LOPRO_SEC_COUNT; ++i) {
+        h.sec_off[i] = L.off[i];
+        h.sec_bytes[i] = L.bytes[i];
+    }
+    // Zero the whole blob (padding bytes included, so that equal layers give equal blobs), then
+    // the header.  The header source is on this stack frame: the copy below is synchronous with
+    // respect to the host for pageable memory, and the stream is synchronised before returning.
+    if (cudaMemsetAsync(packed, 0, L.total, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (cudaMemcpyAsync(packed, &h, sizeof(h), cudaMemcpyHostToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (launch_validate(*desc, codes, scales_f16, zeros_f16, perm, packed, L, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (launch_pack(*desc, codes, scales_f16, zeros_f16, perm, A_f16, B_f16, packed, L, s) != cudaSuccess)
+        return LOPRO_ERR_CUDA;
+    BlobHeader back;
+    if (cudaMemcpyAsync(&back, packed, sizeof(back), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (back.magic != kBlobMagic) return LOPRO_ERR_CUDA;
+    if (back.invalid != 0) return LOPRO_ERR_INVALID_DATA;
+    return LOPRO_OK;
+}
+
+lopro_status lopro_unpack(const lopro_desc* desc, const void* packed, uint8_t* codes, uint32_t* words,
+                          uint16_t* scales_f16, uint16_t* zeros_f16, int32_t* perm, uint16_t* A_f16,
+                          uint16_t* B_f16, void* stream) {
+    if (!desc || !packed) return LOPRO_ERR_INVALID_ARG;
+    BlobLayout L;
+    lopro_status st = blob_layout(*desc, &L);
+    if (st != LOPRO_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    BlobHeader h;
+    if (cudaMemcpyAsync(&h, packed, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (h.magic != kBlobMagic || h.version != kBlobVersion || memcmp(&h.desc, desc, sizeof(lopro_desc)) != 0 ||
+        h.total_bytes != L.total || h.invalid != 0)
+        return LOPRO_ERR_INVALID_DATA;
+    if (launch_unpack(*desc, packed, L, codes, words, scales_f16, zeros_f16, perm, A_f16, B_f16, s) != cudaSuccess)
+        return LOPRO_ERR_CUDA;
+    return LOPRO_OK;
+}
+
+lopro_status lopro_rotate(const lopro_desc* desc, const int32_t* perm, const uint16_t* x_bf16, int64_t ldx,
+                          uint16_t* xrot_bf16, int64_t ldo, int32_t T, void* stream) {
+    if (!desc) return LOPRO_ERR_INVALID_ARG;
+    lopro_status st = check_desc(*desc);
+    if (st != LOPRO_OK) return st;
+    if (T < 0) return LOPRO_ERR_INVALID_ARG;
+    if (T == 0) return LOPRO_OK;
+    if (!perm || !x_bf16 || !xrot_bf16) return LOPRO_ERR_INVALID_ARG;
+    if (ldx < desc->d_in || ldo < desc->d_in || (ldx % 8) || (ldo % 8)) return LOPRO_ERR_INVALID_ARG;
+    if (!aligned(x_bf16, 16) || !aligned(xrot_bf16, 16) || !aligned(perm, 4)) return LOPRO_ERR_INVALID_ARG;
+    cudaError_t e = launch_rotate(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, (__nv_bfloat16*)xrot_bf16, ldo,
+                                  nullptr, T, (cudaStream_t)stream);
+    return e == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
+}
+
+lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const uint16_t* x_bf16, int64_t ldx,
+                              void* y, int64_t ldy, int32_t out_dtype, int32_t T, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+    if (!desc) return LOPRO_ERR_INVALID_ARG;
+    BlobLayout L;
+    lopro_status st = blob_layout(*desc, &L);
+    if (st != LOPRO_OK) return st;
+    if (desc->layout != LOPRO_LAYOUT_FRAGMENT) return LOPRO_ERR_UNSUPPORTED;
+    if (T < 0 || (out_dtype != LOPRO_OUT_BF16 && out_dtype != LOPRO_OUT_F32)) return LOPRO_ERR_INVALID_ARG;
+    if (T == 0) return LOPRO_OK;
+    if (!packed || !x_bf16 || !y || !workspace) return LOPRO_ERR_INVALID_ARG;
+    if (ldx < desc->d_in || (ldx % 8) || ldy < desc->d_out) return LOPRO_ERR_INVALID_ARG;
+    if (!aligned(packed, 256) || !aligned(workspace, 256) || !aligned(x_bf16, 16) ||
+        !aligned(y, out_dtype == LOPRO_OUT_F32 ? 4 : 2))
+        return LOPRO_ERR_INVALID_ARG;
+    WorkspaceLayout W;
+    st = workspace_layout(*desc, T, &W);
+    if (st != LOPRO_OK) return st;
+    if (workspace_bytes < W.total) return LOPRO_ERR_BUFFER_TOO_SMALL;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t* ws = (uint8_t*)workspace;
+    const uint8_t* blob = (const uint8_t*)packed;
+    // Status word and split-K tickets start at zero.
+    if (cudaMemsetAsync(ws, 0, W.off_xrot, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    const int32_t* perm = (const int32_t*)(blob + L.off[LOPRO_SEC_PERM]);
+    __nv_bfloat16* xrot = (__nv_bfloat16*)(ws + W.off_xrot);
+    float* s64 = (float*)(ws + W.off_s64);
+    if (launch_rotate(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, xrot, desc->d_in, s64, T, s) != cudaSuccess)
+        return LOPRO_ERR_CUDA;
+    if (desc->rank > 0) {
+        if (launch_lowrank_down(*desc, (const __half*)(blob + L.off[LOPRO_SEC_B]), L.r_pad,
+                                (const __nv_bfloat16*)x_bf16, ldx, (__half*)(ws + W.off_t), T, s) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
+    }
+    if (launch_decode(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    return LOPRO_OK;
+}
+
+size_t lopro_host_staging_bytes(const lopro_desc* desc, int32_t T, int32_t out_dtype) {
+    if (!desc || check_desc(*desc) != LOPRO_OK || T < 0) return 0;
+    const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;
+    return round_up_size((size_t)T * desc->d_in * 2, 256) + round_up_size((size_t)T * desc->d_out * esz, 256);
+}
+
+lopro_status lopro_linear_fwd_host(const lopro_desc* desc, const void* packed, const uint16_t* x_host,
+                                   void* y_host, int32_t out_dtype, int32_t T, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+    if (!desc) return LOPRO_ERR_INVALID_ARG;
+    if (out_dtype != LOPRO_OUT_BF16 && out_dtype != LOPRO_OUT_F32) return LOPRO_ERR_INVALID_ARG;
+    WorkspaceLayout W;
+    lopro_status st = workspace_layout(*desc, T, &W);
+    if (st != LOPRO_OK) return st;
+    if (T == 0) return LOPRO_OK;
+    if (!x_host || !y_host || !workspace) return LOPRO_ERR_INVALID_ARG;
+    const size_t stage = lopro_host_staging_bytes(desc, T, out_dtype);
+    if (workspace_bytes < W.total + stage) return LOPRO_ERR_BUFFER_TOO_SMALL;
+    if (!aligned(workspace, 256)) return LOPRO_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;
+    uint8_t* xd = (uint8_t*)workspace + W.total;
+    uint8_t* yd = xd + round_up_size((size_t)T * desc->d_in * 2, 256);
+    if (cudaMemcpyAsync(xd, x_host, (size_t)T * desc->d_in * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return LOPRO_ERR_CUDA;
+    st = lopro_linear_fwd(desc, packed, (const uint16_t*)xd, desc->d_in, yd, desc->d_out, out_dtype, T, workspace,
+                          W.total, stream);
+    if (st != LOPRO_OK) return st;
+    if (cudaMemcpyAsync(y_host, yd, (size_t)T * desc->d_out * esz, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return LOPRO_ERR_CUDA;
+    return LOPRO_OK;
+}
+
+}  // extern "C"

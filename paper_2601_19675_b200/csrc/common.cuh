@@ -1,0 +1,136 @@
+// Internal declarations shared by the translation units of liblopro (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lopro.h"
+
+namespace lopro {
+
+constexpr uint32_t kBlobMagic = 0x4F52504Cu;  // "LPRO"
+constexpr uint32_t kBlobVersion = 1;
+constexpr int kHeaderBytes = 256;
+constexpr int kSectionAlign = 256;
+
+// Header at offset 0 of the packed blob (256 bytes reserved).
+struct BlobHeader {
+    uint32_t magic;
+    uint32_t version;
+    lopro_desc desc;
+    uint64_t total_bytes;
+    uint64_t sec_off[LOPRO_SEC_COUNT];
+    uint64_t sec_bytes[LOPRO_SEC_COUNT];
+    uint32_t invalid;  // validation flags written by lopro_pack's check kernels (0 = clean)
+    uint32_t reserved[3];
+};
+static_assert(sizeof(BlobHeader) <= kHeaderBytes, "header must fit its slot");
+
+enum : uint32_t {
+    kInvalidPermRange = 1u,
+    kInvalidPermDuplicate = 2u,
+    kInvalidCode = 4u,
+    kInvalidScale = 8u,
+    kInvalidZero = 16u,
+};
+
+struct BlobLayout {
+    size_t off[LOPRO_SEC_COUNT];
+    size_t bytes[LOPRO_SEC_COUNT];
+    size_t total;
+    int r_pad;
+};
+
+// Host: validates the descriptor and fills the section table.
+lopro_status check_desc(const lopro_desc& d);
+lopro_status blob_layout(const lopro_desc& d, BlobLayout* out);
+
+inline int round_up_int(int v, int a) { return (v + a - 1) / a * a; }
+inline size_t round_up_size(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Workspace of lopro_linear_fwd: status word, split-K tickets, rotated activations, 64-column
+// sums of the rotated activations, low-rank intermediate, split-K partial sums.
+struct WorkspaceLayout {
+    size_t off_status, off_tickets, off_xrot, off_s64, off_t, off_partial, total;
+    int t_pad;       // tokens padded to a multiple of 8
+    int max_tickets;
+    size_t partial_bytes;
+};
+constexpr int kMaxTickets = 4096;
+constexpr int kDecodeMaxT = 32;      // tokens per launch of the small-batch kernel
+constexpr int kDecodeMaxSplit = 16;  // upper bound of the split-K factor
+lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* out);
+// Split-K factor the small-batch kernel uses for T tokens (host).
+int decode_split(const lopro_desc& d, int T);
+
+// ---- launchers (each returns the CUDA status of its launches) -------------------------------
+cudaError_t launch_validate(const lopro_desc& d, const uint8_t* codes, const uint16_t* scales,
+                            const uint16_t* zeros, const int32_t* perm, void* blob, const BlobLayout& L,
+                            cudaStream_t s);
+cudaError_t launch_pack(const lopro_desc& d, const uint8_t* codes, const uint16_t* scales, const uint16_t* zeros,
+                        const int32_t* perm, const uint16_t* A, const uint16_t* B, void* blob,
+                        const BlobLayout& L, cudaStream_t s);
+cudaError_t launch_unpack(const lopro_desc& d, const void* blob, const BlobLayout& L, uint8_t* codes,
+                          uint32_t* words, uint16_t* scales, uint16_t* zeros, int32_t* perm, uint16_t* A,
+                          uint16_t* B, cudaStream_t s);
+// Rotation; s64 (optional) receives the sums of each aligned run of 64 rotated (bf16-rounded)
+// entries, [T][n/64] fp32.
+cudaError_t launch_rotate(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
+                          __nv_bfloat16* xrot, int64_t ldo, float* s64, int T, cudaStream_t s);
+// t[T][r_pad] (fp16) = B x, fp32 accumulation.
+cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,
+                                int64_t ldx, __half* t, int T, cudaStream_t s);
+// Small-batch forward over the fragment layout (T tokens, any T: processed 32 at a time).
+cudaError_t launch_decode(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
+                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
+
+// ---- fragment layout ----------------------------------------------------------------------
+// Codes are stored per tile of 16 rows x 64 columns as [32 lanes][q words].  Lane l = 4 gq + tg
+// owns, for each of the four 16-column sub-steps j, the four register pairs rho = 0..3 of the
+// A operand of mma.m16n8k16:  row = gq + 8 (rho & 1),  column = 16 j + 8 (rho >> 1) + 2 tg + h,
+// h = 0 (low half) or 1 (high half).  Pair index pi = 4 j + rho.
+//   4-bit: word j;      low code at bit 4 rho,       high code at bit 16 + 4 rho
+//   2-bit: word pi / 8; low code at bit 2 (pi % 8),  high code at bit 16 + 2 (pi % 8)
+//   3-bit: pi < 15: word pi / 5, low at bit 3 (pi % 5), high at bit 16 + 3 (pi % 5);
+//          pi = 15: bit b of the low code is bit 15 of word b, of the high code bit 31 of word b.
+struct FragPos {
+    size_t word;     // index of the uint32 inside the blob's code section
+    uint32_t shift;  // bit position of the code's bit 0 (2- and 4-bit, 3-bit with pi < 15)
+    bool scattered;  // 3-bit pi = 15: bit b lives at bit `shift` of word + b
+};
+
+__host__ __device__ inline FragPos frag_pos(int bits, int n, int row, int k) {
+    const int rt = row >> 4, rr = row & 15, gq = rr & 7, hi8 = rr >> 3;
+    const int ks = k >> 6, kk = k & 63, j = kk >> 4, c = kk & 15;
+    const int rho = hi8 + 2 * (c >> 3), c8 = c & 7, tg = c8 >> 1, h = c8 & 1;
+    const int lane = 4 * gq + tg, pi = 4 * j + rho;
+    const size_t base = (((size_t)rt * (size_t)(n >> 6) + (size_t)ks) * 32u + (size_t)lane) * (size_t)bits;
+    FragPos p;
+    p.scattered = false;
+    if (bits == 4) {
+        p.word = base + j;
+        p.shift = 4 * rho + 16 * h;
+    } else if (bits == 2) {
+        p.word = base + (pi >> 3);
+        p.shift = 2 * (pi & 7) + 16 * h;
+    } else {
+        if (pi < 15) {
+            p.word = base + pi / 5;
+            p.shift = 3 * (pi % 5) + 16 * h;
+        } else {
+            p.word = base;
+            p.shift = 15 + 16 * h;
+            p.scattered = true;
+        }
+    }
+    return p;
+}
+
+// (scale, zero) pairs in the fragment layout: [m/16][n/g][16 rows] half2.
+__host__ __device__ inline size_t sz_frag_index(int n_groups, int row, int grp) {
+    return ((size_t)(row >> 4) * (size_t)n_groups + (size_t)grp) * 16u + (size_t)(row & 15);
+}
+
+}  // namespace lopro

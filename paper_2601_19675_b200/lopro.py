@@ -1,0 +1,227 @@
+"""ctypes binding of liblopro.so: the same entry points as include/lopro.h, argument marshalling only.
+
+Tensors are torch tensors (torch supplies device memory and streams); every computation runs in the
+library's CUDA kernels.  The library must have been built (`python -m paper_2601_19675_b200.build`);
+loading fails loudly otherwise -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblopro.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT, ERR_INVALID_DATA = range(7)
+OUT_BF16, OUT_F32 = 0, 1
+LAYOUT_CANONICAL, LAYOUT_FRAGMENT = 0, 1
+SEC_HEADER, SEC_CODES, SEC_SCALEZERO, SEC_PERM, SEC_A, SEC_B = range(6)
+
+# every symbol include/lopro.h declares
+SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packed_bytes", "lopro_packed_section",
+           "lopro_workspace_bytes", "lopro_pack", "lopro_unpack", "lopro_rotate", "lopro_linear_fwd",
+           "lopro_host_staging_bytes", "lopro_linear_fwd_host"]
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32), ("bits", ctypes.c_int32),
+                ("group_size", ctypes.c_int32), ("block_size", ctypes.c_int32), ("identity_cols", ctypes.c_int32),
+                ("rank", ctypes.c_int32), ("layout", ctypes.c_int32)]
+
+    def __repr__(self):
+        return "Desc(" + ", ".join(f"{n}={getattr(self, n)}" for n, _ in self._fields_) + ")"
+
+
+class LoproError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        super().__init__(f"{where}: {status_str(status)} (status {int(status)})")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library (loads it on first use)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_19675_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        dp = ctypes.POINTER(Desc)
+        L.lopro_version.restype = ctypes.c_int
+        L.lopro_version.argtypes = []
+        L.lopro_status_str.restype = ctypes.c_char_p
+        L.lopro_status_str.argtypes = [ctypes.c_int]
+        L.lopro_check_desc.restype = ctypes.c_int
+        L.lopro_check_desc.argtypes = [dp]
+        L.lopro_packed_bytes.restype = sz
+        L.lopro_packed_bytes.argtypes = [dp]
+        L.lopro_packed_section.restype = ctypes.c_int
+        L.lopro_packed_section.argtypes = [dp, i32, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.lopro_workspace_bytes.restype = sz
+        L.lopro_workspace_bytes.argtypes = [dp, i32]
+        L.lopro_pack.restype = ctypes.c_int
+        L.lopro_pack.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.lopro_unpack.restype = ctypes.c_int
+        L.lopro_unpack.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.lopro_rotate.restype = ctypes.c_int
+        L.lopro_rotate.argtypes = [dp, vp, vp, i64, vp, i64, i32, vp]
+        L.lopro_linear_fwd.restype = ctypes.c_int
+        L.lopro_linear_fwd.argtypes = [dp, vp, vp, i64, vp, i64, i32, i32, vp, sz, vp]
+        L.lopro_host_staging_bytes.restype = sz
+        L.lopro_host_staging_bytes.argtypes = [dp, i32, i32]
+        L.lopro_linear_fwd_host.restype = ctypes.c_int
+        L.lopro_linear_fwd_host.argtypes = [dp, vp, vp, vp, i32, i32, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def version():
+    return lib().lopro_version()
+
+
+def status_str(status):
+    return lib().lopro_status_str(int(status)).decode()
+
+
+def make_desc(d_in, d_out, bits, group_size, block_size, identity_cols=None, rank=0, layout=LAYOUT_FRAGMENT):
+    """Descriptor of one layer; identity_cols defaults to block_size (the paper's b_I = b_H)."""
+    if identity_cols is None:
+        identity_cols = block_size
+    return Desc(d_in, d_out, bits, group_size, block_size, identity_cols, rank, layout)
+
+
+def check_desc(desc):
+    return lib().lopro_check_desc(ctypes.byref(desc))
+
+
+def packed_bytes(desc):
+    return int(lib().lopro_packed_bytes(ctypes.byref(desc)))
+
+
+def packed_section(desc, section):
+    off, nbytes = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    st = lib().lopro_packed_section(ctypes.byref(desc), section, ctypes.byref(off), ctypes.byref(nbytes))
+    if st != OK:
+        raise LoproError(st, "lopro_packed_section")
+    return int(off.value), int(nbytes.value)
+
+
+def workspace_bytes(desc, T):
+    return int(lib().lopro_workspace_bytes(ctypes.byref(desc), int(T)))
+
+
+def host_staging_bytes(desc, T, out_dtype=OUT_BF16):
+    return int(lib().lopro_host_staging_bytes(ctypes.byref(desc), int(T), int(out_dtype)))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(st, where):
+    if st != OK:
+        raise LoproError(st, where)
+
+
+def _dev(t, dtype_bytes):
+    assert t.is_cuda and t.is_contiguous() and t.element_size() == dtype_bytes, "expects a contiguous device tensor"
+    return t
+
+
+def pack(desc, codes, scales_f16, zeros_f16, perm, A_f16=None, B_f16=None, out=None):
+    """lopro_pack: device tensors in (uint8 codes [m][n]; 2-byte scales/zeros/A/B; int32 perm) -> uint8 blob."""
+    nbytes = packed_bytes(desc)
+    if nbytes == 0:
+        raise LoproError(check_desc(desc) or ERR_INVALID_ARG, "lopro_packed_bytes")
+    if out is None:
+        out = torch.empty(nbytes, dtype=torch.uint8, device=codes.device)
+    st = lib().lopro_pack(ctypes.byref(desc), _ptr(_dev(codes, 1)), _ptr(_dev(scales_f16, 2)), _ptr(_dev(zeros_f16, 2)),
+                          _ptr(_dev(perm, 4)), _ptr(A_f16), _ptr(B_f16), _ptr(out), out.numel(), _stream())
+    _check(st, "lopro_pack")
+    return out
+
+
+def unpack(desc, packed, want=("codes", "words", "scales", "zeros", "perm", "A", "B")):
+    """lopro_unpack: returns a dict of freshly allocated device tensors (16-bit floats as int16 bit patterns)."""
+    m, n, g, r = desc.d_out, desc.d_in, desc.group_size, desc.rank
+    dev = packed.device
+    out = {}
+    if "codes" in want:
+        out["codes"] = torch.empty((m, n), dtype=torch.uint8, device=dev)
+    if "words" in want:
+        out["words"] = torch.empty((m, n * desc.bits // 32), dtype=torch.int32, device=dev)
+    if "scales" in want:
+        out["scales"] = torch.empty((m, n // g), dtype=torch.int16, device=dev)
+    if "zeros" in want:
+        out["zeros"] = torch.empty((m, n // g), dtype=torch.int16, device=dev)
+    if "perm" in want:
+        out["perm"] = torch.empty((n,), dtype=torch.int32, device=dev)
+    if "A" in want and r > 0:
+        out["A"] = torch.empty((m, r), dtype=torch.int16, device=dev)
+    if "B" in want and r > 0:
+        out["B"] = torch.empty((r, n), dtype=torch.int16, device=dev)
+    st = lib().lopro_unpack(ctypes.byref(desc), _ptr(packed), _ptr(out.get("codes")), _ptr(out.get("words")),
+                            _ptr(out.get("scales")), _ptr(out.get("zeros")), _ptr(out.get("perm")), _ptr(out.get("A")),
+                            _ptr(out.get("B")), _stream())
+    _check(st, "lopro_unpack")
+    return out
+
+
+def perm_of(desc, packed):
+    """View of the permutation section of a blob (int32 [n], device)."""
+    off, nbytes = packed_section(desc, SEC_PERM)
+    return packed[off:off + nbytes].view(torch.int32)
+
+
+def rotate(desc, perm, x, out=None):
+    """lopro_rotate: x bf16 [T][n] (rows may be strided) -> rotated bf16 [T][n]."""
+    assert x.is_cuda and x.dim() == 2 and x.element_size() == 2 and x.stride(1) == 1
+    T = x.shape[0]
+    if out is None:
+        out = torch.empty((T, desc.d_in), dtype=x.dtype, device=x.device)
+    st = lib().lopro_rotate(ctypes.byref(desc), _ptr(perm), _ptr(x), x.stride(0) if T > 1 else max(x.stride(0), desc.d_in),
+                            _ptr(out), out.stride(0) if T > 1 else max(out.stride(0), desc.d_in), T, _stream())
+    _check(st, "lopro_rotate")
+    return out
+
+
+def linear_fwd(desc, packed, x, out_dtype=OUT_BF16, workspace=None, y=None):
+    """lopro_linear_fwd: x bf16 [T][n] device -> y [T][m] (bf16 or fp32)."""
+    assert x.is_cuda and x.dim() == 2 and x.element_size() == 2 and x.stride(1) == 1
+    T = x.shape[0]
+    if workspace is None:
+        workspace = torch.empty(max(workspace_bytes(desc, T), 256), dtype=torch.uint8, device=x.device)
+    if y is None:
+        y = torch.empty((T, desc.d_out), dtype=torch.float32 if out_dtype == OUT_F32 else torch.bfloat16,
+                        device=x.device)
+    ldx = x.stride(0) if T > 1 else max(x.stride(0), desc.d_in)
+    ldy = y.stride(0) if T > 1 else max(y.stride(0), desc.d_out)
+    st = lib().lopro_linear_fwd(ctypes.byref(desc), _ptr(packed), _ptr(x), ldx, _ptr(y), ldy, int(out_dtype), T,
+                                _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "lopro_linear_fwd")
+    return y
+
+
+def linear_fwd_host(desc, packed, x_host, y_host, workspace, out_dtype=OUT_BF16):
+    """lopro_linear_fwd_host: x_host / y_host are HOST tensors (pinned for asynchronous copies); enqueues
+    copy-in, forward and copy-out on the current stream and returns without synchronising."""
+    assert not x_host.is_cuda and not y_host.is_cuda and x_host.is_contiguous() and y_host.is_contiguous()
+    T = x_host.shape[0]
+    st = lib().lopro_linear_fwd_host(ctypes.byref(desc), _ptr(packed), _ptr(x_host), _ptr(y_host), int(out_dtype), T,
+                                     _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "lopro_linear_fwd_host")
+    return y_host
+
+
+def workspace_status(workspace):
+    """Status word a kernel leaves at the start of the workspace (synchronises)."""
+    return int(workspace[:4].view(torch.int32).item())

@@ -1,0 +1,109 @@
+"""Host-only checks of the C ABI: the library loads without a GPU, exports every symbol the header
+declares, validates descriptors, and sizes the blob by the storage accounting of Eq. 13."""
+import os
+import re
+
+import pytest
+
+from oracle import lopro_oracle as o
+from paper_2601_19675_b200 import build, lopro
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "lopro.h")).read()
+    return sorted(set(re.findall(r"LOPRO_API[^;(]*?\b(lopro_\w+)\s*\(", text)))
+
+
+def test_header_declares_what_binding_lists():
+    assert _declared_symbols() == sorted(lopro.SYMBOLS)
+
+
+def test_library_exports_every_declared_symbol():
+    L = lopro.lib()
+    for name in _declared_symbols():
+        assert hasattr(L, name), name
+    assert lopro.version() >= 100
+    assert lopro.status_str(lopro.OK) == "ok"
+    assert "timed out" in lopro.status_str(lopro.ERR_TIMEOUT)
+
+
+@pytest.mark.parametrize("kw,expect", [
+    (dict(), lopro.OK),
+    (dict(bits=5), lopro.ERR_INVALID_ARG),
+    (dict(bits=1), lopro.ERR_INVALID_ARG),
+    (dict(block_size=96), lopro.ERR_INVALID_ARG),          # b_H must be a power of two (Eq. 6)
+    (dict(block_size=2048), lopro.ERR_INVALID_ARG),
+    (dict(identity_cols=100), lopro.ERR_INVALID_ARG),      # (n - b_I) must be a whole number of blocks
+    (dict(identity_cols=0), lopro.OK),
+    (dict(identity_cols=4096), lopro.OK),                  # rotation disabled
+    (dict(group_size=100), lopro.ERR_INVALID_ARG),         # g must divide n
+    (dict(group_size=32), lopro.ERR_UNSUPPORTED),
+    (dict(d_in=4096 + 32, identity_cols=32 + 128), lopro.ERR_INVALID_ARG),
+    (dict(d_out=4100), lopro.ERR_UNSUPPORTED),
+    (dict(rank=-1), lopro.ERR_INVALID_ARG),
+    (dict(rank=17), lopro.OK),
+    (dict(layout=7), lopro.ERR_INVALID_ARG),
+])
+def test_descriptor_domain(kw, expect):
+    base = dict(d_in=4096, d_out=4096, bits=4, group_size=128, block_size=128, identity_cols=128, rank=32)
+    base.update(kw)
+    d = lopro.make_desc(**base)
+    assert lopro.check_desc(d) == expect
+    assert (lopro.packed_bytes(d) > 0) == (expect == lopro.OK)
+
+
+@pytest.mark.parametrize("m,n,bits,g,r", [(4096, 4096, 4, 128, 32), (11008, 4096, 3, 64, 64), (28672, 8192, 2, 64, 128),
+                                          (512, 512, 4, 128, 16)])
+def test_blob_size_follows_eq13_accounting(m, n, bits, g, r):
+    # Eq. 13 with this library's widths: d_q bits per code, 16-bit scale and 16-bit zero per group,
+    # 16-bit factor entries (rank padded to 16), 32-bit permutation entries; plus a 256-byte header
+    # and at most 255 bytes of padding after each of the six sections.
+    d = lopro.make_desc(n, m, bits, g, 64, rank=r)
+    r_pad = (r + 15) // 16 * 16
+    payload_bits = m * n * (o.average_bits(m, n, bits, 32, g, r_pad, 16) - 2 * 32 / n - r_pad * 32 / (m * n)) + 32 * n
+    nbytes = lopro.packed_bytes(d)
+    assert payload_bits / 8 + 256 <= nbytes <= payload_bits / 8 + 256 + 6 * 256
+    total = 0
+    for sec in range(6):
+        off, sz = lopro.packed_section(d, sec)
+        assert off % 256 == 0 and off >= total
+        total = off + sz
+    assert total <= nbytes
+
+
+def test_workspace_size_is_monotone_in_tokens():
+    d = lopro.make_desc(4096, 4096, 4, 128, 128, rank=32)
+    sizes = [lopro.workspace_bytes(d, t) for t in (0, 1, 7, 8, 9, 32, 33, 2048)]
+    assert all(a <= b for a, b in zip(sizes, sizes[1:])) and sizes[0] > 0
+    assert lopro.workspace_bytes(d, -1) == 0
+    assert lopro.host_staging_bytes(d, 8) >= 8 * 4096 * 2 * 2
+
+
+def test_null_and_bad_arguments_are_rejected_before_any_cuda_call():
+    import ctypes
+    L = lopro.lib()
+    d = lopro.make_desc(512, 512, 4, 128, 64, rank=16)
+    assert L.lopro_pack(None, None, None, None, None, None, None, None, 0, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_pack(ctypes.byref(d), None, None, None, None, None, None, None, 0, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_rotate(ctypes.byref(d), None, None, 512, None, 512, 4, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_rotate(ctypes.byref(d), None, None, 512, None, 512, 0, None) == lopro.OK      # T = 0: no-op
+    assert L.lopro_rotate(ctypes.byref(d), None, None, 512, None, 512, -1, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_linear_fwd(ctypes.byref(d), None, None, 512, None, 512, 0, 0, None, 0, None) == lopro.OK
+    assert L.lopro_linear_fwd(ctypes.byref(d), None, None, 512, None, 512, 0, 4, None, 0, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_linear_fwd(ctypes.byref(d), None, None, 512, None, 512, 9, 4, None, 0, None) == lopro.ERR_INVALID_ARG
+    dc = lopro.make_desc(512, 512, 4, 128, 64, rank=16, layout=lopro.LAYOUT_CANONICAL)
+    assert L.lopro_linear_fwd(ctypes.byref(dc), None, None, 512, None, 512, 0, 4, None, 0, None) == lopro.ERR_UNSUPPORTED
+    # misaligned pointers and short leading dimensions (fake non-null addresses are never dereferenced)
+    fake = ctypes.c_void_p(0x1000)
+    odd = ctypes.c_void_p(0x1002)
+    assert L.lopro_rotate(ctypes.byref(d), fake, odd, 512, fake, 512, 4, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_rotate(ctypes.byref(d), fake, fake, 500, fake, 512, 4, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_linear_fwd(ctypes.byref(d), fake, fake, 512, fake, 100, 0, 4, fake, 1 << 30, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_linear_fwd(ctypes.byref(d), fake, fake, 512, fake, 512, 0, 4, fake, 16, None) == lopro.ERR_BUFFER_TOO_SMALL

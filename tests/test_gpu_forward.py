@@ -1,0 +1,140 @@
+"""GPU parity of lopro_linear_fwd with the fp64 oracle of Eq. 8.
+
+Gate A: bf16 output against the exact oracle, max relative error <= 2e-2.
+Gate B: fp32 output (fp32 accumulation) against the mirrored oracle, which applies the roundings the
+library declares (rotated activations to bf16, low-rank intermediate to fp16), <= 1e-3.
+The error measure is oracle.max_rel_err (element-wise, relative to max(|y|, rms of the token's row))."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lopro_oracle as o
+from paper_2601_19675_b200 import lopro, synth
+from tests._layers import bf16_bits_to_device, device_bf16_to_f64, oracle_args, random_layer_np, to_device
+
+pytestmark = pytest.mark.gpu
+
+GATE_A = 2e-2
+GATE_B = 1e-3
+
+
+def _pack(layer, d):
+    dev = to_device(layer)
+    return lopro.pack(d, dev["codes"], dev["scales"], dev["zeros"], dev["perm"], dev["A"], dev["B"])
+
+
+def _check_forward(layer, d, x_bits, rows=None, gate_a=GATE_A, gate_b=GATE_B):
+    blob = _pack(layer, d)
+    x = bf16_bits_to_device(x_bits)
+    T = x.shape[0]
+    ws = torch.zeros(lopro.workspace_bytes(d, T), dtype=torch.uint8, device="cuda")
+    y_bf = lopro.linear_fwd(d, blob, x, lopro.OUT_BF16, workspace=ws)
+    y_f32 = lopro.linear_fwd(d, blob, x, lopro.OUT_F32, workspace=ws)
+    torch.cuda.synchronize()
+    assert lopro.workspace_status(ws) == lopro.OK
+    args = oracle_args(layer, d.group_size, d.identity_cols, d.block_size, rows=rows)
+    x64 = o.bf16_bits_to_f64(x_bits)
+    exact = o.forward_exact(x64, **args)
+    mirrored = o.forward_mirrored(x64, **args, round_w=False, round_t="f16", out="f32")
+    assert o.max_rel_err(mirrored, exact) <= 1e-2            # declared roundings cannot hide an error
+    got_bf = device_bf16_to_f64(y_bf)
+    got_f32 = y_f32.cpu().numpy().astype(np.float64)
+    if rows is not None:
+        got_bf, got_f32 = got_bf[:, rows], got_f32[:, rows]
+    err_a = o.max_rel_err(got_bf, exact)
+    err_b = o.max_rel_err(got_f32, mirrored)
+    assert err_a <= gate_a, f"gate A: {err_a}"
+    assert err_b <= gate_b, f"gate B: {err_b}"
+    # bf16 output is the rounding of the fp32 output path (same accumulation order)
+    assert np.array_equal(got_bf, o.round_bf16(got_f32))
+    return err_a, err_b
+
+
+def test_cfg1_layer_quantized_by_the_oracle():
+    # configuration 1: 512 x 512, 16 tokens, weights ~ N(0, 0.02) quantized by the oracle to 4-bit
+    # asymmetric g = 128, random permutation, b_I = b_H = 64, rank 16.
+    c = synth.CONFIGS["cfg1"]
+    n, m, r = c["d_in"], c["d_out"], c["rank"]
+    w = synth.weights(m, n, seed=0)
+    perm = synth.permutation(n, seed=0)
+    q = o.lopro_quantize(w, perm, c["identity_cols"], c["block_size"], r, c["bits"], c["group_size"], method="svd")
+    layer = dict(codes=q["codes"], scales=o.f64_to_f16_bits(q["scales"]), zeros=o.f64_to_f16_bits(q["zeros"]),
+                 perm=perm, A=o.f64_to_f16_bits(q["A"]), B=o.f64_to_f16_bits(q["B"]))
+    d = lopro.make_desc(n, m, c["bits"], c["group_size"], c["block_size"], c["identity_cols"], r)
+    x_bits = synth.activations(16, n, seed=0)
+    _check_forward(layer, d, x_bits)
+    # and the quantized layer approximates the dense one: y ~= W x (quantization error only)
+    blob = _pack(layer, d)
+    y = device_bf16_to_f64(lopro.linear_fwd(d, blob, bf16_bits_to_device(x_bits)))
+    dense = o.bf16_bits_to_f64(x_bits) @ w.astype(np.float64).T
+    assert np.linalg.norm(y - dense) / np.linalg.norm(dense) < 0.12
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("g", [64, 128])
+@pytest.mark.parametrize("T", [1, 2, 3, 7, 8, 9, 15, 16, 17, 31, 32, 33, 65])
+def test_token_count_edges(bits, g, T):
+    n, m, r = 768, 144, 17                                    # ragged row tile (144 = 128 + 16), odd rank
+    layer = random_layer_np(n, m, bits, g, r, seed=100 + bits + g)
+    d = lopro.make_desc(n, m, bits, g, 128, identity_cols=128, rank=r)
+    _check_forward(layer, d, synth.activations(T, n, seed=T))
+
+
+@pytest.mark.parametrize("n,m,bits,g,b_i,b_h,r,T", [
+    (64, 16, 4, 64, 0, 64, 0, 1),            # smallest layer, no low-rank branch
+    (64, 16, 2, 64, 64, 2, 1, 5),            # rotation disabled (b_I = n)
+    (1024, 256, 3, 256, 0, 1024, 64, 4),     # full-width Hadamard (the full-rotation ablation)
+    (2048, 128, 4, 128, 0, 512, 8, 8),
+    (4096, 512, 4, 128, 256, 256, 32, 8),    # several K slices and panels
+    (8192, 256, 2, 64, 256, 256, 128, 16),
+    (4096, 384, 3, 64, 128, 128, 64, 40),
+    (11008, 128, 4, 128, 128, 128, 32, 2),   # the 7B 'down' projection width
+])
+def test_shapes_in_the_parameter_domain(n, m, bits, g, b_i, b_h, r, T):
+    layer = random_layer_np(n, m, bits, g, r, seed=n + m + bits)
+    d = lopro.make_desc(n, m, bits, g, b_h, identity_cols=b_i, rank=r)
+    _check_forward(layer, d, synth.activations(T, n, seed=7, outlier_frac=0.01))
+
+
+def test_outputs_can_be_strided_and_calls_repeat_bitwise():
+    n, m, bits, g, r, T = 1024, 256, 4, 128, 16, 8
+    layer = random_layer_np(n, m, bits, g, r, seed=1)
+    d = lopro.make_desc(n, m, bits, g, 128, rank=r)
+    blob = _pack(layer, d)
+    x = bf16_bits_to_device(synth.activations(T, n, seed=2))
+    y1 = lopro.linear_fwd(d, blob, x)
+    ybuf = torch.zeros((T, m + 32), dtype=torch.bfloat16, device="cuda")
+    lopro.linear_fwd(d, blob, x, y=ybuf[:, :m])
+    y2 = lopro.linear_fwd(d, blob, x)
+    assert torch.equal(y1, ybuf[:, :m]) and torch.equal(y1, y2)     # split-K order is fixed
+    assert torch.count_nonzero(ybuf[:, m:]) == 0
+
+
+def test_forward_argument_errors():
+    n, m = 512, 64
+    layer = random_layer_np(n, m, 4, 128, 0, seed=1)
+    d = lopro.make_desc(n, m, 4, 128, 64, rank=0)
+    blob = _pack(layer, d)
+    x = torch.zeros((4, n), dtype=torch.bfloat16, device="cuda")
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(lopro.LoproError) as e:
+        lopro.linear_fwd(d, blob, x, workspace=small)
+    assert e.value.status == lopro.ERR_BUFFER_TOO_SMALL
+    y = lopro.linear_fwd(d, blob, x[:0])                        # T = 0
+    assert y.shape == (0, m)
+
+
+def test_host_entry_point_matches_device_entry_point():
+    n, m, bits, g, r, T = 1024, 256, 4, 128, 16, 8
+    layer = random_layer_np(n, m, bits, g, r, seed=4)
+    d = lopro.make_desc(n, m, bits, g, 128, rank=r)
+    blob = _pack(layer, d)
+    x_bits = synth.activations(T, n, seed=5)
+    x = bf16_bits_to_device(x_bits)
+    y_dev = lopro.linear_fwd(d, blob, x)
+    xh = torch.from_numpy(x_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    yh = torch.empty((T, m), dtype=torch.bfloat16).pin_memory()
+    ws = torch.zeros(lopro.workspace_bytes(d, T) + lopro.host_staging_bytes(d, T), dtype=torch.uint8, device="cuda")
+    lopro.linear_fwd_host(d, blob, xh, yh, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(yh, y_dev.cpu())
