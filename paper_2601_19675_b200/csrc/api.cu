@@ -45,30 +45,6 @@ lopro_status blob_layout(const lopro_desc& d, BlobLayout* out) {
     return LOPRO_OK;
 }
 
-// Split-K factor of the small-batch kernel: enough CTAs to cover the SMs about twice, K slices
-// that are whole groups and at least 256 columns long.
-int decode_split(const lopro_desc& d, int T) {
-    static int forced = -1;
-    if (forced < 0) {
-        const char* e = getenv("LOPRO_DECODE_SPLIT");
-        forced = e ? atoi(e) : 0;
-    }
-    const int mt = (d.d_out + 127) / 128;
-    const int zc = (T + kDecodeMaxT - 1) / kDecodeMaxT;
-    int split = 1;
-    if (forced > 0) {
-        split = forced;
-    } else {
-        while (split < kDecodeMaxSplit && mt * zc * split < 2 * 148) split *= 2;
-    }
-    const int unit = d.group_size > 512 ? d.group_size : 512;
-    while (split > 1 && (d.d_in % (split * unit) != 0)) split /= 2;
-    if (split > kDecodeMaxSplit) split = kDecodeMaxSplit;
-    while (split > 1 && (d.d_in % (split * d.group_size) != 0)) split /= 2;
-    if (zc > 1) split = 1;  // many tokens: the token chunks already fill the machine
-    return split;
-}
-
 lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
     lopro_status st = check_desc(d);
     if (st != LOPRO_OK) return st;
@@ -79,21 +55,18 @@ lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
     W->t_pad = t_pad;
     W->off_status = off;
     off += 256;
-    W->max_tickets = kMaxTickets;
-    W->off_tickets = off;
-    off += round_up_size((size_t)kMaxTickets * 4, 256);
     W->off_xrot = off;
-    off += round_up_size((size_t)t_pad * d.d_in * 2, 256);
+    {
+        size_t xb = (size_t)t_pad * d.d_in * 2;
+        if (t_pad <= kDecodeMaxT && act_image_bytes(d.d_in, t_pad) > xb) xb = act_image_bytes(d.d_in, t_pad);
+        off += round_up_size(xb, 256);
+    }
     W->off_s64 = off;
-    off += round_up_size((size_t)t_pad * (d.d_in / 64) * 4, 256);
+    off += round_up_size((size_t)t_pad * s64_stride(d.d_in) * 4, 256);
     W->off_t = off;
     off += round_up_size((size_t)t_pad * (r_pad > 0 ? r_pad : 16) * 2, 256);
-    W->off_partial = off;
-    // Partial sums exist only while one launch covers all tokens (T <= 32); sized for the
-    // largest split so that the size does not depend on tuning.
-    const int tp = t_pad < kDecodeMaxT ? t_pad : kDecodeMaxT;
-    W->partial_bytes = (size_t)kDecodeMaxSplit * tp * d.d_out * 4;
-    off += round_up_size(W->partial_bytes, 256);
+    W->off_tpart = off;
+    if (t_pad <= kDecodeMaxT) off += round_up_size((size_t)((d.d_in + 255) / 256) * t_pad * r_pad * 4, 256);
     W->total = off;
     return LOPRO_OK;
 }
@@ -217,7 +190,7 @@ lopro_status lopro_rotate(const lopro_desc* desc, const int32_t* perm, const uin
     if (ldx < desc->d_in || ldo < desc->d_in || (ldx % 8) || (ldo % 8)) return LOPRO_ERR_INVALID_ARG;
     if (!aligned(x_bf16, 16) || !aligned(xrot_bf16, 16) || !aligned(perm, 4)) return LOPRO_ERR_INVALID_ARG;
     cudaError_t e = launch_rotate(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, (__nv_bfloat16*)xrot_bf16, ldo,
-                                  nullptr, T, (cudaStream_t)stream);
+                                  nullptr, nullptr, T, (cudaStream_t)stream);
     return e == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }
 
@@ -244,16 +217,25 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     cudaStream_t s = (cudaStream_t)stream;
     uint8_t* ws = (uint8_t*)workspace;
     const uint8_t* blob = (const uint8_t*)packed;
-    // Status word and split-K tickets start at zero.
-    if (cudaMemsetAsync(ws, 0, W.off_xrot, s) != cudaSuccess) return LOPRO_ERR_CUDA;
     const int32_t* perm = (const int32_t*)(blob + L.off[LOPRO_SEC_PERM]);
+    const __half* B = (const __half*)(blob + L.off[LOPRO_SEC_B]);
     __nv_bfloat16* xrot = (__nv_bfloat16*)(ws + W.off_xrot);
     float* s64 = (float*)(ws + W.off_s64);
-    if (launch_rotate(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, xrot, desc->d_in, s64, T, s) != cudaSuccess)
+    int* status = (int*)(ws + W.off_status);
+    if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
+        // small batch: prologue + streaming kernel, chained by programmatic launches
+        if (launch_prologue(*desc, perm, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot,
+                            (float*)(ws + W.off_tpart), W.t_pad, status, T, s) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
+        if (launch_stream(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+        return LOPRO_OK;
+    }
+    if (launch_rotate(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, xrot, desc->d_in, s64, status, T, s) !=
+        cudaSuccess)
         return LOPRO_ERR_CUDA;
     if (desc->rank > 0) {
-        if (launch_lowrank_down(*desc, (const __half*)(blob + L.off[LOPRO_SEC_B]), L.r_pad,
-                                (const __nv_bfloat16*)x_bf16, ldx, (__half*)(ws + W.off_t), T, s) != cudaSuccess)
+        if (launch_lowrank_down(*desc, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, (__half*)(ws + W.off_t), T, s) !=
+            cudaSuccess)
             return LOPRO_ERR_CUDA;
     }
     if (launch_decode(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;

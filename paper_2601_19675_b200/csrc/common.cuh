@@ -47,23 +47,42 @@ struct BlobLayout {
 lopro_status check_desc(const lopro_desc& d);
 lopro_status blob_layout(const lopro_desc& d, BlobLayout* out);
 
+// Raises a kernel's dynamic shared-memory limit once per device (function attributes are per device);
+// later calls, e.g. during stream capture, make no CUDA call.  `done` is a per-kernel bit mask.
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long long* done) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (__atomic_load_n(done, __ATOMIC_ACQUIRE) & bit) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) __atomic_fetch_or(done, bit, __ATOMIC_RELEASE);
+    return e;
+}
+
 inline int round_up_int(int v, int a) { return (v + a - 1) / a * a; }
 inline size_t round_up_size(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Workspace of lopro_linear_fwd: status word, split-K tickets, rotated activations, 64-column
-// sums of the rotated activations, low-rank intermediate, split-K partial sums.
+// Workspace of lopro_linear_fwd: status word, rotated activations, 64-column sums of the rotated
+// activations, low-rank intermediate (fp16, general path), per-chunk partial sums of the low-rank
+// intermediate (fp32, small-batch path).
 struct WorkspaceLayout {
-    size_t off_status, off_tickets, off_xrot, off_s64, off_t, off_partial, total;
-    int t_pad;       // tokens padded to a multiple of 8
-    int max_tickets;
-    size_t partial_bytes;
+    size_t off_status, off_xrot, off_s64, off_t, off_tpart, total;
+    int t_pad;  // tokens padded to a multiple of 8
 };
-constexpr int kMaxTickets = 4096;
-constexpr int kDecodeMaxT = 32;      // tokens per launch of the small-batch kernel
-constexpr int kDecodeMaxSplit = 16;  // upper bound of the split-K factor
+constexpr int kDecodeMaxT = 32;               // tokens per CTA of the streaming kernels
+constexpr int kStreamMaxSmem = 220 * 1024;    // dynamic shared memory the small-batch kernel may use
+// Row stride of the 64-column sums: a whole number of 16-step stages, so that a stage's sums of one
+// token are one aligned 64-byte piece.
+inline int s64_stride(int n) { return ((n / 64 + 15) / 16) * 16; }
+// Small-batch path: the prologue stores the rotated activations as the shared-memory image of the
+// streaming kernel's stages, [stage of 1024 columns][token][kActRecord bytes]: 1024 bf16 entries, the
+// sixteen 64-column sums (fp32), 16 bytes of padding (the odd multiple of 16 bytes keeps ldmatrix
+// reads of eight tokens conflict-free).  One bulk copy then brings a stage's activations.
+constexpr int kActRecord = 2048 + 64 + 16;
+inline size_t act_image_bytes(int n, int t_pad) { return (size_t)((n + 1023) / 1024) * t_pad * kActRecord; }
 lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* out);
-// Split-K factor the small-batch kernel uses for T tokens (host).
-int decode_split(const lopro_desc& d, int T);
 
 // ---- launchers (each returns the CUDA status of its launches) -------------------------------
 cudaError_t launch_validate(const lopro_desc& d, const uint8_t* codes, const uint16_t* scales,
@@ -78,12 +97,21 @@ cudaError_t launch_unpack(const lopro_desc& d, const void* blob, const BlobLayou
 // Rotation; s64 (optional) receives the sums of each aligned run of 64 rotated (bf16-rounded)
 // entries, [T][n/64] fp32.
 cudaError_t launch_rotate(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
-                          __nv_bfloat16* xrot, int64_t ldo, float* s64, int T, cudaStream_t s);
+                          __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s);
+// Small-batch prologue: rotation, 64-column sums and per-chunk partial sums of B x in one launch.
+bool prologue_supported(const lopro_desc& d, int T);
+cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
+                            const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, float* t_part, int t_pad,
+                            int* status, int T, cudaStream_t s);
 // t[T][r_pad] (fp16) = B x, fp32 accumulation.
 cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,
                                 int64_t ldx, __half* t, int T, cudaStream_t s);
-// Small-batch forward over the fragment layout (T tokens, any T: processed 32 at a time).
+// General forward over the fragment layout: any T, after launch_rotate and launch_lowrank_down.
 cudaError_t launch_decode(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
+                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
+// Small-batch forward (T <= 32) after launch_prologue: bulk-copy ring, one CTA per 32 output rows.
+bool stream_supported(const lopro_desc& d, int T);
+cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
 
 // ---- fragment layout ----------------------------------------------------------------------

@@ -1,4 +1,4 @@
-// Small-batch forward (decode): y = W^ x~ + A t for up to 32 tokens per launch, streaming the
+// Small-batch forward (decode): y = W^ x~ + A t for up to 32 tokens per CTA, streaming the
 // packed codes once from HBM (steps "Dequant(W_q) X" and "U (Sigma Y)" of Appendix A.3, summed
 // as in Eq. 8).
 //
@@ -28,8 +28,7 @@ struct DecodeParams {
     const __nv_bfloat16* xrot;  // [T][n]
     const float* s64;           // [T][n/64]
     const __half* t;            // [T][r_pad]
-    float* partial;             // [split][tp][m]
-    int* tickets;               // [m tiles]
+    int s64_stride;
     void* y;
     int64_t ldy;
     int out_f32;
@@ -37,8 +36,7 @@ struct DecodeParams {
     int gshift;      // log2(group_size / 64)
     int ng;          // groups per row
     int r_pad;
-    int split;       // K slices
-    int slice_steps; // 64-column steps per slice
+    int slice_steps; // 64-column steps (the whole K range)
     int panel_steps; // steps staged in shared memory at a time (multiple of kPrefetch)
 };
 
@@ -98,6 +96,8 @@ __device__ __forceinline__ void expand_codes(uint32_t (&a)[16], const uint32_t (
     }
 }
 
+// General path: grid (row tiles of 128, 1, token chunks of 32); every warp streams the codes of its
+// 16 rows over the whole K range with a register ring and writes its outputs directly.
 template <int BITS, int NT>
 __global__ void __launch_bounds__(kThreads)
 decode_kernel(const DecodeParams p) {
@@ -107,17 +107,16 @@ decode_kernel(const DecodeParams p) {
     const int xs_stride = panel_cols + 8;  // bf16 elements; +16 bytes makes the fragment loads conflict-free
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);
     float* ss = reinterpret_cast<float*>(smem_raw + (size_t)kTok * xs_stride * 2);  // [kTok][panel_steps]
-    __shared__ int s_ticket;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tg = lane & 3;
-    const int mtile = blockIdx.x, ksl = blockIdx.y;
+    const int mtile = blockIdx.x;
     const int tok0 = blockIdx.z * kDecodeMaxT;
-    const int tc = min(kTok, p.T - tok0);  // live tokens of this launch slice
+    const int tc = min(kTok, p.T - tok0);  // live tokens of this CTA
     const int row0 = mtile * kRowsPerCta + warp * 16;
     const bool active = row0 < p.m;
     const int nsteps = p.n >> 6;
-    const int s_begin = ksl * p.slice_steps, s_end = s_begin + p.slice_steps;
+    const int s_begin = 0, s_end = p.slice_steps;
 
     float yacc[NT][4];
 #pragma unroll
@@ -125,7 +124,8 @@ decode_kernel(const DecodeParams p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) yacc[nt][i] = 0.0f;
 
-    // Register ring of code words and (scale, zero) pairs, kPrefetch steps deep.
+    // Register ring of code words and (scale, zero) pairs, kPrefetch steps deep.  The layer's own
+    // data does not depend on the previous kernel, so the first loads are issued before the wait.
     uint32_t wbuf[kPrefetch][BITS];
     uint32_t szbuf[kPrefetch][2];
     const uint32_t* wbase = p.codes + ((size_t)(row0 >> 4) * nsteps * 32 + lane) * BITS;
@@ -155,12 +155,12 @@ decode_kernel(const DecodeParams p) {
         for (int i = tid; i < kTok * (pcols / 8); i += kThreads) {
             const int tk = i / (pcols / 8), c = i % (pcols / 8);
             uint4 v = make_uint4(0, 0, 0, 0);
-            if (tk < tc) v = __ldg(reinterpret_cast<const uint4*>(p.xrot + (size_t)(tok0 + tk) * p.n + ps * 64) + c);
+            if (tk < tc) v = __ldcg(reinterpret_cast<const uint4*>(p.xrot + (size_t)(tok0 + tk) * p.n + ps * 64) + c);
             *reinterpret_cast<uint4*>(xs + (size_t)tk * xs_stride + c * 8) = v;
         }
         for (int i = tid; i < kTok * (pe - ps); i += kThreads) {
             const int tk = i / (pe - ps), st = i % (pe - ps);
-            ss[tk * p.panel_steps + st] = tk < tc ? __ldg(p.s64 + (size_t)(tok0 + tk) * nsteps + ps + st) : 0.0f;
+            ss[tk * p.panel_steps + st] = tk < tc ? __ldcg(p.s64 + (size_t)(tok0 + tk) * p.s64_stride + ps + st) : 0.0f;
         }
         __syncthreads();
         if (!active) continue;
@@ -205,8 +205,8 @@ decode_kernel(const DecodeParams p) {
         }
     }
 
-    // low-rank up-projection A t, added by the first K slice (fp16 tensor-core product, fp32 sum)
-    if (active && ksl == 0 && p.r_pad > 0) {
+    // low-rank up-projection A t (fp16 tensor-core product, fp32 sum)
+    if (active && p.r_pad > 0) {
         const __half* arow_lo = p.A + (size_t)(row0 + gq) * p.r_pad + 2 * tg;
         const __half* arow_hi = arow_lo + (size_t)8 * p.r_pad;
         for (int jj = 0; jj < p.r_pad; jj += 16) {
@@ -220,8 +220,8 @@ decode_kernel(const DecodeParams p) {
                 uint32_t b0 = 0, b1 = 0;
                 if (nt * 8 + gq < tc) {
                     const __half* trow = p.t + (size_t)(tok0 + nt * 8 + gq) * p.r_pad + jj + 2 * tg;
-                    b0 = __ldg(reinterpret_cast<const uint32_t*>(trow));
-                    b1 = __ldg(reinterpret_cast<const uint32_t*>(trow + 8));
+                    b0 = __ldcg(reinterpret_cast<const uint32_t*>(trow));
+                    b1 = __ldcg(reinterpret_cast<const uint32_t*>(trow + 8));
                 }
                 mma_f16(yacc[nt], a, b0, b1);
             }
@@ -230,56 +230,28 @@ decode_kernel(const DecodeParams p) {
 
     // ---- write-out ---------------------------------------------------------------------------
     // accumulator element (nt, i): token nt*8 + 2 tg + (i & 1), row row0 + gq + 8 (i >> 1)
-    if (p.split == 1) {
-        if (active) {
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int tk = nt * 8 + 2 * tg + (i & 1), row = row0 + gq + 8 * (i >> 1);
-                    if (tk < tc) {
-                        const size_t o = (size_t)(tok0 + tk) * p.ldy + row;
-                        if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = yacc[nt][i];
-                        else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(yacc[nt][i]);
-                    }
-                }
-        }
-        return;
-    }
-
-    // split-K: every slice stores its partial sums; the CTA that draws the last ticket of the row
-    // tile adds the slices in index order (deterministic) and writes y.
     if (active) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int tk = nt * 8 + 2 * tg + (i & 1), row = row0 + gq + 8 * (i >> 1);
-                if (tk < tc) p.partial[((size_t)ksl * kTok + tk) * p.m + row] = yacc[nt][i];
+                if (tk < tc) {
+                    const size_t o = (size_t)(tok0 + tk) * p.ldy + row;
+                    if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = yacc[nt][i];
+                    else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(yacc[nt][i]);
+                }
             }
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_ticket = atomicAdd(p.tickets + mtile, 1);
-    __syncthreads();
-    if (s_ticket != p.split - 1) return;
-    __threadfence();
-    const int rows_here = min(kRowsPerCta, p.m - mtile * kRowsPerCta);
-    for (int i = tid; i < tc * rows_here; i += kThreads) {
-        const int tk = i / rows_here, row = mtile * kRowsPerCta + i % rows_here;
-        float s = 0.0f;
-        for (int k = 0; k < p.split; ++k) s += __ldcg(p.partial + ((size_t)k * kTok + tk) * p.m + row);
-        const size_t o = (size_t)(tok0 + tk) * p.ldy + row;
-        if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = s;
-        else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(s);
-    }
-    if (tid == 0) p.tickets[mtile] = 0;
 }
 
 template <int BITS, int NT>
 cudaError_t launch_nt(const DecodeParams& p, dim3 grid, cudaStream_t s) {
     const size_t smem = (size_t)NT * 8 * (p.panel_steps * 64 + 8) * 2 + (size_t)NT * 8 * p.panel_steps * 4;
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static unsigned long long attr_done = 0;
+    constexpr int kMaxPanel = NT == 4 ? 16 : 32;
+    constexpr int kMaxSmem = NT * 8 * (kMaxPanel * 64 + 8) * 2 + NT * 8 * kMaxPanel * 4;
+    cudaError_t e = ensure_dynamic_smem(decode_kernel<BITS, NT>, kMaxSmem, &attr_done);
     if (e != cudaSuccess) return e;
     decode_kernel<BITS, NT><<<grid, kThreads, smem, s>>>(p);
     return cudaGetLastError();
@@ -302,9 +274,8 @@ cudaError_t launch_decode(const lopro_desc& d, const uint8_t* blob, const BlobLa
     p.A = reinterpret_cast<const __half*>(blob + L.off[LOPRO_SEC_A]);
     p.xrot = reinterpret_cast<const __nv_bfloat16*>(ws + W.off_xrot);
     p.s64 = reinterpret_cast<const float*>(ws + W.off_s64);
+    p.s64_stride = s64_stride(d.d_in);
     p.t = reinterpret_cast<const __half*>(ws + W.off_t);
-    p.partial = reinterpret_cast<float*>(const_cast<uint8_t*>(ws) + W.off_partial);
-    p.tickets = reinterpret_cast<int*>(const_cast<uint8_t*>(ws) + W.off_tickets);
     p.y = y;
     p.ldy = ldy;
     p.out_f32 = out_dtype == LOPRO_OUT_F32;
@@ -316,16 +287,15 @@ cudaError_t launch_decode(const lopro_desc& d, const uint8_t* blob, const BlobLa
     p.gshift = gshift;
     p.ng = d.d_in / d.group_size;
     p.r_pad = d.rank > 0 ? L.r_pad : 0;
-    p.split = decode_split(d, T);
-    p.slice_steps = (d.d_in / 64) / p.split;
+    p.slice_steps = d.d_in / 64;
     const int zc = (T + kDecodeMaxT - 1) / kDecodeMaxT;
     const int tl = T < kDecodeMaxT ? T : kDecodeMaxT;
     const int nt = tl <= 8 ? 1 : (tl <= 16 ? 2 : 4);
     const int max_panel = nt == 4 ? 16 : 32;  // 1024 or 2048 columns of x~ per panel
     p.panel_steps = p.slice_steps < max_panel ? round_up_int(p.slice_steps, kPrefetch) : max_panel;
     const int mt = (d.d_out + kRowsPerCta - 1) / kRowsPerCta;
-    if (mt > W.max_tickets || zc > 65535 || p.split > 65535) return cudaErrorInvalidValue;
-    dim3 grid(mt, p.split, zc);
+    if (zc > 65535) return cudaErrorInvalidValue;
+    dim3 grid(mt, 1, zc);
     switch (d.bits) {
         case 2: return launch_bits<2>(p, nt, grid, s);
         case 3: return launch_bits<3>(p, nt, grid, s);

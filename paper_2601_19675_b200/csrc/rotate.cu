@@ -20,8 +20,8 @@ constexpr int kRotThreads = 256;
 template <int E>
 __global__ void __launch_bounds__(kRotThreads)
 rotate_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
-              __nv_bfloat16* __restrict__ xrot, int64_t ldo, float* __restrict__ s64, int n, int b_i, int b_h,
-              float inv_sqrt_bh) {
+              __nv_bfloat16* __restrict__ xrot, int64_t ldo, float* __restrict__ s64, int s64_ld,
+              int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __nv_bfloat16* xin = reinterpret_cast<__nv_bfloat16*>(smem_raw);
     __nv_bfloat16* xout = xin + n;
@@ -29,6 +29,7 @@ rotate_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* _
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kRotThreads / 32;
     constexpr int kRun = 32 * E;
+    if (status != nullptr && t == 0 && tid == 0) *status = LOPRO_OK;
 
     const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * ldx);
     for (int i = tid; i < n / 8; i += kRotThreads) reinterpret_cast<uint4*>(xin)[i] = __ldg(src + i);
@@ -90,7 +91,7 @@ rotate_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* _
             float s = __low2float(p) + __high2float(p);
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-            if (lane == 0) s64[(size_t)t * nsteps + st] = s;
+            if (lane == 0) s64[(size_t)t * s64_ld + st] = s;
         }
     }
 }
@@ -141,27 +142,163 @@ lowrank_down_kernel(const __half* __restrict__ B, const __nv_bfloat16* __restric
     }
 }
 
+// Prologue of the small-batch forward (T <= 32, b_H <= 256, b_I a multiple of b_H): one CTA per
+// chunk of 256 columns and group of 8 tokens.
+//  (1) warp w rotates the chunk's 256 output columns of token w: the 8 entries of a lane are
+//      gathered from global memory through perm, transformed with register and shuffle
+//      butterflies, rounded to bf16 and stored together with their 64-column sums in the
+//      activation image the streaming kernel copies to shared memory;
+//  (2) the CTA multiplies the 256 ORIGINAL columns of the chunk with B: partial sums
+//      t_part[chunk][token][j] (fp32) of the low-rank intermediate t = B x, which the forward
+//      kernel adds up in chunk order.
+// Launched with programmatic stream serialization: perm (layer data) is read before the wait, the
+// activations after it.
+__global__ void __launch_bounds__(256)
+prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
+                const __half* __restrict__ B, unsigned char* __restrict__ act_image, float* __restrict__ t_part,
+                int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T) {
+    constexpr int kXs = 258;       // fp32 row stride of the staged activations
+    constexpr int kBs = 256 + 8;   // fp16 row stride of the staged slab of B
+    __shared__ __align__(16) float xsf[8 * kXs];
+    __shared__ __align__(16) __half bs[32 * kBs];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int chunk = blockIdx.x, tok0 = blockIdx.y * 8;
+    const int col0 = chunk * 256 + lane * 8;
+
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    int pidx[8];
+    if (col0 < n) {
+        const int4 p0 = __ldg(reinterpret_cast<const int4*>(perm + col0));
+        const int4 p1 = __ldg(reinterpret_cast<const int4*>(perm + col0 + 4));
+        pidx[0] = p0.x; pidx[1] = p0.y; pidx[2] = p0.z; pidx[3] = p0.w;
+        pidx[4] = p1.x; pidx[5] = p1.y; pidx[6] = p1.z; pidx[7] = p1.w;
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (status != nullptr && chunk == 0 && tok0 == 0 && tid == 0) *status = LOPRO_OK;
+
+    // (1) rotation: token tok0 + warp
+    const int tok = tok0 + warp;
+    if (tok < T) {
+        float v[8];
+        const __nv_bfloat16* xrow = x + (size_t)tok * ldx;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = col0 < n ? __bfloat162float(xrow[pidx[e]]) : 0.0f;
+        const bool rot = col0 >= b_i;  // whole Hadamard blocks lie on one side of b_I
+        float r[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) r[e] = v[e];
+#pragma unroll
+        for (int h = 1; h < 8; h <<= 1) {
+            if (h < b_h) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    if ((e & h) == 0) {
+                        const float a = r[e], b = r[e + h];
+                        r[e] = a + b;
+                        r[e + h] = a - b;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            if (d * 8 < b_h) {
+                const bool upper = (lane & d) != 0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float other = __shfl_xor_sync(0xffffffffu, r[e], d);
+                    r[e] = upper ? other - r[e] : r[e] + other;
+                }
+            }
+        }
+        __nv_bfloat16 o[8];
+        float sum = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            o[e] = rot ? __float2bfloat16_rn(r[e] * inv_sqrt_bh) : __float2bfloat16_rn(v[e]);
+            sum += __bfloat162float(o[e]);
+        }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+        if (col0 < n) {
+            // record of (stage, token) in the activation image: 1024 entries, then the 16 sums
+            unsigned char* rec = act_image + ((size_t)(col0 >> 10) * t_pad + tok) * kActRecord;
+            *reinterpret_cast<uint4*>(rec + (col0 & 1023) * 2) = *reinterpret_cast<const uint4*>(o);
+            if ((lane & 7) == 0) reinterpret_cast<float*>(rec + 2048)[(col0 & 1023) >> 6] = sum;
+        }
+    }
+
+    // (2) partial low-rank down-projection over the chunk's original columns
+    if (r_pad == 0) return;
+    for (int i = tid; i < 8 * 256; i += 256) {
+        const int tk = i >> 8, k = i & 255, col = chunk * 256 + k;
+        xsf[tk * kXs + k] = (tok0 + tk < T && col < n) ? __bfloat162float(x[(size_t)(tok0 + tk) * ldx + col]) : 0.0f;
+    }
+    const int j = tid >> 3, tk = tid & 7;
+    for (int jg = 0; jg < r_pad; jg += 32) {
+        __syncthreads();
+        for (int i = tid; i < 32 * 32; i += 256) {
+            const int jr = i >> 5, c8 = (i & 31) * 8, col = chunk * 256 + c8;
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (jg + jr < r_pad && col < n) w = __ldg(reinterpret_cast<const uint4*>(B + (size_t)(jg + jr) * n + col));
+            *reinterpret_cast<uint4*>(bs + jr * kBs + c8) = w;
+        }
+        __syncthreads();
+        float acc = 0.0f;
+#pragma unroll 8
+        for (int k = 0; k < 256; k += 2) {
+            const float2 bf = __half22float2(*reinterpret_cast<const __half2*>(bs + j * kBs + k));
+            const float2 xf = *reinterpret_cast<const float2*>(xsf + tk * kXs + k);
+            acc = fmaf(bf.x, xf.x, acc);
+            acc = fmaf(bf.y, xf.y, acc);
+        }
+        if (jg + j < r_pad) t_part[((size_t)chunk * t_pad + tok0 + tk) * r_pad + jg + j] = acc;
+    }
+}
+
 template <int E>
 cudaError_t launch_rotate_e(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
-                            __nv_bfloat16* xrot, int64_t ldo, float* s64, int T, cudaStream_t s) {
+                            __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s) {
     const size_t smem = (size_t)d.d_in * 4;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(rotate_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(rotate_kernel<E>, 32768 * 4, &attr_done);  // largest supported row
+    if (e != cudaSuccess) return e;
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
-    rotate_kernel<E><<<T, kRotThreads, smem, s>>>(x, ldx, perm, xrot, ldo, s64, d.d_in, d.identity_cols,
-                                                  d.block_size, inv);
+    rotate_kernel<E><<<T, kRotThreads, smem, s>>>(x, ldx, perm, xrot, ldo, s64, s64_stride(d.d_in), status, d.d_in,
+                                                  d.identity_cols, d.block_size, inv);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_rotate(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
-                          __nv_bfloat16* xrot, int64_t ldo, float* s64, int T, cudaStream_t s) {
-    if (d.block_size <= 256) return launch_rotate_e<8>(d, perm, x, ldx, xrot, ldo, s64, T, s);
-    if (d.block_size == 512) return launch_rotate_e<16>(d, perm, x, ldx, xrot, ldo, s64, T, s);
-    return launch_rotate_e<32>(d, perm, x, ldx, xrot, ldo, s64, T, s);
+                          __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s) {
+    if (d.block_size <= 256) return launch_rotate_e<8>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
+    if (d.block_size == 512) return launch_rotate_e<16>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
+    return launch_rotate_e<32>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
+}
+
+bool prologue_supported(const lopro_desc& d, int T) {
+    return T <= kDecodeMaxT && d.block_size <= 256 && d.identity_cols % d.block_size == 0;
+}
+
+cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
+                            const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, float* t_part, int t_pad,
+                            int* status, int T, cudaStream_t s) {
+    const float inv = (float)(1.0 / sqrt((double)d.block_size));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((d.d_in + 255) / 256, (T + 7) / 8);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prologue_kernel, x, ldx, perm, B, act_image, t_part, status, d.d_in,
+                              d.identity_cols, d.block_size, inv, d.rank > 0 ? r_pad : 0, t_pad, T);
 }
 
 cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,

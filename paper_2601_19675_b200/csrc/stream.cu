@@ -1,0 +1,461 @@
+// Small-batch forward (decode, T <= 32): y = W^ x~ + A t, the packed codes streamed once from HBM
+// by bulk asynchronous copies (steps "Dequant(W_q) X" and "U (Sigma Y)" of Appendix A.3, summed as
+// in Eq. 8).
+//
+// One CTA owns 32 output rows (two 16-row tiles of the fragment layout) over the WHOLE K range, so
+// no partial sums ever cross CTAs.  A producer warp fills a ring of shared-memory stages with
+// cp.async.bulk copies (16 steps of 64 columns per stage): the layer's own data -- codes,
+// (scale, zero) pairs, the rows of A -- is requested before griddepcontrol.wait, i.e. while the
+// prologue kernel of the same forward still runs; the rotated activations and their 64-column
+// sums follow after the wait.  Sixteen consumer warps split each stage by K step (warp w takes
+// step w), multiply with mma.sync and keep their sums in registers; one shared-memory reduction
+// over the warps at the end, then the low-rank term and the store.
+//
+// Arithmetic: as in the general path, sum_k s (c_k - z) x~_k = s (sum_k (128 + c_k) x~_k
+// - (128 + z) sum_k x~_k), the first sum on the tensor cores with exact bf16 operands 128 + c_k,
+// fp32 accumulation, scale and zero-point applied in fp32 once per 64 columns.
+//
+// Every wait on an mbarrier is bounded; a wait that runs out stores LOPRO_ERR_TIMEOUT in the
+// workspace status word and the CTA stops waiting (its outputs are then unspecified).
+#include "common.cuh"
+
+namespace lopro {
+
+namespace {
+
+constexpr int kConsumerWarps = 16;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
+constexpr int kStageSteps = 16;                      // 64-column steps per stage = one per consumer warp
+constexpr int kStageCols = kStageSteps * 64;
+constexpr int kXsStride = kActRecord / 2;            // bf16 elements between the token rows of a stage
+constexpr int kRowTiles = 2;                         // 16-row tiles per CTA
+constexpr int kMaxStages = 8;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct StreamParams {
+    const uint32_t* codes;
+    const uint32_t* sz;
+    const __half* A;
+    const unsigned char* act;   // activation image [stage][t_pad][kActRecord]
+    const float* t_part;        // [chunks][t_pad][r_pad]
+    int* status;
+    void* y;
+    int64_t ldy;
+    int out_f32;
+    int m, n, T, t_pad;
+    int nsteps, gshift, ng, r_pad;
+    int n_stages;  // ring depth
+    int total_stages;
+    // shared-memory layout (bytes from the dynamic base)
+    int off_sz, off_a, off_t, off_ring, stage_bytes, off_stage_x;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the limit ran out (the caller records the time-out and carries on).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+constexpr uint32_t kMagic128 = 0x43004300u;  // two bf16 128.0 (ulp 1): 128.0 | c == 128 + c
+
+template <int BITS>
+__device__ __forceinline__ void expand_codes(uint32_t (&a)[16], const uint32_t (&w)[BITS]) {
+    if constexpr (BITS == 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = ((w[j] >> (4 * rho)) & 0x000F000Fu) | kMagic128;
+    } else if constexpr (BITS == 2) {
+#pragma unroll
+        for (int pi = 0; pi < 16; ++pi) a[pi] = ((w[pi >> 3] >> (2 * (pi & 7))) & 0x00030003u) | kMagic128;
+    } else {
+#pragma unroll
+        for (int pi = 0; pi < 15; ++pi) a[pi] = ((w[pi / 5] >> (3 * (pi % 5))) & 0x00070007u) | kMagic128;
+        a[15] = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u) | kMagic128;
+    }
+}
+
+template <int BITS, int NT>
+__global__ void __launch_bounds__(kThreads, 1)
+stream_kernel(const StreamParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) uint64_t bars[3 * kMaxStages + 1];  // wfull, xfull, empty per stage; one for sz / A
+    __shared__ int s_timeout;
+    constexpr int kTok = NT * 8;
+    constexpr int kStepBytes = 128 * BITS;  // codes of one 16-row tile and one 64-column step
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gq = lane >> 2, tg = lane & 3;
+    const int rt0 = blockIdx.x * kRowTiles;                         // first 16-row tile of this CTA
+    const int n_rt = min(kRowTiles, (p.m >> 4) - rt0);              // live row tiles (1 or 2)
+    const int tc = min(kTok, p.T);                                  // live tokens
+    const uint32_t bar0 = smem_u32(bars);
+    auto wfull = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto xfull = [&](int s) { return bar0 + 8u * (uint32_t)(kMaxStages + s); };
+    auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kMaxStages + s); };
+    const uint32_t cbar = bar0 + 8u * (uint32_t)(3 * kMaxStages);
+    const uint32_t smem0 = smem_u32(smem);
+
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (tid == 0) {
+        for (int s = 0; s < p.n_stages; ++s) {
+            mbar_init(wfull(s), 1);
+            mbar_init(xfull(s), 1);
+            mbar_init(empty(s), kConsumerWarps);
+        }
+        mbar_init(cbar, 1);
+        s_timeout = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    auto steps_of = [&](int stage) { return min(kStageSteps, p.nsteps - stage * kStageSteps); };
+    // weights of one stage: for each live row tile, `steps` consecutive steps of packed codes
+    auto issue_w = [&](int stage, int slot) {
+        const int steps = steps_of(stage);
+        const uint32_t bytes = (uint32_t)(steps * kStepBytes);
+        mbar_expect_tx(wfull(slot), bytes * (uint32_t)n_rt);
+        for (int r = 0; r < n_rt; ++r) {
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(p.codes) +
+                                       ((size_t)(rt0 + r) * p.nsteps + (size_t)stage * kStageSteps) * kStepBytes;
+            bulk_g2s(smem0 + p.off_ring + slot * p.stage_bytes + r * kStageSteps * kStepBytes, src, bytes, wfull(slot));
+        }
+    };
+    // activations of one stage: the records of the live tokens, one contiguous piece of the image
+    auto issue_x = [&](int stage, int slot) {
+        const uint32_t bytes = (uint32_t)(tc * kActRecord);
+        mbar_expect_tx(xfull(slot), bytes);
+        bulk_g2s(smem0 + p.off_ring + slot * p.stage_bytes + p.off_stage_x,
+                 p.act + (size_t)stage * p.t_pad * kActRecord, bytes, xfull(slot));
+    };
+
+    float yacc[kRowTiles][NT][4];
+#pragma unroll
+    for (int r = 0; r < kRowTiles; ++r)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) yacc[r][nt][i] = 0.0f;
+
+    if (warp == kConsumerWarps) {
+        // ---------------- producer warp ----------------
+        const int first = min(p.n_stages, p.total_stages);
+        if (lane == 0) {
+            // layer data: (scale, zero) pairs and rows of A of the live row tiles, then the first stages of codes
+            const uint32_t sz_bytes = (uint32_t)(n_rt * p.ng * 64);
+            const uint32_t a_bytes = (uint32_t)(n_rt * 16 * p.r_pad * 2);
+            mbar_expect_tx(cbar, sz_bytes + a_bytes);
+            bulk_g2s(smem0 + p.off_sz, p.sz + (size_t)rt0 * p.ng * 16, sz_bytes, cbar);
+            if (a_bytes) bulk_g2s(smem0 + p.off_a, p.A + (size_t)rt0 * 16 * p.r_pad, a_bytes, cbar);
+            for (int s = 0; s < first; ++s) issue_w(s, s);
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (lane == 0)
+            for (int s = 0; s < first; ++s) issue_x(s, s);
+        // low-rank intermediate t = sum over the prologue's column chunks (chunk order), rounded to fp16
+        if (p.r_pad > 0) {
+            __half* ts = reinterpret_cast<__half*>(smem + p.off_t);
+            const int nchunks = (p.n + 255) >> 8;
+            for (int i = lane; i < kTok * p.r_pad; i += 32) {
+                const int tk = i / p.r_pad, j = i - tk * p.r_pad;
+                float acc = 0.0f;
+                if (tk < tc) {
+                    const float* src = p.t_part + (size_t)tk * p.r_pad + j;
+                    for (int c = 0; c < nchunks; ++c) acc += __ldcg(src + (size_t)c * p.t_pad * p.r_pad);
+                }
+                ts[i] = __float2half_rn(acc);
+            }
+        }
+        if (lane == 0) {
+            for (int s = first; s < p.total_stages; ++s) {
+                const int slot = s % p.n_stages;
+                const uint32_t parity = (uint32_t)((s / p.n_stages) - 1) & 1u;
+                if (!s_timeout && !mbar_wait(empty(slot), parity)) {
+                    s_timeout = 1;
+                    atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+                }
+                issue_w(s, slot);
+                issue_x(s, slot);
+            }
+        }
+    } else {
+        // ---------------- consumer warps ----------------
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (!mbar_wait(cbar, 0)) {
+            s_timeout = 1;
+            if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+        }
+        const uint32_t* szs = reinterpret_cast<const uint32_t*>(smem + p.off_sz);
+        const uint32_t ldm_off = (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
+        for (int s = 0; s < p.total_stages; ++s) {
+            const int slot = s % p.n_stages;
+            const uint32_t parity = (uint32_t)(s / p.n_stages) & 1u;
+            if (!s_timeout && !(mbar_wait(wfull(slot), parity) && mbar_wait(xfull(slot), parity))) {
+                s_timeout = 1;
+                if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+            }
+            const int steps = steps_of(s);
+            if (warp < steps) {
+                const unsigned char* stage = smem + p.off_ring + slot * p.stage_bytes;
+                const uint32_t xs_u32 = smem0 + p.off_ring + slot * p.stage_bytes + p.off_stage_x;
+                const unsigned char* srec = stage + p.off_stage_x + 2048;  // sums of token 0
+                const int grp = (s * kStageSteps + warp) >> p.gshift;
+                // B operand: the 64 columns of step `warp`, all token tiles
+                uint32_t b[NT][8];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint32_t base = xs_u32 + (uint32_t)(nt * 8 * kXsStride + warp * 64) * 2u + ldm_off;
+                    ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][0]), base);
+                    ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][4]), base + 64u);
+                }
+                float sx[NT][2];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    sx[nt][0] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg) * kActRecord)[warp];
+                    sx[nt][1] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg + 1) * kActRecord)[warp];
+                }
+#pragma unroll
+                for (int r = 0; r < kRowTiles; ++r) {
+                    if (r < n_rt) {
+                        uint32_t w[BITS];
+                        const uint32_t* wp = reinterpret_cast<const uint32_t*>(stage + (r * kStageSteps + warp) * kStepBytes) +
+                                             lane * BITS;
+                        if constexpr (BITS == 4) {
+                            const uint4 v = *reinterpret_cast<const uint4*>(wp);
+                            w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+                        } else if constexpr (BITS == 2) {
+                            const uint2 v = *reinterpret_cast<const uint2*>(wp);
+                            w[0] = v.x; w[1] = v.y;
+                        } else {
+#pragma unroll
+                            for (int q = 0; q < BITS; ++q) w[q] = wp[q];
+                        }
+                        uint32_t a[16];
+                        expand_codes<BITS>(a, w);
+                        const uint32_t sz_lo = szs[(r * p.ng + grp) * 16 + gq], sz_hi = szs[(r * p.ng + grp) * 16 + gq + 8];
+                        const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
+                        const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
+                        const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                            mma_bf16(acc, &a[0], b[nt][0], b[nt][1]);
+                            mma_bf16(acc, &a[4], b[nt][2], b[nt][3]);
+                            mma_bf16(acc, &a[8], b[nt][4], b[nt][5]);
+                            mma_bf16(acc, &a[12], b[nt][6], b[nt][7]);
+                            yacc[r][nt][0] = fmaf(f_lo.x, acc[0], fmaf(nsz_lo, sx[nt][0], yacc[r][nt][0]));
+                            yacc[r][nt][1] = fmaf(f_lo.x, acc[1], fmaf(nsz_lo, sx[nt][1], yacc[r][nt][1]));
+                            yacc[r][nt][2] = fmaf(f_hi.x, acc[2], fmaf(nsz_hi, sx[nt][0], yacc[r][nt][2]));
+                            yacc[r][nt][3] = fmaf(f_hi.x, acc[3], fmaf(nsz_hi, sx[nt][1], yacc[r][nt][3]));
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty(slot));
+        }
+    }
+    __syncthreads();  // every stage consumed, t staged: the ring can be reused for the reduction
+
+    // low-rank up-projection A t: warp r adds the term of row tile r (fp16 tensor-core product into
+    // the fp32 sums)
+    auto lowrank_up = [&](float (&acc)[NT][4], int r) {
+        const __half* as = reinterpret_cast<const __half*>(smem + p.off_a) + (size_t)r * 16 * p.r_pad;
+        const __half* ts = reinterpret_cast<const __half*>(smem + p.off_t);
+        for (int jj = 0; jj < p.r_pad; jj += 16) {
+            uint32_t a[4];
+            a[0] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 2 * tg);
+            a[1] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 2 * tg);
+            a[2] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 8 + 2 * tg);
+            a[3] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 8 + 2 * tg);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const __half* trow = ts + (nt * 8 + gq) * p.r_pad + jj + 2 * tg;
+                mma_f16(acc[nt], a, *reinterpret_cast<const uint32_t*>(trow), *reinterpret_cast<const uint32_t*>(trow + 8));
+            }
+        }
+    };
+    if (p.r_pad > 0) {
+        if (warp == 0) lowrank_up(yacc[0], 0);
+        else if (warp == 1 && n_rt > 1) lowrank_up(yacc[1], 1);
+    }
+
+    // reduction over the consumer warps: red[warp][token][32 rows]
+    float* red = reinterpret_cast<float*>(smem + p.off_ring);
+    if (warp < kConsumerWarps) {
+#pragma unroll
+        for (int r = 0; r < kRowTiles; ++r)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int tk = nt * 8 + 2 * tg + (i & 1), rl = r * 16 + gq + 8 * (i >> 1);
+                    red[(warp * kTok + tk) * 32 + rl] = yacc[r][nt][i];
+                }
+    }
+    __syncthreads();
+    const int rows_here = n_rt * 16;
+    for (int i = tid; i < tc * 32; i += kThreads) {
+        const int tk = i >> 5, rl = i & 31;
+        if (rl < rows_here) {
+            float sum = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) sum += red[(w * kTok + tk) * 32 + rl];
+            const size_t o = (size_t)tk * p.ldy + (size_t)rt0 * 16 + rl;
+            if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = sum;
+            else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(sum);
+        }
+    }
+}
+
+template <int BITS, int NT>
+cudaError_t launch_stream_nt(const StreamParams& p, int smem_bytes, cudaStream_t s) {
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(stream_kernel<BITS, NT>, kStreamMaxSmem, &attr_done);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((p.m / 16 + kRowTiles - 1) / kRowTiles);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, stream_kernel<BITS, NT>, p);
+}
+
+template <int BITS>
+cudaError_t launch_stream_bits(const StreamParams& p, int nt, int smem_bytes, cudaStream_t s) {
+    if (nt == 1) return launch_stream_nt<BITS, 1>(p, smem_bytes, s);
+    if (nt == 2) return launch_stream_nt<BITS, 2>(p, smem_bytes, s);
+    return launch_stream_nt<BITS, 4>(p, smem_bytes, s);
+}
+
+struct StreamPlan {
+    int nt, n_stages, total_stages, smem_bytes;
+    int off_sz, off_a, off_t, off_ring, stage_bytes, off_stage_x;
+};
+
+bool plan_stream(const lopro_desc& d, int T, StreamPlan* pl) {
+    if (T < 1 || T > kDecodeMaxT) return false;
+    const int r_pad = d.rank > 0 ? round_up_int(d.rank, 16) : 0;
+    const int ng = d.d_in / d.group_size;
+    pl->nt = T <= 8 ? 1 : (T <= 16 ? 2 : 4);
+    const int ktok = pl->nt * 8;
+    int off = 0;
+    pl->off_sz = off;
+    off += round_up_int(kRowTiles * ng * 64, 128);
+    pl->off_a = off;
+    off += round_up_int(kRowTiles * 16 * r_pad * 2, 128);
+    pl->off_t = off;
+    off += round_up_int(ktok * r_pad * 2, 128);
+    pl->off_ring = off;
+    const int w_bytes = kRowTiles * kStageSteps * 128 * d.bits;
+    pl->off_stage_x = w_bytes;
+    pl->stage_bytes = round_up_int(w_bytes + ktok * kActRecord, 128);
+    pl->total_stages = (d.d_in / 64 + kStageSteps - 1) / kStageSteps;
+    const int red_bytes = kConsumerWarps * ktok * 32 * 4;
+    int stages = (kStreamMaxSmem - off) / pl->stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages > pl->total_stages) stages = pl->total_stages;
+    if (stages < 1) return false;
+    int ring = stages * pl->stage_bytes;
+    if (ring < red_bytes) ring = red_bytes;
+    pl->n_stages = stages;
+    pl->smem_bytes = off + ring;
+    return pl->smem_bytes <= kStreamMaxSmem;
+}
+
+}  // namespace
+
+bool stream_supported(const lopro_desc& d, int T) {
+    StreamPlan pl;
+    return plan_stream(d, T, &pl);
+}
+
+cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
+                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s) {
+    StreamPlan pl;
+    if (!plan_stream(d, T, &pl)) return cudaErrorInvalidValue;
+    StreamParams p;
+    p.codes = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_CODES]);
+    p.sz = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_SCALEZERO]);
+    p.A = reinterpret_cast<const __half*>(blob + L.off[LOPRO_SEC_A]);
+    p.act = ws + W.off_xrot;
+    p.t_part = reinterpret_cast<const float*>(ws + W.off_tpart);
+    p.status = reinterpret_cast<int*>(const_cast<uint8_t*>(ws) + W.off_status);
+    p.y = y;
+    p.ldy = ldy;
+    p.out_f32 = out_dtype == LOPRO_OUT_F32;
+    p.m = d.d_out;
+    p.n = d.d_in;
+    p.T = T;
+    p.t_pad = W.t_pad;
+    p.nsteps = d.d_in / 64;
+    int gs = d.group_size / 64, gshift = 0;
+    while ((1 << gshift) < gs) ++gshift;
+    p.gshift = gshift;
+    p.ng = d.d_in / d.group_size;
+    p.r_pad = d.rank > 0 ? L.r_pad : 0;
+    p.n_stages = pl.n_stages;
+    p.total_stages = pl.total_stages;
+    p.off_sz = pl.off_sz;
+    p.off_a = pl.off_a;
+    p.off_t = pl.off_t;
+    p.off_ring = pl.off_ring;
+    p.stage_bytes = pl.stage_bytes;
+    p.off_stage_x = pl.off_stage_x;
+    switch (d.bits) {
+        case 2: return launch_stream_bits<2>(p, pl.nt, pl.smem_bytes, s);
+        case 3: return launch_stream_bits<3>(p, pl.nt, pl.smem_bytes, s);
+        default: return launch_stream_bits<4>(p, pl.nt, pl.smem_bytes, s);
+    }
+}
+
+}  // namespace lopro
