@@ -65,8 +65,6 @@ lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
     off += round_up_size((size_t)t_pad * s64_stride(d.d_in) * 4, 256);
     W->off_t = off;
     off += round_up_size((size_t)t_pad * (r_pad > 0 ? r_pad : 16) * 2, 256);
-    W->off_tpart = off;
-    if (t_pad <= kDecodeMaxT) off += round_up_size((size_t)((d.d_in + 255) / 256) * t_pad * r_pad * 4, 256);
     W->total = off;
     return LOPRO_OK;
 }
@@ -225,7 +223,7 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
         // small batch: prologue + streaming kernel, chained by programmatic launches
         if (launch_prologue(*desc, perm, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot,
-                            (float*)(ws + W.off_tpart), W.t_pad, status, T, s) != cudaSuccess)
+                            (__half*)(ws + W.off_t), W.t_pad, status, T, s) != cudaSuccess)
             return LOPRO_ERR_CUDA;
         if (launch_stream(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;
         return LOPRO_OK;

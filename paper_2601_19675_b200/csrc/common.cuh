@@ -68,7 +68,7 @@ inline size_t round_up_size(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // activations, low-rank intermediate (fp16, general path), per-chunk partial sums of the low-rank
 // intermediate (fp32, small-batch path).
 struct WorkspaceLayout {
-    size_t off_status, off_xrot, off_s64, off_t, off_tpart, total;
+    size_t off_status, off_xrot, off_s64, off_t, total;
     int t_pad;  // tokens padded to a multiple of 8
 };
 constexpr int kDecodeMaxT = 32;               // tokens per CTA of the streaming kernels
@@ -98,10 +98,10 @@ cudaError_t launch_unpack(const lopro_desc& d, const void* blob, const BlobLayou
 // entries, [T][n/64] fp32.
 cudaError_t launch_rotate(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
                           __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s);
-// Small-batch prologue: rotation, 64-column sums and per-chunk partial sums of B x in one launch.
+// Small-batch prologue: rotation, 64-column sums and t = B x in one launch.
 bool prologue_supported(const lopro_desc& d, int T);
 cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
-                            const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, float* t_part, int t_pad,
+                            const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, __half* t, int t_pad,
                             int* status, int T, cudaStream_t s);
 // t[T][r_pad] (fp16) = B x, fp32 accumulation.
 cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,

@@ -142,30 +142,114 @@ lowrank_down_kernel(const __half* __restrict__ B, const __nv_bfloat16* __restric
     }
 }
 
-// Prologue of the small-batch forward (T <= 32, b_H <= 256, b_I a multiple of b_H): one CTA per
-// chunk of 256 columns and group of 8 tokens.
-//  (1) warp w rotates the chunk's 256 output columns of token w: the 8 entries of a lane are
-//      gathered from global memory through perm, transformed with register and shuffle
-//      butterflies, rounded to bf16 and stored together with their 64-column sums in the
-//      activation image the streaming kernel copies to shared memory;
-//  (2) the CTA multiplies the 256 ORIGINAL columns of the chunk with B: partial sums
-//      t_part[chunk][token][j] (fp32) of the low-rank intermediate t = B x, which the forward
-//      kernel adds up in chunk order.
-// Launched with programmatic stream serialization: perm (layer data) is read before the wait, the
-// activations after it.
+// Prologue of the small-batch forward (T <= 32, b_H <= 256, b_I a multiple of b_H).  Grid:
+// x = column chunks of 256, then pairs of rows of B; y = groups of 8 tokens.
+//  * a chunk CTA rotates 256 output columns, warp w for token w: the 8 entries of a lane are
+//    gathered from global memory through perm, transformed with register and shuffle butterflies,
+//    rounded to bf16 and stored together with their 64-column sums in the activation image that the
+//    streaming kernel copies to shared memory;
+//  * a row-pair CTA computes t[token][j] = sum_k B[j][k] x[token][k] for two rows j and the 8 tokens
+//    (fp32 accumulation over all of K, one rounding to fp16): the low-rank intermediate "Y = V X".
+// Launched with programmatic stream serialization: perm and B (layer data) are read before the
+// wait, the activations after it.
 __global__ void __launch_bounds__(256)
 prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
-                const __half* __restrict__ B, unsigned char* __restrict__ act_image, float* __restrict__ t_part,
+                const __half* __restrict__ B, unsigned char* __restrict__ act_image, __half* __restrict__ t,
                 int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T) {
-    constexpr int kXs = 258;       // fp32 row stride of the staged activations
-    constexpr int kBs = 256 + 8;   // fp16 row stride of the staged slab of B
-    __shared__ __align__(16) float xsf[8 * kXs];
-    __shared__ __align__(16) __half bs[32 * kBs];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int chunk = blockIdx.x, tok0 = blockIdx.y * 8;
-    const int col0 = chunk * 256 + lane * 8;
-
+    const int nchunks = (n + 255) >> 8;
+    const int tok0 = blockIdx.y * 8;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    if ((int)blockIdx.x >= nchunks) {
+        // ---- two rows of B against eight tokens ----
+        __shared__ float part[8][16];
+        const int j0 = 2 * ((int)blockIdx.x - nchunks);
+        const __half* b0 = B + (size_t)j0 * n;
+        const __half* b1 = b0 + n;
+        const int npass = (n + 2047) >> 11;
+        uint4 pre[2][2];
+#pragma unroll
+        for (int ps = 0; ps < 2; ++ps) {
+            const int k = ps * 2048 + tid * 8;
+            pre[ps][0] = pre[ps][1] = make_uint4(0, 0, 0, 0);
+            if (k < n) {
+                pre[ps][0] = __ldg(reinterpret_cast<const uint4*>(b0 + k));
+                pre[ps][1] = __ldg(reinterpret_cast<const uint4*>(b1 + k));
+            }
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        float acc[2][8];
+#pragma unroll
+        for (int r = 0; r < 2; ++r)
+#pragma unroll
+            for (int tk = 0; tk < 8; ++tk) acc[r][tk] = 0.0f;
+        for (int ps = 0; ps < npass; ++ps) {
+            const int k = ps * 2048 + tid * 8;
+            if (k >= n) break;
+            uint4 bw[2];
+            if (ps == 0) {
+                bw[0] = pre[0][0];
+                bw[1] = pre[0][1];
+            } else if (ps == 1) {
+                bw[0] = pre[1][0];
+                bw[1] = pre[1][1];
+            } else {
+                bw[0] = __ldg(reinterpret_cast<const uint4*>(b0 + k));
+                bw[1] = __ldg(reinterpret_cast<const uint4*>(b1 + k));
+            }
+            float bf[2][8];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const __half2* h = reinterpret_cast<const __half2*>(&bw[r]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 f = __half22float2(h[i]);
+                    bf[r][2 * i] = f.x;
+                    bf[r][2 * i + 1] = f.y;
+                }
+            }
+            uint4 xw[8];
+#pragma unroll
+            for (int tk = 0; tk < 8; ++tk)
+                xw[tk] = tok0 + tk < T ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tok0 + tk) * ldx + k))
+                                       : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int tk = 0; tk < 8; ++tk) {
+                const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xw[tk]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 f = __bfloat1622float2(xh[i]);
+                    acc[0][tk] = fmaf(bf[0][2 * i], f.x, acc[0][tk]);
+                    acc[0][tk] = fmaf(bf[0][2 * i + 1], f.y, acc[0][tk]);
+                    acc[1][tk] = fmaf(bf[1][2 * i], f.x, acc[1][tk]);
+                    acc[1][tk] = fmaf(bf[1][2 * i + 1], f.y, acc[1][tk]);
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r)
+#pragma unroll
+            for (int tk = 0; tk < 8; ++tk) {
+                float v = acc[r][tk];
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+                if (lane == 0) part[warp][r * 8 + tk] = v;
+            }
+        __syncthreads();
+        if (tid < 16) {
+            float v = 0.0f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) v += part[w][tid];
+            const int r = tid >> 3, tk = tid & 7;
+            if (tok0 + tk < T && j0 + r < r_pad) t[(size_t)(tok0 + tk) * r_pad + j0 + r] = __float2half_rn(v);
+        }
+        return;
+    }
+
+    // ---- rotation of one chunk of 256 output columns, warp = token ----
+    const int chunk = blockIdx.x;
+    const int col0 = chunk * 256 + lane * 8;
     int pidx[8];
     if (col0 < n) {
         const int4 p0 = __ldg(reinterpret_cast<const int4*>(perm + col0));
@@ -228,33 +312,6 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
             if ((lane & 7) == 0) reinterpret_cast<float*>(rec + 2048)[(col0 & 1023) >> 6] = sum;
         }
     }
-
-    // (2) partial low-rank down-projection over the chunk's original columns
-    if (r_pad == 0) return;
-    for (int i = tid; i < 8 * 256; i += 256) {
-        const int tk = i >> 8, k = i & 255, col = chunk * 256 + k;
-        xsf[tk * kXs + k] = (tok0 + tk < T && col < n) ? __bfloat162float(x[(size_t)(tok0 + tk) * ldx + col]) : 0.0f;
-    }
-    const int j = tid >> 3, tk = tid & 7;
-    for (int jg = 0; jg < r_pad; jg += 32) {
-        __syncthreads();
-        for (int i = tid; i < 32 * 32; i += 256) {
-            const int jr = i >> 5, c8 = (i & 31) * 8, col = chunk * 256 + c8;
-            uint4 w = make_uint4(0, 0, 0, 0);
-            if (jg + jr < r_pad && col < n) w = __ldg(reinterpret_cast<const uint4*>(B + (size_t)(jg + jr) * n + col));
-            *reinterpret_cast<uint4*>(bs + jr * kBs + c8) = w;
-        }
-        __syncthreads();
-        float acc = 0.0f;
-#pragma unroll 8
-        for (int k = 0; k < 256; k += 2) {
-            const float2 bf = __half22float2(*reinterpret_cast<const __half2*>(bs + j * kBs + k));
-            const float2 xf = *reinterpret_cast<const float2*>(xsf + tk * kXs + k);
-            acc = fmaf(bf.x, xf.x, acc);
-            acc = fmaf(bf.y, xf.y, acc);
-        }
-        if (jg + j < r_pad) t_part[((size_t)chunk * t_pad + tok0 + tk) * r_pad + jg + j] = acc;
-    }
 }
 
 template <int E>
@@ -284,11 +341,11 @@ bool prologue_supported(const lopro_desc& d, int T) {
 }
 
 cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
-                            const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, float* t_part, int t_pad,
+                            const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, __half* t, int t_pad,
                             int* status, int T, cudaStream_t s) {
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((d.d_in + 255) / 256, (T + 7) / 8);
+    cfg.gridDim = dim3((d.d_in + 255) / 256 + (d.rank > 0 ? r_pad / 2 : 0), (T + 7) / 8);
     cfg.blockDim = dim3(256);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = s;
@@ -297,7 +354,7 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prologue_kernel, x, ldx, perm, B, act_image, t_part, status, d.d_in,
+    return cudaLaunchKernelEx(&cfg, prologue_kernel, x, ldx, perm, B, act_image, t, status, d.d_in,
                               d.identity_cols, d.block_size, inv, d.rank > 0 ? r_pad : 0, t_pad, T);
 }
 

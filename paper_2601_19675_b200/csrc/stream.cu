@@ -37,7 +37,7 @@ struct StreamParams {
     const uint32_t* sz;
     const __half* A;
     const unsigned char* act;   // activation image [stage][t_pad][kActRecord]
-    const float* t_part;        // [chunks][t_pad][r_pad]
+    const __half* t;            // [T][r_pad] low-rank intermediate
     int* status;
     void* y;
     int64_t ldy;
@@ -123,7 +123,7 @@ template <int BITS, int NT>
 __global__ void __launch_bounds__(kThreads, 1)
 stream_kernel(const StreamParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t bars[3 * kMaxStages + 1];  // wfull, xfull, empty per stage; one for sz / A
+    __shared__ __align__(8) uint64_t bars[3 * kMaxStages + 2];  // wfull, xfull, empty per stage; sz + A; t
     __shared__ int s_timeout;
     constexpr int kTok = NT * 8;
     constexpr int kStepBytes = 128 * BITS;  // codes of one 16-row tile and one 64-column step
@@ -138,6 +138,7 @@ stream_kernel(const StreamParams p) {
     auto xfull = [&](int s) { return bar0 + 8u * (uint32_t)(kMaxStages + s); };
     auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kMaxStages + s); };
     const uint32_t cbar = bar0 + 8u * (uint32_t)(3 * kMaxStages);
+    const uint32_t tbar = cbar + 8u;
     const uint32_t smem0 = smem_u32(smem);
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -148,6 +149,7 @@ stream_kernel(const StreamParams p) {
             mbar_init(empty(s), kConsumerWarps);
         }
         mbar_init(cbar, 1);
+        mbar_init(tbar, 1);
         s_timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -194,20 +196,12 @@ stream_kernel(const StreamParams p) {
             for (int s = 0; s < first; ++s) issue_w(s, s);
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (lane == 0)
+        if (lane == 0) {
             for (int s = 0; s < first; ++s) issue_x(s, s);
-        // low-rank intermediate t = sum over the prologue's column chunks (chunk order), rounded to fp16
-        if (p.r_pad > 0) {
-            __half* ts = reinterpret_cast<__half*>(smem + p.off_t);
-            const int nchunks = (p.n + 255) >> 8;
-            for (int i = lane; i < kTok * p.r_pad; i += 32) {
-                const int tk = i / p.r_pad, j = i - tk * p.r_pad;
-                float acc = 0.0f;
-                if (tk < tc) {
-                    const float* src = p.t_part + (size_t)tk * p.r_pad + j;
-                    for (int c = 0; c < nchunks; ++c) acc += __ldcg(src + (size_t)c * p.t_pad * p.r_pad);
-                }
-                ts[i] = __float2half_rn(acc);
+            if (p.r_pad > 0) {  // low-rank intermediate of the live tokens
+                const uint32_t t_bytes = (uint32_t)(tc * p.r_pad * 2);
+                mbar_expect_tx(tbar, t_bytes);
+                bulk_g2s(smem0 + p.off_t, p.t, t_bytes, tbar);
             }
         }
         if (lane == 0) {
@@ -319,9 +313,10 @@ stream_kernel(const StreamParams p) {
             }
         }
     };
-    if (p.r_pad > 0) {
+    if (p.r_pad > 0 && warp < n_rt) {
+        if (!mbar_wait(tbar, 0) && lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
         if (warp == 0) lowrank_up(yacc[0], 0);
-        else if (warp == 1 && n_rt > 1) lowrank_up(yacc[1], 1);
+        else lowrank_up(yacc[1], 1);
     }
 
     // reduction over the consumer warps: red[warp][token][32 rows]
@@ -428,7 +423,7 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
     p.sz = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_SCALEZERO]);
     p.A = reinterpret_cast<const __half*>(blob + L.off[LOPRO_SEC_A]);
     p.act = ws + W.off_xrot;
-    p.t_part = reinterpret_cast<const float*>(ws + W.off_tpart);
+    p.t = reinterpret_cast<const __half*>(ws + W.off_t);
     p.status = reinterpret_cast<int*>(const_cast<uint8_t*>(ws) + W.off_status);
     p.y = y;
     p.ldy = ldy;
