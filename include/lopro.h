@@ -185,6 +185,31 @@ LOPRO_API lopro_status lopro_linear_fwd_host(const lopro_desc* desc, const void*
                                    void* y_host, int32_t out_dtype, int32_t T, void* workspace,
                                    size_t workspace_bytes, void* stream);
 
+/* Forward for callers that cannot allocate device memory (the paper has no counterpart of this entry
+ * point; it is a deployment convenience of this library).  Meant for code that runs where asking the
+ * driver for memory is not an option: a plug-in inside a host program that owns the whole device
+ * heap and hands out none of it, a latency-critical serving loop in which cudaMalloc's implicit
+ * device synchronisation would stall every other stream, or a process started with a fixed memory
+ * budget.  It computes exactly what lopro_linear_fwd computes, with the same arguments minus the
+ * workspace: the scratch is a fixed array of LOPRO_NOALLOC_SCRATCH_BYTES inside the library itself
+ * (every GPU that loads the library holds that memory until the process ends).
+ *   - Accepted sizes: lopro_workspace_bytes(desc, T) <= LOPRO_NOALLOC_SCRATCH_BYTES, which covers
+ *     the small-batch (decode) range of ordinary layers, e.g. d_in = 8192 with T <= 32.  Anything
+ *     larger returns LOPRO_ERR_BUFFER_TOO_SMALL and does nothing.
+ *   - The call allocates and frees nothing and does not synchronise.  The first call on each device
+ *     looks up the array's device address (once per device, with that device current); make that
+ *     first call before any stream capture begins.
+ *   - All calls on one device share the one array and it keeps what the last call left in it.  No
+ *     part of it needs clearing between calls (each forward rewrites what it reads), but two calls
+ *     whose kernels overlap on the GPU -- different streams, or concurrent host threads -- race on
+ *     it: order every use of this entry point on a device through one stream.
+ *   - The workspace status word of lopro_linear_fwd is not visible here; use lopro_linear_fwd when
+ *     the device-side status matters. */
+#define LOPRO_NOALLOC_SCRATCH_BYTES (2 * 1024 * 1024)
+LOPRO_API lopro_status lopro_linear_fwd_noalloc(const lopro_desc* desc, const void* packed, const uint16_t* x_bf16,
+                                                int64_t ldx, void* y, int64_t ldy, int32_t out_dtype, int32_t T,
+                                                void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,7 @@ SEC_HEADER, SEC_CODES, SEC_SCALEZERO, SEC_PERM, SEC_A, SEC_B = range(6)
 # every symbol include/lopro.h declares
 SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packed_bytes", "lopro_packed_section",
            "lopro_workspace_bytes", "lopro_pack", "lopro_unpack", "lopro_rotate", "lopro_linear_fwd",
-           "lopro_host_staging_bytes", "lopro_linear_fwd_host"]
+           "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc"]
 
 
 class Desc(ctypes.Structure):
@@ -76,6 +76,8 @@ def lib():
         L.lopro_host_staging_bytes.argtypes = [dp, i32, i32]
         L.lopro_linear_fwd_host.restype = ctypes.c_int
         L.lopro_linear_fwd_host.argtypes = [dp, vp, vp, vp, i32, i32, vp, sz, vp]
+        L.lopro_linear_fwd_noalloc.restype = ctypes.c_int
+        L.lopro_linear_fwd_noalloc.argtypes = [dp, vp, vp, i64, vp, i64, i32, i32, vp]
         _lib = L
     return _lib
 
@@ -220,6 +222,24 @@ def linear_fwd_host(desc, packed, x_host, y_host, workspace, out_dtype=OUT_BF16)
                                      _ptr(workspace), workspace.numel(), _stream())
     _check(st, "lopro_linear_fwd_host")
     return y_host
+
+
+NOALLOC_SCRATCH_BYTES = 2 * 1024 * 1024
+
+
+def linear_fwd_noalloc(desc, packed, x, y, out_dtype=OUT_BF16):
+    """lopro_linear_fwd_noalloc: the forward without a workspace argument, for callers that may not allocate
+    device memory (the scratch is a fixed array inside the library).  The binding allocates nothing either:
+    the caller passes the output tensor y [T][m].  Raises LoproError(ERR_BUFFER_TOO_SMALL) when the layer and
+    token count need more than NOALLOC_SCRATCH_BYTES of scratch."""
+    assert x.is_cuda and x.dim() == 2 and x.element_size() == 2 and x.stride(1) == 1
+    T = x.shape[0]
+    ldx = x.stride(0) if T > 1 else max(x.stride(0), desc.d_in)
+    ldy = y.stride(0) if T > 1 else max(y.stride(0), desc.d_out)
+    st = lib().lopro_linear_fwd_noalloc(ctypes.byref(desc), _ptr(packed), _ptr(x), ldx, _ptr(y), ldy, int(out_dtype), T,
+                                        _stream())
+    _check(st, "lopro_linear_fwd_noalloc")
+    return y
 
 
 def workspace_status(workspace):
