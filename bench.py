@@ -347,7 +347,7 @@ def main():
         ach = algorithmic_bytes(c, T) / dur_s / 1e9
         roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
                         traffic=None, peak_source=f"of {peaks['source']}",
-                        frac_of_nominal_8000=ach / 8000.0, kernel="decode_kernel",
+                        frac_of_nominal_8000=ach / 8000.0, kernel="stream_kernel" if T <= 32 else "decode_kernel",
                         algorithmic_bytes_per_launch=algorithmic_bytes(c, T),
                         launch_us=dur_s * 1e6, note="duration = step time / layer forwards (includes the prologue kernels)")
     else:
@@ -357,7 +357,8 @@ def main():
                         peak_source=f"of {peaks['source']} (sustained)", kernel="decode_kernel",
                         algorithmic_flops_per_launch=algorithmic_flops(c, T), launch_us=dur_s * 1e6,
                         note="duration = step time / layer forwards (includes the prologue kernels)")
-    kernels_per_forward = 3 if c["rank"] > 0 else 2
+    # T <= 32: prologue + streaming kernel; larger T: rotate + low-rank down + general kernel
+    kernels_per_forward = 2 if T <= 32 else (3 if c["rank"] > 0 else 2)
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic", config=workload_config(args.workload), clocks=clocks,
