@@ -166,10 +166,12 @@ LOPRO_API lopro_status lopro_rotate(const lopro_desc* desc, const int32_t* perm,
  *             first 4 bytes are a status word: it is set to LOPRO_OK when the call starts and a
  *             kernel that gives up on a bounded wait stores LOPRO_ERR_TIMEOUT there (read it
  *             after synchronising).  Calls that share a workspace must be ordered on one stream.
- * Arithmetic: rotated activations rounded to bf16; the code-times-activation products are
- * accumulated in fp32 (tensor cores), scales and zero-points applied in fp32; B x accumulated in
- * fp32 and rounded to fp16; A times that accumulated in fp32 into the same sum; one final
- * rounding to the output type.  T = 0 is a no-op. */
+ * Arithmetic: rotated activations rounded to bf16; B x accumulated in fp32 and rounded to fp16; A
+ * times that accumulated in fp32 into the same sum as the quantized part; one final rounding to the
+ * output type.  Quantized part, T <= 32: code-times-activation products accumulated in fp32 on the
+ * tensor cores, scales and zero-points applied in fp32 (the weights are never rounded).  T > 32:
+ * weights dequantized in fp32 and rounded once to bf16, bf16 x bf16 products accumulated in fp32.
+ * T = 0 is a no-op. */
 LOPRO_API lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const uint16_t* x_bf16, int64_t ldx,
                               void* y, int64_t ldy, int32_t out_dtype, int32_t T, void* workspace,
                               size_t workspace_bytes, void* stream);

@@ -236,6 +236,10 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
             cudaSuccess)
             return LOPRO_ERR_CUDA;
     }
+    if (prefill_supported(*desc, T)) {
+        if (launch_prefill(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+        return LOPRO_OK;
+    }
     if (launch_decode(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;
     return LOPRO_OK;
 }

@@ -114,6 +114,11 @@ bool stream_supported(const lopro_desc& d, int T);
 cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
 
+// Prefill forward (T > 32) on tcgen05 / TMEM, after launch_rotate and launch_lowrank_down.
+bool prefill_supported(const lopro_desc& d, int T);
+cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
+                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
+
 // ---- fragment layout ----------------------------------------------------------------------
 // Codes are stored per tile of 16 rows x 64 columns as [32 lanes][q words].  Lane l = 4 gq + tg
 // owns, for each of the four 16-column sub-steps j, the four register pairs rho = 0..3 of the

@@ -1,0 +1,411 @@
+// Prefill forward (T > 32): y = W^ x~ + A t as one tensor-core GEMM on tcgen05 / TMEM
+// (steps "Dequant(W_q) X" and "U (Sigma Y)" of Appendix A.3, summed as in Eq. 8).
+//
+// CTA tile: 128 weight rows (the M side of the MMA, one TMEM lane per row) x N tokens (N = 64, 128
+// or 256 TMEM columns, fp32) x 64 columns of K per pipeline stage.
+//   * warps 0-7 (dequant): each owns one 16-row tile of the fragment layout; per stage it reads its
+//     packed codes from global memory (a register ring a few stages ahead), turns them into
+//     bf16(s (c - z)) -- fp32 arithmetic, one rounding -- and writes them into the stage's A tile in
+//     the K-major 128-byte-swizzled layout the MMA reads;
+//   * warp 8 (loader): one thread brings the stage's tile of rotated activations (B operand) with a
+//     tiled TMA copy, and for the low-rank stages the tiles of A (fp16) and t (fp16);
+//   * warp 9 (MMA): one thread issues four tcgen05.mma (K = 16 each) per stage into the TMEM
+//     accumulator and commits the stage back to the producers; the rank-r term A t runs as extra K
+//     stages with fp16 operands into the same accumulator, so the sum of Eq. 8 costs no extra pass;
+//   * warps 8-11 (epilogue): tcgen05.ld the accumulator, round once, store y[token][row].
+// All mbarrier waits are bounded; a wait that runs out sets LOPRO_ERR_TIMEOUT in the workspace status
+// word, the CTA stops waiting, still frees its TMEM and returns (outputs then unspecified).
+#include <cuda.h>
+#include <stdlib.h>
+
+#include "common.cuh"
+
+namespace lopro {
+
+namespace {
+
+constexpr int kDequantWarps = 8;
+constexpr int kThreads = 12 * 32;
+constexpr int kTileM = 128;      // weight rows per CTA
+constexpr int kMaxTileN = 256;   // tokens per CTA
+constexpr int kStageK = 64;      // K columns per stage = 128 bytes of bf16 = one swizzle atom
+constexpr int kStages = 4;
+constexpr int kABytes = kTileM * 128;       // 16 KB
+constexpr int kBBytes = kMaxTileN * 128;    // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024;  // + slack for 1024-byte alignment
+constexpr int kTmemCols = 256;
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr int kCodeRing = 4;  // stages of packed codes held in registers ahead of use
+
+struct PrefillParams {
+    const uint32_t* codes;
+    const uint32_t* sz;
+    int* status;
+    void* y;
+    int64_t ldy;
+    int out_f32;
+    int m, n, T;
+    int nsteps, gshift, ng, r_pad;
+    int tile_n;      // 64, 128 or 256
+    int lr_stages;   // ceil(r_pad / 64)
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// tiled TMA load of a 2-D box (no multicast), completion counted on an mbarrier of this CTA
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem desc] * B[smem desc], M x N x 16, issued by one thread
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+// arrive on an mbarrier once every MMA issued so far by this thread has finished reading shared memory
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// K-major, 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart
+__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                        // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;              // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                        // SWIZZLE_128B
+    return d;
+}
+// instruction descriptor: fp32 accumulator, K-major A and B, M = 128, N = tile_n; fmt 1 = bf16, 0 = fp16
+__device__ __forceinline__ uint32_t make_idesc(int tile_n, uint32_t fmt) {
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+constexpr uint32_t kMagic128 = 0x43004300u;
+template <int BITS>
+__device__ __forceinline__ void expand_codes(uint32_t (&a)[16], const uint32_t (&w)[BITS]) {
+    if constexpr (BITS == 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = ((w[j] >> (4 * rho)) & 0x000F000Fu) | kMagic128;
+    } else if constexpr (BITS == 2) {
+#pragma unroll
+        for (int pi = 0; pi < 16; ++pi) a[pi] = ((w[pi >> 3] >> (2 * (pi & 7))) & 0x00030003u) | kMagic128;
+    } else {
+#pragma unroll
+        for (int pi = 0; pi < 15; ++pi) a[pi] = ((w[pi / 5] >> (3 * (pi % 5))) & 0x00070007u) | kMagic128;
+        a[15] = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u) | kMagic128;
+    }
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a,
+               const __grid_constant__ CUtensorMap map_t) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bars[3 * kStages + 1];  // full_a, full_b, empty per stage; accumulator ready
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_timeout;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tile_m = blockIdx.x, tile_t = blockIdx.y;
+    const int row_base = tile_m * kTileM, tok_base = tile_t * p.tile_n;
+    const int total = p.nsteps + p.lr_stages;
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
+    unsigned char* base_ptr = smem_raw + (base - raw);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_a = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto full_b = [&](int s) { return bar0 + 8u * (uint32_t)(kStages + s); };
+    auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kStages + s); };
+    const uint32_t acc_ready = bar0 + 8u * (uint32_t)(3 * kStages);
+    auto time_out = [&]() {
+        s_timeout = 1;
+        atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+    };
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_a(s), kDequantWarps);
+            mbar_init(full_b(s), 1);
+            mbar_init(empty(s), 1);
+        }
+        mbar_init(acc_ready, 1);
+        s_timeout = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 9) {  // one warp allocates the accumulator columns and later frees them
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                     "r"((uint32_t)kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+
+    if (warp < kDequantWarps) {
+        // ---------------- dequant warps: fill the A tile of every weight stage ----------------
+        const int gq = lane >> 2, tg = lane & 3;
+        const int rt = tile_m * (kTileM / 16) + warp;
+        const bool valid = rt * 16 < p.m;
+        uint32_t wbuf[kCodeRing][BITS];
+        uint32_t szbuf[kCodeRing][2];
+        const uint32_t* wbase = p.codes + ((size_t)rt * p.nsteps * 32 + lane) * BITS;
+        const uint32_t* szbase = p.sz + (size_t)rt * p.ng * 16 + gq;
+        auto issue = [&](int slot, int s) {
+#pragma unroll
+            for (int q = 0; q < BITS; ++q) wbuf[slot][q] = __ldg(wbase + (size_t)s * 32 * BITS + q);
+            const uint32_t* z = szbase + (size_t)(s >> p.gshift) * 16;
+            szbuf[slot][0] = __ldg(z);
+            szbuf[slot][1] = __ldg(z + 8);
+        };
+        if (valid) {
+#pragma unroll
+            for (int i = 0; i < kCodeRing; ++i)
+                if (i < p.nsteps) issue(i, i);
+        }
+        for (int s0 = 0; s0 < total; s0 += kCodeRing) {
+#pragma unroll
+            for (int i = 0; i < kCodeRing; ++i) {
+                const int s = s0 + i;
+                if (s < total) {
+                    const int slot = s % kStages;
+                    if (s >= kStages && !s_timeout && !mbar_wait(empty(slot), (uint32_t)((s / kStages) - 1) & 1u) && lane == 0)
+                        time_out();
+                    if (s < p.nsteps && valid) {
+                        uint32_t w[BITS];
+#pragma unroll
+                        for (int q = 0; q < BITS; ++q) w[q] = wbuf[i][q];
+                        const uint32_t sz_lo = szbuf[i][0], sz_hi = szbuf[i][1];
+                        if (s + kCodeRing < p.nsteps) issue(i, s + kCodeRing);
+                        uint32_t a[16];
+                        expand_codes<BITS>(a, w);
+                        const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
+                        const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
+                        const float sc[2] = {f_lo.x, f_hi.x};
+                        const float zs[2] = {128.0f + f_lo.y, 128.0f + f_hi.y};  // exact in fp32
+                        unsigned char* a_tile = base_ptr + slot * kStageBytes;
+#pragma unroll
+                        for (int pi = 0; pi < 16; ++pi) {
+                            const int j = pi >> 2, rho = pi & 3, hi8 = rho & 1;
+                            const float lo_f = __uint_as_float(a[pi] << 16), hi_f = __uint_as_float(a[pi] & 0xFFFF0000u);
+                            // (128 + c) - (128 + z) is exact, so s (c - z) is rounded once to fp32, once to bf16
+                            const __nv_bfloat162 wv =
+                                __floats2bfloat162_rn((lo_f - zs[hi8]) * sc[hi8], (hi_f - zs[hi8]) * sc[hi8]);
+                            const int row = warp * 16 + gq + 8 * hi8;          // row & 7 == gq
+                            const int chunk = (2 * j + (rho >> 1)) ^ gq;       // 16-byte chunk after the 128-byte swizzle
+                            *reinterpret_cast<__nv_bfloat162*>(a_tile + row * 128 + chunk * 16 + tg * 4) = wv;
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(full_a(slot));
+                }
+            }
+        }
+    } else if (warp == 8) {
+        // ---------------- loader: activation tiles, and the fp16 tiles of the low-rank stages ----------------
+        if (lane == 0) {
+            for (int s = 0; s < total; ++s) {
+                const int slot = s % kStages;
+                if (s >= kStages && !s_timeout && !mbar_wait(empty(slot), (uint32_t)((s / kStages) - 1) & 1u)) time_out();
+                const uint32_t a_tile = base + slot * kStageBytes, b_tile = a_tile + kABytes;
+                if (s < p.nsteps) {
+                    mbar_expect_tx(full_b(slot), (uint32_t)(p.tile_n * 128));
+                    tma_load_2d(b_tile, &map_x, s * kStageK, tok_base, full_b(slot));
+                } else {
+                    const int lr = s - p.nsteps;
+                    mbar_expect_tx(full_b(slot), (uint32_t)(p.tile_n * 128 + kABytes));
+                    tma_load_2d(b_tile, &map_t, lr * kStageK, tok_base, full_b(slot));
+                    tma_load_2d(a_tile, &map_a, lr * kStageK, row_base, full_b(slot));
+                }
+            }
+        }
+    } else if (warp == 9) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc_w = make_idesc(p.tile_n, 1u), idesc_lr = make_idesc(p.tile_n, 0u);
+            for (int s = 0; s < total; ++s) {
+                const int slot = s % kStages;
+                const uint32_t parity = (uint32_t)(s / kStages) & 1u;
+                if (!s_timeout && !(mbar_wait(full_a(slot), parity) && mbar_wait(full_b(slot), parity))) time_out();
+                tc_fence_after();
+                const uint32_t a_tile = base + slot * kStageBytes, b_tile = a_tile + kABytes;
+                const uint64_t da = make_desc_sw128(a_tile), db = make_desc_sw128(b_tile);
+                const bool lowrank = s >= p.nsteps;
+                const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
+                for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
+                    umma_f16(tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), lowrank ? idesc_lr : idesc_w,
+                             (s > 0 || k > 0) ? 1u : 0u);
+                umma_commit(empty(slot));  // the stage may be refilled once these MMAs have read it
+            }
+            umma_commit(acc_ready);
+        }
+    }
+
+    if (warp >= 8) {
+        // ---------------- epilogue: TMEM -> registers -> y[token][row] ----------------
+        __syncwarp();
+        if (!mbar_wait(acc_ready, 0) && lane == 0) time_out();
+        tc_fence_after();
+        const int lane_base = (warp & 3) * 32;  // a warp may read the 32 TMEM lanes of its quarter
+        const int row = row_base + lane_base + lane;
+        for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
+            uint32_t v[32];
+            const uint32_t taddr = tmem + ((uint32_t)lane_base << 16) + (uint32_t)c0;
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                : "r"(taddr)
+                : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (row < p.m) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int tok = tok_base + c0 + i;
+                    if (tok < p.T) {
+                        const size_t o = (size_t)tok * p.ldy + row;
+                        if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = __uint_as_float(v[i]);
+                        else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 9) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime so that the library does not link
+// against the driver library (it must load on machines without one).
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D row-major tensor [rows][cols] of 2-byte elements, box {64 columns, box_rows}, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool make_map(CUtensorMap* map, CUtensorMapDataType dt, const void* ptr, uint64_t cols, uint64_t rows, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kStageK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BITS>
+cudaError_t launch_prefill_bits(const PrefillParams& p, const CUtensorMap& mx, const CUtensorMap& ma, const CUtensorMap& mt,
+                                dim3 grid, cudaStream_t s) {
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(prefill_kernel<BITS>, kSmemBytes, &attr_done);
+    if (e != cudaSuccess) return e;
+    prefill_kernel<BITS><<<grid, kThreads, kSmemBytes, s>>>(p, mx, ma, mt);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool prefill_supported(const lopro_desc& d, int T) {
+    static int off = -1;
+    if (off < 0) {
+        const char* e = getenv("LOPRO_NO_TCGEN05");  // tuning / A-B comparison only
+        off = (e != nullptr && e[0] == '1') ? 1 : 0;
+    }
+    return off == 0 && T > kDecodeMaxT && encode_tiled_fn() != nullptr && (d.d_in % 64) == 0;
+}
+
+cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
+                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s) {
+    PrefillParams p;
+    p.codes = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_CODES]);
+    p.sz = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_SCALEZERO]);
+    p.status = reinterpret_cast<int*>(const_cast<uint8_t*>(ws) + W.off_status);
+    p.y = y;
+    p.ldy = ldy;
+    p.out_f32 = out_dtype == LOPRO_OUT_F32;
+    p.m = d.d_out;
+    p.n = d.d_in;
+    p.T = T;
+    p.nsteps = d.d_in / 64;
+    int gs = d.group_size / 64, gshift = 0;
+    while ((1 << gshift) < gs) ++gshift;
+    p.gshift = gshift;
+    p.ng = d.d_in / d.group_size;
+    p.r_pad = d.rank > 0 ? L.r_pad : 0;
+    p.tile_n = T <= 64 ? 64 : (T <= 128 ? 128 : 256);
+    p.lr_stages = (p.r_pad + kStageK - 1) / kStageK;
+    CUtensorMap mx, ma, mt;
+    if (!make_map(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ws + W.off_xrot, (uint64_t)d.d_in, (uint64_t)T, (uint32_t)p.tile_n))
+        return cudaErrorInvalidValue;
+    ma = mx;
+    mt = mx;
+    if (p.r_pad > 0) {
+        if (!make_map(&ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, blob + L.off[LOPRO_SEC_A], (uint64_t)p.r_pad, (uint64_t)d.d_out,
+                      (uint32_t)kTileM) ||
+            !make_map(&mt, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ws + W.off_t, (uint64_t)p.r_pad, (uint64_t)T, (uint32_t)p.tile_n))
+            return cudaErrorInvalidValue;
+    }
+    dim3 grid((d.d_out + kTileM - 1) / kTileM, (T + p.tile_n - 1) / p.tile_n);
+    if (grid.y > 65535) return cudaErrorInvalidValue;
+    switch (d.bits) {
+        case 2: return launch_prefill_bits<2>(p, mx, ma, mt, grid, s);
+        case 3: return launch_prefill_bits<3>(p, mx, ma, mt, grid, s);
+        default: return launch_prefill_bits<4>(p, mx, ma, mt, grid, s);
+    }
+}
+
+}  // namespace lopro

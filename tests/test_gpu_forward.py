@@ -2,7 +2,8 @@
 
 Gate A: bf16 output against the exact oracle, max relative error <= 2e-2.
 Gate B: fp32 output (fp32 accumulation) against the mirrored oracle, which applies the roundings the
-library declares (rotated activations to bf16, low-rank intermediate to fp16), <= 1e-3.
+library declares (rotated activations to bf16, low-rank intermediate to fp16, and for more than 32
+tokens -- the tensor-core prefill kernel -- the dequantized weights to bf16), <= 1e-3.
 The error measure is oracle.max_rel_err (element-wise, relative to max(|y|, rms of the token's row))."""
 import numpy as np
 import pytest
@@ -35,8 +36,10 @@ def _check_forward(layer, d, x_bits, rows=None, gate_a=GATE_A, gate_b=GATE_B):
     args = oracle_args(layer, d.group_size, d.identity_cols, d.block_size, rows=rows)
     x64 = o.bf16_bits_to_f64(x_bits)
     exact = o.forward_exact(x64, **args)
-    mirrored = o.forward_mirrored(x64, **args, round_w=False, round_t="f16", out="f32")
-    assert o.max_rel_err(mirrored, exact) <= 1e-2            # declared roundings cannot hide an error
+    mirrored = o.forward_mirrored(x64, **args, round_w=T > 32, round_t="f16", out="f32")
+    # declared roundings cannot hide an error (rounding the weights to bf16 alone reaches ~1 % on the
+    # max-over-entries measure, hence the wider guard for the prefill path)
+    assert o.max_rel_err(mirrored, exact) <= (2e-2 if T > 32 else 1e-2)
     got_bf = device_bf16_to_f64(y_bf)
     got_f32 = y_f32.cpu().numpy().astype(np.float64)
     if rows is not None:
