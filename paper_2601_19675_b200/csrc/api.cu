@@ -65,6 +65,8 @@ lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
     off += round_up_size((size_t)t_pad * s64_stride(d.d_in) * 4, 256);
     W->off_t = off;
     off += round_up_size((size_t)t_pad * (r_pad > 0 ? r_pad : 16) * 2, 256);
+    W->off_lrpart = off;
+    if (T > kDecodeMaxT && d.rank > 0) off += round_up_size(lowrank_mma_scratch_bytes(d, T), 256);
     W->total = off;
     return LOPRO_OK;
 }
@@ -232,9 +234,12 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
         cudaSuccess)
         return LOPRO_ERR_CUDA;
     if (desc->rank > 0) {
-        if (launch_lowrank_down(*desc, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, (__half*)(ws + W.off_t), T, s) !=
-            cudaSuccess)
-            return LOPRO_ERR_CUDA;
+        cudaError_t e = T > kDecodeMaxT
+                            ? launch_lowrank_down_mma(*desc, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx,
+                                                      (float*)(ws + W.off_lrpart), (__half*)(ws + W.off_t), T, s)
+                            : launch_lowrank_down(*desc, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx,
+                                                  (__half*)(ws + W.off_t), T, s);
+        if (e != cudaSuccess) return LOPRO_ERR_CUDA;
     }
     if (prefill_supported(*desc, T)) {
         if (launch_prefill(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;

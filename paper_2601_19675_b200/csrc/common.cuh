@@ -68,7 +68,7 @@ inline size_t round_up_size(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // activations, low-rank intermediate (fp16, general path), per-chunk partial sums of the low-rank
 // intermediate (fp32, small-batch path).
 struct WorkspaceLayout {
-    size_t off_status, off_xrot, off_s64, off_t, total;
+    size_t off_status, off_xrot, off_s64, off_t, off_lrpart, total;
     int t_pad;  // tokens padded to a multiple of 8
 };
 constexpr int kDecodeMaxT = 32;               // tokens per CTA of the streaming kernels
@@ -114,6 +114,10 @@ bool stream_supported(const lopro_desc& d, int T);
 cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
 
+// t = B x on the tensor cores for many tokens; `partial` holds lowrank_mma_scratch_bytes of fp32 K-slice sums.
+size_t lowrank_mma_scratch_bytes(const lopro_desc& d, int T);
+cudaError_t launch_lowrank_down_mma(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x, int64_t ldx,
+                                    float* partial, __half* t, int T, cudaStream_t s);
 // Prefill forward (T > 32) on tcgen05 / TMEM, after launch_rotate and launch_lowrank_down.
 bool prefill_supported(const lopro_desc& d, int T);
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,

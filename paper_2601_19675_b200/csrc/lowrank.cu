@@ -1,0 +1,171 @@
+// Low-rank down-projection t = B x for many tokens (Appendix A.3, "Y = V X"), on the tensor cores.
+//
+// x is bf16 and B is fp16; to keep the products exact each fp16 entry of B is split into two bf16
+// numbers, B = B_hi + B_lo (the 11-bit significand of fp16 fits 8 + 8 bits), and both parts are
+// multiplied with x by mma.sync with fp32 accumulation.  Grid: (128-token tiles, K slices); every
+// CTA writes the fp32 partial sums of its K slice, a second small kernel adds the slices in order
+// and rounds once to fp16.
+#include "common.cuh"
+
+namespace lopro {
+
+namespace {
+
+constexpr int kLrThreads = 256;
+constexpr int kLrTokens = 128;       // tokens per CTA (8 warps x 16)
+constexpr int kLrChunk = 64;         // K columns staged per iteration
+constexpr int kLrStride = kLrChunk + 8;  // bf16 elements per shared-memory row (+16 bytes: conflict-free ldmatrix)
+constexpr int kLrMaxRank = 128;      // rows of B per CTA
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// NJ = 8-wide column tiles of the output handled per CTA (rows of B / 8)
+template <int NJ>
+__global__ void __launch_bounds__(kLrThreads)
+lowrank_down_mma_kernel(const __half* __restrict__ B, const __nv_bfloat16* __restrict__ x, int64_t ldx,
+                        float* __restrict__ partial, int n, int r_pad, int T, int j0, int slice_cols) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);   // [128][kLrStride]
+    __nv_bfloat16* bh = xs + kLrTokens * kLrStride;                    // [NJ*8][kLrStride]
+    __nv_bfloat16* bl = bh + NJ * 8 * kLrStride;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tok0 = blockIdx.x * kLrTokens;
+    const int kb = blockIdx.y * slice_cols, ke = min(n, kb + slice_cols);
+    const int rows_b = min(NJ * 8, r_pad - j0);
+
+    float acc[NJ][4];
+#pragma unroll
+    for (int j = 0; j < NJ; ++j)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[j][i] = 0.0f;
+
+    const uint32_t xs_u = (uint32_t)__cvta_generic_to_shared(xs);
+    const uint32_t bh_u = (uint32_t)__cvta_generic_to_shared(bh), bl_u = (uint32_t)__cvta_generic_to_shared(bl);
+    // ldmatrix lane addresses: A operand (16 tokens x 16 columns), B operand (16 rows of B x 16 columns)
+    const uint32_t a_off = (uint32_t)((warp * 16 + (lane & 7) + 8 * ((lane >> 3) & 1)) * kLrStride + 8 * (lane >> 4)) * 2u;
+    const uint32_t b_off = (uint32_t)(((lane & 7) + 8 * (lane >> 4)) * kLrStride + 8 * ((lane >> 3) & 1)) * 2u;
+
+    for (int k0 = kb; k0 < ke; k0 += kLrChunk) {
+        __syncthreads();
+        // activations: 128 tokens x 64 columns, 16 bytes per thread and step
+        for (int i = tid; i < kLrTokens * 8; i += kLrThreads) {
+            const int r = i >> 3, c = i & 7;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (tok0 + r < T) v = __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tok0 + r) * ldx + k0) + c);
+            *reinterpret_cast<uint4*>(xs + r * kLrStride + c * 8) = v;
+        }
+        // rows of B: fp16 -> (hi, lo) bf16
+        for (int i = tid; i < NJ * 8 * 8; i += kLrThreads) {
+            const int r = i >> 3, c = i & 7;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (r < rows_b) v = __ldg(reinterpret_cast<const uint4*>(B + (size_t)(j0 + r) * n + k0) + c);
+            const __half2* h = reinterpret_cast<const __half2*>(&v);
+            uint4 hi, lo;
+            uint32_t* hp = reinterpret_cast<uint32_t*>(&hi);
+            uint32_t* lp = reinterpret_cast<uint32_t*>(&lo);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 f = __half22float2(h[e]);
+                const __nv_bfloat162 bhi = __floats2bfloat162_rn(f.x, f.y);
+                const float2 fh = __bfloat1622float2(bhi);
+                const __nv_bfloat162 blo = __floats2bfloat162_rn(f.x - fh.x, f.y - fh.y);  // exact remainder
+                hp[e] = *reinterpret_cast<const uint32_t*>(&bhi);
+                lp[e] = *reinterpret_cast<const uint32_t*>(&blo);
+            }
+            *reinterpret_cast<uint4*>(bh + r * kLrStride + c * 8) = hi;
+            *reinterpret_cast<uint4*>(bl + r * kLrStride + c * 8) = lo;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < kLrChunk; kk += 16) {
+            uint32_t a[4];
+            ldsm_x4(a, xs_u + a_off + kk * 2);
+#pragma unroll
+            for (int jp = 0; jp < NJ / 2; ++jp) {
+                uint32_t b[4];
+                ldsm_x4(b, bh_u + b_off + (uint32_t)(jp * 16 * kLrStride + kk) * 2u);
+                mma_bf16_16816(acc[2 * jp], a, b[0], b[1]);
+                mma_bf16_16816(acc[2 * jp + 1], a, b[2], b[3]);
+                ldsm_x4(b, bl_u + b_off + (uint32_t)(jp * 16 * kLrStride + kk) * 2u);
+                mma_bf16_16816(acc[2 * jp], a, b[0], b[1]);
+                mma_bf16_16816(acc[2 * jp + 1], a, b[2], b[3]);
+            }
+        }
+    }
+    // partial[slice][token][j]
+    const int gq = lane >> 2, tg = lane & 3;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int tok = tok0 + warp * 16 + gq + 8 * (i >> 1), col = j0 + j * 8 + 2 * tg + (i & 1);
+            if (tok < T && col < r_pad) partial[((size_t)blockIdx.y * T + tok) * r_pad + col] = acc[j][i];
+        }
+}
+
+__global__ void lowrank_finish_kernel(const float* __restrict__ partial, __half* __restrict__ t, size_t count, int slices) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    float s = 0.0f;
+    for (int k = 0; k < slices; ++k) s += partial[(size_t)k * count + i];
+    t[i] = __float2half_rn(s);
+}
+
+}  // namespace
+
+int lowrank_mma_slices(const lopro_desc& d, int T) {
+    const int tiles = (T + kLrTokens - 1) / kLrTokens;
+    int slices = 1;
+    while (slices < 16 && tiles * slices < 128 && d.d_in / (slices * 2) >= 512 && (d.d_in / 64) % (slices * 2) == 0) slices *= 2;
+    return slices;
+}
+
+size_t lowrank_mma_scratch_bytes(const lopro_desc& d, int T) {
+    const int r_pad = round_up_int(d.rank, 16);
+    return (size_t)lowrank_mma_slices(d, T) * T * r_pad * 4;
+}
+
+cudaError_t launch_lowrank_down_mma(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x, int64_t ldx,
+                                    float* partial, __half* t, int T, cudaStream_t s) {
+    const int slices = lowrank_mma_slices(d, T);
+    const int slice_cols = d.d_in / slices;
+    dim3 grid((T + kLrTokens - 1) / kLrTokens, slices);
+    for (int j0 = 0; j0 < r_pad; j0 += kLrMaxRank) {
+        const int rows = r_pad - j0 < kLrMaxRank ? r_pad - j0 : kLrMaxRank;
+        cudaError_t e;
+        static unsigned long long done16 = 0, done8 = 0, done4 = 0, done2 = 0;
+        if (rows > 64) {
+            const int smem = (kLrTokens + 2 * 128) * kLrStride * 2;
+            if ((e = ensure_dynamic_smem(lowrank_down_mma_kernel<16>, smem, &done16)) != cudaSuccess) return e;
+            lowrank_down_mma_kernel<16><<<grid, kLrThreads, smem, s>>>(B, x, ldx, partial, d.d_in, r_pad, T, j0, slice_cols);
+        } else if (rows > 32) {
+            const int smem = (kLrTokens + 2 * 64) * kLrStride * 2;
+            if ((e = ensure_dynamic_smem(lowrank_down_mma_kernel<8>, smem, &done8)) != cudaSuccess) return e;
+            lowrank_down_mma_kernel<8><<<grid, kLrThreads, smem, s>>>(B, x, ldx, partial, d.d_in, r_pad, T, j0, slice_cols);
+        } else if (rows > 16) {
+            const int smem = (kLrTokens + 2 * 32) * kLrStride * 2;
+            if ((e = ensure_dynamic_smem(lowrank_down_mma_kernel<4>, smem, &done4)) != cudaSuccess) return e;
+            lowrank_down_mma_kernel<4><<<grid, kLrThreads, smem, s>>>(B, x, ldx, partial, d.d_in, r_pad, T, j0, slice_cols);
+        } else {
+            const int smem = (kLrTokens + 2 * 16) * kLrStride * 2;
+            if ((e = ensure_dynamic_smem(lowrank_down_mma_kernel<2>, smem, &done2)) != cudaSuccess) return e;
+            lowrank_down_mma_kernel<2><<<grid, kLrThreads, smem, s>>>(B, x, ldx, partial, d.d_in, r_pad, T, j0, slice_cols);
+        }
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    const size_t count = (size_t)T * r_pad;
+    lowrank_finish_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(partial, t, count, slices);
+    return cudaGetLastError();
+}
+
+}  // namespace lopro

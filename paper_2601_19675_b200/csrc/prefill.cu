@@ -3,20 +3,22 @@
 //
 // CTA tile: 128 weight rows (the M side of the MMA, one TMEM lane per row) x N tokens (N = 64, 128
 // or 256 TMEM columns, fp32) x 64 columns of K per pipeline stage.
-//   * warps 0-7 (dequant): each owns one 16-row tile of the fragment layout; per stage it reads its
+//   * warps 0-15 (dequant): two per 16-row tile of the fragment layout; per stage each reads the tile's
 //     packed codes from global memory (a register ring a few stages ahead), turns them into
 //     bf16(s (c - z)) -- fp32 arithmetic, one rounding -- and writes them into the stage's A tile in
 //     the K-major 128-byte-swizzled layout the MMA reads;
-//   * warp 8 (loader): one thread brings the stage's tile of rotated activations (B operand) with a
+//   * warp 16 (loader): one thread brings the stage's tile of rotated activations (B operand) with a
 //     tiled TMA copy, and for the low-rank stages the tiles of A (fp16) and t (fp16);
-//   * warp 9 (MMA): one thread issues four tcgen05.mma (K = 16 each) per stage into the TMEM
+//   * warp 17 (MMA): one thread issues four tcgen05.mma (K = 16 each) per stage into the TMEM
 //     accumulator and commits the stage back to the producers; the rank-r term A t runs as extra K
 //     stages with fp16 operands into the same accumulator, so the sum of Eq. 8 costs no extra pass;
-//   * warps 8-11 (epilogue): tcgen05.ld the accumulator, round once, store y[token][row].
+//   * warps 16-19 (epilogue): tcgen05.ld the accumulator, round once, store y[token][row].
 // All mbarrier waits are bounded; a wait that runs out sets LOPRO_ERR_TIMEOUT in the workspace status
 // word, the CTA stops waiting, still frees its TMEM and returns (outputs then unspecified).
 #include <cuda.h>
 #include <stdlib.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -24,17 +26,16 @@ namespace lopro {
 
 namespace {
 
-constexpr int kDequantWarps = 8;
-constexpr int kThreads = 12 * 32;
+constexpr int kDequantWarps = 16;  // two warps per 16-row tile, eight register pairs (32 columns) each
+constexpr int kThreads = (kDequantWarps + 4) * 32;
 constexpr int kTileM = 128;      // weight rows per CTA
 constexpr int kMaxTileN = 256;   // tokens per CTA
 constexpr int kStageK = 64;      // K columns per stage = 128 bytes of bf16 = one swizzle atom
-constexpr int kStages = 4;
-constexpr int kABytes = kTileM * 128;       // 16 KB
-constexpr int kBBytes = kMaxTileN * 128;    // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024;  // + slack for 1024-byte alignment
-constexpr int kTmemCols = 256;
+constexpr int kAStages = 4;      // ring of weight tiles (16 KB each)
+constexpr int kBStages = 2;      // ring of activation tiles (one or two accumulators' worth, 64 KB each)
+constexpr int kABytes = kTileM * 128;           // 16 KB
+constexpr int kBBytes = 2 * kMaxTileN * 128;    // 64 KB: two 256-token tiles
+constexpr int kSmemBytes = kAStages * kABytes + kBStages * kBBytes + 1024;  // + slack for 1024-byte alignment
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr int kCodeRing = 4;  // stages of packed codes held in registers ahead of use
 
@@ -47,7 +48,8 @@ struct PrefillParams {
     int out_f32;
     int m, n, T;
     int nsteps, gshift, ng, r_pad;
-    int tile_n;      // 64, 128 or 256
+    int tile_n;      // tokens per accumulator: 64, 128 or 256
+    int n_acc;       // accumulators per CTA (1 or 2): the CTA covers tile_n * n_acc tokens
     int lr_stages;   // ceil(r_pad / 64)
 };
 
@@ -133,40 +135,52 @@ __global__ void __launch_bounds__(kThreads, 1)
 prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a,
                const __grid_constant__ CUtensorMap map_t) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t bars[3 * kStages + 1];  // full_a, full_b, empty per stage; accumulator ready
+    // full_a, empty_a per A slot; full_b, empty_b per B slot; accumulator ready
+    __shared__ __align__(8) uint64_t bars[2 * kAStages + 2 * kBStages + 1];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_timeout;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile_m = blockIdx.x, tile_t = blockIdx.y;
-    const int row_base = tile_m * kTileM, tok_base = tile_t * p.tile_n;
+    const int row_base = tile_m * kTileM, tok_base = tile_t * p.tile_n * p.n_acc;
     const int total = p.nsteps + p.lr_stages;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
     unsigned char* base_ptr = smem_raw + (base - raw);
+    const uint32_t b_ring = base + kAStages * kABytes;  // B slots follow the A slots
     const uint32_t bar0 = smem_u32(bars);
     auto full_a = [&](int s) { return bar0 + 8u * (uint32_t)s; };
-    auto full_b = [&](int s) { return bar0 + 8u * (uint32_t)(kStages + s); };
-    auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kStages + s); };
-    const uint32_t acc_ready = bar0 + 8u * (uint32_t)(3 * kStages);
+    auto empty_a = [&](int s) { return bar0 + 8u * (uint32_t)(kAStages + s); };
+    auto full_b = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kAStages + s); };
+    auto empty_b = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kAStages + kBStages + s); };
+    const uint32_t acc_ready = bar0 + 8u * (uint32_t)(2 * kAStages + 2 * kBStages);
     auto time_out = [&]() {
         s_timeout = 1;
         atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
     };
+    // one lane polls, the warp follows (bar.warp.sync orders the other lanes' accesses after the wait)
+    auto warp_wait = [&](uint32_t bar, uint32_t parity) {
+        if (lane == 0 && !s_timeout && !mbar_wait(bar, parity)) time_out();
+        __syncwarp();
+    };
+    const uint32_t tmem_cols = p.n_acc == 2 ? 512u : 256u;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_a(s), kDequantWarps);
+        for (int s = 0; s < kAStages; ++s) {
+            mbar_init(full_a(s), kDequantWarps + 1);  // every dequant warp and the loader
+            mbar_init(empty_a(s), 1);
+        }
+        for (int s = 0; s < kBStages; ++s) {
             mbar_init(full_b(s), 1);
-            mbar_init(empty(s), 1);
+            mbar_init(empty_b(s), 1);
         }
         mbar_init(acc_ready, 1);
         s_timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 9) {  // one warp allocates the accumulator columns and later frees them
+    if (warp == kDequantWarps + 1) {  // one warp allocates the accumulator columns and later frees them
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                     "r"((uint32_t)kTmemCols)
+                     "r"(tmem_cols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -178,7 +192,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     if (warp < kDequantWarps) {
         // ---------------- dequant warps: fill the A tile of every weight stage ----------------
         const int gq = lane >> 2, tg = lane & 3;
-        const int rt = tile_m * (kTileM / 16) + warp;
+        const int rt = tile_m * (kTileM / 16) + (warp & 7);
         const bool valid = rt * 16 < p.m;
         uint32_t wbuf[kCodeRing][BITS];
         uint32_t szbuf[kCodeRing][2];
@@ -196,38 +210,48 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
             for (int i = 0; i < kCodeRing; ++i)
                 if (i < p.nsteps) issue(i, i);
         }
+        // byte offset of this lane's 4-byte slot in 16-byte chunk c of its row (row & 7 == gq, 128-byte swizzle)
+        uint32_t off[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) off[c] = (uint32_t)(((warp & 7) * 16 + gq) * 128 + ((c ^ gq) << 4) + tg * 4);
+        // the warp converts eight of the tile's sixteen register pairs: HALF = 0 -> columns 0..31, 1 -> 32..63
+        auto convert = [&](auto half_tag, const uint32_t (&w)[BITS], uint32_t sz_lo, uint32_t sz_hi, unsigned char* a_tile) {
+            constexpr int HALF = decltype(half_tag)::value;
+            uint32_t a[16];
+            expand_codes<BITS>(a, w);  // pairs of the other half are dead code after unrolling
+            const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
+            const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
+            const float sc[2] = {f_lo.x, f_hi.x};
+            const float zs[2] = {128.0f + f_lo.y, 128.0f + f_hi.y};  // exact in fp32
+#pragma unroll
+            for (int pp = 0; pp < 8; ++pp) {
+                constexpr int kBase = HALF * 8;
+                const int pi = kBase + pp;
+                const int j = pi >> 2, rho = pi & 3, hi8 = rho & 1;
+                const uint32_t av = a[pi];
+                const float lo_f = __uint_as_float(av << 16), hi_f = __uint_as_float(av & 0xFFFF0000u);
+                // (128 + c) - (128 + z) is exact, so s (c - z) is rounded once to fp32, once to bf16
+                const __nv_bfloat162 wv = __floats2bfloat162_rn((lo_f - zs[hi8]) * sc[hi8], (hi_f - zs[hi8]) * sc[hi8]);
+                *reinterpret_cast<__nv_bfloat162*>(a_tile + off[2 * j + (rho >> 1)] + hi8 * 1024) = wv;
+            }
+        };
+        const bool upper = (warp >> 3) != 0;
         for (int s0 = 0; s0 < total; s0 += kCodeRing) {
 #pragma unroll
             for (int i = 0; i < kCodeRing; ++i) {
                 const int s = s0 + i;
                 if (s < total) {
-                    const int slot = s % kStages;
-                    if (s >= kStages && !s_timeout && !mbar_wait(empty(slot), (uint32_t)((s / kStages) - 1) & 1u) && lane == 0)
-                        time_out();
+                    const int slot = s % kAStages;
+                    if (s >= kAStages) warp_wait(empty_a(slot), (uint32_t)((s / kAStages) - 1) & 1u);
                     if (s < p.nsteps && valid) {
                         uint32_t w[BITS];
 #pragma unroll
                         for (int q = 0; q < BITS; ++q) w[q] = wbuf[i][q];
                         const uint32_t sz_lo = szbuf[i][0], sz_hi = szbuf[i][1];
                         if (s + kCodeRing < p.nsteps) issue(i, s + kCodeRing);
-                        uint32_t a[16];
-                        expand_codes<BITS>(a, w);
-                        const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
-                        const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
-                        const float sc[2] = {f_lo.x, f_hi.x};
-                        const float zs[2] = {128.0f + f_lo.y, 128.0f + f_hi.y};  // exact in fp32
-                        unsigned char* a_tile = base_ptr + slot * kStageBytes;
-#pragma unroll
-                        for (int pi = 0; pi < 16; ++pi) {
-                            const int j = pi >> 2, rho = pi & 3, hi8 = rho & 1;
-                            const float lo_f = __uint_as_float(a[pi] << 16), hi_f = __uint_as_float(a[pi] & 0xFFFF0000u);
-                            // (128 + c) - (128 + z) is exact, so s (c - z) is rounded once to fp32, once to bf16
-                            const __nv_bfloat162 wv =
-                                __floats2bfloat162_rn((lo_f - zs[hi8]) * sc[hi8], (hi_f - zs[hi8]) * sc[hi8]);
-                            const int row = warp * 16 + gq + 8 * hi8;          // row & 7 == gq
-                            const int chunk = (2 * j + (rho >> 1)) ^ gq;       // 16-byte chunk after the 128-byte swizzle
-                            *reinterpret_cast<__nv_bfloat162*>(a_tile + row * 128 + chunk * 16 + tg * 4) = wv;
-                        }
+                        unsigned char* a_tile = base_ptr + slot * kABytes;
+                        if (upper) convert(std::integral_constant<int, 1>{}, w, sz_lo, sz_hi, a_tile);
+                        else convert(std::integral_constant<int, 0>{}, w, sz_lo, sz_hi, a_tile);
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
                     }
                     __syncwarp();
@@ -235,74 +259,87 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                 }
             }
         }
-    } else if (warp == 8) {
+    } else if (warp == kDequantWarps) {
         // ---------------- loader: activation tiles, and the fp16 tiles of the low-rank stages ----------------
         if (lane == 0) {
+            const uint32_t b_bytes = (uint32_t)(p.n_acc * p.tile_n * 128);
             for (int s = 0; s < total; ++s) {
-                const int slot = s % kStages;
-                if (s >= kStages && !s_timeout && !mbar_wait(empty(slot), (uint32_t)((s / kStages) - 1) & 1u)) time_out();
-                const uint32_t a_tile = base + slot * kStageBytes, b_tile = a_tile + kABytes;
+                const int sa = s % kAStages, sb = s % kBStages;
+                if (s >= kAStages && !s_timeout && !mbar_wait(empty_a(sa), (uint32_t)((s / kAStages) - 1) & 1u)) time_out();
+                if (s >= kBStages && !s_timeout && !mbar_wait(empty_b(sb), (uint32_t)((s / kBStages) - 1) & 1u)) time_out();
+                const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
+                mbar_expect_tx(full_b(sb), b_bytes);
                 if (s < p.nsteps) {
-                    mbar_expect_tx(full_b(slot), (uint32_t)(p.tile_n * 128));
-                    tma_load_2d(b_tile, &map_x, s * kStageK, tok_base, full_b(slot));
+                    for (int acc = 0; acc < p.n_acc; ++acc)
+                        tma_load_2d(b_tile + acc * (kBBytes / 2), &map_x, s * kStageK, tok_base + acc * p.tile_n, full_b(sb));
+                    mbar_arrive(full_a(sa));
                 } else {
                     const int lr = s - p.nsteps;
-                    mbar_expect_tx(full_b(slot), (uint32_t)(p.tile_n * 128 + kABytes));
-                    tma_load_2d(b_tile, &map_t, lr * kStageK, tok_base, full_b(slot));
-                    tma_load_2d(a_tile, &map_a, lr * kStageK, row_base, full_b(slot));
+                    for (int acc = 0; acc < p.n_acc; ++acc)
+                        tma_load_2d(b_tile + acc * (kBBytes / 2), &map_t, lr * kStageK, tok_base + acc * p.tile_n, full_b(sb));
+                    mbar_expect_tx(full_a(sa), (uint32_t)kABytes);
+                    tma_load_2d(a_tile, &map_a, lr * kStageK, row_base, full_a(sa));
                 }
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == kDequantWarps + 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             const uint32_t idesc_w = make_idesc(p.tile_n, 1u), idesc_lr = make_idesc(p.tile_n, 0u);
             for (int s = 0; s < total; ++s) {
-                const int slot = s % kStages;
-                const uint32_t parity = (uint32_t)(s / kStages) & 1u;
-                if (!s_timeout && !(mbar_wait(full_a(slot), parity) && mbar_wait(full_b(slot), parity))) time_out();
+                const int sa = s % kAStages, sb = s % kBStages;
+                if (!s_timeout && !(mbar_wait(full_a(sa), (uint32_t)(s / kAStages) & 1u) &&
+                                    mbar_wait(full_b(sb), (uint32_t)(s / kBStages) & 1u)))
+                    time_out();
                 tc_fence_after();
-                const uint32_t a_tile = base + slot * kStageBytes, b_tile = a_tile + kABytes;
-                const uint64_t da = make_desc_sw128(a_tile), db = make_desc_sw128(b_tile);
+                const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
+                const uint64_t da = make_desc_sw128(a_tile);
                 const bool lowrank = s >= p.nsteps;
                 const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
-                for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
-                    umma_f16(tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), lowrank ? idesc_lr : idesc_w,
-                             (s > 0 || k > 0) ? 1u : 0u);
-                umma_commit(empty(slot));  // the stage may be refilled once these MMAs have read it
+                for (int acc = 0; acc < p.n_acc; ++acc) {
+                    const uint64_t db = make_desc_sw128(b_tile + acc * (kBBytes / 2));
+                    for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
+                        umma_f16(tmem + (uint32_t)(acc * 256), da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
+                                 lowrank ? idesc_lr : idesc_w, (s > 0 || k > 0) ? 1u : 0u);
+                }
+                umma_commit(empty_a(sa));  // the slots may be refilled once these MMAs have read them
+                umma_commit(empty_b(sb));
             }
             umma_commit(acc_ready);
         }
     }
 
-    if (warp >= 8) {
+    if (warp >= kDequantWarps) {
         // ---------------- epilogue: TMEM -> registers -> y[token][row] ----------------
         __syncwarp();
-        if (!mbar_wait(acc_ready, 0) && lane == 0) time_out();
+        if (lane == 0 && !mbar_wait(acc_ready, 0)) time_out();
+        __syncwarp();
         tc_fence_after();
         const int lane_base = (warp & 3) * 32;  // a warp may read the 32 TMEM lanes of its quarter
         const int row = row_base + lane_base + lane;
-        for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
-            uint32_t v[32];
-            const uint32_t taddr = tmem + ((uint32_t)lane_base << 16) + (uint32_t)c0;
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                : "r"(taddr)
-                : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (row < p.m) {
+        for (int acc = 0; acc < p.n_acc; ++acc) {
+            for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
+                uint32_t v[32];
+                const uint32_t taddr = tmem + ((uint32_t)lane_base << 16) + (uint32_t)(acc * 256 + c0);
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                      "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                      "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                      "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                    : "r"(taddr)
+                    : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (row < p.m) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int tok = tok_base + c0 + i;
-                    if (tok < p.T) {
-                        const size_t o = (size_t)tok * p.ldy + row;
-                        if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = __uint_as_float(v[i]);
-                        else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                    for (int i = 0; i < 32; ++i) {
+                        const int tok = tok_base + acc * p.tile_n + c0 + i;
+                        if (tok < p.T) {
+                            const size_t o = (size_t)tok * p.ldy + row;
+                            if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = __uint_as_float(v[i]);
+                            else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                        }
                     }
                 }
             }
@@ -310,9 +347,9 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) {
+    if (warp == kDequantWarps + 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
     }
 }
 
@@ -387,6 +424,7 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     p.ng = d.d_in / d.group_size;
     p.r_pad = d.rank > 0 ? L.r_pad : 0;
     p.tile_n = T <= 64 ? 64 : (T <= 128 ? 128 : 256);
+    p.n_acc = T > 256 ? 2 : 1;
     p.lr_stages = (p.r_pad + kStageK - 1) / kStageK;
     CUtensorMap mx, ma, mt;
     if (!make_map(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ws + W.off_xrot, (uint64_t)d.d_in, (uint64_t)T, (uint32_t)p.tile_n))
@@ -399,7 +437,8 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
             !make_map(&mt, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ws + W.off_t, (uint64_t)p.r_pad, (uint64_t)T, (uint32_t)p.tile_n))
             return cudaErrorInvalidValue;
     }
-    dim3 grid((d.d_out + kTileM - 1) / kTileM, (T + p.tile_n - 1) / p.tile_n);
+    const int cta_tokens = p.tile_n * p.n_acc;
+    dim3 grid((d.d_out + kTileM - 1) / kTileM, (T + cta_tokens - 1) / cta_tokens);
     if (grid.y > 65535) return cudaErrorInvalidValue;
     switch (d.bits) {
         case 2: return launch_prefill_bits<2>(p, mx, ma, mt, grid, s);
