@@ -143,12 +143,12 @@ lowrank_down_kernel(const __half* __restrict__ B, const __nv_bfloat16* __restric
 }
 
 // Prologue of the small-batch forward (T <= 32, b_H <= 256, b_I a multiple of b_H).  Grid:
-// x = column chunks of 256, then pairs of rows of B; y = groups of 8 tokens.
+// x = column chunks of 256, then the rows of B; y = groups of 8 tokens.
 //  * a chunk CTA rotates 256 output columns, warp w for token w: the 8 entries of a lane are
 //    gathered from global memory through perm, transformed with register and shuffle butterflies,
 //    rounded to bf16 and stored together with their 64-column sums in the activation image that the
 //    streaming kernel copies to shared memory;
-//  * a row-pair CTA computes t[token][j] = sum_k B[j][k] x[token][k] for two rows j and the 8 tokens
+//  * a row CTA computes t[token][j] = sum_k B[j][k] x[token][k] for one row j of B and the 8 tokens
 //    (fp32 accumulation over all of K, one rounding to fp16): the low-rank intermediate "Y = V X".
 // Launched with programmatic stream serialization: perm and B (layer data) are read before the
 // wait, the activations after it.
@@ -162,87 +162,75 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if ((int)blockIdx.x >= nchunks) {
-        // ---- two rows of B against eight tokens ----
-        __shared__ float part[8][16];
-        const int j0 = 2 * ((int)blockIdx.x - nchunks);
-        const __half* b0 = B + (size_t)j0 * n;
-        const __half* b1 = b0 + n;
+        // ---- one row of B against eight tokens ----
+        __shared__ float part[8][8];
+        const int j = (int)blockIdx.x - nchunks;
+        const __half* brow = B + (size_t)j * n;
         const int npass = (n + 2047) >> 11;
-        uint4 pre[2][2];
+        uint4 pre[2];
 #pragma unroll
         for (int ps = 0; ps < 2; ++ps) {
             const int k = ps * 2048 + tid * 8;
-            pre[ps][0] = pre[ps][1] = make_uint4(0, 0, 0, 0);
-            if (k < n) {
-                pre[ps][0] = __ldg(reinterpret_cast<const uint4*>(b0 + k));
-                pre[ps][1] = __ldg(reinterpret_cast<const uint4*>(b1 + k));
-            }
+            pre[ps] = k < n ? __ldg(reinterpret_cast<const uint4*>(brow + k)) : make_uint4(0, 0, 0, 0);
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        float acc[2][8];
+        float acc[8];
 #pragma unroll
-        for (int r = 0; r < 2; ++r)
-#pragma unroll
-            for (int tk = 0; tk < 8; ++tk) acc[r][tk] = 0.0f;
-        for (int ps = 0; ps < npass; ++ps) {
-            const int k = ps * 2048 + tid * 8;
-            if (k >= n) break;
-            uint4 bw[2];
-            if (ps == 0) {
-                bw[0] = pre[0][0];
-                bw[1] = pre[0][1];
-            } else if (ps == 1) {
-                bw[0] = pre[1][0];
-                bw[1] = pre[1][1];
-            } else {
-                bw[0] = __ldg(reinterpret_cast<const uint4*>(b0 + k));
-                bw[1] = __ldg(reinterpret_cast<const uint4*>(b1 + k));
-            }
-            float bf[2][8];
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const __half2* h = reinterpret_cast<const __half2*>(&bw[r]);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float2 f = __half22float2(h[i]);
-                    bf[r][2 * i] = f.x;
-                    bf[r][2 * i + 1] = f.y;
-                }
-            }
-            uint4 xw[8];
+        for (int tk = 0; tk < 8; ++tk) acc[tk] = 0.0f;
+        auto load_x = [&](uint4 (&xw)[8], int k) {
 #pragma unroll
             for (int tk = 0; tk < 8; ++tk)
-                xw[tk] = tok0 + tk < T ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tok0 + tk) * ldx + k))
-                                       : make_uint4(0, 0, 0, 0);
+                xw[tk] = (k < n && tok0 + tk < T) ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tok0 + tk) * ldx + k))
+                                                  : make_uint4(0, 0, 0, 0);
+        };
+        auto accumulate = [&](const uint4& bw, const uint4 (&xw)[8]) {
+            float bf[8];
+            const __half2* h = reinterpret_cast<const __half2*>(&bw);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(h[i]);
+                bf[2 * i] = f.x;
+                bf[2 * i + 1] = f.y;
+            }
 #pragma unroll
             for (int tk = 0; tk < 8; ++tk) {
                 const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xw[tk]);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const float2 f = __bfloat1622float2(xh[i]);
-                    acc[0][tk] = fmaf(bf[0][2 * i], f.x, acc[0][tk]);
-                    acc[0][tk] = fmaf(bf[0][2 * i + 1], f.y, acc[0][tk]);
-                    acc[1][tk] = fmaf(bf[1][2 * i], f.x, acc[1][tk]);
-                    acc[1][tk] = fmaf(bf[1][2 * i + 1], f.y, acc[1][tk]);
+                    acc[tk] = fmaf(bf[2 * i], f.x, acc[tk]);
+                    acc[tk] = fmaf(bf[2 * i + 1], f.y, acc[tk]);
                 }
             }
+        };
+        {   // the first two passes (all of K up to 4096 columns): every load is in flight before the first use,
+            // so the dependent chain after the wait is one memory round trip
+            uint4 x0[8], x1[8];
+            load_x(x0, tid * 8);
+            load_x(x1, 2048 + tid * 8);
+            accumulate(pre[0], x0);
+            accumulate(pre[1], x1);
+        }
+        for (int ps = 2; ps < npass; ++ps) {
+            const int k = ps * 2048 + tid * 8;
+            if (k >= n) break;
+            uint4 xw[8];
+            load_x(xw, k);
+            accumulate(__ldg(reinterpret_cast<const uint4*>(brow + k)), xw);
         }
 #pragma unroll
-        for (int r = 0; r < 2; ++r)
+        for (int tk = 0; tk < 8; ++tk) {
+            float v = acc[tk];
 #pragma unroll
-            for (int tk = 0; tk < 8; ++tk) {
-                float v = acc[r][tk];
-#pragma unroll
-                for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-                if (lane == 0) part[warp][r * 8 + tk] = v;
-            }
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+            if (lane == 0) part[warp][tk] = v;
+        }
         __syncthreads();
-        if (tid < 16) {
+        if (tid < 8) {
             float v = 0.0f;
 #pragma unroll
             for (int w = 0; w < 8; ++w) v += part[w][tid];
-            const int r = tid >> 3, tk = tid & 7;
-            if (tok0 + tk < T && j0 + r < r_pad) t[(size_t)(tok0 + tk) * r_pad + j0 + r] = __float2half_rn(v);
+            if (tok0 + tid < T) t[(size_t)(tok0 + tid) * r_pad + j] = __float2half_rn(v);
         }
         return;
     }
@@ -345,7 +333,7 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
                             int* status, int T, cudaStream_t s) {
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((d.d_in + 255) / 256 + (d.rank > 0 ? r_pad / 2 : 0), (T + 7) / 8);
+    cfg.gridDim = dim3((d.d_in + 255) / 256 + (d.rank > 0 ? r_pad : 0), (T + 7) / 8);
     cfg.blockDim = dim3(256);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = s;
