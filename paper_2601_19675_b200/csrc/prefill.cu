@@ -49,7 +49,7 @@ struct PrefillParams {
     int m, n, T;
     int nsteps, gshift, ng, r_pad;
     int tile_n;      // tokens per accumulator: 64, 128 or 256
-    int n_acc;       // accumulators per CTA (1 or 2): the CTA covers tile_n * n_acc tokens
+    int pair_tiles;  // CTAs along y that own two accumulators (2 * tile_n tokens); the others own one
     int lr_stages;   // ceil(r_pad / 64)
 };
 
@@ -142,7 +142,10 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile_m = blockIdx.x, tile_t = blockIdx.y;
-    const int row_base = tile_m * kTileM, tok_base = tile_t * p.tile_n * p.n_acc;
+    // token tiles: the first p.pair_tiles CTAs along y own two accumulators (2 * tile_n tokens), the rest one
+    const int n_acc = tile_t < p.pair_tiles ? 2 : 1;
+    const int row_base = tile_m * kTileM;
+    const int tok_base = tile_t < p.pair_tiles ? tile_t * 2 * p.tile_n : (p.pair_tiles + tile_t) * p.tile_n;
     const int total = p.nsteps + p.lr_stages;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
@@ -163,7 +166,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
         if (lane == 0 && !s_timeout && !mbar_wait(bar, parity)) time_out();
         __syncwarp();
     };
-    const uint32_t tmem_cols = p.n_acc == 2 ? 512u : 256u;
+    const uint32_t tmem_cols = n_acc == 2 ? 512u : 256u;
 
     if (tid == 0) {
         for (int s = 0; s < kAStages; ++s) {
@@ -262,7 +265,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     } else if (warp == kDequantWarps) {
         // ---------------- loader: activation tiles, and the fp16 tiles of the low-rank stages ----------------
         if (lane == 0) {
-            const uint32_t b_bytes = (uint32_t)(p.n_acc * p.tile_n * 128);
+            const uint32_t b_bytes = (uint32_t)(n_acc * p.tile_n * 128);
             for (int s = 0; s < total; ++s) {
                 const int sa = s % kAStages, sb = s % kBStages;
                 if (s >= kAStages && !s_timeout && !mbar_wait(empty_a(sa), (uint32_t)((s / kAStages) - 1) & 1u)) time_out();
@@ -270,12 +273,12 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                 const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
                 mbar_expect_tx(full_b(sb), b_bytes);
                 if (s < p.nsteps) {
-                    for (int acc = 0; acc < p.n_acc; ++acc)
+                    for (int acc = 0; acc < n_acc; ++acc)
                         tma_load_2d(b_tile + acc * (kBBytes / 2), &map_x, s * kStageK, tok_base + acc * p.tile_n, full_b(sb));
                     mbar_arrive(full_a(sa));
                 } else {
                     const int lr = s - p.nsteps;
-                    for (int acc = 0; acc < p.n_acc; ++acc)
+                    for (int acc = 0; acc < n_acc; ++acc)
                         tma_load_2d(b_tile + acc * (kBBytes / 2), &map_t, lr * kStageK, tok_base + acc * p.tile_n, full_b(sb));
                     mbar_expect_tx(full_a(sa), (uint32_t)kABytes);
                     tma_load_2d(a_tile, &map_a, lr * kStageK, row_base, full_a(sa));
@@ -296,7 +299,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                 const uint64_t da = make_desc_sw128(a_tile);
                 const bool lowrank = s >= p.nsteps;
                 const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
-                for (int acc = 0; acc < p.n_acc; ++acc) {
+                for (int acc = 0; acc < n_acc; ++acc) {
                     const uint64_t db = make_desc_sw128(b_tile + acc * (kBBytes / 2));
                     for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
                         umma_f16(tmem + (uint32_t)(acc * 256), da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
@@ -317,7 +320,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
         tc_fence_after();
         const int lane_base = (warp & 3) * 32;  // a warp may read the 32 TMEM lanes of its quarter
         const int row = row_base + lane_base + lane;
-        for (int acc = 0; acc < p.n_acc; ++acc) {
+        for (int acc = 0; acc < n_acc; ++acc) {
             for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
                 uint32_t v[32];
                 const uint32_t taddr = tmem + ((uint32_t)lane_base << 16) + (uint32_t)(acc * 256 + c0);
@@ -424,7 +427,6 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     p.ng = d.d_in / d.group_size;
     p.r_pad = d.rank > 0 ? L.r_pad : 0;
     p.tile_n = T <= 64 ? 64 : (T <= 128 ? 128 : 256);
-    p.n_acc = T > 256 ? 2 : 1;
     p.lr_stages = (p.r_pad + kStageK - 1) / kStageK;
     CUtensorMap mx, ma, mt;
     if (!make_map(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ws + W.off_xrot, (uint64_t)d.d_in, (uint64_t)T, (uint32_t)p.tile_n))
@@ -437,8 +439,48 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
             !make_map(&mt, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ws + W.off_t, (uint64_t)p.r_pad, (uint64_t)T, (uint32_t)p.tile_n))
             return cudaErrorInvalidValue;
     }
-    const int cta_tokens = p.tile_n * p.n_acc;
-    dim3 grid((d.d_out + kTileM - 1) / kTileM, (T + cta_tokens - 1) / cta_tokens);
+    // Token tiling: U units of tile_n tokens per row tile.  A CTA with two accumulators dequantizes its
+    // weights once for two units (cost ~1.5 per stage against 1.0 for a single unit) but coarser tiles
+    // waste more of the last wave; pick the number of pair tiles that minimises the makespan of a greedy
+    // schedule over the 148 SMs (pairs are dispatched first, then singles).
+    const int units = (T + p.tile_n - 1) / p.tile_n;
+    const int m_tiles = (d.d_out + kTileM - 1) / kTileM;
+    int best_pairs = units / 2;
+    if ((long long)m_tiles * units <= 20000) {
+        // list scheduling of the tiles (pairs first, dispatch order = block order) on 148 SMs
+        double best_cost = 1e30;
+        for (int pairs = units / 2; pairs >= 0; --pairs) {
+            const int singles = units - 2 * pairs;
+            double finish[148];
+            for (int i = 0; i < 148; ++i) finish[i] = 0.0;
+            auto place = [&](long long count, double dur) {
+                for (long long c = 0; c < count; ++c) {
+                    int best = 0;
+                    for (int i = 1; i < 148; ++i)
+                        if (finish[i] < finish[best]) best = i;
+                    finish[best] += dur;
+                }
+            };
+            place((long long)m_tiles * pairs, 1.5);
+            place((long long)m_tiles * singles, 1.0);
+            double cost = 0.0;
+            for (int i = 0; i < 148; ++i) cost = finish[i] > cost ? finish[i] : cost;
+            if (cost < best_cost - 1e-9) {
+                best_cost = cost;
+                best_pairs = pairs;
+            }
+        }
+    }
+    {
+        static int forced = -2;  // LOPRO_PREFILL_PAIRS overrides the choice (tuning only)
+        if (forced == -2) {
+            const char* e = getenv("LOPRO_PREFILL_PAIRS");
+            forced = e ? atoi(e) : -1;
+        }
+        if (forced >= 0 && forced <= units / 2) best_pairs = forced;
+    }
+    p.pair_tiles = best_pairs;
+    dim3 grid(m_tiles, best_pairs + (units - 2 * best_pairs));
     if (grid.y > 65535) return cudaErrorInvalidValue;
     switch (d.bits) {
         case 2: return launch_prefill_bits<2>(p, mx, ma, mt, grid, s);

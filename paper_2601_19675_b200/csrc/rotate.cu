@@ -11,87 +11,100 @@ namespace {
 
 constexpr int kRotThreads = 256;
 
-// One CTA per token row.  The row is staged in shared memory with coalesced 16-byte loads, the
-// gather through `perm` reads shared memory (a 2-byte gather from global memory would use 1/16 of
-// every sector), each warp transforms runs of 32*E consecutive rotated columns: lane l holds E
-// consecutive entries, the first log2(E) butterfly stages stay in registers, the next five go
-// through warp shuffles.  Results are rounded to bf16 once, collected in shared memory and stored
-// with coalesced 16-byte stores.  E = 8 covers b_H <= 256, E = 16 and 32 cover 512 and 1024.
-template <int E>
+// One CTA per TOK token rows.  The rows are staged in shared memory with coalesced 16-byte loads,
+// the gather through `perm` reads shared memory (a 2-byte gather from global memory would use 1/16
+// of every sector; with TOK > 1 each index of perm is fetched once for all rows), each warp transforms
+// runs of 32*E consecutive rotated columns: lane l holds E consecutive entries, the first log2(E)
+// butterfly stages stay in registers, the next five go through warp shuffles.  Results are rounded to
+// bf16 once, collected in shared memory and stored with coalesced 16-byte stores.  E = 8 covers
+// b_H <= 256, E = 16 and 32 cover 512 and 1024.
+template <int E, int TOK>
 __global__ void __launch_bounds__(kRotThreads)
 rotate_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
               __nv_bfloat16* __restrict__ xrot, int64_t ldo, float* __restrict__ s64, int s64_ld,
-              int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh) {
+              int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int T) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __nv_bfloat16* xin = reinterpret_cast<__nv_bfloat16*>(smem_raw);
-    __nv_bfloat16* xout = xin + n;
-    const int t = blockIdx.x;
+    __nv_bfloat16* xin = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [TOK][n]
+    __nv_bfloat16* xout = xin + (size_t)TOK * n;                       // [TOK][n]
+    const int t0 = blockIdx.x * TOK;
+    const int nt = min(TOK, T - t0);  // live rows of this CTA
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kRotThreads / 32;
     constexpr int kRun = 32 * E;
-    if (status != nullptr && t == 0 && tid == 0) *status = LOPRO_OK;
+    if (status != nullptr && blockIdx.x == 0 && tid == 0) *status = LOPRO_OK;
 
-    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * ldx);
-    for (int i = tid; i < n / 8; i += kRotThreads) reinterpret_cast<uint4*>(xin)[i] = __ldg(src + i);
+    for (int r = 0; r < nt; ++r) {
+        const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)(t0 + r) * ldx);
+        for (int i = tid; i < n / 8; i += kRotThreads) reinterpret_cast<uint4*>(xin + (size_t)r * n)[i] = __ldg(src + i);
+    }
     __syncthreads();
 
     // identity prefix: permuted only
-    for (int k = tid; k < b_i; k += kRotThreads) xout[k] = xin[__ldg(perm + k)];
+    for (int k = tid; k < b_i; k += kRotThreads) {
+        const int pk = __ldg(perm + k);
+#pragma unroll
+        for (int r = 0; r < TOK; ++r)
+            if (r < nt) xout[(size_t)r * n + k] = xin[(size_t)r * n + pk];
+    }
 
     const int nrot = n - b_i;
     const int nruns = (nrot + kRun - 1) / kRun;
     for (int run = warp; run < nruns; run += kWarps) {
         const int rel = run * kRun + lane * E;  // offset inside the rotated region
-        float v[E];
+        int pidx[E];
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            const int idx = rel + e;
-            v[e] = idx < nrot ? __bfloat162float(xin[__ldg(perm + b_i + idx)]) : 0.0f;
-        }
-        // stages inside the lane: distance h = 1, 2, ..., E/2
+        for (int e = 0; e < E; ++e) pidx[e] = rel + e < nrot ? __ldg(perm + b_i + rel + e) : 0;
+        for (int r = 0; r < nt; ++r) {
+            const __nv_bfloat16* row = xin + (size_t)r * n;
+            float v[E];
 #pragma unroll
-        for (int h = 1; h < E; h <<= 1) {
-            if (h < b_h) {
+            for (int e = 0; e < E; ++e) v[e] = rel + e < nrot ? __bfloat162float(row[pidx[e]]) : 0.0f;
+            // stages inside the lane: distance h = 1, 2, ..., E/2
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    if ((e & h) == 0) {
-                        const float a = v[e], b = v[e + h];
-                        v[e] = a + b;
-                        v[e + h] = a - b;
+            for (int h = 1; h < E; h <<= 1) {
+                if (h < b_h) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        if ((e & h) == 0) {
+                            const float a = v[e], b = v[e + h];
+                            v[e] = a + b;
+                            v[e + h] = a - b;
+                        }
                     }
                 }
             }
-        }
-        // stages across lanes: distance h = E, 2E, ..., 16E  (lane distance h / E)
+            // stages across lanes: distance h = E, 2E, ..., 16E  (lane distance h / E)
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            if (d * E < b_h) {
-                const bool upper = (lane & d) != 0;
+            for (int d = 1; d < 32; d <<= 1) {
+                if (d * E < b_h) {
+                    const bool upper = (lane & d) != 0;
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const float other = __shfl_xor_sync(0xffffffffu, v[e], d);
-                    v[e] = upper ? other - v[e] : v[e] + other;
+                    for (int e = 0; e < E; ++e) {
+                        const float other = __shfl_xor_sync(0xffffffffu, v[e], d);
+                        v[e] = upper ? other - v[e] : v[e] + other;
+                    }
                 }
             }
-        }
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            const int idx = rel + e;
-            if (idx < nrot) xout[b_i + idx] = __float2bfloat16_rn(v[e] * inv_sqrt_bh);
+            for (int e = 0; e < E; ++e)
+                if (rel + e < nrot) xout[(size_t)r * n + b_i + rel + e] = __float2bfloat16_rn(v[e] * inv_sqrt_bh);
         }
     }
     __syncthreads();
 
-    uint4* dst = reinterpret_cast<uint4*>(xrot + (size_t)t * ldo);
-    for (int i = tid; i < n / 8; i += kRotThreads) dst[i] = reinterpret_cast<const uint4*>(xout)[i];
-    if (s64 != nullptr) {
-        const int nsteps = n / 64;
-        for (int st = warp; st < nsteps; st += kWarps) {
-            const __nv_bfloat162 p = reinterpret_cast<const __nv_bfloat162*>(xout)[st * 32 + lane];
-            float s = __low2float(p) + __high2float(p);
+    for (int r = 0; r < nt; ++r) {
+        const __nv_bfloat16* out_row = xout + (size_t)r * n;
+        uint4* dst = reinterpret_cast<uint4*>(xrot + (size_t)(t0 + r) * ldo);
+        for (int i = tid; i < n / 8; i += kRotThreads) dst[i] = reinterpret_cast<const uint4*>(out_row)[i];
+        if (s64 != nullptr) {
+            const int nsteps = n / 64;
+            for (int st = warp; st < nsteps; st += kWarps) {
+                const __nv_bfloat162 p = reinterpret_cast<const __nv_bfloat162*>(out_row)[st * 32 + lane];
+                float s = __low2float(p) + __high2float(p);
 #pragma unroll
-            for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-            if (lane == 0) s64[(size_t)t * s64_ld + st] = s;
+                for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+                if (lane == 0) s64[(size_t)(t0 + r) * s64_ld + st] = s;
+            }
         }
     }
 }
@@ -302,17 +315,27 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
     }
 }
 
+template <int E, int TOK>
+cudaError_t launch_rotate_et(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
+                             __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s) {
+    const size_t smem = (size_t)d.d_in * 4 * TOK;
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(rotate_kernel<E, TOK>, TOK == 1 ? 32768 * 4 : 160 * 1024, &attr_done);
+    if (e != cudaSuccess) return e;
+    const float inv = (float)(1.0 / sqrt((double)d.block_size));
+    rotate_kernel<E, TOK><<<(T + TOK - 1) / TOK, kRotThreads, smem, s>>>(x, ldx, perm, xrot, ldo, s64, s64_stride(d.d_in),
+                                                                       status, d.d_in, d.identity_cols, d.block_size,
+                                                                       inv, T);
+    return cudaGetLastError();
+}
+
+// Four rows per CTA when there are many tokens and the rows fit shared memory, else one.
 template <int E>
 cudaError_t launch_rotate_e(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
                             __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s) {
-    const size_t smem = (size_t)d.d_in * 4;
-    static unsigned long long attr_done = 0;
-    cudaError_t e = ensure_dynamic_smem(rotate_kernel<E>, 32768 * 4, &attr_done);  // largest supported row
-    if (e != cudaSuccess) return e;
-    const float inv = (float)(1.0 / sqrt((double)d.block_size));
-    rotate_kernel<E><<<T, kRotThreads, smem, s>>>(x, ldx, perm, xrot, ldo, s64, s64_stride(d.d_in), status, d.d_in,
-                                                  d.identity_cols, d.block_size, inv);
-    return cudaGetLastError();
+    if (T >= 256 && (size_t)d.d_in * 16 <= 160 * 1024)
+        return launch_rotate_et<E, 4>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
+    return launch_rotate_et<E, 1>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
 }
 
 }  // namespace
