@@ -99,6 +99,16 @@ def test_shapes_in_the_parameter_domain(n, m, bits, g, b_i, b_h, r, T):
     _check_forward(layer, d, synth.activations(T, n, seed=7, outlier_frac=0.01))
 
 
+@pytest.mark.parametrize("bits,g", [(4, 128), (3, 64), (2, 64)])
+@pytest.mark.parametrize("T", [1, 2, 5, 8])
+@pytest.mark.parametrize("n,m,r,b", [(2048, 144, 17, 128), (4096, 528, 32, 256), (4096, 64, 0, 64)])
+def test_small_batch_path_row_and_token_edges(bits, g, T, n, m, r, b):
+    # small-batch path with row counts that leave the last CTA half empty (m % 32 = 16) and few rows overall
+    layer = random_layer_np(n, m, bits, g, r, seed=n + m + bits + T)
+    d = lopro.make_desc(n, m, bits, g, b, identity_cols=b, rank=r)
+    _check_forward(layer, d, synth.activations(T, n, seed=T + 3, outlier_frac=0.01))
+
+
 def test_outputs_can_be_strided_and_calls_repeat_bitwise():
     n, m, bits, g, r, T = 1024, 256, 4, 128, 16, 8
     layer = random_layer_np(n, m, bits, g, r, seed=1)
