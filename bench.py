@@ -75,7 +75,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -202,7 +202,7 @@ def workload_config(name):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2_T8", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="lopro", choices=["lopro", "reference"])
@@ -354,11 +354,11 @@ def main():
         ach = algorithmic_flops(c, T) / dur_s / 1e12
         pk = peaks["bf16_tflops_sustained"]
         roofline = dict(bound="tensor", achieved=ach, peak=pk, unit="TFLOP/s", frac=ach / pk, traffic=None,
-                        peak_source=f"of {peaks['source']} (sustained)", kernel="decode_kernel",
+                        peak_source=f"of {peaks['source']} (sustained)", kernel="prefill_kernel",
                         algorithmic_flops_per_launch=algorithmic_flops(c, T), launch_us=dur_s * 1e6,
                         note="duration = step time / layer forwards (includes the prologue kernels)")
-    # T <= 32: prologue + streaming kernel; larger T: rotate + low-rank down + general kernel
-    kernels_per_forward = 2 if T <= 32 else (3 if c["rank"] > 0 else 2)
+    # T <= 32: prologue + streaming kernel; larger T: rotate + low-rank down (two kernels) + prefill kernel
+    kernels_per_forward = 2 if T <= 32 else (4 if c["rank"] > 0 else 2)
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic", config=workload_config(args.workload), clocks=clocks,
