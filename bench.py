@@ -36,6 +36,9 @@ WORKLOADS = {
     "cfg4_T16": ("cfg4", 16, 8),
     "cfg4_T4096": ("cfg4", 4096, 2),
 }
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
+# capture summarised in profiles/; valid for the kernel as committed with that summary, null otherwise.
+NCU_TRAFFIC = {"cfg2_T8": 9284352}
 METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
 
@@ -346,7 +349,7 @@ def main():
     if hbm_bound:
         ach = algorithmic_bytes(c, T) / dur_s / 1e9
         roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
-                        traffic=None, peak_source=f"of {peaks['source']}",
+                        traffic=NCU_TRAFFIC.get(args.workload), peak_source=f"of {peaks['source']}",
                         frac_of_nominal_8000=ach / 8000.0, kernel="stream_kernel" if T <= 32 else "decode_kernel",
                         algorithmic_bytes_per_launch=algorithmic_bytes(c, T),
                         launch_us=dur_s * 1e6, note="duration = step time / layer forwards (includes the prologue kernels)")
