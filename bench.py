@@ -38,7 +38,7 @@ WORKLOADS = {
 }
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
 # capture summarised in profiles/; valid for the kernel as committed with that summary, null otherwise.
-NCU_TRAFFIC = {"cfg2_T8": 9284352}
+NCU_TRAFFIC = {("cfg2_T8", "stream_kernel"): 9284352}
 METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
 
@@ -340,34 +340,36 @@ def main():
     tokens_per_step = T * ring * world
     value = tokens_per_step / (ms_per_step * 1e-3)
     e2e_value = T * ring * world / (e2e_ms / e2e_steps * 1e-3)
-    # Dominant kernel: the streaming forward kernel, launched once per layer.  Its launch duration is
-    # taken as (step time / launches), i.e. the whole per-layer time including the two small
-    # prologue kernels -- an upper bound on the kernel's own duration, a lower bound on `achieved`.
+    # Dominant kernel: the forward kernel that reads the packed weights, launched once per layer.  Its
+    # launch duration is taken as (step time / launches), i.e. the whole per-layer time including any
+    # prologue kernels of the path -- an upper bound on the kernel's own duration, a lower bound on
+    # `achieved`.
+    path, kernels_per_forward = lopro.linear_fwd_path(d, T)
+    path_name = lopro.PATH_NAMES.get(path, "?")
+    kernel_name = {"stream": "stream_kernel", "general": "decode_kernel",
+                   "prefill": "prefill_kernel"}.get(path_name, "?")
+    note = "duration = step time / layer forwards (includes the prologue kernels)"
     launches_per_step = ring
     dur_s = ms_per_step * 1e-3 / launches_per_step
     hbm_bound = T <= 64
     if hbm_bound:
         ach = algorithmic_bytes(c, T) / dur_s / 1e9
         roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
-                        traffic=NCU_TRAFFIC.get(args.workload), peak_source=f"of {peaks['source']}",
-                        frac_of_nominal_8000=ach / 8000.0, kernel="stream_kernel" if T <= 32 else "decode_kernel",
-                        algorithmic_bytes_per_launch=algorithmic_bytes(c, T),
-                        launch_us=dur_s * 1e6, note="duration = step time / layer forwards (includes the prologue kernels)")
+                        traffic=NCU_TRAFFIC.get((args.workload, kernel_name)), peak_source=f"of {peaks['source']}",
+                        frac_of_nominal_8000=ach / 8000.0, kernel=kernel_name,
+                        algorithmic_bytes_per_launch=algorithmic_bytes(c, T), launch_us=dur_s * 1e6, note=note)
     else:
         ach = algorithmic_flops(c, T) / dur_s / 1e12
         pk = peaks["bf16_tflops_sustained"]
         roofline = dict(bound="tensor", achieved=ach, peak=pk, unit="TFLOP/s", frac=ach / pk, traffic=None,
-                        peak_source=f"of {peaks['source']} (sustained)", kernel="prefill_kernel",
-                        algorithmic_flops_per_launch=algorithmic_flops(c, T), launch_us=dur_s * 1e6,
-                        note="duration = step time / layer forwards (includes the prologue kernels)")
-    # T <= 32: prologue + streaming kernel; larger T: rotate + low-rank down (two kernels) + prefill kernel
-    kernels_per_forward = 2 if T <= 32 else (4 if c["rank"] > 0 else 2)
+                        peak_source=f"of {peaks['source']} (sustained)", kernel=kernel_name,
+                        algorithmic_flops_per_launch=algorithmic_flops(c, T), launch_us=dur_s * 1e6, note=note)
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic", config=workload_config(args.workload), clocks=clocks,
                 e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=ring * T * c["d_in"] * 2,
                          d2h_bytes_per_step=ring * T * c["d_out"] * 2, steps=e2e_steps),
-                gpu_launches=kernels_per_forward * ring * args.steps, roofline=roofline,
+                gpu_launches=kernels_per_forward * ring * args.steps, path=path_name, roofline=roofline,
                 step_ms_min=min(step_ms), step_ms_median=statistics.median(step_ms),
                 cuda_graph=graph is not None)
     if not args.no_cpu_baseline and world == 1:

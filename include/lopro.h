@@ -176,6 +176,21 @@ LOPRO_API lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* pack
                               void* y, int64_t ldy, int32_t out_dtype, int32_t T, void* workspace,
                               size_t workspace_bytes, void* stream);
 
+/* Which kernels lopro_linear_fwd runs for this layer and token count on the current device (an
+ * implementation detail of this library, exposed so that tests and benchmarks can name what they
+ * measure; the paper's Appendix A.3 lists the steps, not their grouping into launches).
+ *   LOPRO_PATH_STREAM   2 launches: prologue (permutation, rotation, B x) + streaming product, T <= 32
+ *   LOPRO_PATH_GENERAL  rotation, B x, register-ring product (any shape the descriptor allows)
+ *   LOPRO_PATH_PREFILL  rotation, B x (2 launches), tcgen05 product, T > 32
+ * Returns the path (> 0) and stores the number of kernel launches in *launches (may be NULL), or
+ * returns 0 for a bad descriptor or T < 1. */
+typedef enum {
+    LOPRO_PATH_STREAM = 2,
+    LOPRO_PATH_GENERAL = 3,
+    LOPRO_PATH_PREFILL = 4
+} lopro_path;
+LOPRO_API int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches);
+
 /* The same forward for callers whose activations live in HOST memory (Eq. 8 end to end):
  * copies x_host [T][n] (dense, bf16; pinned memory makes the copy asynchronous) to the device,
  * runs lopro_linear_fwd and copies y [T][m] back to y_host.  `workspace` must hold

@@ -194,6 +194,21 @@ lopro_status lopro_rotate(const lopro_desc* desc, const int32_t* perm, const uin
     return e == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }
 
+int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches) {
+    if (!desc || check_desc(*desc) != LOPRO_OK || desc->layout != LOPRO_LAYOUT_FRAGMENT || T < 1) return 0;
+    int32_t path, n;
+    if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
+        path = LOPRO_PATH_STREAM;
+        n = 2;
+    } else {
+        const int pre = 1 + (desc->rank > 0 ? (T > kDecodeMaxT ? 2 : 1) : 0);
+        path = prefill_supported(*desc, T) ? LOPRO_PATH_PREFILL : LOPRO_PATH_GENERAL;
+        n = pre + 1;
+    }
+    if (launches) *launches = n;
+    return path;
+}
+
 lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const uint16_t* x_bf16, int64_t ldx,
                               void* y, int64_t ldy, int32_t out_dtype, int32_t T, void* workspace,
                               size_t workspace_bytes, void* stream) {

@@ -2,7 +2,7 @@
 // by bulk asynchronous copies (steps "Dequant(W_q) X" and "U (Sigma Y)" of Appendix A.3, summed as
 // in Eq. 8).
 //
-// One CTA owns 32 output rows (two 16-row tiles of the fragment layout) over the WHOLE K range, so
+// One CTA owns 32 or 64 output rows (two or four 16-row tiles of the fragment layout) over the WHOLE K range, so
 // no partial sums ever cross CTAs.  A producer warp fills a ring of shared-memory stages with
 // cp.async.bulk copies (16 steps of 64 columns per stage): the layer's own data -- codes,
 // (scale, zero) pairs, the rows of A -- is requested before griddepcontrol.wait, i.e. while the
@@ -18,6 +18,7 @@
 // Every wait on an mbarrier is bounded; a wait that runs out stores LOPRO_ERR_TIMEOUT in the
 // workspace status word and the CTA stops waiting (its outputs are then unspecified).
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace lopro {
 
@@ -26,11 +27,8 @@ namespace {
 constexpr int kConsumerWarps = 16;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
 constexpr int kStageSteps = 16;                      // 64-column steps per stage = one per consumer warp
-constexpr int kStageCols = kStageSteps * 64;
 constexpr int kXsStride = kActRecord / 2;            // bf16 elements between the token rows of a stage
-constexpr int kRowTiles = 2;                         // 16-row tiles per CTA
 constexpr int kMaxStages = 8;
-constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct StreamParams {
     const uint32_t* codes;
@@ -50,76 +48,7 @@ struct StreamParams {
     int off_sz, off_a, off_t, off_ring, stage_bytes, off_stage_x;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the limit ran out (the caller records the time-out and carries on).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t* a, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t* a, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-
-constexpr uint32_t kMagic128 = 0x43004300u;  // two bf16 128.0 (ulp 1): 128.0 | c == 128 + c
-
-template <int BITS>
-__device__ __forceinline__ void expand_codes(uint32_t (&a)[16], const uint32_t (&w)[BITS]) {
-    if constexpr (BITS == 4) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = ((w[j] >> (4 * rho)) & 0x000F000Fu) | kMagic128;
-    } else if constexpr (BITS == 2) {
-#pragma unroll
-        for (int pi = 0; pi < 16; ++pi) a[pi] = ((w[pi >> 3] >> (2 * (pi & 7))) & 0x00030003u) | kMagic128;
-    } else {
-#pragma unroll
-        for (int pi = 0; pi < 15; ++pi) a[pi] = ((w[pi / 5] >> (3 * (pi % 5))) & 0x00070007u) | kMagic128;
-        a[15] = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u) | kMagic128;
-    }
-}
-
-template <int BITS, int NT>
+template <int BITS, int NT, int RT>
 __global__ void __launch_bounds__(kThreads, 1)
 stream_kernel(const StreamParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -130,8 +59,8 @@ stream_kernel(const StreamParams p) {
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tg = lane & 3;
-    const int rt0 = blockIdx.x * kRowTiles;                         // first 16-row tile of this CTA
-    const int n_rt = min(kRowTiles, (p.m >> 4) - rt0);              // live row tiles (1 or 2)
+    const int rt0 = blockIdx.x * RT;                     // first 16-row tile of this CTA
+    const int n_rt = min(RT, (p.m >> 4) - rt0);          // live row tiles
     const int tc = min(kTok, p.T);                                  // live tokens
     const uint32_t bar0 = smem_u32(bars);
     auto wfull = [&](int s) { return bar0 + 8u * (uint32_t)s; };
@@ -175,9 +104,9 @@ stream_kernel(const StreamParams p) {
                  p.act + (size_t)stage * p.t_pad * kActRecord, bytes, xfull(slot));
     };
 
-    float yacc[kRowTiles][NT][4];
+    float yacc[RT][NT][4];
 #pragma unroll
-    for (int r = 0; r < kRowTiles; ++r)
+    for (int r = 0; r < RT; ++r)
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -253,7 +182,7 @@ stream_kernel(const StreamParams p) {
                     sx[nt][1] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg + 1) * kActRecord)[warp];
                 }
 #pragma unroll
-                for (int r = 0; r < kRowTiles; ++r) {
+                for (int r = 0; r < RT; ++r) {
                     if (r < n_rt) {
                         uint32_t w[BITS];
                         const uint32_t* wp = reinterpret_cast<const uint32_t*>(stage + (r * kStageSteps + warp) * kStepBytes) +
@@ -315,31 +244,33 @@ stream_kernel(const StreamParams p) {
     };
     if (p.r_pad > 0 && warp < n_rt) {
         if (!mbar_wait(tbar, 0) && lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
-        if (warp == 0) lowrank_up(yacc[0], 0);
-        else lowrank_up(yacc[1], 1);
+#pragma unroll
+        for (int r = 0; r < RT; ++r)
+            if (warp == r) lowrank_up(yacc[r], r);
     }
 
-    // reduction over the consumer warps: red[warp][token][32 rows]
+    // reduction over the consumer warps: red[warp][token][RT * 16 rows]
+    constexpr int kRows = RT * 16;
     float* red = reinterpret_cast<float*>(smem + p.off_ring);
     if (warp < kConsumerWarps) {
 #pragma unroll
-        for (int r = 0; r < kRowTiles; ++r)
+        for (int r = 0; r < RT; ++r)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int tk = nt * 8 + 2 * tg + (i & 1), rl = r * 16 + gq + 8 * (i >> 1);
-                    red[(warp * kTok + tk) * 32 + rl] = yacc[r][nt][i];
+                    red[(warp * kTok + tk) * kRows + rl] = yacc[r][nt][i];
                 }
     }
     __syncthreads();
     const int rows_here = n_rt * 16;
-    for (int i = tid; i < tc * 32; i += kThreads) {
-        const int tk = i >> 5, rl = i & 31;
+    for (int i = tid; i < tc * kRows; i += kThreads) {
+        const int tk = i / kRows, rl = i - tk * kRows;
         if (rl < rows_here) {
             float sum = 0.0f;
 #pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) sum += red[(w * kTok + tk) * 32 + rl];
+            for (int w = 0; w < kConsumerWarps; ++w) sum += red[(w * kTok + tk) * kRows + rl];
             const size_t o = (size_t)tk * p.ldy + (size_t)rt0 * 16 + rl;
             if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = sum;
             else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(sum);
@@ -347,13 +278,13 @@ stream_kernel(const StreamParams p) {
     }
 }
 
-template <int BITS, int NT>
-cudaError_t launch_stream_nt(const StreamParams& p, int smem_bytes, cudaStream_t s) {
+template <int BITS, int NT, int RT>
+cudaError_t launch_stream_k(const StreamParams& p, int smem_bytes, cudaStream_t s) {
     static unsigned long long attr_done = 0;
-    cudaError_t e = ensure_dynamic_smem(stream_kernel<BITS, NT>, kStreamMaxSmem, &attr_done);
+    cudaError_t e = ensure_dynamic_smem(stream_kernel<BITS, NT, RT>, kStreamMaxSmem, &attr_done);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.m / 16 + kRowTiles - 1) / kRowTiles);
+    cfg.gridDim = dim3((p.m / 16 + RT - 1) / RT);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = s;
@@ -362,20 +293,22 @@ cudaError_t launch_stream_nt(const StreamParams& p, int smem_bytes, cudaStream_t
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, stream_kernel<BITS, NT>, p);
+    return cudaLaunchKernelEx(&cfg, stream_kernel<BITS, NT, RT>, p);
 }
 
 template <int BITS>
-cudaError_t launch_stream_bits(const StreamParams& p, int nt, int smem_bytes, cudaStream_t s) {
-    if (nt == 1) return launch_stream_nt<BITS, 1>(p, smem_bytes, s);
-    if (nt == 2) return launch_stream_nt<BITS, 2>(p, smem_bytes, s);
-    return launch_stream_nt<BITS, 4>(p, smem_bytes, s);
+cudaError_t launch_stream_bits(const StreamParams& p, int nt, int rt, int smem_bytes, cudaStream_t s) {
+    if (nt == 1) return rt == 4 ? launch_stream_k<BITS, 1, 4>(p, smem_bytes, s) : launch_stream_k<BITS, 1, 2>(p, smem_bytes, s);
+    if (nt == 2) return rt == 4 ? launch_stream_k<BITS, 2, 4>(p, smem_bytes, s) : launch_stream_k<BITS, 2, 2>(p, smem_bytes, s);
+    return launch_stream_k<BITS, 4, 2>(p, smem_bytes, s);
 }
 
 struct StreamPlan {
-    int nt, n_stages, total_stages, smem_bytes;
+    int nt, rt, n_stages, total_stages, smem_bytes;
     int off_sz, off_a, off_t, off_ring, stage_bytes, off_stage_x;
 };
+
+bool plan_layout(const lopro_desc& d, StreamPlan* pl, int r_pad, int ng, int ktok);
 
 bool plan_stream(const lopro_desc& d, int T, StreamPlan* pl) {
     if (T < 1 || T > kDecodeMaxT) return false;
@@ -383,23 +316,35 @@ bool plan_stream(const lopro_desc& d, int T, StreamPlan* pl) {
     const int ng = d.d_in / d.group_size;
     pl->nt = T <= 8 ? 1 : (T <= 16 ? 2 : 4);
     const int ktok = pl->nt * 8;
+    // Rows per CTA: 64 instead of 32 when the layer is tall enough to keep two CTAs per SM busy anyway --
+    // every CTA reads all of x~ from L2, so taller CTAs halve that traffic.
+    pl->rt = (pl->nt <= 2 && (d.d_out / 16) / 4 >= 296) ? 4 : 2;
+    for (;;) {
+        if (plan_layout(d, pl, r_pad, ng, ktok)) return true;
+        if (pl->rt == 2) return false;
+        pl->rt = 2;
+    }
+}
+
+bool plan_layout(const lopro_desc& d, StreamPlan* pl, int r_pad, int ng, int ktok) {
     int off = 0;
     pl->off_sz = off;
-    off += round_up_int(kRowTiles * ng * 64, 128);
+    off += round_up_int(pl->rt * ng * 64, 128);
     pl->off_a = off;
-    off += round_up_int(kRowTiles * 16 * r_pad * 2, 128);
+    off += round_up_int(pl->rt * 16 * r_pad * 2, 128);
     pl->off_t = off;
     off += round_up_int(ktok * r_pad * 2, 128);
     pl->off_ring = off;
-    const int w_bytes = kRowTiles * kStageSteps * 128 * d.bits;
+    const int w_bytes = pl->rt * kStageSteps * 128 * d.bits;
     pl->off_stage_x = w_bytes;
     pl->stage_bytes = round_up_int(w_bytes + ktok * kActRecord, 128);
     pl->total_stages = (d.d_in / 64 + kStageSteps - 1) / kStageSteps;
-    const int red_bytes = kConsumerWarps * ktok * 32 * 4;
+    const int red_bytes = kConsumerWarps * ktok * pl->rt * 16 * 4;
     int stages = (kStreamMaxSmem - off) / pl->stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages > pl->total_stages) stages = pl->total_stages;
     if (stages < 1) return false;
+    if (pl->rt > 2 && stages < pl->total_stages && stages < 3) return false;  // too shallow a ring: fall back to 32 rows
     int ring = stages * pl->stage_bytes;
     if (ring < red_bytes) ring = red_bytes;
     pl->n_stages = stages;
@@ -447,9 +392,9 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
     p.stage_bytes = pl.stage_bytes;
     p.off_stage_x = pl.off_stage_x;
     switch (d.bits) {
-        case 2: return launch_stream_bits<2>(p, pl.nt, pl.smem_bytes, s);
-        case 3: return launch_stream_bits<3>(p, pl.nt, pl.smem_bytes, s);
-        default: return launch_stream_bits<4>(p, pl.nt, pl.smem_bytes, s);
+        case 2: return launch_stream_bits<2>(p, pl.nt, pl.rt, pl.smem_bytes, s);
+        case 3: return launch_stream_bits<3>(p, pl.nt, pl.rt, pl.smem_bytes, s);
+        default: return launch_stream_bits<4>(p, pl.nt, pl.rt, pl.smem_bytes, s);
     }
 }
 

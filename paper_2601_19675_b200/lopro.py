@@ -22,7 +22,7 @@ SEC_HEADER, SEC_CODES, SEC_SCALEZERO, SEC_PERM, SEC_A, SEC_B = range(6)
 # every symbol include/lopro.h declares
 SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packed_bytes", "lopro_packed_section",
            "lopro_workspace_bytes", "lopro_pack", "lopro_unpack", "lopro_rotate", "lopro_linear_fwd",
-           "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc"]
+           "lopro_linear_fwd_path", "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc"]
 
 
 class Desc(ctypes.Structure):
@@ -72,6 +72,8 @@ def lib():
         L.lopro_rotate.argtypes = [dp, vp, vp, i64, vp, i64, i32, vp]
         L.lopro_linear_fwd.restype = ctypes.c_int
         L.lopro_linear_fwd.argtypes = [dp, vp, vp, i64, vp, i64, i32, i32, vp, sz, vp]
+        L.lopro_linear_fwd_path.restype = i32
+        L.lopro_linear_fwd_path.argtypes = [dp, i32, ctypes.POINTER(i32)]
         L.lopro_host_staging_bytes.restype = sz
         L.lopro_host_staging_bytes.argtypes = [dp, i32, i32]
         L.lopro_linear_fwd_host.restype = ctypes.c_int
@@ -115,6 +117,17 @@ def packed_section(desc, section):
 
 def workspace_bytes(desc, T):
     return int(lib().lopro_workspace_bytes(ctypes.byref(desc), int(T)))
+
+
+PATH_STREAM, PATH_GENERAL, PATH_PREFILL = 2, 3, 4
+PATH_NAMES = {PATH_STREAM: "stream", PATH_GENERAL: "general", PATH_PREFILL: "prefill"}
+
+
+def linear_fwd_path(desc, T):
+    """(path, launches) of lopro_linear_fwd for this layer and token count; path 0 = bad arguments."""
+    n = ctypes.c_int32(0)
+    path = int(lib().lopro_linear_fwd_path(ctypes.byref(desc), int(T), ctypes.byref(n)))
+    return path, int(n.value)
 
 
 def host_staging_bytes(desc, T, out_dtype=OUT_BF16):

@@ -86,6 +86,18 @@ def test_workspace_size_is_monotone_in_tokens():
     assert lopro.host_staging_bytes(d, 8) >= 8 * 4096 * 2 * 2
 
 
+def test_forward_path_query_names_the_small_batch_and_general_paths():
+    d = lopro.make_desc(4096, 4096, 4, 128, 128, rank=32)
+    assert lopro.linear_fwd_path(d, 8) == (lopro.PATH_STREAM, 2)       # prologue + streaming kernel
+    assert lopro.linear_fwd_path(d, 0) == (0, 0) and lopro.linear_fwd_path(d, -3) == (0, 0)
+    wide = lopro.make_desc(4096, 4096, 4, 128, 1024, identity_cols=0, rank=32)  # b_H beyond the prologue's 256
+    path, launches = lopro.linear_fwd_path(wide, 8)
+    assert path == lopro.PATH_GENERAL and launches == 3                # rotation, B x, product
+    assert lopro.linear_fwd_path(lopro.make_desc(4096, 4096, 4, 128, 1024, identity_cols=0, rank=0), 8)[1] == 2
+    bad = lopro.make_desc(4096, 4096, 5, 128, 128, rank=32)
+    assert lopro.linear_fwd_path(bad, 8)[0] == 0
+
+
 def test_null_and_bad_arguments_are_rejected_before_any_cuda_call():
     import ctypes
     L = lopro.lib()
