@@ -346,7 +346,7 @@ def main():
     # `achieved`.
     path, kernels_per_forward = lopro.linear_fwd_path(d, T)
     path_name = lopro.PATH_NAMES.get(path, "?")
-    kernel_name = {"stream": "stream_kernel", "general": "decode_kernel",
+    kernel_name = {"stream": "stream_kernel", "tall": "tall_kernel", "general": "decode_kernel",
                    "prefill": "prefill_kernel"}.get(path_name, "?")
     note = "duration = step time / layer forwards (includes the prologue kernels)"
     launches_per_step = ring

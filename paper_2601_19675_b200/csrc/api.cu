@@ -194,11 +194,18 @@ lopro_status lopro_rotate(const lopro_desc* desc, const int32_t* perm, const uin
     return e == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }
 
+// LOPRO_NO_TALL=1 keeps the persistent kernel for tall layers off (A/B comparison and tests of the other kernel).
+static bool use_tall(const lopro_desc& d, int T) {
+    const char* e = getenv("LOPRO_NO_TALL");
+    if (e && e[0] == '1') return false;
+    return tall_supported(d, T);
+}
+
 int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches) {
     if (!desc || check_desc(*desc) != LOPRO_OK || desc->layout != LOPRO_LAYOUT_FRAGMENT || T < 1) return 0;
     int32_t path, n;
     if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
-        path = LOPRO_PATH_STREAM;
+        path = use_tall(*desc, T) ? LOPRO_PATH_TALL : LOPRO_PATH_STREAM;
         n = 2;
     } else {
         const int pre = 1 + (desc->rank > 0 ? (T > kDecodeMaxT ? 2 : 1) : 0);
@@ -242,7 +249,9 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
         if (launch_prologue(*desc, perm, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot,
                             (__half*)(ws + W.off_t), W.t_pad, status, T, s) != cudaSuccess)
             return LOPRO_ERR_CUDA;
-        if (launch_stream(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+        const cudaError_t e = use_tall(*desc, T) ? launch_tall(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s)
+                                                 : launch_stream(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s);
+        if (e != cudaSuccess) return LOPRO_ERR_CUDA;
         return LOPRO_OK;
     }
     if (launch_rotate(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, xrot, desc->d_in, s64, status, T, s) !=

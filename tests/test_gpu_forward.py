@@ -37,9 +37,9 @@ def _check_forward(layer, d, x_bits, rows=None, gate_a=GATE_A, gate_b=GATE_B):
     x64 = o.bf16_bits_to_f64(x_bits)
     exact = o.forward_exact(x64, **args)
     mirrored = o.forward_mirrored(x64, **args, round_w=T > 32, round_t="f16", out="f32")
-    # declared roundings cannot hide an error (rounding the weights to bf16 alone reaches ~1 % on the
-    # max-over-entries measure, hence the wider guard for the prefill path)
-    assert o.max_rel_err(mirrored, exact) <= (2e-2 if T > 32 else 1e-2)
+    # declared roundings cannot hide an error: by themselves they stay inside gate A (rounding x~ to bf16 alone
+    # reaches ~1 % on the max-over-entries measure once a layer has a few hundred thousand outputs)
+    assert o.max_rel_err(mirrored, exact) <= GATE_A
     got_bf = device_bf16_to_f64(y_bf)
     got_f32 = y_f32.cpu().numpy().astype(np.float64)
     if rows is not None:
@@ -107,6 +107,40 @@ def test_small_batch_path_row_and_token_edges(bits, g, T, n, m, r, b):
     layer = random_layer_np(n, m, bits, g, r, seed=n + m + bits + T)
     d = lopro.make_desc(n, m, bits, g, b, identity_cols=b, rank=r)
     _check_forward(layer, d, synth.activations(T, n, seed=T + 3, outlier_frac=0.01))
+
+
+def _tall_rows(tiles_per_sm, extra_tiles):
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    return 16 * (sms * tiles_per_sm + extra_tiles)
+
+
+@pytest.mark.parametrize("bits,g,r", [(4, 128, 32), (3, 64, 17), (2, 64, 128), (4, 256, 0)])
+@pytest.mark.parametrize("T", [1, 8, 16, 32])
+@pytest.mark.parametrize("per_sm,extra", [(2, 1), (4, 100), (5, 7), (6, 3)])
+def test_tall_layers_persistent_kernel(bits, g, r, T, per_sm, extra):
+    # more 16-row tiles than twice the SM count: the persistent kernel, with runs of tiles per CTA that end in
+    # groups of 1, 2 and 3 tiles (2/3, 4/4+1, 4+1/4+2, 4+2/4+3 tiles per CTA) and a ragged last stage (36 steps)
+    n, m = 2304, _tall_rows(per_sm, extra)
+    d = lopro.make_desc(n, m, bits, g, 64, identity_cols=64, rank=r)
+    assert lopro.linear_fwd_path(d, T)[0] == lopro.PATH_TALL
+    layer = random_layer_np(n, m, bits, g, r, seed=m + bits + T)
+    _check_forward(layer, d, synth.activations(T, n, seed=T + 11, outlier_frac=0.01))
+
+
+def test_tall_kernel_agrees_with_the_per_group_kernel(monkeypatch):
+    # both small-batch kernels sum the same products in fp32 in different orders: outputs agree to fp32 rounding
+    n, m, bits, g, r, T = 1024, _tall_rows(4, 9), 4, 128, 32, 8
+    d = lopro.make_desc(n, m, bits, g, 128, rank=r)
+    layer = random_layer_np(n, m, bits, g, r, seed=3)
+    blob = _pack(layer, d)
+    x = bf16_bits_to_device(synth.activations(T, n, seed=4))
+    y_tall = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
+    monkeypatch.setenv("LOPRO_NO_TALL", "1")
+    assert lopro.linear_fwd_path(d, T)[0] == lopro.PATH_STREAM
+    y_stream = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
+    torch.cuda.synchronize()
+    scale = y_stream.abs().max().item()
+    assert (y_tall - y_stream).abs().max().item() <= 1e-5 * scale
 
 
 def test_outputs_can_be_strided_and_calls_repeat_bitwise():
