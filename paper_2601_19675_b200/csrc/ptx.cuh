@@ -60,19 +60,31 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
 
 constexpr uint32_t kMagic128 = 0x43004300u;  // two bf16 128.0 (ulp 1): 128.0 | c == 128 + c
 
+// (a & mask) | magic in ONE logic instruction (truth table 0xEA), both constants held in registers --
+// left to the compiler this becomes two instructions, since only one operand may be an immediate.
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t mask, uint32_t magic) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(magic));
+    return d;
+}
+
 template <int BITS>
 __device__ __forceinline__ void expand_codes(uint32_t (&a)[16], const uint32_t (&w)[BITS]) {
+    const uint32_t magic = kMagic128;
     if constexpr (BITS == 4) {
+        const uint32_t mask = 0x000F000Fu;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = ((w[j] >> (4 * rho)) & 0x000F000Fu) | kMagic128;
+            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = and_or(w[j] >> (4 * rho), mask, magic);
     } else if constexpr (BITS == 2) {
+        const uint32_t mask = 0x00030003u;
 #pragma unroll
-        for (int pi = 0; pi < 16; ++pi) a[pi] = ((w[pi >> 3] >> (2 * (pi & 7))) & 0x00030003u) | kMagic128;
+        for (int pi = 0; pi < 16; ++pi) a[pi] = and_or(w[pi >> 3] >> (2 * (pi & 7)), mask, magic);
     } else {
+        const uint32_t mask = 0x00070007u;
 #pragma unroll
-        for (int pi = 0; pi < 15; ++pi) a[pi] = ((w[pi / 5] >> (3 * (pi % 5))) & 0x00070007u) | kMagic128;
+        for (int pi = 0; pi < 15; ++pi) a[pi] = and_or(w[pi / 5] >> (3 * (pi % 5)), mask, magic);
         a[15] = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u) | kMagic128;
     }
 }

@@ -67,6 +67,80 @@ __device__ __forceinline__ void named_arrive(int id) {
     asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(kConsumerThreads) : "memory");
 }
 
+// One 16-row tile times one 64-column step: expand the packed codes to bf16 operands 128 + c, four
+// m16n8k16 products per token tile, then scale and zero-point in fp32 against the 64-column sums.
+template <int BITS, int NT>
+__device__ __forceinline__ void tile_step(const unsigned char* codes_rt, const uint32_t* szs, const unsigned char* srec,
+                                          uint32_t xs_u32, int st, int gl, int lane, float (&yacc)[NT][4]) {
+    constexpr int kStepBytes = 128 * BITS;
+    const int gq = lane >> 2, tg = lane & 3;
+    uint32_t b[NT][8];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const uint32_t addr = xs_u32 + (uint32_t)(nt * 8 * kActRecord + st * 128);
+        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][0]), addr);
+        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][4]), addr + 64u);
+    }
+    float sx[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        sx[nt][0] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg) * kActRecord)[st];
+        sx[nt][1] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg + 1) * kActRecord)[st];
+    }
+    uint32_t w[BITS];
+    const uint32_t* wp = reinterpret_cast<const uint32_t*>(codes_rt + st * kStepBytes) + lane * BITS;
+    if constexpr (BITS == 4) {
+        const uint4 v = *reinterpret_cast<const uint4*>(wp);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else if constexpr (BITS == 2) {
+        const uint2 v = *reinterpret_cast<const uint2*>(wp);
+        w[0] = v.x; w[1] = v.y;
+    } else {
+#pragma unroll
+        for (int q = 0; q < BITS; ++q) w[q] = wp[q];
+    }
+    uint32_t a[16];
+    expand_codes<BITS>(a, w);
+    const uint32_t sz_lo = szs[gl * 16 + gq], sz_hi = szs[gl * 16 + gq + 8];
+    const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
+    const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
+    const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        mma_bf16(acc, &a[0], b[nt][0], b[nt][1]);
+        mma_bf16(acc, &a[4], b[nt][2], b[nt][3]);
+        mma_bf16(acc, &a[8], b[nt][4], b[nt][5]);
+        mma_bf16(acc, &a[12], b[nt][6], b[nt][7]);
+        yacc[nt][0] = fmaf(f_lo.x, acc[0], fmaf(nsz_lo, sx[nt][0], yacc[nt][0]));
+        yacc[nt][1] = fmaf(f_lo.x, acc[1], fmaf(nsz_lo, sx[nt][1], yacc[nt][1]));
+        yacc[nt][2] = fmaf(f_hi.x, acc[2], fmaf(nsz_hi, sx[nt][0], yacc[nt][2]));
+        yacc[nt][3] = fmaf(f_hi.x, acc[3], fmaf(nsz_hi, sx[nt][1], yacc[nt][3]));
+    }
+}
+
+// The steps kq, kq + KQ, ... of one stage for tile slot r (KQ = 16 >> RBITS phases): unrolled with
+// constant strides for a full stage, a plain loop for the ragged last one.
+template <int BITS, int NT, int RBITS>
+__device__ __forceinline__ void consume_stage(const TallParams& p, const unsigned char* stage, uint32_t xs_u32, int r,
+                                              int kq, int s, int steps, int lane, float (&yacc)[NT][4]) {
+    constexpr int KQ = kConsumerWarps >> RBITS, PER = kStageSteps / KQ;
+    const unsigned char* codes_rt = stage + r * kStageSteps * (128 * BITS);
+    const uint32_t* szs = reinterpret_cast<const uint32_t*>(stage + p.off_stage_sz + r * kSzTile);
+    const unsigned char* srec = stage + p.off_stage_x + 2048;  // sums of token 0
+    const int g0 = (s * kStageSteps) >> p.gshift;
+    if (steps == kStageSteps) {
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int st = kq + i * KQ;
+            tile_step<BITS, NT>(codes_rt, szs, srec, xs_u32, st, ((s * kStageSteps + st) >> p.gshift) - g0, lane, yacc);
+        }
+    } else {
+        for (int st = kq; st < steps; st += KQ)
+            tile_step<BITS, NT>(codes_rt, szs, srec, xs_u32, st, ((s * kStageSteps + st) >> p.gshift) - g0, lane, yacc);
+    }
+}
+
 template <int BITS, int NT>
 __global__ void __launch_bounds__(kThreads, 1)
 tall_kernel(const TallParams p) {
@@ -226,59 +300,12 @@ tall_kernel(const TallParams p) {
                 if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
             }
             if (active) {
-                const int steps = steps_of(s);
                 const unsigned char* stage = smem + p.off_ring + slot * p.stage_bytes;
-                const uint32_t xs_u32 = smem0 + p.off_ring + slot * p.stage_bytes + p.off_stage_x;
-                const unsigned char* srec = stage + p.off_stage_x + 2048;  // sums of token 0
-                const uint32_t* szs = reinterpret_cast<const uint32_t*>(stage + p.off_stage_sz + r * kSzTile);
-                const int g0 = (s * kStageSteps) >> p.gshift;
-                for (int st = kq; st < steps; st += KQ) {
-                    uint32_t b[NT][8];
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        const uint32_t addr = xs_u32 + (uint32_t)(nt * 8 * kActRecord + st * 128) + ldm_off;
-                        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][0]), addr);
-                        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][4]), addr + 64u);
-                    }
-                    float sx[NT][2];
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        sx[nt][0] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg) * kActRecord)[st];
-                        sx[nt][1] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg + 1) * kActRecord)[st];
-                    }
-                    uint32_t w[BITS];
-                    const uint32_t* wp =
-                        reinterpret_cast<const uint32_t*>(stage + (r * kStageSteps + st) * kStepBytes) + lane * BITS;
-                    if constexpr (BITS == 4) {
-                        const uint4 v = *reinterpret_cast<const uint4*>(wp);
-                        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-                    } else if constexpr (BITS == 2) {
-                        const uint2 v = *reinterpret_cast<const uint2*>(wp);
-                        w[0] = v.x; w[1] = v.y;
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < BITS; ++q) w[q] = wp[q];
-                    }
-                    uint32_t a[16];
-                    expand_codes<BITS>(a, w);
-                    const int gl = ((s * kStageSteps + st) >> p.gshift) - g0;
-                    const uint32_t sz_lo = szs[gl * 16 + gq], sz_hi = szs[gl * 16 + gq + 8];
-                    const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
-                    const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
-                    const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                        mma_bf16(acc, &a[0], b[nt][0], b[nt][1]);
-                        mma_bf16(acc, &a[4], b[nt][2], b[nt][3]);
-                        mma_bf16(acc, &a[8], b[nt][4], b[nt][5]);
-                        mma_bf16(acc, &a[12], b[nt][6], b[nt][7]);
-                        yacc[nt][0] = fmaf(f_lo.x, acc[0], fmaf(nsz_lo, sx[nt][0], yacc[nt][0]));
-                        yacc[nt][1] = fmaf(f_lo.x, acc[1], fmaf(nsz_lo, sx[nt][1], yacc[nt][1]));
-                        yacc[nt][2] = fmaf(f_hi.x, acc[2], fmaf(nsz_hi, sx[nt][0], yacc[nt][2]));
-                        yacc[nt][3] = fmaf(f_hi.x, acc[3], fmaf(nsz_hi, sx[nt][1], yacc[nt][3]));
-                    }
-                }
+                const uint32_t xs_u32 = smem0 + p.off_ring + slot * p.stage_bytes + p.off_stage_x + ldm_off;
+                const int steps = steps_of(s);
+                if (rbits == 2) consume_stage<BITS, NT, 2>(p, stage, xs_u32, r, kq, s, steps, lane, yacc);
+                else if (rbits == 1) consume_stage<BITS, NT, 1>(p, stage, xs_u32, r, kq, s, steps, lane, yacc);
+                else consume_stage<BITS, NT, 0>(p, stage, xs_u32, r, kq, s, steps, lane, yacc);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty(slot));
