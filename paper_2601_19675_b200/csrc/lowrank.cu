@@ -55,36 +55,55 @@ lowrank_down_mma_kernel(const __half* __restrict__ B, const __nv_bfloat16* __res
     const uint32_t a_off = (uint32_t)((warp * 16 + (lane & 7) + 8 * ((lane >> 3) & 1)) * kLrStride + 8 * (lane >> 4)) * 2u;
     const uint32_t b_off = (uint32_t)(((lane & 7) + 8 * (lane >> 4)) * kLrStride + 8 * ((lane >> 3) & 1)) * 2u;
 
+    // global loads of one 64-column chunk, kept in registers while the previous chunk is multiplied
+    constexpr int kXPer = kLrTokens * 8 / kLrThreads;                     // 16-byte pieces of x per thread
+    constexpr int kBPer = (NJ * 8 * 8 + kLrThreads - 1) / kLrThreads;     // 16-byte pieces of B per thread
+    uint4 xr[kXPer], br[kBPer];
+    auto load_chunk = [&](int k0) {
+#pragma unroll
+        for (int u = 0; u < kXPer; ++u) {
+            const int i = tid + u * kLrThreads, r = i >> 3, c = i & 7;
+            xr[u] = tok0 + r < T ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tok0 + r) * ldx + k0) + c)
+                                 : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kBPer; ++u) {
+            const int i = tid + u * kLrThreads, r = i >> 3, c = i & 7;
+            br[u] = (i < NJ * 64 && r < rows_b) ? __ldg(reinterpret_cast<const uint4*>(B + (size_t)(j0 + r) * n + k0) + c)
+                                                : make_uint4(0, 0, 0, 0);
+        }
+    };
+    if (kb < ke) load_chunk(kb);
     for (int k0 = kb; k0 < ke; k0 += kLrChunk) {
-        __syncthreads();
-        // activations: 128 tokens x 64 columns, 16 bytes per thread and step
-        for (int i = tid; i < kLrTokens * 8; i += kLrThreads) {
-            const int r = i >> 3, c = i & 7;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (tok0 + r < T) v = __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tok0 + r) * ldx + k0) + c);
-            *reinterpret_cast<uint4*>(xs + r * kLrStride + c * 8) = v;
+        __syncthreads();  // the previous chunk has been multiplied
+#pragma unroll
+        for (int u = 0; u < kXPer; ++u) {
+            const int i = tid + u * kLrThreads, r = i >> 3, c = i & 7;
+            *reinterpret_cast<uint4*>(xs + r * kLrStride + c * 8) = xr[u];
         }
         // rows of B: fp16 -> (hi, lo) bf16
-        for (int i = tid; i < NJ * 8 * 8; i += kLrThreads) {
-            const int r = i >> 3, c = i & 7;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (r < rows_b) v = __ldg(reinterpret_cast<const uint4*>(B + (size_t)(j0 + r) * n + k0) + c);
-            const __half2* h = reinterpret_cast<const __half2*>(&v);
-            uint4 hi, lo;
-            uint32_t* hp = reinterpret_cast<uint32_t*>(&hi);
-            uint32_t* lp = reinterpret_cast<uint32_t*>(&lo);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 f = __half22float2(h[e]);
-                const __nv_bfloat162 bhi = __floats2bfloat162_rn(f.x, f.y);
-                const float2 fh = __bfloat1622float2(bhi);
-                const __nv_bfloat162 blo = __floats2bfloat162_rn(f.x - fh.x, f.y - fh.y);  // exact remainder
-                hp[e] = *reinterpret_cast<const uint32_t*>(&bhi);
-                lp[e] = *reinterpret_cast<const uint32_t*>(&blo);
+        for (int u = 0; u < kBPer; ++u) {
+            const int i = tid + u * kLrThreads, r = i >> 3, c = i & 7;
+            if (i < NJ * 64) {
+                const __half2* h = reinterpret_cast<const __half2*>(&br[u]);
+                uint4 hi, lo;
+                uint32_t* hp = reinterpret_cast<uint32_t*>(&hi);
+                uint32_t* lp = reinterpret_cast<uint32_t*>(&lo);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __half22float2(h[e]);
+                    const __nv_bfloat162 bhi = __floats2bfloat162_rn(f.x, f.y);
+                    const float2 fh = __bfloat1622float2(bhi);
+                    const __nv_bfloat162 blo = __floats2bfloat162_rn(f.x - fh.x, f.y - fh.y);  // exact remainder
+                    hp[e] = *reinterpret_cast<const uint32_t*>(&bhi);
+                    lp[e] = *reinterpret_cast<const uint32_t*>(&blo);
+                }
+                *reinterpret_cast<uint4*>(bh + r * kLrStride + c * 8) = hi;
+                *reinterpret_cast<uint4*>(bl + r * kLrStride + c * 8) = lo;
             }
-            *reinterpret_cast<uint4*>(bh + r * kLrStride + c * 8) = hi;
-            *reinterpret_cast<uint4*>(bl + r * kLrStride + c * 8) = lo;
         }
+        if (k0 + kLrChunk < ke) load_chunk(k0 + kLrChunk);  // in flight during the products below
         __syncthreads();
 #pragma unroll
         for (int kk = 0; kk < kLrChunk; kk += 16) {
@@ -126,7 +145,7 @@ __global__ void lowrank_finish_kernel(const float* __restrict__ partial, __half*
 int lowrank_mma_slices(const lopro_desc& d, int T) {
     const int tiles = (T + kLrTokens - 1) / kLrTokens;
     int slices = 1;
-    while (slices < 16 && tiles * slices < 128 && d.d_in / (slices * 2) >= 512 && (d.d_in / 64) % (slices * 2) == 0) slices *= 2;
+    while (slices < 32 && tiles * slices < 512 && d.d_in / (slices * 2) >= 256 && (d.d_in / 64) % (slices * 2) == 0) slices *= 2;
     return slices;
 }
 

@@ -18,14 +18,14 @@ constexpr int kRotThreads = 256;
 // butterfly stages stay in registers, the next five go through warp shuffles.  Results are rounded to
 // bf16 once, collected in shared memory and stored with coalesced 16-byte stores.  E = 8 covers
 // b_H <= 256, E = 16 and 32 cover 512 and 1024.
-template <int E, int TOK>
+template <int E, int TOK, bool DIRECT>
 __global__ void __launch_bounds__(kRotThreads)
 rotate_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
               __nv_bfloat16* __restrict__ xrot, int64_t ldo, float* __restrict__ s64, int s64_ld,
               int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int T) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __nv_bfloat16* xin = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [TOK][n]
-    __nv_bfloat16* xout = xin + (size_t)TOK * n;                       // [TOK][n]
+    __nv_bfloat16* xout = xin + (size_t)TOK * n;                       // [TOK][n], staged variant only
     const int t0 = blockIdx.x * TOK;
     const int nt = min(TOK, T - t0);  // live rows of this CTA
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -39,12 +39,46 @@ rotate_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* _
     }
     __syncthreads();
 
-    // identity prefix: permuted only
-    for (int k = tid; k < b_i; k += kRotThreads) {
-        const int pk = __ldg(perm + k);
+    if constexpr (DIRECT) {
+        // identity prefix, b_I a multiple of 64: lane l of a warp gathers eight consecutive columns and stores
+        // them as one 16-byte piece; eight lanes cover one 64-column step and add up its sum
+        const int n8 = b_i >> 3;
+        for (int base = warp * 32; base < n8; base += kWarps * 32) {
+            const int k8 = base + lane;
+            const bool on = k8 < n8;
+            int pk[8];
+            if (on) {
+                const int4 p0 = __ldg(reinterpret_cast<const int4*>(perm + k8 * 8));
+                const int4 p1 = __ldg(reinterpret_cast<const int4*>(perm + k8 * 8 + 4));
+                pk[0] = p0.x; pk[1] = p0.y; pk[2] = p0.z; pk[3] = p0.w;
+                pk[4] = p1.x; pk[5] = p1.y; pk[6] = p1.z; pk[7] = p1.w;
+            }
+            for (int r = 0; r < nt; ++r) {
+                const __nv_bfloat16* row = xin + (size_t)r * n;
+                __nv_bfloat16 o[8];
+                float sum = 0.0f;
 #pragma unroll
-        for (int r = 0; r < TOK; ++r)
-            if (r < nt) xout[(size_t)r * n + k] = xin[(size_t)r * n + pk];
+                for (int e = 0; e < 8; ++e) {
+                    o[e] = on ? row[pk[e]] : __float2bfloat16_rn(0.0f);
+                    sum += __bfloat162float(o[e]);
+                }
+                sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+                if (on) {
+                    *reinterpret_cast<uint4*>(xrot + (size_t)(t0 + r) * ldo + k8 * 8) = *reinterpret_cast<const uint4*>(o);
+                    if (s64 != nullptr && (lane & 7) == 0) s64[(size_t)(t0 + r) * s64_ld + (k8 >> 3)] = sum;
+                }
+            }
+        }
+    } else {
+        // identity prefix: permuted only
+        for (int k = tid; k < b_i; k += kRotThreads) {
+            const int pk = __ldg(perm + k);
+#pragma unroll
+            for (int r = 0; r < TOK; ++r)
+                if (r < nt) xout[(size_t)r * n + k] = xin[(size_t)r * n + pk];
+        }
     }
 
     const int nrot = n - b_i;
@@ -85,11 +119,33 @@ rotate_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* _
                     }
                 }
             }
+            if constexpr (DIRECT) {
+                // rounded results leave from registers: 16-byte stores, contiguous across the warp; the lanes of a
+                // 64-column step add up its sum
+                __nv_bfloat16 o[E];
+                float sum = 0.0f;
 #pragma unroll
-            for (int e = 0; e < E; ++e)
-                if (rel + e < nrot) xout[(size_t)r * n + b_i + rel + e] = __float2bfloat16_rn(v[e] * inv_sqrt_bh);
+                for (int e = 0; e < E; ++e) {
+                    o[e] = __float2bfloat16_rn(v[e] * inv_sqrt_bh);
+                    sum += __bfloat162float(o[e]);
+                }
+#pragma unroll
+                for (int d = 1; d < 64 / E; d <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+                if (rel < nrot) {
+                    uint4* dst = reinterpret_cast<uint4*>(xrot + (size_t)(t0 + r) * ldo + b_i + rel);
+#pragma unroll
+                    for (int q = 0; q < E / 8; ++q) dst[q] = reinterpret_cast<const uint4*>(o)[q];
+                    if (s64 != nullptr && (lane & (64 / E - 1)) == 0)
+                        s64[(size_t)(t0 + r) * s64_ld + ((b_i + rel) >> 6)] = sum;
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    if (rel + e < nrot) xout[(size_t)r * n + b_i + rel + e] = __float2bfloat16_rn(v[e] * inv_sqrt_bh);
+            }
         }
     }
+    if constexpr (DIRECT) return;
     __syncthreads();
 
     for (int r = 0; r < nt; ++r) {
@@ -315,27 +371,32 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
     }
 }
 
-template <int E, int TOK>
-cudaError_t launch_rotate_et(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
-                             __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s) {
-    const size_t smem = (size_t)d.d_in * 4 * TOK;
+template <int E, int TOK, bool DIRECT>
+cudaError_t launch_rotate_etd(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
+                              __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s) {
+    const size_t smem = (size_t)d.d_in * (DIRECT ? 2 : 4) * TOK;
     static unsigned long long attr_done = 0;
-    cudaError_t e = ensure_dynamic_smem(rotate_kernel<E, TOK>, TOK == 1 ? 32768 * 4 : 160 * 1024, &attr_done);
+    cudaError_t e = ensure_dynamic_smem(rotate_kernel<E, TOK, DIRECT>, TOK == 1 ? 32768 * 4 : 160 * 1024, &attr_done);
     if (e != cudaSuccess) return e;
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
-    rotate_kernel<E, TOK><<<(T + TOK - 1) / TOK, kRotThreads, smem, s>>>(x, ldx, perm, xrot, ldo, s64, s64_stride(d.d_in),
-                                                                       status, d.d_in, d.identity_cols, d.block_size,
-                                                                       inv, T);
+    rotate_kernel<E, TOK, DIRECT><<<(T + TOK - 1) / TOK, kRotThreads, smem, s>>>(
+        x, ldx, perm, xrot, ldo, s64, s64_stride(d.d_in), status, d.d_in, d.identity_cols, d.block_size, inv, T);
     return cudaGetLastError();
 }
 
+// Results go straight from registers to global memory when the identity prefix ends on a 64-column step
+// (16-byte stores and whole steps per lane group); otherwise they are collected in shared memory first.
 // Four rows per CTA when there are many tokens and the rows fit shared memory, else one.
 template <int E>
 cudaError_t launch_rotate_e(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
                             __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s) {
-    if (T >= 256 && (size_t)d.d_in * 16 <= 160 * 1024)
-        return launch_rotate_et<E, 4>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
-    return launch_rotate_et<E, 1>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
+    const bool direct = d.identity_cols % 64 == 0;
+    const bool four = T >= 256 && (size_t)d.d_in * (direct ? 8 : 16) <= 160 * 1024;
+    if (direct)
+        return four ? launch_rotate_etd<E, 4, true>(d, perm, x, ldx, xrot, ldo, s64, status, T, s)
+                    : launch_rotate_etd<E, 1, true>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
+    return four ? launch_rotate_etd<E, 4, false>(d, perm, x, ldx, xrot, ldo, s64, status, T, s)
+                : launch_rotate_etd<E, 1, false>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
 }
 
 }  // namespace
