@@ -1,12 +1,15 @@
 // Prefill forward (T > 32): y = W^ x~ + A t as one tensor-core GEMM on tcgen05 / TMEM
 // (steps "Dequant(W_q) X" and "U (Sigma Y)" of Appendix A.3, summed as in Eq. 8).
 //
-// CTA tile: 128 weight rows (the M side of the MMA, one TMEM lane per row) x N tokens (N = 64, 128
-// or 256 TMEM columns, fp32) x 64 columns of K per pipeline stage.
-//   * warps 0-15 (dequant): two per 16-row tile of the fragment layout; per stage each reads the tile's
-//     packed codes from global memory (a register ring a few stages ahead), turns them into
-//     bf16(s (c - z)) -- fp32 arithmetic, one rounding -- and writes them into the stage's A tile in
-//     the K-major 128-byte-swizzled layout the MMA reads;
+// CTA tile: one or two blocks of 128 weight rows (the M side of the MMA, one TMEM lane per row, one
+// accumulator per block) x N tokens (N = 64, 128 or 256 TMEM columns, fp32) x 64 columns of K per
+// pipeline stage.  Two row blocks share every activation tile, which halves the traffic of the
+// activation operand from L2 (each CTA streams all K columns of its tokens).
+//   * warps 0-15 (dequant): one per 16-row tile of the fragment layout (with a single row block: two
+//     per tile, taking turns by pairs of stages);
+//     each reads the tile's packed codes from global memory (registers, two visits ahead), turns them
+//     into bf16(s (c - z)) -- fp32 arithmetic, one rounding -- and writes them into the stages' A tiles
+//     in the K-major 128-byte-swizzled layout the MMA reads;
 //   * warp 16 (loader): one thread brings the stage's tile of rotated activations (B operand) with a
 //     tiled TMA copy, and for the low-rank stages the tiles of A (fp16) and t (fp16);
 //   * warp 17 (MMA): one thread issues four tcgen05.mma (K = 16 each) per stage into the TMEM
@@ -31,13 +34,14 @@ constexpr int kThreads = (kDequantWarps + 4) * 32;
 constexpr int kTileM = 128;      // weight rows per CTA
 constexpr int kMaxTileN = 256;   // tokens per CTA
 constexpr int kStageK = 64;      // K columns per stage = 128 bytes of bf16 = one swizzle atom
-constexpr int kAStages = 4;      // ring of weight tiles (16 KB each)
-constexpr int kBStages = 2;      // ring of activation tiles (one or two accumulators' worth, 64 KB each)
-constexpr int kABytes = kTileM * 128;           // 16 KB
-constexpr int kBBytes = 2 * kMaxTileN * 128;    // 64 KB: two 256-token tiles
+constexpr int kAStages = 4;      // ring of weight tiles (two row blocks of 16 KB each)
+constexpr int kBStages = 3;      // ring of activation tiles (32 KB each)
+constexpr int kABlock = kTileM * 128;           // 16 KB: one row block of one stage
+constexpr int kABytes = 2 * kABlock;            // 32 KB
+constexpr int kBBytes = kMaxTileN * 128;        // 32 KB: one 256-token tile
+constexpr double kPairCost = 1.25;  // duration of a two-block CTA relative to a one-block CTA (scheduling estimate)
 constexpr int kSmemBytes = kAStages * kABytes + kBStages * kBBytes + 1024;  // + slack for 1024-byte alignment
 constexpr uint32_t kSpinLimit = 1u << 24;
-constexpr int kCodeRing = 4;  // stages of packed codes held in registers ahead of use
 
 struct PrefillParams {
     const uint32_t* codes;
@@ -46,10 +50,11 @@ struct PrefillParams {
     void* y;
     int64_t ldy;
     int out_f32;
+    int y_vec;       // bf16 output whose rows allow 16-byte stores (y 16-byte aligned, ldy a multiple of 8)
     int m, n, T;
     int nsteps, gshift, ng, r_pad;
     int tile_n;      // tokens per accumulator: 64, 128 or 256
-    int pair_tiles;  // CTAs along y that own two accumulators (2 * tile_n tokens); the others own one
+    int pair_tiles;  // CTAs along x that own two row blocks (256 rows, two accumulators); the others own one
     int lr_stages;   // ceil(r_pad / 64)
 };
 
@@ -113,19 +118,29 @@ __device__ __forceinline__ uint32_t make_idesc(int tile_n, uint32_t fmt) {
 }
 
 constexpr uint32_t kMagic128 = 0x43004300u;
+// (a & mask) | magic in one logic instruction, both constants in registers
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t mask, uint32_t magic) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(magic));
+    return d;
+}
 template <int BITS>
 __device__ __forceinline__ void expand_codes(uint32_t (&a)[16], const uint32_t (&w)[BITS]) {
+    const uint32_t magic = kMagic128;
     if constexpr (BITS == 4) {
+        const uint32_t mask = 0x000F000Fu;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = ((w[j] >> (4 * rho)) & 0x000F000Fu) | kMagic128;
+            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = and_or(w[j] >> (4 * rho), mask, magic);
     } else if constexpr (BITS == 2) {
+        const uint32_t mask = 0x00030003u;
 #pragma unroll
-        for (int pi = 0; pi < 16; ++pi) a[pi] = ((w[pi >> 3] >> (2 * (pi & 7))) & 0x00030003u) | kMagic128;
+        for (int pi = 0; pi < 16; ++pi) a[pi] = and_or(w[pi >> 3] >> (2 * (pi & 7)), mask, magic);
     } else {
+        const uint32_t mask = 0x00070007u;
 #pragma unroll
-        for (int pi = 0; pi < 15; ++pi) a[pi] = ((w[pi / 5] >> (3 * (pi % 5))) & 0x00070007u) | kMagic128;
+        for (int pi = 0; pi < 15; ++pi) a[pi] = and_or(w[pi / 5] >> (3 * (pi % 5)), mask, magic);
         a[15] = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u) | kMagic128;
     }
 }
@@ -141,11 +156,10 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     __shared__ int s_timeout;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int tile_m = blockIdx.x, tile_t = blockIdx.y;
-    // token tiles: the first p.pair_tiles CTAs along y own two accumulators (2 * tile_n tokens), the rest one
-    const int n_acc = tile_t < p.pair_tiles ? 2 : 1;
-    const int row_base = tile_m * kTileM;
-    const int tok_base = tile_t < p.pair_tiles ? tile_t * 2 * p.tile_n : (p.pair_tiles + tile_t) * p.tile_n;
+    // row tiles: the first p.pair_tiles CTAs along x own two blocks of 128 rows (two accumulators), the rest one
+    const int n_acc = (int)blockIdx.x < p.pair_tiles ? 2 : 1;
+    const int row_base = ((int)blockIdx.x < p.pair_tiles ? (int)blockIdx.x * 2 : p.pair_tiles + (int)blockIdx.x) * kTileM;
+    const int tok_base = (int)blockIdx.y * p.tile_n;
     const int total = p.nsteps + p.lr_stages;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
@@ -170,7 +184,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
 
     if (tid == 0) {
         for (int s = 0; s < kAStages; ++s) {
-            mbar_init(full_a(s), kDequantWarps + 1);  // every dequant warp and the loader
+            mbar_init(full_a(s), (n_acc == 2 ? kDequantWarps : kDequantWarps / 2) + 1);  // the slot's dequant warps and the loader
             mbar_init(empty_a(s), 1);
         }
         for (int s = 0; s < kBStages; ++s) {
@@ -194,42 +208,49 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
 
     if (warp < kDequantWarps) {
         // ---------------- dequant warps: fill the A tile of every weight stage ----------------
+        // A visit converts two consecutive stages of one 16-row tile (2 x 64 columns, 32 register pairs per
+        // lane) between one pair of waits and one proxy fence.  Two row blocks: warp w owns tile w and visits
+        // every pair of stages.  One row block: warps w and w + 8 share tile w, group g = w >> 3 takes the
+        // stages 4 v + 2 g and 4 v + 2 g + 1, so the two groups work on different stages at the same time.
+        static_assert(kAStages == 4, "the visit schedule assumes four weight slots");
         const int gq = lane >> 2, tg = lane & 3;
-        const int rt = tile_m * (kTileM / 16) + (warp & 7);
+        const int g = n_acc == 2 ? 0 : warp >> 3;
+        const int vstride = n_acc == 2 ? 2 : 4;  // stages between the visits of this warp
+        const int rt = row_base / 16 + (n_acc == 2 ? warp : (warp & 7));
         const bool valid = rt * 16 < p.m;
-        uint32_t wbuf[kCodeRing][BITS];
-        uint32_t szbuf[kCodeRing][2];
+        uint32_t wbuf[2][2][BITS];
+        uint32_t szbuf[2][2][2];
         const uint32_t* wbase = p.codes + ((size_t)rt * p.nsteps * 32 + lane) * BITS;
         const uint32_t* szbase = p.sz + (size_t)rt * p.ng * 16 + gq;
-        auto issue = [&](int slot, int s) {
+        auto load_visit = [&](int buf, int v) {
 #pragma unroll
-            for (int q = 0; q < BITS; ++q) wbuf[slot][q] = __ldg(wbase + (size_t)s * 32 * BITS + q);
-            const uint32_t* z = szbase + (size_t)(s >> p.gshift) * 16;
-            szbuf[slot][0] = __ldg(z);
-            szbuf[slot][1] = __ldg(z + 8);
+            for (int j = 0; j < 2; ++j) {
+                const int s = vstride * v + 2 * g + j;
+                if (valid && s < p.nsteps) {
+#pragma unroll
+                    for (int q = 0; q < BITS; ++q) wbuf[buf][j][q] = __ldg(wbase + (size_t)s * 32 * BITS + q);
+                    const uint32_t* z = szbase + (size_t)(s >> p.gshift) * 16;
+                    szbuf[buf][j][0] = __ldg(z);
+                    szbuf[buf][j][1] = __ldg(z + 8);
+                }
+            }
         };
-        if (valid) {
-#pragma unroll
-            for (int i = 0; i < kCodeRing; ++i)
-                if (i < p.nsteps) issue(i, i);
-        }
+        load_visit(0, 0);
+        load_visit(1, 1);
         // byte offset of this lane's 4-byte slot in 16-byte chunk c of its row (row & 7 == gq, 128-byte swizzle)
         uint32_t off[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) off[c] = (uint32_t)(((warp & 7) * 16 + gq) * 128 + ((c ^ gq) << 4) + tg * 4);
-        // the warp converts eight of the tile's sixteen register pairs: HALF = 0 -> columns 0..31, 1 -> 32..63
-        auto convert = [&](auto half_tag, const uint32_t (&w)[BITS], uint32_t sz_lo, uint32_t sz_hi, unsigned char* a_tile) {
-            constexpr int HALF = decltype(half_tag)::value;
+        // all sixteen register pairs of the tile and stage: 64 columns of rows gq and gq + 8
+        auto convert = [&](const uint32_t (&w)[BITS], uint32_t sz_lo, uint32_t sz_hi, unsigned char* a_tile) {
             uint32_t a[16];
-            expand_codes<BITS>(a, w);  // pairs of the other half are dead code after unrolling
+            expand_codes<BITS>(a, w);
             const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
             const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
             const float sc[2] = {f_lo.x, f_hi.x};
             const float zs[2] = {128.0f + f_lo.y, 128.0f + f_hi.y};  // exact in fp32
 #pragma unroll
-            for (int pp = 0; pp < 8; ++pp) {
-                constexpr int kBase = HALF * 8;
-                const int pi = kBase + pp;
+            for (int pi = 0; pi < 16; ++pi) {
                 const int j = pi >> 2, rho = pi & 3, hi8 = rho & 1;
                 const uint32_t av = a[pi];
                 const float lo_f = __uint_as_float(av << 16), hi_f = __uint_as_float(av & 0xFFFF0000u);
@@ -238,34 +259,38 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                 *reinterpret_cast<__nv_bfloat162*>(a_tile + off[2 * j + (rho >> 1)] + hi8 * 1024) = wv;
             }
         };
-        const bool upper = (warp >> 3) != 0;
-        for (int s0 = 0; s0 < total; s0 += kCodeRing) {
+        unsigned char* const blk_ptr = base_ptr + (n_acc == 2 ? (warp >> 3) * kABlock : 0);
+        const int n_visits = total > 2 * g ? (total - 2 * g + vstride - 1) / vstride : 0;
+        for (int v0 = 0; v0 < n_visits; v0 += 2) {
 #pragma unroll
-            for (int i = 0; i < kCodeRing; ++i) {
-                const int s = s0 + i;
-                if (s < total) {
-                    const int slot = s % kAStages;
-                    if (s >= kAStages) warp_wait(empty_a(slot), (uint32_t)((s / kAStages) - 1) & 1u);
-                    if (s < p.nsteps && valid) {
-                        uint32_t w[BITS];
+            for (int u = 0; u < 2; ++u) {  // u = register buffer of the visit
+                const int v = v0 + u;
+                if (v < n_visits) {
 #pragma unroll
-                        for (int q = 0; q < BITS; ++q) w[q] = wbuf[i][q];
-                        const uint32_t sz_lo = szbuf[i][0], sz_hi = szbuf[i][1];
-                        if (s + kCodeRing < p.nsteps) issue(i, s + kCodeRing);
-                        unsigned char* a_tile = base_ptr + slot * kABytes;
-                        if (upper) convert(std::integral_constant<int, 1>{}, w, sz_lo, sz_hi, a_tile);
-                        else convert(std::integral_constant<int, 0>{}, w, sz_lo, sz_hi, a_tile);
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
+                    for (int j = 0; j < 2; ++j) {
+                        const int s = vstride * v + 2 * g + j;
+                        if (s < total) {
+                            const int slot = s & 3, use = s >> 2;
+                            if (use >= 1) warp_wait(empty_a(slot), (uint32_t)(use - 1) & 1u);
+                            if (valid && s < p.nsteps)
+                                convert(wbuf[u][j], szbuf[u][j][0], szbuf[u][j][1], blk_ptr + slot * kABytes);
+                        }
                     }
+                    load_visit(u, v + 2);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(full_a(slot));
+                    if (lane == 0) {
+                        const int s0 = vstride * v + 2 * g;
+                        mbar_arrive(full_a(s0 & 3));
+                        if (s0 + 1 < total) mbar_arrive(full_a((s0 + 1) & 3));
+                    }
                 }
             }
         }
     } else if (warp == kDequantWarps) {
         // ---------------- loader: activation tiles, and the fp16 tiles of the low-rank stages ----------------
         if (lane == 0) {
-            const uint32_t b_bytes = (uint32_t)(n_acc * p.tile_n * 128);
+            const uint32_t b_bytes = (uint32_t)(p.tile_n * 128);
             for (int s = 0; s < total; ++s) {
                 const int sa = s % kAStages, sb = s % kBStages;
                 if (s >= kAStages && !s_timeout && !mbar_wait(empty_a(sa), (uint32_t)((s / kAStages) - 1) & 1u)) time_out();
@@ -273,15 +298,14 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                 const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
                 mbar_expect_tx(full_b(sb), b_bytes);
                 if (s < p.nsteps) {
-                    for (int acc = 0; acc < n_acc; ++acc)
-                        tma_load_2d(b_tile + acc * (kBBytes / 2), &map_x, s * kStageK, tok_base + acc * p.tile_n, full_b(sb));
+                    tma_load_2d(b_tile, &map_x, s * kStageK, tok_base, full_b(sb));
                     mbar_arrive(full_a(sa));
                 } else {
                     const int lr = s - p.nsteps;
+                    tma_load_2d(b_tile, &map_t, lr * kStageK, tok_base, full_b(sb));
+                    mbar_expect_tx(full_a(sa), (uint32_t)(n_acc * kABlock));
                     for (int acc = 0; acc < n_acc; ++acc)
-                        tma_load_2d(b_tile + acc * (kBBytes / 2), &map_t, lr * kStageK, tok_base + acc * p.tile_n, full_b(sb));
-                    mbar_expect_tx(full_a(sa), (uint32_t)kABytes);
-                    tma_load_2d(a_tile, &map_a, lr * kStageK, row_base, full_a(sa));
+                        tma_load_2d(a_tile + acc * kABlock, &map_a, lr * kStageK, row_base + acc * kTileM, full_a(sa));
                 }
             }
         }
@@ -296,11 +320,11 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                     time_out();
                 tc_fence_after();
                 const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
-                const uint64_t da = make_desc_sw128(a_tile);
+                const uint64_t db = make_desc_sw128(b_tile);
                 const bool lowrank = s >= p.nsteps;
                 const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
                 for (int acc = 0; acc < n_acc; ++acc) {
-                    const uint64_t db = make_desc_sw128(b_tile + acc * (kBBytes / 2));
+                    const uint64_t da = make_desc_sw128(a_tile + acc * kABlock);
                     for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
                         umma_f16(tmem + (uint32_t)(acc * 256), da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
                                  lowrank ? idesc_lr : idesc_w, (s > 0 || k > 0) ? 1u : 0u);
@@ -319,8 +343,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
         __syncwarp();
         tc_fence_after();
         const int lane_base = (warp & 3) * 32;  // a warp may read the 32 TMEM lanes of its quarter
-        const int row = row_base + lane_base + lane;
         for (int acc = 0; acc < n_acc; ++acc) {
+            const int row = row_base + acc * kTileM + lane_base + lane;
             for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
                 uint32_t v[32];
                 const uint32_t taddr = tmem + ((uint32_t)lane_base << 16) + (uint32_t)(acc * 256 + c0);
@@ -334,10 +358,26 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                     : "r"(taddr)
                     : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row < p.m) {
+                if (p.y_vec) {
+                    // bf16 rows of 32 tokens meet in shared memory (the rings are idle now), [token][32 rows], and
+                    // leave as 16-byte pieces of eight consecutive rows
+                    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(base_ptr + (warp - kDequantWarps) * 2048);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) stg[i * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int piece = q * 32 + lane, ti = piece >> 2, r8 = (piece & 3) * 8;
+                        const int tok = tok_base + c0 + ti, prow = row_base + acc * kTileM + lane_base + r8;
+                        if (tok < p.T && prow < p.m)
+                            *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.y) + (size_t)tok * p.ldy + prow) =
+                                *reinterpret_cast<const uint4*>(stg + ti * 32 + r8);
+                    }
+                } else if (row < p.m) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        const int tok = tok_base + acc * p.tile_n + c0 + i;
+                        const int tok = tok_base + c0 + i;
                         if (tok < p.T) {
                             const size_t o = (size_t)tok * p.ldy + row;
                             if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = __uint_as_float(v[i]);
@@ -417,6 +457,7 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     p.y = y;
     p.ldy = ldy;
     p.out_f32 = out_dtype == LOPRO_OUT_F32;
+    p.y_vec = !p.out_f32 && (ldy % 8) == 0 && (reinterpret_cast<uintptr_t>(y) % 16) == 0 && (d.d_out % 8) == 0;
     p.m = d.d_out;
     p.n = d.d_in;
     p.T = T;
@@ -439,18 +480,17 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
             !make_map(&mt, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ws + W.off_t, (uint64_t)p.r_pad, (uint64_t)T, (uint32_t)p.tile_n))
             return cudaErrorInvalidValue;
     }
-    // Token tiling: U units of tile_n tokens per row tile.  A CTA with two accumulators dequantizes its
-    // weights once for two units (cost ~1.5 per stage against 1.0 for a single unit) but coarser tiles
-    // waste more of the last wave; pick the number of pair tiles that minimises the makespan of a greedy
-    // schedule over the 148 SMs (pairs are dispatched first, then singles).
+    // Row tiling: R blocks of 128 rows.  A CTA with two blocks streams its activations once for both (the
+    // kernel is bound by that stream, so it costs little more than a CTA with one block), but coarser
+    // tiles waste more of the last wave; pick the number of two-block CTAs that minimises the makespan of a
+    // greedy schedule over the SMs (two-block CTAs are dispatched first, then the single blocks).
     const int units = (T + p.tile_n - 1) / p.tile_n;
     const int m_tiles = (d.d_out + kTileM - 1) / kTileM;
-    int best_pairs = units / 2;
+    int best_pairs = m_tiles / 2;
     if ((long long)m_tiles * units <= 20000) {
-        // list scheduling of the tiles (pairs first, dispatch order = block order) on 148 SMs
         double best_cost = 1e30;
-        for (int pairs = units / 2; pairs >= 0; --pairs) {
-            const int singles = units - 2 * pairs;
+        for (int pairs = m_tiles / 2; pairs >= 0; --pairs) {
+            const int singles = m_tiles - 2 * pairs;
             double finish[148];
             for (int i = 0; i < 148; ++i) finish[i] = 0.0;
             auto place = [&](long long count, double dur) {
@@ -461,8 +501,8 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
                     finish[best] += dur;
                 }
             };
-            place((long long)m_tiles * pairs, 1.5);
-            place((long long)m_tiles * singles, 1.0);
+            place((long long)pairs * units, kPairCost);
+            place((long long)singles * units, 1.0);
             double cost = 0.0;
             for (int i = 0; i < 148; ++i) cost = finish[i] > cost ? finish[i] : cost;
             if (cost < best_cost - 1e-9) {
@@ -477,10 +517,10 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
             const char* e = getenv("LOPRO_PREFILL_PAIRS");
             forced = e ? atoi(e) : -1;
         }
-        if (forced >= 0 && forced <= units / 2) best_pairs = forced;
+        if (forced >= 0 && forced <= m_tiles / 2) best_pairs = forced;
     }
     p.pair_tiles = best_pairs;
-    dim3 grid(m_tiles, best_pairs + (units - 2 * best_pairs));
+    dim3 grid(best_pairs + (m_tiles - 2 * best_pairs), units);
     if (grid.y > 65535) return cudaErrorInvalidValue;
     switch (d.bits) {
         case 2: return launch_prefill_bits<2>(p, mx, ma, mt, grid, s);
