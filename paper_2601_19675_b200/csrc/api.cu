@@ -208,7 +208,9 @@ int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launch
         path = use_tall(*desc, T) ? LOPRO_PATH_TALL : LOPRO_PATH_STREAM;
         n = 2;
     } else {
-        const int pre = 1 + (desc->rank > 0 ? (T > kDecodeMaxT ? 2 : 1) : 0);
+        const int pre = (T > kDecodeMaxT && rotate_lowrank_supported(*desc, T))
+                            ? 2
+                            : 1 + (desc->rank > 0 ? (T > kDecodeMaxT ? 2 : 1) : 0);
         path = prefill_supported(*desc, T) ? LOPRO_PATH_PREFILL : LOPRO_PATH_GENERAL;
         n = pre + 1;
     }
@@ -254,6 +256,12 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
         if (e != cudaSuccess) return LOPRO_ERR_CUDA;
         return LOPRO_OK;
     }
+    if (T > kDecodeMaxT && rotate_lowrank_supported(*desc, T)) {
+        // many tokens: rotation and B x side by side in one grid, then the sum over K slices
+        if (launch_rotate_lowrank(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, xrot, desc->d_in, s64, status, B, L.r_pad,
+                                  (float*)(ws + W.off_lrpart), (__half*)(ws + W.off_t), T, s) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
+    } else {
     if (launch_rotate(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, xrot, desc->d_in, s64, status, T, s) !=
         cudaSuccess)
         return LOPRO_ERR_CUDA;
@@ -264,6 +272,7 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
                             : launch_lowrank_down(*desc, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx,
                                                   (__half*)(ws + W.off_t), T, s);
         if (e != cudaSuccess) return LOPRO_ERR_CUDA;
+    }
     }
     if (prefill_supported(*desc, T)) {
         if (launch_prefill(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;

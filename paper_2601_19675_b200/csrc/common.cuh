@@ -123,6 +123,11 @@ cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayo
 size_t lowrank_mma_scratch_bytes(const lopro_desc& d, int T);
 cudaError_t launch_lowrank_down_mma(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x, int64_t ldx,
                                     float* partial, __half* t, int T, cudaStream_t s);
+// Rotation and t = B x of a many-token forward in one grid (plus the dependent launch that adds the K slices).
+bool rotate_lowrank_supported(const lopro_desc& d, int T);
+cudaError_t launch_rotate_lowrank(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
+                                  __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, const __half* B, int r_pad,
+                                  float* partial, __half* t, int T, cudaStream_t s);
 // Prefill forward (T > 32) on tcgen05 / TMEM, after launch_rotate and launch_lowrank_down.
 bool prefill_supported(const lopro_desc& d, int T);
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,

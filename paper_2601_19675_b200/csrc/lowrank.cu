@@ -5,7 +5,10 @@
 // multiplied with x by mma.sync with fp32 accumulation.  Grid: (128-token tiles, K slices); every
 // CTA writes the fp32 partial sums of its K slice, a second small kernel adds the slices in order
 // and rounds once to fp16.
+#include <math.h>
+
 #include "common.cuh"
+#include "rotate_body.cuh"
 
 namespace lopro {
 
@@ -31,16 +34,16 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
 
 // NJ = 8-wide column tiles of the output handled per CTA (rows of B / 8)
 template <int NJ>
-__global__ void __launch_bounds__(kLrThreads)
-lowrank_down_mma_kernel(const __half* __restrict__ B, const __nv_bfloat16* __restrict__ x, int64_t ldx,
-                        float* __restrict__ partial, int n, int r_pad, int T, int j0, int slice_cols) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ __forceinline__ void lowrank_body(unsigned char* smem_raw, int bx, int by, const __half* __restrict__ B,
+                                             const __nv_bfloat16* __restrict__ x, int64_t ldx,
+                                             float* __restrict__ partial, int n, int r_pad, int T, int j0,
+                                             int slice_cols) {
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);   // [128][kLrStride]
     __nv_bfloat16* bh = xs + kLrTokens * kLrStride;                    // [NJ*8][kLrStride]
     __nv_bfloat16* bl = bh + NJ * 8 * kLrStride;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int tok0 = blockIdx.x * kLrTokens;
-    const int kb = blockIdx.y * slice_cols, ke = min(n, kb + slice_cols);
+    const int tok0 = bx * kLrTokens;
+    const int kb = by * slice_cols, ke = min(n, kb + slice_cols);
     const int rows_b = min(NJ * 8, r_pad - j0);
 
     float acc[NJ][4];
@@ -128,11 +131,44 @@ lowrank_down_mma_kernel(const __half* __restrict__ B, const __nv_bfloat16* __res
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int tok = tok0 + warp * 16 + gq + 8 * (i >> 1), col = j0 + j * 8 + 2 * tg + (i & 1);
-            if (tok < T && col < r_pad) partial[((size_t)blockIdx.y * T + tok) * r_pad + col] = acc[j][i];
+            if (tok < T && col < r_pad) partial[((size_t)by * T + tok) * r_pad + col] = acc[j][i];
         }
 }
 
+template <int NJ>
+__global__ void __launch_bounds__(kLrThreads)
+lowrank_down_mma_kernel(const __half* __restrict__ B, const __nv_bfloat16* __restrict__ x, int64_t ldx,
+                        float* __restrict__ partial, int n, int r_pad, int T, int j0, int slice_cols) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    lowrank_body<NJ>(smem_raw, (int)blockIdx.x, (int)blockIdx.y, B, x, ldx, partial, n, r_pad, T, j0, slice_cols);
+}
+
+// Rotation and low-rank down-projection of a many-token forward in ONE grid: the two read the same activations
+// and do not depend on each other, so their CTAs run side by side (blocks [0, n_rot) rotate four token rows each,
+// the rest are the (token tile, K slice) CTAs of the down-projection).  Launched with programmatic stream
+// serialization: the dependents may be scheduled at once, the activations are read after the wait.
+template <int NJ>
+__global__ void __launch_bounds__(kLrThreads)
+rotate_lowrank_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
+                      __nv_bfloat16* __restrict__ xrot, int64_t ldo, float* __restrict__ s64, int s64_ld,
+                      int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int T, int n_rot,
+                      const __half* __restrict__ B, float* __restrict__ partial, int r_pad, int lr_gx, int slice_cols) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if ((int)blockIdx.x < n_rot) {
+        rotate_body<8, 4, true>(smem_raw, (int)blockIdx.x, x, ldx, perm, xrot, ldo, s64, s64_ld, status, n, b_i, b_h,
+                                inv_sqrt_bh, T);
+    } else {
+        const int b = (int)blockIdx.x - n_rot;
+        lowrank_body<NJ>(smem_raw, b % lr_gx, b / lr_gx, B, x, ldx, partial, n, r_pad, T, 0, slice_cols);
+    }
+}
+
+// Adds the K slices in order and rounds once to fp16.  Safe under a programmatic launch: waits for the producer.
 __global__ void lowrank_finish_kernel(const float* __restrict__ partial, __half* __restrict__ t, size_t count, int slices) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= count) return;
     float s = 0.0f;
@@ -185,6 +221,66 @@ cudaError_t launch_lowrank_down_mma(const lopro_desc& d, const __half* B, int r_
     const size_t count = (size_t)T * r_pad;
     lowrank_finish_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(partial, t, count, slices);
     return cudaGetLastError();
+}
+
+namespace {
+
+template <int NJ>
+cudaError_t launch_rotate_lowrank_nj(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
+                                     __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, const __half* B, int r_pad,
+                                     float* partial, int T, cudaStream_t s) {
+    const int slices = lowrank_mma_slices(d, T);
+    const int slice_cols = d.d_in / slices;
+    const int n_rot = (T + 3) / 4, lr_gx = (T + kLrTokens - 1) / kLrTokens;
+    const size_t smem_rot = (size_t)d.d_in * 8, smem_lr = (size_t)(kLrTokens + 2 * NJ * 8) * kLrStride * 2;
+    const size_t smem = smem_rot > smem_lr ? smem_rot : smem_lr;
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(rotate_lowrank_kernel<NJ>, 160 * 1024, &attr_done);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(n_rot + lr_gx * slices));
+    cfg.blockDim = dim3(kLrThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const float inv = (float)(1.0 / sqrt((double)d.block_size));
+    return cudaLaunchKernelEx(&cfg, rotate_lowrank_kernel<NJ>, x, ldx, perm, xrot, ldo, s64, s64_stride(d.d_in), status,
+                              d.d_in, d.identity_cols, d.block_size, inv, T, n_rot, B, partial, r_pad, lr_gx, slice_cols);
+}
+
+}  // namespace
+
+bool rotate_lowrank_supported(const lopro_desc& d, int T) {
+    const int r_pad = round_up_int(d.rank, 16);
+    return d.rank > 0 && r_pad <= kLrMaxRank && T >= 256 && d.block_size <= 256 && d.identity_cols % 64 == 0 &&
+           (size_t)d.d_in * 8 <= 160 * 1024;
+}
+
+cudaError_t launch_rotate_lowrank(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
+                                  __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, const __half* B, int r_pad,
+                                  float* partial, __half* t, int T, cudaStream_t s) {
+    cudaError_t e;
+    if (r_pad > 64) e = launch_rotate_lowrank_nj<16>(d, perm, x, ldx, xrot, ldo, s64, status, B, r_pad, partial, T, s);
+    else if (r_pad > 32) e = launch_rotate_lowrank_nj<8>(d, perm, x, ldx, xrot, ldo, s64, status, B, r_pad, partial, T, s);
+    else if (r_pad > 16) e = launch_rotate_lowrank_nj<4>(d, perm, x, ldx, xrot, ldo, s64, status, B, r_pad, partial, T, s);
+    else e = launch_rotate_lowrank_nj<2>(d, perm, x, ldx, xrot, ldo, s64, status, B, r_pad, partial, T, s);
+    if (e != cudaSuccess) return e;
+    // the K slices are added by a dependent launch that waits for the grid above
+    const size_t count = (size_t)T * r_pad;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((count + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, lowrank_finish_kernel, (const float*)partial, t, count, lowrank_mma_slices(d, T));
 }
 
 }  // namespace lopro

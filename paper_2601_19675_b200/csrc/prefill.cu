@@ -290,6 +290,9 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     } else if (warp == kDequantWarps) {
         // ---------------- loader: activation tiles, and the fp16 tiles of the low-rank stages ----------------
         if (lane == 0) {
+            // under a programmatic launch the rotated activations and t of the preceding kernels are complete
+            // only after this wait; the dequant warps start on the layer's own data right away
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             const uint32_t b_bytes = (uint32_t)(p.tile_n * 128);
             for (int s = 0; s < total; ++s) {
                 const int sa = s % kAStages, sb = s % kBStages;
@@ -433,8 +436,17 @@ cudaError_t launch_prefill_bits(const PrefillParams& p, const CUtensorMap& mx, c
     static unsigned long long attr_done = 0;
     cudaError_t e = ensure_dynamic_smem(prefill_kernel<BITS>, kSmemBytes, &attr_done);
     if (e != cudaSuccess) return e;
-    prefill_kernel<BITS><<<grid, kThreads, kSmemBytes, s>>>(p, mx, ma, mt);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_kernel<BITS>, p, mx, ma, mt);
 }
 
 }  // namespace
