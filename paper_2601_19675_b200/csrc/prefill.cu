@@ -39,7 +39,7 @@ constexpr int kBStages = 3;      // ring of activation tiles (32 KB each)
 constexpr int kABlock = kTileM * 128;           // 16 KB: one row block of one stage
 constexpr int kABytes = 2 * kABlock;            // 32 KB
 constexpr int kBBytes = kMaxTileN * 128;        // 32 KB: one 256-token tile
-constexpr double kPairCost = 1.25;  // duration of a two-block CTA relative to a one-block CTA (scheduling estimate)
+constexpr double kPairCost = 1.4;  // duration of a two-block CTA relative to a one-block CTA (scheduling estimate)
 constexpr int kSmemBytes = kAStages * kABytes + kBStages * kBBytes + 1024;  // + slack for 1024-byte alignment
 constexpr uint32_t kSpinLimit = 1u << 24;
 
@@ -54,7 +54,9 @@ struct PrefillParams {
     int m, n, T;
     int nsteps, gshift, ng, r_pad;
     int tile_n;      // tokens per accumulator: 64, 128 or 256
-    int pair_tiles;  // CTAs along x that own two row blocks (256 rows, two accumulators); the others own one
+    int pair_tiles;    // row tiles of two blocks (256 rows, two accumulators)
+    int single_tiles;  // row tiles of one block
+    int units;         // token tiles
     int lr_stages;   // ceil(r_pad / 64)
 };
 
@@ -156,10 +158,17 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     __shared__ int s_timeout;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // row tiles: the first p.pair_tiles CTAs along x own two blocks of 128 rows (two accumulators), the rest one
-    const int n_acc = (int)blockIdx.x < p.pair_tiles ? 2 : 1;
-    const int row_base = ((int)blockIdx.x < p.pair_tiles ? (int)blockIdx.x * 2 : p.pair_tiles + (int)blockIdx.x) * kTileM;
-    const int tok_base = (int)blockIdx.y * p.tile_n;
+    // The grid is one-dimensional and lists every two-block CTA (256 rows, two accumulators) before the
+    // one-block CTAs, so that the cheaper tiles fill the last wave: pair_tiles two-block row tiles and
+    // single_tiles one-block row tiles per token tile.
+    const int n_pair_ctas = p.pair_tiles * p.units;
+    const bool is_pair = (int)blockIdx.x < n_pair_ctas;
+    const int n_acc = is_pair ? 2 : 1;
+    const int rest = (int)blockIdx.x - n_pair_ctas;
+    const int tile_x = is_pair ? (int)blockIdx.x % p.pair_tiles : p.pair_tiles + rest % p.single_tiles;
+    const int tile_y = is_pair ? (int)blockIdx.x / p.pair_tiles : rest / p.single_tiles;
+    const int row_base = (is_pair ? tile_x * 2 : p.pair_tiles + tile_x) * kTileM;
+    const int tok_base = tile_y * p.tile_n;
     const int total = p.nsteps + p.lr_stages;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
@@ -532,8 +541,11 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
         if (forced >= 0 && forced <= m_tiles / 2) best_pairs = forced;
     }
     p.pair_tiles = best_pairs;
-    dim3 grid(best_pairs + (m_tiles - 2 * best_pairs), units);
-    if (grid.y > 65535) return cudaErrorInvalidValue;
+    p.single_tiles = m_tiles - 2 * best_pairs;
+    p.units = units;
+    const long long n_ctas = (long long)(p.pair_tiles + p.single_tiles) * units;
+    if (n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;
+    dim3 grid((unsigned)n_ctas);
     switch (d.bits) {
         case 2: return launch_prefill_bits<2>(p, mx, ma, mt, grid, s);
         case 3: return launch_prefill_bits<3>(p, mx, ma, mt, grid, s);
