@@ -8,8 +8,8 @@
 // (scale, zero) pairs, the rows of A -- is requested before griddepcontrol.wait, i.e. while the
 // prologue kernel of the same forward still runs; the rotated activations and their 64-column
 // sums follow after the wait.  Sixteen consumer warps split each stage by K step (warp w takes
-// step w), multiply with mma.sync and keep their sums in registers; one shared-memory reduction
-// over the warps at the end, then the low-rank term and the store.
+// step w), multiply with mma.sync and keep their sums in registers (the warps 0 .. RT-1 start theirs
+// from the low-rank term A t); one shared-memory reduction over the warps at the end, then the store.
 //
 // Arithmetic: as in the general path, sum_k s (c_k - z) x~_k = s (sum_k (128 + c_k) x~_k
 // - (128 + z) sum_k x~_k), the first sum on the tensor cores with exact bf16 operands 128 + c_k,
@@ -112,6 +112,24 @@ stream_kernel(const StreamParams p) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) yacc[r][nt][i] = 0.0f;
 
+    // low-rank up-projection A t: warp r starts the sums of row tile r with it (fp16 tensor-core product
+    // into the fp32 sums), before the first stage, so that nothing but the reduction follows the last one
+    auto lowrank_up = [&](float (&acc)[NT][4], int r) {
+        const __half* as = reinterpret_cast<const __half*>(smem + p.off_a) + (size_t)r * 16 * p.r_pad;
+        const __half* ts = reinterpret_cast<const __half*>(smem + p.off_t);
+        for (int jj = 0; jj < p.r_pad; jj += 16) {
+            uint32_t a[4];
+            a[0] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 2 * tg);
+            a[1] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 2 * tg);
+            a[2] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 8 + 2 * tg);
+            a[3] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 8 + 2 * tg);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const __half* trow = ts + (nt * 8 + gq) * p.r_pad + jj + 2 * tg;
+                mma_f16(acc[nt], a, *reinterpret_cast<const uint32_t*>(trow), *reinterpret_cast<const uint32_t*>(trow + 8));
+            }
+        }
+    };
     if (warp == kConsumerWarps) {
         // ---------------- producer warp ----------------
         const int first = min(p.n_stages, p.total_stages);
@@ -151,6 +169,12 @@ stream_kernel(const StreamParams p) {
         if (!mbar_wait(cbar, 0)) {
             s_timeout = 1;
             if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+        }
+        if (p.r_pad > 0 && warp < n_rt) {
+            if (!mbar_wait(tbar, 0) && lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+#pragma unroll
+            for (int r = 0; r < RT; ++r)
+                if (warp == r) lowrank_up(yacc[r], r);
         }
         const uint32_t* szs = reinterpret_cast<const uint32_t*>(smem + p.off_sz);
         const uint32_t ldm_off = (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
@@ -222,32 +246,7 @@ stream_kernel(const StreamParams p) {
             if (lane == 0) mbar_arrive(empty(slot));
         }
     }
-    __syncthreads();  // every stage consumed, t staged: the ring can be reused for the reduction
-
-    // low-rank up-projection A t: warp r adds the term of row tile r (fp16 tensor-core product into
-    // the fp32 sums)
-    auto lowrank_up = [&](float (&acc)[NT][4], int r) {
-        const __half* as = reinterpret_cast<const __half*>(smem + p.off_a) + (size_t)r * 16 * p.r_pad;
-        const __half* ts = reinterpret_cast<const __half*>(smem + p.off_t);
-        for (int jj = 0; jj < p.r_pad; jj += 16) {
-            uint32_t a[4];
-            a[0] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 2 * tg);
-            a[1] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 2 * tg);
-            a[2] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 8 + 2 * tg);
-            a[3] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 8 + 2 * tg);
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const __half* trow = ts + (nt * 8 + gq) * p.r_pad + jj + 2 * tg;
-                mma_f16(acc[nt], a, *reinterpret_cast<const uint32_t*>(trow), *reinterpret_cast<const uint32_t*>(trow + 8));
-            }
-        }
-    };
-    if (p.r_pad > 0 && warp < n_rt) {
-        if (!mbar_wait(tbar, 0) && lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
-#pragma unroll
-        for (int r = 0; r < RT; ++r)
-            if (warp == r) lowrank_up(yacc[r], r);
-    }
+    __syncthreads();  // every stage consumed: the ring can be reused for the reduction
 
     // reduction over the consumer warps: red[warp][token][RT * 16 rows]
     constexpr int kRows = RT * 16;
