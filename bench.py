@@ -35,10 +35,45 @@ WORKLOADS = {
     "cfg3_T2048": ("cfg3", 2048, 8),
     "cfg4_T16": ("cfg4", 16, 8),
     "cfg4_T4096": ("cfg4", 4096, 2),
+    # the linears of the synthetic 32-layer decoder stack (7 per layer, 224 distinct layers, 3.6 GB of packed weights);
+    # attention, norms and activations are not part of the method and are not run
+    "cfg5_T1": ("cfg5", 1, 224),
+    "cfg5_T32": ("cfg5", 32, 224),
 }
+# linears of one layer of the stack: name, d_in, d_out (hidden 4096, MLP 11008)
+STACK_LINEARS = [("q", 4096, 4096), ("k", 4096, 4096), ("v", 4096, 4096), ("o", 4096, 4096),
+                 ("gate", 4096, 11008), ("up", 4096, 11008), ("down", 11008, 4096)]
+STACK_LAYERS = 32
+STACK_QUANT = dict(bits=4, group_size=128, block_size=128, identity_cols=128, rank=32)
+
+
+def stack_shape(n, m):
+    return dict(d_in=n, d_out=m, **STACK_QUANT)
+
+
+def stack_bytes(T):
+    return STACK_LAYERS * sum(algorithmic_bytes(stack_shape(n, m), T) for _, n, m in STACK_LINEARS)
+
+
+def time_oracle_stack(T, budget_s):
+    """The oracle on the three linear shapes of the stack (1024 sampled output rows each), combined into the
+    time of one pass through all 224 linears."""
+    shapes = {}
+    for _, n, m in STACK_LINEARS:
+        shapes[(n, m)] = shapes.get((n, m), 0) + 1
+    total, cores, desc = 0.0, 1, []
+    for (n, m), count in shapes.items():
+        r = time_oracle(stack_shape(n, m), T, budget_s / len(shapes), 1024, None)
+        total += STACK_LAYERS * count * r["seconds_per_layer"]
+        cores = r["cores"]
+        desc.append(f"{n}->{m}: {r['rows']} rows x {r['reps']} reps")
+    return dict(value=T / total, cores=cores, sample="oracle.forward_exact (fp64 numpy) on sampled rows of the three "
+                "linear shapes (" + "; ".join(desc) + f"), {T} tokens, scaled linearly to 32 layers x 7 linears")
+
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
 # capture summarised in profiles/; valid for the kernel as committed with that summary, null otherwise.
-NCU_TRAFFIC = {("cfg2_T8", "stream_kernel"): 9284352}
+NCU_TRAFFIC = {("cfg2_T8", "stream_kernel"): 9283456, ("cfg4_T16", "tall_kernel"): 83354880,
+               ("cfg3_T2048", "prefill_kernel"): 52772608}
 METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
 
@@ -167,6 +202,21 @@ def run_reference(args):
         return 0
     from paper_2601_19675_b200 import synth
     cfg, T, ring = WORKLOADS[args.workload]
+    if cfg == "cfg5":
+        for _ in range(args.warmup):
+            time_oracle_stack(T, 0.0)
+        t0 = time.perf_counter()
+        results = [time_oracle_stack(T, 1.5) for _ in range(args.steps)]
+        wall = time.perf_counter() - t0
+        value = statistics.median(r["value"] for r in results)
+        line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=int(os.environ.get("WORLD_SIZE", "1")),
+                    steps=args.steps, warmup=args.warmup, ms_per_step=wall / args.steps * 1e3, higher_is_better=True,
+                    scaling="weak", vs_baseline=None, dtype="f64", data="synthetic", config=workload_config(args.workload),
+                    cpu_baseline=dict(value=value, unit=UNIT, cores=results[0]["cores"], kind="oracle",
+                                      sample=results[0]["sample"]),
+                    e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+        print(json.dumps(line))
+        return 0
     c = synth.CONFIGS[cfg]
     max_rows = 1024 if c["d_out"] * c["d_in"] > (1 << 24) or T > 64 else None
     max_tokens = 16 if T > 64 else None
@@ -193,6 +243,11 @@ def run_reference(args):
 def workload_config(name):
     from paper_2601_19675_b200 import synth
     cfg, T, ring = WORKLOADS[name]
+    if cfg == "cfg5":
+        return dict(workload=f"{name}: the 224 LoPRo linears of a 32-layer decoder stack (hidden 4096, MLP 11008; 4-bit g128 "
+                             f"block 128 rank 32), batch {T}, one token per sequence; attention/norm/activation glue not run",
+                    tokens=T, ring_layers=ring,
+                    l2="inputs larger than L2: one step reads %.0f MB of packed weights" % (stack_bytes(T) / 1e6))
     c = synth.CONFIGS[cfg]
     ring_bytes = ring * algorithmic_bytes(c, T)
     return dict(workload=f"{name}: LoPRo linear forward d_in={c['d_in']} d_out={c['d_out']} {c['bits']}-bit g{c['group_size']} "
@@ -200,6 +255,138 @@ def workload_config(name):
                 tokens=T, ring_layers=ring,
                 l2="inputs larger than L2: every step walks a ring of %d distinct layers (%.0f MB of packed weights)"
                    % (ring, ring_bytes / 1e6))
+
+
+def run_stack(args, T, rank, world, local, dev, dev16):
+    """The 224 linears of the 32-layer stack, one forward each per step, every linear with its own packed layer.
+    Linears with 4096 inputs read one fixed activation tensor, the `down` projections another (the glue between
+    them is not part of the method and is not run; the kernels' work does not depend on the values)."""
+    import torch
+    from paper_2601_19675_b200 import lopro, synth
+    if world > 1:
+        import torch.distributed as dist
+    q = STACK_QUANT
+    shapes = sorted({(n, m) for _, n, m in STACK_LINEARS})
+    base, descs = {}, {}
+    for n, m in shapes:
+        layer = synth.random_layer(n, m, q["bits"], q["group_size"], q["rank"], seed=rank + n // 64)
+        base[(n, m)] = dict(codes=torch.from_numpy(layer["codes"]).to(dev), sc=dev16(layer["scales"]), zr=dev16(layer["zeros"]),
+                            pm=torch.from_numpy(layer["perm"]).to(dev), A=dev16(layer["A"]), B=dev16(layer["B"]))
+        descs[(n, m)] = lopro.make_desc(n, m, q["bits"], q["group_size"], q["block_size"], q["identity_cols"], q["rank"])
+    xs, x_bits = {}, {}
+    for n in sorted({n for n, _ in shapes}):
+        x_bits[n] = synth.activations(T, n, seed=rank + n)
+        xs[n] = dev16(x_bits[n]).view(torch.bfloat16)
+    ys = {m: [torch.empty((T, m), dtype=torch.bfloat16, device=dev) for _ in range(2)] for m in sorted({m for _, m in shapes})}
+    ws_bytes = max(lopro.workspace_bytes(descs[k], T) for k in shapes)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    linears = []  # (desc, blob, x, y)
+    for li in range(STACK_LAYERS):
+        for j, (_, n, m) in enumerate(STACK_LINEARS):
+            b = base[(n, m)]
+            i = li * len(STACK_LINEARS) + j
+            codes = torch.roll(b["codes"], shifts=(i, 3 * i), dims=(0, 1)) if i else b["codes"]
+            blob = lopro.pack(descs[(n, m)], codes, b["sc"], b["zr"], b["pm"], b["A"], b["B"])
+            linears.append((descs[(n, m)], blob, xs[n], ys[m][i % 2]))
+    del codes
+    for b in base.values():
+        del b["codes"]
+
+    def one_step():
+        for d, blob, x, y in linears:
+            lopro.linear_fwd(d, blob, x, lopro.OUT_BF16, workspace=ws, y=y)
+
+    stream = torch.cuda.Stream(device=dev)
+    graph = None
+    with torch.cuda.stream(stream):
+        one_step()
+        stream.synchronize()
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                one_step()
+        run_step = graph.replay if graph is not None else one_step
+        for _ in range(args.warmup):
+            run_step()
+        stream.synchronize()
+        if world > 1:
+            dist.barrier()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        ev[0].record(stream)
+        for k in range(args.steps):
+            run_step()
+            ev[k + 1].record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        clocks = sampler.stop() if rank == 0 else None
+        total_ms = ev[0].elapsed_time(ev[-1])
+        step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+        # end to end: the batch's activations come from pinned host memory every step, the last linear's output
+        # goes back to the host
+        xh = torch.from_numpy(x_bits[4096].view(np.int16)).view(torch.bfloat16).pin_memory()
+        y_last = linears[-1][3]
+        yh = torch.empty(tuple(y_last.shape), dtype=torch.bfloat16).pin_memory()
+        e2e_steps = max(3, min(args.steps, 20))
+
+        def e2e_step():
+            xs[4096].copy_(xh, non_blocking=True)
+            run_step()
+            yh.copy_(y_last, non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        stream.synchronize()
+        if world > 1:
+            dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        stream.synchronize()
+        e2e_ms = e0.elapsed_time(e1)
+        status = lopro.workspace_status(ws)
+        assert status == lopro.OK, f"device status {status}"
+        assert torch.isfinite(yh.float()).all()
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+        dist.barrier()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+    peaks = measured_peaks()
+    ms_per_step = total_ms / args.steps
+    value = T * world / (ms_per_step * 1e-3)
+    e2e_value = T * world / (e2e_ms / e2e_steps * 1e-3)
+    paths = [lopro.linear_fwd_path(d, T) for d, _, _, _ in linears]
+    names = sorted({lopro.PATH_NAMES.get(p, "?") for p, _ in paths})
+    ach = stack_bytes(T) / (ms_per_step * 1e-3) / 1e9
+    roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"], traffic=None,
+                    peak_source=f"of {peaks['source']}", frac_of_nominal_8000=ach / 8000.0,
+                    kernel=" + ".join(n + "_kernel" for n in names), algorithmic_bytes_per_step=stack_bytes(T),
+                    launch_us=ms_per_step * 1e3 / len(linears),
+                    note="whole step: 224 linear forwards (prologue kernels included); launch_us = step time / 224")
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic", config=workload_config(args.workload), clocks=clocks,
+                e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=T * 4096 * 2, d2h_bytes_per_step=T * y_last.shape[1] * 2,
+                         steps=e2e_steps),
+                gpu_launches=sum(n for _, n in paths) * args.steps, path="+".join(names), roofline=roofline,
+                step_ms_min=min(step_ms), step_ms_median=statistics.median(step_ms), cuda_graph=graph is not None)
+    if not args.no_cpu_baseline and world == 1:
+        r = time_oracle_stack(T, 12.0)
+        line["cpu_baseline"] = dict(value=r["value"], unit=UNIT, cores=r["cores"], kind="oracle", sample=r["sample"])
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
 
 
 def main():
@@ -236,12 +423,15 @@ def main():
     lopro.lib()
 
     cfg, T, ring = WORKLOADS[args.workload]
-    c = synth.CONFIGS[cfg]
-    d = lopro.make_desc(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"])
     dev = torch.device("cuda", local)
 
     def dev16(a):
         return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev)
+
+    if cfg == "cfg5":
+        return run_stack(args, T, rank, world, local, dev, dev16)
+    c = synth.CONFIGS[cfg]
+    d = lopro.make_desc(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"])
 
     # ring of distinct layers: layer 0 drawn by the seeded generator, the others re-use its tensors with
     # freshly drawn codes (generated on the host once, shifted per layer) so that set-up stays short
@@ -361,7 +551,8 @@ def main():
     else:
         ach = algorithmic_flops(c, T) / dur_s / 1e12
         pk = peaks["bf16_tflops_sustained"]
-        roofline = dict(bound="tensor", achieved=ach, peak=pk, unit="TFLOP/s", frac=ach / pk, traffic=None,
+        roofline = dict(bound="tensor", achieved=ach, peak=pk, unit="TFLOP/s", frac=ach / pk,
+                        traffic=NCU_TRAFFIC.get((args.workload, kernel_name)),
                         peak_source=f"of {peaks['source']} (sustained)", kernel=kernel_name,
                         algorithmic_flops_per_launch=algorithmic_flops(c, T), launch_us=dur_s * 1e6, note=note)
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,

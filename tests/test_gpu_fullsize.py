@@ -1,5 +1,6 @@
 """Parity at the full sizes of the benchmark workloads, in the launch configuration bench.py times,
-on sampled output rows the oracle computes one by one (configurations 2, 3 and 4)."""
+on sampled output rows the oracle computes one by one (configurations 2, 3 and 4, and the three linear
+shapes of the stack of configuration 5)."""
 import numpy as np
 import pytest
 import torch
@@ -12,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 
 def _sampled(cfg, T, n_rows=48, seed=0):
-    c = synth.CONFIGS[cfg]
+    c = synth.CONFIGS[cfg] if isinstance(cfg, str) else cfg
     n, m = c["d_in"], c["d_out"]
     layer = random_layer_np(n, m, c["bits"], c["group_size"], c["rank"], seed=seed)
     d = lopro.make_desc(n, m, c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"])
@@ -54,3 +55,15 @@ def test_cfg3_prefill():
 @pytest.mark.parametrize("T", [16, 4096])
 def test_cfg4_large_layer(T):
     _sampled("cfg4", T, n_rows=24)
+
+
+# the three linear shapes of the 32-layer stack configuration (hidden 4096, MLP 11008; 4-bit, g = 128, rank 32,
+# block 128): attention projections, gate/up, and down -- whose 11008 input columns are neither a multiple of
+# 1024 (ragged last stage of the streaming kernels) nor of 256 x 8
+_STACK = dict(bits=4, group_size=128, block_size=128, identity_cols=128, rank=32)
+
+
+@pytest.mark.parametrize("T", [1, 32])
+@pytest.mark.parametrize("n,m", [(4096, 4096), (4096, 11008), (11008, 4096)])
+def test_stack_linear_shapes(n, m, T):
+    _sampled(dict(d_in=n, d_out=m, **_STACK), T, n_rows=32, seed=n // 64 + T)
