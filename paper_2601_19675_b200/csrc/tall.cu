@@ -107,8 +107,8 @@ __device__ __forceinline__ void tile_step(const unsigned char* codes_rt, const u
     const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        mma_bf16(acc, &a[0], b[nt][0], b[nt][1]);
+        float acc[4];
+        mma_bf16_first(acc, &a[0], b[nt][0], b[nt][1]);
         mma_bf16(acc, &a[4], b[nt][2], b[nt][3]);
         mma_bf16(acc, &a[8], b[nt][4], b[nt][5]);
         mma_bf16(acc, &a[12], b[nt][6], b[nt][7]);
