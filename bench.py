@@ -151,6 +151,17 @@ class ClockSampler:
                     samples=len(sm), reasons=sorted(reasons))
 
 
+def max_over_ranks(values, device):
+    """Replicas: every rank times its own copy of the job; the job's time is the slowest rank's.  Element-wise
+    maximum of `values` over the ranks of the default process group, followed by a barrier."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.barrier()
+    return [float(v) for v in t]
+
+
 def oracle_layer_inputs(c, T, seed):
     from oracle import lopro_oracle as o
     from paper_2601_19675_b200 import synth
@@ -353,10 +364,7 @@ def run_stack(args, T, rank, world, local, dev, dev16):
         assert status == lopro.OK, f"device status {status}"
         assert torch.isfinite(yh.float()).all()
     if world > 1:
-        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
-        dist.barrier()
+        total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -516,10 +524,7 @@ def main():
         assert torch.isfinite(yh.float()).all()
 
     if world > 1:
-        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
-        dist.barrier()
+        total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
