@@ -17,6 +17,8 @@
 //
 // Every wait on an mbarrier is bounded; a wait that runs out stores LOPRO_ERR_TIMEOUT in the
 // workspace status word and the CTA stops waiting (its outputs are then unspecified).
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -277,6 +279,193 @@ stream_kernel(const StreamParams p) {
     }
 }
 
+// Variant for up to 8 tokens when the whole K range fits the ring (no refills): 32 consumer warps and no
+// producer warp.  Warp w takes step w & 15 of every stage for row tile w >> 4, i.e. ONE tile step per stage, so
+// each scheduler has eight warps to hide the expand -> MMA -> FMA chains behind; lane 0 of warp 0 issues every
+// copy (layer data before griddepcontrol.wait, activations and t after it).
+constexpr int kWideWarps = 32;
+constexpr int kWideThreads = kWideWarps * 32;
+
+template <int BITS>
+__global__ void __launch_bounds__(kWideThreads, 1)
+stream_wide_kernel(const StreamParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) uint64_t bars[2 * kMaxStages + 2];  // wfull, xfull per stage; sz + A; t
+    __shared__ int s_timeout;
+    constexpr int kTok = 8;
+    constexpr int kStepBytes = 128 * BITS;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gq = lane >> 2, tg = lane & 3;
+    const int step = warp & 15, r = warp >> 4;
+    const int rt0 = blockIdx.x * 2;
+    const int n_rt = min(2, (p.m >> 4) - rt0);
+    const int tc = min(kTok, p.T);
+    const uint32_t bar0 = smem_u32(bars);
+    auto wfull = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto xfull = [&](int s) { return bar0 + 8u * (uint32_t)(kMaxStages + s); };
+    const uint32_t cbar = bar0 + 8u * (uint32_t)(2 * kMaxStages);
+    const uint32_t tbar = cbar + 8u;
+    const uint32_t smem0 = smem_u32(smem);
+
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (tid == 0) {
+        for (int s = 0; s < p.total_stages; ++s) {
+            mbar_init(wfull(s), 1);
+            mbar_init(xfull(s), 1);
+        }
+        mbar_init(cbar, 1);
+        mbar_init(tbar, 1);
+        s_timeout = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    auto steps_of = [&](int stage) { return min(kStageSteps, p.nsteps - stage * kStageSteps); };
+
+    if (tid == 0) {
+        // layer data: (scale, zero) pairs and rows of A of the live row tiles, the codes of every stage
+        const uint32_t sz_bytes = (uint32_t)(n_rt * p.ng * 64);
+        const uint32_t a_bytes = (uint32_t)(n_rt * 16 * p.r_pad * 2);
+        mbar_expect_tx(cbar, sz_bytes + a_bytes);
+        bulk_g2s(smem0 + p.off_sz, p.sz + (size_t)rt0 * p.ng * 16, sz_bytes, cbar);
+        if (a_bytes) bulk_g2s(smem0 + p.off_a, p.A + (size_t)rt0 * 16 * p.r_pad, a_bytes, cbar);
+        for (int s = 0; s < p.total_stages; ++s) {
+            const uint32_t bytes = (uint32_t)(steps_of(s) * kStepBytes);
+            mbar_expect_tx(wfull(s), bytes * (uint32_t)n_rt);
+            for (int q = 0; q < n_rt; ++q)
+                bulk_g2s(smem0 + p.off_ring + s * p.stage_bytes + q * kStageSteps * kStepBytes,
+                         reinterpret_cast<const unsigned char*>(p.codes) +
+                             ((size_t)(rt0 + q) * p.nsteps + (size_t)s * kStageSteps) * kStepBytes,
+                         bytes, wfull(s));
+        }
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (tid == 0) {
+        const uint32_t bytes = (uint32_t)(tc * kActRecord);
+        for (int s = 0; s < p.total_stages; ++s) {
+            mbar_expect_tx(xfull(s), bytes);
+            bulk_g2s(smem0 + p.off_ring + s * p.stage_bytes + p.off_stage_x, p.act + (size_t)s * p.t_pad * kActRecord, bytes,
+                     xfull(s));
+        }
+        if (p.r_pad > 0) {
+            const uint32_t t_bytes = (uint32_t)(tc * p.r_pad * 2);
+            mbar_expect_tx(tbar, t_bytes);
+            bulk_g2s(smem0 + p.off_t, p.t, t_bytes, tbar);
+        }
+    }
+
+    float yacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    const bool live = r < n_rt;
+    if (!mbar_wait(cbar, 0)) {
+        s_timeout = 1;
+        if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+    }
+    if (p.r_pad > 0 && step == 0) {
+        // low-rank term A t of row tile r starts the sums of its step-0 warp
+        if (!mbar_wait(tbar, 0) && lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+        if (live) {
+            const __half* as = reinterpret_cast<const __half*>(smem + p.off_a) + (size_t)r * 16 * p.r_pad;
+            const __half* ts = reinterpret_cast<const __half*>(smem + p.off_t);
+            for (int jj = 0; jj < p.r_pad; jj += 16) {
+                uint32_t a[4];
+                a[0] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 2 * tg);
+                a[1] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 2 * tg);
+                a[2] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 8 + 2 * tg);
+                a[3] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 8 + 2 * tg);
+                const __half* trow = ts + gq * p.r_pad + jj + 2 * tg;
+                mma_f16(yacc, a, *reinterpret_cast<const uint32_t*>(trow), *reinterpret_cast<const uint32_t*>(trow + 8));
+            }
+        }
+    }
+    const uint32_t* szs = reinterpret_cast<const uint32_t*>(smem + p.off_sz);
+    const uint32_t ldm_off = (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
+    for (int s = 0; s < p.total_stages; ++s) {
+        if (!s_timeout && !(mbar_wait(wfull(s), 0) && mbar_wait(xfull(s), 0))) {
+            s_timeout = 1;
+            if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+        }
+        if (live && step < steps_of(s)) {
+            const unsigned char* stage = smem + p.off_ring + s * p.stage_bytes;
+            const uint32_t xs_u32 = smem0 + p.off_ring + s * p.stage_bytes + p.off_stage_x;
+            const unsigned char* srec = stage + p.off_stage_x + 2048;  // sums of token 0
+            const int grp = (s * kStageSteps + step) >> p.gshift;
+            uint32_t b[8];
+            const uint32_t base = xs_u32 + (uint32_t)(step * 64) * 2u + ldm_off;
+            ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[0]), base);
+            ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[4]), base + 64u);
+            const float sx0 = reinterpret_cast<const float*>(srec + (2 * tg) * kActRecord)[step];
+            const float sx1 = reinterpret_cast<const float*>(srec + (2 * tg + 1) * kActRecord)[step];
+            uint32_t w[BITS];
+            const uint32_t* wp = reinterpret_cast<const uint32_t*>(stage + (r * kStageSteps + step) * kStepBytes) + lane * BITS;
+            if constexpr (BITS == 4) {
+                const uint4 v = *reinterpret_cast<const uint4*>(wp);
+                w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+            } else if constexpr (BITS == 2) {
+                const uint2 v = *reinterpret_cast<const uint2*>(wp);
+                w[0] = v.x; w[1] = v.y;
+            } else {
+#pragma unroll
+                for (int q = 0; q < BITS; ++q) w[q] = wp[q];
+            }
+            uint32_t a[16];
+            expand_codes<BITS>(a, w);
+            const uint32_t sz_lo = szs[(r * p.ng + grp) * 16 + gq], sz_hi = szs[(r * p.ng + grp) * 16 + gq + 8];
+            const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
+            const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
+            const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
+            float acc[4];
+            mma_bf16_first(acc, &a[0], b[0], b[1]);
+            mma_bf16(acc, &a[4], b[2], b[3]);
+            mma_bf16(acc, &a[8], b[4], b[5]);
+            mma_bf16(acc, &a[12], b[6], b[7]);
+            yacc[0] = fmaf(f_lo.x, acc[0], fmaf(nsz_lo, sx0, yacc[0]));
+            yacc[1] = fmaf(f_lo.x, acc[1], fmaf(nsz_lo, sx1, yacc[1]));
+            yacc[2] = fmaf(f_hi.x, acc[2], fmaf(nsz_hi, sx0, yacc[2]));
+            yacc[3] = fmaf(f_hi.x, acc[3], fmaf(nsz_hi, sx1, yacc[3]));
+        }
+    }
+    __syncthreads();  // every stage consumed: the ring can be reused for the reduction
+
+    // reduction over the 16 steps of a tile: red[step][token][32 rows]
+    float* red = reinterpret_cast<float*>(smem + p.off_ring);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int tk = 2 * tg + (i & 1), rl = r * 16 + gq + 8 * (i >> 1);
+        red[(step * kTok + tk) * 32 + rl] = yacc[i];
+    }
+    __syncthreads();
+    const int rows_here = n_rt * 16;
+    for (int i = tid; i < tc * 32; i += kWideThreads) {
+        const int tk = i >> 5, rl = i & 31;
+        if (rl < rows_here) {
+            float sum = 0.0f;
+#pragma unroll
+            for (int w = 0; w < 16; ++w) sum += red[(w * kTok + tk) * 32 + rl];
+            const size_t o = (size_t)tk * p.ldy + (size_t)rt0 * 16 + rl;
+            if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = sum;
+            else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(sum);
+        }
+    }
+}
+
+template <int BITS>
+cudaError_t launch_stream_wide(const StreamParams& p, int smem_bytes, cudaStream_t s) {
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(stream_wide_kernel<BITS>, kStreamMaxSmem, &attr_done);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((p.m / 16 + 1) / 2);
+    cfg.blockDim = dim3(kWideThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, stream_wide_kernel<BITS>, p);
+}
+
 template <int BITS, int NT, int RT>
 cudaError_t launch_stream_k(const StreamParams& p, int smem_bytes, cudaStream_t s) {
     static unsigned long long attr_done = 0;
@@ -390,6 +579,18 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
     p.off_ring = pl.off_ring;
     p.stage_bytes = pl.stage_bytes;
     p.off_stage_x = pl.off_stage_x;
+    static int no_wide = -1;  // LOPRO_NO_WIDE=1 keeps the 32-warp variant off (A/B comparison and tests)
+    if (no_wide < 0) {
+        const char* e = getenv("LOPRO_NO_WIDE");
+        no_wide = (e != nullptr && e[0] == '1') ? 1 : 0;
+    }
+    if (!no_wide && pl.nt == 1 && pl.rt == 2 && pl.n_stages == pl.total_stages) {
+        switch (d.bits) {
+            case 2: return launch_stream_wide<2>(p, pl.smem_bytes, s);
+            case 3: return launch_stream_wide<3>(p, pl.smem_bytes, s);
+            default: return launch_stream_wide<4>(p, pl.smem_bytes, s);
+        }
+    }
     switch (d.bits) {
         case 2: return launch_stream_bits<2>(p, pl.nt, pl.rt, pl.smem_bytes, s);
         case 3: return launch_stream_bits<3>(p, pl.nt, pl.rt, pl.smem_bytes, s);
