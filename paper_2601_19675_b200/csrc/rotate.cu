@@ -66,96 +66,111 @@ lowrank_down_kernel(const __half* __restrict__ B, const __nv_bfloat16* __restric
     }
 }
 
+// One row j of B against TPR tokens: t[token][j] = sum_k B[j][k] x[token][k], fp32 accumulation over all of K, one
+// rounding to fp16.  The row of B is read before griddepcontrol.wait, every activation load of the first 4096 columns
+// is in flight before the first use.  Fewer tokens per CTA mean more CTAs and less to load per SM: this chain decides
+// when the prologue ends.
+template <int TPR>
+__device__ __forceinline__ void lowrank_row(const __nv_bfloat16* __restrict__ x, int64_t ldx, const __half* __restrict__ B,
+                                            __half* __restrict__ t, int n, int r_pad, int T, int rb, int tok0) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ float part[8][TPR];
+    const int j = rb % r_pad, tq = tok0 + TPR * (rb / r_pad);
+    const __half* brow = B + (size_t)j * n;
+    const int npass = (n + 2047) >> 11;
+    uint4 pre[2];
+#pragma unroll
+    for (int ps = 0; ps < 2; ++ps) {
+        const int k = ps * 2048 + tid * 8;
+        pre[ps] = k < n ? __ldg(reinterpret_cast<const uint4*>(brow + k)) : make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    float acc[TPR];
+#pragma unroll
+    for (int tk = 0; tk < TPR; ++tk) acc[tk] = 0.0f;
+    auto load_x = [&](uint4 (&xw)[TPR], int k) {
+#pragma unroll
+        for (int tk = 0; tk < TPR; ++tk)
+            xw[tk] = (k < n && tq + tk < T) ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tq + tk) * ldx + k))
+                                            : make_uint4(0, 0, 0, 0);
+    };
+    auto accumulate = [&](const uint4& bw, const uint4 (&xw)[TPR]) {
+        float bf[8];
+        const __half2* h = reinterpret_cast<const __half2*>(&bw);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(h[i]);
+            bf[2 * i] = f.x;
+            bf[2 * i + 1] = f.y;
+        }
+#pragma unroll
+        for (int tk = 0; tk < TPR; ++tk) {
+            const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xw[tk]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(xh[i]);
+                acc[tk] = fmaf(bf[2 * i], f.x, acc[tk]);
+                acc[tk] = fmaf(bf[2 * i + 1], f.y, acc[tk]);
+            }
+        }
+    };
+    {   // the first two passes (all of K up to 4096 columns): every load is in flight before the first use,
+        // so the dependent chain after the wait is one memory round trip
+        uint4 x0[TPR], x1[TPR];
+        load_x(x0, tid * 8);
+        load_x(x1, 2048 + tid * 8);
+        accumulate(pre[0], x0);
+        accumulate(pre[1], x1);
+    }
+    for (int ps = 2; ps < npass; ++ps) {
+        const int k = ps * 2048 + tid * 8;
+        if (k >= n) break;
+        uint4 xw[TPR];
+        load_x(xw, k);
+        accumulate(__ldg(reinterpret_cast<const uint4*>(brow + k)), xw);
+    }
+#pragma unroll
+    for (int tk = 0; tk < TPR; ++tk) {
+        float v = acc[tk];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+        if (lane == 0) part[warp][tk] = v;
+    }
+    __syncthreads();
+    if (tid < TPR) {
+        float v = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += part[w][tid];
+        if (tq + tid < T) t[(size_t)(tq + tid) * r_pad + j] = __float2half_rn(v);
+    }
+}
+
 // Prologue of the small-batch forward (T <= 32, b_H <= 256, b_I a multiple of b_H).  Grid:
 // x = column chunks of 256, then the rows of B; y = groups of 8 tokens.
 //  * a chunk CTA rotates 256 output columns, warp w for token w: the 8 entries of a lane are
 //    gathered from global memory through perm, transformed with register and shuffle butterflies,
 //    rounded to bf16 and stored together with their 64-column sums in the activation image that the
 //    streaming kernel copies to shared memory;
-//  * a row CTA computes t[token][j] = sum_k B[j][k] x[token][k] for one row j of B and the 8 tokens
-//    (fp32 accumulation over all of K, one rounding to fp16): the low-rank intermediate "Y = V X".
+//  * a row CTA computes t[token][j] = sum_k B[j][k] x[token][k] for one row j of B and `tpr` of the 8 tokens
+//    (8 / tpr CTAs per row): the low-rank intermediate "Y = V X".
 // Launched with programmatic stream serialization: perm and B (layer data) are read before the
 // wait, the activations after it.
 __global__ void __launch_bounds__(256)
 prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
                 const __half* __restrict__ B, unsigned char* __restrict__ act_image, __half* __restrict__ t,
-                int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T) {
+                int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T,
+                int tpr) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nchunks = (n + 255) >> 8;
     const int tok0 = blockIdx.y * 8;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if ((int)blockIdx.x >= nchunks) {
-        // ---- one row of B against eight tokens ----
-        __shared__ float part[8][8];
-        const int j = (int)blockIdx.x - nchunks;
-        const __half* brow = B + (size_t)j * n;
-        const int npass = (n + 2047) >> 11;
-        uint4 pre[2];
-#pragma unroll
-        for (int ps = 0; ps < 2; ++ps) {
-            const int k = ps * 2048 + tid * 8;
-            pre[ps] = k < n ? __ldg(reinterpret_cast<const uint4*>(brow + k)) : make_uint4(0, 0, 0, 0);
-        }
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        float acc[8];
-#pragma unroll
-        for (int tk = 0; tk < 8; ++tk) acc[tk] = 0.0f;
-        auto load_x = [&](uint4 (&xw)[8], int k) {
-#pragma unroll
-            for (int tk = 0; tk < 8; ++tk)
-                xw[tk] = (k < n && tok0 + tk < T) ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tok0 + tk) * ldx + k))
-                                                  : make_uint4(0, 0, 0, 0);
-        };
-        auto accumulate = [&](const uint4& bw, const uint4 (&xw)[8]) {
-            float bf[8];
-            const __half2* h = reinterpret_cast<const __half2*>(&bw);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 f = __half22float2(h[i]);
-                bf[2 * i] = f.x;
-                bf[2 * i + 1] = f.y;
-            }
-#pragma unroll
-            for (int tk = 0; tk < 8; ++tk) {
-                const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xw[tk]);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float2 f = __bfloat1622float2(xh[i]);
-                    acc[tk] = fmaf(bf[2 * i], f.x, acc[tk]);
-                    acc[tk] = fmaf(bf[2 * i + 1], f.y, acc[tk]);
-                }
-            }
-        };
-        {   // the first two passes (all of K up to 4096 columns): every load is in flight before the first use,
-            // so the dependent chain after the wait is one memory round trip
-            uint4 x0[8], x1[8];
-            load_x(x0, tid * 8);
-            load_x(x1, 2048 + tid * 8);
-            accumulate(pre[0], x0);
-            accumulate(pre[1], x1);
-        }
-        for (int ps = 2; ps < npass; ++ps) {
-            const int k = ps * 2048 + tid * 8;
-            if (k >= n) break;
-            uint4 xw[8];
-            load_x(xw, k);
-            accumulate(__ldg(reinterpret_cast<const uint4*>(brow + k)), xw);
-        }
-#pragma unroll
-        for (int tk = 0; tk < 8; ++tk) {
-            float v = acc[tk];
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-            if (lane == 0) part[warp][tk] = v;
-        }
-        __syncthreads();
-        if (tid < 8) {
-            float v = 0.0f;
-#pragma unroll
-            for (int w = 0; w < 8; ++w) v += part[w][tid];
-            if (tok0 + tid < T) t[(size_t)(tok0 + tid) * r_pad + j] = __float2half_rn(v);
-        }
+        const int rb = (int)blockIdx.x - nchunks;
+        if (tpr == 8) lowrank_row<8>(x, ldx, B, t, n, r_pad, T, rb, tok0);
+        else if (tpr == 4) lowrank_row<4>(x, ldx, B, t, n, r_pad, T, rb, tok0);
+        else if (tpr == 2) lowrank_row<2>(x, ldx, B, t, n, r_pad, T, rb, tok0);
+        else lowrank_row<1>(x, ldx, B, t, n, r_pad, T, rb, tok0);
         return;
     }
 
@@ -272,7 +287,12 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
                             int* status, int T, cudaStream_t s) {
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((d.d_in + 255) / 256 + (d.rank > 0 ? r_pad : 0), (T + 7) / 8);
+    // tokens per row CTA: as few as it takes to put about one CTA on every SM
+    const int live = T < 8 ? T : 8;
+    int tpr = 8;
+    while (tpr > 1 && r_pad * ((live + tpr - 1) / tpr) * ((T + 7) / 8) < 120) tpr >>= 1;
+    const int row_ctas = d.rank > 0 ? r_pad * ((live + tpr - 1) / tpr) : 0;
+    cfg.gridDim = dim3((d.d_in + 255) / 256 + row_ctas, (T + 7) / 8);
     cfg.blockDim = dim3(256);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = s;
@@ -282,7 +302,7 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, prologue_kernel, x, ldx, perm, B, act_image, t, status, d.d_in,
-                              d.identity_cols, d.block_size, inv, d.rank > 0 ? r_pad : 0, t_pad, T);
+                              d.identity_cols, d.block_size, inv, d.rank > 0 ? r_pad : 0, t_pad, T, tpr);
 }
 
 cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,
