@@ -294,6 +294,10 @@ stream_wide_kernel(const StreamParams p) {
     __shared__ int s_timeout;
     constexpr int kTok = 8;
     constexpr int kStepBytes = 128 * BITS;
+    // stage geometry of this variant (8 tokens, two row tiles) as compile-time constants: the unrolled stage loop
+    // then addresses everything with immediates
+    constexpr int kOffX = 2 * kStageSteps * kStepBytes;                             // activations after the codes
+    constexpr int kStageBytes = (kOffX + kTok * kActRecord + 127) / 128 * 128;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tg = lane & 3;
@@ -333,7 +337,7 @@ stream_wide_kernel(const StreamParams p) {
             const uint32_t bytes = (uint32_t)(steps_of(s) * kStepBytes);
             mbar_expect_tx(wfull(s), bytes * (uint32_t)n_rt);
             for (int q = 0; q < n_rt; ++q)
-                bulk_g2s(smem0 + p.off_ring + s * p.stage_bytes + q * kStageSteps * kStepBytes,
+                bulk_g2s(smem0 + p.off_ring + s * kStageBytes + q * kStageSteps * kStepBytes,
                          reinterpret_cast<const unsigned char*>(p.codes) +
                              ((size_t)(rt0 + q) * p.nsteps + (size_t)s * kStageSteps) * kStepBytes,
                          bytes, wfull(s));
@@ -344,7 +348,7 @@ stream_wide_kernel(const StreamParams p) {
         const uint32_t bytes = (uint32_t)(tc * kActRecord);
         for (int s = 0; s < p.total_stages; ++s) {
             mbar_expect_tx(xfull(s), bytes);
-            bulk_g2s(smem0 + p.off_ring + s * p.stage_bytes + p.off_stage_x, p.act + (size_t)s * p.t_pad * kActRecord, bytes,
+            bulk_g2s(smem0 + p.off_ring + s * kStageBytes + kOffX, p.act + (size_t)s * p.t_pad * kActRecord, bytes,
                      xfull(s));
         }
         if (p.r_pad > 0) {
@@ -379,15 +383,18 @@ stream_wide_kernel(const StreamParams p) {
     }
     const uint32_t* szs = reinterpret_cast<const uint32_t*>(smem + p.off_sz);
     const uint32_t ldm_off = (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
+    const unsigned char* ring = smem + p.off_ring;
+    const uint32_t ring_u32 = smem0 + p.off_ring;
+#pragma unroll 4
     for (int s = 0; s < p.total_stages; ++s) {
         if (!s_timeout && !(mbar_wait(wfull(s), 0) && mbar_wait(xfull(s), 0))) {
             s_timeout = 1;
             if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
         }
         if (live && step < steps_of(s)) {
-            const unsigned char* stage = smem + p.off_ring + s * p.stage_bytes;
-            const uint32_t xs_u32 = smem0 + p.off_ring + s * p.stage_bytes + p.off_stage_x;
-            const unsigned char* srec = stage + p.off_stage_x + 2048;  // sums of token 0
+            const unsigned char* stage = ring + s * kStageBytes;
+            const uint32_t xs_u32 = ring_u32 + s * kStageBytes + kOffX;
+            const unsigned char* srec = stage + kOffX + 2048;  // sums of token 0
             const int grp = (s * kStageSteps + step) >> p.gshift;
             uint32_t b[8];
             const uint32_t base = xs_u32 + (uint32_t)(step * 64) * 2u + ldm_off;
@@ -584,7 +591,8 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
         const char* e = getenv("LOPRO_NO_WIDE");
         no_wide = (e != nullptr && e[0] == '1') ? 1 : 0;
     }
-    if (!no_wide && pl.nt == 1 && pl.rt == 2 && pl.n_stages == pl.total_stages) {
+    if (!no_wide && pl.nt == 1 && pl.rt == 2 && pl.n_stages == pl.total_stages &&
+        pl.off_stage_x == 2 * kStageSteps * 128 * d.bits) {  // the variant's compile-time stage geometry
         switch (d.bits) {
             case 2: return launch_stream_wide<2>(p, pl.smem_bytes, s);
             case 3: return launch_stream_wide<3>(p, pl.smem_bytes, s);
