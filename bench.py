@@ -72,7 +72,7 @@ def time_oracle_stack(T, budget_s):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
 # capture summarised in profiles/; valid for the kernel as committed with that summary, null otherwise.
-NCU_TRAFFIC = {("cfg2_T8", "stream_kernel"): 9283456, ("cfg4_T16", "tall_kernel"): 83354880,
+NCU_TRAFFIC = {("cfg2_T8", "stream_wide_kernel"): 9299840, ("cfg4_T16", "tall_kernel"): 83354880,
                ("cfg3_T2048", "prefill_kernel"): 52772608}
 METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
@@ -541,7 +541,7 @@ def main():
     # `achieved`.
     path, kernels_per_forward = lopro.linear_fwd_path(d, T)
     path_name = lopro.PATH_NAMES.get(path, "?")
-    kernel_name = {"stream": "stream_kernel", "tall": "tall_kernel", "general": "decode_kernel",
+    kernel_name = {"stream": "stream_kernel", "wide": "stream_wide_kernel", "tall": "tall_kernel", "general": "decode_kernel",
                    "prefill": "prefill_kernel"}.get(path_name, "?")
     note = "duration = step time / layer forwards (includes the prologue kernels)"
     launches_per_step = ring

@@ -180,6 +180,7 @@ LOPRO_API lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* pack
  * implementation detail of this library, exposed so that tests and benchmarks can name what they
  * measure; the paper's Appendix A.3 lists the steps, not their grouping into launches).
  *   LOPRO_PATH_STREAM   2 launches: prologue (permutation, rotation, B x) + streaming product, T <= 32
+ *   LOPRO_PATH_WIDE     the same with the 32-warp variant of the streaming kernel (T <= 8, all of K in the ring)
  *   LOPRO_PATH_TALL     the same with the persistent streaming kernel for layers with many output rows
  *   LOPRO_PATH_GENERAL  rotation, B x, register-ring product (any shape the descriptor allows)
  *   LOPRO_PATH_PREFILL  rotation, B x (2 launches), tcgen05 product, T > 32
@@ -189,7 +190,8 @@ typedef enum {
     LOPRO_PATH_STREAM = 2,
     LOPRO_PATH_GENERAL = 3,
     LOPRO_PATH_PREFILL = 4,
-    LOPRO_PATH_TALL = 5
+    LOPRO_PATH_TALL = 5,
+    LOPRO_PATH_WIDE = 6
 } lopro_path;
 LOPRO_API int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches);
 

@@ -205,7 +205,7 @@ int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launch
     if (!desc || check_desc(*desc) != LOPRO_OK || desc->layout != LOPRO_LAYOUT_FRAGMENT || T < 1) return 0;
     int32_t path, n;
     if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
-        path = use_tall(*desc, T) ? LOPRO_PATH_TALL : LOPRO_PATH_STREAM;
+        path = use_tall(*desc, T) ? LOPRO_PATH_TALL : (stream_uses_wide(*desc, T) ? LOPRO_PATH_WIDE : LOPRO_PATH_STREAM);
         n = 2;
     } else {
         const int pre = (T > kDecodeMaxT && rotate_lowrank_supported(*desc, T))

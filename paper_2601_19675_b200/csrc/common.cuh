@@ -111,6 +111,7 @@ cudaError_t launch_decode(const lopro_desc& d, const uint8_t* blob, const BlobLa
                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
 // Small-batch forward (T <= 32) after launch_prologue: bulk-copy ring, one CTA per 32 output rows.
 bool stream_supported(const lopro_desc& d, int T);
+bool stream_uses_wide(const lopro_desc& d, int T);  // the 32-warp variant of the kernel will run
 cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
 

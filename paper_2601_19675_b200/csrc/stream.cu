@@ -549,6 +549,23 @@ bool plan_layout(const lopro_desc& d, StreamPlan* pl, int r_pad, int ng, int kto
 
 }  // namespace
 
+// The 32-warp variant runs for up to 8 tokens when all of K fits the ring; LOPRO_NO_WIDE=1 keeps it off (A/B
+// comparison and tests).
+static bool wide_variant(const lopro_desc& d, const StreamPlan& pl) {
+    static int no_wide = -1;
+    if (no_wide < 0) {
+        const char* e = getenv("LOPRO_NO_WIDE");
+        no_wide = (e != nullptr && e[0] == '1') ? 1 : 0;
+    }
+    return !no_wide && pl.nt == 1 && pl.rt == 2 && pl.n_stages == pl.total_stages &&
+           pl.off_stage_x == 2 * kStageSteps * 128 * d.bits;  // the variant's compile-time stage geometry
+}
+
+bool stream_uses_wide(const lopro_desc& d, int T) {
+    StreamPlan pl;
+    return plan_stream(d, T, &pl) && wide_variant(d, pl);
+}
+
 bool stream_supported(const lopro_desc& d, int T) {
     StreamPlan pl;
     return plan_stream(d, T, &pl);
@@ -586,13 +603,7 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
     p.off_ring = pl.off_ring;
     p.stage_bytes = pl.stage_bytes;
     p.off_stage_x = pl.off_stage_x;
-    static int no_wide = -1;  // LOPRO_NO_WIDE=1 keeps the 32-warp variant off (A/B comparison and tests)
-    if (no_wide < 0) {
-        const char* e = getenv("LOPRO_NO_WIDE");
-        no_wide = (e != nullptr && e[0] == '1') ? 1 : 0;
-    }
-    if (!no_wide && pl.nt == 1 && pl.rt == 2 && pl.n_stages == pl.total_stages &&
-        pl.off_stage_x == 2 * kStageSteps * 128 * d.bits) {  // the variant's compile-time stage geometry
+    if (wide_variant(d, pl)) {
         switch (d.bits) {
             case 2: return launch_stream_wide<2>(p, pl.smem_bytes, s);
             case 3: return launch_stream_wide<3>(p, pl.smem_bytes, s);

@@ -119,8 +119,8 @@ def workspace_bytes(desc, T):
     return int(lib().lopro_workspace_bytes(ctypes.byref(desc), int(T)))
 
 
-PATH_STREAM, PATH_GENERAL, PATH_PREFILL, PATH_TALL = 2, 3, 4, 5
-PATH_NAMES = {PATH_TALL: "tall", PATH_STREAM: "stream", PATH_GENERAL: "general", PATH_PREFILL: "prefill"}
+PATH_STREAM, PATH_GENERAL, PATH_PREFILL, PATH_TALL, PATH_WIDE = 2, 3, 4, 5, 6
+PATH_NAMES = {PATH_TALL: "tall", PATH_WIDE: "wide", PATH_STREAM: "stream", PATH_GENERAL: "general", PATH_PREFILL: "prefill"}
 
 
 def linear_fwd_path(desc, T):

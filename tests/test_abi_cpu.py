@@ -88,7 +88,8 @@ def test_workspace_size_is_monotone_in_tokens():
 
 def test_forward_path_query_names_the_small_batch_and_general_paths():
     d = lopro.make_desc(4096, 4096, 4, 128, 128, rank=32)
-    assert lopro.linear_fwd_path(d, 8) == (lopro.PATH_STREAM, 2)       # prologue + streaming kernel
+    assert lopro.linear_fwd_path(d, 8) == (lopro.PATH_WIDE, 2)         # prologue + streaming kernel, 32-warp variant
+    assert lopro.linear_fwd_path(d, 16) == (lopro.PATH_STREAM, 2)      # prologue + streaming kernel
     assert lopro.linear_fwd_path(d, 0) == (0, 0) and lopro.linear_fwd_path(d, -3) == (0, 0)
     wide = lopro.make_desc(4096, 4096, 4, 128, 1024, identity_cols=0, rank=32)  # b_H beyond the prologue's 256
     path, launches = lopro.linear_fwd_path(wide, 8)

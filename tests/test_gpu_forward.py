@@ -136,7 +136,7 @@ def test_tall_kernel_agrees_with_the_per_group_kernel(monkeypatch):
     x = bf16_bits_to_device(synth.activations(T, n, seed=4))
     y_tall = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
     monkeypatch.setenv("LOPRO_NO_TALL", "1")
-    assert lopro.linear_fwd_path(d, T)[0] == lopro.PATH_STREAM
+    assert lopro.linear_fwd_path(d, T)[0] in (lopro.PATH_STREAM, lopro.PATH_WIDE)
     y_stream = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
     torch.cuda.synchronize()
     scale = y_stream.abs().max().item()
