@@ -148,7 +148,7 @@ lowrank_down_mma_kernel(const __half* __restrict__ B, const __nv_bfloat16* __res
 // the rest are the (token tile, K slice) CTAs of the down-projection).  Launched with programmatic stream
 // serialization: the dependents may be scheduled at once, the activations are read after the wait.
 template <int NJ>
-__global__ void __launch_bounds__(kLrThreads)
+__global__ void __launch_bounds__(kLrThreads, NJ <= 8 ? 3 : 2)
 rotate_lowrank_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
                       __nv_bfloat16* __restrict__ xrot, int64_t ldo, float* __restrict__ s64, int s64_ld,
                       int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int T, int n_rot,
