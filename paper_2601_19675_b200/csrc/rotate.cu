@@ -303,10 +303,13 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
                             int* status, int T, cudaStream_t s) {
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
     cudaLaunchConfig_t cfg = {};
-    // tokens per row CTA: as few as it takes to put about one CTA on every SM
+    // tokens per row CTA: as few as it takes to fill the SMs
     const int live = T < 8 ? T : 8;
     int tpr = 8;
-    while (tpr > 1 && r_pad * ((live + tpr - 1) / tpr) * ((T + 7) / 8) < 120) tpr >>= 1;
+    // (measured: with one group of tokens a CTA per (row, token) is best -- 256 CTAs for cfg2 --, with several
+    // groups about one CTA per SM)
+    const int want = T <= 8 ? 256 : 120;
+    while (tpr > 1 && r_pad * ((live + tpr - 1) / tpr) * ((T + 7) / 8) < want) tpr >>= 1;
     const int row_ctas = d.rank > 0 ? r_pad * ((live + tpr - 1) / tpr) : 0;
     cfg.gridDim = dim3((d.d_in + 255) / 256 + row_ctas, (T + 7) / 8);
     cfg.blockDim = dim3(256);
