@@ -109,6 +109,17 @@ def test_small_batch_path_row_and_token_edges(bits, g, T, n, m, r, b):
     _check_forward(layer, d, synth.activations(T, n, seed=T + 3, outlier_frac=0.01))
 
 
+@pytest.mark.parametrize("r", [40, 64, 128, 256])
+@pytest.mark.parametrize("T", [3, 8])
+def test_prologue_row_ctas_for_one_two_four_and_eight_tokens(r, T):
+    # the prologue gives a row CTA of t = B x 1, 2, 4 or 8 tokens depending on the padded rank (48, 64, 128, 256 here)
+    n, m, bits, g = 2304, 80, 4, 128                          # 36 steps: a ragged third stage; 80 rows: half-empty CTA
+    d = lopro.make_desc(n, m, bits, g, 128, identity_cols=128, rank=r)
+    assert lopro.linear_fwd_path(d, T)[0] == lopro.PATH_WIDE
+    layer = random_layer_np(n, m, bits, g, r, seed=r + T)
+    _check_forward(layer, d, synth.activations(T, n, seed=r, outlier_frac=0.01))
+
+
 def _tall_rows(tiles_per_sm, extra_tiles):
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     return 16 * (sms * tiles_per_sm + extra_tiles)
