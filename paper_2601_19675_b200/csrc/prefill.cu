@@ -335,11 +335,14 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                 const uint64_t db = make_desc_sw128(b_tile);
                 const bool lowrank = s >= p.nsteps;
                 const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
-                for (int acc = 0; acc < n_acc; ++acc) {
-                    const uint64_t da = make_desc_sw128(a_tile + acc * kABlock);
-                    for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
-                        umma_f16(tmem + (uint32_t)(acc * 256), da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
-                                 lowrank ? idesc_lr : idesc_w, (s > 0 || k > 0) ? 1u : 0u);
+                // the two accumulators alternate, so that consecutive MMAs never write the same accumulator
+                const uint64_t da0 = make_desc_sw128(a_tile), da1 = make_desc_sw128(a_tile + kABlock);
+                for (int k = 0; k < ksub; ++k) {  // 16 columns = 32 bytes = 2 descriptor address units
+                    const uint32_t accumulate = (s > 0 || k > 0) ? 1u : 0u;
+                    umma_f16(tmem, da0 + (uint64_t)(2 * k), db + (uint64_t)(2 * k), lowrank ? idesc_lr : idesc_w, accumulate);
+                    if (n_acc == 2)
+                        umma_f16(tmem + 256u, da1 + (uint64_t)(2 * k), db + (uint64_t)(2 * k), lowrank ? idesc_lr : idesc_w,
+                                 accumulate);
                 }
                 umma_commit(empty_a(sa));  // the slots may be refilled once these MMAs have read them
                 umma_commit(empty_b(sb));
