@@ -168,6 +168,23 @@ def test_outputs_can_be_strided_and_calls_repeat_bitwise():
     assert torch.count_nonzero(ybuf[:, m:]) == 0
 
 
+@pytest.mark.parametrize("T,pad", [(8, 3), (16, 5), (40, 3), (300, 8), (300, 1)])
+def test_strided_outputs_on_every_path(T, pad):
+    # y with a row stride that is not the row length: odd strides take the scalar stores of the prefill epilogue,
+    # strides that are multiples of 8 its 16-byte stores; the columns beyond m must stay untouched
+    n, m, bits, g, r = 1024, 16 * (2 * torch.cuda.get_device_properties(0).multi_processor_count + 3) if T == 16 else 400, 4, 128, 16
+    d = lopro.make_desc(n, m, bits, g, 128, rank=r)
+    layer = random_layer_np(n, m, bits, g, r, seed=T + pad)
+    blob = _pack(layer, d)
+    x = bf16_bits_to_device(synth.activations(T, n, seed=pad))
+    y_ref = lopro.linear_fwd(d, blob, x)
+    ybuf = torch.full((T, m + pad), 7.0, dtype=torch.bfloat16, device="cuda")
+    lopro.linear_fwd(d, blob, x, y=ybuf[:, :m])
+    torch.cuda.synchronize()
+    assert torch.equal(ybuf[:, :m], y_ref)
+    assert torch.all(ybuf[:, m:] == 7.0)
+
+
 def test_forward_argument_errors():
     n, m = 512, 64
     layer = random_layer_np(n, m, 4, 128, 0, seed=1)
