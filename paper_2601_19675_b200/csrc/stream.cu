@@ -286,12 +286,16 @@ stream_kernel(const StreamParams p) {
 constexpr int kWideWarps = 32;
 constexpr int kWideThreads = kWideWarps * 32;
 
+// Partial sums of the 16 step warps of a tile, red[step][token][row] with padded strides: the four token pairs of
+// a warp's store fall into different banks, and so do the four partial sums that a thread adds afterwards.
+constexpr int kRedTok = 36;                 // floats between tokens
+constexpr int kRedStep = 8 * kRedTok + 8;   // floats between steps
+
 template <int BITS>
 __global__ void __launch_bounds__(kWideThreads, 1)
 stream_wide_kernel(const StreamParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t bars[2 * kMaxStages + 2];  // wfull, xfull per stage; sz + A; t
-    __shared__ int s_timeout;
+    __shared__ __align__(8) uint64_t bars[kMaxStages + 2];  // full per stage (codes and activations); sz + A; t
     constexpr int kTok = 8;
     constexpr int kStepBytes = 128 * BITS;
     // stage geometry of this variant (8 tokens, two row tiles) as compile-time constants: the unrolled stage loop
@@ -306,21 +310,16 @@ stream_wide_kernel(const StreamParams p) {
     const int n_rt = min(2, (p.m >> 4) - rt0);
     const int tc = min(kTok, p.T);
     const uint32_t bar0 = smem_u32(bars);
-    auto wfull = [&](int s) { return bar0 + 8u * (uint32_t)s; };
-    auto xfull = [&](int s) { return bar0 + 8u * (uint32_t)(kMaxStages + s); };
-    const uint32_t cbar = bar0 + 8u * (uint32_t)(2 * kMaxStages);
+    auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    const uint32_t cbar = bar0 + 8u * (uint32_t)kMaxStages;
     const uint32_t tbar = cbar + 8u;
     const uint32_t smem0 = smem_u32(smem);
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
-        for (int s = 0; s < p.total_stages; ++s) {
-            mbar_init(wfull(s), 1);
-            mbar_init(xfull(s), 1);
-        }
+        for (int s = 0; s < p.total_stages; ++s) mbar_init(full(s), 2);  // two arrivals: codes, activations
         mbar_init(cbar, 1);
         mbar_init(tbar, 1);
-        s_timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -335,21 +334,21 @@ stream_wide_kernel(const StreamParams p) {
         if (a_bytes) bulk_g2s(smem0 + p.off_a, p.A + (size_t)rt0 * 16 * p.r_pad, a_bytes, cbar);
         for (int s = 0; s < p.total_stages; ++s) {
             const uint32_t bytes = (uint32_t)(steps_of(s) * kStepBytes);
-            mbar_expect_tx(wfull(s), bytes * (uint32_t)n_rt);
+            mbar_expect_tx(full(s), bytes * (uint32_t)n_rt);
             for (int q = 0; q < n_rt; ++q)
                 bulk_g2s(smem0 + p.off_ring + s * kStageBytes + q * kStageSteps * kStepBytes,
                          reinterpret_cast<const unsigned char*>(p.codes) +
                              ((size_t)(rt0 + q) * p.nsteps + (size_t)s * kStageSteps) * kStepBytes,
-                         bytes, wfull(s));
+                         bytes, full(s));
         }
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 0) {
         const uint32_t bytes = (uint32_t)(tc * kActRecord);
         for (int s = 0; s < p.total_stages; ++s) {
-            mbar_expect_tx(xfull(s), bytes);
+            mbar_expect_tx(full(s), bytes);
             bulk_g2s(smem0 + p.off_ring + s * kStageBytes + kOffX, p.act + (size_t)s * p.t_pad * kActRecord, bytes,
-                     xfull(s));
+                     full(s));
         }
         if (p.r_pad > 0) {
             const uint32_t t_bytes = (uint32_t)(tc * p.r_pad * 2);
@@ -358,15 +357,24 @@ stream_wide_kernel(const StreamParams p) {
         }
     }
 
-    float yacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    // Everything a warp needs to address its tile steps, worked out while the copies are in flight: the stage
+    // loop below adds compile-time offsets only.
     const bool live = r < n_rt;
-    if (!mbar_wait(cbar, 0)) {
-        s_timeout = 1;
-        if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
-    }
+    const int my_stages = live ? min(p.total_stages, (p.nsteps - step + kStageSteps - 1) / kStageSteps) : 0;
+    const unsigned char* ring = smem + p.off_ring;
+    const unsigned char* wptr = ring + (r * kStageSteps + step) * kStepBytes + lane * (BITS * 4);
+    const uint32_t xaddr = smem0 + p.off_ring + kOffX + (uint32_t)(step * 64) * 2u +
+                           (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
+    const float* sxp = reinterpret_cast<const float*>(ring + kOffX + 2048 + (2 * tg) * kActRecord) + step;
+    const uint32_t* szp = reinterpret_cast<const uint32_t*>(smem + p.off_sz) + (r * p.ng + (step >> p.gshift)) * 16 + gq;
+    const int sz_stage = (kStageSteps >> p.gshift) * 16;  // (scale, zero) words between the stages of a warp
+    bool timed_out = false;
+
+    float yacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    if (!mbar_wait(cbar, 0)) timed_out = true;
     if (p.r_pad > 0 && step == 0) {
         // low-rank term A t of row tile r starts the sums of its step-0 warp
-        if (!mbar_wait(tbar, 0) && lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+        if (!mbar_wait(tbar, 0)) timed_out = true;
         if (live) {
             const __half* as = reinterpret_cast<const __half*>(smem + p.off_a) + (size_t)r * 16 * p.r_pad;
             const __half* ts = reinterpret_cast<const __half*>(smem + p.off_t);
@@ -381,76 +389,67 @@ stream_wide_kernel(const StreamParams p) {
             }
         }
     }
-    const uint32_t* szs = reinterpret_cast<const uint32_t*>(smem + p.off_sz);
-    const uint32_t ldm_off = (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
-    const unsigned char* ring = smem + p.off_ring;
-    const uint32_t ring_u32 = smem0 + p.off_ring;
-#pragma unroll 4
-    for (int s = 0; s < p.total_stages; ++s) {
-        if (!s_timeout && !(mbar_wait(wfull(s), 0) && mbar_wait(xfull(s), 0))) {
-            s_timeout = 1;
-            if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
-        }
-        if (live && step < steps_of(s)) {
-            const unsigned char* stage = ring + s * kStageBytes;
-            const uint32_t xs_u32 = ring_u32 + s * kStageBytes + kOffX;
-            const unsigned char* srec = stage + kOffX + 2048;  // sums of token 0
-            const int grp = (s * kStageSteps + step) >> p.gshift;
-            uint32_t b[8];
-            const uint32_t base = xs_u32 + (uint32_t)(step * 64) * 2u + ldm_off;
-            ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[0]), base);
-            ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[4]), base + 64u);
-            const float sx0 = reinterpret_cast<const float*>(srec + (2 * tg) * kActRecord)[step];
-            const float sx1 = reinterpret_cast<const float*>(srec + (2 * tg + 1) * kActRecord)[step];
-            uint32_t w[BITS];
-            const uint32_t* wp = reinterpret_cast<const uint32_t*>(stage + (r * kStageSteps + step) * kStepBytes) + lane * BITS;
-            if constexpr (BITS == 4) {
-                const uint4 v = *reinterpret_cast<const uint4*>(wp);
-                w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-            } else if constexpr (BITS == 2) {
-                const uint2 v = *reinterpret_cast<const uint2*>(wp);
-                w[0] = v.x; w[1] = v.y;
-            } else {
 #pragma unroll
-                for (int q = 0; q < BITS; ++q) w[q] = wp[q];
-            }
-            uint32_t a[16];
-            expand_codes<BITS>(a, w);
-            const uint32_t sz_lo = szs[(r * p.ng + grp) * 16 + gq], sz_hi = szs[(r * p.ng + grp) * 16 + gq + 8];
-            const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
-            const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
-            const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
-            float acc[4];
-            mma_bf16_first(acc, &a[0], b[0], b[1]);
-            mma_bf16(acc, &a[4], b[2], b[3]);
-            mma_bf16(acc, &a[8], b[4], b[5]);
-            mma_bf16(acc, &a[12], b[6], b[7]);
-            yacc[0] = fmaf(f_lo.x, acc[0], fmaf(nsz_lo, sx0, yacc[0]));
-            yacc[1] = fmaf(f_lo.x, acc[1], fmaf(nsz_lo, sx1, yacc[1]));
-            yacc[2] = fmaf(f_hi.x, acc[2], fmaf(nsz_hi, sx0, yacc[2]));
-            yacc[3] = fmaf(f_hi.x, acc[3], fmaf(nsz_hi, sx1, yacc[3]));
+    for (int s = 0; s < kMaxStages; ++s) {
+        if (s >= my_stages) break;
+        if (!mbar_wait(full(s), 0)) timed_out = true;
+        uint32_t b[8];
+        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[0]), xaddr + s * kStageBytes);
+        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[4]), xaddr + s * kStageBytes + 64u);
+        const float sx0 = sxp[s * (kStageBytes / 4)];
+        const float sx1 = sxp[s * (kStageBytes / 4) + kActRecord / 4];
+        uint32_t w[BITS];
+        const uint32_t* wp = reinterpret_cast<const uint32_t*>(wptr + s * kStageBytes);
+        if constexpr (BITS == 4) {
+            const uint4 v = *reinterpret_cast<const uint4*>(wp);
+            w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        } else if constexpr (BITS == 2) {
+            const uint2 v = *reinterpret_cast<const uint2*>(wp);
+            w[0] = v.x; w[1] = v.y;
+        } else {
+#pragma unroll
+            for (int q = 0; q < BITS; ++q) w[q] = wp[q];
         }
+        uint32_t a[16];
+        expand_codes<BITS>(a, w);
+        const uint32_t sz_lo = szp[s * sz_stage], sz_hi = szp[s * sz_stage + 8];
+        const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
+        const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
+        const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
+        float acc[4];
+        mma_bf16_first(acc, &a[0], b[0], b[1]);
+        mma_bf16(acc, &a[4], b[2], b[3]);
+        mma_bf16(acc, &a[8], b[4], b[5]);
+        mma_bf16(acc, &a[12], b[6], b[7]);
+        yacc[0] = fmaf(f_lo.x, acc[0], fmaf(nsz_lo, sx0, yacc[0]));
+        yacc[1] = fmaf(f_lo.x, acc[1], fmaf(nsz_lo, sx1, yacc[1]));
+        yacc[2] = fmaf(f_hi.x, acc[2], fmaf(nsz_hi, sx0, yacc[2]));
+        yacc[3] = fmaf(f_hi.x, acc[3], fmaf(nsz_hi, sx1, yacc[3]));
     }
-    __syncthreads();  // every stage consumed: the ring can be reused for the reduction
+    if (timed_out && lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+    // Every stage has a step-0 warp that waited for it, so after this barrier every copy has landed and the ring
+    // can be reused for the reduction.
+    __syncthreads();
 
-    // reduction over the 16 steps of a tile: red[step][token][32 rows]
     float* red = reinterpret_cast<float*>(smem + p.off_ring);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int tk = 2 * tg + (i & 1), rl = r * 16 + gq + 8 * (i >> 1);
-        red[(step * kTok + tk) * 32 + rl] = yacc[i];
+        red[step * kRedStep + tk * kRedTok + rl] = yacc[i];
     }
     __syncthreads();
-    const int rows_here = n_rt * 16;
-    for (int i = tid; i < tc * 32; i += kWideThreads) {
-        const int tk = i >> 5, rl = i & 31;
-        if (rl < rows_here) {
-            float sum = 0.0f;
-#pragma unroll
-            for (int w = 0; w < 16; ++w) sum += red[(w * kTok + tk) * 32 + rl];
-            const size_t o = (size_t)tk * p.ldy + (size_t)rt0 * 16 + rl;
-            if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = sum;
-            else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(sum);
+    // four threads per output: each adds four of the 16 partial sums, two shuffles finish
+    {
+        const int o = tid >> 2, part = tid & 3;
+        const int tk = o >> 5, rl = o & 31;
+        const float* src = red + part * kRedStep + tk * kRedTok + rl;
+        float sum = (src[0] + src[4 * kRedStep]) + (src[8 * kRedStep] + src[12 * kRedStep]);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        if (part == 0 && tk < tc && rl < n_rt * 16) {
+            const size_t idx = (size_t)tk * p.ldy + (size_t)rt0 * 16 + rl;
+            if (p.out_f32) reinterpret_cast<float*>(p.y)[idx] = sum;
+            else reinterpret_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(sum);
         }
     }
 }
