@@ -178,41 +178,49 @@ stream_kernel(const StreamParams p) {
             for (int r = 0; r < RT; ++r)
                 if (warp == r) lowrank_up(yacc[r], r);
         }
-        const uint32_t* szs = reinterpret_cast<const uint32_t*>(smem + p.off_sz);
-        const uint32_t ldm_off = (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
+        // Offsets of what this warp (step `warp` of every stage) reads, from the start of a stage; the stage loop
+        // keeps a running slot, parity and address instead of dividing by the ring depth.
+        const uint32_t wofs = (uint32_t)(warp * kStepBytes + lane * (BITS * 4));
+        const uint32_t xofs = (uint32_t)p.off_stage_x + (uint32_t)(warp * 64) * 2u +
+                              (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
+        const uint32_t sxofs = (uint32_t)(p.off_stage_x + 2048 + 2 * tg * kActRecord + warp * 4);
+        const uint32_t* szs = reinterpret_cast<const uint32_t*>(smem + p.off_sz) + gq;
+        const int sz_tile = p.ng * 16;  // (scale, zero) words between row tiles
+        int kstep = warp;               // this warp's 64-column step of the current stage
+        int slot = 0;
+        uint32_t parity = 0;
+        const unsigned char* stage = smem + p.off_ring;
+        uint32_t stage_u32 = smem0 + (uint32_t)p.off_ring;
+        bool dead = false;  // a wait of this warp ran out
+        int steps_left = p.nsteps;
         for (int s = 0; s < p.total_stages; ++s) {
-            const int slot = s % p.n_stages;
-            const uint32_t parity = (uint32_t)(s / p.n_stages) & 1u;
-            if (!s_timeout && !(mbar_wait(wfull(slot), parity) && mbar_wait(xfull(slot), parity))) {
+            if (!dead && !(mbar_wait(wfull(slot), parity) && mbar_wait(xfull(slot), parity))) {
+                dead = true;
                 s_timeout = 1;
                 if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
             }
-            const int steps = steps_of(s);
-            if (warp < steps) {
-                const unsigned char* stage = smem + p.off_ring + slot * p.stage_bytes;
-                const uint32_t xs_u32 = smem0 + p.off_ring + slot * p.stage_bytes + p.off_stage_x;
-                const unsigned char* srec = stage + p.off_stage_x + 2048;  // sums of token 0
-                const int grp = (s * kStageSteps + warp) >> p.gshift;
+            if (warp < steps_left) {
                 // B operand: the 64 columns of step `warp`, all token tiles
                 uint32_t b[NT][8];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    const uint32_t base = xs_u32 + (uint32_t)(nt * 8 * kXsStride + warp * 64) * 2u + ldm_off;
+                    const uint32_t base = stage_u32 + xofs + (uint32_t)(nt * 8 * kXsStride) * 2u;
                     ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][0]), base);
                     ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][4]), base + 64u);
                 }
+                const float* sxp = reinterpret_cast<const float*>(stage + sxofs);
+                const uint32_t* szp = szs + (kstep >> p.gshift) * 16;
                 float sx[NT][2];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    sx[nt][0] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg) * kActRecord)[warp];
-                    sx[nt][1] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg + 1) * kActRecord)[warp];
+                    sx[nt][0] = sxp[nt * 8 * (kActRecord / 4)];
+                    sx[nt][1] = sxp[(nt * 8 + 1) * (kActRecord / 4)];
                 }
 #pragma unroll
                 for (int r = 0; r < RT; ++r) {
                     if (r < n_rt) {
                         uint32_t w[BITS];
-                        const uint32_t* wp = reinterpret_cast<const uint32_t*>(stage + (r * kStageSteps + warp) * kStepBytes) +
-                                             lane * BITS;
+                        const uint32_t* wp = reinterpret_cast<const uint32_t*>(stage + wofs + r * kStageSteps * kStepBytes);
                         if constexpr (BITS == 4) {
                             const uint4 v = *reinterpret_cast<const uint4*>(wp);
                             w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
@@ -225,7 +233,7 @@ stream_kernel(const StreamParams p) {
                         }
                         uint32_t a[16];
                         expand_codes<BITS>(a, w);
-                        const uint32_t sz_lo = szs[(r * p.ng + grp) * 16 + gq], sz_hi = szs[(r * p.ng + grp) * 16 + gq + 8];
+                        const uint32_t sz_lo = szp[r * sz_tile], sz_hi = szp[r * sz_tile + 8];
                         const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
                         const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
                         const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
@@ -246,6 +254,18 @@ stream_kernel(const StreamParams p) {
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty(slot));
+            // next stage: its steps, its slot of the ring
+            kstep += kStageSteps;
+            steps_left -= kStageSteps;
+            ++slot;
+            stage += p.stage_bytes;
+            stage_u32 += (uint32_t)p.stage_bytes;
+            if (slot == p.n_stages) {
+                slot = 0;
+                parity ^= 1u;
+                stage = smem + p.off_ring;
+                stage_u32 = smem0 + (uint32_t)p.off_ring;
+            }
         }
     }
     __syncthreads();  // every stage consumed: the ring can be reused for the reduction
@@ -366,8 +386,7 @@ stream_wide_kernel(const StreamParams p) {
     const uint32_t xaddr = smem0 + p.off_ring + kOffX + (uint32_t)(step * 64) * 2u +
                            (uint32_t)((lane & 7) * kXsStride + (lane >> 3) * 8) * 2u;
     const float* sxp = reinterpret_cast<const float*>(ring + kOffX + 2048 + (2 * tg) * kActRecord) + step;
-    const uint32_t* szp = reinterpret_cast<const uint32_t*>(smem + p.off_sz) + (r * p.ng + (step >> p.gshift)) * 16 + gq;
-    const int sz_stage = (kStageSteps >> p.gshift) * 16;  // (scale, zero) words between the stages of a warp
+    const uint32_t* szs = reinterpret_cast<const uint32_t*>(smem + p.off_sz) + r * p.ng * 16 + gq;
     bool timed_out = false;
 
     float yacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -412,7 +431,8 @@ stream_wide_kernel(const StreamParams p) {
         }
         uint32_t a[16];
         expand_codes<BITS>(a, w);
-        const uint32_t sz_lo = szp[s * sz_stage], sz_hi = szp[s * sz_stage + 8];
+        const uint32_t* szp = szs + ((s * kStageSteps + step) >> p.gshift) * 16;  // the step's group
+        const uint32_t sz_lo = szp[0], sz_hi = szp[8];
         const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
         const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
         const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
@@ -431,6 +451,7 @@ stream_wide_kernel(const StreamParams p) {
     // can be reused for the reduction.
     __syncthreads();
 
+    static_assert(kStageSteps * kRedStep * 4 <= kStageBytes, "the partial sums fit one stage of the ring");
     float* red = reinterpret_cast<float*>(smem + p.off_ring);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {

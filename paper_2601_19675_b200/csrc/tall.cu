@@ -69,26 +69,24 @@ __device__ __forceinline__ void named_arrive(int id) {
 
 // One 16-row tile times one 64-column step: expand the packed codes to bf16 operands 128 + c, four
 // m16n8k16 products per token tile, then scale and zero-point in fp32 against the 64-column sums.
+// wp: the lane's words of the step; xaddr: the lane's ldmatrix row of the step (shared-space address);
+// sxp: the step's 64-column sum of token 2 * tg; szp: the (scale, zero) pair of row gq in the step's group.
 template <int BITS, int NT>
-__device__ __forceinline__ void tile_step(const unsigned char* codes_rt, const uint32_t* szs, const unsigned char* srec,
-                                          uint32_t xs_u32, int st, int gl, int lane, float (&yacc)[NT][4]) {
-    constexpr int kStepBytes = 128 * BITS;
-    const int gq = lane >> 2, tg = lane & 3;
+__device__ __forceinline__ void tile_step(const uint32_t* wp, uint32_t xaddr, const float* sxp, const uint32_t* szp,
+                                          float (&yacc)[NT][4]) {
     uint32_t b[NT][8];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        const uint32_t addr = xs_u32 + (uint32_t)(nt * 8 * kActRecord + st * 128);
-        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][0]), addr);
-        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][4]), addr + 64u);
+        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][0]), xaddr + (uint32_t)(nt * 8 * kActRecord));
+        ldmatrix_x4(*reinterpret_cast<uint32_t(*)[4]>(&b[nt][4]), xaddr + (uint32_t)(nt * 8 * kActRecord) + 64u);
     }
     float sx[NT][2];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        sx[nt][0] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg) * kActRecord)[st];
-        sx[nt][1] = reinterpret_cast<const float*>(srec + (nt * 8 + 2 * tg + 1) * kActRecord)[st];
+        sx[nt][0] = sxp[nt * 8 * (kActRecord / 4)];
+        sx[nt][1] = sxp[(nt * 8 + 1) * (kActRecord / 4)];
     }
     uint32_t w[BITS];
-    const uint32_t* wp = reinterpret_cast<const uint32_t*>(codes_rt + st * kStepBytes) + lane * BITS;
     if constexpr (BITS == 4) {
         const uint4 v = *reinterpret_cast<const uint4*>(wp);
         w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
@@ -101,7 +99,7 @@ __device__ __forceinline__ void tile_step(const unsigned char* codes_rt, const u
     }
     uint32_t a[16];
     expand_codes<BITS>(a, w);
-    const uint32_t sz_lo = szs[gl * 16 + gq], sz_hi = szs[gl * 16 + gq + 8];
+    const uint32_t sz_lo = szp[0], sz_hi = szp[8];
     const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
     const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
     const float nsz_lo = -f_lo.x * (128.0f + f_lo.y), nsz_hi = -f_hi.x * (128.0f + f_hi.y);
@@ -119,25 +117,30 @@ __device__ __forceinline__ void tile_step(const unsigned char* codes_rt, const u
     }
 }
 
-// The steps kq, kq + KQ, ... of one stage for tile slot r (KQ = 16 >> RBITS phases): unrolled with
-// constant strides for a full stage, a plain loop for the ragged last one.
+// Byte offsets, from the start of a stage, of what a warp reads in its first step (step kq of tile slot r); they
+// change only when the split of the warps changes, i.e. once per group of tiles.
+struct WarpOffsets {
+    uint32_t w, x, sx, sz;
+};
+
+// The steps kq, kq + KQ, ... of one stage for tile slot r (KQ = 16 >> RBITS phases), unrolled with constant
+// strides; gs = min(gshift, 4): a stage starts on a group boundary or lies inside one group, so the group of
+// step st within the stage's (scale, zero) block is st >> gs.
 template <int BITS, int NT, int RBITS>
-__device__ __forceinline__ void consume_stage(const TallParams& p, const unsigned char* stage, uint32_t xs_u32, int r,
-                                              int kq, int s, int steps, int lane, float (&yacc)[NT][4]) {
+__device__ __forceinline__ void consume_stage(const unsigned char* stage, uint32_t stage_u32, const WarpOffsets& o, int kq,
+                                              int gs, int steps, float (&yacc)[NT][4]) {
     constexpr int KQ = kConsumerWarps >> RBITS, PER = kStageSteps / KQ;
-    const unsigned char* codes_rt = stage + r * kStageSteps * (128 * BITS);
-    const uint32_t* szs = reinterpret_cast<const uint32_t*>(stage + p.off_stage_sz + r * kSzTile);
-    const unsigned char* srec = stage + p.off_stage_x + 2048;  // sums of token 0
-    const int g0 = (s * kStageSteps) >> p.gshift;
-    if (steps == kStageSteps) {
+    constexpr int kStepBytes = 128 * BITS;
+    const unsigned char* wbase = stage + o.w;
+    const float* sxbase = reinterpret_cast<const float*>(stage + o.sx);
+    const uint32_t* szbase = reinterpret_cast<const uint32_t*>(stage + o.sz);
 #pragma unroll
-        for (int i = 0; i < PER; ++i) {
-            const int st = kq + i * KQ;
-            tile_step<BITS, NT>(codes_rt, szs, srec, xs_u32, st, ((s * kStageSteps + st) >> p.gshift) - g0, lane, yacc);
-        }
-    } else {
-        for (int st = kq; st < steps; st += KQ)
-            tile_step<BITS, NT>(codes_rt, szs, srec, xs_u32, st, ((s * kStageSteps + st) >> p.gshift) - g0, lane, yacc);
+    for (int i = 0; i < PER; ++i) {
+        const int st = kq + i * KQ;
+        if (st < steps)
+            tile_step<BITS, NT>(reinterpret_cast<const uint32_t*>(wbase + i * KQ * kStepBytes),
+                                stage_u32 + o.x + (uint32_t)(i * KQ * 128), sxbase + i * KQ, szbase + (st >> gs) * 16,
+                                yacc);
     }
 }
 
@@ -248,7 +251,13 @@ tall_kernel(const TallParams p) {
     const uint32_t ldm_off = (uint32_t)((lane & 7) * kActRecord + (lane >> 3) * 16);
     float* red = reinterpret_cast<float*>(smem + p.off_red);  // [writer][NT * 4][32 lanes]
     bool wrote_red = false;  // this warp handed sums over in an earlier group
-    int S = 0;
+    bool dead = false;       // a wait of this warp ran out
+    const int gs = min(p.gshift, 4);
+    // the ring slot of the next stage, its parity and its address
+    int slot = 0;
+    uint32_t phase = 0;
+    const unsigned char* stage = smem + p.off_ring;
+    uint32_t stage_u32 = smem0 + (uint32_t)p.off_ring;
     for (int gi = 0; gi < n_groups; ++gi) {
         const int tile0 = my_start + gi * p.gt;
         const int n_rt = min(p.gt, my_cnt - gi * p.gt);
@@ -293,22 +302,35 @@ tall_kernel(const TallParams p) {
             }
         }
 
-        for (int s = 0; s < TS; ++s, ++S) {
-            const int slot = S % p.n_stages;
-            if (!s_timeout && !mbar_wait(full(slot), (uint32_t)(S / p.n_stages) & 1u)) {
+        WarpOffsets wo;
+        wo.w = (uint32_t)((r * kStageSteps + kq) * kStepBytes + lane * (BITS * 4));
+        wo.x = (uint32_t)p.off_stage_x + ldm_off + (uint32_t)(kq * 128);
+        wo.sx = (uint32_t)(p.off_stage_x + 2048 + 2 * tg * kActRecord + kq * 4);
+        wo.sz = (uint32_t)(p.off_stage_sz + r * kSzTile + gq * 4);
+        for (int s = 0; s < TS; ++s) {
+            if (!dead && !mbar_wait(full(slot), phase)) {
+                dead = true;  // this warp stops waiting; its outputs are unspecified
                 s_timeout = 1;
                 if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
             }
             if (active) {
-                const unsigned char* stage = smem + p.off_ring + slot * p.stage_bytes;
-                const uint32_t xs_u32 = smem0 + p.off_ring + slot * p.stage_bytes + p.off_stage_x + ldm_off;
                 const int steps = steps_of(s);
-                if (rbits == 2) consume_stage<BITS, NT, 2>(p, stage, xs_u32, r, kq, s, steps, lane, yacc);
-                else if (rbits == 1) consume_stage<BITS, NT, 1>(p, stage, xs_u32, r, kq, s, steps, lane, yacc);
-                else consume_stage<BITS, NT, 0>(p, stage, xs_u32, r, kq, s, steps, lane, yacc);
+                if (rbits == 2) consume_stage<BITS, NT, 2>(stage, stage_u32, wo, kq, gs, steps, yacc);
+                else if (rbits == 1) consume_stage<BITS, NT, 1>(stage, stage_u32, wo, kq, gs, steps, yacc);
+                else consume_stage<BITS, NT, 0>(stage, stage_u32, wo, kq, gs, steps, yacc);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty(slot));
+            // next slot of the ring
+            ++slot;
+            stage += p.stage_bytes;
+            stage_u32 += (uint32_t)p.stage_bytes;
+            if (slot == p.n_stages) {
+                slot = 0;
+                phase ^= 1u;
+                stage = smem + p.off_ring;
+                stage_u32 = smem0 + (uint32_t)p.off_ring;
+            }
         }
 
         // ---- end of the group: the K phases of a tile meet in the warp kq = 0, which stores the rows ----

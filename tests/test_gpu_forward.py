@@ -138,6 +138,20 @@ def test_tall_layers_persistent_kernel(bits, g, r, T, per_sm, extra):
     _check_forward(layer, d, synth.activations(T, n, seed=T + 11, outlier_frac=0.01))
 
 
+@pytest.mark.parametrize("g", [1024, 2048, 4096])
+@pytest.mark.parametrize("T,m", [(8, 160), (16, 160), (8, None)])
+def test_groups_as_long_as_or_longer_than_a_stage(g, T, m):
+    # a stage of the small-batch kernels holds 1024 columns: groups of exactly one stage, of two stages and of
+    # the whole row (one scale per row), on the 32-warp, the 16-warp and the persistent kernel
+    n = 4096
+    m = _tall_rows(2, 5) if m is None else m
+    d = lopro.make_desc(n, m, 4, g, 128, identity_cols=128, rank=16)
+    want = {(8, False): lopro.PATH_WIDE, (16, False): lopro.PATH_STREAM, (8, True): lopro.PATH_TALL}[(T, m > 160)]
+    assert lopro.linear_fwd_path(d, T)[0] == want
+    layer = random_layer_np(n, m, 4, g, 16, seed=g + T)
+    _check_forward(layer, d, synth.activations(T, n, seed=T + g))
+
+
 def test_tall_kernel_agrees_with_the_per_group_kernel(monkeypatch):
     # both small-batch kernels sum the same products in fp32 in different orders: outputs agree to fp32 rounding
     n, m, bits, g, r, T = 1024, _tall_rows(4, 9), 4, 128, 32, 8
