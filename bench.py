@@ -74,7 +74,7 @@ def time_oracle_stack(T, budget_s):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
 # capture summarised in profiles/; valid for the kernel as committed with that summary, null otherwise.
-NCU_TRAFFIC = {("cfg2_T8", "stream_wide_kernel"): 9300096, ("cfg4_T16", "tall_kernel"): 83239040,
+NCU_TRAFFIC = {("cfg2_T8", "stream_wide_kernel"): 9296640, ("cfg4_T16", "tall_kernel"): 83635840,
                ("cfg3_T2048", "prefill_kernel"): 53210752}
 METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
