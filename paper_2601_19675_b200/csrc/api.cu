@@ -201,10 +201,33 @@ static bool use_tall(const lopro_desc& d, int T) {
     return tall_supported(d, T);
 }
 
+// Token counts a little above the small-batch range run as chunks of kDecodeMaxT tokens through the small-batch
+// kernels when that costs less than the tensor-core path: a prefill CTA walks all of K for its 128 or 256 rows
+// whatever the token count, and a layer with few rows fills few SMs.  Both sides are estimated from timings on
+// B200 (microseconds): a chunk 4 + 0.6e-6 d_out d_in (15 for 4096 x 4096, 25-32 for 4096 x 11008 either way
+// round), the prefill chain 8 + 0.017 d_in per wave of CTAs (74 for d_in = 4096, 205 for 11008, flat from 33 to
+// 256 tokens).  LOPRO_NO_CHUNKS=1 turns this off (A/B runs, tests of the prefill kernel on small layers).
+static int small_batch_chunks(const lopro_desc& d, int T) {
+    if (T <= kDecodeMaxT) return 0;
+    const char* e = getenv("LOPRO_NO_CHUNKS");
+    if (e && e[0] == '1') return 0;
+    if (!prefill_supported(d, T)) return 0;  // keep the general path's behaviour where there is no prefill kernel
+    const int chunks = (T + kDecodeMaxT - 1) / kDecodeMaxT;
+    const double chunk_us = 4.0 + 0.6e-6 * (double)d.d_out * (double)d.d_in;
+    const int ctas = ((d.d_out + 255) / 256) * ((T + 255) / 256);  // two 128-row blocks per CTA
+    const double prefill_us = 8.0 + 0.017 * (double)d.d_in * (double)((ctas + 147) / 148);
+    if ((double)chunks * chunk_us >= prefill_us) return 0;
+    if (!prologue_supported(d, kDecodeMaxT) || !stream_supported(d, kDecodeMaxT)) return 0;
+    return chunks;
+}
+
 int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches) {
     if (!desc || check_desc(*desc) != LOPRO_OK || desc->layout != LOPRO_LAYOUT_FRAGMENT || T < 1) return 0;
     int32_t path, n;
-    if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
+    if (const int chunks = small_batch_chunks(*desc, T)) {
+        path = use_tall(*desc, kDecodeMaxT) ? LOPRO_PATH_TALL : LOPRO_PATH_STREAM;
+        n = 2 * chunks;
+    } else if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
         path = use_tall(*desc, T) ? LOPRO_PATH_TALL : (stream_uses_wide(*desc, T) ? LOPRO_PATH_WIDE : LOPRO_PATH_STREAM);
         n = 2;
     } else {
@@ -246,6 +269,25 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     __nv_bfloat16* xrot = (__nv_bfloat16*)(ws + W.off_xrot);
     float* s64 = (float*)(ws + W.off_s64);
     int* status = (int*)(ws + W.off_status);
+    if (const int chunks = small_batch_chunks(*desc, T)) {
+        // chunks of kDecodeMaxT tokens through the small-batch kernels; the status word is reset by the first
+        // chunk's prologue only, so a time-out in any chunk stays recorded
+        const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;
+        for (int c = 0; c < chunks; ++c) {
+            const int t0 = c * kDecodeMaxT, tc = T - t0 < kDecodeMaxT ? T - t0 : kDecodeMaxT;
+            WorkspaceLayout Wc;  // never larger than the layout for all T tokens
+            if ((st = workspace_layout(*desc, tc, &Wc)) != LOPRO_OK) return st;
+            const __nv_bfloat16* xc = (const __nv_bfloat16*)x_bf16 + (size_t)t0 * ldx;
+            void* yc = (uint8_t*)y + (size_t)t0 * ldy * esz;
+            if (launch_prologue(*desc, perm, B, L.r_pad, xc, ldx, ws + Wc.off_xrot, (__half*)(ws + Wc.off_t), Wc.t_pad,
+                                c == 0 ? status : nullptr, tc, s) != cudaSuccess)
+                return LOPRO_ERR_CUDA;
+            const cudaError_t e = use_tall(*desc, tc) ? launch_tall(*desc, blob, L, ws, Wc, yc, ldy, out_dtype, tc, s)
+                                                      : launch_stream(*desc, blob, L, ws, Wc, yc, ldy, out_dtype, tc, s);
+            if (e != cudaSuccess) return LOPRO_ERR_CUDA;
+        }
+        return LOPRO_OK;
+    }
     if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
         // small batch: prologue + streaming kernel, chained by programmatic launches
         if (launch_prologue(*desc, perm, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot,

@@ -34,7 +34,7 @@ def _sampled(cfg, T, n_rows=48, seed=0):
     args = oracle_args(layer, d.group_size, d.identity_cols, d.block_size, rows=rows)
     x64 = o.bf16_bits_to_f64(x_bits[toks])
     exact = o.forward_exact(x64, **args)
-    mirrored = o.forward_mirrored(x64, **args, round_w=T > 32, round_t="f16", out="f32")
+    mirrored = o.forward_mirrored(x64, **args, round_w=lopro.linear_fwd_path(d, T)[0] == lopro.PATH_PREFILL, round_t="f16", out="f32")
     # error relative to the rms of the sampled entries of each token's row
     got_bf = device_bf16_to_f64(y_bf[torch.from_numpy(toks).cuda()])[:, rows]
     got_f32 = y_f32[torch.from_numpy(toks).cuda()].cpu().numpy().astype(np.float64)[:, rows]
