@@ -31,6 +31,7 @@ constexpr int kThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
 constexpr int kStageSteps = 16;                      // 64-column steps per stage = one per consumer warp
 constexpr int kXsStride = kActRecord / 2;            // bf16 elements between the token rows of a stage
 constexpr int kMaxStages = 8;
+constexpr int kRedPad = 4;  // floats of padding per token row of the reduction buffer
 
 struct StreamParams {
     const uint32_t* codes;
@@ -270,8 +271,9 @@ stream_kernel(const StreamParams p) {
     }
     __syncthreads();  // every stage consumed: the ring can be reused for the reduction
 
-    // reduction over the consumer warps: red[warp][token][RT * 16 rows]
-    constexpr int kRows = RT * 16;
+    // reduction over the consumer warps: red[warp][token][RT * 16 rows + 4] -- the padding puts the four token
+    // pairs of a warp's store into different banks
+    constexpr int kRows = RT * 16, kRowsP = kRows + kRedPad;
     float* red = reinterpret_cast<float*>(smem + p.off_ring);
     if (warp < kConsumerWarps) {
 #pragma unroll
@@ -281,7 +283,7 @@ stream_kernel(const StreamParams p) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int tk = nt * 8 + 2 * tg + (i & 1), rl = r * 16 + gq + 8 * (i >> 1);
-                    red[(warp * kTok + tk) * kRows + rl] = yacc[r][nt][i];
+                    red[(warp * kTok + tk) * kRowsP + rl] = yacc[r][nt][i];
                 }
     }
     __syncthreads();
@@ -289,9 +291,11 @@ stream_kernel(const StreamParams p) {
     for (int i = tid; i < tc * kRows; i += kThreads) {
         const int tk = i / kRows, rl = i - tk * kRows;
         if (rl < rows_here) {
-            float sum = 0.0f;
+            // four independent partial sums, then their sum
+            float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) sum += red[(w * kTok + tk) * kRows + rl];
+            for (int w = 0; w < kConsumerWarps; ++w) s4[w & 3] += red[(w * kTok + tk) * kRowsP + rl];
+            const float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
             const size_t o = (size_t)tk * p.ldy + (size_t)rt0 * 16 + rl;
             if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = sum;
             else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(sum);
@@ -554,7 +558,7 @@ bool plan_layout(const lopro_desc& d, StreamPlan* pl, int r_pad, int ng, int kto
     pl->off_stage_x = w_bytes;
     pl->stage_bytes = round_up_int(w_bytes + ktok * kActRecord, 128);
     pl->total_stages = (d.d_in / 64 + kStageSteps - 1) / kStageSteps;
-    const int red_bytes = kConsumerWarps * ktok * pl->rt * 16 * 4;
+    const int red_bytes = kConsumerWarps * ktok * (pl->rt * 16 + kRedPad) * 4;
     int stages = (kStreamMaxSmem - off) / pl->stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages > pl->total_stages) stages = pl->total_stages;
