@@ -32,6 +32,8 @@ WORKLOADS = {
     # name: (config, tokens, layers in the ring)
     "cfg2_T8": ("cfg2", 8, 64),
     "cfg2_T1": ("cfg2", 1, 64),
+    "cfg2_T16": ("cfg2", 16, 64),
+    "cfg2_T32": ("cfg2", 32, 64),
     # one layer repeated: its 9.5 MB of packed weights stay in the 126 MB L2 (reported as such, never the bench line)
     "cfg2_T8_L2": ("cfg2", 8, 64),
     "cfg3_T2048": ("cfg3", 2048, 8),
