@@ -185,8 +185,8 @@ LOPRO_API lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* pack
  *   LOPRO_PATH_GENERAL  rotation, B x, register-ring product (any shape the descriptor allows)
  *   LOPRO_PATH_PREFILL  rotation, B x (2 launches), tcgen05 product, T > 32
  * For T a little above 32, where the library estimates it to be faster than the tensor-core path (layers with
- * few output rows; e.g. up to 128 tokens for 4096 x 4096), the forward runs as chunks of 32 tokens through the
- * small-batch kernels: STREAM or TALL with 2 launches per chunk.
+ * few output rows; e.g. up to 192 tokens for 4096 x 4096), the forward runs as chunks of 32 tokens through the
+ * small-batch kernels: STREAM or TALL with one prologue launch and one launch per chunk.
  * Returns the path (> 0) and stores the number of kernel launches in *launches (may be NULL), or
  * returns 0 for a bad descriptor or T < 1. */
 typedef enum {

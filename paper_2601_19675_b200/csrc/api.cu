@@ -57,8 +57,9 @@ lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
     off += 256;
     W->off_xrot = off;
     {
+        // rotated activations, or the activation image of the small-batch kernels (a little larger)
         size_t xb = (size_t)t_pad * d.d_in * 2;
-        if (t_pad <= kDecodeMaxT && act_image_bytes(d.d_in, t_pad) > xb) xb = act_image_bytes(d.d_in, t_pad);
+        if (act_image_bytes(d.d_in, t_pad) > xb) xb = act_image_bytes(d.d_in, t_pad);
         off += round_up_size(xb, 256);
     }
     W->off_s64 = off;
@@ -201,21 +202,22 @@ static bool use_tall(const lopro_desc& d, int T) {
     return tall_supported(d, T);
 }
 
-// Token counts a little above the small-batch range run as chunks of kDecodeMaxT tokens through the small-batch
-// kernels when that costs less than the tensor-core path: a prefill CTA walks all of K for its 128 or 256 rows
-// whatever the token count, and a layer with few rows fills few SMs.  Both sides are estimated from timings on
-// B200 (microseconds): a chunk 4 + 0.6e-6 d_out d_in (15 for 4096 x 4096, 25-32 for 4096 x 11008 either way
-// round), the prefill chain 8 + 0.017 d_in per wave of CTAs (74 for d_in = 4096, 205 for 11008, flat from 33 to
-// 256 tokens).  LOPRO_NO_CHUNKS=1 turns this off (A/B runs, tests of the prefill kernel on small layers).
+// Token counts a little above the small-batch range run as ONE prologue plus chunks of kDecodeMaxT tokens through
+// the small-batch kernels when that costs less than the tensor-core path: a prefill CTA walks all of K for its
+// 128 or 256 rows whatever the token count, and a layer with few rows fills few SMs.  Both sides are estimated from
+// timings on B200 (microseconds, beyond a common 8 for the first launches): a chunk 3 + 0.45e-6 d_out d_in (10.9 for
+// 4096 x 4096, 23.4 for 4096 x 11008 either way round), the prefill kernel 0.017 d_in per wave of CTAs (74 in all
+// for d_in = 4096, 205 for 11008, flat from 33 to 256 tokens).  LOPRO_NO_CHUNKS=1 turns this off (A/B runs, tests
+// of the prefill kernel on small layers).
 static int small_batch_chunks(const lopro_desc& d, int T) {
     if (T <= kDecodeMaxT) return 0;
     const char* e = getenv("LOPRO_NO_CHUNKS");
     if (e && e[0] == '1') return 0;
     if (!prefill_supported(d, T)) return 0;  // keep the general path's behaviour where there is no prefill kernel
     const int chunks = (T + kDecodeMaxT - 1) / kDecodeMaxT;
-    const double chunk_us = 4.0 + 0.6e-6 * (double)d.d_out * (double)d.d_in;
+    const double chunk_us = 3.0 + 0.45e-6 * (double)d.d_out * (double)d.d_in;
     const int ctas = ((d.d_out + 255) / 256) * ((T + 255) / 256);  // two 128-row blocks per CTA
-    const double prefill_us = 8.0 + 0.017 * (double)d.d_in * (double)((ctas + 147) / 148);
+    const double prefill_us = 0.017 * (double)d.d_in * (double)((ctas + 147) / 148);
     if ((double)chunks * chunk_us >= prefill_us) return 0;
     if (!prologue_supported(d, kDecodeMaxT) || !stream_supported(d, kDecodeMaxT)) return 0;
     return chunks;
@@ -226,7 +228,7 @@ int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launch
     int32_t path, n;
     if (const int chunks = small_batch_chunks(*desc, T)) {
         path = use_tall(*desc, kDecodeMaxT) ? LOPRO_PATH_TALL : LOPRO_PATH_STREAM;
-        n = 2 * chunks;
+        n = 1 + chunks;
     } else if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
         path = use_tall(*desc, T) ? LOPRO_PATH_TALL : (stream_uses_wide(*desc, T) ? LOPRO_PATH_WIDE : LOPRO_PATH_STREAM);
         n = 2;
@@ -270,20 +272,17 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     float* s64 = (float*)(ws + W.off_s64);
     int* status = (int*)(ws + W.off_status);
     if (const int chunks = small_batch_chunks(*desc, T)) {
-        // chunks of kDecodeMaxT tokens through the small-batch kernels; the status word is reset by the first
-        // chunk's prologue only, so a time-out in any chunk stays recorded
+        // one prologue for all tokens, then chunks of kDecodeMaxT tokens through the small-batch kernels, each
+        // reading its tokens' records of the activation image and rows of t
+        if (launch_prologue(*desc, perm, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot,
+                            (__half*)(ws + W.off_t), W.t_pad, status, T, s) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
         const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;
         for (int c = 0; c < chunks; ++c) {
             const int t0 = c * kDecodeMaxT, tc = T - t0 < kDecodeMaxT ? T - t0 : kDecodeMaxT;
-            WorkspaceLayout Wc;  // never larger than the layout for all T tokens
-            if ((st = workspace_layout(*desc, tc, &Wc)) != LOPRO_OK) return st;
-            const __nv_bfloat16* xc = (const __nv_bfloat16*)x_bf16 + (size_t)t0 * ldx;
             void* yc = (uint8_t*)y + (size_t)t0 * ldy * esz;
-            if (launch_prologue(*desc, perm, B, L.r_pad, xc, ldx, ws + Wc.off_xrot, (__half*)(ws + Wc.off_t), Wc.t_pad,
-                                c == 0 ? status : nullptr, tc, s) != cudaSuccess)
-                return LOPRO_ERR_CUDA;
-            const cudaError_t e = use_tall(*desc, tc) ? launch_tall(*desc, blob, L, ws, Wc, yc, ldy, out_dtype, tc, s)
-                                                      : launch_stream(*desc, blob, L, ws, Wc, yc, ldy, out_dtype, tc, s);
+            const cudaError_t e = use_tall(*desc, tc) ? launch_tall(*desc, blob, L, ws, W, yc, ldy, out_dtype, tc, s, t0)
+                                                      : launch_stream(*desc, blob, L, ws, W, yc, ldy, out_dtype, tc, s, t0);
             if (e != cudaSuccess) return LOPRO_ERR_CUDA;
         }
         return LOPRO_OK;

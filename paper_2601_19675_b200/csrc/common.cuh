@@ -113,12 +113,12 @@ cudaError_t launch_decode(const lopro_desc& d, const uint8_t* blob, const BlobLa
 bool stream_supported(const lopro_desc& d, int T);
 bool stream_uses_wide(const lopro_desc& d, int T);  // the 32-warp variant of the kernel will run
 cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
+                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0 = 0);
 
 // Small-batch forward for tall layers after launch_prologue: persistent CTAs, one ring across tile groups.
 bool tall_supported(const lopro_desc& d, int T);
 cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                        const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
+                        const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0 = 0);
 
 // t = B x on the tensor cores for many tokens; `partial` holds lowrank_mma_scratch_bytes of fp32 K-slice sums.
 size_t lowrank_mma_scratch_bytes(const lopro_desc& d, int T);

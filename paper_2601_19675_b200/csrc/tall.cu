@@ -453,15 +453,16 @@ bool tall_supported(const lopro_desc& d, int T) {
 }
 
 cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                        const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s) {
+                        const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0) {
     TallPlan pl;
     if (!plan_tall(d, T, &pl)) return cudaErrorInvalidValue;
     TallParams p;
     p.codes = blob + L.off[LOPRO_SEC_CODES];
     p.sz = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_SCALEZERO]);
     p.A = reinterpret_cast<const __half*>(blob + L.off[LOPRO_SEC_A]);
-    p.act = ws + W.off_xrot;
-    p.t = reinterpret_cast<const __half*>(ws + W.off_t);
+    // t0: first token of this launch within the activation image and t (a chunk of a longer batch)
+    p.act = ws + W.off_xrot + (size_t)t0 * kActRecord;
+    p.t = reinterpret_cast<const __half*>(ws + W.off_t) + (size_t)t0 * (d.rank > 0 ? L.r_pad : 0);
     p.status = reinterpret_cast<int*>(const_cast<uint8_t*>(ws) + W.off_status);
     p.y = y;
     p.ldy = ldy;
