@@ -251,8 +251,9 @@ def test_forward_argument_errors():
     assert y.shape == (0, m)
 
 
-def test_host_entry_point_matches_device_entry_point():
-    n, m, bits, g, r, T = 1024, 256, 4, 128, 16, 8
+@pytest.mark.parametrize("T", [8, 40, 300])  # small batch, chunks of 32 tokens, tensor-core path
+def test_host_entry_point_matches_device_entry_point(T):
+    n, m, bits, g, r = 1024, 256, 4, 128, 16
     layer = random_layer_np(n, m, bits, g, r, seed=4)
     d = lopro.make_desc(n, m, bits, g, 128, rank=r)
     blob = _pack(layer, d)
