@@ -65,11 +65,54 @@ def _check_forward_once(layer, d, x_bits, rows, gate_a, gate_b):
         got_bf, got_f32 = got_bf[:, rows], got_f32[:, rows]
     err_a = o.max_rel_err(got_bf, exact)
     err_b = o.max_rel_err(got_f32, mirrored)
+    if err_b > gate_b:
+        err_b = _gate_b_with_ties(x64, args, round_w, mirrored, got_f32)
     assert err_a <= gate_a, f"gate A: {err_a}"
     assert err_b <= gate_b, f"gate B: {err_b}"
     # bf16 output is the rounding of the fp32 output path (same accumulation order)
     assert np.array_equal(got_bf, o.round_bf16(got_f32))
     return err_a, err_b
+
+
+def _gate_b_with_ties(x64, args, round_w, mirrored, got_f32):
+    """Gate B when a rotated entry sits on a bf16 rounding boundary.  The kernels run the butterflies in fp32,
+    the oracle in fp64; an entry of the exact x~ that lies within 1e-6 of its block's maximum of the midpoint
+    between two bf16 values may legitimately round to either side (the rotation's own tolerance allows it).
+    Everything here comes from the oracle: for each token with such entries the mirrored result is re-evaluated
+    with such entries moved to the other side -- y is linear in x~, so flipping entry k of token t adds
+    (other - chosen) * W^[:, k] -- and the token's outputs must meet the gate for one such choice."""
+    b_i, b_h, g = args["b_i"], args["b_h"], args["g"]
+    xt = o.rotate(x64, args["perm"], b_i, b_h)
+    chosen = o.round_bf16(xt)
+    # the neighbouring bf16 value on the other side of xt
+    step = np.abs(chosen) * 2.0 ** -7
+    other = np.where(xt > chosen, o.round_bf16(chosen + step), np.where(xt < chosen, o.round_bf16(chosen - step), chosen))
+    mid = 0.5 * (chosen + other)
+    n = xt.shape[1]
+    blockmax = np.empty_like(xt)
+    blockmax[:, :b_i] = np.abs(xt[:, :b_i])
+    if n > b_i:
+        bm = np.abs(xt[:, b_i:]).reshape(xt.shape[0], -1, b_h).max(axis=2, keepdims=True)
+        blockmax[:, b_i:] = np.broadcast_to(bm, (xt.shape[0], (n - b_i) // b_h, b_h)).reshape(xt.shape[0], n - b_i)
+    near = (other != chosen) & (np.abs(xt - mid) <= 1e-6 * blockmax)
+    w_hat = o.dequant(args["codes"], args["scales"], args["zeros"], g)
+    if round_w:
+        w_hat = o.round_bf16(o.round_f32(w_hat))
+    worst = 0.0
+    for t in range(xt.shape[0]):
+        # greedy search for a witness, largest rounding steps first: a flip is kept when it lowers the token's
+        # error (a few entries per token qualify; only one with a large step can matter)
+        ks = np.flatnonzero(near[t])
+        ks = ks[np.argsort(-np.abs(other[t, ks] - chosen[t, ks]))]
+        y = mirrored[t].copy()
+        best = o.max_rel_err(got_f32[t:t + 1], y[None, :])
+        for k in ks:
+            y_alt = y + (other[t, k] - chosen[t, k]) * w_hat[:, k]
+            e = o.max_rel_err(got_f32[t:t + 1], y_alt[None, :])
+            if e < best:
+                y, best = y_alt, e
+        worst = max(worst, best)
+    return worst
 
 
 def test_cfg1_layer_quantized_by_the_oracle():
@@ -184,10 +227,18 @@ def test_token_counts_above_32_run_as_chunks_where_that_is_estimated_faster(T, n
         assert launches == 1 + (T + 31) // 32
     layer = random_layer_np(n, m, 4, 128, 16, seed=T + m)
     rows = None if n * m <= 1 << 22 else np.arange(0, m, 7)
-    # (seed: with seed = T the 128-token case has one rotated outlier entry within rounding distance of a bf16 tie,
-    # which the fp32 butterflies and the fp64 oracle round to different sides -- inside the rotation's own tolerance
-    # -- and which alone moves one output of that token to 1.03e-3 against the mirrored oracle)
     _check_forward(layer, d, synth.activations(T, n, seed=T + 1), rows=rows)
+
+
+def test_rotated_entry_on_a_bf16_rounding_boundary():
+    # 128 tokens drawn with seed 128: one rotated outlier entry lies within fp32 rounding distance of the midpoint of
+    # two bf16 values; the fp32 butterflies of the kernel and the fp64 oracle may round it to different sides (inside
+    # the rotation's own tolerance), which alone moves one output of that token past 1e-3.  Gate B then holds
+    # against the mirrored oracle evaluated for either side (_gate_b_with_ties).
+    T, n, m = 128, 1024, 4096
+    d = lopro.make_desc(n, m, 4, 128, 128, identity_cols=128, rank=16)
+    layer = random_layer_np(n, m, 4, 128, 16, seed=T + m)
+    _check_forward(layer, d, synth.activations(T, n, seed=T))
 
 
 def test_tall_kernel_agrees_with_the_per_group_kernel(monkeypatch):

@@ -249,3 +249,81 @@ def test_max_rel_err_definition():
     y = np.array([[3.3, 4.0, 0.25, 0.0]])
     # |0.3| / 3 = 0.1 ; |0.25| / max(0, 2.5) = 0.1
     assert abs(o.max_rel_err(y, y_ref) - 0.1) < 1e-12
+
+
+def _lib_bf16(a):
+    """fp64 -> bf16 values by torch's cast (independent of the oracle's rounding helpers)."""
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float64)).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def _mirrored_by_hand(L, round_w, round_t, out):
+    """Eq. 8 with the declared roundings written out step by step: explicit dense P and Q, scalar loops for the
+    dequantization, library casts (torch bfloat16, numpy float16 / float32) for every rounding."""
+    x, codes, scales, zeros, perm = L["x"], L["codes"], L["scales"], L["zeros"], L["perm"]
+    a, b, g, b_i, b_h = L["a"], L["b"], L["g"], L["b_i"], L["b_h"]
+    T, n = x.shape
+    m = codes.shape[0]
+    p = np.zeros((n, n))
+    for k in range(n):
+        p[int(perm[k]), k] = 1.0                       # (x P)[k] = x[perm[k]]
+    q = np.zeros((n, n))
+    for k in range(b_i):
+        q[k, k] = 1.0
+    for s in range(b_i, n, b_h):
+        for i in range(b_h):
+            for j in range(b_h):
+                q[s + i, s + j] = (-1.0 if bin(i & j).count("1") & 1 else 1.0) / math.sqrt(b_h)
+    xt = _lib_bf16(x @ p @ q)                          # rotated activations, stored as bf16
+    w = np.zeros((m, n))
+    for i in range(m):
+        for k in range(n):
+            w[i, k] = float(scales[i, k // g]) * (float(codes[i, k]) - float(zeros[i, k // g]))
+    if round_w:
+        w = _lib_bf16(w.astype(np.float32).astype(np.float64))   # fp32 product, then one rounding to bf16
+    t = x @ b.T
+    if round_t == "f16":
+        t = t.astype(np.float16).astype(np.float64)
+    elif round_t == "bf16":
+        t = _lib_bf16(t)
+    y = xt @ w.T + t @ a.T
+    return _lib_bf16(y) if out == "bf16" else y.astype(np.float32).astype(np.float64)
+
+
+@pytest.mark.parametrize("round_w", [False, True])
+@pytest.mark.parametrize("round_t", ["f16", "bf16", "none"])
+@pytest.mark.parametrize("out", ["f32", "bf16"])
+def test_forward_mirrored_equals_the_steps_written_out(round_w, round_t, out):
+    # every product and partial sum of this tiny layer is exact in fp64 (8-bit activations, 11-bit scales and
+    # factors, a narrow exponent range), so the two evaluations may differ in nothing but a misplaced rounding
+    L = _tiny_layer(31, m=8, n=64, g=16, bits=4, b_i=16, b_h=16, r=3, T=5)
+    got = o.forward_mirrored(**L, round_w=round_w, round_t=round_t, out=out)
+    np.testing.assert_array_equal(got, _mirrored_by_hand(L, round_w, round_t, out))
+
+
+def test_each_switch_of_forward_mirrored_touches_only_the_operand_it_names():
+    L = _tiny_layer(32, m=8, n=64, g=16, bits=4, b_i=16, b_h=16, r=3, T=5)
+    base = o.forward_mirrored(**L, round_w=False, round_t="none", out="f32")
+    # weights that are bf16 values already (power-of-two scales, integer zero-points): round_w changes nothing,
+    # while with generic fp16 scales it does
+    Lp = dict(L)
+    Lp["scales"] = np.full_like(L["scales"], 2.0 ** -5)
+    Lp["zeros"] = np.rint(L["zeros"])
+    np.testing.assert_array_equal(o.forward_mirrored(**Lp, round_w=True, round_t="none"),
+                                  o.forward_mirrored(**Lp, round_w=False, round_t="none"))
+    assert not np.array_equal(o.forward_mirrored(**L, round_w=True, round_t="none"), base)
+    # no low-rank branch: round_t changes nothing; with one it does, and by exactly A (round(t) - t)
+    L0 = dict(L)
+    L0["a"], L0["b"] = np.zeros((8, 0)), np.zeros((0, 64))
+    np.testing.assert_array_equal(o.forward_mirrored(**L0, round_t="f16"), o.forward_mirrored(**L0, round_t="none"))
+    t = L["x"] @ L["b"].T
+    d_t = (t.astype(np.float16).astype(np.float64) - t) @ L["a"].T
+    full = o.forward_mirrored(**L, round_w=False, round_t="f16", out="f32")
+    np.testing.assert_allclose(full - base, d_t, atol=2e-6)       # both sides carry one fp32 rounding of y
+    assert np.abs(d_t).max() > 0.0
+    # activations: always rounded -- x~ that is bf16 already (rotation off, b_I = n) makes mirrored == exact
+    Li = dict(L)
+    Li["b_i"] = 64
+    y_exact = o.forward_exact(**Li)
+    np.testing.assert_array_equal(o.forward_mirrored(**Li, round_t="none"), y_exact.astype(np.float32).astype(np.float64))
+    # out: the bf16 result is one rounding of the fp64 sum, not of the fp32 result
+    np.testing.assert_array_equal(o.forward_mirrored(**Li, round_t="none", out="bf16"), _lib_bf16(y_exact))

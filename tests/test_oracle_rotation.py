@@ -133,10 +133,14 @@ def test_perm_from_stats_moves_large_ratio_first():
     np.testing.assert_array_equal(o.perm_from_stats(diag_h, r), [1, 2, 3, 0])
 
 
-def test_activation_scale_formula():
-    x = np.array([[1.0, -2.0, 4.0], [3.0, 2.0, -4.0]])     # Xbar = 2, 2, 4
+def test_activation_scale_worked_by_hand():
+    # Algorithm 1: Xbar = column means of |X| = (2, 2, 4); max * min = 8, so s = Xbar^2.5 / sqrt(8):
+    # 2^2.5 / 2^1.5 = 2 and 4^2.5 / 2^1.5 = 32 / (2 sqrt 2) = 8 sqrt 2 -- numbers worked out on paper
+    x = np.array([[1.0, -2.0, 4.0], [3.0, 2.0, -4.0]])
     s = o.activation_scale(x)
-    np.testing.assert_allclose(s, np.array([2.0, 2.0, 4.0]) ** 2.5 / np.sqrt(4.0 * 2.0), rtol=1e-15)
+    np.testing.assert_allclose(s, [2.0, 2.0, 11.313708498984761], rtol=1e-14)
+    # homogeneous of degree 1.5 in X (2.5 - 2 / 2): scaling the calibration data by 4 scales s by 8
+    np.testing.assert_allclose(o.activation_scale(4.0 * x), 8.0 * s, rtol=1e-14)
 
 
 def test_rotate_is_orthogonal_map_of_x():

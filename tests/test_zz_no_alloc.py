@@ -29,11 +29,8 @@ def _layer(n, m, bits, g, b, r, seed):
     return d, blob
 
 
-@pytest.mark.parametrize("n,m,bits,g,b,r", [(1024, 272, 4, 128, 128, 16), (2048, 144, 2, 64, 256, 33)])
-def test_two_calls_in_a_row_match_the_workspace_entry_point(n, m, bits, g, b, r):
-    d, blob = _layer(n, m, bits, g, b, r, seed=11)
-    outs = []
-    for call, T in enumerate((8, 3)):           # second call: fewer tokens, other values, same shared scratch
+def _two_calls(d, blob, n, m, token_counts):
+    for call, T in enumerate(token_counts):     # second call: fewer tokens, other values, same shared scratch
         x = bf16_bits_to_device(synth.activations(T, n, seed=50 + call, outlier_frac=0.01))
         ref_bf = lopro.linear_fwd(d, blob, x, lopro.OUT_BF16)
         ref_f32 = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
@@ -42,13 +39,33 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(n, m, bits, g, b, r)
         lopro.linear_fwd_noalloc(d, blob, x, y_bf, lopro.OUT_BF16)
         lopro.linear_fwd_noalloc(d, blob, x, y_f32, lopro.OUT_F32)
         torch.cuda.synchronize()
-        # same tolerances as the forward tests (gate A for bf16, gate B for fp32), here against the
-        # workspace entry point instead of the oracle
+        # Both entry points launch the same kernels on the same inputs in the same fixed order, so the outputs
+        # agree bit for bit -- a sharper check than the forward tests' tolerances (which it implies): anything
+        # stale read from the shared scratch, or a misplaced offset inside it, would show.
+        assert torch.isfinite(y_f32).all()
+        assert torch.equal(y_bf, ref_bf)
+        assert torch.equal(y_f32, ref_f32)
         assert o.max_rel_err(device_bf16_to_f64(y_bf), device_bf16_to_f64(ref_bf)) <= 2e-2
         assert o.max_rel_err(y_f32.cpu().numpy().astype(np.float64), ref_f32.cpu().numpy().astype(np.float64)) <= 1e-3
-        assert torch.isfinite(y_f32).all()
-        outs.append(y_f32.clone())
-    assert outs[0].shape != outs[1].shape
+
+
+@pytest.mark.parametrize("n,m,bits,g,b,r", [(1024, 272, 4, 128, 128, 16), (2048, 144, 2, 64, 256, 33)])
+def test_two_calls_in_a_row_match_the_workspace_entry_point(n, m, bits, g, b, r):
+    d, blob = _layer(n, m, bits, g, b, r, seed=11)
+    _two_calls(d, blob, n, m, (8, 3))
+
+
+@pytest.mark.parametrize("no_chunks", [False, True])
+def test_more_than_32_tokens_inside_the_fixed_scratch(no_chunks, monkeypatch):
+    # 40 and 33 tokens still fit the built-in array: as chunks of 32 through the small-batch kernels, and (with the
+    # library's switch for it) through the tensor-core kernel
+    n, m = 1024, 256
+    d, blob = _layer(n, m, 4, 128, 128, 16, seed=13)
+    if no_chunks:
+        monkeypatch.setenv("LOPRO_NO_CHUNKS", "1")
+    assert lopro.workspace_bytes(d, 40) <= lopro.NOALLOC_SCRATCH_BYTES
+    assert (lopro.linear_fwd_path(d, 40)[0] == lopro.PATH_PREFILL) == no_chunks
+    _two_calls(d, blob, n, m, (40, 33))
 
 
 def test_requests_beyond_the_fixed_scratch_are_refused():
