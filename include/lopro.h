@@ -98,6 +98,22 @@ enum {
     LOPRO_SEC_COUNT = 6
 };
 
+/* Tuning switches of lopro_configure.  They change which kernels a forward runs, never what it computes; they
+ * exist for A/B timing and for tests that must reach a particular kernel (the paper has no counterpart).  The
+ * initial value of each is read once per process from the environment variable of the same name
+ * (LOPRO_NO_WIDE=1, ...); 0 = default behaviour. */
+enum {
+    LOPRO_OPT_NO_WIDE = 0,       /* 1: never the 32-warp variant of the streaming kernel                       */
+    LOPRO_OPT_NO_TALL = 1,       /* 1: never the persistent streaming kernel for layers with many rows         */
+    LOPRO_OPT_NO_CHUNKS = 2,     /* 1: token counts above 32 always take the tensor-core (prefill) kernel      */
+    LOPRO_OPT_NO_TCGEN05 = 3,    /* 1: never the tcgen05 prefill kernel (general register-ring product)        */
+    LOPRO_OPT_PREFILL_PAIRS = 4, /* >= 0: number of two-block row tiles of the prefill grid; -1: chosen by it  */
+    LOPRO_OPT_COUNT = 5
+};
+/* Sets one switch for the whole process (not thread-safe against forwards running on other host threads).
+ * Returns LOPRO_ERR_INVALID_ARG for an unknown option. */
+LOPRO_API lopro_status lopro_configure(int32_t option, int32_t value);
+
 /* Library version (major * 10000 + minor * 100 + patch). */
 LOPRO_API int lopro_version(void);
 
@@ -118,8 +134,8 @@ LOPRO_API size_t lopro_packed_bytes(const lopro_desc* desc);
  * bad descriptor or section id. */
 LOPRO_API lopro_status lopro_packed_section(const lopro_desc* desc, int32_t section, size_t* offset, size_t* bytes);
 
-/* Bytes of device workspace lopro_linear_fwd needs for up to T tokens (0 on bad arguments).
- * Monotone in T. */
+/* Bytes of device workspace lopro_linear_fwd needs for up to T tokens (0 on bad arguments).  Non-decreasing
+ * in T: a workspace sized for the largest batch serves every smaller one. */
 LOPRO_API size_t lopro_workspace_bytes(const lopro_desc* desc, int32_t T);
 
 /* Build the packed blob from plain arrays -- the record (W_q, U, V, Sigma, p, s) that
@@ -233,6 +249,15 @@ LOPRO_API lopro_status lopro_linear_fwd_host(const lopro_desc* desc, const void*
 LOPRO_API lopro_status lopro_linear_fwd_noalloc(const lopro_desc* desc, const void* packed, const uint16_t* x_bf16,
                                                 int64_t ldx, void* y, int64_t ldy, int32_t out_dtype, int32_t T,
                                                 void* stream);
+
+/* Self-test of the library's failure detection (the paper has no counterpart).  Every wait of the forward
+ * kernels on a shared-memory barrier is bounded: when the limit runs out the kernel stores LOPRO_ERR_TIMEOUT in
+ * the workspace status word and returns normally instead of hanging.  This call exercises exactly that code path
+ * without any fault: it launches one thread block that initialises a barrier, announces bytes that no copy will
+ * ever deliver (nothing is in flight when the block exits), waits on it with the library's bounded wait under a
+ * short limit (4096 polls), and on expiry stores LOPRO_ERR_TIMEOUT in *status_word (device memory, 4 bytes,
+ * 4-byte aligned; the kernel first stores LOPRO_OK there).  Asynchronous: read the word after synchronising. */
+LOPRO_API lopro_status lopro_selftest_wait(void* status_word, void* stream);
 
 #ifdef __cplusplus
 }

@@ -74,6 +74,45 @@ lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
+namespace {
+int g_options[LOPRO_OPT_COUNT];
+int g_options_ready = 0;  // 0 = not read yet, 1 = being read, 2 = ready
+
+void read_options_once() {
+    int expected = 0;
+    if (__atomic_compare_exchange_n(&g_options_ready, &expected, 1, false, __ATOMIC_ACQ_REL, __ATOMIC_ACQUIRE)) {
+        static const char* const names[LOPRO_OPT_COUNT] = {"LOPRO_NO_WIDE", "LOPRO_NO_TALL", "LOPRO_NO_CHUNKS",
+                                                           "LOPRO_NO_TCGEN05", "LOPRO_PREFILL_PAIRS"};
+        for (int i = 0; i < LOPRO_OPT_COUNT; ++i) {
+            const char* e = getenv(names[i]);
+            g_options[i] = e ? atoi(e) : (i == LOPRO_OPT_PREFILL_PAIRS ? -1 : 0);
+        }
+        __atomic_store_n(&g_options_ready, 2, __ATOMIC_RELEASE);
+    } else {
+        while (__atomic_load_n(&g_options_ready, __ATOMIC_ACQUIRE) != 2) {
+        }
+    }
+}
+}  // namespace
+
+int option(int id) {
+    if (__atomic_load_n(&g_options_ready, __ATOMIC_ACQUIRE) != 2) read_options_once();
+    return __atomic_load_n(&g_options[id], __ATOMIC_RELAXED);
+}
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    int& c = cached[dev & 63];
+    if (c == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        c = v;
+    }
+    return c;
+}
+
 }  // namespace lopro
 
 using namespace lopro;
@@ -157,7 +196,15 @@ lopro_status lopro_pack(const lopro_desc* desc, const uint8_t* codes, const uint
     if (cudaMemcpyAsync(&back, packed, sizeof(back), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOPRO_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return LOPRO_ERR_CUDA;
     if (back.magic != kBlobMagic) return LOPRO_ERR_CUDA;
-    if (back.invalid != 0) return LOPRO_ERR_INVALID_DATA;
+    if (back.invalid != 0) {
+        // A rejected blob must stay harmless if a caller ignores the status and runs a forward on it: the kernels
+        // gather x[perm[k]] without a range check, so the permutation section is cleared (every entry 0, in range;
+        // codes were masked to their width while packing).  The header keeps the validation flags.
+        if (cudaMemsetAsync((uint8_t*)packed + L.off[LOPRO_SEC_PERM], 0, L.bytes[LOPRO_SEC_PERM], s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
+        return LOPRO_ERR_INVALID_DATA;
+    }
     return LOPRO_OK;
 }
 
@@ -195,10 +242,9 @@ lopro_status lopro_rotate(const lopro_desc* desc, const int32_t* perm, const uin
     return e == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }
 
-// LOPRO_NO_TALL=1 keeps the persistent kernel for tall layers off (A/B comparison and tests of the other kernel).
+// LOPRO_OPT_NO_TALL keeps the persistent kernel for tall layers off (A/B comparison and tests of the other kernel).
 static bool use_tall(const lopro_desc& d, int T) {
-    const char* e = getenv("LOPRO_NO_TALL");
-    if (e && e[0] == '1') return false;
+    if (option(LOPRO_OPT_NO_TALL) == 1) return false;
     return tall_supported(d, T);
 }
 
@@ -207,17 +253,17 @@ static bool use_tall(const lopro_desc& d, int T) {
 // 128 or 256 rows whatever the token count, and a layer with few rows fills few SMs.  Both sides are estimated from
 // timings on B200 (microseconds, beyond a common 8 for the first launches): a chunk 3 + 0.45e-6 d_out d_in (10.9 for
 // 4096 x 4096, 23.4 for 4096 x 11008 either way round), the prefill kernel 0.017 d_in per wave of CTAs (74 in all
-// for d_in = 4096, 205 for 11008, flat from 33 to 256 tokens).  LOPRO_NO_CHUNKS=1 turns this off (A/B runs, tests
+// for d_in = 4096, 205 for 11008, flat from 33 to 256 tokens).  LOPRO_OPT_NO_CHUNKS turns this off (A/B runs, tests
 // of the prefill kernel on small layers).
 static int small_batch_chunks(const lopro_desc& d, int T) {
     if (T <= kDecodeMaxT) return 0;
-    const char* e = getenv("LOPRO_NO_CHUNKS");
-    if (e && e[0] == '1') return 0;
+    if (option(LOPRO_OPT_NO_CHUNKS) == 1) return 0;
     if (!prefill_supported(d, T)) return 0;  // keep the general path's behaviour where there is no prefill kernel
     const int chunks = (T + kDecodeMaxT - 1) / kDecodeMaxT;
     const double chunk_us = 3.0 + 0.45e-6 * (double)d.d_out * (double)d.d_in;
     const int ctas = ((d.d_out + 255) / 256) * ((T + 255) / 256);  // two 128-row blocks per CTA
-    const double prefill_us = 0.017 * (double)d.d_in * (double)((ctas + 147) / 148);
+    const int sms = sm_count();
+    const double prefill_us = 0.017 * (double)d.d_in * (double)((ctas + sms - 1) / sms);
     if ((double)chunks * chunk_us >= prefill_us) return 0;
     if (!prologue_supported(d, kDecodeMaxT) || !stream_supported(d, kDecodeMaxT)) return 0;
     return chunks;
@@ -320,6 +366,13 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
         return LOPRO_OK;
     }
     if (launch_decode(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    return LOPRO_OK;
+}
+
+lopro_status lopro_configure(int32_t opt, int32_t value) {
+    if (opt < 0 || opt >= LOPRO_OPT_COUNT) return LOPRO_ERR_INVALID_ARG;
+    (void)option(opt);  // make sure the environment has been read, so that it cannot overwrite this value later
+    __atomic_store_n(&g_options[opt], (int)value, __ATOMIC_RELAXED);
     return LOPRO_OK;
 }
 

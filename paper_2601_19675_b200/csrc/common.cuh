@@ -61,6 +61,11 @@ inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long l
     return e;
 }
 
+// Tuning switches (lopro_configure; initial values from the environment, read once per process).
+int option(int id);
+// Multiprocessors of the current device (cached per device; 148 if the query fails).
+int sm_count();
+
 inline int round_up_int(int v, int a) { return (v + a - 1) / a * a; }
 inline size_t round_up_size(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

@@ -11,6 +11,7 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace lopro {
 
@@ -40,26 +41,6 @@ struct DecodeParams {
     int panel_steps; // steps staged in shared memory at a time (multiple of kPrefetch)
 };
 
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t smem_addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(smem_addr));
-}
-
 // Streaming load of one lane's `BITS` code words (read once: keep them out of L1).
 template <int BITS>
 __device__ __forceinline__ void load_codes(uint32_t (&w)[BITS], const uint32_t* p) {
@@ -73,26 +54,6 @@ __device__ __forceinline__ void load_codes(uint32_t (&w)[BITS], const uint32_t* 
         w[0] = __ldg(p);
         w[1] = __ldg(p + 1);
         w[2] = __ldg(p + 2);
-    }
-}
-
-constexpr uint32_t kMagic128 = 0x43004300u;  // two bf16 128.0: ulp 1, so 128.0 | c == 128 + c for c < 128
-
-// The sixteen A-operand register pairs (128 + code as bf16) of one 16 x 64 tile, pair pi = 4 j + rho.
-template <int BITS>
-__device__ __forceinline__ void expand_codes(uint32_t (&a)[16], const uint32_t (&w)[BITS]) {
-    if constexpr (BITS == 4) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = ((w[j] >> (4 * rho)) & 0x000F000Fu) | kMagic128;
-    } else if constexpr (BITS == 2) {
-#pragma unroll
-        for (int pi = 0; pi < 16; ++pi) a[pi] = ((w[pi >> 3] >> (2 * (pi & 7))) & 0x00030003u) | kMagic128;
-    } else {
-#pragma unroll
-        for (int pi = 0; pi < 15; ++pi) a[pi] = ((w[pi / 5] >> (3 * (pi % 5))) & 0x00070007u) | kMagic128;
-        a[15] = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u) | kMagic128;
     }
 }
 

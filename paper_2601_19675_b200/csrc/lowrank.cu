@@ -8,6 +8,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 #include "rotate_body.cuh"
 
 namespace lopro {
@@ -19,18 +20,6 @@ constexpr int kLrTokens = 128;       // tokens per CTA (8 warps x 16)
 constexpr int kLrChunk = 64;         // K columns staged per iteration
 constexpr int kLrStride = kLrChunk + 8;  // bf16 elements per shared-memory row (+16 bytes: conflict-free ldmatrix)
 constexpr int kLrMaxRank = 128;      // rows of B per CTA
-
-__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 
 // NJ = 8-wide column tiles of the output handled per CTA (rows of B / 8)
 template <int NJ>
@@ -111,16 +100,16 @@ __device__ __forceinline__ void lowrank_body(unsigned char* smem_raw, int bx, in
 #pragma unroll
         for (int kk = 0; kk < kLrChunk; kk += 16) {
             uint32_t a[4];
-            ldsm_x4(a, xs_u + a_off + kk * 2);
+            ldmatrix_x4(a, xs_u + a_off + kk * 2);
 #pragma unroll
             for (int jp = 0; jp < NJ / 2; ++jp) {
                 uint32_t b[4];
-                ldsm_x4(b, bh_u + b_off + (uint32_t)(jp * 16 * kLrStride + kk) * 2u);
-                mma_bf16_16816(acc[2 * jp], a, b[0], b[1]);
-                mma_bf16_16816(acc[2 * jp + 1], a, b[2], b[3]);
-                ldsm_x4(b, bl_u + b_off + (uint32_t)(jp * 16 * kLrStride + kk) * 2u);
-                mma_bf16_16816(acc[2 * jp], a, b[0], b[1]);
-                mma_bf16_16816(acc[2 * jp + 1], a, b[2], b[3]);
+                ldmatrix_x4(b, bh_u + b_off + (uint32_t)(jp * 16 * kLrStride + kk) * 2u);
+                mma_bf16(acc[2 * jp], a, b[0], b[1]);
+                mma_bf16(acc[2 * jp + 1], a, b[2], b[3]);
+                ldmatrix_x4(b, bl_u + b_off + (uint32_t)(jp * 16 * kLrStride + kk) * 2u);
+                mma_bf16(acc[2 * jp], a, b[0], b[1]);
+                mma_bf16(acc[2 * jp + 1], a, b[2], b[3]);
             }
         }
     }
@@ -185,9 +174,19 @@ int lowrank_mma_slices(const lopro_desc& d, int T) {
     return slices;
 }
 
+// Bytes reserved for the K-slice sums of up to T tokens.  The slice count falls as the token tiles grow, so the
+// need of a launch, slices(T) * T rows, is not monotone in T; the reservation is the largest need of any token
+// count up to T (the slice count is constant within a tile count, so the last T of each tile count decides).
 size_t lowrank_mma_scratch_bytes(const lopro_desc& d, int T) {
     const int r_pad = round_up_int(d.rank, 16);
-    return (size_t)lowrank_mma_slices(d, T) * T * r_pad * 4;
+    const int tiles = (T + kLrTokens - 1) / kLrTokens;
+    size_t rows = 0;
+    for (int tl = 1; tl <= tiles; ++tl) {
+        const int t_last = tl * kLrTokens < T ? tl * kLrTokens : T;
+        const size_t need = (size_t)lowrank_mma_slices(d, t_last) * (size_t)t_last;
+        if (need > rows) rows = need;
+    }
+    return rows * (size_t)r_pad * 4;
 }
 
 cudaError_t launch_lowrank_down_mma(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x, int64_t ldx,

@@ -2,6 +2,7 @@
 // The scratch the forward needs lives in a fixed array inside the library image instead of a
 // caller-provided workspace.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace {
 
@@ -45,4 +46,26 @@ extern "C" lopro_status lopro_linear_fwd_noalloc(const lopro_desc* desc, const v
     // word and every other region is written before it is read.
     return lopro_linear_fwd(desc, packed, x_bf16, ldx, y, ldy, out_dtype, T, scratch, (size_t)LOPRO_NOALLOC_SCRATCH_BYTES,
                             stream);
+}
+
+namespace {
+
+// One block, one thread: a barrier that expects bytes nobody sends, the library's bounded wait, the time-out path.
+__global__ void selftest_wait_kernel(int* status) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x != 0) return;
+    *status = (int)LOPRO_OK;
+    const uint32_t b = lopro::smem_u32(&bar);
+    lopro::mbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    lopro::mbar_expect_tx(b, 16);                    // one arrival, 16 bytes announced; no copy is ever issued
+    if (!lopro::mbar_wait(b, 0, 1u << 12)) atomicExch(status, (int)LOPRO_ERR_TIMEOUT);
+}
+
+}  // namespace
+
+extern "C" lopro_status lopro_selftest_wait(void* status_word, void* stream) {
+    if (!status_word || ((uintptr_t)status_word % 4) != 0) return LOPRO_ERR_INVALID_ARG;
+    selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((int*)status_word);
+    return cudaGetLastError() == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }

@@ -18,12 +18,13 @@
 //   * warps 16-19 (epilogue): tcgen05.ld the accumulator, round once, store y[token][row].
 // All mbarrier waits are bounded; a wait that runs out sets LOPRO_ERR_TIMEOUT in the workspace status
 // word, the CTA stops waiting, still frees its TMEM and returns (outputs then unspecified).
-#include <cuda.h>
 #include <stdlib.h>
 
 #include <type_traits>
 
 #include "common.cuh"
+#include "ptx.cuh"
+#include "tc5.cuh"
 
 namespace lopro {
 
@@ -41,7 +42,7 @@ constexpr int kABytes = 2 * kABlock;            // 32 KB
 constexpr int kBBytes = kMaxTileN * 128;        // 32 KB: one 256-token tile
 constexpr double kPairCost = 1.4;  // duration of a two-block CTA relative to a one-block CTA (scheduling estimate)
 constexpr int kSmemBytes = kAStages * kABytes + kBStages * kBBytes + 1024;  // + slack for 1024-byte alignment
-constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr uint32_t kPrefillSpin = 1u << 24;  // polls of one wait: a CTA's stages are milliseconds apart at most
 
 struct PrefillParams {
     const uint32_t* codes;
@@ -59,93 +60,6 @@ struct PrefillParams {
     int units;         // token tiles
     int lr_stages;   // ceil(r_pad / 64)
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// tiled TMA load of a 2-D box (no multicast), completion counted on an mbarrier of this CTA
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// D[tmem] (+)= A[smem desc] * B[smem desc], M x N x 16, issued by one thread
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u)
-        : "memory");
-}
-// arrive on an mbarrier once every MMA issued so far by this thread has finished reading shared memory
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// K-major, 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart
-__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                        // leading byte offset (unused with swizzle)
-    d |= (uint64_t)(1024 >> 4) << 32;              // stride between 8-row groups
-    d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                        // SWIZZLE_128B
-    return d;
-}
-// instruction descriptor: fp32 accumulator, K-major A and B, M = 128, N = tile_n; fmt 1 = bf16, 0 = fp16
-__device__ __forceinline__ uint32_t make_idesc(int tile_n, uint32_t fmt) {
-    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-}
-
-constexpr uint32_t kMagic128 = 0x43004300u;
-// (a & mask) | magic in one logic instruction, both constants in registers
-__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t mask, uint32_t magic) {
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(magic));
-    return d;
-}
-template <int BITS>
-__device__ __forceinline__ void expand_codes(uint32_t (&a)[16], const uint32_t (&w)[BITS]) {
-    const uint32_t magic = kMagic128;
-    if constexpr (BITS == 4) {
-        const uint32_t mask = 0x000F000Fu;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int rho = 0; rho < 4; ++rho) a[4 * j + rho] = and_or(w[j] >> (4 * rho), mask, magic);
-    } else if constexpr (BITS == 2) {
-        const uint32_t mask = 0x00030003u;
-#pragma unroll
-        for (int pi = 0; pi < 16; ++pi) a[pi] = and_or(w[pi >> 3] >> (2 * (pi & 7)), mask, magic);
-    } else {
-        const uint32_t mask = 0x00070007u;
-#pragma unroll
-        for (int pi = 0; pi < 15; ++pi) a[pi] = and_or(w[pi / 5] >> (3 * (pi % 5)), mask, magic);
-        a[15] = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u) | kMagic128;
-    }
-}
 
 template <int BITS>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -186,7 +100,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     };
     // one lane polls, the warp follows (bar.warp.sync orders the other lanes' accesses after the wait)
     auto warp_wait = [&](uint32_t bar, uint32_t parity) {
-        if (lane == 0 && !s_timeout && !mbar_wait(bar, parity)) time_out();
+        if (lane == 0 && !s_timeout && !mbar_wait(bar, parity, kPrefillSpin)) time_out();
         __syncwarp();
     };
     const uint32_t tmem_cols = n_acc == 2 ? 512u : 256u;
@@ -205,10 +119,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kDequantWarps + 1) {  // one warp allocates the accumulator columns and later frees them
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                     "r"(tmem_cols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc(smem_u32(&s_tmem_base), tmem_cols);
     }
     tc_fence_before();
     __syncthreads();
@@ -305,8 +216,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
             const uint32_t b_bytes = (uint32_t)(p.tile_n * 128);
             for (int s = 0; s < total; ++s) {
                 const int sa = s % kAStages, sb = s % kBStages;
-                if (s >= kAStages && !s_timeout && !mbar_wait(empty_a(sa), (uint32_t)((s / kAStages) - 1) & 1u)) time_out();
-                if (s >= kBStages && !s_timeout && !mbar_wait(empty_b(sb), (uint32_t)((s / kBStages) - 1) & 1u)) time_out();
+                if (s >= kAStages && !s_timeout && !mbar_wait(empty_a(sa), (uint32_t)((s / kAStages) - 1) & 1u, kPrefillSpin)) time_out();
+                if (s >= kBStages && !s_timeout && !mbar_wait(empty_b(sb), (uint32_t)((s / kBStages) - 1) & 1u, kPrefillSpin)) time_out();
                 const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
                 mbar_expect_tx(full_b(sb), b_bytes);
                 if (s < p.nsteps) {
@@ -327,8 +238,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
             const uint32_t idesc_w = make_idesc(p.tile_n, 1u), idesc_lr = make_idesc(p.tile_n, 0u);
             for (int s = 0; s < total; ++s) {
                 const int sa = s % kAStages, sb = s % kBStages;
-                if (!s_timeout && !(mbar_wait(full_a(sa), (uint32_t)(s / kAStages) & 1u) &&
-                                    mbar_wait(full_b(sb), (uint32_t)(s / kBStages) & 1u)))
+                if (!s_timeout && !(mbar_wait(full_a(sa), (uint32_t)(s / kAStages) & 1u, kPrefillSpin) &&
+                                    mbar_wait(full_b(sb), (uint32_t)(s / kBStages) & 1u, kPrefillSpin)))
                     time_out();
                 tc_fence_after();
                 const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
@@ -354,7 +265,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     if (warp >= kDequantWarps) {
         // ---------------- epilogue: TMEM -> registers -> y[token][row] ----------------
         __syncwarp();
-        if (lane == 0 && !mbar_wait(acc_ready, 0)) time_out();
+        if (lane == 0 && !mbar_wait(acc_ready, 0, kPrefillSpin)) time_out();
         __syncwarp();
         tc_fence_after();
         const int lane_base = (warp & 3) * 32;  // a warp may read the 32 TMEM lanes of its quarter
@@ -407,7 +318,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     __syncthreads();
     if (warp == kDequantWarps + 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+        tmem_dealloc(tmem, tmem_cols);
     }
 }
 
@@ -464,11 +375,7 @@ cudaError_t launch_prefill_bits(const PrefillParams& p, const CUtensorMap& mx, c
 }  // namespace
 
 bool prefill_supported(const lopro_desc& d, int T) {
-    static int off = -1;
-    if (off < 0) {
-        const char* e = getenv("LOPRO_NO_TCGEN05");  // tuning / A-B comparison only
-        off = (e != nullptr && e[0] == '1') ? 1 : 0;
-    }
+    const int off = option(LOPRO_OPT_NO_TCGEN05) == 1 ? 1 : 0;  // tuning / A-B comparison only
     return off == 0 && T > kDecodeMaxT && encode_tiled_fn() != nullptr && (d.d_in % 64) == 0;
 }
 
@@ -511,16 +418,17 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     const int units = (T + p.tile_n - 1) / p.tile_n;
     const int m_tiles = (d.d_out + kTileM - 1) / kTileM;
     int best_pairs = m_tiles / 2;
+    const int n_sm = sm_count() < 256 ? sm_count() : 256;
     if ((long long)m_tiles * units <= 20000) {
         double best_cost = 1e30;
         for (int pairs = m_tiles / 2; pairs >= 0; --pairs) {
             const int singles = m_tiles - 2 * pairs;
-            double finish[148];
-            for (int i = 0; i < 148; ++i) finish[i] = 0.0;
+            double finish[256];
+            for (int i = 0; i < n_sm; ++i) finish[i] = 0.0;
             auto place = [&](long long count, double dur) {
                 for (long long c = 0; c < count; ++c) {
                     int best = 0;
-                    for (int i = 1; i < 148; ++i)
+                    for (int i = 1; i < n_sm; ++i)
                         if (finish[i] < finish[best]) best = i;
                     finish[best] += dur;
                 }
@@ -528,7 +436,7 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
             place((long long)pairs * units, kPairCost);
             place((long long)singles * units, 1.0);
             double cost = 0.0;
-            for (int i = 0; i < 148; ++i) cost = finish[i] > cost ? finish[i] : cost;
+            for (int i = 0; i < n_sm; ++i) cost = finish[i] > cost ? finish[i] : cost;
             if (cost < best_cost - 1e-9) {
                 best_cost = cost;
                 best_pairs = pairs;
@@ -536,11 +444,7 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
         }
     }
     {
-        static int forced = -2;  // LOPRO_PREFILL_PAIRS overrides the choice (tuning only)
-        if (forced == -2) {
-            const char* e = getenv("LOPRO_PREFILL_PAIRS");
-            forced = e ? atoi(e) : -1;
-        }
+        const int forced = option(LOPRO_OPT_PREFILL_PAIRS);  // overrides the choice (tuning only)
         if (forced >= 0 && forced <= m_tiles / 2) best_pairs = forced;
     }
     p.pair_tiles = best_pairs;

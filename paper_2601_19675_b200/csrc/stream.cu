@@ -573,14 +573,10 @@ bool plan_layout(const lopro_desc& d, StreamPlan* pl, int r_pad, int ng, int kto
 
 }  // namespace
 
-// The 32-warp variant runs for up to 8 tokens when all of K fits the ring; LOPRO_NO_WIDE=1 keeps it off (A/B
+// The 32-warp variant runs for up to 8 tokens when all of K fits the ring; LOPRO_OPT_NO_WIDE keeps it off (A/B
 // comparison and tests).
 static bool wide_variant(const lopro_desc& d, const StreamPlan& pl) {
-    static int no_wide = -1;
-    if (no_wide < 0) {
-        const char* e = getenv("LOPRO_NO_WIDE");
-        no_wide = (e != nullptr && e[0] == '1') ? 1 : 0;
-    }
+    const bool no_wide = option(LOPRO_OPT_NO_WIDE) == 1;
     return !no_wide && pl.nt == 1 && pl.rt == 2 && pl.n_stages == pl.total_stages &&
            pl.off_stage_x == 2 * kStageSteps * 128 * d.bits;  // the variant's compile-time stage geometry
 }

@@ -375,19 +375,6 @@ struct TallPlan {
     int off_a, a_bytes, off_t, off_red, off_ring, stage_bytes, off_stage_sz, off_stage_x, smem_bytes;
 };
 
-int sm_count() {
-    static int cached[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    int& c = cached[dev & 63];
-    if (c == 0) {
-        int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
-        c = v;
-    }
-    return c;
-}
-
 bool plan_tall(const lopro_desc& d, int T, TallPlan* pl) {
     if (T < 1 || T > kDecodeMaxT) return false;
     const int n_sm = sm_count();

@@ -22,7 +22,8 @@ SEC_HEADER, SEC_CODES, SEC_SCALEZERO, SEC_PERM, SEC_A, SEC_B = range(6)
 # every symbol include/lopro.h declares
 SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packed_bytes", "lopro_packed_section",
            "lopro_workspace_bytes", "lopro_pack", "lopro_unpack", "lopro_rotate", "lopro_linear_fwd",
-           "lopro_linear_fwd_path", "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc"]
+           "lopro_linear_fwd_path", "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc",
+           "lopro_configure", "lopro_selftest_wait"]
 
 
 class Desc(ctypes.Structure):
@@ -80,8 +81,39 @@ def lib():
         L.lopro_linear_fwd_host.argtypes = [dp, vp, vp, vp, i32, i32, vp, sz, vp]
         L.lopro_linear_fwd_noalloc.restype = ctypes.c_int
         L.lopro_linear_fwd_noalloc.argtypes = [dp, vp, vp, i64, vp, i64, i32, i32, vp]
+        L.lopro_configure.restype = ctypes.c_int
+        L.lopro_configure.argtypes = [i32, i32]
+        L.lopro_selftest_wait.restype = ctypes.c_int
+        L.lopro_selftest_wait.argtypes = [vp, vp]
         _lib = L
     return _lib
+
+
+OPT_NO_WIDE, OPT_NO_TALL, OPT_NO_CHUNKS, OPT_NO_TCGEN05, OPT_PREFILL_PAIRS = range(5)
+
+
+def configure(option, value):
+    """lopro_configure: set one tuning switch for the process (which kernels run, never what they compute)."""
+    _check(lib().lopro_configure(int(option), int(value)), "lopro_configure")
+
+
+class configured:
+    """Context manager: a tuning switch set for the duration of a block, then back to its default (0; -1 for
+    OPT_PREFILL_PAIRS)."""
+
+    def __init__(self, option, value):
+        self.option, self.value = option, value
+
+    def __enter__(self):
+        configure(self.option, self.value)
+
+    def __exit__(self, *exc):
+        configure(self.option, -1 if self.option == OPT_PREFILL_PAIRS else 0)
+
+
+def selftest_wait(status_word):
+    """lopro_selftest_wait: status_word is a device int32 tensor of one element; read it after synchronising."""
+    _check(lib().lopro_selftest_wait(_ptr(status_word), _stream()), "lopro_selftest_wait")
 
 
 def version():

@@ -120,3 +120,27 @@ def test_null_and_bad_arguments_are_rejected_before_any_cuda_call():
     assert L.lopro_rotate(ctypes.byref(d), fake, fake, 500, fake, 512, 4, None) == lopro.ERR_INVALID_ARG
     assert L.lopro_linear_fwd(ctypes.byref(d), fake, fake, 512, fake, 100, 0, 4, fake, 1 << 30, None) == lopro.ERR_INVALID_ARG
     assert L.lopro_linear_fwd(ctypes.byref(d), fake, fake, 512, fake, 512, 0, 4, fake, 16, None) == lopro.ERR_BUFFER_TOO_SMALL
+
+
+@pytest.mark.parametrize("n,r", [(4096, 32), (8192, 128), (32768, 17), (4096, 0)])
+def test_workspace_size_never_decreases_with_the_token_count(n, r):
+    # a workspace sized once for the largest batch must serve every smaller one
+    d = lopro.make_desc(n, 256, 2, 64, 256, rank=r)
+    prev = 0
+    for t in range(1, 8193):
+        cur = lopro.workspace_bytes(d, t)
+        assert cur >= prev, (t, cur, prev)
+        prev = cur
+
+
+def test_configure_rejects_unknown_options():
+    import ctypes
+    L = lopro.lib()
+    assert L.lopro_configure(99, 1) == lopro.ERR_INVALID_ARG
+    assert L.lopro_configure(-1, 1) == lopro.ERR_INVALID_ARG
+    d = lopro.make_desc(4096, 4096, 4, 128, 128, rank=32)
+    with lopro.configured(lopro.OPT_NO_WIDE, 1):
+        assert lopro.linear_fwd_path(d, 8) == (lopro.PATH_STREAM, 2)
+    assert lopro.linear_fwd_path(d, 8) == (lopro.PATH_WIDE, 2)
+    assert L.lopro_selftest_wait(None, None) == lopro.ERR_INVALID_ARG
+    assert L.lopro_selftest_wait(ctypes.c_void_p(0x1002), None) == lopro.ERR_INVALID_ARG

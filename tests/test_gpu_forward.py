@@ -5,8 +5,6 @@ Gate B: fp32 output (fp32 accumulation) against the mirrored oracle, which appli
 library declares (rotated activations to bf16, low-rank intermediate to fp16, and where the forward
 runs the tensor-core prefill kernel the dequantized weights to bf16), <= 1e-3.
 The error measure is oracle.max_rel_err (element-wise, relative to max(|y|, rms of the token's row))."""
-import os
-
 import numpy as np
 import pytest
 import torch
@@ -31,13 +29,10 @@ def _check_forward(layer, d, x_bits, rows=None, gate_a=GATE_A, gate_b=GATE_B):
     (more than 32 tokens, few output rows) the tensor-core prefill path is checked as well."""
     T = x_bits.shape[0]
     res = _check_forward_once(layer, d, x_bits, rows, gate_a, gate_b)
-    if T > 32 and lopro.linear_fwd_path(d, T)[0] != lopro.PATH_PREFILL and "LOPRO_NO_CHUNKS" not in os.environ:
-        os.environ["LOPRO_NO_CHUNKS"] = "1"
-        try:
+    if T > 32 and lopro.linear_fwd_path(d, T)[0] != lopro.PATH_PREFILL:
+        with lopro.configured(lopro.OPT_NO_CHUNKS, 1):
             if lopro.linear_fwd_path(d, T)[0] == lopro.PATH_PREFILL:
                 _check_forward_once(layer, d, x_bits, rows, gate_a, gate_b)
-        finally:
-            del os.environ["LOPRO_NO_CHUNKS"]
     return res
 
 
@@ -241,7 +236,7 @@ def test_rotated_entry_on_a_bf16_rounding_boundary():
     _check_forward(layer, d, synth.activations(T, n, seed=T))
 
 
-def test_tall_kernel_agrees_with_the_per_group_kernel(monkeypatch):
+def test_tall_kernel_agrees_with_the_per_group_kernel():
     # both small-batch kernels sum the same products in fp32 in different orders: outputs agree to fp32 rounding
     n, m, bits, g, r, T = 1024, _tall_rows(4, 9), 4, 128, 32, 8
     d = lopro.make_desc(n, m, bits, g, 128, rank=r)
@@ -249,9 +244,9 @@ def test_tall_kernel_agrees_with_the_per_group_kernel(monkeypatch):
     blob = _pack(layer, d)
     x = bf16_bits_to_device(synth.activations(T, n, seed=4))
     y_tall = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
-    monkeypatch.setenv("LOPRO_NO_TALL", "1")
-    assert lopro.linear_fwd_path(d, T)[0] in (lopro.PATH_STREAM, lopro.PATH_WIDE)
-    y_stream = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
+    with lopro.configured(lopro.OPT_NO_TALL, 1):
+        assert lopro.linear_fwd_path(d, T)[0] in (lopro.PATH_STREAM, lopro.PATH_WIDE)
+        y_stream = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
     torch.cuda.synchronize()
     scale = y_stream.abs().max().item()
     assert (y_tall - y_stream).abs().max().item() <= 1e-5 * scale
@@ -317,3 +312,20 @@ def test_host_entry_point_matches_device_entry_point(T):
     lopro.linear_fwd_host(d, blob, xh, yh, ws)
     torch.cuda.synchronize()
     assert torch.equal(yh, y_dev.cpu())
+
+
+def test_a_bounded_wait_that_runs_out_reports_a_timeout():
+    # the library's own self-test: a barrier that nothing completes, waited on with the bounded wait every
+    # forward kernel uses; the wait gives up, the kernel returns normally and the status word says so
+    word = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    lopro.selftest_wait(word)
+    torch.cuda.synchronize()
+    assert int(word.item()) == lopro.ERR_TIMEOUT
+    # the context is intact: an ordinary forward still runs and reports OK
+    n, m = 512, 64
+    d = lopro.make_desc(n, m, 4, 128, 64, rank=0)
+    blob = _pack(random_layer_np(n, m, 4, 128, 0, seed=1), d)
+    ws = torch.zeros(lopro.workspace_bytes(d, 4), dtype=torch.uint8, device="cuda")
+    y = lopro.linear_fwd(d, blob, torch.ones((4, n), dtype=torch.bfloat16, device="cuda"), workspace=ws)
+    torch.cuda.synchronize()
+    assert lopro.workspace_status(ws) == lopro.OK and torch.isfinite(y.float()).all()

@@ -121,3 +121,20 @@ def test_unpack_rejects_mismatched_descriptor():
     with pytest.raises(lopro.LoproError) as e:
         lopro.unpack(d2, blob)
     assert e.value.status == lopro.ERR_INVALID_DATA
+
+
+def test_a_rejected_blob_holds_no_out_of_range_index():
+    # a permutation with entries outside [0, n) is rejected, and what is left in the blob cannot send a forward
+    # out of bounds: the permutation section reads back all zeros (checked on the host; no forward is run on it)
+    n, m, bits, g, r = 512, 64, 4, 128, 0
+    layer = random_layer_np(n, m, bits, g, r, seed=8)
+    d = lopro.make_desc(n, m, bits, g, 64, rank=r)
+    bad = layer["perm"].copy()
+    bad[5], bad[77] = n + 1000, -3
+    dev = to_device(dict(layer, perm=bad))
+    blob = torch.full((lopro.packed_bytes(d),), 0xFF, dtype=torch.uint8, device="cuda")
+    with pytest.raises(lopro.LoproError) as e:
+        lopro.pack(d, dev["codes"], dev["scales"], dev["zeros"], dev["perm"], out=blob)
+    assert e.value.status == lopro.ERR_INVALID_DATA
+    perm_back = lopro.perm_of(d, blob).cpu().numpy()
+    assert perm_back.min() >= 0 and perm_back.max() < n

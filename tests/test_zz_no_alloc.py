@@ -56,16 +56,15 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(n, m, bits, g, b, r)
 
 
 @pytest.mark.parametrize("no_chunks", [False, True])
-def test_more_than_32_tokens_inside_the_fixed_scratch(no_chunks, monkeypatch):
+def test_more_than_32_tokens_inside_the_fixed_scratch(no_chunks):
     # 40 and 33 tokens still fit the built-in array: as chunks of 32 through the small-batch kernels, and (with the
     # library's switch for it) through the tensor-core kernel
     n, m = 1024, 256
     d, blob = _layer(n, m, 4, 128, 128, 16, seed=13)
-    if no_chunks:
-        monkeypatch.setenv("LOPRO_NO_CHUNKS", "1")
-    assert lopro.workspace_bytes(d, 40) <= lopro.NOALLOC_SCRATCH_BYTES
-    assert (lopro.linear_fwd_path(d, 40)[0] == lopro.PATH_PREFILL) == no_chunks
-    _two_calls(d, blob, n, m, (40, 33))
+    with lopro.configured(lopro.OPT_NO_CHUNKS, 1 if no_chunks else 0):
+        assert lopro.workspace_bytes(d, 40) <= lopro.NOALLOC_SCRATCH_BYTES
+        assert (lopro.linear_fwd_path(d, 40)[0] == lopro.PATH_PREFILL) == no_chunks
+        _two_calls(d, blob, n, m, (40, 33))
 
 
 def test_requests_beyond_the_fixed_scratch_are_refused():
