@@ -289,7 +289,8 @@ def run_stack(args, T, rank, world, local, dev, dev16):
         layer = synth.random_layer(n, m, q["bits"], q["group_size"], q["rank"], seed=rank + n // 64)
         base[(n, m)] = dict(codes=torch.from_numpy(layer["codes"]).to(dev), sc=dev16(layer["scales"]), zr=dev16(layer["zeros"]),
                             pm=torch.from_numpy(layer["perm"]).to(dev), A=dev16(layer["A"]), B=dev16(layer["B"]))
-        descs[(n, m)] = lopro.make_desc(n, m, q["bits"], q["group_size"], q["block_size"], q["identity_cols"], q["rank"])
+        descs[(n, m)] = lopro.make_desc(n, m, q["bits"], q["group_size"], q["block_size"], q["identity_cols"], q["rank"],
+                                        layout=lopro.LAYOUT_ROWBLOCK if args.layout == "rowblock" else lopro.LAYOUT_FRAGMENT)
     xs, x_bits = {}, {}
     for n in sorted({n for n, _ in shapes}):
         x_bits[n] = synth.activations(T, n, seed=rank + n)
@@ -412,6 +413,7 @@ def main():
     ap.add_argument("--impl", default="lopro", choices=["lopro", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch through the stream instead of a CUDA graph")
+    ap.add_argument("--layout", default="fragment", choices=["fragment", "rowblock"], help="code layout of the packed layers")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -445,7 +447,8 @@ def main():
     if cfg == "cfg5":
         return run_stack(args, T, rank, world, local, dev, dev16)
     c = synth.CONFIGS[cfg]
-    d = lopro.make_desc(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"])
+    d = lopro.make_desc(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"],
+                        layout=lopro.LAYOUT_ROWBLOCK if args.layout == "rowblock" else lopro.LAYOUT_FRAGMENT)
 
     # ring of distinct layers: layer 0 drawn by the seeded generator, the others re-use its tensors with
     # freshly drawn codes (generated on the host once, shifted per layer) so that set-up stays short
@@ -551,7 +554,7 @@ def main():
     path, kernels_per_forward = lopro.linear_fwd_path(d, T)
     path_name = lopro.PATH_NAMES.get(path, "?")
     kernel_name = {"stream": "stream_kernel", "wide": "stream_wide_kernel", "tall": "tall_kernel", "general": "decode_kernel",
-                   "prefill": "prefill_kernel"}.get(path_name, "?")
+                   "prefill": "prefill_kernel", "rowblock": "rowblock_kernel"}.get(path_name, "?")
     note = "duration = step time / layer forwards (includes the prologue kernels)"
     launches_per_step = ring
     dur_s = ms_per_step * 1e-3 / launches_per_step

@@ -66,7 +66,9 @@ enum {
     LOPRO_LAYOUT_CANONICAL = 0, /* per row, code k occupies bits [k q, (k+1) q) of a little-endian
                                    bit stream stored as uint32 words (4-bit: 8 codes per word, low
                                    nibble first); interchange format, not accepted by the forward */
-    LOPRO_LAYOUT_FRAGMENT = 1   /* tensor-core fragment order read by the forward kernels         */
+    LOPRO_LAYOUT_FRAGMENT = 1,  /* register-fragment order of the warp-level tensor-core kernels   */
+    LOPRO_LAYOUT_ROWBLOCK = 2   /* blocks of 128 rows x 64 columns, a row's codes together: the order
+                                   the tcgen05 kernels expand into shared-memory operand tiles    */
 };
 
 /* Descriptor of one quantized layer (plain data, host memory).
@@ -210,7 +212,9 @@ typedef enum {
     LOPRO_PATH_GENERAL = 3,
     LOPRO_PATH_PREFILL = 4,
     LOPRO_PATH_TALL = 5,
-    LOPRO_PATH_WIDE = 6
+    LOPRO_PATH_WIDE = 6,
+    LOPRO_PATH_ROWBLOCK = 7  /* row-block layout: operand image (1 launch; 2-3 for descriptors the prologue kernel
+                                does not take) + one tcgen05 small-batch launch per group of up to 32 tokens   */
 } lopro_path;
 LOPRO_API int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches);
 
@@ -245,7 +249,7 @@ LOPRO_API lopro_status lopro_linear_fwd_host(const lopro_desc* desc, const void*
  *     it: order every use of this entry point on a device through one stream.
  *   - The workspace status word of lopro_linear_fwd is not visible here; use lopro_linear_fwd when
  *     the device-side status matters. */
-#define LOPRO_NOALLOC_SCRATCH_BYTES (2 * 1024 * 1024)
+#define LOPRO_NOALLOC_SCRATCH_BYTES (8 * 1024 * 1024)
 LOPRO_API lopro_status lopro_linear_fwd_noalloc(const lopro_desc* desc, const void* packed, const uint16_t* x_bf16,
                                                 int64_t ldx, void* y, int64_t ldy, int32_t out_dtype, int32_t T,
                                                 void* stream);

@@ -14,7 +14,8 @@ lopro_status check_desc(const lopro_desc& d) {
     if (d.identity_cols < 0 || d.identity_cols > d.d_in) return LOPRO_ERR_INVALID_ARG;
     if ((d.d_in - d.identity_cols) % d.block_size != 0) return LOPRO_ERR_INVALID_ARG;
     if (d.rank < 0 || d.rank > 512) return LOPRO_ERR_INVALID_ARG;
-    if (d.layout != LOPRO_LAYOUT_CANONICAL && d.layout != LOPRO_LAYOUT_FRAGMENT) return LOPRO_ERR_INVALID_ARG;
+    if (d.layout != LOPRO_LAYOUT_CANONICAL && d.layout != LOPRO_LAYOUT_FRAGMENT && d.layout != LOPRO_LAYOUT_ROWBLOCK)
+        return LOPRO_ERR_INVALID_ARG;
     // Kernel coverage: 64-column steps, 16-row tiles, rows short enough for one CTA's shared memory.
     if (d.d_in % 64 != 0 || d.d_out % 16 != 0 || d.group_size % 64 != 0) return LOPRO_ERR_UNSUPPORTED;
     if ((d.group_size / 64) & (d.group_size / 64 - 1)) return LOPRO_ERR_UNSUPPORTED;  // g = 64 * 2^k
@@ -68,8 +69,42 @@ lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
     off += round_up_size((size_t)t_pad * (r_pad > 0 ? r_pad : 16) * 2, 256);
     W->off_lrpart = off;
     if (T > kDecodeMaxT && d.rank > 0) off += round_up_size(lowrank_mma_scratch_bytes(d, T), 256);
+    // operand image of the tcgen05 small-batch kernel (row-block layout)
+    W->np = T <= 16 ? 16 : 32;
+    W->n_tgroups = T <= 16 ? 1 : (T + 31) / 32;
+    W->off_counters = W->off_ximg = W->off_sums = W->off_timg = W->off_partial = off;
+    if (d.layout == LOPRO_LAYOUT_ROWBLOCK) {
+        const size_t tg = (size_t)W->n_tgroups;
+        W->off_counters = off;
+        off += round_up_size((size_t)((d.d_out + kRbRows - 1) / kRbRows) * 4, 256);
+        W->off_ximg = round_up_size(off, 1024);
+        off = W->off_ximg + tg * ximg_bytes(d.d_in, W->np);
+        W->off_sums = off;
+        off += round_up_size(tg * (size_t)(d.d_in / sum_run(d)) * W->np * 4, 1024);
+        W->off_timg = off;
+        off += tg * (size_t)((r_pad + 63) / 64) * W->np * 128;
+        W->off_partial = off;
+        off += (size_t)2 * kRbMaxGrid * W->np * kRbRows * 4;
+    }
     W->total = off;
     return LOPRO_OK;
+}
+
+ImageOut image_out(const lopro_desc& d, uint8_t* ws, const WorkspaceLayout& W) {
+    ImageOut o;
+    o.ximg = ws + W.off_ximg;
+    o.sums = reinterpret_cast<float*>(ws + W.off_sums);
+    o.timg = ws + W.off_timg;
+    o.counters = reinterpret_cast<int*>(ws + W.off_counters);
+    o.n_counters = (d.d_out + kRbRows - 1) / kRbRows;
+    o.np = W.np;
+    o.np_shift = W.np == 16 ? 4 : 5;
+    o.nsteps = d.d_in / 64;
+    const int gs = sum_run(d);
+    o.gs_shift = gs == 64 ? 0 : (gs == 128 ? 1 : 2);
+    o.n_sums = d.d_in / gs;
+    o.lr_steps = (round_up_int(d.rank, 16) + 63) / 64;
+    return o;
 }
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
@@ -269,8 +304,19 @@ static int small_batch_chunks(const lopro_desc& d, int T) {
     return chunks;
 }
 
+// Row-block layout: launches before the product (the prologue, or rotation + B x + image conversion).
+static int rowblock_pre_launches(const lopro_desc& d, int T) {
+    if (prologue_supported(d, 1)) return 1;
+    return 2 + (d.rank > 0 ? 1 : 0);
+}
+
 int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches) {
-    if (!desc || check_desc(*desc) != LOPRO_OK || desc->layout != LOPRO_LAYOUT_FRAGMENT || T < 1) return 0;
+    if (!desc || check_desc(*desc) != LOPRO_OK || desc->layout == LOPRO_LAYOUT_CANONICAL || T < 1) return 0;
+    if (desc->layout == LOPRO_LAYOUT_ROWBLOCK) {
+        if (!rowblock_supported(*desc)) return 0;
+        if (launches) *launches = rowblock_pre_launches(*desc, T) + (T <= 16 ? 1 : (T + 31) / 32);
+        return LOPRO_PATH_ROWBLOCK;
+    }
     int32_t path, n;
     if (const int chunks = small_batch_chunks(*desc, T)) {
         path = use_tall(*desc, kDecodeMaxT) ? LOPRO_PATH_TALL : LOPRO_PATH_STREAM;
@@ -296,7 +342,8 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     BlobLayout L;
     lopro_status st = blob_layout(*desc, &L);
     if (st != LOPRO_OK) return st;
-    if (desc->layout != LOPRO_LAYOUT_FRAGMENT) return LOPRO_ERR_UNSUPPORTED;
+    if (desc->layout == LOPRO_LAYOUT_CANONICAL) return LOPRO_ERR_UNSUPPORTED;
+    if (desc->layout == LOPRO_LAYOUT_ROWBLOCK && !rowblock_supported(*desc)) return LOPRO_ERR_UNSUPPORTED;
     if (T < 0 || (out_dtype != LOPRO_OUT_BF16 && out_dtype != LOPRO_OUT_F32)) return LOPRO_ERR_INVALID_ARG;
     if (T == 0) return LOPRO_OK;
     if (!packed || !x_bf16 || !y || !workspace) return LOPRO_ERR_INVALID_ARG;
@@ -317,6 +364,31 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     __nv_bfloat16* xrot = (__nv_bfloat16*)(ws + W.off_xrot);
     float* s64 = (float*)(ws + W.off_s64);
     int* status = (int*)(ws + W.off_status);
+    if (desc->layout == LOPRO_LAYOUT_ROWBLOCK) {
+        // operand image (one launch where the prologue kernel takes the descriptor), then one tcgen05 launch per
+        // group of up to 32 tokens
+        const ImageOut img = image_out(*desc, ws, W);
+        if (prologue_supported(*desc, 1)) {
+            if (launch_prologue(*desc, perm, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, nullptr, nullptr, W.t_pad, status,
+                                T, s, &img) != cudaSuccess)
+                return LOPRO_ERR_CUDA;
+        } else {
+            if (launch_rotate(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, xrot, desc->d_in, s64, status, T, s) !=
+                cudaSuccess)
+                return LOPRO_ERR_CUDA;
+            if (desc->rank > 0 && launch_lowrank_down(*desc, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx,
+                                                      (__half*)(ws + W.off_t), T, s) != cudaSuccess)
+                return LOPRO_ERR_CUDA;
+            if (launch_image_convert(*desc, xrot, s64, s64_stride(desc->d_in), (const __half*)(ws + W.off_t), L.r_pad, img, T,
+                                     s) != cudaSuccess)
+                return LOPRO_ERR_CUDA;
+        }
+        for (int tg = 0; tg < W.n_tgroups; ++tg) {
+            const int live = T - tg * W.np < W.np ? T - tg * W.np : W.np;
+            if (launch_rowblock(*desc, blob, L, ws, W, y, ldy, out_dtype, tg, live, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+        }
+        return LOPRO_OK;
+    }
     if (const int chunks = small_batch_chunks(*desc, T)) {
         // one prologue for all tokens, then chunks of kDecodeMaxT tokens through the small-batch kernels, each
         // reading its tokens' records of the activation image and rows of t

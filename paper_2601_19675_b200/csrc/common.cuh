@@ -75,6 +75,10 @@ inline size_t round_up_size(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct WorkspaceLayout {
     size_t off_status, off_xrot, off_s64, off_t, off_lrpart, total;
     int t_pad;  // tokens padded to a multiple of 8
+    // row-block layout only: the operand image of the tcgen05 small-batch kernel (see ImageOut)
+    size_t off_counters, off_ximg, off_sums, off_timg, off_partial;
+    int np;        // tokens per image tile: 16 (T <= 16) or 32
+    int n_tgroups; // token groups of np tokens
 };
 constexpr int kDecodeMaxT = 32;               // tokens per CTA of the streaming kernels
 constexpr int kStreamMaxSmem = 220 * 1024;    // dynamic shared memory the small-batch kernel may use
@@ -88,6 +92,29 @@ inline int s64_stride(int n) { return ((n / 64 + 15) / 16) * 16; }
 constexpr int kActRecord = 2048 + 64 + 16;
 inline size_t act_image_bytes(int n, int t_pad) { return (size_t)((n + 1023) / 1024) * t_pad * kActRecord; }
 lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* out);
+
+// Operand image of the tcgen05 small-batch kernel, written by the prologue (or converted from the plain rotated
+// activations): per group of NP tokens and 64-column step one K-major tile [NP tokens][64 columns] of bf16 with the
+// 128-byte swizzle the MMA reads (token row tl, 16-byte piece c at byte tl * 128 + ((c ^ (tl & 7)) << 4)), so that a
+// plain bulk copy brings a tile; sums of the rotated (bf16-rounded) activations over runs of gs = min(g, 256) columns,
+// [token group][run][NP] fp32; the low-rank intermediate t = B x as fp16 tiles of the same shape over the rank; and
+// the per-row-block arrival counters of the split-K reduction, cleared by whoever writes the image.
+constexpr int kRbMaxGrid = 160;  // CTAs of the tcgen05 small-batch kernel (one per SM), bound used to size the partial sums
+struct ImageOut {
+    unsigned char* ximg;  // nullptr: the record format of the warp-level kernels is written instead
+    float* sums;
+    unsigned char* timg;
+    int* counters;
+    int n_counters;
+    int np, np_shift;   // tokens per tile (16 or 32) and its log2
+    int nsteps;         // 64-column steps of K
+    int gs_shift;       // log2(gs / 64): 0, 1 or 2
+    int n_sums;         // d_in / gs
+    int lr_steps;       // 64-column steps of the padded rank
+};
+inline size_t ximg_bytes(int n, int np) { return (size_t)(n / 64) * np * 128; }
+inline int sum_run(const lopro_desc& d) { return d.group_size < 256 ? d.group_size : 256; }
+ImageOut image_out(const lopro_desc& d, uint8_t* ws, const WorkspaceLayout& W);
 
 // ---- launchers (each returns the CUDA status of its launches) -------------------------------
 cudaError_t launch_validate(const lopro_desc& d, const uint8_t* codes, const uint16_t* scales,
@@ -107,7 +134,15 @@ cudaError_t launch_rotate(const lopro_desc& d, const int32_t* perm, const __nv_b
 bool prologue_supported(const lopro_desc& d, int T);
 cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
                             const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, __half* t, int t_pad,
-                            int* status, int T, cudaStream_t s);
+                            int* status, int T, cudaStream_t s, const ImageOut* img = nullptr);
+// Plain rotated activations, 64-column sums and t (the general path's outputs) -> operand image.
+cudaError_t launch_image_convert(const lopro_desc& d, const __nv_bfloat16* xrot, const float* s64, int s64_ld,
+                                 const __half* t, int r_pad, const ImageOut& img, int T, cudaStream_t s);
+// tcgen05 small-batch forward over the row-block layout, one launch per group of up to 32 tokens.
+bool rowblock_supported(const lopro_desc& d);
+cudaError_t launch_rowblock(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, uint8_t* ws,
+                            const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int tgroup, int t_live,
+                            cudaStream_t s);
 // t[T][r_pad] (fp16) = B x, fp32 accumulation.
 cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,
                                 int64_t ldx, __half* t, int T, cudaStream_t s);
@@ -179,6 +214,61 @@ __host__ __device__ inline FragPos frag_pos(int bits, int n, int row, int k) {
         }
     }
     return p;
+}
+
+// ---- row-block layout -------------------------------------------------------------------------
+// Codes are stored per block of up to 128 rows (the last block holds the remaining rows, a multiple of 16) and
+// 64-column step: R rows x 2 q words, the steps of a block one after the other, so that any run of steps of a block
+// is one contiguous piece.  A row's 2 q words of a step are its two 32-column half-steps, each q words in the bit
+// order of expand_codes with pair pi = columns (2 pi, 2 pi + 1) of the half-step: expanding a half-step yields the
+// row's 32 columns as sixteen bf16 pairs in memory order, i.e. four 16-byte pieces of a K-major operand tile.  Inside
+// a (block, step) the words are kept as planes of 4 words per row (the last plane of a 3-bit step has 2), [plane][row],
+// so that thread r of a warp reads its row's plane with one conflict-free 16-byte (8-byte) load.
+constexpr int kRbRows = 128;
+
+__host__ __device__ inline int rb_rows(int m, int rb) { return m - rb * kRbRows < kRbRows ? m - rb * kRbRows : kRbRows; }
+// word offset of the (block, step) piece inside the code section
+__host__ __device__ inline size_t rb_step_word(int bits, int nsteps, int m, int rb, int ks) {
+    return ((size_t)rb * kRbRows * (size_t)nsteps + (size_t)ks * (size_t)rb_rows(m, rb)) * (size_t)(2 * bits);
+}
+// word offset of word w (0 .. 2 q - 1) of row r inside a (block, step) piece of R rows
+__host__ __device__ inline int rb_word_in_step(int bits, int R, int r, int w) {
+    const int plane = w >> 2, len = (2 * bits - 4 * plane) < 4 ? (2 * bits - 4 * plane) : 4;
+    return 4 * plane * R + r * len + (w & 3);
+}
+__host__ __device__ inline FragPos rb_pos(int bits, int n, int m, int row, int k) {
+    const int rb = row >> 7, r = row & 127, ks = k >> 6, kk = k & 63, hs = kk >> 5, c = kk & 31, pi = c >> 1, h = c & 1;
+    const int R = rb_rows(m, rb);
+    const size_t base = rb_step_word(bits, n >> 6, m, rb, ks);
+    FragPos p;
+    p.scattered = false;
+    int wi;
+    if (bits == 4) {
+        wi = pi >> 2;
+        p.shift = 4 * (pi & 3) + 16 * h;
+    } else if (bits == 2) {
+        wi = pi >> 3;
+        p.shift = 2 * (pi & 7) + 16 * h;
+    } else if (pi < 15) {
+        wi = pi / 5;
+        p.shift = 3 * (pi % 5) + 16 * h;
+    } else {
+        wi = 0;  // bit b of the code sits at bit `shift` of half-step word b
+        p.shift = 15 + 16 * h;
+        p.scattered = true;
+    }
+    p.word = base + (size_t)rb_word_in_step(bits, R, r, hs * bits + wi);
+    return p;
+}
+// word index of half-step word b (scattered 3-bit codes): words of one half-step may straddle two planes
+__host__ __device__ inline size_t rb_halfstep_word(int bits, int n, int m, int row, int k, int b) {
+    const int rb = row >> 7, r = row & 127, ks = k >> 6, hs = (k & 63) >> 5;
+    return rb_step_word(bits, n >> 6, m, rb, ks) + (size_t)rb_word_in_step(bits, rb_rows(m, rb), r, hs * bits + b);
+}
+// (scale, zero) pairs in the row-block layout: [block][group][R rows] half2.
+__host__ __device__ inline size_t sz_rb_index(int n_groups, int m, int row, int grp) {
+    const int rb = row >> 7;
+    return (size_t)rb * kRbRows * (size_t)n_groups + (size_t)grp * (size_t)rb_rows(m, rb) + (size_t)(row & 127);
 }
 
 // (scale, zero) pairs in the fragment layout: [m/16][n/g][16 rows] half2.

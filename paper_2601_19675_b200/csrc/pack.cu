@@ -83,8 +83,43 @@ __global__ void pack_fragment_kernel(const uint8_t* __restrict__ codes, uint32_t
     for (int b = 0; b < bits; ++b) words[idx * bits + b] = w[b];
 }
 
-__device__ __forceinline__ uint32_t read_code(const uint32_t* __restrict__ words, int layout, int bits, int n, int row,
-                                              int k) {
+// Row-block layout: one thread per (row, 64-column step); writes the row's 2 q words of the step.
+__global__ void pack_rowblock_kernel(const uint8_t* __restrict__ codes, uint32_t* __restrict__ words, int m, int n,
+                                     int bits) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int nsteps = n / 64;
+    if (idx >= (size_t)m * nsteps) return;
+    const int row = (int)(idx / nsteps), ks = (int)(idx % nsteps);
+    const int rb = row >> 7, r = row & 127, R = rb_rows(m, rb);
+    uint32_t* dst = words + rb_step_word(bits, nsteps, m, rb, ks);
+    for (int hs = 0; hs < 2; ++hs) {
+        uint32_t w[4] = {0, 0, 0, 0};
+        for (int pi = 0; pi < 16; ++pi) {
+            const int k = ks * 64 + hs * 32 + 2 * pi;
+            const uint32_t lo = load_code(codes, n, bits, row, k), hi = load_code(codes, n, bits, row, k + 1);
+            if (bits == 4) {
+                w[pi >> 2] |= (lo << (4 * (pi & 3))) | (hi << (16 + 4 * (pi & 3)));
+            } else if (bits == 2) {
+                w[pi >> 3] |= (lo << (2 * (pi & 7))) | (hi << (16 + 2 * (pi & 7)));
+            } else if (pi < 15) {
+                w[pi / 5] |= (lo << (3 * (pi % 5))) | (hi << (16 + 3 * (pi % 5)));
+            } else {
+                for (int b = 0; b < 3; ++b) w[b] |= (((lo >> b) & 1u) << 15) | (((hi >> b) & 1u) << 31);
+            }
+        }
+        for (int b = 0; b < bits; ++b) dst[rb_word_in_step(bits, R, r, hs * bits + b)] = w[b];
+    }
+}
+
+__device__ __forceinline__ uint32_t read_code(const uint32_t* __restrict__ words, int layout, int bits, int m, int n,
+                                              int row, int k) {
+    if (layout == LOPRO_LAYOUT_ROWBLOCK) {
+        const FragPos p = rb_pos(bits, n, m, row, k);
+        if (!p.scattered) return (words[p.word] >> p.shift) & ((1u << bits) - 1u);
+        uint32_t c = 0;
+        for (int b = 0; b < 3; ++b) c |= ((words[rb_halfstep_word(bits, n, m, row, k, b)] >> p.shift) & 1u) << b;
+        return c;
+    }
     if (layout == LOPRO_LAYOUT_FRAGMENT) {
         const FragPos p = frag_pos(bits, n, row, k);
         if (!p.scattered) return (words[p.word] >> p.shift) & ((1u << bits) - 1u);
@@ -104,7 +139,7 @@ __global__ void unpack_codes_kernel(const uint32_t* __restrict__ words, uint8_t*
                                     int bits, int layout) {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)m * n) return;
-    codes[idx] = (uint8_t)read_code(words, layout, bits, n, (int)(idx / n), (int)(idx % n));
+    codes[idx] = (uint8_t)read_code(words, layout, bits, m, n, (int)(idx / n), (int)(idx % n));
 }
 
 __global__ void unpack_words_kernel(const uint32_t* __restrict__ words, uint32_t* __restrict__ out, int m, int n,
@@ -116,7 +151,7 @@ __global__ void unpack_words_kernel(const uint32_t* __restrict__ words, uint32_t
     const int bit0 = 32 * w;
     uint32_t o = 0;
     for (int k = bit0 / bits; k * bits < bit0 + 32 && k < n; ++k) {
-        const uint32_t c = read_code(words, layout, bits, n, row, k);
+        const uint32_t c = read_code(words, layout, bits, m, n, row, k);
         const int pos = k * bits - bit0;
         o |= pos >= 0 ? (c << pos) : (c >> (-pos));
     }
@@ -129,7 +164,8 @@ __global__ void scalezero_kernel(uint16_t* __restrict__ scales, uint16_t* __rest
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)m * ng) return;
     const int row = (int)(idx / ng), grp = (int)(idx % ng);
-    const size_t pos = layout == LOPRO_LAYOUT_FRAGMENT ? sz_frag_index(ng, row, grp) : idx;
+    const size_t pos = layout == LOPRO_LAYOUT_FRAGMENT ? sz_frag_index(ng, row, grp)
+                       : layout == LOPRO_LAYOUT_ROWBLOCK ? sz_rb_index(ng, m, row, grp) : idx;
     if (to_blob) {
         sz[pos] = (uint32_t)scales[idx] | ((uint32_t)zeros[idx] << 16);
     } else {
@@ -175,6 +211,9 @@ cudaError_t launch_pack(const lopro_desc& d, const uint8_t* codes, const uint16_
     if (d.layout == LOPRO_LAYOUT_FRAGMENT) {
         const size_t total = (size_t)(m / 16) * (n / 64) * 32;
         pack_fragment_kernel<<<blocks_for(total, 256), 256, 0, s>>>(codes, words, m, n, d.bits);
+    } else if (d.layout == LOPRO_LAYOUT_ROWBLOCK) {
+        const size_t total = (size_t)m * (n / 64);
+        pack_rowblock_kernel<<<blocks_for(total, 256), 256, 0, s>>>(codes, words, m, n, d.bits);
     } else {
         const size_t total = (size_t)m * (n * d.bits / 32);
         pack_canonical_kernel<<<blocks_for(total, 256), 256, 0, s>>>(codes, words, m, n, d.bits);

@@ -28,6 +28,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// try_wait with a suspend-time hint (ns): the thread may stay parked that long before the instruction returns false
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait for warps that expect to wait long: a failed poll backs off before the next one, so that the polls
+// of many waiting warps do not crowd the shared-memory pipeline of the warps that work.
+__device__ __forceinline__ bool mbar_wait_backoff(uint32_t bar, uint32_t parity, uint32_t limit = kSpinLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
+#if defined(RB_WAIT_HINT)
+        if (mbar_try_wait_hint(bar, parity, RB_WAIT_HINT)) return true;
+#else
+        if (mbar_try_wait(bar, parity)) return true;
+#endif
+#if defined(RB_WAIT_SLEEP)
+        __nanosleep(RB_WAIT_SLEEP);
+#endif
+    }
+    return false;
+}
 // Bounded wait: false if the limit ran out (the caller records the time-out and carries on).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = kSpinLimit) {
     for (uint32_t i = 0; i < limit; ++i)

@@ -79,7 +79,8 @@ __device__ __forceinline__ void prefetch_l2(const void* p) {
 // when the prologue ends.
 template <int TPR>
 __device__ __forceinline__ void lowrank_row(const __nv_bfloat16* __restrict__ x, int64_t ldx, const __half* __restrict__ B,
-                                            __half* __restrict__ t, int n, int r_pad, int T, int rb, int tok0) {
+                                            __half* __restrict__ t, int n, int r_pad, int T, int rb, int tok0,
+                                            const ImageOut& img) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ float part[8][TPR];
     const int j = rb % r_pad, tq = tok0 + TPR * (rb / r_pad);
@@ -155,7 +156,18 @@ __device__ __forceinline__ void lowrank_row(const __nv_bfloat16* __restrict__ x,
         float v = 0.0f;
 #pragma unroll
         for (int w = 0; w < 8; ++w) v += part[w][tid];
-        if (tq + tid < T) t[(size_t)(tq + tid) * r_pad + j] = __float2half_rn(v);
+        if (tq + tid < T) {
+            const int tok = tq + tid;
+            if (img.ximg == nullptr) {
+                t[(size_t)tok * r_pad + j] = __float2half_rn(v);
+            } else {
+                // operand image: tile (token group, 64-column step of the rank), token row tl, swizzled 16-byte piece
+                const int tgp = tok >> img.np_shift, tl = tok & (img.np - 1);
+                unsigned char* tile = img.timg + ((size_t)tgp * img.lr_steps + (j >> 6)) * img.np * 128;
+                *reinterpret_cast<__half*>(tile + tl * 128 + ((((j & 63) >> 3) ^ (tl & 7)) << 4) + (j & 7) * 2) =
+                    __float2half_rn(v);
+            }
+        }
     }
 }
 
@@ -163,7 +175,8 @@ __device__ __forceinline__ void lowrank_row(const __nv_bfloat16* __restrict__ x,
 // gathered entries of the lane.  Register and shuffle butterflies, rounding to bf16, and the store of the entries
 // and of their 64-column sums into the record of (stage, token) in the activation image.
 __device__ __forceinline__ void rotate_tail(const float (&v)[8], unsigned char* __restrict__ act_image, int n, int b_i,
-                                            int b_h, float inv_sqrt_bh, int t_pad, int tok, int col0, int lane) {
+                                            int b_h, float inv_sqrt_bh, int t_pad, int tok, int col0, int lane,
+                                            const ImageOut& img) {
     const bool rot = col0 >= b_i;  // whole Hadamard blocks lie on one side of b_I
     float r[8];
 #pragma unroll
@@ -202,6 +215,21 @@ __device__ __forceinline__ void rotate_tail(const float (&v)[8], unsigned char* 
     sum += __shfl_xor_sync(0xffffffffu, sum, 1);
     sum += __shfl_xor_sync(0xffffffffu, sum, 2);
     sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+    if (img.ximg != nullptr) {
+        // operand image of the tcgen05 kernel: swizzled 16-byte piece of the (token group, step) tile, and the sum
+        // over the run of 64, 128 or 256 columns (a warp's chunk of 256 columns holds whole runs)
+        if (img.gs_shift >= 1) sum += __shfl_xor_sync(0xffffffffu, sum, 8);
+        if (img.gs_shift >= 2) sum += __shfl_xor_sync(0xffffffffu, sum, 16);
+        if (col0 < n) {
+            const int tgp = tok >> img.np_shift, tl = tok & (img.np - 1);
+            unsigned char* tile = img.ximg + ((size_t)tgp * img.nsteps + (col0 >> 6)) * img.np * 128;
+            *reinterpret_cast<uint4*>(tile + tl * 128 + ((((col0 & 63) >> 3) ^ (tl & 7)) << 4)) =
+                *reinterpret_cast<const uint4*>(o);
+            if ((lane & ((8 << img.gs_shift) - 1)) == 0)
+                img.sums[((size_t)tgp * img.n_sums + (col0 >> (6 + img.gs_shift))) * img.np + tl] = sum;
+        }
+        return;
+    }
     if (col0 < n) {
         // record of (stage, token) in the activation image: 1024 entries, then the 16 sums
         unsigned char* rec = act_image + ((size_t)(col0 >> 10) * t_pad + tok) * kActRecord;
@@ -229,7 +257,7 @@ __global__ void __launch_bounds__(256)
 prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
                 const __half* __restrict__ B, unsigned char* __restrict__ act_image, __half* __restrict__ t,
                 int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T,
-                int tpr) {
+                int tpr, const ImageOut img) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nchunks = (n + 255) >> 8;
     const int tok0 = blockIdx.y * 8;
@@ -240,10 +268,10 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
     const int nrow = (int)gridDim.x - (STAGED ? live * ((nchunks + 7) >> 3) : nchunks);
     if ((int)blockIdx.x < nrow) {
         const int rb = (int)blockIdx.x;
-        if (tpr == 8) lowrank_row<8>(x, ldx, B, t, n, r_pad, T, rb, tok0);
-        else if (tpr == 4) lowrank_row<4>(x, ldx, B, t, n, r_pad, T, rb, tok0);
-        else if (tpr == 2) lowrank_row<2>(x, ldx, B, t, n, r_pad, T, rb, tok0);
-        else lowrank_row<1>(x, ldx, B, t, n, r_pad, T, rb, tok0);
+        if (tpr == 8) lowrank_row<8>(x, ldx, B, t, n, r_pad, T, rb, tok0, img);
+        else if (tpr == 4) lowrank_row<4>(x, ldx, B, t, n, r_pad, T, rb, tok0, img);
+        else if (tpr == 2) lowrank_row<2>(x, ldx, B, t, n, r_pad, T, rb, tok0, img);
+        else lowrank_row<1>(x, ldx, B, t, n, r_pad, T, rb, tok0, img);
         return;
     }
 
@@ -261,14 +289,18 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
             pidx[0] = p0.x; pidx[1] = p0.y; pidx[2] = p0.z; pidx[3] = p0.w;
             pidx[4] = p1.x; pidx[5] = p1.y; pidx[6] = p1.z; pidx[7] = p1.w;
         }
-        if (status != nullptr && c == 0 && tok0 == 0 && tid == 0) *status = LOPRO_OK;
+        if (c == 0 && tok0 == 0) {
+            if (status != nullptr && tid == 0) *status = LOPRO_OK;
+            if (img.ximg != nullptr)
+                for (int i = tid; i < img.n_counters; i += 256) img.counters[i] = 0;
+        }
         const int tok = tok0 + warp;
         if (tok < T) {
             float v[8];
             const __nv_bfloat16* xrow = x + (size_t)tok * ldx;
 #pragma unroll
             for (int e = 0; e < 8; ++e) v[e] = col0 < n ? __bfloat162float(xrow[pidx[e]]) : 0.0f;
-            rotate_tail(v, act_image, n, b_i, b_h, inv_sqrt_bh, t_pad, tok, col0, lane);
+            rotate_tail(v, act_image, n, b_i, b_h, inv_sqrt_bh, t_pad, tok, col0, lane, img);
         }
     } else {
         // one token, 8 chunks: warp w takes chunk 8 * (c / live) + w.  perm and the token's row of x are independent
@@ -302,11 +334,15 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
             }
         }
         __syncthreads();
-        if (status != nullptr && c == 0 && tok0 == 0 && tid == 0) *status = LOPRO_OK;  // (token 0 exists: T >= 1)
+        if (c == 0 && tok0 == 0) {  // (token 0 exists: T >= 1)
+            if (status != nullptr && tid == 0) *status = LOPRO_OK;
+            if (img.ximg != nullptr)
+                for (int i = tid; i < img.n_counters; i += 256) img.counters[i] = 0;
+        }
         float v[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) v[e] = col0 < n ? __bfloat162float(xs[pidx[e]]) : 0.0f;
-        rotate_tail(v, act_image, n, b_i, b_h, inv_sqrt_bh, t_pad, tok, col0, lane);
+        rotate_tail(v, act_image, n, b_i, b_h, inv_sqrt_bh, t_pad, tok, col0, lane, img);
     }
 }
 
@@ -354,8 +390,10 @@ bool prologue_supported(const lopro_desc& d, int T) {
 
 cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
                             const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, __half* t, int t_pad,
-                            int* status, int T, cudaStream_t s) {
+                            int* status, int T, cudaStream_t s, const ImageOut* img_out) {
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
+    ImageOut img = {};
+    if (img_out != nullptr) img = *img_out;
     cudaLaunchConfig_t cfg = {};
     // tokens per row CTA: as few as it takes to fill the SMs
     const int live = T < 8 ? T : 8;
@@ -387,9 +425,9 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
     cfg.numAttrs = 1;
     const int rp = d.rank > 0 ? r_pad : 0;
     return staged ? cudaLaunchKernelEx(&cfg, prologue_kernel<true>, x, ldx, perm, B, act_image, t, status, d.d_in,
-                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr)
+                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img)
                   : cudaLaunchKernelEx(&cfg, prologue_kernel<false>, x, ldx, perm, B, act_image, t, status, d.d_in,
-                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr);
+                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img);
 }
 
 cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,

@@ -12,11 +12,12 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liblopro.so")
+# LOPRO_LIBRARY names another build of the library (A/B timing of kernel variants)
+LIB_PATH = os.environ.get("LOPRO_LIBRARY") or os.path.join(_HERE, "liblopro.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT, ERR_INVALID_DATA = range(7)
 OUT_BF16, OUT_F32 = 0, 1
-LAYOUT_CANONICAL, LAYOUT_FRAGMENT = 0, 1
+LAYOUT_CANONICAL, LAYOUT_FRAGMENT, LAYOUT_ROWBLOCK = 0, 1, 2
 SEC_HEADER, SEC_CODES, SEC_SCALEZERO, SEC_PERM, SEC_A, SEC_B = range(6)
 
 # every symbol include/lopro.h declares
@@ -151,8 +152,9 @@ def workspace_bytes(desc, T):
     return int(lib().lopro_workspace_bytes(ctypes.byref(desc), int(T)))
 
 
-PATH_STREAM, PATH_GENERAL, PATH_PREFILL, PATH_TALL, PATH_WIDE = 2, 3, 4, 5, 6
-PATH_NAMES = {PATH_TALL: "tall", PATH_WIDE: "wide", PATH_STREAM: "stream", PATH_GENERAL: "general", PATH_PREFILL: "prefill"}
+PATH_STREAM, PATH_GENERAL, PATH_PREFILL, PATH_TALL, PATH_WIDE, PATH_ROWBLOCK = 2, 3, 4, 5, 6, 7
+PATH_NAMES = {PATH_TALL: "tall", PATH_WIDE: "wide", PATH_STREAM: "stream", PATH_GENERAL: "general", PATH_PREFILL: "prefill",
+              PATH_ROWBLOCK: "rowblock"}
 
 
 def linear_fwd_path(desc, T):
@@ -269,7 +271,7 @@ def linear_fwd_host(desc, packed, x_host, y_host, workspace, out_dtype=OUT_BF16)
     return y_host
 
 
-NOALLOC_SCRATCH_BYTES = 2 * 1024 * 1024
+NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
 def linear_fwd_noalloc(desc, packed, x, y, out_dtype=OUT_BF16):

@@ -29,6 +29,12 @@ def _check_forward(layer, d, x_bits, rows=None, gate_a=GATE_A, gate_b=GATE_B):
     (more than 32 tokens, few output rows) the tensor-core prefill path is checked as well."""
     T = x_bits.shape[0]
     res = _check_forward_once(layer, d, x_bits, rows, gate_a, gate_b)
+    if d.layout == lopro.LAYOUT_FRAGMENT:
+        # the same layer packed in the row-block layout: the tcgen05 small-batch kernel
+        d2 = lopro.make_desc(d.d_in, d.d_out, d.bits, d.group_size, d.block_size, d.identity_cols, d.rank,
+                             layout=lopro.LAYOUT_ROWBLOCK)
+        assert lopro.linear_fwd_path(d2, T)[0] == lopro.PATH_ROWBLOCK
+        _check_forward_once(layer, d2, x_bits, rows, gate_a, gate_b)
     if T > 32 and lopro.linear_fwd_path(d, T)[0] != lopro.PATH_PREFILL:
         with lopro.configured(lopro.OPT_NO_CHUNKS, 1):
             if lopro.linear_fwd_path(d, T)[0] == lopro.PATH_PREFILL:

@@ -12,11 +12,11 @@ from tests._layers import bf16_bits_to_device, device_bf16_to_f64, oracle_args, 
 pytestmark = pytest.mark.gpu
 
 
-def _sampled(cfg, T, n_rows=48, seed=0):
+def _sampled(cfg, T, n_rows=48, seed=0, layout=lopro.LAYOUT_FRAGMENT):
     c = synth.CONFIGS[cfg] if isinstance(cfg, str) else cfg
     n, m = c["d_in"], c["d_out"]
     layer = random_layer_np(n, m, c["bits"], c["group_size"], c["rank"], seed=seed)
-    d = lopro.make_desc(n, m, c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"])
+    d = lopro.make_desc(n, m, c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"], layout=layout)
     dev = to_device(layer)
     blob = lopro.pack(d, dev["codes"], dev["scales"], dev["zeros"], dev["perm"], dev["A"], dev["B"])
     del dev
@@ -43,18 +43,24 @@ def _sampled(cfg, T, n_rows=48, seed=0):
     assert torch.isfinite(y_f32).all()
 
 
+LAYOUTS = [lopro.LAYOUT_FRAGMENT, lopro.LAYOUT_ROWBLOCK]
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
 @pytest.mark.parametrize("T", [1, 8])
-def test_cfg2_decode(T):
-    _sampled("cfg2", T)
+def test_cfg2_decode(T, layout):
+    _sampled("cfg2", T, layout=layout)
 
 
-def test_cfg3_prefill():
-    _sampled("cfg3", 2048, n_rows=32)
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_cfg3_prefill(layout):
+    _sampled("cfg3", 2048, n_rows=32, layout=layout)
 
 
+@pytest.mark.parametrize("layout", LAYOUTS)
 @pytest.mark.parametrize("T", [16, 4096])
-def test_cfg4_large_layer(T):
-    _sampled("cfg4", T, n_rows=24)
+def test_cfg4_large_layer(T, layout):
+    _sampled("cfg4", T, n_rows=24, layout=layout)
 
 
 # the three linear shapes of the 32-layer stack configuration (hidden 4096, MLP 11008; 4-bit, g = 128, rank 32,
@@ -63,7 +69,8 @@ def test_cfg4_large_layer(T):
 _STACK = dict(bits=4, group_size=128, block_size=128, identity_cols=128, rank=32)
 
 
+@pytest.mark.parametrize("layout", LAYOUTS)
 @pytest.mark.parametrize("T", [1, 32])
 @pytest.mark.parametrize("n,m", [(4096, 4096), (4096, 11008), (11008, 4096)])
-def test_stack_linear_shapes(n, m, T):
-    _sampled(dict(d_in=n, d_out=m, **_STACK), T, n_rows=32, seed=n // 64 + T)
+def test_stack_linear_shapes(n, m, T, layout):
+    _sampled(dict(d_in=n, d_out=m, **_STACK), T, n_rows=32, seed=n // 64 + T, layout=layout)

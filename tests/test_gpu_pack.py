@@ -26,7 +26,7 @@ def _same_bits(t, ref_np):
 
 
 @pytest.mark.parametrize("n,m,bits,g,r", CASES)
-@pytest.mark.parametrize("layout", [lopro.LAYOUT_CANONICAL, lopro.LAYOUT_FRAGMENT])
+@pytest.mark.parametrize("layout", [lopro.LAYOUT_CANONICAL, lopro.LAYOUT_FRAGMENT, lopro.LAYOUT_ROWBLOCK])
 def test_pack_unpack_bit_exact(n, m, bits, g, r, layout):
     layer = random_layer_np(n, m, bits, g, r, seed=3)
     dev = to_device(layer)
@@ -52,11 +52,12 @@ def test_pack_unpack_bit_exact(n, m, bits, g, r, layout):
 
 
 @pytest.mark.parametrize("bits", [2, 3, 4])
-def test_walking_patterns_roundtrip(bits):
+@pytest.mark.parametrize("layout", [lopro.LAYOUT_FRAGMENT, lopro.LAYOUT_ROWBLOCK])
+def test_walking_patterns_roundtrip(bits, layout):
     # every code value at every position of a 16 x 64 tile, one at a time in a field of the complement
     n, m, g = 64, 16, 64
     qmax = 2 ** bits - 1
-    d = lopro.make_desc(n, m, bits, g, 64, rank=0)
+    d = lopro.make_desc(n, m, bits, g, 64, rank=0, layout=layout)
     ones = np.full((m, n // g), 0x3C00, dtype=np.uint16)
     perm = torch.arange(n, dtype=torch.int32, device="cuda")
     sc = torch.from_numpy(ones.view(np.int16)).cuda()

@@ -21,9 +21,9 @@ from tests._layers import bf16_bits_to_device, device_bf16_to_f64, random_layer_
 pytestmark = pytest.mark.gpu
 
 
-def _layer(n, m, bits, g, b, r, seed):
+def _layer(n, m, bits, g, b, r, seed, layout=lopro.LAYOUT_FRAGMENT):
     layer = random_layer_np(n, m, bits, g, r, seed=seed)
-    d = lopro.make_desc(n, m, bits, g, b, rank=r)
+    d = lopro.make_desc(n, m, bits, g, b, rank=r, layout=layout)
     dev = to_device(layer)
     blob = lopro.pack(d, dev["codes"], dev["scales"], dev["zeros"], dev["perm"], dev["A"], dev["B"])
     return d, blob
@@ -49,9 +49,12 @@ def _two_calls(d, blob, n, m, token_counts):
         assert o.max_rel_err(y_f32.cpu().numpy().astype(np.float64), ref_f32.cpu().numpy().astype(np.float64)) <= 1e-3
 
 
+@pytest.mark.parametrize("layout", [lopro.LAYOUT_FRAGMENT, lopro.LAYOUT_ROWBLOCK])
 @pytest.mark.parametrize("n,m,bits,g,b,r", [(1024, 272, 4, 128, 128, 16), (2048, 144, 2, 64, 256, 33)])
-def test_two_calls_in_a_row_match_the_workspace_entry_point(n, m, bits, g, b, r):
-    d, blob = _layer(n, m, bits, g, b, r, seed=11)
+def test_two_calls_in_a_row_match_the_workspace_entry_point(n, m, bits, g, b, r, layout):
+    # (row-block layout: blocks of rows shared between thread blocks leave arrival counters and partial sums in the
+    # scratch; the counters must read zero again when the second call starts)
+    d, blob = _layer(n, m, bits, g, b, r, seed=11, layout=layout)
     _two_calls(d, blob, n, m, (8, 3))
 
 
@@ -70,7 +73,7 @@ def test_more_than_32_tokens_inside_the_fixed_scratch(no_chunks):
 def test_requests_beyond_the_fixed_scratch_are_refused():
     n, m = 4096, 64
     d, blob = _layer(n, m, 4, 128, 128, 0, seed=12)
-    T = 1024                                      # needs ~8 MB of scratch: more than the built-in array
+    T = 2048                                      # needs ~17 MB of scratch: more than the built-in array
     assert lopro.workspace_bytes(d, T) > lopro.NOALLOC_SCRATCH_BYTES
     x = torch.zeros((T, n), dtype=torch.bfloat16, device="cuda")
     y = torch.zeros((T, m), dtype=torch.bfloat16, device="cuda")
