@@ -8,21 +8,31 @@
 // when the group's last MMA has completed, the slice is read back and scale and zero-point enter once, in fp32,
 // with the pre-computed column sums of x~.  The rank-r term A t runs as fp16 MMAs into a slice of its own (scale 1).
 //
+// The expanded weights never touch shared memory: a thread expands the 64 codes of one row and step into 32
+// registers of bf16 pairs and stores them with one tcgen05.st into 32 columns of tensor memory, from where the MMA
+// reads its A operand (row = lane).  Shared memory carries only what arrives by bulk copy: packed codes,
+// (scale, zero) pairs, activation tiles and column sums.
+//
 // Work split ("stream-K").  A unit is one quantization group of one block of 128 rows; the units of the layer,
 // ordered [block][group], are cut into one contiguous run per CTA.  A CTA whose run covers a whole block stores
 // its rows; where a block is shared, every contributor writes its fp32 partial sums to the workspace and counts
 // itself in; whoever arrives last adds the partial sums in the fixed order of the contributors (the result does
 // not depend on who was last) and stores the rows.  Nobody waits for another CTA.
 //
-// Roles of a CTA (15 warps):
-//   warps 0-3   epilogue: thread = row; tcgen05.ld of a finished slice, scale / zero-point, running sums, output;
-//   warps 4-11  expansion: thread = row; reads the row's packed codes of a 64-column step from the code ring,
-//               expands them to bf16 128 + c and stores eight 16-byte pieces into the step's K-major, 128-byte
-//               swizzled A tile (for the low-rank steps: copies the row's fp16 entries of A);
+// A CTA walks its run in stages of up to four 64-column steps (a wait on a shared-memory barrier costs a thread
+// about 125 cycles even when it is satisfied, so every role waits once per stage, not once per step).
+// Roles (16 warps):
+//   warps 0-3   epilogue: thread = row; per stage, the slices of the groups that end in it: tcgen05.ld,
+//               scale / zero-point, running sums; at the end of a block's piece the output or the partial sums;
+//   warps 4-11  expansion, two sets of four warps (one warp per 32-row quarter) taking turns by stage: thread = row;
+//               reads the row's packed codes from the code ring, expands, tcgen05.st (for the low-rank steps:
+//               the row's fp16 entries of A); the set's first warp also waits for the stage's activation tiles
+//               and for the accumulator slices the stage opens, so that the MMA thread has a single wait;
 //   warp 12     one thread streams packed codes and (scale, zero) pairs with bulk copies -- layer data, requested
 //               before griddepcontrol.wait, i.e. while the prologue of the same forward still runs;
 //   warp 13     one thread waits for the prologue and streams the activation tiles and column sums;
-//   warp 14     one thread issues tcgen05.mma (M 128, N = NP, K 16) and commits stages, tiles and slices back.
+//   warps 14-15 one thread each issues tcgen05.mma (M 128, N = NP, K 16; A from tensor memory, B from shared memory)
+//               and commits stages, tiles and slices back; the two take turns by stage.
 // Every mbarrier wait is bounded; a wait that runs out stores LOPRO_ERR_TIMEOUT in the workspace status word, the
 // CTA stops waiting, frees its tensor memory and returns (outputs then unspecified).
 #include "common.cuh"
@@ -34,25 +44,19 @@ namespace lopro {
 namespace {
 
 constexpr int kEpiWarps = 4;
-constexpr int kExpWarps = 8;  // two sets of four warps (one warp per 32-row quarter), alternating steps
-constexpr int kWarpW = kEpiWarps + kExpWarps, kWarpX = kWarpW + 1, kWarpMma = kWarpW + 2;
-constexpr int kThreads = (kWarpMma + 1) * 32;
-#ifndef RB_XSLOTS
-#define RB_XSLOTS 6
-#endif
-#ifndef RB_GSLOTS
-#define RB_GSLOTS 8
-#endif
-#ifndef RB_POLL_ALL
-#define RB_POLL_ALL 1
-#endif
-constexpr int kASlots = 4;             // ring of expanded A tiles
-constexpr int kATile = kRbRows * 128;  // 16 KB: 128 rows x 64 columns of bf16
-constexpr int kXSlots = RB_XSLOTS;     // ring of activation tiles
-constexpr int kGSlots = RB_GSLOTS;     // ring of group records: (scale, zero) pairs and column sums
-constexpr int kSlices = 8;             // accumulator slices in tensor memory
-constexpr int kMaxCSlots = 32;         // ring of packed-code steps (depth chosen at launch)
+constexpr int kExpWarps = 8;
+constexpr int kWarpW = kEpiWarps + kExpWarps, kWarpX = kWarpW + 1, kWarpMma = kWarpW + 2;  // two MMA warps
+constexpr int kThreads = (kWarpMma + 2) * 32;
+constexpr int kStageItems = 4;  // 64-column steps per stage
+constexpr int kAStages = 2;     // stages of expanded weights in tensor memory (128 columns each)
+constexpr int kXSlots = 4;      // ring of activation stages
+constexpr int kGSlots = 6;      // ring of group records: (scale, zero) pairs and column sums of the groups a stage ends
+constexpr int kGSlotBytes = 4096;
+constexpr int kSlices = 8;      // accumulator slices in tensor memory
+constexpr int kMaxCSlots = 16;  // ring of packed-code stages (depth chosen at launch)
 constexpr int kSmemLimit = 200 * 1024;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kSliceCol0 = kAStages * kStageItems * 32;  // tensor-memory column of slice 0
 
 struct RbParams {
     const uint32_t* codes;
@@ -68,28 +72,108 @@ struct RbParams {
     int64_t ldy;
     int out_f32;
     int m, T;                   // T: live tokens of this launch (<= NP)
-    int nsteps, ng, gsteps;     // 64-column steps of K, groups per row, steps per group
+    int nsteps, ng, gshift;     // 64-column steps of K, groups per row, log2(steps per group)
     int r_pad, lr_steps;
     int units;                  // blocks * ng
     int spg;                    // column-sum runs per group (1 unless g > 256)
     int c_slots;                // depth of the code ring
-    int g_slot_bytes;
-    int bits;
+    int two_issuers;            // the two MMA threads take turns by stage (no group spans two stages)
 };
 
 // Ring position: slot and the parity of its current use.
 struct Ring {
     int slot = 0;
     uint32_t phase = 0;
+    bool wrapped = false;
     int n;
     __device__ explicit Ring(int n_) : n(n_) {}
     __device__ void next() {
         if (++slot == n) {
             slot = 0;
             phase ^= 1u;
+            wrapped = true;
         }
     }
 };
+
+// One stage of a CTA's run: up to four consecutive 64-column steps of one block of rows -- either steps of the
+// quantized part or (first in a piece that starts its block) steps of the low-rank term.
+struct Stage {
+    int rb;          // block of rows
+    bool lr;         // low-rank steps (operands A and t) instead of quantized steps
+    int i0, ni;      // first step (of the block's K range, or of the padded rank) and number of steps
+    int first_mask, last_mask;  // bit i: step i0 + i is the first / the last of its group (lr: of the low-rank term)
+    int n_open, n_close;        // groups that begin / end in the stage (popcounts of the masks)
+    int close0;      // index of the first group that ends in the stage
+    bool piece_end;  // last stage of this CTA's piece of the block
+    bool piece_whole, piece_first;  // the piece covers the whole block / starts at the block's first unit
+};
+
+// Walks the stages of the run of units [u, u1) in the order every role of the CTA follows.
+struct Walker {
+    int u, u1, ng, gshift, lr_steps;
+    int rb = 0, gb = 0, ge = 0, n_lr = 0, total = 0, j = 0, q_first = 0, q_last = 0;
+    __device__ Walker(int u0_, int u1_, int ng_, int gshift_, int lr_steps_)
+        : u(u0_), u1(u1_), ng(ng_), gshift(gshift_), lr_steps(lr_steps_) {}
+    __device__ __noinline__ bool next(Stage& s) {
+        if (j == total) {  // next piece: the units of the run that lie in one block
+            u += ge - gb;
+            if (u >= u1) return false;
+            rb = u / ng;
+            gb = u - rb * ng;
+            ge = min(ng, gb + (u1 - u));
+            n_lr = gb == 0 ? (lr_steps + kStageItems - 1) / kStageItems : 0;
+            q_first = gb << gshift;
+            q_last = ge << gshift;
+            total = n_lr + (q_last - q_first + kStageItems - 1) / kStageItems;
+            j = 0;
+        }
+        s.rb = rb;
+        s.piece_first = gb == 0;
+        s.piece_whole = gb == 0 && ge == ng;
+        s.lr = j < n_lr;
+        if (s.lr) {
+            s.i0 = j * kStageItems;
+            s.ni = min(kStageItems, lr_steps - s.i0);
+            s.first_mask = j == 0 ? 1 : 0;
+            s.last_mask = j == n_lr - 1 ? 1 << (s.ni - 1) : 0;
+            s.close0 = 0;
+        } else {
+            s.i0 = q_first + (j - n_lr) * kStageItems;
+            s.ni = min(kStageItems, q_last - s.i0);
+            const int gmask = (1 << gshift) - 1, live = (1 << s.ni) - 1;
+            if (gshift == 0) {
+                s.first_mask = s.last_mask = live;
+            } else if (gshift == 1) {
+                s.first_mask = 0x5 & live;  // stages start on even steps
+                s.last_mask = 0xA & live;
+            } else {  // groups of four steps or more: at most one begins and one ends in a stage
+                s.first_mask = (s.i0 & gmask) == 0 ? 1 : 0;
+                s.last_mask = ((s.i0 + s.ni) & gmask) == 0 ? 1 << (s.ni - 1) : 0;
+            }
+            s.close0 = (s.i0 + gmask + 1) >> gshift;
+            s.close0 -= 1;
+        }
+        s.n_open = __popc(s.first_mask);
+        s.n_close = __popc(s.last_mask);
+        ++j;
+        s.piece_end = j == total;
+        return true;
+    }
+};
+
+// Out-of-line slow path of every wait of this file (one copy of the polling loop for all roles: the kernel is bound
+// by instruction fetch as soon as its hot loops outgrow the instruction caches).  Polls with a suspend-time hint, so a
+// waiting warp issues few instructions.  False if the limit ran out.
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
+    return false;
+}
+__device__ __noinline__ void report_timeout(int* status, int* flag) {
+    *flag = 1;
+    atomicExch(status, (int)LOPRO_ERR_TIMEOUT);
+}
 
 template <int NP>
 __device__ __forceinline__ void tmem_ld(uint32_t (&v)[NP], uint32_t taddr) {
@@ -114,33 +198,58 @@ __device__ __forceinline__ void tmem_ld(uint32_t (&v)[NP], uint32_t taddr) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 32 registers of one thread -> 32 consecutive columns of its lane of tensor memory
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+          "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+          "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem desc], 128 x N x 16, issued by one thread
+__device__ __forceinline__ void umma_f16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"r"(kEpiWarps * 32) : "memory"); }
 
 template <int BITS, int NP>
 __global__ void __launch_bounds__(kThreads, 1)
 rowblock_kernel(const RbParams p) {
     extern __shared__ unsigned char smem_raw[];
-    // full / empty per slot of the five rings
-    __shared__ __align__(8) uint64_t bars[2 * (kASlots + kXSlots + kGSlots + kSlices + kMaxCSlots)];
+    // full / empty per slot: A stages, activation stages, group records, slices, code stages
+    __shared__ __align__(8) uint64_t bars[2 * (kAStages + kXSlots + kGSlots + kSlices + kMaxCSlots)];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_timeout;
     __shared__ int s_last;
+    // what the MMA thread needs to know about the stage in A slot k, written by the expansion warps that fill it:
+    // x = first_mask | last_mask << 4 | steps << 8 | low-rank << 12 | end << 13 | MMAs of the last step << 16,
+    // y = activation slot, z = slices opened before the stage
+    __shared__ uint4 s_cmd[kAStages];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // operand tiles are 1024-byte aligned (swizzle atoms)
     unsigned char* base_ptr = smem_raw + (base - raw);
-    constexpr int kXTile = NP * 128;
+    constexpr int kXTile = NP * 128, kXStage = kStageItems * kXTile;
     constexpr int kStepBytes = kRbRows * 8 * BITS;  // packed codes of 128 rows x 64 columns
-    const uint32_t a_ring = base, x_ring = a_ring + kASlots * kATile, g_ring = x_ring + kXSlots * kXTile;
-    const uint32_t c_ring = g_ring + (uint32_t)(kGSlots * p.g_slot_bytes);
-    const unsigned char* g_ring_ptr = base_ptr + kASlots * kATile + kXSlots * kXTile;
-    const unsigned char* c_ring_ptr = g_ring_ptr + kGSlots * p.g_slot_bytes;
+    constexpr int kCStage = kStageItems * kStepBytes;
+    const uint32_t x_ring = base, g_ring = x_ring + kXSlots * kXStage, c_ring = g_ring + kGSlots * kGSlotBytes;
+    const unsigned char* g_ring_ptr = base_ptr + kXSlots * kXStage;
+    const unsigned char* c_ring_ptr = g_ring_ptr + kGSlots * kGSlotBytes;
 
     const uint32_t bar0 = smem_u32(bars);
     int bi = 0;
-    const uint32_t full_a = bar0 + 8u * bi; bi += kASlots;
-    const uint32_t empty_a = bar0 + 8u * bi; bi += kASlots;
+    const uint32_t full_a = bar0 + 8u * bi; bi += kAStages;
+    const uint32_t empty_a = bar0 + 8u * bi; bi += kAStages;
     const uint32_t full_x = bar0 + 8u * bi; bi += kXSlots;
     const uint32_t empty_x = bar0 + 8u * bi; bi += kXSlots;
     const uint32_t full_g = bar0 + 8u * bi; bi += kGSlots;
@@ -152,8 +261,8 @@ rowblock_kernel(const RbParams p) {
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
-        for (int s = 0; s < kASlots; ++s) {
-            mbar_init(full_a + 8u * s, 4);   // the four expansion warps of a step
+        for (int s = 0; s < kAStages; ++s) {
+            mbar_init(full_a + 8u * s, 4);   // the four expansion warps of the stage's set
             mbar_init(empty_a + 8u * s, 1);  // tcgen05.commit
         }
         for (int s = 0; s < kXSlots; ++s) {
@@ -175,7 +284,6 @@ rowblock_kernel(const RbParams p) {
         s_timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    constexpr uint32_t kTmemCols = kSlices * NP;  // 128 or 256: a power of two >= 32
     if (warp == kWarpMma) tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
     tc_fence_before();
     __syncthreads();
@@ -185,55 +293,39 @@ rowblock_kernel(const RbParams p) {
     // this CTA's run of units [u0, u1)
     const long long G = gridDim.x;
     const int u0 = (int)((long long)blockIdx.x * p.units / G), u1 = (int)(((long long)blockIdx.x + 1) * p.units / G);
+    Walker walk(u0, u1, p.ng, p.gshift, p.lr_steps);
+    Stage st;
 
-    auto time_out = [&]() {
-        s_timeout = 1;
-        atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
-    };
-    // bounded wait of one thread / of every lane of a warp (all lanes poll: they all read what the wait guards)
+    bool dead = false;  // a wait of this thread ran out: it stops waiting
     auto wait = [&](uint32_t bar, uint32_t parity) {
-        if (!*(volatile int*)&s_timeout && !mbar_wait(bar, parity)) time_out();
-    };
-    // wait of a whole warp: one lane polls, the warp follows (bar.warp.sync orders the other lanes' accesses after it)
-    auto slow_wait = [&](uint32_t bar, uint32_t parity) {
-        if (!*(volatile int*)&s_timeout && !mbar_wait_backoff(bar, parity)) time_out();
-    };
-    auto warp_wait = [&](uint32_t bar, uint32_t parity) {
-#if RB_POLL_ALL
-        slow_wait(bar, parity);
-#else
-        if (lane == 0) slow_wait(bar, parity);
-        __syncwarp();
-#endif
+        if (dead || mbar_try_wait(bar, parity)) return;
+        if (!wait_slow(bar, parity)) {
+            dead = true;
+            report_timeout(p.status, &s_timeout);
+        }
     };
 
     if (warp == kWarpW) {
         // ---------------- layer-data producer: packed codes and (scale, zero) pairs ----------------
         if (lane == 0) {
             Ring rc(p.c_slots), rg(kGSlots);
-            bool c_wrapped = false, g_wrapped = false;
-            for (int u = u0; u < u1;) {
-                const int rb = u / p.ng, gb = u - rb * p.ng, ge = min(p.ng, gb + (u1 - u));
-                const int R = rb_rows(p.m, rb);
-                const uint32_t step_bytes = (uint32_t)(R * 8 * BITS), sz_bytes = (uint32_t)(R * 4);
-                const uint32_t* cblock = p.codes + rb_step_word(BITS, p.nsteps, p.m, rb, 0);
-                const uint32_t* szblock = p.sz + (size_t)rb * kRbRows * p.ng;
-                for (int g = gb; g < ge; ++g) {
-                    if (g_wrapped) slow_wait(empty_g + 8u * rg.slot, rg.phase ^ 1u);
+            while (walk.next(st)) {
+                if (st.lr) continue;
+                const int R = rb_rows(p.m, st.rb);
+                const uint32_t bytes = (uint32_t)(st.ni * R * 8 * BITS);
+                if (rc.wrapped) wait(empty_c + 8u * rc.slot, rc.phase ^ 1u);
+                mbar_expect_tx(full_c + 8u * rc.slot, bytes);
+                bulk_g2s(c_ring + (uint32_t)(rc.slot * kCStage), p.codes + rb_step_word(BITS, p.nsteps, p.m, st.rb, st.i0), bytes,
+                         full_c + 8u * rc.slot);
+                rc.next();
+                if (st.n_close > 0) {
+                    const uint32_t sz_bytes = (uint32_t)(st.n_close * R * 4);
+                    if (rg.wrapped) wait(empty_g + 8u * rg.slot, rg.phase ^ 1u);
                     mbar_expect_tx(full_g + 8u * rg.slot, sz_bytes);
-                    bulk_g2s(g_ring + (uint32_t)(rg.slot * p.g_slot_bytes), szblock + (size_t)g * R, sz_bytes, full_g + 8u * rg.slot);
+                    bulk_g2s(g_ring + (uint32_t)(rg.slot * kGSlotBytes),
+                             p.sz + (size_t)st.rb * kRbRows * p.ng + (size_t)st.close0 * R, sz_bytes, full_g + 8u * rg.slot);
                     rg.next();
-                    if (rg.slot == 0) g_wrapped = true;
-                    for (int st = 0; st < p.gsteps; ++st) {
-                        if (c_wrapped) slow_wait(empty_c + 8u * rc.slot, rc.phase ^ 1u);
-                        mbar_expect_tx(full_c + 8u * rc.slot, step_bytes);
-                        bulk_g2s(c_ring + (uint32_t)(rc.slot * kStepBytes),
-                                 cblock + (size_t)(g * p.gsteps + st) * R * (2 * BITS), step_bytes, full_c + 8u * rc.slot);
-                        rc.next();
-                        if (rc.slot == 0) c_wrapped = true;
-                    }
                 }
-                u += ge - gb;
             }
         }
     } else if (warp == kWarpX) {
@@ -241,199 +333,216 @@ rowblock_kernel(const RbParams p) {
         if (lane == 0) {
             asm volatile("griddepcontrol.wait;" ::: "memory");  // the prologue's image is complete
             Ring rx(kXSlots), rg(kGSlots);
-            bool x_wrapped = false, g_wrapped = false;
-            const uint32_t sum_bytes = (uint32_t)(p.spg * NP * 4);
-            auto issue_x = [&](const unsigned char* src) {
-                if (x_wrapped) slow_wait(empty_x + 8u * rx.slot, rx.phase ^ 1u);
-                mbar_expect_tx(full_x + 8u * rx.slot, kXTile);
-                bulk_g2s(x_ring + (uint32_t)(rx.slot * kXTile), src, kXTile, full_x + 8u * rx.slot);
+            while (walk.next(st)) {
+                const uint32_t bytes = (uint32_t)(st.ni * kXTile);
+                if (rx.wrapped) wait(empty_x + 8u * rx.slot, rx.phase ^ 1u);
+                mbar_expect_tx(full_x + 8u * rx.slot, bytes);
+                bulk_g2s(x_ring + (uint32_t)(rx.slot * kXStage), (st.lr ? p.timg : p.ximg) + (size_t)st.i0 * kXTile, bytes,
+                         full_x + 8u * rx.slot);
                 rx.next();
-                if (rx.slot == 0) x_wrapped = true;
-            };
-            for (int u = u0; u < u1;) {
-                const int rb = u / p.ng, gb = u - rb * p.ng, ge = min(p.ng, gb + (u1 - u));
-                if (gb == 0)
-                    for (int j = 0; j < p.lr_steps; ++j) issue_x(p.timg + (size_t)j * kXTile);
-                for (int g = gb; g < ge; ++g) {
-                    if (g_wrapped) slow_wait(empty_g + 8u * rg.slot, rg.phase ^ 1u);
+                if (!st.lr && st.n_close > 0) {
+                    const uint32_t sum_bytes = (uint32_t)(st.n_close * p.spg * NP * 4);
+                    if (rg.wrapped) wait(empty_g + 8u * rg.slot, rg.phase ^ 1u);
                     mbar_expect_tx(full_g + 8u * rg.slot, sum_bytes);
-                    bulk_g2s(g_ring + (uint32_t)(rg.slot * p.g_slot_bytes) + 512u, p.sums + (size_t)g * p.spg * NP, sum_bytes,
+                    bulk_g2s(g_ring + (uint32_t)(rg.slot * kGSlotBytes) + 2048u, p.sums + (size_t)st.close0 * p.spg * NP, sum_bytes,
                              full_g + 8u * rg.slot);
                     rg.next();
-                    if (rg.slot == 0) g_wrapped = true;
-                    for (int st = 0; st < p.gsteps; ++st) issue_x(p.ximg + (size_t)(g * p.gsteps + st) * kXTile);
                 }
-                u += ge - gb;
             }
         }
-    } else if (warp == kWarpMma) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+    } else if (warp >= kWarpMma) {
+        // ---------------- MMA issuers: one wait per stage, everything else comes ready-made ----------------
+        // A single thread runs a few hundred cycles per stage on bookkeeping alone, about as long as the stage's MMAs
+        // take in the tensor pipe; two issuing threads on two schedulers taking turns by stage hide that.  (Only when no
+        // accumulator slice spans two stages -- otherwise the order of the MMAs into it would be open -- else the first
+        // thread issues every stage.)
+        const int k = warp - kWarpMma;
+        if (lane == 0 && (k == 0 || p.two_issuers)) {
             const uint32_t idesc_w = make_idesc(NP, 1u), idesc_lr = make_idesc(NP, 0u);
-            Ring ra(kASlots), rx(kXSlots), rs(kSlices);
-            bool s_wrapped = false;
-            // one 64-column step: up to four MMAs of K = 16 into slice `d`
-            auto step = [&](uint32_t d, uint32_t idesc, int ksub, bool first) {
-                wait(full_a + 8u * ra.slot, ra.phase);
-                wait(full_x + 8u * rx.slot, rx.phase);
+            const uint64_t desc_x0 = make_desc_sw128(x_ring);
+            int slot = k;
+            uint32_t phase = 0;
+            for (;;) {
+                wait(full_a + 8u * slot, phase);  // expanded weights in tensor memory, tiles and slices ready
                 tc_fence_after();
-                const uint64_t da = make_desc_sw128(a_ring + ra.slot * kATile), db = make_desc_sw128(x_ring + rx.slot * kXTile);
-                for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
-                    umma_f16(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (first && k == 0) ? 0u : 1u);
-                umma_commit(empty_a + 8u * ra.slot);  // the tiles may be refilled once these MMAs have read them
-                umma_commit(empty_x + 8u * rx.slot);
-                ra.next();
-                rx.next();
-            };
-            auto open_slice = [&]() {
-                if (s_wrapped) wait(empty_s + 8u * rs.slot, rs.phase ^ 1u);
-                tc_fence_after();
-                return tmem + (uint32_t)(rs.slot * NP);
-            };
-            auto close_slice = [&]() {
-                umma_commit(full_s + 8u * rs.slot);
-                rs.next();
-                if (rs.slot == 0) s_wrapped = true;
-            };
-            for (int u = u0; u < u1;) {
-                const int rb = u / p.ng, gb = u - rb * p.ng, ge = min(p.ng, gb + (u1 - u));
-                if (gb == 0 && p.lr_steps > 0) {
-                    const uint32_t d = open_slice();
-                    for (int j = 0; j < p.lr_steps; ++j) step(d, idesc_lr, min(4, (p.r_pad - j * 64) / 16), j == 0);
-                    close_slice();
+                const uint4 cmd = s_cmd[slot];
+                if (dead || ((cmd.x >> 13) & 1u)) break;
+                const uint32_t ni = (cmd.x >> 8) & 15u, lr = (cmd.x >> 12) & 1u, ksub_last = (cmd.x >> 16) & 7u;
+                uint32_t first_mask = cmd.x & 15u, last_mask = (cmd.x >> 4) & 15u, spos = cmd.z;
+                uint32_t a = tmem + (uint32_t)(slot * kStageItems * 32);
+                uint64_t db = desc_x0 + (uint64_t)(cmd.y * (uint32_t)(kXStage >> 4));
+                const uint32_t idesc = lr ? idesc_lr : idesc_w;
+#pragma unroll
+                for (int i = 0; i < kStageItems; ++i) {
+                    if (i < (int)ni) {
+                        const uint32_t first = first_mask & 1u;
+                        spos += first;
+                        const uint32_t sl = (spos - 1u) & (kSlices - 1);
+                        const uint32_t d = tmem + kSliceCol0 + sl * NP;
+                        if (i + 1 < (int)ni || ksub_last == 4u) {
+                            // a whole step: four MMAs of 16 columns (8 columns of tensor memory, 32 bytes of the B tile)
+                            umma_f16_ta(d, a, db, idesc, first ^ 1u);
+                            umma_f16_ta(d, a + 8u, db + 2u, idesc, 1u);
+                            umma_f16_ta(d, a + 16u, db + 4u, idesc, 1u);
+                            umma_f16_ta(d, a + 24u, db + 6u, idesc, 1u);
+                        } else {
+                            // the last step of a padded rank that is not a multiple of 64
+                            for (uint32_t kk = 0; kk < ksub_last; ++kk)
+                                umma_f16_ta(d, a + 8u * kk, db + (uint64_t)(2u * kk), idesc, (first && kk == 0) ? 0u : 1u);
+                        }
+                        if (last_mask & 1u) umma_commit(full_s + 8u * sl);  // the group's slice is complete
+                        first_mask >>= 1;
+                        last_mask >>= 1;
+                        a += 32u;
+                        db += (uint64_t)(kXTile >> 4);
+                    }
                 }
-                for (int g = gb; g < ge; ++g) {
-                    const uint32_t d = open_slice();
-                    for (int st = 0; st < p.gsteps; ++st) step(d, idesc_w, 4, st == 0);
-                    close_slice();
+                umma_commit(empty_a + 8u * slot);  // the stage may be refilled once these MMAs have read it
+                umma_commit(empty_x + 8u * cmd.y);
+                if (p.two_issuers) {
+                    phase ^= 1u;
+                } else {
+                    slot ^= 1;
+                    if (slot == 0) phase ^= 1u;
                 }
-                u += ge - gb;
             }
         }
     } else if (warp >= kEpiWarps) {
         // ---------------- expansion warps ----------------
         const int e = warp - kEpiWarps, quarter = e & 3, set = e >> 2;
         const int r = quarter * 32 + lane;
-        // byte offset of 16-byte piece 0 of row r in an A tile; piece c sits at (off ^ (c << 4))
-        const uint32_t row_off = (uint32_t)(r * 128 + ((r & 7) << 4));
-        Ring rc(p.c_slots);
-        int it = 0;  // steps seen so far by this CTA: set `it & 1` expands it into A slot `it & 3`
-        auto a_slot_ready = [&](int item) {
-            if (item >= kASlots) warp_wait(empty_a + 8u * (item & (kASlots - 1)), (uint32_t)((item / kASlots) - 1) & 1u);
-        };
-        auto publish = [&](int item) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full_a + 8u * (item & (kASlots - 1)));
-        };
-        for (int u = u0; u < u1;) {
-            const int rb = u / p.ng, gb = u - rb * p.ng, ge = min(p.ng, gb + (u1 - u));
-            const int R = rb_rows(p.m, rb);
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        Ring rc(p.c_slots), rx(kXSlots);
+        int sidx = 0;   // stages seen so far: set `sidx & 1` expands stage sidx into A stage `sidx & 1`
+        int spos = 0;   // slices opened so far
+        for (; walk.next(st); ++sidx) {
+            const bool mine = (sidx & 1) == set;
+            const int R = rb_rows(p.m, st.rb);
             const bool live = r < R;
-            if (gb == 0) {
-                // low-rank steps: the row's fp16 entries of A, 64 columns of the rank per step
-                const __half* arow = p.A + (size_t)(rb * kRbRows + r) * p.r_pad;
-                for (int j = 0; j < p.lr_steps; ++j, ++it) {
-                    if ((it & 1) != set) continue;
-                    a_slot_ready(it);
-                    unsigned char* tile = base_ptr + (it & (kASlots - 1)) * kATile;
-                    if (live) {
-                        const int pieces = min(8, (p.r_pad - j * 64) / 8);
-#pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            if (c < pieces)
-                                *reinterpret_cast<uint4*>(tile + (row_off ^ (uint32_t)(c << 4))) =
-                                    __ldg(reinterpret_cast<const uint4*>(arow + j * 64) + c);
-                    }
-                    publish(it);
-                }
-            }
-            const int n_q = (ge - gb) * p.gsteps;
-            for (int q = 0; q < n_q; ++q, ++it, rc.next()) {
-                if ((it & 1) != set) continue;
-                warp_wait(full_c + 8u * rc.slot, rc.phase);
-                uint32_t w[2 * BITS];
-                if (live) {
-                    const unsigned char* src = c_ring_ptr + rc.slot * kStepBytes;
-                    const uint4 v0 = *reinterpret_cast<const uint4*>(src + r * 16);
-                    w[0] = v0.x; w[1] = v0.y; w[2] = v0.z; w[3] = v0.w;
-                    if constexpr (BITS == 4) {
-                        const uint4 v1 = *reinterpret_cast<const uint4*>(src + R * 16 + r * 16);
-                        w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
-                    } else if constexpr (BITS == 3) {
-                        const uint2 v1 = *reinterpret_cast<const uint2*>(src + R * 16 + r * 8);
-                        w[4] = v1.x; w[5] = v1.y;
-                    }
-                }
+            const int opened = st.n_open;
+            if (mine) {
+                const uint32_t a0 = tmem + lane_addr + (uint32_t)(set * kStageItems * 32);
+                if (!st.lr) wait(full_c + 8u * rc.slot, rc.phase);
+                if (sidx >= kAStages) wait(empty_a + 8u * set, (uint32_t)((sidx >> 1) - 1) & 1u);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty_c + 8u * rc.slot);  // the words are in registers
-                a_slot_ready(it);
-                if (live) {
-                    unsigned char* tile = base_ptr + (it & (kASlots - 1)) * kATile;
+                tc_fence_after();
+                if (st.lr) {
+                    // low-rank steps: the row's fp16 entries of A, 64 columns of the rank per step
+                    const __half* arow = p.A + (size_t)(st.rb * kRbRows + r) * p.r_pad;
+#pragma unroll 1
+                    for (int i = 0; i < st.ni; ++i) {
+                        uint32_t a[32];
+                        const int pieces = min(8, (p.r_pad - (st.i0 + i) * 64) / 8);
 #pragma unroll
-                    for (int hs = 0; hs < 2; ++hs) {
-                        uint32_t wh[BITS], a[16];
+                        for (int c = 0; c < 8; ++c) {
+                            uint4 v = make_uint4(0, 0, 0, 0);
+                            if (live && c < pieces) v = __ldg(reinterpret_cast<const uint4*>(arow + (st.i0 + i) * 64) + c);
+                            a[4 * c] = v.x; a[4 * c + 1] = v.y; a[4 * c + 2] = v.z; a[4 * c + 3] = v.w;
+                        }
+                        tmem_st32(a0 + (uint32_t)(i * 32), a);
+                    }
+                } else {
+                    const unsigned char* src = c_ring_ptr + rc.slot * kCStage;
+#pragma unroll 1
+                    for (int i = 0; i < st.ni; ++i, src += R * 8 * BITS) {
+                        uint32_t w[2 * BITS];
 #pragma unroll
-                        for (int b = 0; b < BITS; ++b) wh[b] = w[hs * BITS + b];
-                        expand_codes<BITS>(a, wh);
+                        for (int b = 0; b < 2 * BITS; ++b) w[b] = 0;
+                        if (live) {
+                            const uint4 v0 = *reinterpret_cast<const uint4*>(src + r * 16);
+                            w[0] = v0.x; w[1] = v0.y; w[2] = v0.z; w[3] = v0.w;
+                            if constexpr (BITS == 4) {
+                                const uint4 v1 = *reinterpret_cast<const uint4*>(src + R * 16 + r * 16);
+                                w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
+                            } else if constexpr (BITS == 3) {
+                                const uint2 v1 = *reinterpret_cast<const uint2*>(src + R * 16 + r * 8);
+                                w[4] = v1.x; w[5] = v1.y;
+                            }
+                        }
+                        uint32_t a[32];
 #pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            *reinterpret_cast<uint4*>(tile + (row_off ^ (uint32_t)((hs * 4 + c) << 4))) =
-                                make_uint4(a[4 * c], a[4 * c + 1], a[4 * c + 2], a[4 * c + 3]);
+                        for (int hs = 0; hs < 2; ++hs) {
+                            uint32_t wh[BITS], ah[16];
+#pragma unroll
+                            for (int b = 0; b < BITS; ++b) wh[b] = w[hs * BITS + b];
+                            expand_codes<BITS>(ah, wh);
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) a[hs * 16 + q] = ah[q];
+                        }
+                        tmem_st32(a0 + (uint32_t)(i * 32), a);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_c + 8u * rc.slot);  // the words have been read
+                }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                if (quarter == 0) {
+                    // on behalf of the MMA thread: the stage's activation tiles have landed, and the slices the stage
+                    // opens have been drained (the slices are opened and drained in order: the last one decides)
+                    wait(full_x + 8u * rx.slot, rx.phase);
+                    if (opened > 0 && spos + opened > kSlices) {
+                        const int use = spos + opened - 1;  // running number of the last slice the stage opens
+                        wait(empty_s + 8u * (use & (kSlices - 1)), (uint32_t)((use / kSlices) - 1) & 1u);
+                    }
+                    if (lane == 0) {
+                        const int ksub_last = st.lr ? min(4, (p.r_pad - (st.i0 + st.ni - 1) * 64) / 16) : 4;
+                        s_cmd[set] =
+                            make_uint4((uint32_t)(st.first_mask | (st.last_mask << 4) | (st.ni << 8) | ((st.lr ? 1 : 0) << 12) |
+                                                  (ksub_last << 16)),
+                                       (uint32_t)rx.slot, (uint32_t)spos, 0u);
                     }
                 }
-                publish(it);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_a + 8u * set);  // (release: the command is visible to the MMA thread)
             }
-            u += ge - gb;
+            if (!st.lr) rc.next();
+            rx.next();
+            spos += opened;
+        }
+        // end of the run: one more (empty) stage per set tells its MMA thread to stop
+        {
+            const int send = sidx + (((sidx & 1) == set) ? 0 : 1);
+            if (send >= kAStages) wait(empty_a + 8u * set, (uint32_t)((send >> 1) - 1) & 1u);
+            if (quarter == 0 && lane == 0) s_cmd[set] = make_uint4(1u << 13, 0u, 0u, 0u);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full_a + 8u * set);
         }
     } else {
         // ---------------- epilogue warps: thread = row ----------------
         asm volatile("griddepcontrol.wait;" ::: "memory");  // y, the partial sums and the counters belong to this call only now
         const int r = warp * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-        Ring rs(kSlices), rg(kGSlots);
-        for (int u = u0; u < u1;) {
-            const int rb = u / p.ng, gb = u - rb * p.ng, ge = min(p.ng, gb + (u1 - u));
-            const int R = rb_rows(p.m, rb);
-            const bool live = r < R;
-            float yacc[NP];
+        Ring rg(kGSlots);
+        int spos = 0;  // slices closed so far
+        float yacc[NP];
 #pragma unroll
-            for (int i = 0; i < NP; ++i) yacc[i] = 0.0f;
-            uint32_t v[NP];
-            auto take_slice = [&]() {
-                warp_wait(full_s + 8u * rs.slot, rs.phase);
+        for (int i = 0; i < NP; ++i) yacc[i] = 0.0f;
+        while (walk.next(st)) {
+            const int R = rb_rows(p.m, st.rb);
+            const bool live = r < R;
+            if (st.n_close > 0) {
+                // the slices close in order: when the last one of the stage is complete, all are
+                const int last_use = spos + st.n_close - 1;
+                wait(full_s + 8u * (last_use & (kSlices - 1)), (uint32_t)(last_use / kSlices) & 1u);
+                if (!st.lr) wait(full_g + 8u * rg.slot, rg.phase);
                 __syncwarp();
                 tc_fence_after();
-                tmem_ld<NP>(v, tmem + lane_addr + (uint32_t)(rs.slot * NP));
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_s + 8u * rs.slot);
-                rs.next();
-            };
-            if (gb == 0 && p.lr_steps > 0) {
-                take_slice();
+                const unsigned char* rec = g_ring_ptr + rg.slot * kGSlotBytes;
+#pragma unroll 1
+                for (int c = 0; c < st.n_close; ++c, ++spos) {
+                    uint32_t v[NP];
+                    tmem_ld<NP>(v, tmem + lane_addr + kSliceCol0 + (uint32_t)((spos & (kSlices - 1)) * NP));
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_s + 8u * (spos & (kSlices - 1)));
+                    if (st.lr) {
 #pragma unroll
-                for (int i = 0; i < NP; ++i) yacc[i] += __uint_as_float(v[i]);
-            }
-            for (int g = gb; g < ge; ++g) {
-                take_slice();
-                warp_wait(full_g + 8u * rg.slot, rg.phase);
-                const unsigned char* rec = g_ring_ptr + rg.slot * p.g_slot_bytes;
-                if (live) {
-                    const uint32_t szw = *reinterpret_cast<const uint32_t*>(rec + r * 4);
-                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&szw));
-                    const float sc = f.x, nsz = -f.x * (128.0f + f.y);
-                    const float4* sp = reinterpret_cast<const float4*>(rec + 512);
-                    if (p.spg == 1) {
-#pragma unroll
-                        for (int i = 0; i < NP / 4; ++i) {
-                            const float4 sx = sp[i];
-                            yacc[4 * i + 0] = fmaf(sc, __uint_as_float(v[4 * i + 0]), fmaf(nsz, sx.x, yacc[4 * i + 0]));
-                            yacc[4 * i + 1] = fmaf(sc, __uint_as_float(v[4 * i + 1]), fmaf(nsz, sx.y, yacc[4 * i + 1]));
-                            yacc[4 * i + 2] = fmaf(sc, __uint_as_float(v[4 * i + 2]), fmaf(nsz, sx.z, yacc[4 * i + 2]));
-                            yacc[4 * i + 3] = fmaf(sc, __uint_as_float(v[4 * i + 3]), fmaf(nsz, sx.w, yacc[4 * i + 3]));
-                        }
-                    } else {
+                        for (int i = 0; i < NP; ++i) yacc[i] += __uint_as_float(v[i]);
+                    } else if (live) {
+                        const uint32_t szw = *reinterpret_cast<const uint32_t*>(rec + (c * R + r) * 4);
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&szw));
+                        const float sc = f.x, nsz = -f.x * (128.0f + f.y);
+                        const float4* sp = reinterpret_cast<const float4*>(rec + 2048 + c * p.spg * NP * 4);
 #pragma unroll
                         for (int i = 0; i < NP / 4; ++i) {
                             float4 sx = sp[i];
@@ -448,13 +557,16 @@ rowblock_kernel(const RbParams p) {
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_g + 8u * rg.slot);
-                rg.next();
+                if (!st.lr) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_g + 8u * rg.slot);
+                    rg.next();
+                }
             }
+            if (!st.piece_end) continue;
 
             // ---- the block's rows: stored directly, or handed over as partial sums ----
-            const int row = rb * kRbRows + r;
+            const int row = st.rb * kRbRows + r;
             auto store_rows = [&](const float (&acc)[NP]) {
                 if (!live) return;
 #pragma unroll
@@ -465,22 +577,22 @@ rowblock_kernel(const RbParams p) {
                         else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(acc[i]);
                     }
             };
-            if (gb == 0 && ge == p.ng) {
+            if (st.piece_whole) {
                 store_rows(yacc);
             } else {
                 // contributors of this block: the CTAs whose runs meet its units, in grid order
-                const long long ub = (long long)rb * p.ng, ue = ub + p.ng - 1;
+                const long long ub = (long long)st.rb * p.ng, ue = ub + p.ng - 1;
                 const int c_first = (int)(((ub + 1) * G - 1) / p.units), c_last = (int)(((ue + 1) * G - 1) / p.units);
-                float* mine = p.partial + (size_t)(2 * blockIdx.x + (gb > 0 ? 0 : 1)) * (NP * kRbRows);
+                float* mine = p.partial + (size_t)(2 * blockIdx.x + (st.piece_first ? 1 : 0)) * (NP * kRbRows);
 #pragma unroll
                 for (int i = 0; i < NP; ++i)
                     if (i < p.T) mine[i * kRbRows + r] = yacc[i];
                 __threadfence();
                 epi_sync();
                 if (tid == 0) {
-                    const int old = atomicAdd(p.counters + rb, 1);
+                    const int old = atomicAdd(p.counters + st.rb, 1);
                     const int last = old == c_last - c_first;
-                    if (last) atomicExch(p.counters + rb, 0);  // ready for the next forward
+                    if (last) atomicExch(p.counters + st.rb, 0);  // ready for the next forward
                     s_last = last;
                 }
                 epi_sync();
@@ -500,7 +612,8 @@ rowblock_kernel(const RbParams p) {
                 }
                 epi_sync();  // s_last is rewritten by the next shared block
             }
-            u += ge - gb;
+#pragma unroll
+            for (int i = 0; i < NP; ++i) yacc[i] = 0.0f;
         }
     }
 
@@ -543,18 +656,17 @@ image_convert_kernel(const __nv_bfloat16* __restrict__ xrot, int n, const float*
 }
 
 struct RbPlan {
-    int c_slots, g_slot_bytes, smem_bytes;
+    int c_slots, smem_bytes;
 };
 
 RbPlan plan_rowblock(const lopro_desc& d, int np) {
     RbPlan pl;
-    const int spg = d.group_size > 256 ? d.group_size / 256 : 1;
-    pl.g_slot_bytes = round_up_int(512 + spg * np * 4, 128);
-    const int fixed = 1024 + kASlots * kATile + kXSlots * np * 128 + kGSlots * pl.g_slot_bytes;
-    int slots = (kSmemLimit - fixed) / (kRbRows * 8 * d.bits);
+    const int fixed = 1024 + kXSlots * kStageItems * np * 128 + kGSlots * kGSlotBytes;
+    const int c_stage = kStageItems * kRbRows * 8 * d.bits;
+    int slots = (kSmemLimit - fixed) / c_stage;
     if (slots > kMaxCSlots) slots = kMaxCSlots;
     pl.c_slots = slots;
-    pl.smem_bytes = fixed + slots * kRbRows * 8 * d.bits;
+    pl.smem_bytes = fixed + slots * c_stage;
     return pl;
 }
 
@@ -622,13 +734,13 @@ cudaError_t launch_rowblock(const lopro_desc& d, const uint8_t* blob, const Blob
     p.m = d.d_out;
     p.T = t_live;
     p.ng = d.d_in / d.group_size;
-    p.gsteps = d.group_size / 64;
+    p.gshift = 0;
+    while ((64 << p.gshift) < d.group_size) ++p.gshift;
     const int blocks = (d.d_out + kRbRows - 1) / kRbRows;
     p.units = blocks * p.ng;
     p.spg = d.group_size > 256 ? d.group_size / 256 : 1;
     p.c_slots = pl.c_slots;
-    p.g_slot_bytes = pl.g_slot_bytes;
-    p.bits = d.bits;
+    p.two_issuers = (p.gshift <= 2 && p.lr_steps <= kStageItems) ? 1 : 0;
     int grid = sm_count();
     if (grid > kRbMaxGrid) grid = kRbMaxGrid;
     if (grid > p.units) grid = p.units;
