@@ -12,8 +12,8 @@
 //     in the K-major 128-byte-swizzled layout the MMA reads;
 //   * warp 16 (loader): one thread brings the stage's tile of rotated activations (B operand) with a
 //     tiled TMA copy, and for the low-rank stages the tiles of A (fp16) and t (fp16);
-//   * warp 17 (MMA): one thread issues four tcgen05.mma (K = 16 each) per stage into the TMEM
-//     accumulator and commits the stage back to the producers; the rank-r term A t runs as extra K
+//   * warps 17, 18 (MMA): one thread per accumulator issues four tcgen05.mma (K = 16 each) per stage into its
+//     TMEM accumulator and commits the stage back to the producers; the rank-r term A t runs as extra K
 //     stages with fp16 operands into the same accumulator, so the sum of Eq. 8 costs no extra pass;
 //   * warps 16-19 (epilogue): tcgen05.ld the accumulator, round once, store y[token][row].
 // All mbarrier waits are bounded; a wait that runs out sets LOPRO_ERR_TIMEOUT in the workspace status
@@ -108,13 +108,13 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     if (tid == 0) {
         for (int s = 0; s < kAStages; ++s) {
             mbar_init(full_a(s), (n_acc == 2 ? kDequantWarps : kDequantWarps / 2) + 1);  // the slot's dequant warps and the loader
-            mbar_init(empty_a(s), 1);
+            mbar_init(empty_a(s), n_acc);  // one commit per MMA-issuing thread
         }
         for (int s = 0; s < kBStages; ++s) {
             mbar_init(full_b(s), 1);
-            mbar_init(empty_b(s), 1);
+            mbar_init(empty_b(s), n_acc);
         }
-        mbar_init(acc_ready, 1);
+        mbar_init(acc_ready, n_acc);
         s_timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -232,31 +232,38 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                 }
             }
         }
-    } else if (warp == kDequantWarps + 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+    } else if (warp == kDequantWarps + 1 || warp == kDequantWarps + 2) {
+        // ---------------- MMA issuers ----------------
+        // One thread per accumulator: a thread spends several hundred cycles per stage on its two barrier waits,
+        // the descriptors and the commits, during which the tensor pipe would idle (an issued MMA occupies the
+        // thread until the pipe takes it); with two row blocks the second thread's MMAs fill those gaps.  Each
+        // accumulator receives its MMAs from one thread only, in program order, so results do not depend on timing.
+        const int acc = warp - (kDequantWarps + 1);
+        if (lane == 0 && acc < n_acc) {
             const uint32_t idesc_w = make_idesc(p.tile_n, 1u), idesc_lr = make_idesc(p.tile_n, 0u);
+            const uint32_t d = tmem + (uint32_t)(acc * 256);
+            int sa = 0, sb = 0;
+            uint32_t pa = 0, pb = 0;
             for (int s = 0; s < total; ++s) {
-                const int sa = s % kAStages, sb = s % kBStages;
-                if (!s_timeout && !(mbar_wait(full_a(sa), (uint32_t)(s / kAStages) & 1u, kPrefillSpin) &&
-                                    mbar_wait(full_b(sb), (uint32_t)(s / kBStages) & 1u, kPrefillSpin)))
-                    time_out();
+                if (!s_timeout && !(mbar_wait(full_a(sa), pa, kPrefillSpin) && mbar_wait(full_b(sb), pb, kPrefillSpin))) time_out();
                 tc_fence_after();
-                const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
-                const uint64_t db = make_desc_sw128(b_tile);
+                const uint64_t da = make_desc_sw128(base + sa * kABytes + acc * kABlock);
+                const uint64_t db = make_desc_sw128(b_ring + sb * kBBytes);
                 const bool lowrank = s >= p.nsteps;
                 const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
-                // the two accumulators alternate, so that consecutive MMAs never write the same accumulator
-                const uint64_t da0 = make_desc_sw128(a_tile), da1 = make_desc_sw128(a_tile + kABlock);
-                for (int k = 0; k < ksub; ++k) {  // 16 columns = 32 bytes = 2 descriptor address units
-                    const uint32_t accumulate = (s > 0 || k > 0) ? 1u : 0u;
-                    umma_f16(tmem, da0 + (uint64_t)(2 * k), db + (uint64_t)(2 * k), lowrank ? idesc_lr : idesc_w, accumulate);
-                    if (n_acc == 2)
-                        umma_f16(tmem + 256u, da1 + (uint64_t)(2 * k), db + (uint64_t)(2 * k), lowrank ? idesc_lr : idesc_w,
-                                 accumulate);
-                }
+                const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
+                for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
+                    umma_f16(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (s > 0 || k > 0) ? 1u : 0u);
                 umma_commit(empty_a(sa));  // the slots may be refilled once these MMAs have read them
                 umma_commit(empty_b(sb));
+                if (++sa == kAStages) {
+                    sa = 0;
+                    pa ^= 1u;
+                }
+                if (++sb == kBStages) {
+                    sb = 0;
+                    pb ^= 1u;
+                }
             }
             umma_commit(acc_ready);
         }
