@@ -305,14 +305,27 @@ def run_stack(args, T, rank, world, local, dev, dev16):
             i = li * len(STACK_LINEARS) + j
             codes = torch.roll(b["codes"], shifts=(i, 3 * i), dims=(0, 1)) if i else b["codes"]
             blob = lopro.pack(descs[(n, m)], codes, b["sc"], b["zr"], b["pm"], b["A"], b["B"])
-            linears.append((descs[(n, m)], blob, xs[n], ys[m][i % 2]))
+            y = torch.empty((T, m), dtype=torch.bfloat16, device=dev) if j in (1, 2, 5) else ys[m][i % 2]
+            linears.append((descs[(n, m)], blob, xs[n], y))
     del codes
     for b in base.values():
         del b["codes"]
+    # sibling linears of a layer read the same activations: (q, k, v) and (gate, up) go through the grouped call
+    groups = []
+    for li in range(STACK_LAYERS):
+        L7 = linears[li * 7:(li + 1) * 7]
+        for idx in ((0, 1, 2), (3,), (4, 5), (6,)) if not args.no_groups else ((0,), (1,), (2,), (3,), (4,), (5,), (6,)):
+            part = [L7[k] for k in idx]
+            groups.append(([g[0] for g in part], [g[1] for g in part], part[0][2], [g[3] for g in part]))
+    gws_bytes = max(lopro.group_workspace_bytes(g[0], T) for g in groups)
+    ws = torch.zeros(max(ws_bytes, gws_bytes), dtype=torch.uint8, device=dev)
 
     def one_step():
-        for d, blob, x, y in linears:
-            lopro.linear_fwd(d, blob, x, lopro.OUT_BF16, workspace=ws, y=y)
+        for ds, blobs_, x, ys_ in groups:
+            if len(ds) == 1:
+                lopro.linear_fwd(ds[0], blobs_[0], x, lopro.OUT_BF16, workspace=ws, y=ys_[0])
+            else:
+                lopro.linear_fwd_group(ds, blobs_, x, lopro.OUT_BF16, workspace=ws, ys=ys_)
 
     stream = torch.cuda.Stream(device=dev)
     graph = None
@@ -382,6 +395,8 @@ def run_stack(args, T, rank, world, local, dev, dev16):
     e2e_value = T * world / (e2e_ms / e2e_steps * 1e-3)
     paths = [lopro.linear_fwd_path(d, T) for d, _, _, _ in linears]
     names = sorted({lopro.PATH_NAMES.get(p, "?") for p, _ in paths})
+    n_launches = sum(lopro.linear_fwd_group_path(g[0], T)[1] if len(g[0]) > 1 else lopro.linear_fwd_path(g[0][0], T)[1]
+                     for g in groups)
     ach = stack_bytes(T) / (ms_per_step * 1e-3) / 1e9
     roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"], traffic=None,
                     peak_source=f"of {peaks['source']}", frac_of_nominal_8000=ach / 8000.0,
@@ -393,7 +408,7 @@ def run_stack(args, T, rank, world, local, dev, dev16):
                 data="synthetic", config=workload_config(args.workload), clocks=clocks,
                 e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=T * 4096 * 2, d2h_bytes_per_step=T * y_last.shape[1] * 2,
                          steps=e2e_steps),
-                gpu_launches=sum(n for _, n in paths) * args.steps, path="+".join(names), roofline=roofline,
+                gpu_launches=n_launches * args.steps, path="+".join(names), launches_per_step=n_launches, roofline=roofline,
                 step_ms_min=min(step_ms), step_ms_median=statistics.median(step_ms), cuda_graph=graph is not None)
     if not args.no_cpu_baseline and world == 1:
         r = time_oracle_stack(T, 12.0)
@@ -413,6 +428,7 @@ def main():
     ap.add_argument("--impl", default="lopro", choices=["lopro", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch through the stream instead of a CUDA graph")
+    ap.add_argument("--no-groups", action="store_true", help="stack workloads: every linear on its own (no grouped siblings)")
     ap.add_argument("--layout", default="fragment", choices=["fragment", "rowblock"], help="code layout of the packed layers")
     args = ap.parse_args()
     if args.impl == "reference":

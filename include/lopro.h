@@ -218,6 +218,25 @@ typedef enum {
 } lopro_path;
 LOPRO_API int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches);
 
+/* Forward of several SIBLING layers that read the same activations -- the q/k/v projections of an attention block,
+ * the gate/up projections of an MLP: y_i[t] = A_i (B_i x[t]) + W^_i (Q^T P_i^T x[t]), each layer with its own
+ * permutation (Eq. 5 depends on the layer's residual and Hessian), low-rank factors and codes.  The paper names the
+ * fusion of these steps as future work; its inference-latency table measures exactly this workload, layer by layer.
+ *   n_layers >= 1; descs[i], packed[i], y[i], ldy[i] per layer (host arrays of n_layers entries); all layers have
+ *   the same d_in; x, out_dtype, T as for lopro_linear_fwd; workspace of lopro_group_workspace_bytes(...) bytes,
+ *   256-byte aligned.  The status word of the group is the first word of the workspace.
+ * When the layers differ in nothing but d_out and their data, are in LOPRO_LAYOUT_FRAGMENT, n_layers <= 4, T <= 32 and
+ * each would run as prologue + streaming kernel, the group runs as TWO launches: one prologue that writes every
+ * layer's rotated activations and B_i x, and one product launch over the row tiles of all layers.  Otherwise the
+ * layers run one after the other (same results, one lopro_linear_fwd each).  lopro_linear_fwd_group_path returns 2
+ * in the first case, 1 in the second (0 on bad arguments) and the number of launches in *launches. */
+LOPRO_API size_t lopro_group_workspace_bytes(int32_t n_layers, const lopro_desc* const* descs, int32_t T);
+LOPRO_API int32_t lopro_linear_fwd_group_path(int32_t n_layers, const lopro_desc* const* descs, int32_t T, int32_t* launches);
+LOPRO_API lopro_status lopro_linear_fwd_group(int32_t n_layers, const lopro_desc* const* descs, const void* const* packed,
+                                              const uint16_t* x_bf16, int64_t ldx, void* const* y, const int64_t* ldy,
+                                              int32_t out_dtype, int32_t T, void* workspace, size_t workspace_bytes,
+                                              void* stream);
+
 /* The same forward for callers whose activations live in HOST memory (Eq. 8 end to end):
  * copies x_host [T][n] (dense, bf16; pinned memory makes the copy asynchronous) to the device,
  * runs lopro_linear_fwd and copies y [T][m] back to y_host.  `workspace` must hold

@@ -448,6 +448,127 @@ lopro_status lopro_configure(int32_t opt, int32_t value) {
     return LOPRO_OK;
 }
 
+// Sibling layers can share launches when they differ in nothing but their rows and data, the batch is small and
+// the per-layer path would be prologue + streaming kernel for each of them.
+static bool group_shares_launches(int32_t n, const lopro_desc* const* descs, int32_t T) {
+    if (n < 2 || n > kMaxSiblings || T < 1 || T > kDecodeMaxT) return false;
+    const lopro_desc& d0 = *descs[0];
+    if (d0.layout != LOPRO_LAYOUT_FRAGMENT) return false;
+    for (int i = 0; i < n; ++i) {
+        const lopro_desc& d = *descs[i];
+        if (d.d_in != d0.d_in || d.bits != d0.bits || d.group_size != d0.group_size || d.block_size != d0.block_size ||
+            d.identity_cols != d0.identity_cols || d.rank != d0.rank || d.layout != d0.layout)
+            return false;
+        if (!prologue_supported(d, T) || !stream_supported(d, T) || use_tall(d, T)) return false;
+    }
+    return true;
+}
+
+static size_t group_region_bytes(const lopro_desc& d, int32_t T) {
+    WorkspaceLayout W;
+    if (workspace_layout(d, T, &W) != LOPRO_OK) return 0;
+    return round_up_size(W.total, 1024);
+}
+
+size_t lopro_group_workspace_bytes(int32_t n_layers, const lopro_desc* const* descs, int32_t T) {
+    if (n_layers < 1 || !descs || T < 0) return 0;
+    size_t total = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        if (!descs[i]) return 0;
+        const size_t r = group_region_bytes(*descs[i], T);
+        if (r == 0) return 0;
+        total += r;
+    }
+    return total;
+}
+
+int32_t lopro_linear_fwd_group_path(int32_t n_layers, const lopro_desc* const* descs, int32_t T, int32_t* launches) {
+    if (n_layers < 1 || !descs || T < 1) return 0;
+    for (int i = 0; i < n_layers; ++i)
+        if (!descs[i] || check_desc(*descs[i]) != LOPRO_OK) return 0;
+    if (group_shares_launches(n_layers, descs, T)) {
+        if (launches) *launches = 2;
+        return 2;
+    }
+    int32_t total = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        int32_t one = 0;
+        if (lopro_linear_fwd_path(descs[i], T, &one) == 0) return 0;
+        total += one;
+    }
+    if (launches) *launches = total;
+    return 1;
+}
+
+lopro_status lopro_linear_fwd_group(int32_t n_layers, const lopro_desc* const* descs, const void* const* packed,
+                                    const uint16_t* x_bf16, int64_t ldx, void* const* y, const int64_t* ldy, int32_t out_dtype,
+                                    int32_t T, void* workspace, size_t workspace_bytes, void* stream) {
+    if (n_layers < 1 || !descs || !packed || !y || !ldy) return LOPRO_ERR_INVALID_ARG;
+    if (T < 0 || (out_dtype != LOPRO_OUT_BF16 && out_dtype != LOPRO_OUT_F32)) return LOPRO_ERR_INVALID_ARG;
+    for (int i = 0; i < n_layers; ++i) {
+        if (!descs[i]) return LOPRO_ERR_INVALID_ARG;
+        const lopro_status st = check_desc(*descs[i]);
+        if (st != LOPRO_OK) return st;
+        if (descs[i]->d_in != descs[0]->d_in) return LOPRO_ERR_INVALID_ARG;  // siblings read the same x
+    }
+    if (T == 0) return LOPRO_OK;
+    if (!workspace || !aligned(workspace, 256)) return LOPRO_ERR_INVALID_ARG;
+    if (workspace_bytes < lopro_group_workspace_bytes(n_layers, descs, T)) return LOPRO_ERR_BUFFER_TOO_SMALL;
+    uint8_t* ws = (uint8_t*)workspace;
+    if (!group_shares_launches(n_layers, descs, T)) {
+        // layer by layer, each in its own region of the workspace
+        for (int i = 0; i < n_layers; ++i) {
+            const size_t region = group_region_bytes(*descs[i], T);
+            const lopro_status st =
+                lopro_linear_fwd(descs[i], packed[i], x_bf16, ldx, y[i], ldy[i], out_dtype, T, ws, region, stream);
+            if (st != LOPRO_OK) return st;
+            ws += region;
+        }
+        return LOPRO_OK;
+    }
+    // one prologue for all siblings (one read of x per rotation CTA set, every layer its own permutation, Eq. 5),
+    // one product launch over the row tiles of all of them
+    const lopro_desc& d0 = *descs[0];
+    if (!x_bf16 || ldx < d0.d_in || (ldx % 8) || !aligned(x_bf16, 16)) return LOPRO_ERR_INVALID_ARG;
+    WorkspaceLayout W;
+    lopro_status st = workspace_layout(d0, T, &W);
+    if (st != LOPRO_OK) return st;
+    const size_t region = group_region_bytes(d0, T);
+    BlobLayout L[kMaxSiblings];
+    for (int i = 0; i < n_layers; ++i) {
+        if (!packed[i] || !y[i] || !aligned(packed[i], 256) || ldy[i] < descs[i]->d_out ||
+            !aligned(y[i], out_dtype == LOPRO_OUT_F32 ? 4 : 2))
+            return LOPRO_ERR_INVALID_ARG;
+        st = blob_layout(*descs[i], &L[i]);
+        if (st != LOPRO_OK) return st;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    PrologueSiblings ps = {};
+    StreamSiblingArgs ss = {};
+    ps.n = ss.n = n_layers - 1;
+    for (int i = 1; i < n_layers; ++i) {
+        const uint8_t* blob = (const uint8_t*)packed[i];
+        uint8_t* wsi = ws + (size_t)i * region;
+        ps.perm[i - 1] = (const int32_t*)(blob + L[i].off[LOPRO_SEC_PERM]);
+        ps.B[i - 1] = (const __half*)(blob + L[i].off[LOPRO_SEC_B]);
+        ps.act[i - 1] = wsi + W.off_xrot;
+        ps.t[i - 1] = (__half*)(wsi + W.off_t);
+        ss.blob[i - 1] = blob;
+        ss.L[i - 1] = L[i];
+        ss.ws[i - 1] = wsi;
+        ss.y[i - 1] = y[i];
+        ss.ldy[i - 1] = ldy[i];
+        ss.d_out[i - 1] = descs[i]->d_out;
+    }
+    const uint8_t* blob0 = (const uint8_t*)packed[0];
+    if (launch_prologue(d0, (const int32_t*)(blob0 + L[0].off[LOPRO_SEC_PERM]), (const __half*)(blob0 + L[0].off[LOPRO_SEC_B]),
+                        L[0].r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot, (__half*)(ws + W.off_t), W.t_pad,
+                        (int*)(ws + W.off_status), T, s, nullptr, &ps) != cudaSuccess)
+        return LOPRO_ERR_CUDA;
+    if (launch_stream(d0, blob0, L[0], ws, W, y[0], ldy[0], out_dtype, T, s, 0, &ss) != cudaSuccess) return LOPRO_ERR_CUDA;
+    return LOPRO_OK;
+}
+
 size_t lopro_host_staging_bytes(const lopro_desc* desc, int32_t T, int32_t out_dtype) {
     if (!desc || check_desc(*desc) != LOPRO_OK || T < 0) return 0;
     const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;

@@ -132,9 +132,19 @@ cudaError_t launch_rotate(const lopro_desc& d, const int32_t* perm, const __nv_b
                           __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s);
 // Small-batch prologue: rotation, 64-column sums and t = B x in one launch.
 bool prologue_supported(const lopro_desc& d, int T);
+// Sibling layers of a grouped forward: they read the same x and differ only in their rows (d_out) and data.
+constexpr int kMaxSiblings = 4;
+struct PrologueSiblings {  // siblings 1 .. n of a grouped prologue (sibling 0 travels in the ordinary arguments)
+    int n;
+    const int32_t* perm[kMaxSiblings - 1];
+    const __half* B[kMaxSiblings - 1];
+    unsigned char* act[kMaxSiblings - 1];
+    __half* t[kMaxSiblings - 1];
+};
 cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
                             const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, __half* t, int t_pad,
-                            int* status, int T, cudaStream_t s, const ImageOut* img = nullptr);
+                            int* status, int T, cudaStream_t s, const ImageOut* img = nullptr,
+                            const PrologueSiblings* siblings = nullptr);
 // Plain rotated activations, 64-column sums and t (the general path's outputs) -> operand image.
 cudaError_t launch_image_convert(const lopro_desc& d, const __nv_bfloat16* xrot, const float* s64, int s64_ld,
                                  const __half* t, int r_pad, const ImageOut& img, int T, cudaStream_t s);
@@ -152,8 +162,20 @@ cudaError_t launch_decode(const lopro_desc& d, const uint8_t* blob, const BlobLa
 // Small-batch forward (T <= 32) after launch_prologue: bulk-copy ring, one CTA per 32 output rows.
 bool stream_supported(const lopro_desc& d, int T);
 bool stream_uses_wide(const lopro_desc& d, int T);  // the 32-warp variant of the kernel will run
+// `more`: sibling layers of a grouped launch (same descriptor but for d_out; each with its own blob, workspace
+// region laid out like W, and output) whose row tiles are appended to the grid.
+struct StreamSiblingArgs {
+    int n;
+    const uint8_t* blob[kMaxSiblings - 1];
+    BlobLayout L[kMaxSiblings - 1];
+    const uint8_t* ws[kMaxSiblings - 1];
+    void* y[kMaxSiblings - 1];
+    int64_t ldy[kMaxSiblings - 1];
+    int d_out[kMaxSiblings - 1];
+};
 cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0 = 0);
+                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0 = 0,
+                          const StreamSiblingArgs* more = nullptr);
 
 // Small-batch forward for tall layers after launch_prologue: persistent CTAs, one ring across tile groups.
 bool tall_supported(const lopro_desc& d, int T);

@@ -254,10 +254,23 @@ constexpr int kPrologueMaxSmem = 200 * 1024;  // one row of x: d_in <= 102400
 // wait, everything is loaded after it.
 template <bool STAGED>
 __global__ void __launch_bounds__(256)
-prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
-                const __half* __restrict__ B, unsigned char* __restrict__ act_image, __half* __restrict__ t,
+prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm0,
+                const __half* __restrict__ B0, unsigned char* __restrict__ act_image0, __half* __restrict__ t0,
                 int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T,
-                int tpr, const ImageOut img) {
+                int tpr, const ImageOut img, const PrologueSiblings sibs) {
+    // sibling layers (grid z): the same x, each layer its own permutation, B and outputs
+    const int32_t* __restrict__ perm = perm0;
+    const __half* __restrict__ B = B0;
+    unsigned char* __restrict__ act_image = act_image0;
+    __half* __restrict__ t = t0;
+#pragma unroll
+    for (int i = 0; i < kMaxSiblings - 1; ++i)
+        if ((int)blockIdx.z == i + 1) {
+            perm = sibs.perm[i];
+            B = sibs.B[i];
+            act_image = sibs.act[i];
+            t = sibs.t[i];
+        }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nchunks = (n + 255) >> 8;
     const int tok0 = blockIdx.y * 8;
@@ -289,7 +302,7 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
             pidx[0] = p0.x; pidx[1] = p0.y; pidx[2] = p0.z; pidx[3] = p0.w;
             pidx[4] = p1.x; pidx[5] = p1.y; pidx[6] = p1.z; pidx[7] = p1.w;
         }
-        if (c == 0 && tok0 == 0) {
+        if (c == 0 && tok0 == 0 && blockIdx.z == 0) {
             if (status != nullptr && tid == 0) *status = LOPRO_OK;
             if (img.ximg != nullptr)
                 for (int i = tid; i < img.n_counters; i += 256) img.counters[i] = 0;
@@ -334,7 +347,7 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
             }
         }
         __syncthreads();
-        if (c == 0 && tok0 == 0) {  // (token 0 exists: T >= 1)
+        if (c == 0 && tok0 == 0 && blockIdx.z == 0) {  // (token 0 exists: T >= 1)
             if (status != nullptr && tid == 0) *status = LOPRO_OK;
             if (img.ximg != nullptr)
                 for (int i = tid; i < img.n_counters; i += 256) img.counters[i] = 0;
@@ -390,10 +403,12 @@ bool prologue_supported(const lopro_desc& d, int T) {
 
 cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
                             const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, __half* t, int t_pad,
-                            int* status, int T, cudaStream_t s, const ImageOut* img_out) {
+                            int* status, int T, cudaStream_t s, const ImageOut* img_out, const PrologueSiblings* siblings) {
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
     ImageOut img = {};
     if (img_out != nullptr) img = *img_out;
+    PrologueSiblings sibs = {};
+    if (siblings != nullptr) sibs = *siblings;
     cudaLaunchConfig_t cfg = {};
     // tokens per row CTA: as few as it takes to fill the SMs
     const int live = T < 8 ? T : 8;
@@ -414,7 +429,7 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
         cudaError_t e = ensure_dynamic_smem(prologue_kernel<true>, kPrologueMaxSmem, &attr_done);
         if (e != cudaSuccess) return e;
     }
-    cfg.gridDim = dim3(row_ctas + rot_ctas, (T + 7) / 8);
+    cfg.gridDim = dim3(row_ctas + rot_ctas, (T + 7) / 8, 1 + sibs.n);
     cfg.blockDim = dim3(256);
     cfg.dynamicSmemBytes = staged ? (size_t)d.d_in * 2 : 0;
     cfg.stream = s;
@@ -425,9 +440,9 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
     cfg.numAttrs = 1;
     const int rp = d.rank > 0 ? r_pad : 0;
     return staged ? cudaLaunchKernelEx(&cfg, prologue_kernel<true>, x, ldx, perm, B, act_image, t, status, d.d_in,
-                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img)
+                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, sibs)
                   : cudaLaunchKernelEx(&cfg, prologue_kernel<false>, x, ldx, perm, B, act_image, t, status, d.d_in,
-                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img);
+                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, sibs);
 }
 
 cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,

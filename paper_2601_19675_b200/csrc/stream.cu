@@ -51,9 +51,45 @@ struct StreamParams {
     int off_sz, off_a, off_t, off_ring, stage_bytes, off_stage_x;
 };
 
+// Sibling layers 1 .. n of a grouped launch (sibling 0 travels in StreamParams): same shape of K, quantization and
+// rank, each its own rows and data; CTAs [cta0[i], cta0[i + 1]) of the grid belong to sibling i + 1.
+struct StreamSiblings {
+    int n;
+    int cta0[kMaxSiblings - 1];
+    const uint32_t* codes[kMaxSiblings - 1];
+    const uint32_t* sz[kMaxSiblings - 1];
+    const __half* A[kMaxSiblings - 1];
+    const unsigned char* act[kMaxSiblings - 1];
+    const __half* t[kMaxSiblings - 1];
+    void* y[kMaxSiblings - 1];
+    int64_t ldy[kMaxSiblings - 1];
+    int m[kMaxSiblings - 1];
+};
+
+// The layer a CTA works on: patches the per-layer fields of the parameters, returns the CTA's index within the layer.
+__device__ __forceinline__ int select_sibling(StreamParams& p, const StreamSiblings& sibs) {
+    int bx = (int)blockIdx.x;
+#pragma unroll
+    for (int i = kMaxSiblings - 2; i >= 0; --i)
+        if (i < sibs.n && (int)blockIdx.x >= sibs.cta0[i] && bx == (int)blockIdx.x) {
+            bx = (int)blockIdx.x - sibs.cta0[i];
+            p.codes = sibs.codes[i];
+            p.sz = sibs.sz[i];
+            p.A = sibs.A[i];
+            p.act = sibs.act[i];
+            p.t = sibs.t[i];
+            p.y = sibs.y[i];
+            p.ldy = sibs.ldy[i];
+            p.m = sibs.m[i];
+        }
+    return bx;
+}
+
 template <int BITS, int NT, int RT>
 __global__ void __launch_bounds__(kThreads, 1)
-stream_kernel(const StreamParams p) {
+stream_kernel(const StreamParams p_in, const StreamSiblings sibs) {
+    StreamParams p = p_in;
+    const int bx = select_sibling(p, sibs);
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t bars[3 * kMaxStages + 2];  // wfull, xfull, empty per stage; sz + A; t
     __shared__ int s_timeout;
@@ -62,7 +98,7 @@ stream_kernel(const StreamParams p) {
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tg = lane & 3;
-    const int rt0 = blockIdx.x * RT;                     // first 16-row tile of this CTA
+    const int rt0 = bx * RT;                             // first 16-row tile of this CTA
     const int n_rt = min(RT, (p.m >> 4) - rt0);          // live row tiles
     const int tc = min(kTok, p.T);                                  // live tokens
     const uint32_t bar0 = smem_u32(bars);
@@ -317,7 +353,9 @@ constexpr int kRedStep = 8 * kRedTok + 8;   // floats between steps
 
 template <int BITS>
 __global__ void __launch_bounds__(kWideThreads, 1)
-stream_wide_kernel(const StreamParams p) {
+stream_wide_kernel(const StreamParams p_in, const StreamSiblings sibs) {
+    StreamParams p = p_in;
+    const int bx = select_sibling(p, sibs);
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t bars[kMaxStages + 2];  // full per stage (codes and activations); sz + A; t
     constexpr int kTok = 8;
@@ -330,7 +368,7 @@ stream_wide_kernel(const StreamParams p) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = lane >> 2, tg = lane & 3;
     const int step = warp & 15, r = warp >> 4;
-    const int rt0 = blockIdx.x * 2;
+    const int rt0 = bx * 2;
     const int n_rt = min(2, (p.m >> 4) - rt0);
     const int tc = min(kTok, p.T);
     const uint32_t bar0 = smem_u32(bars);
@@ -480,12 +518,12 @@ stream_wide_kernel(const StreamParams p) {
 }
 
 template <int BITS>
-cudaError_t launch_stream_wide(const StreamParams& p, int smem_bytes, cudaStream_t s) {
+cudaError_t launch_stream_wide(const StreamParams& p, const StreamSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
     static unsigned long long attr_done = 0;
     cudaError_t e = ensure_dynamic_smem(stream_wide_kernel<BITS>, kStreamMaxSmem, &attr_done);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.m / 16 + 1) / 2);
+    cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kWideThreads);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = s;
@@ -494,16 +532,16 @@ cudaError_t launch_stream_wide(const StreamParams& p, int smem_bytes, cudaStream
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, stream_wide_kernel<BITS>, p);
+    return cudaLaunchKernelEx(&cfg, stream_wide_kernel<BITS>, p, sibs);
 }
 
 template <int BITS, int NT, int RT>
-cudaError_t launch_stream_k(const StreamParams& p, int smem_bytes, cudaStream_t s) {
+cudaError_t launch_stream_k(const StreamParams& p, const StreamSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
     static unsigned long long attr_done = 0;
     cudaError_t e = ensure_dynamic_smem(stream_kernel<BITS, NT, RT>, kStreamMaxSmem, &attr_done);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.m / 16 + RT - 1) / RT);
+    cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = s;
@@ -512,14 +550,17 @@ cudaError_t launch_stream_k(const StreamParams& p, int smem_bytes, cudaStream_t 
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, stream_kernel<BITS, NT, RT>, p);
+    return cudaLaunchKernelEx(&cfg, stream_kernel<BITS, NT, RT>, p, sibs);
 }
 
 template <int BITS>
-cudaError_t launch_stream_bits(const StreamParams& p, int nt, int rt, int smem_bytes, cudaStream_t s) {
-    if (nt == 1) return rt == 4 ? launch_stream_k<BITS, 1, 4>(p, smem_bytes, s) : launch_stream_k<BITS, 1, 2>(p, smem_bytes, s);
-    if (nt == 2) return rt == 4 ? launch_stream_k<BITS, 2, 4>(p, smem_bytes, s) : launch_stream_k<BITS, 2, 2>(p, smem_bytes, s);
-    return launch_stream_k<BITS, 4, 2>(p, smem_bytes, s);
+cudaError_t launch_stream_bits(const StreamParams& p, const StreamSiblings& sibs, int grid, int nt, int rt, int smem_bytes,
+                               cudaStream_t s) {
+    if (nt == 1)
+        return rt == 4 ? launch_stream_k<BITS, 1, 4>(p, sibs, grid, smem_bytes, s) : launch_stream_k<BITS, 1, 2>(p, sibs, grid, smem_bytes, s);
+    if (nt == 2)
+        return rt == 4 ? launch_stream_k<BITS, 2, 4>(p, sibs, grid, smem_bytes, s) : launch_stream_k<BITS, 2, 2>(p, sibs, grid, smem_bytes, s);
+    return launch_stream_k<BITS, 4, 2>(p, sibs, grid, smem_bytes, s);
 }
 
 struct StreamPlan {
@@ -592,7 +633,8 @@ bool stream_supported(const lopro_desc& d, int T) {
 }
 
 cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0) {
+                          const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0,
+                          const StreamSiblingArgs* more) {
     StreamPlan pl;
     if (!plan_stream(d, T, &pl)) return cudaErrorInvalidValue;
     StreamParams p;
@@ -624,17 +666,40 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
     p.off_ring = pl.off_ring;
     p.stage_bytes = pl.stage_bytes;
     p.off_stage_x = pl.off_stage_x;
-    if (wide_variant(d, pl)) {
+    const bool wide = wide_variant(d, pl);
+    const int rows_per_cta = wide ? 32 : pl.rt * 16;
+    int grid = (d.d_out + rows_per_cta - 1) / rows_per_cta;
+    // sibling layers: the CTAs of each follow those of the one before
+    StreamSiblings sibs = {};
+    if (more != nullptr) {
+        sibs.n = more->n;
+        for (int i = 0; i < more->n; ++i) {
+            const uint8_t* b = more->blob[i];
+            const BlobLayout& Li = more->L[i];
+            const uint8_t* wsi = more->ws[i];
+            sibs.cta0[i] = grid;
+            sibs.codes[i] = reinterpret_cast<const uint32_t*>(b + Li.off[LOPRO_SEC_CODES]);
+            sibs.sz[i] = reinterpret_cast<const uint32_t*>(b + Li.off[LOPRO_SEC_SCALEZERO]);
+            sibs.A[i] = reinterpret_cast<const __half*>(b + Li.off[LOPRO_SEC_A]);
+            sibs.act[i] = wsi + W.off_xrot + (size_t)t0 * kActRecord;
+            sibs.t[i] = reinterpret_cast<const __half*>(wsi + W.off_t) + (size_t)t0 * (d.rank > 0 ? L.r_pad : 0);
+            sibs.y[i] = more->y[i];
+            sibs.ldy[i] = more->ldy[i];
+            sibs.m[i] = more->d_out[i];
+            grid += (more->d_out[i] + rows_per_cta - 1) / rows_per_cta;
+        }
+    }
+    if (wide) {
         switch (d.bits) {
-            case 2: return launch_stream_wide<2>(p, pl.smem_bytes, s);
-            case 3: return launch_stream_wide<3>(p, pl.smem_bytes, s);
-            default: return launch_stream_wide<4>(p, pl.smem_bytes, s);
+            case 2: return launch_stream_wide<2>(p, sibs, grid, pl.smem_bytes, s);
+            case 3: return launch_stream_wide<3>(p, sibs, grid, pl.smem_bytes, s);
+            default: return launch_stream_wide<4>(p, sibs, grid, pl.smem_bytes, s);
         }
     }
     switch (d.bits) {
-        case 2: return launch_stream_bits<2>(p, pl.nt, pl.rt, pl.smem_bytes, s);
-        case 3: return launch_stream_bits<3>(p, pl.nt, pl.rt, pl.smem_bytes, s);
-        default: return launch_stream_bits<4>(p, pl.nt, pl.rt, pl.smem_bytes, s);
+        case 2: return launch_stream_bits<2>(p, sibs, grid, pl.nt, pl.rt, pl.smem_bytes, s);
+        case 3: return launch_stream_bits<3>(p, sibs, grid, pl.nt, pl.rt, pl.smem_bytes, s);
+        default: return launch_stream_bits<4>(p, sibs, grid, pl.nt, pl.rt, pl.smem_bytes, s);
     }
 }
 

@@ -24,7 +24,8 @@ SEC_HEADER, SEC_CODES, SEC_SCALEZERO, SEC_PERM, SEC_A, SEC_B = range(6)
 SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packed_bytes", "lopro_packed_section",
            "lopro_workspace_bytes", "lopro_pack", "lopro_unpack", "lopro_rotate", "lopro_linear_fwd",
            "lopro_linear_fwd_path", "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc",
-           "lopro_configure", "lopro_selftest_wait"]
+           "lopro_configure", "lopro_selftest_wait", "lopro_group_workspace_bytes", "lopro_linear_fwd_group_path",
+           "lopro_linear_fwd_group"]
 
 
 class Desc(ctypes.Structure):
@@ -82,6 +83,14 @@ def lib():
         L.lopro_linear_fwd_host.argtypes = [dp, vp, vp, vp, i32, i32, vp, sz, vp]
         L.lopro_linear_fwd_noalloc.restype = ctypes.c_int
         L.lopro_linear_fwd_noalloc.argtypes = [dp, vp, vp, i64, vp, i64, i32, i32, vp]
+        dpp = ctypes.POINTER(ctypes.POINTER(Desc))
+        L.lopro_group_workspace_bytes.restype = sz
+        L.lopro_group_workspace_bytes.argtypes = [i32, dpp, i32]
+        L.lopro_linear_fwd_group_path.restype = i32
+        L.lopro_linear_fwd_group_path.argtypes = [i32, dpp, i32, ctypes.POINTER(i32)]
+        L.lopro_linear_fwd_group.restype = ctypes.c_int
+        L.lopro_linear_fwd_group.argtypes = [i32, dpp, ctypes.POINTER(vp), vp, i64, ctypes.POINTER(vp), ctypes.POINTER(i64), i32,
+                                             i32, vp, sz, vp]
         L.lopro_configure.restype = ctypes.c_int
         L.lopro_configure.argtypes = [i32, i32]
         L.lopro_selftest_wait.restype = ctypes.c_int
@@ -269,6 +278,43 @@ def linear_fwd_host(desc, packed, x_host, y_host, workspace, out_dtype=OUT_BF16)
                                      _ptr(workspace), workspace.numel(), _stream())
     _check(st, "lopro_linear_fwd_host")
     return y_host
+
+
+def _desc_array(descs):
+    arr = (ctypes.POINTER(Desc) * len(descs))()
+    for i, d in enumerate(descs):
+        arr[i] = ctypes.pointer(d)
+    return arr
+
+
+def group_workspace_bytes(descs, T):
+    return int(lib().lopro_group_workspace_bytes(len(descs), _desc_array(descs), int(T)))
+
+
+def linear_fwd_group_path(descs, T):
+    """(2, launches) when the sibling layers share their two launches, (1, launches) when they run one by one."""
+    n = ctypes.c_int32(0)
+    path = int(lib().lopro_linear_fwd_group_path(len(descs), _desc_array(descs), int(T), ctypes.byref(n)))
+    return path, int(n.value)
+
+
+def linear_fwd_group(descs, packed, x, out_dtype=OUT_BF16, workspace=None, ys=None):
+    """lopro_linear_fwd_group: sibling layers on the same x bf16 [T][n] -> list of y_i [T][m_i]."""
+    assert x.is_cuda and x.dim() == 2 and x.element_size() == 2 and x.stride(1) == 1
+    T, k = x.shape[0], len(descs)
+    if workspace is None:
+        workspace = torch.empty(max(group_workspace_bytes(descs, T), 256), dtype=torch.uint8, device=x.device)
+    if ys is None:
+        ys = [torch.empty((T, d.d_out), dtype=torch.float32 if out_dtype == OUT_F32 else torch.bfloat16, device=x.device)
+              for d in descs]
+    ldx = x.stride(0) if T > 1 else max(x.stride(0), descs[0].d_in)
+    blobs = (ctypes.c_void_p * k)(*[b.data_ptr() for b in packed])
+    outs = (ctypes.c_void_p * k)(*[y.data_ptr() for y in ys])
+    ldys = (ctypes.c_int64 * k)(*[(y.stride(0) if T > 1 else max(y.stride(0), d.d_out)) for y, d in zip(ys, descs)])
+    st = lib().lopro_linear_fwd_group(k, _desc_array(descs), blobs, _ptr(x), ldx, outs, ldys, int(out_dtype), T, _ptr(workspace),
+                                      workspace.numel(), _stream())
+    _check(st, "lopro_linear_fwd_group")
+    return ys
 
 
 NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
