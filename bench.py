@@ -4,7 +4,9 @@
 Default workload: the decode configuration (4096 x 4096, 4-bit g128, block 128, rank 32, 8 tokens).
 One step = one forward of the token batch through every layer of a ring of distinct synthetic
 layers; the ring is larger than the L2 cache, so every layer's packed weights come from HBM.
-Prints ONE JSON line (see README / DESIGN for the keys).
+A step repeats that pass until it lasts --step-ms (50 ms), so that a run of 20 steps loads the GPU for a second.
+Prints ONE JSON line: the contract's keys for the named workload, `roofline`, `cpu_baseline`, `e2e`, and under
+`workloads` one record per other regime (decode at other batch sizes, the large layer, the decoder stack, prefill).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
@@ -274,70 +276,214 @@ def workload_config(name):
                    % (ring, ring_bytes / 1e6))
 
 
-def run_stack(args, T, rank, world, local, dev, dev16):
-    """The 224 linears of the 32-layer stack, one forward each per step, every linear with its own packed layer.
-    Linears with 4096 inputs read one fixed activation tensor, the `down` projections another (the glue between
-    them is not part of the method and is not run; the kernels' work does not depend on the values)."""
-    import torch
-    from paper_2601_19675_b200 import lopro, synth
-    if world > 1:
-        import torch.distributed as dist
-    q = STACK_QUANT
-    shapes = sorted({(n, m) for _, n, m in STACK_LINEARS})
-    base, descs = {}, {}
-    for n, m in shapes:
-        layer = synth.random_layer(n, m, q["bits"], q["group_size"], q["rank"], seed=rank + n // 64)
-        base[(n, m)] = dict(codes=torch.from_numpy(layer["codes"]).to(dev), sc=dev16(layer["scales"]), zr=dev16(layer["zeros"]),
-                            pm=torch.from_numpy(layer["perm"]).to(dev), A=dev16(layer["A"]), B=dev16(layer["B"]))
-        descs[(n, m)] = lopro.make_desc(n, m, q["bits"], q["group_size"], q["block_size"], q["identity_cols"], q["rank"],
-                                        layout=lopro.LAYOUT_ROWBLOCK if args.layout == "rowblock" else lopro.LAYOUT_FRAGMENT)
-    xs, x_bits = {}, {}
-    for n in sorted({n for n, _ in shapes}):
-        x_bits[n] = synth.activations(T, n, seed=rank + n)
-        xs[n] = dev16(x_bits[n]).view(torch.bfloat16)
-    ys = {m: [torch.empty((T, m), dtype=torch.bfloat16, device=dev) for _ in range(2)] for m in sorted({m for _, m in shapes})}
-    ws_bytes = max(lopro.workspace_bytes(descs[k], T) for k in shapes)
-    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
-    linears = []  # (desc, blob, x, y)
-    for li in range(STACK_LAYERS):
-        for j, (_, n, m) in enumerate(STACK_LINEARS):
-            b = base[(n, m)]
-            i = li * len(STACK_LINEARS) + j
-            codes = torch.roll(b["codes"], shifts=(i, 3 * i), dims=(0, 1)) if i else b["codes"]
-            blob = lopro.pack(descs[(n, m)], codes, b["sc"], b["zr"], b["pm"], b["A"], b["B"])
-            y = torch.empty((T, m), dtype=torch.bfloat16, device=dev) if j in (1, 2, 5) else ys[m][i % 2]
-            linears.append((descs[(n, m)], blob, xs[n], y))
-    del codes
-    for b in base.values():
-        del b["codes"]
-    # sibling linears of a layer read the same activations: (q, k, v) and (gate, up) go through the grouped call
-    groups = []
-    for li in range(STACK_LAYERS):
-        L7 = linears[li * 7:(li + 1) * 7]
-        for idx in ((0, 1, 2), (3,), (4, 5), (6,)) if not args.no_groups else ((0,), (1,), (2,), (3,), (4,), (5,), (6,)):
-            part = [L7[k] for k in idx]
-            groups.append(([g[0] for g in part], [g[1] for g in part], part[0][2], [g[3] for g in part]))
-    gws_bytes = max(lopro.group_workspace_bytes(g[0], T) for g in groups)
-    ws = torch.zeros(max(ws_bytes, gws_bytes), dtype=torch.uint8, device=dev)
+def cpu_model():
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
 
-    def one_step():
-        for ds, blobs_, x, ys_ in groups:
+
+def cpu_baseline_record(c_or_stack, T, budget_s, stack=False):
+    """The oracle as it stands on the host cores: all BLAS threads, and capped to one thread."""
+    def run(budget):
+        if stack:
+            return time_oracle_stack(T, budget)
+        max_rows = 1024 if c_or_stack["d_out"] * c_or_stack["d_in"] > (1 << 24) or T > 64 else None
+        max_tokens = 16 if T > 64 else None
+        return time_oracle(c_or_stack, T, budget, max_rows, max_tokens)
+    r = run(budget_s)
+    if stack:
+        sample = r["sample"]
+    else:
+        sample = (f"oracle.forward_exact (fp64 numpy) on {r['rows']} of {c_or_stack['d_out']} output rows, {r['tokens']} of {T} "
+                  f"tokens of one layer, {r['reps']} repetitions, scaled linearly to a full layer forward")
+    rec = dict(value=r["value"], unit=UNIT, cores=r["cores"], kind="oracle", sample=sample, cpu_model=cpu_model(),
+               host_cores=os.cpu_count())
+    try:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            r1 = run(max(2.0, budget_s / 3))
+        rec["single_thread"] = dict(value=r1["value"], unit=UNIT, cores=1)
+    except Exception as e:  # threadpoolctl missing: the all-threads leg stands alone
+        rec["single_thread"] = dict(value=None, note=f"not measured: {e}")
+    return rec
+
+
+class Workload:
+    """One benchmark workload resident on the device: a pass (every layer forward once), a verification pass that reads
+    the status word after every forward, and the end-to-end pass with host buffers."""
+
+    def __init__(self, args, name, rank, dev):
+        import torch
+        from paper_2601_19675_b200 import lopro, synth
+        self.torch, self.lopro, self.name, self.dev, self.args = torch, lopro, name, dev, args
+        cfg, T, ring = WORKLOADS[name]
+        self.cfg, self.T, self.ring = cfg, T, ring
+        layout = lopro.LAYOUT_ROWBLOCK if args.layout == "rowblock" else lopro.LAYOUT_FRAGMENT
+
+        def dev16(a):
+            return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev)
+
+        if cfg == "cfg5":
+            q = STACK_QUANT
+            shapes = sorted({(n, m) for _, n, m in STACK_LINEARS})
+            base, descs = {}, {}
+            for n, m in shapes:
+                layer = synth.random_layer(n, m, q["bits"], q["group_size"], q["rank"], seed=rank + n // 64)
+                base[(n, m)] = dict(codes=torch.from_numpy(layer["codes"]).to(dev), sc=dev16(layer["scales"]),
+                                    zr=dev16(layer["zeros"]), pm=torch.from_numpy(layer["perm"]).to(dev), A=dev16(layer["A"]),
+                                    B=dev16(layer["B"]))
+                descs[(n, m)] = lopro.make_desc(n, m, q["bits"], q["group_size"], q["block_size"], q["identity_cols"], q["rank"],
+                                                layout=layout)
+            self.x_bits = {n: synth.activations(T, n, seed=rank + n) for n in sorted({n for n, _ in shapes})}
+            xs = {n: dev16(b).view(torch.bfloat16) for n, b in self.x_bits.items()}
+            linears = []
+            for li in range(STACK_LAYERS):
+                for j, (_, n, m) in enumerate(STACK_LINEARS):
+                    b = base[(n, m)]
+                    i = li * len(STACK_LINEARS) + j
+                    codes = torch.roll(b["codes"], shifts=(i, 3 * i), dims=(0, 1)) if i else b["codes"]
+                    blob = lopro.pack(descs[(n, m)], codes, b["sc"], b["zr"], b["pm"], b["A"], b["B"])
+                    linears.append((descs[(n, m)], blob, xs[n], torch.empty((T, m), dtype=torch.bfloat16, device=dev)))
+            del codes
+            for b in base.values():
+                del b["codes"]
+            # sibling linears of a layer read the same activations: (q, k, v) and (gate, up) go through the grouped call
+            split = ((0,), (1,), (2,), (3,), (4,), (5,), (6,)) if args.no_groups else ((0, 1, 2), (3,), (4, 5), (6,))
+            self.calls = []   # (descs, blobs, x, ys)
+            for li in range(STACK_LAYERS):
+                L7 = linears[li * 7:(li + 1) * 7]
+                for idx in split:
+                    part = [L7[k] for k in idx]
+                    self.calls.append(([g[0] for g in part], [g[1] for g in part], part[0][2], [g[3] for g in part]))
+            self.x_dev, self.x_host_bits, self.y_last = xs[4096], self.x_bits[4096], self.calls[-1][3][-1]
+            self.forwards = len(linears)
+            self.tokens_per_pass = T
+            self.bytes_per_pass = stack_bytes(T)
+            self.flops_per_pass = None
+            self.h2d, self.d2h = T * 4096 * 2, T * self.y_last.shape[1] * 2
+            ws_bytes = max(lopro.group_workspace_bytes(c[0], T) for c in self.calls)
+            self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+            self.paths = sorted({lopro.PATH_NAMES.get(lopro.linear_fwd_path(d, T)[0], "?") for d, _, _, _ in linears})
+            self.launches_per_pass = sum(lopro.linear_fwd_group_path(c[0], T)[1] if len(c[0]) > 1
+                                         else lopro.linear_fwd_path(c[0][0], T)[1] for c in self.calls)
+            self.c = None
+            return
+        c = synth.CONFIGS[cfg]
+        self.c = c
+        d = lopro.make_desc(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"],
+                            layout=layout)
+        # ring of distinct layers: layer 0 drawn by the seeded generator, the others re-use its small tensors with the
+        # code matrix rolled per layer (set-up time only; every blob is a separate allocation)
+        base = synth.random_layer(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["rank"], seed=rank)
+        sc, zr, pm, A, B = dev16(base["scales"]), dev16(base["zeros"]), torch.from_numpy(base["perm"]).to(dev), \
+            dev16(base["A"]), dev16(base["B"])
+        codes0 = torch.from_numpy(base["codes"]).to(dev)
+        blobs = []
+        for i in range(ring):
+            if name.endswith("_L2") and i:
+                blobs.append(blobs[0])  # the same packed layer again: L2-resident measurement
+                continue
+            codes = torch.roll(codes0, shifts=(i, 3 * i), dims=(0, 1)) if i else codes0
+            blobs.append(lopro.pack(d, codes, sc, zr, pm, A, B))
+        del codes0, codes
+        self.x_host_bits = synth.activations(T, c["d_in"], seed=rank, outlier_frac=c.get("outlier_frac", 0.0),
+                                             outlier_scale=c.get("outlier_scale", 20.0))
+        x = dev16(self.x_host_bits).view(torch.bfloat16)
+        ys = [torch.empty((T, c["d_out"]), dtype=torch.bfloat16, device=dev) for _ in range(min(ring, 4))]
+        self.ws = torch.zeros(lopro.workspace_bytes(d, T) + lopro.host_staging_bytes(d, T), dtype=torch.uint8, device=dev)
+        self.calls = [([d], [blob], x, [ys[i % len(ys)]]) for i, blob in enumerate(blobs)]
+        self.d = d
+        self.forwards = ring
+        self.tokens_per_pass = T * ring
+        self.bytes_per_pass = ring * algorithmic_bytes(c, T)
+        self.flops_per_pass = ring * algorithmic_flops(c, T)
+        self.h2d, self.d2h = ring * T * c["d_in"] * 2, ring * T * c["d_out"] * 2
+        path, per_forward = lopro.linear_fwd_path(d, T)
+        self.paths = [lopro.PATH_NAMES.get(path, "?")]
+        self.launches_per_pass = per_forward * ring
+
+    def one_pass(self):
+        lopro = self.lopro
+        for ds, blobs, x, ys in self.calls:
             if len(ds) == 1:
-                lopro.linear_fwd(ds[0], blobs_[0], x, lopro.OUT_BF16, workspace=ws, y=ys_[0])
+                lopro.linear_fwd(ds[0], blobs[0], x, lopro.OUT_BF16, workspace=self.ws, y=ys[0])
             else:
-                lopro.linear_fwd_group(ds, blobs_, x, lopro.OUT_BF16, workspace=ws, ys=ys_)
+                lopro.linear_fwd_group(ds, blobs, x, lopro.OUT_BF16, workspace=self.ws, ys=ys)
 
+    def verify_pass(self):
+        """Untimed: every forward of the pass on its own, the device status word read after each of them (a forward
+        resets the word when it starts, so reading it once at the end would report the last forward only)."""
+        lopro, torch = self.lopro, self.torch
+        for k, (ds, blobs, x, ys) in enumerate(self.calls):
+            if len(ds) == 1:
+                lopro.linear_fwd(ds[0], blobs[0], x, lopro.OUT_BF16, workspace=self.ws, y=ys[0])
+            else:
+                lopro.linear_fwd_group(ds, blobs, x, lopro.OUT_BF16, workspace=self.ws, ys=ys)
+            torch.cuda.current_stream().synchronize()
+            status = lopro.workspace_status(self.ws)
+            assert status == lopro.OK, f"device status {status} after call {k} of {self.name}"
+            assert torch.isfinite(ys[-1].float()).all(), f"non-finite output after call {k} of {self.name}"
+
+    def e2e_setup(self):
+        torch = self.torch
+        self.xh = torch.from_numpy(self.x_host_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+        if self.cfg == "cfg5":
+            self.yh = torch.empty(tuple(self.y_last.shape), dtype=torch.bfloat16).pin_memory()
+        else:
+            self.yh = torch.empty((self.T, self.c["d_out"]), dtype=torch.bfloat16).pin_memory()
+
+    def e2e_pass(self, run_graph):
+        """The same work with host buffers: activations from pinned host memory, results back to the host."""
+        lopro = self.lopro
+        if self.cfg == "cfg5":
+            self.x_dev.copy_(self.xh, non_blocking=True)
+            run_graph()
+            self.yh.copy_(self.y_last, non_blocking=True)
+        else:
+            for ds, blobs, _, _ in self.calls:
+                lopro.linear_fwd_host(ds[0], blobs[0], self.xh, self.yh, self.ws, lopro.OUT_BF16)
+
+
+def measure(args, name, steps, warmup, rank, world, local, dev, dist, with_e2e=True):
+    """Builds the workload, times `steps` steps (each a whole number of passes lasting at least args.step_ms) and
+    returns the bench record."""
+    import torch
+    from paper_2601_19675_b200 import lopro
+    w = Workload(args, name, rank, dev)
     stream = torch.cuda.Stream(device=dev)
-    graph = None
     with torch.cuda.stream(stream):
-        one_step()
-        stream.synchronize()
+        w.verify_pass()
+        graph = None
         if not args.no_graph:
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=stream):
-                one_step()
-        run_step = graph.replay if graph is not None else one_step
-        for _ in range(args.warmup):
+                w.one_pass()
+        run_pass = graph.replay if graph is not None else w.one_pass
+        # passes per step: as many as it takes for a step to last args.step_ms
+        for _ in range(3):
+            run_pass()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(3):
+            run_pass()
+        e1.record(stream)
+        stream.synchronize()
+        pass_ms = e0.elapsed_time(e1) / 3
+        passes = max(1, int(np.ceil(args.step_ms / max(pass_ms, 1e-6))))
+        if world > 1:
+            passes = int(max_over_ranks([passes], dev)[0])
+
+        def run_step():
+            for _ in range(passes):
+                run_pass()
+
+        for _ in range(warmup):
             run_step()
         stream.synchronize()
         if world > 1:
@@ -346,89 +492,89 @@ def run_stack(args, T, rank, world, local, dev, dev16):
         if rank == 0:
             sampler.start()
         torch.cuda.synchronize()
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
         ev[0].record(stream)
-        for k in range(args.steps):
+        for k in range(steps):
             run_step()
             ev[k + 1].record(stream)
         stream.synchronize()
         torch.cuda.synchronize()
         clocks = sampler.stop() if rank == 0 else None
         total_ms = ev[0].elapsed_time(ev[-1])
-        step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
-        # end to end: the batch's activations come from pinned host memory every step, the last linear's output
-        # goes back to the host
-        xh = torch.from_numpy(x_bits[4096].view(np.int16)).view(torch.bfloat16).pin_memory()
-        y_last = linears[-1][3]
-        yh = torch.empty(tuple(y_last.shape), dtype=torch.bfloat16).pin_memory()
-        e2e_steps = max(3, min(args.steps, 20))
-
-        def e2e_step():
-            xs[4096].copy_(xh, non_blocking=True)
-            run_step()
-            yh.copy_(y_last, non_blocking=True)
-
-        for _ in range(3):
-            e2e_step()
-        stream.synchronize()
-        if world > 1:
-            dist.barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(e2e_steps):
-            e2e_step()
-        e1.record(stream)
-        stream.synchronize()
-        e2e_ms = e0.elapsed_time(e1)
-        status = lopro.workspace_status(ws)
-        assert status == lopro.OK, f"device status {status}"
-        assert torch.isfinite(yh.float()).all()
+        step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(steps)]
+        e2e_ms, e2e_steps = None, 0
+        if with_e2e:
+            w.e2e_setup()
+            e2e_steps = 5
+            for _ in range(2):
+                w.e2e_pass(run_pass)
+            stream.synchronize()
+            if world > 1:
+                dist.barrier()
+            e0.record(stream)
+            for _ in range(e2e_steps):
+                w.e2e_pass(run_pass)
+            e1.record(stream)
+            stream.synchronize()
+            e2e_ms = e0.elapsed_time(e1)
+            assert torch.isfinite(w.yh.float()).all()
+        w.verify_pass()
     if world > 1:
-        total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dev)
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return 0
+        total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms if e2e_ms is not None else 0.0], dev)
     peaks = measured_peaks()
-    ms_per_step = total_ms / args.steps
-    value = T * world / (ms_per_step * 1e-3)
-    e2e_value = T * world / (e2e_ms / e2e_steps * 1e-3)
-    paths = [lopro.linear_fwd_path(d, T) for d, _, _, _ in linears]
-    names = sorted({lopro.PATH_NAMES.get(p, "?") for p, _ in paths})
-    n_launches = sum(lopro.linear_fwd_group_path(g[0], T)[1] if len(g[0]) > 1 else lopro.linear_fwd_path(g[0][0], T)[1]
-                     for g in groups)
-    ach = stack_bytes(T) / (ms_per_step * 1e-3) / 1e9
-    roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"], traffic=None,
-                    peak_source=f"of {peaks['source']}", frac_of_nominal_8000=ach / 8000.0,
-                    kernel=" + ".join(n + "_kernel" for n in names), algorithmic_bytes_per_step=stack_bytes(T),
-                    launch_us=ms_per_step * 1e3 / len(linears),
-                    note="whole step: 224 linear forwards (prologue kernels included); launch_us = step time / 224")
-    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
-                ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
-                data="synthetic", config=workload_config(args.workload), clocks=clocks,
-                e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=T * 4096 * 2, d2h_bytes_per_step=T * y_last.shape[1] * 2,
-                         steps=e2e_steps),
-                gpu_launches=n_launches * args.steps, path="+".join(names), launches_per_step=n_launches, roofline=roofline,
-                step_ms_min=min(step_ms), step_ms_median=statistics.median(step_ms), cuda_graph=graph is not None)
-    if not args.no_cpu_baseline and world == 1:
-        r = time_oracle_stack(T, 12.0)
-        line["cpu_baseline"] = dict(value=r["value"], unit=UNIT, cores=r["cores"], kind="oracle", sample=r["sample"])
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
-    return 0
+    ms_per_step = total_ms / steps
+    ms_per_pass = ms_per_step / passes
+    value = w.tokens_per_pass * passes * world / (ms_per_step * 1e-3)
+    per_forward_s = ms_per_pass * 1e-3 / w.forwards
+    kernel = " + ".join({"stream": "stream_kernel", "wide": "stream_wide_kernel", "tall": "tall_kernel", "general": "decode_kernel",
+                         "prefill": "prefill_kernel", "rowblock": "rowblock_kernel"}.get(n, n) for n in w.paths)
+    note = ("duration = step time / layer forwards (includes the prologue kernels of each forward): an upper bound on the "
+            "product kernel's own duration, a lower bound on `achieved`")
+    if w.T <= 64:
+        ach = w.bytes_per_pass / (ms_per_pass * 1e-3) / 1e9
+        roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
+                        traffic=NCU_TRAFFIC.get((name, kernel)), peak_source=f"of {peaks['source']}",
+                        frac_of_nominal_8000=ach / 8000.0, kernel=kernel, algorithmic_bytes_per_launch=w.bytes_per_pass // w.forwards,
+                        launch_us=per_forward_s * 1e6, note=note)
+    else:
+        ach = w.flops_per_pass / (ms_per_pass * 1e-3) / 1e12
+        pk = peaks["bf16_tflops_sustained"]
+        roofline = dict(bound="tensor", achieved=ach, peak=pk, unit="TFLOP/s", frac=ach / pk, traffic=NCU_TRAFFIC.get((name, kernel)),
+                        peak_source=f"of {peaks['source']} (sustained, the kernel runs inside a long step)",
+                        frac_of_burst_peak=ach / peaks["bf16_tflops"], burst_peak=peaks["bf16_tflops"], kernel=kernel,
+                        algorithmic_flops_per_launch=w.flops_per_pass // w.forwards, launch_us=per_forward_s * 1e6, note=note)
+    rec = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps, warmup=warmup, ms_per_step=ms_per_step,
+               higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+               config=dict(workload_config(name), passes_per_step=passes, layout=args.layout), clocks=clocks,
+               gpu_launches=w.launches_per_pass * passes * steps, path="+".join(w.paths), roofline=roofline,
+               ms_per_forward=per_forward_s * 1e3, ms_per_pass=ms_per_pass, step_ms_min=min(step_ms),
+               step_ms_median=statistics.median(step_ms), cuda_graph=graph is not None,
+               status_checked="after every forward of an untimed pass before and after the timed region")
+    if e2e_ms is not None:
+        rec["e2e"] = dict(value=w.tokens_per_pass * world / (e2e_ms / e2e_steps * 1e-3), unit=UNIT, h2d_bytes_per_step=w.h2d,
+                          d2h_bytes_per_step=w.d2h, steps=e2e_steps,
+                          note="one pass per step through the host-buffer entry point (pinned host x in, host y out)")
+    rec["_workload"] = w
+    return rec
+
+
+# workloads reported beside the bench line (driver-run evidence for every regime), with the steps each gets
+EXTRA_WORKLOADS = [("cfg2_T1", 5), ("cfg2_T32", 5), ("cfg4_T16", 5), ("cfg5_T1", 5), ("cfg5_T32", 5), ("cfg3_T2048", 5),
+                   ("cfg4_T4096", 4)]
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2_T8", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="lopro", choices=["lopro", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch through the stream instead of a CUDA graph")
     ap.add_argument("--no-groups", action="store_true", help="stack workloads: every linear on its own (no grouped siblings)")
+    ap.add_argument("--no-extras", action="store_true", help="only the named workload, not the table of the other regimes")
+    ap.add_argument("--step-ms", type=float, default=50.0, help="a step repeats the pass until it lasts this long")
     ap.add_argument("--layout", default="fragment", choices=["fragment", "rowblock"], help="code layout of the packed layers")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -445,6 +591,7 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
+    dist = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -453,160 +600,35 @@ def main():
     if world > 1:
         dist.barrier()
     lopro.lib()
-
-    cfg, T, ring = WORKLOADS[args.workload]
     dev = torch.device("cuda", local)
 
-    def dev16(a):
-        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev)
-
-    if cfg == "cfg5":
-        return run_stack(args, T, rank, world, local, dev, dev16)
-    c = synth.CONFIGS[cfg]
-    d = lopro.make_desc(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"],
-                        layout=lopro.LAYOUT_ROWBLOCK if args.layout == "rowblock" else lopro.LAYOUT_FRAGMENT)
-
-    # ring of distinct layers: layer 0 drawn by the seeded generator, the others re-use its tensors with
-    # freshly drawn codes (generated on the host once, shifted per layer) so that set-up stays short
-    base = synth.random_layer(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["rank"], seed=rank)
-    sc, zr, pm, A, B = dev16(base["scales"]), dev16(base["zeros"]), torch.from_numpy(base["perm"]).to(dev), \
-        dev16(base["A"]), dev16(base["B"])
-    codes0 = torch.from_numpy(base["codes"]).to(dev)
-    blobs = []
-    for i in range(ring):
-        if args.workload.endswith("_L2") and i:
-            blobs.append(blobs[0])  # the same packed layer again: L2-resident measurement
-            continue
-        codes = torch.roll(codes0, shifts=(i, 3 * i), dims=(0, 1)) if i else codes0
-        blobs.append(lopro.pack(d, codes, sc, zr, pm, A, B))
-    del codes0, codes
-    x_bits = synth.activations(T, c["d_in"], seed=rank, outlier_frac=c.get("outlier_frac", 0.0),
-                               outlier_scale=c.get("outlier_scale", 20.0))
-    x = dev16(x_bits).view(torch.bfloat16)
-    ys = [torch.empty((T, c["d_out"]), dtype=torch.bfloat16, device=dev) for _ in range(min(ring, 4))]
-    ws = torch.zeros(lopro.workspace_bytes(d, T) + lopro.host_staging_bytes(d, T), dtype=torch.uint8, device=dev)
-
-    def one_step():
-        for i, blob in enumerate(blobs):
-            lopro.linear_fwd(d, blob, x, lopro.OUT_BF16, workspace=ws, y=ys[i % len(ys)])
-
-    stream = torch.cuda.Stream(device=dev)
-    graph = None
-    with torch.cuda.stream(stream):
-        one_step()
-        stream.synchronize()
-        if not args.no_graph:
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                one_step()
-
-        def run_step():
-            if graph is not None:
-                graph.replay()
-            else:
-                one_step()
-
-        for _ in range(args.warmup):
-            run_step()
-        stream.synchronize()
-        if world > 1:
-            dist.barrier()
-        sampler = ClockSampler(local)
-        if rank == 0:
-            sampler.start()
-        torch.cuda.synchronize()
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-        ev[0].record(stream)
-        for k in range(args.steps):
-            run_step()
-            ev[k + 1].record(stream)
-        stream.synchronize()
-        torch.cuda.synchronize()
-        clocks = sampler.stop() if rank == 0 else None
-        total_ms = ev[0].elapsed_time(ev[-1])
-        step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
-
-        # end to end through the host entry point: pinned host activations in, host result out, every layer
-        xh = torch.from_numpy(x_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
-        yh = torch.empty((T, c["d_out"]), dtype=torch.bfloat16).pin_memory()
-        e2e_steps = max(3, min(args.steps, 20))
-
-        def e2e_step():
-            for blob in blobs:
-                lopro.linear_fwd_host(d, blob, xh, yh, ws, lopro.OUT_BF16)
-
-        for _ in range(3):
-            e2e_step()
-        stream.synchronize()
-        if world > 1:
-            dist.barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(e2e_steps):
-            e2e_step()
-        e1.record(stream)
-        stream.synchronize()
-        e2e_ms = e0.elapsed_time(e1)
-        status = lopro.workspace_status(ws)
-        assert status == lopro.OK, f"device status {status}"
-        assert torch.isfinite(yh.float()).all()
-
-    if world > 1:
-        total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dev)
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return 0
-
-    peaks = measured_peaks()
-    ms_per_step = total_ms / args.steps
-    tokens_per_step = T * ring * world
-    value = tokens_per_step / (ms_per_step * 1e-3)
-    e2e_value = T * ring * world / (e2e_ms / e2e_steps * 1e-3)
-    # Dominant kernel: the forward kernel that reads the packed weights, launched once per layer.  Its
-    # launch duration is taken as (step time / launches), i.e. the whole per-layer time including any
-    # prologue kernels of the path -- an upper bound on the kernel's own duration, a lower bound on
-    # `achieved`.
-    path, kernels_per_forward = lopro.linear_fwd_path(d, T)
-    path_name = lopro.PATH_NAMES.get(path, "?")
-    kernel_name = {"stream": "stream_kernel", "wide": "stream_wide_kernel", "tall": "tall_kernel", "general": "decode_kernel",
-                   "prefill": "prefill_kernel", "rowblock": "rowblock_kernel"}.get(path_name, "?")
-    note = "duration = step time / layer forwards (includes the prologue kernels)"
-    launches_per_step = ring
-    dur_s = ms_per_step * 1e-3 / launches_per_step
-    hbm_bound = T <= 64
-    if hbm_bound:
-        ach = algorithmic_bytes(c, T) / dur_s / 1e9
-        roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
-                        traffic=NCU_TRAFFIC.get((args.workload, kernel_name)), peak_source=f"of {peaks['source']}",
-                        frac_of_nominal_8000=ach / 8000.0, kernel=kernel_name,
-                        algorithmic_bytes_per_launch=algorithmic_bytes(c, T), launch_us=dur_s * 1e6, note=note)
-    else:
-        ach = algorithmic_flops(c, T) / dur_s / 1e12
-        pk = peaks["bf16_tflops_sustained"]
-        roofline = dict(bound="tensor", achieved=ach, peak=pk, unit="TFLOP/s", frac=ach / pk,
-                        traffic=NCU_TRAFFIC.get((args.workload, kernel_name)),
-                        peak_source=f"of {peaks['source']} (sustained)", kernel=kernel_name,
-                        algorithmic_flops_per_launch=algorithmic_flops(c, T), launch_us=dur_s * 1e6, note=note)
-    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
-                ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
-                data="synthetic", config=workload_config(args.workload), clocks=clocks,
-                e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=ring * T * c["d_in"] * 2,
-                         d2h_bytes_per_step=ring * T * c["d_out"] * 2, steps=e2e_steps),
-                gpu_launches=kernels_per_forward * ring * args.steps, path=path_name, roofline=roofline,
-                step_ms_min=min(step_ms), step_ms_median=statistics.median(step_ms),
-                cuda_graph=graph is not None)
-    if not args.no_cpu_baseline and world == 1:
-        max_rows = 1024 if c["d_out"] * c["d_in"] > (1 << 24) or T > 64 else None
-        max_tokens = 16 if T > 64 else None
-        r = time_oracle(c, T, 12.0, max_rows, max_tokens)
-        line["cpu_baseline"] = dict(
-            value=r["value"], unit=UNIT, cores=r["cores"], kind="oracle",
-            sample=(f"oracle.forward_exact (fp64 numpy) on {r['rows']} of {c['d_out']} output rows, {r['tokens']} of {T} "
-                    f"tokens of one layer, {r['reps']} repetitions, scaled linearly to a full layer forward"))
+    line = measure(args, args.workload, args.steps, args.warmup, rank, world, local, dev, dist)
+    w = line.pop("_workload")
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline_record(w.c, w.T, 10.0, stack=w.cfg == "cfg5")
+    del w
+    torch.cuda.empty_cache()
+    # the other regimes, each measured the same way with fewer steps (1 GPU only: replicas would repeat them)
+    if world == 1 and not args.no_extras:
+        table = {}
+        for name, st in EXTRA_WORKLOADS:
+            if name == args.workload:
+                continue
+            r = measure(args, name, st, 3, rank, world, local, dev, dist, with_e2e=False)
+            r.pop("_workload")
+            torch.cuda.empty_cache()
+            table[name] = dict(value=r["value"], unit=UNIT, ms_per_forward=r["ms_per_forward"], ms_per_step=r["ms_per_step"],
+                               steps=st, path=r["path"], gpu_launches=r["gpu_launches"],
+                               roofline={k: r["roofline"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "kernel")
+                                         } | ({"frac_of_burst_peak": r["roofline"]["frac_of_burst_peak"]}
+                                              if "frac_of_burst_peak" in r["roofline"] else
+                                              {"frac_of_nominal_8000": r["roofline"]["frac_of_nominal_8000"]}),
+                               clocks=r["clocks"], workload=r["config"]["workload"])
+        line["workloads"] = table
+    if rank == 0:
+        print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
-    print(json.dumps(line))
     return 0
 
 
