@@ -86,7 +86,16 @@ typedef struct {
     int32_t identity_cols;
     int32_t rank;
     int32_t layout;
+    int32_t lowrank_format; /* LOPRO_LOWRANK_FOLDED_F16 or LOPRO_LOWRANK_FP8 */
 } lopro_desc;
+
+/* Storage of the rank-r term W_r.
+ *   FOLDED_F16: A = U Sigma [m][r] and B = V diag(s)^-1 [r][n] in fp16, the W_L W_R of Eq. 4; y_lr = A (B x).
+ *   FP8: the record Algorithm 1 saves, (U, V, Sigma, s): U [m][r] and V [r][n] in fp8 e4m3 (Sec. 3.3 casts the unit
+ *   vectors of every R1SVD step to fp8), Sigma [r] and the activation scale s [n] in fp16;
+ *   y_lr = U (Sigma (V (x / s))).  Half the bytes per factor entry (Appendix A.2: about 0.05 bit per weight at r = 16).
+ *   Served by the small-batch kernels of LOPRO_LAYOUT_FRAGMENT (any T: more than 32 tokens run as chunks of 32). */
+enum { LOPRO_LOWRANK_FOLDED_F16 = 0, LOPRO_LOWRANK_FP8 = 1 };
 
 /* Sections of the packed blob, for lopro_packed_section. */
 enum {
@@ -95,9 +104,11 @@ enum {
     LOPRO_SEC_SCALEZERO = 2, /* (scale, zero) fp16 pairs: canonical [m][n/g]; fragment layout
                                 [m/16][n/g][16]                                                    */
     LOPRO_SEC_PERM = 3,   /* int32 [n]                                                             */
-    LOPRO_SEC_A = 4,      /* fp16 [m][r_pad]                                                       */
-    LOPRO_SEC_B = 5,      /* fp16 [r_pad][n]                                                       */
-    LOPRO_SEC_COUNT = 6
+    LOPRO_SEC_A = 4,      /* fp16 [m][r_pad]  (FP8 format: U, e4m3 [m][r_pad])                      */
+    LOPRO_SEC_B = 5,      /* fp16 [r_pad][n]  (FP8 format: V, e4m3 [r_pad][n])                      */
+    LOPRO_SEC_SIGMA = 6,  /* FP8 format only: fp16 [r_pad]                                         */
+    LOPRO_SEC_S = 7,      /* FP8 format only: fp16 [n]                                             */
+    LOPRO_SEC_COUNT = 8
 };
 
 /* Tuning switches of lopro_configure.  They change which kernels a forward runs, never what it computes; they
@@ -129,7 +140,8 @@ LOPRO_API lopro_status lopro_check_desc(const lopro_desc* desc);
  * flat, relocatable byte buffer: a 256-byte header followed by 256-byte aligned sections;
  * copying it (device to device, to the host, to a file) copies the layer.  Its size follows
  * the storage accounting of Eq. 13 with this library's widths: d_q bits per code, 2 x 16 bits
- * per group (scale and zero-point), 16 bits per factor entry, 32 bits per permutation entry. */
+ * per group (scale and zero-point), 16 bits per factor entry (8 in the FP8 low-rank format, plus 16 bits per entry of
+ * Sigma and s), 32 bits per permutation entry. */
 LOPRO_API size_t lopro_packed_bytes(const lopro_desc* desc);
 
 /* Offset and size in bytes of one section of the blob.  Returns LOPRO_ERR_INVALID_ARG for a
@@ -153,6 +165,21 @@ LOPRO_API size_t lopro_workspace_bytes(const lopro_desc* desc, int32_t T);
 LOPRO_API lopro_status lopro_pack(const lopro_desc* desc, const uint8_t* codes, const uint16_t* scales_f16,
                         const uint16_t* zeros_f16, const int32_t* perm, const uint16_t* A_f16,
                         const uint16_t* B_f16, void* packed, size_t packed_bytes, void* stream);
+
+/* The same for a layer whose descriptor says LOPRO_LOWRANK_FP8: the saved record (W_q, U, V, Sigma, p, s) of
+ * Algorithm 1 as it is, nothing folded.
+ *   U_e4m3 uint8 [m][r]   V_e4m3 uint8 [r][n]   (fp8 e4m3 bit patterns; NaN patterns are rejected)
+ *   sigma_f16 fp16 [r]    s_f16 fp16 [n]        (finite; s non-zero)
+ * Everything else as lopro_pack (which returns LOPRO_ERR_INVALID_ARG for such a descriptor, as this call does for
+ * a LOPRO_LOWRANK_FOLDED_F16 one).  rank must be > 0. */
+LOPRO_API lopro_status lopro_pack_lr8(const lopro_desc* desc, const uint8_t* codes, const uint16_t* scales_f16,
+                                      const uint16_t* zeros_f16, const int32_t* perm, const uint8_t* U_e4m3,
+                                      const uint8_t* V_e4m3, const uint16_t* sigma_f16, const uint16_t* s_f16, void* packed,
+                                      size_t packed_bytes, void* stream);
+/* Reads the low-rank record of an FP8-format blob back, bit for bit (any pointer may be NULL).  For such a blob
+ * lopro_unpack returns the codes, scales, zero-points and perm; its A and B pointers must be NULL. */
+LOPRO_API lopro_status lopro_unpack_lr8(const lopro_desc* desc, const void* packed, uint8_t* U_e4m3, uint8_t* V_e4m3,
+                                        uint16_t* sigma_f16, uint16_t* s_f16, void* stream);
 
 /* Exact inverse of lopro_pack for either layout: writes the arrays lopro_pack was given, bit
  * for bit.  Any output pointer may be NULL to skip that array.  `words` (optional) receives

@@ -447,6 +447,72 @@ def forward_mirrored(x, codes, scales, zeros, perm, a, b, g, b_i, b_h,
     return round_bf16(y) if out == "bf16" else round_f32(y)
 
 
+def forward_exact_unfolded(x, codes, scales, zeros, perm, u, sigma, v, s, g, b_i, b_h):
+    """Eq. 8 with the low-rank branch in the form Algorithm 1 saves, the record (W_q, U, V, Sigma, p, s):
+    y = U (Sigma (V (x / s))) + W^ (Q^T P^T x), i.e. W_r = U Sigma V diag(s)^-1 (Eq. 4 with alpha = diag(s); Sec. 3.3
+    keeps s apart so that the fp8 factors U, V stay unit vectors).  u [m][r], sigma [r], v [r][n], s [n]; all fp64,
+    no intermediate rounding."""
+    x = np.asarray(x, dtype=np.float64)
+    xt = rotate(x, perm, b_i, b_h)
+    y_q = xt @ dequant(codes, scales, zeros, g).T
+    t = (x / np.asarray(s, dtype=np.float64)[None, :]) @ np.asarray(v, dtype=np.float64).T   # Y = V (X / s)
+    t = t * np.asarray(sigma, dtype=np.float64)[None, :]                                    # Sigma Y
+    return y_q + t @ np.asarray(u, dtype=np.float64).T                                      # O = U (Sigma Y)
+
+
+def forward_mirrored_unfolded(x, codes, scales, zeros, perm, u, sigma, v, s, g, b_i, b_h, round_t="f16", out="f32"):
+    """forward_exact_unfolded with the declared roundings: x~ -> bf16, t = Sigma V (x / s) -> fp16 (or none),
+    y -> fp32 or bf16."""
+    x = np.asarray(x, dtype=np.float64)
+    xt = round_bf16(rotate(x, perm, b_i, b_h))
+    y_q = xt @ dequant(codes, scales, zeros, g).T
+    t = ((x / np.asarray(s, dtype=np.float64)[None, :]) @ np.asarray(v, dtype=np.float64).T) * np.asarray(sigma, dtype=np.float64)[None, :]
+    if round_t == "f16":
+        t = round_f16(t)
+    y = y_q + t @ np.asarray(u, dtype=np.float64).T
+    return round_bf16(y) if out == "bf16" else round_f32(y)
+
+
+def lopro_quantize_unfolded(w, perm, b_i, b_h, r, bits, g, s, it, sketches):
+    """Algorithm 1 for one layer with the low-rank factors kept as the paper stores them: W_s = W diag(s); R1SVD of
+    W_s with U_1, V_1 cast to fp8 e4m3 inside the loop (Sec. 3.3), Sigma rounded to fp16; the residual is taken against
+    the STORED factors, R = W - U Sigma V diag(s)^-1, then R' = R P Q and RTN group quantization as in lopro_quantize.
+    Returns dict(codes, scales, zeros, U, sigma, V, s) (fp64 arrays holding e4m3 / fp16 values; s rounded to fp16)."""
+    w = np.asarray(w, dtype=np.float64)
+    s = round_f16(np.asarray(s, dtype=np.float64))
+    u, sig, v = r1svd(w * s[None, :], r, it, sketches, cast=round_e4m3)
+    sig = round_f16(sig)
+    resid = w - (u * sig[None, :]) @ (v / s[None, :])
+    rp = partial_block_rotate(permute_columns(resid, perm), b_i, b_h)
+    codes, scales, zeros = rtn_quantize(rp, bits, g)
+    return dict(codes=codes, scales=scales, zeros=zeros, U=u, sigma=sig, V=v, s=s)
+
+
+def f64_to_e4m3_bits(x):
+    """Exactly representable fp64 values -> fp8 e4m3 bit patterns (uint8): sign, 4 exponent bits (bias 7), 3 mantissa
+    bits; subnormals below 2^-6; no infinities (the finite-only format of the ML fp8 proposal)."""
+    x = np.asarray(x, dtype=np.float64)
+    sign = (np.signbit(x)).astype(np.uint8) << 7
+    a = np.abs(x)
+    out = np.zeros(x.shape, dtype=np.uint8)
+    nz = a > 0
+    m, e = np.frexp(a[nz])                    # a = m 2^e, 0.5 <= m < 1  ->  a = (2m) 2^(e-1)
+    exp = e - 1
+    normal = exp >= -6
+    bits = np.zeros(m.shape, dtype=np.int64)
+    bits[normal] = ((exp[normal] + 7) << 3) | np.rint((2.0 * m[normal] - 1.0) * 8.0).astype(np.int64)
+    bits[~normal] = np.rint(a[nz][~normal] * 2.0 ** 9).astype(np.int64)       # subnormal: k 2^-9, k = 1..7
+    out[nz] = bits.astype(np.uint8)
+    return out | sign
+
+
+def e4m3_bits_to_f64(b):
+    b = np.asarray(b, dtype=np.uint8).astype(np.int64)
+    sign = np.where(b & 0x80, -1.0, 1.0)
+    exp, man = (b >> 3) & 15, b & 7
+    return sign * np.where(exp == 0, man * 2.0 ** -9, (1.0 + man / 8.0) * 2.0 ** (exp - 7.0))
+
+
 def max_rel_err(y, y_ref):
     """Element-wise error relative to max(|y_ref[t, i]|, rms_i y_ref[t, :]): the
     'max relative error' of the acceptance gates, floored at the row RMS so that

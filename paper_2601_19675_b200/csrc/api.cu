@@ -14,6 +14,8 @@ lopro_status check_desc(const lopro_desc& d) {
     if (d.identity_cols < 0 || d.identity_cols > d.d_in) return LOPRO_ERR_INVALID_ARG;
     if ((d.d_in - d.identity_cols) % d.block_size != 0) return LOPRO_ERR_INVALID_ARG;
     if (d.rank < 0 || d.rank > 512) return LOPRO_ERR_INVALID_ARG;
+    if (d.lowrank_format != LOPRO_LOWRANK_FOLDED_F16 && d.lowrank_format != LOPRO_LOWRANK_FP8) return LOPRO_ERR_INVALID_ARG;
+    if (d.lowrank_format == LOPRO_LOWRANK_FP8 && d.rank == 0) return LOPRO_ERR_INVALID_ARG;
     if (d.layout != LOPRO_LAYOUT_CANONICAL && d.layout != LOPRO_LAYOUT_FRAGMENT && d.layout != LOPRO_LAYOUT_ROWBLOCK)
         return LOPRO_ERR_INVALID_ARG;
     // Kernel coverage: 64-column steps, 16-row tiles, rows short enough for one CTA's shared memory.
@@ -33,8 +35,11 @@ lopro_status blob_layout(const lopro_desc& d, BlobLayout* out) {
     bytes[LOPRO_SEC_CODES] = m * n * (size_t)d.bits / 8;
     bytes[LOPRO_SEC_SCALEZERO] = m * ng * 4;
     bytes[LOPRO_SEC_PERM] = n * 4;
-    bytes[LOPRO_SEC_A] = m * (size_t)r_pad * 2;
-    bytes[LOPRO_SEC_B] = (size_t)r_pad * n * 2;
+    const size_t esz = d.lowrank_format == LOPRO_LOWRANK_FP8 ? 1 : 2;
+    bytes[LOPRO_SEC_A] = m * (size_t)r_pad * esz;
+    bytes[LOPRO_SEC_B] = (size_t)r_pad * n * esz;
+    bytes[LOPRO_SEC_SIGMA] = d.lowrank_format == LOPRO_LOWRANK_FP8 ? (size_t)r_pad * 2 : 0;
+    bytes[LOPRO_SEC_S] = d.lowrank_format == LOPRO_LOWRANK_FP8 ? n * 2 : 0;
     size_t off = 0;
     for (int s = 0; s < LOPRO_SEC_COUNT; ++s) {
         out->off[s] = off;
@@ -196,15 +201,17 @@ size_t lopro_workspace_bytes(const lopro_desc* desc, int32_t T) {
     return W.total;
 }
 
-lopro_status lopro_pack(const lopro_desc* desc, const uint8_t* codes, const uint16_t* scales_f16,
-                        const uint16_t* zeros_f16, const int32_t* perm, const uint16_t* A_f16,
-                        const uint16_t* B_f16, void* packed, size_t packed_bytes, void* stream) {
-    if (!desc) return LOPRO_ERR_INVALID_ARG;
+static lopro_status pack_any(const lopro_desc* desc, const uint8_t* codes, const uint16_t* scales_f16,
+                             const uint16_t* zeros_f16, const int32_t* perm, const uint16_t* A_f16, const uint16_t* B_f16,
+                             const uint8_t* U8, const uint8_t* V8, const uint16_t* sigma, const uint16_t* svec, void* packed,
+                             size_t packed_bytes, void* stream) {
     BlobLayout L;
     lopro_status st = blob_layout(*desc, &L);
     if (st != LOPRO_OK) return st;
+    const bool lr8 = desc->lowrank_format == LOPRO_LOWRANK_FP8;
     if (!codes || !scales_f16 || !zeros_f16 || !perm || !packed) return LOPRO_ERR_INVALID_ARG;
-    if (desc->rank > 0 && (!A_f16 || !B_f16)) return LOPRO_ERR_INVALID_ARG;
+    if (!lr8 && desc->rank > 0 && (!A_f16 || !B_f16)) return LOPRO_ERR_INVALID_ARG;
+    if (lr8 && (!U8 || !V8 || !sigma || !svec)) return LOPRO_ERR_INVALID_ARG;
     if (!aligned(packed, 256)) return LOPRO_ERR_INVALID_ARG;
     if (packed_bytes < L.total) return LOPRO_ERR_BUFFER_TOO_SMALL;
     cudaStream_t s = (cudaStream_t)stream;
@@ -225,8 +232,10 @@ lopro_status lopro_pack(const lopro_desc* desc, const uint8_t* codes, const uint
     if (cudaMemsetAsync(packed, 0, L.total, s) != cudaSuccess) return LOPRO_ERR_CUDA;
     if (cudaMemcpyAsync(packed, &h, sizeof(h), cudaMemcpyHostToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
     if (launch_validate(*desc, codes, scales_f16, zeros_f16, perm, packed, L, s) != cudaSuccess) return LOPRO_ERR_CUDA;
-    if (launch_pack(*desc, codes, scales_f16, zeros_f16, perm, A_f16, B_f16, packed, L, s) != cudaSuccess)
+    if (launch_pack(*desc, codes, scales_f16, zeros_f16, perm, lr8 ? nullptr : A_f16, lr8 ? nullptr : B_f16, packed, L, s) !=
+        cudaSuccess)
         return LOPRO_ERR_CUDA;
+    if (lr8 && launch_pack_lr8(*desc, U8, V8, sigma, svec, packed, L, s) != cudaSuccess) return LOPRO_ERR_CUDA;
     BlobHeader back;
     if (cudaMemcpyAsync(&back, packed, sizeof(back), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOPRO_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return LOPRO_ERR_CUDA;
@@ -243,6 +252,47 @@ lopro_status lopro_pack(const lopro_desc* desc, const uint8_t* codes, const uint
     return LOPRO_OK;
 }
 
+lopro_status lopro_pack(const lopro_desc* desc, const uint8_t* codes, const uint16_t* scales_f16,
+                        const uint16_t* zeros_f16, const int32_t* perm, const uint16_t* A_f16,
+                        const uint16_t* B_f16, void* packed, size_t packed_bytes, void* stream) {
+    if (!desc) return LOPRO_ERR_INVALID_ARG;
+    if (check_desc(*desc) == LOPRO_OK && desc->lowrank_format != LOPRO_LOWRANK_FOLDED_F16) return LOPRO_ERR_INVALID_ARG;
+    return pack_any(desc, codes, scales_f16, zeros_f16, perm, A_f16, B_f16, nullptr, nullptr, nullptr, nullptr, packed,
+                    packed_bytes, stream);
+}
+
+lopro_status lopro_pack_lr8(const lopro_desc* desc, const uint8_t* codes, const uint16_t* scales_f16,
+                            const uint16_t* zeros_f16, const int32_t* perm, const uint8_t* U_e4m3, const uint8_t* V_e4m3,
+                            const uint16_t* sigma_f16, const uint16_t* s_f16, void* packed, size_t packed_bytes, void* stream) {
+    if (!desc) return LOPRO_ERR_INVALID_ARG;
+    if (check_desc(*desc) == LOPRO_OK && desc->lowrank_format != LOPRO_LOWRANK_FP8) return LOPRO_ERR_INVALID_ARG;
+    return pack_any(desc, codes, scales_f16, zeros_f16, perm, nullptr, nullptr, U_e4m3, V_e4m3, sigma_f16, s_f16, packed,
+                    packed_bytes, stream);
+}
+
+static lopro_status read_header(const lopro_desc* desc, const void* packed, const BlobLayout& L, cudaStream_t s) {
+    BlobHeader h;
+    if (cudaMemcpyAsync(&h, packed, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (h.magic != kBlobMagic || h.version != kBlobVersion || memcmp(&h.desc, desc, sizeof(lopro_desc)) != 0 ||
+        h.total_bytes != L.total || h.invalid != 0)
+        return LOPRO_ERR_INVALID_DATA;
+    return LOPRO_OK;
+}
+
+lopro_status lopro_unpack_lr8(const lopro_desc* desc, const void* packed, uint8_t* U_e4m3, uint8_t* V_e4m3,
+                              uint16_t* sigma_f16, uint16_t* s_f16, void* stream) {
+    if (!desc || !packed) return LOPRO_ERR_INVALID_ARG;
+    BlobLayout L;
+    lopro_status st = blob_layout(*desc, &L);
+    if (st != LOPRO_OK) return st;
+    if (desc->lowrank_format != LOPRO_LOWRANK_FP8) return LOPRO_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    st = read_header(desc, packed, L, s);
+    if (st != LOPRO_OK) return st;
+    return launch_unpack_lr8(*desc, packed, L, U_e4m3, V_e4m3, sigma_f16, s_f16, s) == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
+}
+
 lopro_status lopro_unpack(const lopro_desc* desc, const void* packed, uint8_t* codes, uint32_t* words,
                           uint16_t* scales_f16, uint16_t* zeros_f16, int32_t* perm, uint16_t* A_f16,
                           uint16_t* B_f16, void* stream) {
@@ -251,12 +301,9 @@ lopro_status lopro_unpack(const lopro_desc* desc, const void* packed, uint8_t* c
     lopro_status st = blob_layout(*desc, &L);
     if (st != LOPRO_OK) return st;
     cudaStream_t s = (cudaStream_t)stream;
-    BlobHeader h;
-    if (cudaMemcpyAsync(&h, packed, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOPRO_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return LOPRO_ERR_CUDA;
-    if (h.magic != kBlobMagic || h.version != kBlobVersion || memcmp(&h.desc, desc, sizeof(lopro_desc)) != 0 ||
-        h.total_bytes != L.total || h.invalid != 0)
-        return LOPRO_ERR_INVALID_DATA;
+    if (desc->lowrank_format == LOPRO_LOWRANK_FP8 && (A_f16 || B_f16)) return LOPRO_ERR_INVALID_ARG;
+    st = read_header(desc, packed, L, s);
+    if (st != LOPRO_OK) return st;
     if (launch_unpack(*desc, packed, L, codes, words, scales_f16, zeros_f16, perm, A_f16, B_f16, s) != cudaSuccess)
         return LOPRO_ERR_CUDA;
     return LOPRO_OK;
@@ -292,6 +339,8 @@ static bool use_tall(const lopro_desc& d, int T) {
 // of the prefill kernel on small layers).
 static int small_batch_chunks(const lopro_desc& d, int T) {
     if (T <= kDecodeMaxT) return 0;
+    if (d.lowrank_format == LOPRO_LOWRANK_FP8)  // served by the small-batch kernels only: always chunks
+        return (prologue_supported(d, kDecodeMaxT) && stream_supported(d, kDecodeMaxT)) ? (T + kDecodeMaxT - 1) / kDecodeMaxT : 0;
     if (option(LOPRO_OPT_NO_CHUNKS) == 1) return 0;
     if (!prefill_supported(d, T)) return 0;  // keep the general path's behaviour where there is no prefill kernel
     const int chunks = (T + kDecodeMaxT - 1) / kDecodeMaxT;
@@ -310,8 +359,15 @@ static int rowblock_pre_launches(const lopro_desc& d, int T) {
     return 2 + (d.rank > 0 ? 1 : 0);
 }
 
+// The FP8 low-rank record is served by the prologue + small-batch kernels of the fragment layout.
+static bool lr8_unsupported(const lopro_desc& d) {
+    return d.lowrank_format == LOPRO_LOWRANK_FP8 &&
+           (d.layout != LOPRO_LAYOUT_FRAGMENT || !prologue_supported(d, 1) || !stream_supported(d, kDecodeMaxT));
+}
+
 int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launches) {
     if (!desc || check_desc(*desc) != LOPRO_OK || desc->layout == LOPRO_LAYOUT_CANONICAL || T < 1) return 0;
+    if (lr8_unsupported(*desc)) return 0;
     if (desc->layout == LOPRO_LAYOUT_ROWBLOCK) {
         if (!rowblock_supported(*desc)) return 0;
         if (launches) *launches = rowblock_pre_launches(*desc, T) + (T <= 16 ? 1 : (T + 31) / 32);
@@ -344,6 +400,7 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     if (st != LOPRO_OK) return st;
     if (desc->layout == LOPRO_LAYOUT_CANONICAL) return LOPRO_ERR_UNSUPPORTED;
     if (desc->layout == LOPRO_LAYOUT_ROWBLOCK && !rowblock_supported(*desc)) return LOPRO_ERR_UNSUPPORTED;
+    if (lr8_unsupported(*desc)) return LOPRO_ERR_UNSUPPORTED;
     if (T < 0 || (out_dtype != LOPRO_OUT_BF16 && out_dtype != LOPRO_OUT_F32)) return LOPRO_ERR_INVALID_ARG;
     if (T == 0) return LOPRO_OK;
     if (!packed || !x_bf16 || !y || !workspace) return LOPRO_ERR_INVALID_ARG;
@@ -364,6 +421,12 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     __nv_bfloat16* xrot = (__nv_bfloat16*)(ws + W.off_xrot);
     float* s64 = (float*)(ws + W.off_s64);
     int* status = (int*)(ws + W.off_status);
+    Lr8Args lr8 = {};
+    if (desc->lowrank_format == LOPRO_LOWRANK_FP8) {
+        lr8.V = blob + L.off[LOPRO_SEC_B];
+        lr8.sigma = (const __half*)(blob + L.off[LOPRO_SEC_SIGMA]);
+        lr8.svec = (const __half*)(blob + L.off[LOPRO_SEC_S]);
+    }
     if (desc->layout == LOPRO_LAYOUT_ROWBLOCK) {
         // operand image (one launch where the prologue kernel takes the descriptor), then one tcgen05 launch per
         // group of up to 32 tokens
@@ -393,7 +456,7 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
         // one prologue for all tokens, then chunks of kDecodeMaxT tokens through the small-batch kernels, each
         // reading its tokens' records of the activation image and rows of t
         if (launch_prologue(*desc, perm, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot,
-                            (__half*)(ws + W.off_t), W.t_pad, status, T, s) != cudaSuccess)
+                            (__half*)(ws + W.off_t), W.t_pad, status, T, s, nullptr, nullptr, &lr8) != cudaSuccess)
             return LOPRO_ERR_CUDA;
         const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;
         for (int c = 0; c < chunks; ++c) {
@@ -408,7 +471,7 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     if (prologue_supported(*desc, T) && stream_supported(*desc, T)) {
         // small batch: prologue + streaming kernel, chained by programmatic launches
         if (launch_prologue(*desc, perm, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot,
-                            (__half*)(ws + W.off_t), W.t_pad, status, T, s) != cudaSuccess)
+                            (__half*)(ws + W.off_t), W.t_pad, status, T, s, nullptr, nullptr, &lr8) != cudaSuccess)
             return LOPRO_ERR_CUDA;
         const cudaError_t e = use_tall(*desc, T) ? launch_tall(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s)
                                                  : launch_stream(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s);
@@ -457,7 +520,8 @@ static bool group_shares_launches(int32_t n, const lopro_desc* const* descs, int
     for (int i = 0; i < n; ++i) {
         const lopro_desc& d = *descs[i];
         if (d.d_in != d0.d_in || d.bits != d0.bits || d.group_size != d0.group_size || d.block_size != d0.block_size ||
-            d.identity_cols != d0.identity_cols || d.rank != d0.rank || d.layout != d0.layout)
+            d.identity_cols != d0.identity_cols || d.rank != d0.rank || d.layout != d0.layout ||
+            d.lowrank_format != LOPRO_LOWRANK_FOLDED_F16)
             return false;
         if (!prologue_supported(d, T) || !stream_supported(d, T) || use_tall(d, T)) return false;
     }

@@ -34,6 +34,7 @@ enum : uint32_t {
     kInvalidCode = 4u,
     kInvalidScale = 8u,
     kInvalidZero = 16u,
+    kInvalidLowrank = 32u,  // FP8 record: NaN pattern in U or V, non-finite Sigma, non-finite or zero s
 };
 
 struct BlobLayout {
@@ -123,6 +124,11 @@ cudaError_t launch_validate(const lopro_desc& d, const uint8_t* codes, const uin
 cudaError_t launch_pack(const lopro_desc& d, const uint8_t* codes, const uint16_t* scales, const uint16_t* zeros,
                         const int32_t* perm, const uint16_t* A, const uint16_t* B, void* blob,
                         const BlobLayout& L, cudaStream_t s);
+// FP8 low-rank record: validation (flags in the header) and the copy into / out of the blob.
+cudaError_t launch_pack_lr8(const lopro_desc& d, const uint8_t* U, const uint8_t* V, const uint16_t* sigma, const uint16_t* svec,
+                            void* blob, const BlobLayout& L, cudaStream_t s);
+cudaError_t launch_unpack_lr8(const lopro_desc& d, const void* blob, const BlobLayout& L, uint8_t* U, uint8_t* V,
+                              uint16_t* sigma, uint16_t* svec, cudaStream_t s);
 cudaError_t launch_unpack(const lopro_desc& d, const void* blob, const BlobLayout& L, uint8_t* codes,
                           uint32_t* words, uint16_t* scales, uint16_t* zeros, int32_t* perm, uint16_t* A,
                           uint16_t* B, cudaStream_t s);
@@ -141,10 +147,16 @@ struct PrologueSiblings {  // siblings 1 .. n of a grouped prologue (sibling 0 t
     unsigned char* act[kMaxSiblings - 1];
     __half* t[kMaxSiblings - 1];
 };
+// FP8 low-rank record: t = Sigma (V (x / s)) instead of t = B x (V null: folded fp16 format).
+struct Lr8Args {
+    const uint8_t* V;      // e4m3 [r_pad][n]
+    const __half* sigma;   // [r_pad]
+    const __half* svec;    // [n]
+};
 cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
                             const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, __half* t, int t_pad,
                             int* status, int T, cudaStream_t s, const ImageOut* img = nullptr,
-                            const PrologueSiblings* siblings = nullptr);
+                            const PrologueSiblings* siblings = nullptr, const Lr8Args* lr8 = nullptr);
 // Plain rotated activations, 64-column sums and t (the general path's outputs) -> operand image.
 cudaError_t launch_image_convert(const lopro_desc& d, const __nv_bfloat16* xrot, const float* s64, int s64_ld,
                                  const __half* t, int r_pad, const ImageOut& img, int T, cudaStream_t s);

@@ -185,6 +185,29 @@ __global__ void copy_padded_kernel(const uint16_t* __restrict__ src, uint16_t* _
     dst[r * dst_ld + c] = src[r * src_ld + c];
 }
 
+// byte matrices of the FP8 low-rank record, rank padded with zeros: U [m][r] <-> [m][r_pad], V [r][n] <-> [r_pad][n]
+__global__ void copy_padded_bytes_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, size_t rows, int cols,
+                                         int src_ld, int dst_ld) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * (size_t)cols) return;
+    const size_t r = idx / cols;
+    const int c = (int)(idx % cols);
+    dst[r * dst_ld + c] = src[r * src_ld + c];
+}
+
+// e4m3 has no infinities; S.1111.111 is NaN.  Sigma finite; s finite and non-zero (the forward divides by it).
+__global__ void validate_lr8_kernel(const uint8_t* __restrict__ U, size_t n_u, const uint8_t* __restrict__ V, size_t n_v,
+                                    const uint16_t* __restrict__ sigma, int r, const uint16_t* __restrict__ svec, int n,
+                                    uint32_t* __restrict__ invalid) {
+    const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (size_t i = tid; i < n_u; i += stride) bad |= (U[i] & 0x7Fu) == 0x7Fu;
+    for (size_t i = tid; i < n_v; i += stride) bad |= (V[i] & 0x7Fu) == 0x7Fu;
+    for (size_t i = tid; i < (size_t)r; i += stride) bad |= !f16_is_finite(sigma[i]);
+    for (size_t i = tid; i < (size_t)n; i += stride) bad |= !f16_is_finite(svec[i]) || (svec[i] & 0x7FFFu) == 0;
+    if (bad) atomicOr(invalid, kInvalidLowrank);
+}
+
 inline unsigned blocks_for(size_t n, int threads) { return (unsigned)((n + threads - 1) / threads); }
 
 }  // namespace
@@ -222,12 +245,40 @@ cudaError_t launch_pack(const lopro_desc& d, const uint8_t* codes, const uint16_
         (uint16_t*)scales, (uint16_t*)zeros, (uint32_t*)(base + L.off[LOPRO_SEC_SCALEZERO]), m, ng, d.layout, true);
     cudaError_t e = cudaMemcpyAsync(base + L.off[LOPRO_SEC_PERM], perm, (size_t)n * 4, cudaMemcpyDeviceToDevice, s);
     if (e != cudaSuccess) return e;
-    if (d.rank > 0) {
+    if (d.rank > 0 && A != nullptr && B != nullptr) {
         copy_padded_kernel<<<blocks_for((size_t)m * d.rank, 256), 256, 0, s>>>(
             A, (uint16_t*)(base + L.off[LOPRO_SEC_A]), (size_t)m, d.rank, d.rank, L.r_pad);
         copy_padded_kernel<<<blocks_for((size_t)d.rank * n, 256), 256, 0, s>>>(
             B, (uint16_t*)(base + L.off[LOPRO_SEC_B]), (size_t)d.rank, n, n, n);
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack_lr8(const lopro_desc& d, const uint8_t* U, const uint8_t* V, const uint16_t* sigma, const uint16_t* svec,
+                            void* blob, const BlobLayout& L, cudaStream_t s) {
+    uint8_t* base = (uint8_t*)blob;
+    const int m = d.d_out, n = d.d_in, r = d.rank;
+    validate_lr8_kernel<<<256, 256, 0, s>>>(U, (size_t)m * r, V, (size_t)r * n, sigma, r, svec, n, &((BlobHeader*)blob)->invalid);
+    copy_padded_bytes_kernel<<<blocks_for((size_t)m * r, 256), 256, 0, s>>>(U, base + L.off[LOPRO_SEC_A], (size_t)m, r, r, L.r_pad);
+    copy_padded_bytes_kernel<<<blocks_for((size_t)r * n, 256), 256, 0, s>>>(V, base + L.off[LOPRO_SEC_B], (size_t)r, n, n, n);
+    cudaError_t e = cudaMemcpyAsync(base + L.off[LOPRO_SEC_SIGMA], sigma, (size_t)r * 2, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return e;
+    e = cudaMemcpyAsync(base + L.off[LOPRO_SEC_S], svec, (size_t)n * 2, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack_lr8(const lopro_desc& d, const void* blob, const BlobLayout& L, uint8_t* U, uint8_t* V,
+                              uint16_t* sigma, uint16_t* svec, cudaStream_t s) {
+    const uint8_t* base = (const uint8_t*)blob;
+    const int m = d.d_out, n = d.d_in, r = d.rank;
+    if (U) copy_padded_bytes_kernel<<<blocks_for((size_t)m * r, 256), 256, 0, s>>>(base + L.off[LOPRO_SEC_A], U, (size_t)m, r, L.r_pad, r);
+    if (V) copy_padded_bytes_kernel<<<blocks_for((size_t)r * n, 256), 256, 0, s>>>(base + L.off[LOPRO_SEC_B], V, (size_t)r, n, n, n);
+    cudaError_t e = cudaSuccess;
+    if (sigma) e = cudaMemcpyAsync(sigma, base + L.off[LOPRO_SEC_SIGMA], (size_t)r * 2, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return e;
+    if (svec) e = cudaMemcpyAsync(svec, base + L.off[LOPRO_SEC_S], (size_t)n * 2, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
@@ -249,7 +300,7 @@ cudaError_t launch_unpack(const lopro_desc& d, const void* blob, const BlobLayou
         cudaError_t e = cudaMemcpyAsync(perm, base + L.off[LOPRO_SEC_PERM], (size_t)n * 4, cudaMemcpyDeviceToDevice, s);
         if (e != cudaSuccess) return e;
     }
-    if (d.rank > 0) {
+    if (d.rank > 0 && d.lowrank_format == LOPRO_LOWRANK_FOLDED_F16) {
         if (A)
             copy_padded_kernel<<<blocks_for((size_t)m * d.rank, 256), 256, 0, s>>>(
                 (const uint16_t*)(base + L.off[LOPRO_SEC_A]), A, (size_t)m, d.rank, L.r_pad, d.rank);

@@ -90,6 +90,32 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
                  : "r"(addr));
 }
 
+// two fp8 e4m3 values (low byte first) -> two fp16 values (exact)
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint16_t v) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(d) : "h"(v));
+    return d;
+}
+
+// A-operand registers (m16n8k16, fp16) of the 16 x 16 piece at columns jj of a 16-row tile of the up-projection
+// factor held in shared memory, rows r_pad entries apart: fp16 entries (A = U Sigma), or fp8 e4m3 entries (U of the
+// FP8 low-rank record) converted exactly to fp16.
+__device__ __forceinline__ void load_up_fragment(uint32_t (&a)[4], const unsigned char* tile, int r_pad, int gq, int tg, int jj,
+                                                 bool lr8) {
+    if (!lr8) {
+        const __half* as = reinterpret_cast<const __half*>(tile);
+        a[0] = *reinterpret_cast<const uint32_t*>(as + gq * r_pad + jj + 2 * tg);
+        a[1] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * r_pad + jj + 2 * tg);
+        a[2] = *reinterpret_cast<const uint32_t*>(as + gq * r_pad + jj + 8 + 2 * tg);
+        a[3] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * r_pad + jj + 8 + 2 * tg);
+    } else {
+        a[0] = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t*>(tile + gq * r_pad + jj + 2 * tg));
+        a[1] = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t*>(tile + (gq + 8) * r_pad + jj + 2 * tg));
+        a[2] = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t*>(tile + gq * r_pad + jj + 8 + 2 * tg));
+        a[3] = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t*>(tile + (gq + 8) * r_pad + jj + 8 + 2 * tg));
+    }
+}
+
 constexpr uint32_t kMagic128 = 0x43004300u;  // two bf16 128.0 (ulp 1): 128.0 | c == 128 + c
 
 // (a & mask) | magic in ONE logic instruction (truth table 0xEA), both constants held in registers --

@@ -4,6 +4,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 #include "rotate_body.cuh"
 
 namespace lopro {
@@ -171,6 +172,67 @@ __device__ __forceinline__ void lowrank_row(const __nv_bfloat16* __restrict__ x,
     }
 }
 
+// The same row job for the FP8 low-rank record (U, V, Sigma, s) that Algorithm 1 saves:
+// t[token][j] = sigma[j] * sum_k V[j][k] * (x[token][k] / s[k]), V in fp8 e4m3 (exact in fp32), the quotient as
+// x * (1 / s) in fp32, fp32 accumulation, one rounding to fp16.
+template <int TPR>
+__device__ __forceinline__ void lowrank_row_lr8(const __nv_bfloat16* __restrict__ x, int64_t ldx, const Lr8Args lr8,
+                                                __half* __restrict__ t, int n, int r_pad, int T, int rb, int tok0) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ float part[8][TPR];
+    const int j = rb % r_pad, tq = tok0 + TPR * (rb / r_pad);
+    const uint8_t* vrow = lr8.V + (size_t)j * n;
+    if ((tid & 15) == 0 && tid * 8 < n) prefetch_l2(vrow + tid * 8);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    float acc[TPR];
+#pragma unroll
+    for (int tk = 0; tk < TPR; ++tk) acc[tk] = 0.0f;
+    for (int k = tid * 8; k < n; k += 2048) {
+        const uint2 vw = __ldg(reinterpret_cast<const uint2*>(vrow + k));
+        const uint4 sw = __ldg(reinterpret_cast<const uint4*>(lr8.svec + k));
+        float vf[8], rs[8];
+        const uint32_t vv[2] = {vw.x, vw.y};
+        const __half2* sh = reinterpret_cast<const __half2*>(&sw);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t h2 = e4m3x2_to_f16x2((uint16_t)(vv[i >> 1] >> (16 * (i & 1))));
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+            const float2 sf = __half22float2(sh[i]);
+            vf[2 * i] = f.x;
+            vf[2 * i + 1] = f.y;
+            rs[2 * i] = __frcp_rn(sf.x);
+            rs[2 * i + 1] = __frcp_rn(sf.y);
+        }
+#pragma unroll
+        for (int tk = 0; tk < TPR; ++tk) {
+            if (tq + tk < T) {
+                const uint4 xw = __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tq + tk) * ldx + k));
+                const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xw);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 f = __bfloat1622float2(xh[i]);
+                    acc[tk] = fmaf(vf[2 * i], f.x * rs[2 * i], acc[tk]);
+                    acc[tk] = fmaf(vf[2 * i + 1], f.y * rs[2 * i + 1], acc[tk]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int tk = 0; tk < TPR; ++tk) {
+        float v = acc[tk];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+        if (lane == 0) part[warp][tk] = v;
+    }
+    __syncthreads();
+    if (tid < TPR) {
+        float v = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += part[w][tid];
+        if (tq + tid < T) t[(size_t)(tq + tid) * r_pad + j] = __float2half_rn(v * __half2float(lr8.sigma[j]));
+    }
+}
+
 // Tail of the prologue's rotation for one (token, chunk of 256 output columns) pair of a warp: v holds the 8
 // gathered entries of the lane.  Register and shuffle butterflies, rounding to bf16, and the store of the entries
 // and of their 64-column sums into the record of (stage, token) in the activation image.
@@ -257,7 +319,7 @@ __global__ void __launch_bounds__(256)
 prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm0,
                 const __half* __restrict__ B0, unsigned char* __restrict__ act_image0, __half* __restrict__ t0,
                 int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T,
-                int tpr, const ImageOut img, const PrologueSiblings sibs) {
+                int tpr, const ImageOut img, const PrologueSiblings sibs, const Lr8Args lr8) {
     // sibling layers (grid z): the same x, each layer its own permutation, B and outputs
     const int32_t* __restrict__ perm = perm0;
     const __half* __restrict__ B = B0;
@@ -281,6 +343,13 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
     const int nrow = (int)gridDim.x - (STAGED ? live * ((nchunks + 7) >> 3) : nchunks);
     if ((int)blockIdx.x < nrow) {
         const int rb = (int)blockIdx.x;
+        if (lr8.V != nullptr) {
+            if (tpr == 8) lowrank_row_lr8<8>(x, ldx, lr8, t, n, r_pad, T, rb, tok0);
+            else if (tpr == 4) lowrank_row_lr8<4>(x, ldx, lr8, t, n, r_pad, T, rb, tok0);
+            else if (tpr == 2) lowrank_row_lr8<2>(x, ldx, lr8, t, n, r_pad, T, rb, tok0);
+            else lowrank_row_lr8<1>(x, ldx, lr8, t, n, r_pad, T, rb, tok0);
+            return;
+        }
         if (tpr == 8) lowrank_row<8>(x, ldx, B, t, n, r_pad, T, rb, tok0, img);
         else if (tpr == 4) lowrank_row<4>(x, ldx, B, t, n, r_pad, T, rb, tok0, img);
         else if (tpr == 2) lowrank_row<2>(x, ldx, B, t, n, r_pad, T, rb, tok0, img);
@@ -403,12 +472,15 @@ bool prologue_supported(const lopro_desc& d, int T) {
 
 cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __half* B, int r_pad,
                             const __nv_bfloat16* x, int64_t ldx, unsigned char* act_image, __half* t, int t_pad,
-                            int* status, int T, cudaStream_t s, const ImageOut* img_out, const PrologueSiblings* siblings) {
+                            int* status, int T, cudaStream_t s, const ImageOut* img_out, const PrologueSiblings* siblings,
+                            const Lr8Args* lr8_args) {
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
     ImageOut img = {};
     if (img_out != nullptr) img = *img_out;
     PrologueSiblings sibs = {};
     if (siblings != nullptr) sibs = *siblings;
+    Lr8Args lr8 = {};
+    if (lr8_args != nullptr) lr8 = *lr8_args;
     cudaLaunchConfig_t cfg = {};
     // tokens per row CTA: as few as it takes to fill the SMs
     const int live = T < 8 ? T : 8;
@@ -440,9 +512,9 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
     cfg.numAttrs = 1;
     const int rp = d.rank > 0 ? r_pad : 0;
     return staged ? cudaLaunchKernelEx(&cfg, prologue_kernel<true>, x, ldx, perm, B, act_image, t, status, d.d_in,
-                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, sibs)
+                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, sibs, lr8)
                   : cudaLaunchKernelEx(&cfg, prologue_kernel<false>, x, ldx, perm, B, act_image, t, status, d.d_in,
-                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, sibs);
+                                       d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, sibs, lr8);
 }
 
 cudaError_t launch_lowrank_down(const lopro_desc& d, const __half* B, int r_pad, const __nv_bfloat16* x,

@@ -47,6 +47,7 @@ struct StreamParams {
     int nsteps, gshift, ng, r_pad;
     int n_stages;  // ring depth
     int total_stages;
+    int lr8;       // the up-projection factor is fp8 e4m3 (U of the FP8 low-rank record), one byte per entry
     // shared-memory layout (bytes from the dynamic base)
     int off_sz, off_a, off_t, off_ring, stage_bytes, off_stage_x;
 };
@@ -154,14 +155,11 @@ stream_kernel(const StreamParams p_in, const StreamSiblings sibs) {
     // low-rank up-projection A t: warp r starts the sums of row tile r with it (fp16 tensor-core product
     // into the fp32 sums), before the first stage, so that nothing but the reduction follows the last one
     auto lowrank_up = [&](float (&acc)[NT][4], int r) {
-        const __half* as = reinterpret_cast<const __half*>(smem + p.off_a) + (size_t)r * 16 * p.r_pad;
+        const unsigned char* as = smem + p.off_a + (size_t)r * 16 * p.r_pad * (p.lr8 ? 1 : 2);
         const __half* ts = reinterpret_cast<const __half*>(smem + p.off_t);
         for (int jj = 0; jj < p.r_pad; jj += 16) {
             uint32_t a[4];
-            a[0] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 2 * tg);
-            a[1] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 2 * tg);
-            a[2] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 8 + 2 * tg);
-            a[3] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 8 + 2 * tg);
+            load_up_fragment(a, as, p.r_pad, gq, tg, jj, p.lr8 != 0);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const __half* trow = ts + (nt * 8 + gq) * p.r_pad + jj + 2 * tg;
@@ -175,10 +173,12 @@ stream_kernel(const StreamParams p_in, const StreamSiblings sibs) {
         if (lane == 0) {
             // layer data: (scale, zero) pairs and rows of A of the live row tiles, then the first stages of codes
             const uint32_t sz_bytes = (uint32_t)(n_rt * p.ng * 64);
-            const uint32_t a_bytes = (uint32_t)(n_rt * 16 * p.r_pad * 2);
+            const uint32_t a_bytes = (uint32_t)(n_rt * 16 * p.r_pad * (p.lr8 ? 1 : 2));
             mbar_expect_tx(cbar, sz_bytes + a_bytes);
             bulk_g2s(smem0 + p.off_sz, p.sz + (size_t)rt0 * p.ng * 16, sz_bytes, cbar);
-            if (a_bytes) bulk_g2s(smem0 + p.off_a, p.A + (size_t)rt0 * 16 * p.r_pad, a_bytes, cbar);
+            if (a_bytes)
+                bulk_g2s(smem0 + p.off_a, reinterpret_cast<const unsigned char*>(p.A) + (size_t)rt0 * 16 * p.r_pad * (p.lr8 ? 1 : 2),
+                         a_bytes, cbar);
             for (int s = 0; s < first; ++s) issue_w(s, s);
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -390,10 +390,12 @@ stream_wide_kernel(const StreamParams p_in, const StreamSiblings sibs) {
     if (tid == 0) {
         // layer data: (scale, zero) pairs and rows of A of the live row tiles, the codes of every stage
         const uint32_t sz_bytes = (uint32_t)(n_rt * p.ng * 64);
-        const uint32_t a_bytes = (uint32_t)(n_rt * 16 * p.r_pad * 2);
+        const uint32_t a_bytes = (uint32_t)(n_rt * 16 * p.r_pad * (p.lr8 ? 1 : 2));
         mbar_expect_tx(cbar, sz_bytes + a_bytes);
         bulk_g2s(smem0 + p.off_sz, p.sz + (size_t)rt0 * p.ng * 16, sz_bytes, cbar);
-        if (a_bytes) bulk_g2s(smem0 + p.off_a, p.A + (size_t)rt0 * 16 * p.r_pad, a_bytes, cbar);
+        if (a_bytes)
+            bulk_g2s(smem0 + p.off_a, reinterpret_cast<const unsigned char*>(p.A) + (size_t)rt0 * 16 * p.r_pad * (p.lr8 ? 1 : 2),
+                     a_bytes, cbar);
         for (int s = 0; s < p.total_stages; ++s) {
             const uint32_t bytes = (uint32_t)(steps_of(s) * kStepBytes);
             mbar_expect_tx(full(s), bytes * (uint32_t)n_rt);
@@ -437,14 +439,11 @@ stream_wide_kernel(const StreamParams p_in, const StreamSiblings sibs) {
         // low-rank term A t of row tile r starts the sums of its step-0 warp
         if (!mbar_wait(tbar, 0)) timed_out = true;
         if (live) {
-            const __half* as = reinterpret_cast<const __half*>(smem + p.off_a) + (size_t)r * 16 * p.r_pad;
+            const unsigned char* as = smem + p.off_a + (size_t)r * 16 * p.r_pad * (p.lr8 ? 1 : 2);
             const __half* ts = reinterpret_cast<const __half*>(smem + p.off_t);
             for (int jj = 0; jj < p.r_pad; jj += 16) {
                 uint32_t a[4];
-                a[0] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 2 * tg);
-                a[1] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 2 * tg);
-                a[2] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 8 + 2 * tg);
-                a[3] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 8 + 2 * tg);
+                load_up_fragment(a, as, p.r_pad, gq, tg, jj, p.lr8 != 0);
                 const __half* trow = ts + gq * p.r_pad + jj + 2 * tg;
                 mma_f16(yacc, a, *reinterpret_cast<const uint32_t*>(trow), *reinterpret_cast<const uint32_t*>(trow + 8));
             }
@@ -658,6 +657,7 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
     p.gshift = gshift;
     p.ng = d.d_in / d.group_size;
     p.r_pad = d.rank > 0 ? L.r_pad : 0;
+    p.lr8 = d.lowrank_format == LOPRO_LOWRANK_FP8 ? 1 : 0;
     p.n_stages = pl.n_stages;
     p.total_stages = pl.total_stages;
     p.off_sz = pl.off_sz;

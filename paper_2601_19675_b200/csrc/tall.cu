@@ -55,6 +55,7 @@ struct TallParams {
     int gt;            // 16-row tiles per group: 4 or 2
     int n_stages;      // ring depth (<= stages per group)
     int total_stages;  // stages per group = ceil(nsteps / 16)
+    int lr8;           // the up-projection factor is fp8 e4m3 (U of the FP8 low-rank record), one byte per entry
     // shared-memory layout (bytes from the dynamic base)
     int off_a, a_bytes, off_t, off_red, off_ring, stage_bytes, off_stage_sz, off_stage_x;
 };
@@ -207,9 +208,10 @@ tall_kernel(const TallParams p) {
                          full(slot));
             }
             if (s == 0 && p.r_pad > 0) {
-                const uint32_t b_a = (uint32_t)(n_rt * 16 * p.r_pad * 2);
+                const uint32_t b_a = (uint32_t)(n_rt * 16 * p.r_pad * (p.lr8 ? 1 : 2));
                 mbar_expect_tx(afull(gi & 1), b_a);
-                bulk_g2s(smem0 + p.off_a + (gi & 1) * p.a_bytes, p.A + (size_t)tile0 * 16 * p.r_pad, b_a, afull(gi & 1));
+                bulk_g2s(smem0 + p.off_a + (gi & 1) * p.a_bytes,
+                         reinterpret_cast<const unsigned char*>(p.A) + (size_t)tile0 * 16 * p.r_pad * (p.lr8 ? 1 : 2), b_a, afull(gi & 1));
             }
         };
         // activations of the stage: the records of the live tokens, one contiguous piece of the image
@@ -284,14 +286,11 @@ tall_kernel(const TallParams p) {
                 if (lane == 0) atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
             }
             if (active) {
-                const __half* as = reinterpret_cast<const __half*>(smem + p.off_a + (gi & 1) * p.a_bytes) + (size_t)r * 16 * p.r_pad;
+                const unsigned char* as = smem + p.off_a + (gi & 1) * p.a_bytes + (size_t)r * 16 * p.r_pad * (p.lr8 ? 1 : 2);
                 const __half* ts = reinterpret_cast<const __half*>(smem + p.off_t);
                 for (int jj = 0; jj < p.r_pad; jj += 16) {
                     uint32_t a[4];
-                    a[0] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 2 * tg);
-                    a[1] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 2 * tg);
-                    a[2] = *reinterpret_cast<const uint32_t*>(as + gq * p.r_pad + jj + 8 + 2 * tg);
-                    a[3] = *reinterpret_cast<const uint32_t*>(as + (gq + 8) * p.r_pad + jj + 8 + 2 * tg);
+                    load_up_fragment(a, as, p.r_pad, gq, tg, jj, p.lr8 != 0);
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
                         const __half* trow = ts + (nt * 8 + gq) * p.r_pad + jj + 2 * tg;
@@ -464,6 +463,7 @@ cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayo
     p.gshift = gshift;
     p.ng = d.d_in / d.group_size;
     p.r_pad = d.rank > 0 ? L.r_pad : 0;
+    p.lr8 = d.lowrank_format == LOPRO_LOWRANK_FP8 ? 1 : 0;
     p.gt = pl.gt;
     p.n_stages = pl.n_stages;
     p.total_stages = pl.total_stages;

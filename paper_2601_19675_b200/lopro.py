@@ -18,20 +18,20 @@ LIB_PATH = os.environ.get("LOPRO_LIBRARY") or os.path.join(_HERE, "liblopro.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT, ERR_INVALID_DATA = range(7)
 OUT_BF16, OUT_F32 = 0, 1
 LAYOUT_CANONICAL, LAYOUT_FRAGMENT, LAYOUT_ROWBLOCK = 0, 1, 2
-SEC_HEADER, SEC_CODES, SEC_SCALEZERO, SEC_PERM, SEC_A, SEC_B = range(6)
+SEC_HEADER, SEC_CODES, SEC_SCALEZERO, SEC_PERM, SEC_A, SEC_B, SEC_SIGMA, SEC_S = range(8)
 
 # every symbol include/lopro.h declares
 SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packed_bytes", "lopro_packed_section",
            "lopro_workspace_bytes", "lopro_pack", "lopro_unpack", "lopro_rotate", "lopro_linear_fwd",
            "lopro_linear_fwd_path", "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc",
            "lopro_configure", "lopro_selftest_wait", "lopro_group_workspace_bytes", "lopro_linear_fwd_group_path",
-           "lopro_linear_fwd_group"]
+           "lopro_linear_fwd_group", "lopro_pack_lr8", "lopro_unpack_lr8"]
 
 
 class Desc(ctypes.Structure):
     _fields_ = [("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32), ("bits", ctypes.c_int32),
                 ("group_size", ctypes.c_int32), ("block_size", ctypes.c_int32), ("identity_cols", ctypes.c_int32),
-                ("rank", ctypes.c_int32), ("layout", ctypes.c_int32)]
+                ("rank", ctypes.c_int32), ("layout", ctypes.c_int32), ("lowrank_format", ctypes.c_int32)]
 
     def __repr__(self):
         return "Desc(" + ", ".join(f"{n}={getattr(self, n)}" for n, _ in self._fields_) + ")"
@@ -91,6 +91,10 @@ def lib():
         L.lopro_linear_fwd_group.restype = ctypes.c_int
         L.lopro_linear_fwd_group.argtypes = [i32, dpp, ctypes.POINTER(vp), vp, i64, ctypes.POINTER(vp), ctypes.POINTER(i64), i32,
                                              i32, vp, sz, vp]
+        L.lopro_pack_lr8.restype = ctypes.c_int
+        L.lopro_pack_lr8.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.lopro_unpack_lr8.restype = ctypes.c_int
+        L.lopro_unpack_lr8.argtypes = [dp, vp, vp, vp, vp, vp, vp]
         L.lopro_configure.restype = ctypes.c_int
         L.lopro_configure.argtypes = [i32, i32]
         L.lopro_selftest_wait.restype = ctypes.c_int
@@ -134,11 +138,15 @@ def status_str(status):
     return lib().lopro_status_str(int(status)).decode()
 
 
-def make_desc(d_in, d_out, bits, group_size, block_size, identity_cols=None, rank=0, layout=LAYOUT_FRAGMENT):
+LOWRANK_FOLDED_F16, LOWRANK_FP8 = 0, 1
+
+
+def make_desc(d_in, d_out, bits, group_size, block_size, identity_cols=None, rank=0, layout=LAYOUT_FRAGMENT,
+              lowrank_format=LOWRANK_FOLDED_F16):
     """Descriptor of one layer; identity_cols defaults to block_size (the paper's b_I = b_H)."""
     if identity_cols is None:
         identity_cols = block_size
-    return Desc(d_in, d_out, bits, group_size, block_size, identity_cols, rank, layout)
+    return Desc(d_in, d_out, bits, group_size, block_size, identity_cols, rank, layout, lowrank_format)
 
 
 def check_desc(desc):
@@ -208,6 +216,31 @@ def pack(desc, codes, scales_f16, zeros_f16, perm, A_f16=None, B_f16=None, out=N
     return out
 
 
+def pack_lr8(desc, codes, scales_f16, zeros_f16, perm, U_e4m3, V_e4m3, sigma_f16, s_f16, out=None):
+    """lopro_pack_lr8: the record (W_q, U, V, Sigma, p, s) with U, V as fp8 e4m3 bytes, Sigma and s as fp16 bit patterns."""
+    nbytes = packed_bytes(desc)
+    if nbytes == 0:
+        raise LoproError(check_desc(desc) or ERR_INVALID_ARG, "lopro_packed_bytes")
+    if out is None:
+        out = torch.empty(nbytes, dtype=torch.uint8, device=codes.device)
+    st = lib().lopro_pack_lr8(ctypes.byref(desc), _ptr(_dev(codes, 1)), _ptr(_dev(scales_f16, 2)), _ptr(_dev(zeros_f16, 2)),
+                              _ptr(_dev(perm, 4)), _ptr(_dev(U_e4m3, 1)), _ptr(_dev(V_e4m3, 1)), _ptr(_dev(sigma_f16, 2)),
+                              _ptr(_dev(s_f16, 2)), _ptr(out), out.numel(), _stream())
+    _check(st, "lopro_pack_lr8")
+    return out
+
+
+def unpack_lr8(desc, packed):
+    """lopro_unpack_lr8: dict(U, V uint8; sigma, s int16 bit patterns) of freshly allocated device tensors."""
+    m, n, r, dev = desc.d_out, desc.d_in, desc.rank, packed.device
+    out = dict(U=torch.empty((m, r), dtype=torch.uint8, device=dev), V=torch.empty((r, n), dtype=torch.uint8, device=dev),
+               sigma=torch.empty((r,), dtype=torch.int16, device=dev), s=torch.empty((n,), dtype=torch.int16, device=dev))
+    st = lib().lopro_unpack_lr8(ctypes.byref(desc), _ptr(packed), _ptr(out["U"]), _ptr(out["V"]), _ptr(out["sigma"]),
+                                _ptr(out["s"]), _stream())
+    _check(st, "lopro_unpack_lr8")
+    return out
+
+
 def unpack(desc, packed, want=("codes", "words", "scales", "zeros", "perm", "A", "B")):
     """lopro_unpack: returns a dict of freshly allocated device tensors (16-bit floats as int16 bit patterns)."""
     m, n, g, r = desc.d_out, desc.d_in, desc.group_size, desc.rank
@@ -223,9 +256,9 @@ def unpack(desc, packed, want=("codes", "words", "scales", "zeros", "perm", "A",
         out["zeros"] = torch.empty((m, n // g), dtype=torch.int16, device=dev)
     if "perm" in want:
         out["perm"] = torch.empty((n,), dtype=torch.int32, device=dev)
-    if "A" in want and r > 0:
+    if "A" in want and r > 0 and desc.lowrank_format == LOWRANK_FOLDED_F16:
         out["A"] = torch.empty((m, r), dtype=torch.int16, device=dev)
-    if "B" in want and r > 0:
+    if "B" in want and r > 0 and desc.lowrank_format == LOWRANK_FOLDED_F16:
         out["B"] = torch.empty((r, n), dtype=torch.int16, device=dev)
     st = lib().lopro_unpack(ctypes.byref(desc), _ptr(packed), _ptr(out.get("codes")), _ptr(out.get("words")),
                             _ptr(out.get("scales")), _ptr(out.get("zeros")), _ptr(out.get("perm")), _ptr(out.get("A")),

@@ -24,7 +24,7 @@ from __future__ import annotations
 import numpy as np
 
 _TAGS = {"x": 1, "perm": 2, "codes": 3, "scales": 4, "zeros": 5, "A": 6, "B": 7, "W": 8,
-         "outliers": 9, "sketch": 10}
+         "outliers": 9, "sketch": 10, "U": 11, "V": 12, "sigma": 13, "s": 14}
 
 CONFIGS = {
     "cfg1": dict(d_in=512, d_out=512, bits=4, group_size=128, block_size=64, identity_cols=64, rank=16, T=(16,)),
@@ -49,6 +49,32 @@ def f32_to_bf16_bits(a):
 
 def f32_to_f16_bits(a):
     return np.asarray(a, dtype=np.float32).astype(np.float16).view(np.uint16)
+
+
+def f32_to_e4m3_bits(a):
+    """float32 -> fp8 e4m3 bit patterns (finite-only format: 4 exponent bits, bias 7, 3 mantissa bits, subnormals
+    below 2^-6, largest value 448), round-to-nearest-even, magnitudes beyond 448 clamped (storage conversion)."""
+    a = np.asarray(a, dtype=np.float32).astype(np.float64)
+    sign = np.signbit(a).astype(np.uint8) << 7
+    mag = np.minimum(np.abs(a), 448.0)
+    m, e = np.frexp(mag)                                   # mag = m 2^e, 0.5 <= m < 1
+    exp = np.maximum(e - 1, -6)                            # exponent of the leading bit, clamped to the subnormal range
+    q = np.rint(np.ldexp(mag, 3 - exp)).astype(np.int64)   # significand in units of 2^(exp - 3): 8..16 (0..8 below 2^-6)
+    exp = np.where(q == 16, exp + 1, exp)                  # rounding carried into the next binade
+    q = np.where(q == 16, 8, q)
+    normal = q >= 8
+    bits = np.where(normal, ((exp + 7) << 3) | (q - 8), q)
+    return (bits.astype(np.uint8) | sign).astype(np.uint8)
+
+
+def lowrank_record(m, n, r, seed=0):
+    """The low-rank record (U, V, Sigma, s) in its stored formats: U [m][r], V [r][n] as e4m3 bit patterns of entries
+    ~ N(0, 1/dim) (unit-vector scale), Sigma [r] ~ U(0.05, 0.5) and the activation scale s [n] ~ U(0.5, 2) as fp16 bits."""
+    u = _rng(seed, "U").standard_normal((m, r), dtype=np.float32) / np.float32(np.sqrt(m))
+    v = _rng(seed, "V").standard_normal((r, n), dtype=np.float32) / np.float32(np.sqrt(n))
+    sigma = _rng(seed, "sigma").uniform(0.05, 0.5, size=r).astype(np.float32)
+    s = _rng(seed, "s").uniform(0.5, 2.0, size=n).astype(np.float32)
+    return dict(U=f32_to_e4m3_bits(u), V=f32_to_e4m3_bits(v), sigma=f32_to_f16_bits(sigma), s=f32_to_f16_bits(s))
 
 
 def activations(T, n, seed=0, outlier_frac=0.0, outlier_scale=20.0):

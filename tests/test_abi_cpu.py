@@ -64,14 +64,14 @@ def test_descriptor_domain(kw, expect):
 def test_blob_size_follows_eq13_accounting(m, n, bits, g, r):
     # Eq. 13 with this library's widths: d_q bits per code, 16-bit scale and 16-bit zero per group,
     # 16-bit factor entries (rank padded to 16), 32-bit permutation entries; plus a 256-byte header
-    # and at most 255 bytes of padding after each of the six sections.
+    # and at most 255 bytes of padding after each of the eight sections.
     d = lopro.make_desc(n, m, bits, g, 64, rank=r)
     r_pad = (r + 15) // 16 * 16
     payload_bits = m * n * (o.average_bits(m, n, bits, 32, g, r_pad, 16) - 2 * 32 / n - r_pad * 32 / (m * n)) + 32 * n
     nbytes = lopro.packed_bytes(d)
-    assert payload_bits / 8 + 256 <= nbytes <= payload_bits / 8 + 256 + 6 * 256
+    assert payload_bits / 8 + 256 <= nbytes <= payload_bits / 8 + 256 + 8 * 256
     total = 0
-    for sec in range(6):
+    for sec in range(8):
         off, sz = lopro.packed_section(d, sec)
         assert off % 256 == 0 and off >= total
         total = off + sz
@@ -144,3 +144,34 @@ def test_configure_rejects_unknown_options():
     assert lopro.linear_fwd_path(d, 8) == (lopro.PATH_WIDE, 2)
     assert L.lopro_selftest_wait(None, None) == lopro.ERR_INVALID_ARG
     assert L.lopro_selftest_wait(ctypes.c_void_p(0x1002), None) == lopro.ERR_INVALID_ARG
+
+
+def test_fp8_lowrank_record_reproduces_the_printed_storage_overhead(golden_dir):
+    # Appendix A.2 / rank-ablation table: U and V in fp8 (d_r = 8) at r = 16 cost about 0.05 bit per weight over the
+    # linears of a 7B model and 0.04 over a 13B model; the blob's A and B sections of the FP8 format hold exactly that
+    gold = {}
+    with open(os.path.join(golden_dir, "avg_bits.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                k, v, tol, _ = line.split()
+                gold[k] = (float(v), float(tol))
+    shapes = {"7b": [(4096, 4096)] * 4 + [(11008, 4096)] * 2 + [(4096, 11008)],
+              "13b": [(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)]}
+    for model, sh in shapes.items():
+        bits = weights = 0
+        for m, n in sh:
+            d = lopro.make_desc(n, m, 4, 128, 128, rank=16, lowrank_format=lopro.LOWRANK_FP8)
+            assert lopro.check_desc(d) == lopro.OK
+            bits += 8 * (lopro.packed_section(d, lopro.SEC_A)[1] + lopro.packed_section(d, lopro.SEC_B)[1])
+            weights += m * n
+            # Sigma and s: 16 bits per entry, as Eq. 13 counts them (r d_o and n d_o)
+            assert lopro.packed_section(d, lopro.SEC_SIGMA)[1] == 16 * 2 and lopro.packed_section(d, lopro.SEC_S)[1] == n * 2
+        val, tol = gold[f"rbit_{model}_r16"]
+        assert abs(bits / weights - val) <= tol
+    # the folded fp16 format has no such sections and twice the factor bytes
+    d16 = lopro.make_desc(4096, 4096, 4, 128, 128, rank=16)
+    d8 = lopro.make_desc(4096, 4096, 4, 128, 128, rank=16, lowrank_format=lopro.LOWRANK_FP8)
+    assert lopro.packed_section(d16, lopro.SEC_SIGMA)[1] == 0 and lopro.packed_section(d16, lopro.SEC_S)[1] == 0
+    assert lopro.packed_section(d16, lopro.SEC_A)[1] == 2 * lopro.packed_section(d8, lopro.SEC_A)[1]
+    assert lopro.check_desc(lopro.make_desc(4096, 4096, 4, 128, 128, rank=0, lowrank_format=lopro.LOWRANK_FP8)) == lopro.ERR_INVALID_ARG
+    assert lopro.check_desc(lopro.make_desc(4096, 4096, 4, 128, 128, rank=16, lowrank_format=3)) == lopro.ERR_INVALID_ARG

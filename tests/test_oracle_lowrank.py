@@ -132,3 +132,95 @@ def test_synth_generators_are_seeded_and_typed():
     assert L["codes"].max() == 15 and o.is_permutation(L["perm"])
     s = o.f16_bits_to_f64(L["scales"])
     assert s.min() >= 0.005 - 1e-5 and s.max() <= 0.02 + 1e-5
+
+
+def _unfolded_layer(seed, m=8, n=32, g=8, bits=3, b_i=8, b_h=8, r=3, T=4, dyadic=False):
+    rng = np.random.default_rng(seed)
+    codes = rng.integers(0, 2 ** bits, size=(m, n)).astype(np.uint8)
+    scales = o.round_f16(rng.uniform(0.01, 0.1, size=(m, n // g)))
+    zeros = o.round_f16(rng.uniform(0, 2 ** bits - 1, size=(m, n // g)))
+    perm = rng.permutation(n).astype(np.int32)
+    if dyadic:   # every product and sum below is exact in fp64
+        u = rng.integers(-8, 9, size=(m, r)) / 8.0
+        v = rng.integers(-8, 9, size=(r, n)) / 8.0
+        sigma = 2.0 ** rng.integers(-2, 3, size=r)
+        s = 2.0 ** rng.integers(-1, 2, size=n)
+        x = rng.integers(-16, 17, size=(T, n)) / 4.0
+    else:
+        u = o.round_e4m3(rng.standard_normal((m, r)) / np.sqrt(m))
+        v = o.round_e4m3(rng.standard_normal((r, n)) / np.sqrt(n))
+        sigma = o.round_f16(rng.uniform(0.5, 2.0, size=r))
+        s = o.round_f16(rng.uniform(0.5, 2.0, size=n))
+        x = o.round_bf16(rng.standard_normal((T, n)))
+    return dict(x=x, codes=codes, scales=scales, zeros=zeros, perm=perm, u=u, sigma=sigma, v=v, s=s, g=g, b_i=b_i, b_h=b_h)
+
+
+def _folded(L):
+    F = {k: L[k] for k in ("x", "codes", "scales", "zeros", "perm", "g", "b_i", "b_h")}
+    F["a"] = L["u"] * L["sigma"][None, :]             # W_L = U Sigma
+    F["b"] = L["v"] / L["s"][None, :]                 # W_R = V alpha^-1, alpha = diag(s)  (Eq. 4)
+    return F
+
+
+def test_unfolded_forward_equals_the_folded_one_on_exact_factors():
+    # with dyadic factors U Sigma and V / s are exact, so the stored form of Algorithm 1's record and the folded form
+    # of Eq. 4 describe the same numbers and every partial sum is exact: the low-rank parts must agree bit for bit
+    L = _unfolded_layer(5, dyadic=True)
+    F = _folded(L)
+    zero_q = dict(L, codes=np.zeros_like(L["codes"]), zeros=np.zeros_like(L["zeros"]))
+    zero_f = dict(F, codes=np.zeros_like(F["codes"]), zeros=np.zeros_like(F["zeros"]))
+    np.testing.assert_array_equal(o.forward_exact_unfolded(**zero_q), o.forward_exact(**zero_f))
+    np.testing.assert_allclose(o.forward_exact_unfolded(**L), o.forward_exact(**F), rtol=0, atol=1e-12)
+
+
+def test_unfolded_forward_equals_dense_eq8():
+    # Eq. 8 literally: W_eff = U Sigma V diag(s)^-1 + W^ Q^T P^T, y = W_eff x
+    L = _unfolded_layer(6)
+    n = L["x"].shape[1]
+    w_hat = o.dequant(L["codes"], L["scales"], L["zeros"], L["g"])
+    w_eff = L["u"] @ np.diag(L["sigma"]) @ L["v"] @ np.diag(1.0 / L["s"]) \
+        + w_hat @ o.q_matrix(n, L["b_i"], L["b_h"]).T @ o.p_matrix(L["perm"]).T
+    np.testing.assert_allclose(o.forward_exact_unfolded(**L), L["x"] @ w_eff.T, atol=1e-12)
+    # the mirrored variant differs only by its declared roundings, and with none left (rotation off, no t rounding)
+    # it is the fp32 rounding of the exact result
+    Li = dict(L, b_i=n)
+    np.testing.assert_array_equal(o.forward_mirrored_unfolded(**Li, round_t="none"),
+                                  o.forward_exact_unfolded(**Li).astype(np.float32).astype(np.float64))
+    e = o.max_rel_err(o.forward_mirrored_unfolded(**L), o.forward_exact_unfolded(**L))
+    assert 0.0 < e < 2e-2
+
+
+def test_e4m3_bit_patterns_round_trip_and_match_the_library_cast():
+    import torch
+    allbits = np.arange(256, dtype=np.uint8)
+    finite = allbits[(allbits & 0x7F) != 0x7F]                       # 0x7F / 0xFF are NaN in the finite-only format
+    vals = o.e4m3_bits_to_f64(finite)
+    ref = torch.from_numpy(finite.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    np.testing.assert_array_equal(vals, ref)
+    back = o.f64_to_e4m3_bits(vals)
+    np.testing.assert_array_equal(back & 0x7F, finite & 0x7F)        # (the sign of zero aside, covered below)
+    np.testing.assert_array_equal(o.e4m3_bits_to_f64(back), vals)
+    np.testing.assert_array_equal(o.round_e4m3(vals), vals)          # representable values are fixed points
+
+
+def test_unfolded_quantizer_absorbs_the_fp8_rounding_in_the_residual():
+    # Algorithm 1 with the casts of Sec. 3.3: the quantized part sees R = W - U Sigma V / s with the STORED factors,
+    # so the layer reproduces W up to the RTN grid alone (same bound as with exact factors)
+    rng = np.random.default_rng(8)
+    m, n, r, g, bits = 32, 64, 4, 16, 4
+    w = rng.standard_normal((m, n)) * 0.05
+    s = rng.uniform(0.5, 2.0, size=n)
+    perm = rng.permutation(n).astype(np.int32)
+    q = o.lopro_quantize_unfolded(w, perm, 16, 16, r, bits, g, s, it=4, sketches=rng.standard_normal((r, n)))
+    np.testing.assert_array_equal(o.round_e4m3(q["U"]), q["U"])
+    np.testing.assert_array_equal(o.round_e4m3(q["V"]), q["V"])
+    np.testing.assert_array_equal(o.round_f16(q["sigma"]), q["sigma"])
+    x = np.eye(n)
+    w_back = o.forward_exact_unfolded(x, q["codes"], q["scales"], q["zeros"], perm, q["U"], q["sigma"], q["V"], q["s"], g, 16, 16).T
+    resid = w - (q["U"] * q["sigma"][None, :]) @ (q["V"] / q["s"][None, :])
+    rp = o.partial_block_rotate(o.permute_columns(resid, perm), 16, 16)
+    step = np.repeat(q["scales"], g, axis=1)
+    err_rot = o.partial_block_rotate(o.permute_columns(w - w_back, perm), 16, 16)   # error in the rotated basis
+    assert np.all(np.abs(err_rot) <= 0.5 * step + 1e-3 * np.abs(rp).max())
+    # and the low-rank part carries most of the weight of the leading directions: the residual is smaller than W
+    assert np.linalg.norm(resid) < np.linalg.norm(w)
