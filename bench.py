@@ -84,10 +84,12 @@ METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
 
 
-def algorithmic_bytes(c, T):
-    """Bytes the method must move per layer forward: codes, (scale, zero) pairs, A and B, perm, x in, y out."""
+def algorithmic_bytes(c, T, lowrank="f16"):
+    """Bytes the method must move per layer forward: codes, (scale, zero) pairs, the low-rank factors (fp16 A and B,
+    or fp8 U and V with fp16 Sigma and s), perm, x in, y out."""
     m, n, q, g, r = c["d_out"], c["d_in"], c["bits"], c["group_size"], c["rank"]
-    return m * n * q // 8 + m * (n // g) * 4 + (m * r + r * n) * 2 + n * 4 + T * (n + m) * 2
+    factors = (m * r + r * n) * 2 if lowrank == "f16" else (m * r + r * n) + 2 * r + 2 * n
+    return m * n * q // 8 + m * (n // g) * 4 + factors + n * 4 + T * (n + m) * 2
 
 
 def algorithmic_flops(c, T):
@@ -375,8 +377,9 @@ class Workload:
             return
         c = synth.CONFIGS[cfg]
         self.c = c
+        fp8 = args.lowrank == "fp8"
         d = lopro.make_desc(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["block_size"], c["identity_cols"], c["rank"],
-                            layout=layout)
+                            layout=layout, lowrank_format=lopro.LOWRANK_FP8 if fp8 else lopro.LOWRANK_FOLDED_F16)
         # ring of distinct layers: layer 0 drawn by the seeded generator, the others re-use its small tensors with the
         # code matrix rolled per layer (set-up time only; every blob is a separate allocation)
         base = synth.random_layer(c["d_in"], c["d_out"], c["bits"], c["group_size"], c["rank"], seed=rank)
@@ -389,7 +392,14 @@ class Workload:
                 blobs.append(blobs[0])  # the same packed layer again: L2-resident measurement
                 continue
             codes = torch.roll(codes0, shifts=(i, 3 * i), dims=(0, 1)) if i else codes0
-            blobs.append(lopro.pack(d, codes, sc, zr, pm, A, B))
+            if fp8:
+                if i == 0:
+                    rec = synth.lowrank_record(c["d_out"], c["d_in"], c["rank"], seed=rank)
+                    U8, V8 = torch.from_numpy(rec["U"]).to(dev), torch.from_numpy(rec["V"]).to(dev)
+                    sg, sv = dev16(rec["sigma"]), dev16(rec["s"])
+                blobs.append(lopro.pack_lr8(d, codes, sc, zr, pm, U8, V8, sg, sv))
+            else:
+                blobs.append(lopro.pack(d, codes, sc, zr, pm, A, B))
         del codes0, codes
         self.x_host_bits = synth.activations(T, c["d_in"], seed=rank, outlier_frac=c.get("outlier_frac", 0.0),
                                              outlier_scale=c.get("outlier_scale", 20.0))
@@ -400,7 +410,7 @@ class Workload:
         self.d = d
         self.forwards = ring
         self.tokens_per_pass = T * ring
-        self.bytes_per_pass = ring * algorithmic_bytes(c, T)
+        self.bytes_per_pass = ring * algorithmic_bytes(c, T, "fp8" if fp8 else "f16")
         self.flops_per_pass = ring * algorithmic_flops(c, T)
         self.h2d, self.d2h = ring * T * c["d_in"] * 2, ring * T * c["d_out"] * 2
         path, per_forward = lopro.linear_fwd_path(d, T)
@@ -545,7 +555,7 @@ def measure(args, name, steps, warmup, rank, world, local, dev, dist, with_e2e=T
                         algorithmic_flops_per_launch=w.flops_per_pass // w.forwards, launch_us=per_forward_s * 1e6, note=note)
     rec = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps, warmup=warmup, ms_per_step=ms_per_step,
                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
-               config=dict(workload_config(name), passes_per_step=passes, layout=args.layout), clocks=clocks,
+               config=dict(workload_config(name), passes_per_step=passes, layout=args.layout, lowrank=args.lowrank), clocks=clocks,
                gpu_launches=w.launches_per_pass * passes * steps, path="+".join(w.paths), roofline=roofline,
                ms_per_forward=per_forward_s * 1e3, ms_per_pass=ms_per_pass, step_ms_min=min(step_ms),
                step_ms_median=statistics.median(step_ms), cuda_graph=graph is not None,
@@ -576,6 +586,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="only the named workload, not the table of the other regimes")
     ap.add_argument("--step-ms", type=float, default=50.0, help="a step repeats the pass until it lasts this long")
     ap.add_argument("--layout", default="fragment", choices=["fragment", "rowblock"], help="code layout of the packed layers")
+    ap.add_argument("--lowrank", default="f16", choices=["f16", "fp8"],
+                    help="storage of the rank-r term of single-layer workloads: folded fp16 A, B or the fp8 record U, V, Sigma, s")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

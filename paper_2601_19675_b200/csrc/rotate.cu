@@ -173,8 +173,8 @@ __device__ __forceinline__ void lowrank_row(const __nv_bfloat16* __restrict__ x,
 }
 
 // The same row job for the FP8 low-rank record (U, V, Sigma, s) that Algorithm 1 saves:
-// t[token][j] = sigma[j] * sum_k V[j][k] * (x[token][k] / s[k]), V in fp8 e4m3 (exact in fp32), the quotient as
-// x * (1 / s) in fp32, fp32 accumulation, one rounding to fp16.
+// t[token][j] = sigma[j] * sum_k V[j][k] * (x[token][k] / s[k]), V in fp8 e4m3 (exact in fp32), the quotient taken on
+// the layer's side as V[j][k] * (1 / s[k]) in fp32 (once for all tokens), fp32 accumulation, one rounding to fp16.
 template <int TPR>
 __device__ __forceinline__ void lowrank_row_lr8(const __nv_bfloat16* __restrict__ x, int64_t ldx, const Lr8Args lr8,
                                                 __half* __restrict__ t, int n, int r_pad, int T, int rb, int tok0) {
@@ -182,15 +182,32 @@ __device__ __forceinline__ void lowrank_row_lr8(const __nv_bfloat16* __restrict_
     __shared__ float part[8][TPR];
     const int j = rb % r_pad, tq = tok0 + TPR * (rb / r_pad);
     const uint8_t* vrow = lr8.V + (size_t)j * n;
-    if ((tid & 15) == 0 && tid * 8 < n) prefetch_l2(vrow + tid * 8);
+    if ((tid & 15) == 0) {  // one request per 128-byte line of the first 4096 columns of the row of V; s likewise
+#pragma unroll
+        for (int ps = 0; ps < 2; ++ps) {
+            const int k = ps * 2048 + tid * 8;
+            if (k < n) prefetch_l2(vrow + k);
+        }
+    }
+    if ((tid & 7) == 0) {
+#pragma unroll
+        for (int ps = 0; ps < 2; ++ps) {
+            const int k = ps * 2048 + tid * 8;
+            if (k < n) prefetch_l2(lr8.svec + k);
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     float acc[TPR];
 #pragma unroll
     for (int tk = 0; tk < TPR; ++tk) acc[tk] = 0.0f;
-    for (int k = tid * 8; k < n; k += 2048) {
-        const uint2 vw = __ldg(reinterpret_cast<const uint2*>(vrow + k));
-        const uint4 sw = __ldg(reinterpret_cast<const uint4*>(lr8.svec + k));
-        float vf[8], rs[8];
+    auto load_x = [&](uint4 (&xw)[TPR], int k) {
+#pragma unroll
+        for (int tk = 0; tk < TPR; ++tk)
+            xw[tk] = (k < n && tq + tk < T) ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tq + tk) * ldx + k))
+                                            : make_uint4(0, 0, 0, 0);
+    };
+    auto accumulate = [&](const uint2& vw, const uint4& sw, const uint4 (&xw)[TPR]) {
+        float vs[8];  // V[j][k] / s[k]
         const uint32_t vv[2] = {vw.x, vw.y};
         const __half2* sh = reinterpret_cast<const __half2*>(&sw);
 #pragma unroll
@@ -198,24 +215,42 @@ __device__ __forceinline__ void lowrank_row_lr8(const __nv_bfloat16* __restrict_
             const uint32_t h2 = e4m3x2_to_f16x2((uint16_t)(vv[i >> 1] >> (16 * (i & 1))));
             const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
             const float2 sf = __half22float2(sh[i]);
-            vf[2 * i] = f.x;
-            vf[2 * i + 1] = f.y;
-            rs[2 * i] = __frcp_rn(sf.x);
-            rs[2 * i + 1] = __frcp_rn(sf.y);
+            vs[2 * i] = f.x * __frcp_rn(sf.x);
+            vs[2 * i + 1] = f.y * __frcp_rn(sf.y);
         }
 #pragma unroll
         for (int tk = 0; tk < TPR; ++tk) {
-            if (tq + tk < T) {
-                const uint4 xw = __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tq + tk) * ldx + k));
-                const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xw);
+            const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xw[tk]);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float2 f = __bfloat1622float2(xh[i]);
-                    acc[tk] = fmaf(vf[2 * i], f.x * rs[2 * i], acc[tk]);
-                    acc[tk] = fmaf(vf[2 * i + 1], f.y * rs[2 * i + 1], acc[tk]);
-                }
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(xh[i]);
+                acc[tk] = fmaf(vs[2 * i], f.x, acc[tk]);
+                acc[tk] = fmaf(vs[2 * i + 1], f.y, acc[tk]);
             }
         }
+    };
+    const uint4 one = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u);  // s = 1 where there is no column
+    {   // the first two passes (all of K up to 4096 columns): every load in flight before the first use
+        uint2 v0 = make_uint2(0, 0), v1 = make_uint2(0, 0);
+        uint4 s0 = one, s1 = one, x0[TPR], x1[TPR];
+        const int k0 = tid * 8, k1 = 2048 + tid * 8;
+        if (k0 < n) {
+            v0 = __ldg(reinterpret_cast<const uint2*>(vrow + k0));
+            s0 = __ldg(reinterpret_cast<const uint4*>(lr8.svec + k0));
+        }
+        if (k1 < n) {
+            v1 = __ldg(reinterpret_cast<const uint2*>(vrow + k1));
+            s1 = __ldg(reinterpret_cast<const uint4*>(lr8.svec + k1));
+        }
+        load_x(x0, k0);
+        load_x(x1, k1);
+        accumulate(v0, s0, x0);
+        accumulate(v1, s1, x1);
+    }
+    for (int k = 4096 + tid * 8; k < n; k += 2048) {
+        uint4 xw[TPR];
+        load_x(xw, k);
+        accumulate(__ldg(reinterpret_cast<const uint2*>(vrow + k)), __ldg(reinterpret_cast<const uint4*>(lr8.svec + k)), xw);
     }
 #pragma unroll
     for (int tk = 0; tk < TPR; ++tk) {
