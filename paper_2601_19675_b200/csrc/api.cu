@@ -370,7 +370,7 @@ int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launch
     if (lr8_unsupported(*desc)) return 0;
     if (desc->layout == LOPRO_LAYOUT_ROWBLOCK) {
         if (!rowblock_supported(*desc)) return 0;
-        if (launches) *launches = rowblock_pre_launches(*desc, T) + (T <= 16 ? 1 : (T + 31) / 32);
+        if (launches) *launches = rowblock_pre_launches(*desc, T) + rowblock_launches(*desc) * (T <= 16 ? 1 : (T + 31) / 32);
         return LOPRO_PATH_ROWBLOCK;
     }
     int32_t path, n;

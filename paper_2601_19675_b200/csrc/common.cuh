@@ -162,6 +162,7 @@ cudaError_t launch_image_convert(const lopro_desc& d, const __nv_bfloat16* xrot,
                                  const __half* t, int r_pad, const ImageOut& img, int T, cudaStream_t s);
 // tcgen05 small-batch forward over the row-block layout, one launch per group of up to 32 tokens.
 bool rowblock_supported(const lopro_desc& d);
+int rowblock_launches(const lopro_desc& d);  // launches per group of up to 32 tokens (1 unless the layer is very large)
 cudaError_t launch_rowblock(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, uint8_t* ws,
                             const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int tgroup, int t_live,
                             cudaStream_t s);

@@ -74,7 +74,8 @@ struct RbParams {
     int m, T;                   // T: live tokens of this launch (<= NP)
     int nsteps, ng, gshift;     // 64-column steps of K, groups per row, log2(steps per group)
     int r_pad, lr_steps;
-    int units;                  // blocks * ng
+    int units;                  // blocks of this launch * ng
+    int rb_base;                // first block of rows of this launch
     int spg;                    // column-sum runs per group (1 unless g > 256)
     int c_slots;                // depth of the code ring
     int two_issuers;            // the two MMA threads take turns by stage (no group spans two stages)
@@ -109,58 +110,95 @@ struct Stage {
     bool piece_whole, piece_first;  // the piece covers the whole block / starts at the block's first unit
 };
 
-// Walks the stages of the run of units [u, u1) in the order every role of the CTA follows.
-struct Walker {
-    int u, u1, ng, gshift, lr_steps;
-    int rb = 0, gb = 0, ge = 0, n_lr = 0, total = 0, j = 0, q_first = 0, q_last = 0;
-    __device__ Walker(int u0_, int u1_, int ng_, int gshift_, int lr_steps_)
-        : u(u0_), u1(u1_), ng(ng_), gshift(gshift_), lr_steps(lr_steps_) {}
-    __device__ __noinline__ bool next(Stage& s) {
-        if (j == total) {  // next piece: the units of the run that lie in one block
-            u += ge - gb;
-            if (u >= u1) return false;
-            rb = u / ng;
-            gb = u - rb * ng;
-            ge = min(ng, gb + (u1 - u));
-            n_lr = gb == 0 ? (lr_steps + kStageItems - 1) / kStageItems : 0;
-            q_first = gb << gshift;
-            q_last = ge << gshift;
-            total = n_lr + (q_last - q_first + kStageItems - 1) / kStageItems;
-            j = 0;
-        }
-        s.rb = rb;
-        s.piece_first = gb == 0;
-        s.piece_whole = gb == 0 && ge == ng;
-        s.lr = j < n_lr;
-        if (s.lr) {
-            s.i0 = j * kStageItems;
-            s.ni = min(kStageItems, lr_steps - s.i0);
-            s.first_mask = j == 0 ? 1 : 0;
-            s.last_mask = j == n_lr - 1 ? 1 << (s.ni - 1) : 0;
-            s.close0 = 0;
-        } else {
-            s.i0 = q_first + (j - n_lr) * kStageItems;
-            s.ni = min(kStageItems, q_last - s.i0);
-            const int gmask = (1 << gshift) - 1, live = (1 << s.ni) - 1;
-            if (gshift == 0) {
-                s.first_mask = s.last_mask = live;
-            } else if (gshift == 1) {
-                s.first_mask = 0x5 & live;  // stages start on even steps
-                s.last_mask = 0xA & live;
-            } else {  // groups of four steps or more: at most one begins and one ends in a stage
-                s.first_mask = (s.i0 & gmask) == 0 ? 1 : 0;
-                s.last_mask = ((s.i0 + s.ni) & gmask) == 0 ? 1 << (s.ni - 1) : 0;
-            }
-            s.close0 = (s.i0 + gmask + 1) >> gshift;
-            s.close0 -= 1;
-        }
-        s.n_open = __popc(s.first_mask);
-        s.n_close = __popc(s.last_mask);
-        ++j;
-        s.piece_end = j == total;
-        return true;
-    }
+// The stages of a CTA's run of units [u0, u1), in the order every role follows, are worked out once, by all threads
+// in parallel, into a table in shared memory (16 bytes per stage): walking the run costs a couple of hundred
+// instructions per stage, which sixteen warps would otherwise each repeat.
+constexpr int kMaxStagesPerCta = 512;
+
+struct RunShape {  // pieces of the run: a first piece (possibly partial), whole blocks, a last partial piece
+    int ng, gshift, lr_steps, nlr;
+    int rb0, gb0, ge0, s0;     // first piece: block, groups [gb0, ge0), stages
+    int full, s_full;          // whole blocks after it and the stages of each
+    int tail, total;           // groups of the last piece (0: none), stages of the run
 };
+
+__device__ __forceinline__ int piece_stages(int gb, int ge, int gshift, int nlr) {
+    return (gb == 0 ? nlr : 0) + ((((ge - gb) << gshift) + kStageItems - 1) / kStageItems);
+}
+
+__device__ __forceinline__ RunShape run_shape(int u0, int u1, int ng, int gshift, int lr_steps) {
+    RunShape r;
+    r.ng = ng;
+    r.gshift = gshift;
+    r.lr_steps = lr_steps;
+    r.nlr = (lr_steps + kStageItems - 1) / kStageItems;
+    r.rb0 = u0 / ng;
+    r.gb0 = u0 - r.rb0 * ng;
+    r.ge0 = min(ng, r.gb0 + (u1 - u0));
+    r.s0 = u1 > u0 ? piece_stages(r.gb0, r.ge0, gshift, r.nlr) : 0;
+    const int rem = (u1 - u0) - (r.ge0 - r.gb0);
+    r.full = rem / ng;
+    r.tail = rem - r.full * ng;
+    r.s_full = piece_stages(0, ng, gshift, r.nlr);
+    r.total = r.s0 + r.full * r.s_full + (r.tail > 0 ? piece_stages(0, r.tail, gshift, r.nlr) : 0);
+    return r;
+}
+
+// Stage k of the run, packed: x = block | steps << 20 | low-rank << 23 | piece_end << 24 | piece_whole << 25 |
+// piece_first << 26;  y = first step | first closing group << 16;  z = first_mask | last_mask << 4;  w = 0.
+__device__ __forceinline__ uint4 stage_record(const RunShape& r, int k) {
+    int rb, gb, ge, j;
+    if (k < r.s0) {
+        rb = r.rb0; gb = r.gb0; ge = r.ge0; j = k;
+    } else {
+        const int k1 = k - r.s0, f = min(k1 / r.s_full, r.full);
+        rb = r.rb0 + 1 + f; gb = 0; ge = f < r.full ? r.ng : r.tail; j = k1 - f * r.s_full;
+    }
+    const int n_lr = gb == 0 ? r.nlr : 0;
+    const int q_first = gb << r.gshift, q_last = ge << r.gshift;
+    const int total = n_lr + (q_last - q_first + kStageItems - 1) / kStageItems;
+    int lr = j < n_lr, i0, ni, first_mask, last_mask, close0 = 0;
+    if (lr) {
+        i0 = j * kStageItems;
+        ni = min(kStageItems, r.lr_steps - i0);
+        first_mask = j == 0 ? 1 : 0;
+        last_mask = j == n_lr - 1 ? 1 << (ni - 1) : 0;
+    } else {
+        i0 = q_first + (j - n_lr) * kStageItems;
+        ni = min(kStageItems, q_last - i0);
+        const int gmask = (1 << r.gshift) - 1, live = (1 << ni) - 1;
+        if (r.gshift == 0) {
+            first_mask = last_mask = live;
+        } else if (r.gshift == 1) {
+            first_mask = 0x5 & live;  // stages start on even steps
+            last_mask = 0xA & live;
+        } else {  // groups of four steps or more: at most one begins and one ends in a stage
+            first_mask = (i0 & gmask) == 0 ? 1 : 0;
+            last_mask = ((i0 + ni) & gmask) == 0 ? 1 << (ni - 1) : 0;
+        }
+        close0 = ((i0 + gmask + 1) >> r.gshift) - 1;
+    }
+    const int piece_end = j == total - 1, piece_first = gb == 0, piece_whole = gb == 0 && ge == r.ng;
+    return make_uint4((uint32_t)(rb | (ni << 20) | (lr << 23) | (piece_end << 24) | (piece_whole << 25) | (piece_first << 26)),
+                      (uint32_t)(i0 | (close0 << 16)), (uint32_t)(first_mask | (last_mask << 4)), 0u);
+}
+
+__device__ __forceinline__ Stage unpack_stage(const uint4& v) {
+    Stage s;
+    s.rb = (int)(v.x & 0xFFFFFu);
+    s.ni = (int)((v.x >> 20) & 7u);
+    s.lr = ((v.x >> 23) & 1u) != 0;
+    s.piece_end = ((v.x >> 24) & 1u) != 0;
+    s.piece_whole = ((v.x >> 25) & 1u) != 0;
+    s.piece_first = ((v.x >> 26) & 1u) != 0;
+    s.i0 = (int)(v.y & 0xFFFFu);
+    s.close0 = (int)(v.y >> 16);
+    s.first_mask = (int)(v.z & 15u);
+    s.last_mask = (int)((v.z >> 4) & 15u);
+    s.n_open = __popc(s.first_mask);
+    s.n_close = __popc(s.last_mask);
+    return s;
+}
 
 // Out-of-line slow path of every wait of this file (one copy of the polling loop for all roles: the kernel is bound
 // by instruction fetch as soon as its hot loops outgrow the instruction caches).  Polls with a suspend-time hint, so a
@@ -234,6 +272,7 @@ rowblock_kernel(const RbParams p) {
     // x = first_mask | last_mask << 4 | steps << 8 | low-rank << 12 | end << 13 | MMAs of the last step << 16,
     // y = activation slot, z = slices opened before the stage
     __shared__ uint4 s_cmd[kAStages];
+    __shared__ uint4 s_stage[kMaxStagesPerCta];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t raw = smem_u32(smem_raw);
@@ -285,16 +324,24 @@ rowblock_kernel(const RbParams p) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kWarpMma) tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
+    // this CTA's run of units [u0, u1) and its table of stages
+    const long long G = gridDim.x;
+    const int u0 = (int)((long long)blockIdx.x * p.units / G), u1 = (int)(((long long)blockIdx.x + 1) * p.units / G);
+    const RunShape shape = run_shape(u0, u1, p.ng, p.gshift, p.lr_steps);
+    const int n_stages = min(shape.total, kMaxStagesPerCta);  // (the host splits a layer so that the table holds a run)
+    for (int k = tid; k < n_stages; k += kThreads) s_stage[k] = stage_record(shape, k);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
-
-    // this CTA's run of units [u0, u1)
-    const long long G = gridDim.x;
-    const int u0 = (int)((long long)blockIdx.x * p.units / G), u1 = (int)(((long long)blockIdx.x + 1) * p.units / G);
-    Walker walk(u0, u1, p.ng, p.gshift, p.lr_steps);
     Stage st;
+    int stage_k = 0;
+    auto next_stage = [&]() {
+        if (stage_k >= n_stages) return false;
+        st = unpack_stage(s_stage[stage_k++]);
+        st.rb += p.rb_base;
+        return true;
+    };
 
     bool dead = false;  // a wait of this thread ran out: it stops waiting
     auto wait = [&](uint32_t bar, uint32_t parity) {
@@ -309,7 +356,7 @@ rowblock_kernel(const RbParams p) {
         // ---------------- layer-data producer: packed codes and (scale, zero) pairs ----------------
         if (lane == 0) {
             Ring rc(p.c_slots), rg(kGSlots);
-            while (walk.next(st)) {
+            while (next_stage()) {
                 if (st.lr) continue;
                 const int R = rb_rows(p.m, st.rb);
                 const uint32_t bytes = (uint32_t)(st.ni * R * 8 * BITS);
@@ -333,7 +380,7 @@ rowblock_kernel(const RbParams p) {
         if (lane == 0) {
             asm volatile("griddepcontrol.wait;" ::: "memory");  // the prologue's image is complete
             Ring rx(kXSlots), rg(kGSlots);
-            while (walk.next(st)) {
+            while (next_stage()) {
                 const uint32_t bytes = (uint32_t)(st.ni * kXTile);
                 if (rx.wrapped) wait(empty_x + 8u * rx.slot, rx.phase ^ 1u);
                 mbar_expect_tx(full_x + 8u * rx.slot, bytes);
@@ -415,7 +462,7 @@ rowblock_kernel(const RbParams p) {
         Ring rc(p.c_slots), rx(kXSlots);
         int sidx = 0;   // stages seen so far: set `sidx & 1` expands stage sidx into A stage `sidx & 1`
         int spos = 0;   // slices opened so far
-        for (; walk.next(st); ++sidx) {
+        for (; next_stage(); ++sidx) {
             const bool mine = (sidx & 1) == set;
             const int R = rb_rows(p.m, st.rb);
             const bool live = r < R;
@@ -517,7 +564,7 @@ rowblock_kernel(const RbParams p) {
         float yacc[NP];
 #pragma unroll
         for (int i = 0; i < NP; ++i) yacc[i] = 0.0f;
-        while (walk.next(st)) {
+        while (next_stage()) {
             const int R = rb_rows(p.m, st.rb);
             const bool live = r < R;
             if (st.n_close > 0) {
@@ -581,7 +628,7 @@ rowblock_kernel(const RbParams p) {
                 store_rows(yacc);
             } else {
                 // contributors of this block: the CTAs whose runs meet its units, in grid order
-                const long long ub = (long long)st.rb * p.ng, ue = ub + p.ng - 1;
+                const long long ub = (long long)(st.rb - p.rb_base) * p.ng, ue = ub + p.ng - 1;
                 const int c_first = (int)(((ub + 1) * G - 1) / p.units), c_last = (int)(((ue + 1) * G - 1) / p.units);
                 float* mine = p.partial + (size_t)(2 * blockIdx.x + (st.piece_first ? 1 : 0)) * (NP * kRbRows);
 #pragma unroll
@@ -695,9 +742,35 @@ cudaError_t launch_rb_bits(const RbParams& p, int np, int grid, int smem_bytes, 
 
 }  // namespace
 
+// Blocks of rows per launch such that no CTA's run exceeds its stage table (0: not even one block fits).
+static int rowblock_blocks_per_launch(const lopro_desc& d) {
+    int sms = sm_count();
+    if (sms > kRbMaxGrid) sms = kRbMaxGrid;
+    const int ng = d.d_in / d.group_size, r_pad = d.rank > 0 ? round_up_int(d.rank, 16) : 0;
+    int gshift = 0;
+    while ((64 << gshift) < d.group_size) ++gshift;
+    const int nlr = ((r_pad + 63) / 64 + kStageItems - 1) / kStageItems;
+    // bound on the stages of a run of `u` units: its steps in fours, plus per piece the low-rank stages and one stage
+    // of rounding
+    auto stages_bound = [&](int nblocks) {
+        const long long units = (long long)nblocks * ng;
+        const int grid = (int)(units < sms ? units : sms);
+        const long long u = (units + grid - 1) / grid;
+        return (long long)(((u << gshift) + kStageItems - 1) / kStageItems) + (u / ng + 3) * (nlr + 1);
+    };
+    int per_launch = (d.d_out + kRbRows - 1) / kRbRows;
+    while (per_launch > 1 && stages_bound(per_launch) > kMaxStagesPerCta) per_launch = (per_launch + 1) / 2;
+    return stages_bound(per_launch) > kMaxStagesPerCta ? 0 : per_launch;
+}
+
+int rowblock_launches(const lopro_desc& d) {
+    const int per_launch = rowblock_blocks_per_launch(d), blocks = (d.d_out + kRbRows - 1) / kRbRows;
+    return per_launch > 0 ? (blocks + per_launch - 1) / per_launch : 0;
+}
+
 bool rowblock_supported(const lopro_desc& d) {
-    // a group record holds 512 bytes of (scale, zero) pairs and the column sums of the group's runs
-    return d.layout == LOPRO_LAYOUT_ROWBLOCK && d.group_size <= 4096;
+    // a group record holds the (scale, zero) pairs and the column sums of up to 16 runs of 256 columns
+    return d.layout == LOPRO_LAYOUT_ROWBLOCK && d.group_size <= 4096 && rowblock_blocks_per_launch(d) > 0;
 }
 
 cudaError_t launch_image_convert(const lopro_desc& d, const __nv_bfloat16* xrot, const float* s64, int s64_ld,
@@ -737,18 +810,29 @@ cudaError_t launch_rowblock(const lopro_desc& d, const uint8_t* blob, const Blob
     p.gshift = 0;
     while ((64 << p.gshift) < d.group_size) ++p.gshift;
     const int blocks = (d.d_out + kRbRows - 1) / kRbRows;
-    p.units = blocks * p.ng;
     p.spg = d.group_size > 256 ? d.group_size / 256 : 1;
     p.c_slots = pl.c_slots;
     p.two_issuers = (p.gshift <= 2 && p.lr_steps <= kStageItems) ? 1 : 0;
-    int grid = sm_count();
-    if (grid > kRbMaxGrid) grid = kRbMaxGrid;
-    if (grid > p.units) grid = p.units;
-    switch (d.bits) {
-        case 2: return launch_rb_bits<2>(p, np, grid, pl.smem_bytes, s);
-        case 3: return launch_rb_bits<3>(p, np, grid, pl.smem_bytes, s);
-        default: return launch_rb_bits<4>(p, np, grid, pl.smem_bytes, s);
+    int sms = sm_count();
+    if (sms > kRbMaxGrid) sms = kRbMaxGrid;
+    // A CTA's table holds kMaxStagesPerCta stages: a layer with more work per CTA than that runs as several launches
+    // over ranges of blocks.
+    const int per_launch = rowblock_blocks_per_launch(d);
+    if (per_launch == 0) return cudaErrorInvalidValue;
+    for (int b0 = 0; b0 < blocks; b0 += per_launch) {
+        const int nb = blocks - b0 < per_launch ? blocks - b0 : per_launch;
+        p.rb_base = b0;
+        p.units = nb * p.ng;
+        const int grid = p.units < sms ? p.units : sms;
+        cudaError_t e;
+        switch (d.bits) {
+            case 2: e = launch_rb_bits<2>(p, np, grid, pl.smem_bytes, s); break;
+            case 3: e = launch_rb_bits<3>(p, np, grid, pl.smem_bytes, s); break;
+            default: e = launch_rb_bits<4>(p, np, grid, pl.smem_bytes, s); break;
+        }
+        if (e != cudaSuccess) return e;
     }
+    return cudaSuccess;
 }
 
 }  // namespace lopro
