@@ -78,8 +78,8 @@ def time_oracle_stack(T, budget_s):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
 # capture summarised in profiles/; valid for the kernel as committed with that summary, null otherwise.
-NCU_TRAFFIC = {("cfg2_T8", "stream_wide_kernel"): 9296640, ("cfg4_T16", "tall_kernel"): 83635840,
-               ("cfg3_T2048", "prefill_kernel"): 53210752}
+NCU_TRAFFIC = {("cfg2_T8", "stream_wide_kernel"): 9295872, ("cfg2_T32", "stream_kernel"): 9488896,
+               ("cfg4_T16", "tall_kernel"): 83944448, ("cfg3_T2048", "prefill_kernel"): 53353984}
 METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
 
