@@ -253,8 +253,10 @@ LOPRO_API int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32
  *   the same d_in; x, out_dtype, T as for lopro_linear_fwd; workspace of lopro_group_workspace_bytes(...) bytes,
  *   256-byte aligned.  The status word of the group is the first word of the workspace.
  * When the layers differ in nothing but d_out and their data, are in LOPRO_LAYOUT_FRAGMENT, n_layers <= 4, T <= 32 and
- * each would run as prologue + streaming kernel, the group runs as TWO launches: one prologue that writes every
- * layer's rotated activations and B_i x, and one product launch over the row tiles of all layers.  Otherwise the
+ * each would run as prologue + small-batch kernel of the same kind (all per-row-group, or all persistent: the
+ * persistent CTAs are then shared out in proportion to the layers' rows), the group runs as TWO launches: one
+ * prologue that writes every layer's rotated activations and B_i x, and one product launch over the row tiles of
+ * all layers.  Otherwise the
  * layers run one after the other (same results, one lopro_linear_fwd each).  lopro_linear_fwd_group_path returns 2
  * in the first case, 1 in the second (0 on bad arguments) and the number of launches in *launches. */
 LOPRO_API size_t lopro_group_workspace_bytes(int32_t n_layers, const lopro_desc* const* descs, int32_t T);

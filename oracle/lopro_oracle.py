@@ -13,8 +13,7 @@ partial block Walsh-Hadamard matrix (Eq. 6), Qz(.) the group quantizer, and
 Every function states the passage it follows.  Nothing here is blocked, fused
 or reordered beyond what the cited definition states.
 
-Readings taken where the paper is silent or inconsistent (all listed in the
-design notes of the repository):
+Readings taken where the paper is silent or inconsistent:
   * permutation direction: gather, (P^T x)[k] = x[perm[k]], i.e. P[perm[k], k] = 1,
     which is the reading under which "sort(...).idx" moves the selected columns
     to the front (Eq. 5 and the sentence after it);

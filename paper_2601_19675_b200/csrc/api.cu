@@ -523,7 +523,10 @@ static bool group_shares_launches(int32_t n, const lopro_desc* const* descs, int
             d.identity_cols != d0.identity_cols || d.rank != d0.rank || d.layout != d0.layout ||
             d.lowrank_format != LOPRO_LOWRANK_FOLDED_F16)
             return false;
-        if (!prologue_supported(d, T) || !stream_supported(d, T) || use_tall(d, T)) return false;
+        if (!prologue_supported(d, T)) return false;
+        // all siblings through the persistent kernel or all through the per-group kernel
+        if (use_tall(d, T) != use_tall(d0, T)) return false;
+        if (!use_tall(d, T) && !stream_supported(d, T)) return false;
     }
     return true;
 }
@@ -629,8 +632,9 @@ lopro_status lopro_linear_fwd_group(int32_t n_layers, const lopro_desc* const* d
                         L[0].r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot, (__half*)(ws + W.off_t), W.t_pad,
                         (int*)(ws + W.off_status), T, s, nullptr, &ps) != cudaSuccess)
         return LOPRO_ERR_CUDA;
-    if (launch_stream(d0, blob0, L[0], ws, W, y[0], ldy[0], out_dtype, T, s, 0, &ss) != cudaSuccess) return LOPRO_ERR_CUDA;
-    return LOPRO_OK;
+    const cudaError_t e = use_tall(d0, T) ? launch_tall(d0, blob0, L[0], ws, W, y[0], ldy[0], out_dtype, T, s, 0, &ss)
+                                          : launch_stream(d0, blob0, L[0], ws, W, y[0], ldy[0], out_dtype, T, s, 0, &ss);
+    return e == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }
 
 size_t lopro_host_staging_bytes(const lopro_desc* desc, int32_t T, int32_t out_dtype) {

@@ -193,7 +193,8 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
 // Small-batch forward for tall layers after launch_prologue: persistent CTAs, one ring across tile groups.
 bool tall_supported(const lopro_desc& d, int T);
 cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                        const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0 = 0);
+                        const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0 = 0,
+                        const StreamSiblingArgs* more = nullptr);
 
 // t = B x on the tensor cores for many tokens; `partial` holds lowrank_mma_scratch_bytes of fp32 K-slice sums.
 size_t lowrank_mma_scratch_bytes(const lopro_desc& d, int T);

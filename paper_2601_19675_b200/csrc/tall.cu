@@ -60,6 +60,42 @@ struct TallParams {
     int off_a, a_bytes, off_t, off_red, off_ring, stage_bytes, off_stage_sz, off_stage_x;
 };
 
+// Sibling layers of a grouped launch: the grid's CTAs from cta0[i] on work on sibling i (the layer of TallParams
+// owns the CTAs before cta0[0]); each sibling walks its own rows with its own share of the persistent CTAs.
+struct TallSiblings {
+    int n;
+    int cta0[kMaxSiblings - 1];
+    const unsigned char* codes[kMaxSiblings - 1];
+    const uint32_t* sz[kMaxSiblings - 1];
+    const __half* A[kMaxSiblings - 1];
+    const unsigned char* act[kMaxSiblings - 1];
+    const __half* t[kMaxSiblings - 1];
+    void* y[kMaxSiblings - 1];
+    int64_t ldy[kMaxSiblings - 1];
+    int m[kMaxSiblings - 1];
+};
+
+// The layer a CTA works on: patches the per-layer fields, returns the CTA's index among the layer's CTAs and
+// their number.
+__device__ __forceinline__ int2 select_sibling(TallParams& p, const TallSiblings& sibs) {
+    int first = 0, end = sibs.n > 0 ? sibs.cta0[0] : (int)gridDim.x;
+#pragma unroll
+    for (int i = 0; i < kMaxSiblings - 1; ++i)
+        if (i < sibs.n && (int)blockIdx.x >= sibs.cta0[i]) {
+            first = sibs.cta0[i];
+            end = i + 1 < sibs.n ? sibs.cta0[i + 1] : (int)gridDim.x;
+            p.codes = sibs.codes[i];
+            p.sz = sibs.sz[i];
+            p.A = sibs.A[i];
+            p.act = sibs.act[i];
+            p.t = sibs.t[i];
+            p.y = sibs.y[i];
+            p.ldy = sibs.ldy[i];
+            p.m = sibs.m[i];
+        }
+    return make_int2((int)blockIdx.x - first, end - first);
+}
+
 __device__ __forceinline__ void named_sync(int id) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kConsumerThreads) : "memory");
 }
@@ -147,7 +183,9 @@ __device__ __forceinline__ void consume_stage(const unsigned char* stage, uint32
 
 template <int BITS, int NT>
 __global__ void __launch_bounds__(kThreads, 1)
-tall_kernel(const TallParams p) {
+tall_kernel(const TallParams p_in, const TallSiblings sibs) {
+    TallParams p = p_in;
+    const int2 cta = select_sibling(p, sibs);  // x: index among the layer's CTAs, y: their number
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t bars[2 * kMaxStages + 3];  // full, empty per stage; A buffers; t
     __shared__ int s_timeout;
@@ -158,9 +196,9 @@ tall_kernel(const TallParams p) {
     const int gq = lane >> 2, tg = lane & 3;
     // this CTA's run of 16-row tiles: the first `extra` CTAs hold one tile more
     const int tiles = p.m >> 4;
-    const int base = tiles / (int)gridDim.x, extra = tiles - base * (int)gridDim.x;
-    const int my_cnt = base + ((int)blockIdx.x < extra ? 1 : 0);
-    const int my_start = (int)blockIdx.x * base + min((int)blockIdx.x, extra);
+    const int base = tiles / cta.y, extra = tiles - base * cta.y;
+    const int my_cnt = base + (cta.x < extra ? 1 : 0);
+    const int my_start = cta.x * base + min(cta.x, extra);
     const int n_groups = (my_cnt + p.gt - 1) / p.gt;
     const int TS = p.total_stages;
     const int tc = min(kTok, p.T);  // live tokens
@@ -407,7 +445,7 @@ bool plan_tall(const lopro_desc& d, int T, TallPlan* pl) {
 }
 
 template <int BITS, int NT>
-cudaError_t launch_tall_k(const TallParams& p, int grid, int smem_bytes, cudaStream_t s) {
+cudaError_t launch_tall_k(const TallParams& p, const TallSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
     static unsigned long long attr_done = 0;
     cudaError_t e = ensure_dynamic_smem(tall_kernel<BITS, NT>, kStreamMaxSmem, &attr_done);
     if (e != cudaSuccess) return e;
@@ -421,14 +459,14 @@ cudaError_t launch_tall_k(const TallParams& p, int grid, int smem_bytes, cudaStr
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tall_kernel<BITS, NT>, p);
+    return cudaLaunchKernelEx(&cfg, tall_kernel<BITS, NT>, p, sibs);
 }
 
 template <int BITS>
-cudaError_t launch_tall_bits(const TallParams& p, int nt, int grid, int smem_bytes, cudaStream_t s) {
-    if (nt == 1) return launch_tall_k<BITS, 1>(p, grid, smem_bytes, s);
-    if (nt == 2) return launch_tall_k<BITS, 2>(p, grid, smem_bytes, s);
-    return launch_tall_k<BITS, 4>(p, grid, smem_bytes, s);
+cudaError_t launch_tall_bits(const TallParams& p, const TallSiblings& sibs, int nt, int grid, int smem_bytes, cudaStream_t s) {
+    if (nt == 1) return launch_tall_k<BITS, 1>(p, sibs, grid, smem_bytes, s);
+    if (nt == 2) return launch_tall_k<BITS, 2>(p, sibs, grid, smem_bytes, s);
+    return launch_tall_k<BITS, 4>(p, sibs, grid, smem_bytes, s);
 }
 
 }  // namespace
@@ -439,7 +477,8 @@ bool tall_supported(const lopro_desc& d, int T) {
 }
 
 cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                        const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0) {
+                        const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0,
+                        const StreamSiblingArgs* more) {
     TallPlan pl;
     if (!plan_tall(d, T, &pl)) return cudaErrorInvalidValue;
     TallParams p;
@@ -475,10 +514,37 @@ cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayo
     p.stage_bytes = pl.stage_bytes;
     p.off_stage_sz = pl.off_stage_sz;
     p.off_stage_x = pl.off_stage_x;
+    TallSiblings sibs = {};
+    if (more != nullptr && more->n > 0) {
+        // the persistent CTAs are shared out in proportion to the layers' row tiles (at least one CTA each)
+        long long tiles_all = d.d_out / 16;
+        for (int i = 0; i < more->n; ++i) tiles_all += more->d_out[i] / 16;
+        sibs.n = more->n;
+        long long tiles_before = d.d_out / 16;
+        for (int i = 0; i < more->n; ++i) {
+            int c0 = (int)((tiles_before * pl.grid + tiles_all / 2) / tiles_all);
+            const int lo = (i == 0 ? 0 : sibs.cta0[i - 1]) + 1, hi = pl.grid - (more->n - i);
+            if (c0 < lo) c0 = lo;
+            if (c0 > hi) c0 = hi;
+            sibs.cta0[i] = c0;
+            tiles_before += more->d_out[i] / 16;
+            const uint8_t* b = more->blob[i];
+            const BlobLayout& Li = more->L[i];
+            const uint8_t* wsi = more->ws[i];
+            sibs.codes[i] = b + Li.off[LOPRO_SEC_CODES];
+            sibs.sz[i] = reinterpret_cast<const uint32_t*>(b + Li.off[LOPRO_SEC_SCALEZERO]);
+            sibs.A[i] = reinterpret_cast<const __half*>(b + Li.off[LOPRO_SEC_A]);
+            sibs.act[i] = wsi + W.off_xrot + (size_t)t0 * kActRecord;
+            sibs.t[i] = reinterpret_cast<const __half*>(wsi + W.off_t) + (size_t)t0 * (d.rank > 0 ? L.r_pad : 0);
+            sibs.y[i] = more->y[i];
+            sibs.ldy[i] = more->ldy[i];
+            sibs.m[i] = more->d_out[i];
+        }
+    }
     switch (d.bits) {
-        case 2: return launch_tall_bits<2>(p, pl.nt, pl.grid, pl.smem_bytes, s);
-        case 3: return launch_tall_bits<3>(p, pl.nt, pl.grid, pl.smem_bytes, s);
-        default: return launch_tall_bits<4>(p, pl.nt, pl.grid, pl.smem_bytes, s);
+        case 2: return launch_tall_bits<2>(p, sibs, pl.nt, pl.grid, pl.smem_bytes, s);
+        case 3: return launch_tall_bits<3>(p, sibs, pl.nt, pl.grid, pl.smem_bytes, s);
+        default: return launch_tall_bits<4>(p, sibs, pl.nt, pl.grid, pl.smem_bytes, s);
     }
 }
 
