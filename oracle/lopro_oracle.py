@@ -255,28 +255,32 @@ def dequant(codes, scales, zeros, g):
     return s * (codes - z)
 
 
-def rtn_quantize(rp, bits, g):
+def rtn_quantize(rp, bits, g, dtype=np.float64):
     """Round-to-nearest asymmetric min/max group quantizer (the RTN row of the
     component ablation).  Per (row, group of g consecutive columns):
     scale = fp16((hi - lo) / (2^q - 1)), zero = fp16(rne(-lo / scale)),
     code = clamp(rne(v / scale) + zero, 0, 2^q - 1).  Degenerate group hi == lo = v:
     scale = |v| (1 if v == 0), zero = 1 if v < 0 else 0, code = 1 if v > 0 else 0.
+    `dtype` is the precision every operation is carried out and rounded in (IEEE, nearest-even):
+    float64 for the definition; float32 where the integer decisions (codes, zero-points) have to
+    be taken in the precision of an implementation that computes in single.
     Returns (codes uint8, scales fp64 holding fp16 values, zeros likewise)."""
-    rp = np.asarray(rp, dtype=np.float64)
+    rp = np.asarray(rp, dtype=dtype)
     m, n = rp.shape
     if n % g:
         raise ValueError("group size must divide n")
-    qmax = float(2 ** bits - 1)
+    qmax = dtype(2 ** bits - 1)
+    one, nil = dtype(1.0), dtype(0.0)
     v = rp.reshape(m, n // g, g)
     lo = v.min(axis=2)
     hi = v.max(axis=2)
     degenerate = hi == lo
-    scale = round_f16(np.where(degenerate, np.where(lo != 0.0, np.abs(lo), 1.0), (hi - lo) / qmax))
-    if np.any(scale == 0.0):
+    scale = round_f16(np.where(degenerate, np.where(lo != nil, np.abs(lo), one), (hi - lo) / qmax)).astype(dtype)
+    if np.any(scale == nil):
         raise ValueError("group range underflows fp16")
-    zero = round_f16(np.where(degenerate, np.where(lo < 0.0, 1.0, 0.0), np.rint(-lo / scale)))
-    code = np.clip(np.rint(v / scale[..., None]) + zero[..., None], 0.0, qmax)
-    return code.reshape(m, n).astype(np.uint8), scale, zero
+    zero = round_f16(np.where(degenerate, np.where(lo < nil, one, nil), np.rint(-lo / scale))).astype(dtype)
+    code = np.clip(np.rint(v / scale[..., None]) + zero[..., None], nil, qmax)
+    return code.reshape(m, n).astype(np.uint8), scale.astype(np.float64), zero.astype(np.float64)
 
 
 def pack_canonical(codes, bits):

@@ -121,10 +121,11 @@ def test_zero_quantization_error_reconstructs_w_exactly():
         resid = w - a @ b
         rp = o.partial_block_rotate(o.permute_columns(resid, perm), b_i, b_h)
         np.testing.assert_array_equal(rp, o.dequant(codes, scales, zeros, g))   # R' recovered exactly
-        c2, s2, z2 = o.rtn_quantize(rp, bits, g)
-        np.testing.assert_array_equal(c2, codes)
-        np.testing.assert_array_equal(s2, scales)
-        np.testing.assert_array_equal(z2, zeros)
+        for dtype in (np.float64, np.float32):      # every operation is exact here, so the precision cannot matter
+            c2, s2, z2 = o.rtn_quantize(rp, bits, g, dtype=dtype)
+            np.testing.assert_array_equal(c2, codes)
+            np.testing.assert_array_equal(s2, scales)
+            np.testing.assert_array_equal(z2, zeros)
         w2 = o.effective_weight(c2, s2, z2, perm, a, b, g, b_i, b_h)
         assert np.max(np.abs(w2 - w)) == 0.0
 
@@ -143,6 +144,24 @@ def test_rtn_error_bound_and_degenerate_groups():
     for c in (0.25, -0.25, 0.0):
         codes, s, z = o.rtn_quantize(np.full((1, 8), c), 4, 8)
         np.testing.assert_array_equal(o.dequant(codes, s, z, 8), np.full((1, 8), c))
+
+
+def test_rtn_precision_switch_worked_by_hand():
+    # 2-bit group {2^-30, 3t, a, 1/2} with t = 1 + 3/2048, the midpoint of the fp16 neighbours 1 + 1/1024 and 1 + 2/1024.
+    # Double precision: hi - lo = 3t - 2^-30 exactly, a third of it lies just below t, so the step rounds DOWN to
+    # 1 + 1/1024.  Single precision: 2^-30 is far below half an ulp of 3t (2^-23), the difference rounds to 3t, the
+    # quotient is t itself, and the tie goes to the even mantissa, 1 + 2/1024.  a = 1 + 1029/2048 then lands on
+    # a / step = 1.50098 (code 2) in double and 1.49951 (code 1) in single; the zero-point is rne(-2^-30 / step) = 0.
+    t = 1.0 + 3.0 / 2048.0
+    a = 1.0 + 1029.0 / 2048.0
+    v = np.array([[2.0 ** -30, 3.0 * t, a, 0.5]])
+    assert np.all(v.astype(np.float32).astype(np.float64) == v)          # the inputs are single-precision numbers
+    c64, s64, z64 = o.rtn_quantize(v, 2, 4)
+    c32, s32, z32 = o.rtn_quantize(v, 2, 4, dtype=np.float32)
+    assert s64[0, 0] == 1.0 + 1.0 / 1024.0 and s32[0, 0] == 1.0 + 2.0 / 1024.0
+    assert z64[0, 0] == 0.0 and z32[0, 0] == 0.0
+    np.testing.assert_array_equal(c64, [[0, 3, 2, 0]])
+    np.testing.assert_array_equal(c32, [[0, 3, 1, 0]])
 
 
 def test_pack_canonical_bit_stream():
