@@ -311,6 +311,58 @@ LOPRO_API lopro_status lopro_linear_fwd_noalloc(const lopro_desc* desc, const vo
  * 4-byte aligned; the kernel first stores LOPRO_OK there).  Asynchronous: read the word after synchronising. */
 LOPRO_API lopro_status lopro_selftest_wait(void* status_word, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------
+ * Offline side of the method on the GPU (Algorithm 1 without its calibration inputs): the step BEFORE the forward
+ * path.  All matrices are fp32 device memory, row-major; every call is asynchronous on `stream`.
+ *
+ * lopro_r1svd -- rank-1 randomized sketch with deflation (Sec. 3.3, Eq. 10-12; inner loop of Algorithm 1).  Per rank
+ *   j: y = (W W^T)^it W v_j, p = W^T y, U_j = y / |y|, V_j = p / |p|, sigma_j = |p| / |y|, optionally U_j, V_j
+ *   rounded to fp8 e4m3 (cast = 1; the values are then those fp8 numbers, held in fp32), then W <- W - sigma_j U_j V_j^T.
+ *   The vector is renormalised after every product (a scaling that cancels in U_j, V_j and sigma_j), so no power of
+ *   W overflows.  A rank whose y or p vanishes (matrix exhausted) and all later ones come out as zeros.
+ *     w        [m][n], IN: the matrix to decompose (W diag(s)); OUT: the deflated remainder
+ *     sketches [r][n] Gaussian test vectors v_j (the call draws nothing)
+ *     U [m][r], sigma [r], V [r][n] outputs; workspace of lopro_r1svd_workspace_bytes(m, n) bytes, 256-byte aligned
+ *   m, n multiples of 4, 1 <= r <= 512, 0 <= it <= 64.  The work is 2 it + 2 matrix-vector products and one
+ *   rank-1 update per rank: memory-bound passes over w.
+ *
+ * lopro_residual_rotate -- R' = (W - Af Bf) P Q (Eq. 3 form ii, Eq. 5, Eq. 6), one row of W at a time: the residual
+ *   against the STORED low-rank factors (Af [m][rank], Bf [rank][n] hold the stored values, e.g. fp16 numbers or
+ *   U Sigma and V diag(s)^-1 formed from the fp8 / fp16 record; rank = desc->rank, may be 0 with null factors), the
+ *   column gather R[:, perm[k]] and the partial block Walsh-Hadamard rotation of every row (the same transform the
+ *   forward applies to an activation row), in fp32.  r_rot [m][n].  d_in <= 24576.
+ *   An index of perm outside [0, n) stores LOPRO_ERR_INVALID_DATA in *status_word (device, 4 bytes) and reads column 0.
+ *
+ * lopro_rtn_quantize -- the group grid of Appendix A.2 by round-to-nearest (ablation row 'RTN'): per row and group of
+ *   g consecutive columns of r_rot, lo = min, hi = max, scale = fp16((hi - lo) / (2^q - 1)),
+ *   zero = fp16(rne(-lo / scale)), code = clamp(rne(v / scale) + zero, 0, 2^q - 1); a constant group v stores scale |v|
+ *   (1 if v = 0), zero 1 if v < 0 else 0, code 1 if v > 0 else 0.  Every operation is an IEEE single-precision operation
+ *   rounded to nearest-even, in this order.  Outputs in the input formats of lopro_pack: codes [m][n] one per byte,
+ *   scales, zeros [m][n/g] fp16 bits.  A non-finite input or a group whose step rounds to zero in fp16 stores
+ *   LOPRO_ERR_INVALID_DATA in *status_word.
+ *
+ * lopro_quantize_layer -- the three steps in sequence for one layer: W_s = W diag(s) (s null: ones; with
+ *   LOPRO_LOWRANK_FP8 s is first rounded to fp16, as stored), R1SVD of W_s (fp8 cast inside the loop for
+ *   LOPRO_LOWRANK_FP8), the record's factors, the residual against them, rotation and quantization.
+ *     lr0..lr3: LOPRO_LOWRANK_FOLDED_F16: lr0 = A [m][r] fp16 = fp16(U Sigma), lr1 = B [r][n] fp16 = fp16(V diag(s)^-1);
+ *               LOPRO_LOWRANK_FP8: lr0 = U [m][r] e4m3, lr1 = V [r][n] e4m3, lr2 = Sigma [r] fp16, lr3 = s [n] fp16
+ *     -- exactly the arguments of lopro_pack / lopro_pack_lr8.  rank = 0: no factors, R = W.
+ *   The first word of the workspace is the status word; workspace of lopro_quantize_workspace_bytes(desc) bytes
+ *   (a copy of W among other things). */
+LOPRO_API size_t lopro_r1svd_workspace_bytes(int32_t m, int32_t n);
+LOPRO_API lopro_status lopro_r1svd(float* w, int32_t m, int32_t n, int32_t r, int32_t it, const float* sketches,
+                                   int32_t cast, float* U, float* sigma, float* V, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+LOPRO_API lopro_status lopro_residual_rotate(const lopro_desc* desc, const float* W, const float* Af, const float* Bf,
+                                             const int32_t* perm, float* r_rot, void* status_word, void* stream);
+LOPRO_API lopro_status lopro_rtn_quantize(const lopro_desc* desc, const float* r_rot, uint8_t* codes, uint16_t* scales,
+                                          uint16_t* zeros, void* status_word, void* stream);
+LOPRO_API size_t lopro_quantize_workspace_bytes(const lopro_desc* desc);
+LOPRO_API lopro_status lopro_quantize_layer(const lopro_desc* desc, const float* W, const float* s, const int32_t* perm,
+                                            const float* sketches, int32_t it, uint8_t* codes, uint16_t* scales,
+                                            uint16_t* zeros, void* lr0, void* lr1, void* lr2, void* lr3, void* workspace,
+                                            size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,7 +25,8 @@ SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packe
            "lopro_workspace_bytes", "lopro_pack", "lopro_unpack", "lopro_rotate", "lopro_linear_fwd",
            "lopro_linear_fwd_path", "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc",
            "lopro_configure", "lopro_selftest_wait", "lopro_group_workspace_bytes", "lopro_linear_fwd_group_path",
-           "lopro_linear_fwd_group", "lopro_pack_lr8", "lopro_unpack_lr8"]
+           "lopro_linear_fwd_group", "lopro_pack_lr8", "lopro_unpack_lr8", "lopro_r1svd_workspace_bytes", "lopro_r1svd",
+           "lopro_residual_rotate", "lopro_rtn_quantize", "lopro_quantize_workspace_bytes", "lopro_quantize_layer"]
 
 
 class Desc(ctypes.Structure):
@@ -99,6 +100,18 @@ def lib():
         L.lopro_configure.argtypes = [i32, i32]
         L.lopro_selftest_wait.restype = ctypes.c_int
         L.lopro_selftest_wait.argtypes = [vp, vp]
+        L.lopro_r1svd_workspace_bytes.restype = sz
+        L.lopro_r1svd_workspace_bytes.argtypes = [i32, i32]
+        L.lopro_r1svd.restype = ctypes.c_int
+        L.lopro_r1svd.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, sz, vp]
+        L.lopro_residual_rotate.restype = ctypes.c_int
+        L.lopro_residual_rotate.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp]
+        L.lopro_rtn_quantize.restype = ctypes.c_int
+        L.lopro_rtn_quantize.argtypes = [dp, vp, vp, vp, vp, vp, vp]
+        L.lopro_quantize_workspace_bytes.restype = sz
+        L.lopro_quantize_workspace_bytes.argtypes = [dp]
+        L.lopro_quantize_layer.restype = ctypes.c_int
+        L.lopro_quantize_layer.argtypes = [dp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -227,6 +240,77 @@ def pack_lr8(desc, codes, scales_f16, zeros_f16, perm, U_e4m3, V_e4m3, sigma_f16
                               _ptr(_dev(perm, 4)), _ptr(_dev(U_e4m3, 1)), _ptr(_dev(V_e4m3, 1)), _ptr(_dev(sigma_f16, 2)),
                               _ptr(_dev(s_f16, 2)), _ptr(out), out.numel(), _stream())
     _check(st, "lopro_pack_lr8")
+    return out
+
+
+def r1svd(w, r, it, sketches, cast=False):
+    """lopro_r1svd on a device fp32 matrix w [m][n] (deflated IN PLACE); returns (U [m][r], sigma [r], V [r][n]) fp32."""
+    m, n = w.shape
+    dev = w.device
+    U = torch.empty((m, r), dtype=torch.float32, device=dev)
+    sigma = torch.empty((r,), dtype=torch.float32, device=dev)
+    V = torch.empty((r, n), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(lib().lopro_r1svd_workspace_bytes(m, n), 256), dtype=torch.uint8, device=dev)
+    st = lib().lopro_r1svd(_ptr(_dev(w, 4)), m, n, r, it, _ptr(_dev(sketches, 4)), 1 if cast else 0, _ptr(U), _ptr(sigma),
+                           _ptr(V), _ptr(ws), ws.numel(), _stream())
+    _check(st, "lopro_r1svd")
+    return U, sigma, V
+
+
+def residual_rotate(desc, W, Af, Bf, perm):
+    """lopro_residual_rotate: R' = (W - Af Bf) P Q as fp32 [m][n], and the device status word (int32 tensor)."""
+    out = torch.empty((desc.d_out, desc.d_in), dtype=torch.float32, device=W.device)
+    status = torch.zeros(1, dtype=torch.int32, device=W.device)
+    st = lib().lopro_residual_rotate(ctypes.byref(desc), _ptr(_dev(W, 4)), _ptr(None if Af is None else _dev(Af, 4)),
+                                     _ptr(None if Bf is None else _dev(Bf, 4)), _ptr(_dev(perm, 4)), _ptr(out),
+                                     _ptr(status), _stream())
+    _check(st, "lopro_residual_rotate")
+    return out, status
+
+
+def rtn_quantize(desc, r_rot):
+    """lopro_rtn_quantize: (codes uint8 [m][n], scales, zeros int16 fp16 bit patterns [m][n/g], status int32 tensor)."""
+    m, n, g, dev = desc.d_out, desc.d_in, desc.group_size, r_rot.device
+    codes = torch.empty((m, n), dtype=torch.uint8, device=dev)
+    scales = torch.empty((m, n // g), dtype=torch.int16, device=dev)
+    zeros = torch.empty((m, n // g), dtype=torch.int16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = lib().lopro_rtn_quantize(ctypes.byref(desc), _ptr(_dev(r_rot, 4)), _ptr(codes), _ptr(scales), _ptr(zeros),
+                                  _ptr(status), _stream())
+    _check(st, "lopro_rtn_quantize")
+    return codes, scales, zeros, status
+
+
+def quantize_workspace_bytes(desc):
+    return lib().lopro_quantize_workspace_bytes(ctypes.byref(desc))
+
+
+def quantize_layer(desc, W, perm, sketches=None, it=8, s=None, workspace=None):
+    """lopro_quantize_layer: a dict with codes, scales, zeros and the low-rank record in the input formats of
+    pack / pack_lr8 (A, B int16 fp16 bits; or U, V uint8, sigma, s int16), plus the workspace (its first word is the
+    status word)."""
+    m, n, g, r, dev = desc.d_out, desc.d_in, desc.group_size, desc.rank, W.device
+    nbytes = quantize_workspace_bytes(desc)
+    if nbytes == 0:
+        raise LoproError(check_desc(desc) or ERR_UNSUPPORTED, "lopro_quantize_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    out = dict(codes=torch.empty((m, n), dtype=torch.uint8, device=dev),
+               scales=torch.empty((m, n // g), dtype=torch.int16, device=dev),
+               zeros=torch.empty((m, n // g), dtype=torch.int16, device=dev), workspace=workspace)
+    lr = [None, None, None, None]
+    if r > 0 and desc.lowrank_format == LOWRANK_FP8:
+        out.update(U=torch.empty((m, r), dtype=torch.uint8, device=dev), V=torch.empty((r, n), dtype=torch.uint8, device=dev),
+                   sigma=torch.empty((r,), dtype=torch.int16, device=dev), s=torch.empty((n,), dtype=torch.int16, device=dev))
+        lr = [out["U"], out["V"], out["sigma"], out["s"]]
+    elif r > 0:
+        out.update(A=torch.empty((m, r), dtype=torch.int16, device=dev), B=torch.empty((r, n), dtype=torch.int16, device=dev))
+        lr = [out["A"], out["B"], None, None]
+    st = lib().lopro_quantize_layer(ctypes.byref(desc), _ptr(_dev(W, 4)), _ptr(None if s is None else _dev(s, 4)),
+                                    _ptr(_dev(perm, 4)), _ptr(None if sketches is None else _dev(sketches, 4)), it,
+                                    _ptr(out["codes"]), _ptr(out["scales"]), _ptr(out["zeros"]), _ptr(lr[0]), _ptr(lr[1]),
+                                    _ptr(lr[2]), _ptr(lr[3]), _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "lopro_quantize_layer")
     return out
 
 

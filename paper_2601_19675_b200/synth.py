@@ -110,8 +110,16 @@ def factors(m, n, r, seed=0, std=0.01):
     return f32_to_f16_bits(a), f32_to_f16_bits(b)
 
 
-def weights(m, n, seed=0, std=0.02):
-    return _rng(seed, "W").standard_normal((m, n), dtype=np.float32) * np.float32(std)
+def weights(m, n, seed=0, std=0.02, spikes=0, spike_gain=24.0):
+    """fp32 weight matrix ~ N(0, std); `spikes` > 0 adds that many rank-1 terms with geometrically decaying weights
+    (separated leading singular values, as trained LLM weights have)."""
+    w = _rng(seed, "W").standard_normal((m, n), dtype=np.float32) * np.float32(std)
+    if spikes:
+        a = _rng(seed, "A").standard_normal((m, spikes), dtype=np.float32)
+        b = _rng(seed, "B").standard_normal((spikes, n), dtype=np.float32)
+        gains = (np.float32(spike_gain * std) * np.float32(0.75) ** np.arange(spikes, dtype=np.float32)) / np.float32(np.sqrt(min(m, n)))
+        w = w + (a * gains[None, :]) @ b
+    return w.astype(np.float32)
 
 
 def sketches(r, n, seed=0):

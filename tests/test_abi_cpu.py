@@ -175,3 +175,16 @@ def test_fp8_lowrank_record_reproduces_the_printed_storage_overhead(golden_dir):
     assert lopro.packed_section(d16, lopro.SEC_A)[1] == 2 * lopro.packed_section(d8, lopro.SEC_A)[1]
     assert lopro.check_desc(lopro.make_desc(4096, 4096, 4, 128, 128, rank=0, lowrank_format=lopro.LOWRANK_FP8)) == lopro.ERR_INVALID_ARG
     assert lopro.check_desc(lopro.make_desc(4096, 4096, 4, 128, 128, rank=16, lowrank_format=3)) == lopro.ERR_INVALID_ARG
+
+
+def test_offline_side_workspace_sizes():
+    # the layer quantizer keeps a copy of W (deflated in place by the rank-1 sketch) besides its small vectors
+    d = lopro.make_desc(4096, 11008, 4, 128, 128, rank=16)
+    need = lopro.quantize_workspace_bytes(d)
+    assert need >= 4096 * 11008 * 4 and need <= 4096 * 11008 * 4 * 1.1
+    assert lopro.lib().lopro_r1svd_workspace_bytes(11008, 4096) >= (11008 // 32) * 4096 * 4
+    # rank 0: no copy, no sketch workspace
+    assert lopro.quantize_workspace_bytes(lopro.make_desc(4096, 4096, 2, 64, 256, rank=0)) < 1 << 20
+    # rows longer than two fp32 copies in one CTA's shared memory are refused
+    assert lopro.quantize_workspace_bytes(lopro.make_desc(32768, 64, 4, 128, 128, rank=0)) == 0
+    assert lopro.lib().lopro_r1svd_workspace_bytes(0, 16) == 0
