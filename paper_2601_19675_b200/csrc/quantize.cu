@@ -13,48 +13,66 @@ namespace {
 
 constexpr int kGemvThreads = 256;  // 8 warps: one row of W per warp
 constexpr int kSlabRows = 32;      // rows of W per CTA in the transposed product
-constexpr int kNormThreads = 1024;
 
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-// y[i] = sum_k W[i][k] (v[k] * scale): one warp per row, 16-byte loads, lanes strided over the row, then a butterfly
-// over the lanes.  `scale` (device, may be null) is the reciprocal norm the previous step left behind.
-__global__ void __launch_bounds__(kGemvThreads) gemv_rows_kernel(const float* __restrict__ W, int m, int n,
-                                                                  const float* __restrict__ v,
-                                                                  const float* __restrict__ scale, float* __restrict__ y) {
-    const int row = blockIdx.x * (kGemvThreads / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (row >= m) return;
-    const float sc = scale ? *scale : 1.0f;
-    const float4* w4 = reinterpret_cast<const float4*>(W + (size_t)row * n);
-    const float4* v4 = reinterpret_cast<const float4*>(v);
+// Sum of squares of a vector by one warp: lanes strided, then a butterfly -- every warp that calls this on the same
+// vector gets the same bits.
+__device__ __forceinline__ float warp_sumsq(const float* __restrict__ v, int len, int lane) {
     float acc = 0.0f;
-    for (int c = lane; c < n / 4; c += 32) {
-        const float4 a = __ldg(w4 + c), b = __ldg(v4 + c);
-        acc = fmaf(a.x, b.x * sc, acc);
-        acc = fmaf(a.y, b.y * sc, acc);
-        acc = fmaf(a.z, b.z * sc, acc);
-        acc = fmaf(a.w, b.w * sc, acc);
-    }
+    for (int i = lane; i < len; i += 32) acc = fmaf(v[i], v[i], acc);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) y[row] = acc;
+    return acc;
+}
+__device__ __forceinline__ float inv_norm(float sumsq) {
+    const float nrm = sqrtf(sumsq);
+    return (nrm > 0.0f && isfinite(nrm)) ? 1.0f / nrm : 0.0f;
 }
 
-// partial[slab][k] = sum over the slab's rows i of W[i][k] (y[i] * scale): a CTA owns kSlabRows rows and 1024
-// columns, a thread four columns; rows in ascending order.
+// y[i] = (sum_k W[i][k] v[k]) / |v|: one warp per row, 16-byte loads, lanes strided over the row, then a butterfly
+// over the lanes.  Every warp reads all of v anyway, so each forms |v|^2 itself (same order, same bits) and no
+// separate reduction launch is needed.
+__global__ void __launch_bounds__(kGemvThreads) gemv_rows_kernel(const float* __restrict__ W, int m, int n,
+                                                                  const float* __restrict__ v, float* __restrict__ y) {
+    const int row = blockIdx.x * (kGemvThreads / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= m) return;
+    const float4* w4 = reinterpret_cast<const float4*>(W + (size_t)row * n);
+    const float4* v4 = reinterpret_cast<const float4*>(v);
+    float acc = 0.0f, vv = 0.0f;
+#pragma unroll 4
+    for (int c = lane; c < n / 4; c += 32) {
+        const float4 a = __ldg(w4 + c), b = __ldg(v4 + c);
+        acc = fmaf(a.x, b.x, acc);
+        acc = fmaf(a.y, b.y, acc);
+        acc = fmaf(a.z, b.z, acc);
+        acc = fmaf(a.w, b.w, acc);
+        vv = fmaf(b.x, b.x, vv);
+        vv = fmaf(b.y, b.y, vv);
+        vv = fmaf(b.z, b.z, vv);
+        vv = fmaf(b.w, b.w, vv);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        vv += __shfl_xor_sync(0xffffffffu, vv, o);
+    }
+    if (lane == 0) y[row] = acc * inv_norm(vv);
+}
+
+// partial[slab][k] = sum over the slab's rows i of W[i][k] y[i]: a CTA owns kSlabRows rows and 1024 columns, a
+// thread four columns; rows in ascending order.
 __global__ void __launch_bounds__(256) gemv_cols_kernel(const float* __restrict__ W, int m, int n,
-                                                        const float* __restrict__ y, const float* __restrict__ scale,
-                                                        float* __restrict__ partial) {
+                                                        const float* __restrict__ y, float* __restrict__ partial) {
     __shared__ float ys[kSlabRows];
     const int slab = blockIdx.y, r0 = slab * kSlabRows, rows = min(kSlabRows, m - r0);
-    const float sc = scale ? *scale : 1.0f;
-    if ((int)threadIdx.x < rows) ys[threadIdx.x] = y[r0 + threadIdx.x] * sc;
+    if ((int)threadIdx.x < rows) ys[threadIdx.x] = y[r0 + threadIdx.x];
     __syncthreads();
     const int c4 = blockIdx.x * 256 + threadIdx.x;
     if (c4 >= n / 4) return;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     const float4* w4 = reinterpret_cast<const float4*>(W + (size_t)r0 * n) + c4;
-#pragma unroll 4
+#pragma unroll 8
     for (int i = 0; i < rows; ++i) {
         const float4 a = __ldg(w4 + (size_t)i * (n / 4));
         const float s = ys[i];
@@ -66,35 +84,20 @@ __global__ void __launch_bounds__(256) gemv_cols_kernel(const float* __restrict_
     reinterpret_cast<float4*>(partial + (size_t)slab * n)[c4] = acc;
 }
 
-// p[k] = sum over slabs (ascending) of partial[slab][k]
+// p[k] = (sum over slabs, ascending, of partial[slab][k]) / |y|; the first warp of every CTA forms |y|^2.
 __global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ partial, int slabs, int n,
-                                                     float* __restrict__ p) {
+                                                     const float* __restrict__ y, int m, float* __restrict__ p) {
+    __shared__ float s_inv;
+    if (threadIdx.x < 32) {
+        const float ss = warp_sumsq(y, m, threadIdx.x);
+        if (threadIdx.x == 0) s_inv = inv_norm(ss);
+    }
+    __syncthreads();
     const int k = blockIdx.x * 256 + threadIdx.x;
     if (k >= n) return;
     float acc = 0.0f;
     for (int s = 0; s < slabs; ++s) acc += partial[(size_t)s * n + k];
-    p[k] = acc;
-}
-
-// out[0] = |v|, out[1] = 1 / |v| (0 when |v| = 0 or not finite): one CTA, fixed order.
-__global__ void __launch_bounds__(kNormThreads) norm_kernel(const float* __restrict__ v, int len, float* __restrict__ out) {
-    __shared__ float red[kNormThreads / 32];
-    float acc = 0.0f;
-    for (int i = threadIdx.x; i < len; i += kNormThreads) acc = fmaf(v[i], v[i], acc);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        float a = red[threadIdx.x];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-        if (threadIdx.x == 0) {
-            const float nrm = sqrtf(a);
-            out[0] = nrm;
-            out[1] = (nrm > 0.0f && isfinite(nrm)) ? 1.0f / nrm : 0.0f;
-        }
-    }
+    p[k] = acc * s_inv;
 }
 
 // fp32 -> nearest fp8 e4m3 value (ties to even, saturating), returned as fp32; bits optionally kept.
@@ -107,27 +110,36 @@ __device__ __forceinline__ float round_e4m3(float x, unsigned char* bits) {
 }
 
 // Rank j is done: U[:, j] = y / |y|, V[j, :] = p / |p| (cast to fp8 values when asked), sigma[j] = |p| where
-// p = W^T (y / |y|).  ny = {|y|, 1/|y|}, np = {|p|, 1/|p|}.  A vanished y or p gives a zero triple.
+// p = W^T (y / |y|).  Every CTA forms the two norms itself.  A vanished y or p gives a zero triple.
 __global__ void __launch_bounds__(256) finish_rank_kernel(const float* __restrict__ y, const float* __restrict__ p,
-                                                          const float* __restrict__ ny, const float* __restrict__ np,
                                                           int m, int n, int r, int j, int cast, float* __restrict__ U,
                                                           float* __restrict__ sigma, float* __restrict__ V,
                                                           float* __restrict__ u1, float* __restrict__ v1) {
-    const bool dead = ny[1] == 0.0f || np[1] == 0.0f;
+    __shared__ float s_ny, s_np;
+    if (threadIdx.x < 32) {
+        const float a = warp_sumsq(y, m, threadIdx.x), b = warp_sumsq(p, n, threadIdx.x);
+        if (threadIdx.x == 0) {
+            s_ny = a;
+            s_np = b;
+        }
+    }
+    __syncthreads();
+    const float iy = inv_norm(s_ny), ip = inv_norm(s_np);
+    const bool dead = iy == 0.0f || ip == 0.0f;
     const int i = blockIdx.x * 256 + threadIdx.x;
     if (i < m) {
-        float u = dead ? 0.0f : y[i] * ny[1];
+        float u = dead ? 0.0f : y[i] * iy;
         if (cast) u = round_e4m3(u, nullptr);
         U[(size_t)i * r + j] = u;
         u1[i] = u;
     }
     if (i < n) {
-        float v = dead ? 0.0f : p[i] * np[1];
+        float v = dead ? 0.0f : p[i] * ip;
         if (cast) v = round_e4m3(v, nullptr);
         V[(size_t)j * n + i] = v;
         v1[i] = v;
     }
-    if (i == 0) sigma[j] = dead ? 0.0f : np[0];
+    if (i == 0) sigma[j] = dead ? 0.0f : sqrtf(s_np);
 }
 
 // W <- W - sigma_j u1 v1^T
@@ -148,7 +160,7 @@ __global__ void __launch_bounds__(256) deflate_kernel(float* __restrict__ W, int
 }
 
 struct R1Workspace {
-    float *y, *p, *u1, *v1, *ny, *np, *partial;
+    float *y, *p, *u1, *v1, *partial;
     int slabs;
     size_t total;
 };
@@ -166,8 +178,6 @@ R1Workspace r1svd_workspace(int m, int n, uint8_t* base) {
     w.p = take((size_t)n * 4);
     w.u1 = take((size_t)m * 4);
     w.v1 = take((size_t)n * 4);
-    w.ny = take(8);
-    w.np = take(8);
     w.partial = take((size_t)w.slabs * n * 4);
     w.total = off;
     return w;
@@ -180,21 +190,18 @@ cudaError_t run_r1svd(float* w, int m, int n, int r, int it, const float* sketch
     const dim3 g_sum((n + 255) / 256);
     const dim3 g_fin((max(m, n) + 255) / 256);
     const dim3 g_def(m, (n / 4 + 255) / 256);
-    auto cols = [&](const float* yv, const float* scale) {
-        gemv_cols_kernel<<<g_cols, 256, 0, s>>>(w, m, n, yv, scale, ws.partial);
-        colsum_kernel<<<g_sum, 256, 0, s>>>(ws.partial, ws.slabs, n, ws.p);
-        norm_kernel<<<1, kNormThreads, 0, s>>>(ws.p, n, ws.np);
+    auto cols = [&]() {  // p = W^T y / |y|
+        gemv_cols_kernel<<<g_cols, 256, 0, s>>>(w, m, n, ws.y, ws.partial);
+        colsum_kernel<<<g_sum, 256, 0, s>>>(ws.partial, ws.slabs, n, ws.y, m, ws.p);
     };
     for (int j = 0; j < r; ++j) {
-        gemv_rows_kernel<<<g_rows, kGemvThreads, 0, s>>>(w, m, n, sketches + (size_t)j * n, nullptr, ws.y);
-        norm_kernel<<<1, kNormThreads, 0, s>>>(ws.y, m, ws.ny);
+        gemv_rows_kernel<<<g_rows, kGemvThreads, 0, s>>>(w, m, n, sketches + (size_t)j * n, ws.y);  // y = W v / |v|
         for (int k = 0; k < it; ++k) {
-            cols(ws.y, ws.ny + 1);                                                              // p = W^T y^
-            gemv_rows_kernel<<<g_rows, kGemvThreads, 0, s>>>(w, m, n, ws.p, ws.np + 1, ws.y);  // y = W p^
-            norm_kernel<<<1, kNormThreads, 0, s>>>(ws.y, m, ws.ny);
+            cols();
+            gemv_rows_kernel<<<g_rows, kGemvThreads, 0, s>>>(w, m, n, ws.p, ws.y);                  // y = W p / |p|
         }
-        cols(ws.y, ws.ny + 1);  // p = W^T y^, |p| = sigma
-        finish_rank_kernel<<<g_fin, 256, 0, s>>>(ws.y, ws.p, ws.ny, ws.np, m, n, r, j, cast, U, sigma, V, ws.u1, ws.v1);
+        cols();  // |p| = sigma
+        finish_rank_kernel<<<g_fin, 256, 0, s>>>(ws.y, ws.p, m, n, r, j, cast, U, sigma, V, ws.u1, ws.v1);
         deflate_kernel<<<g_def, 256, 0, s>>>(w, m, n, ws.u1, ws.v1, sigma + j);
     }
     return cudaGetLastError();
