@@ -16,15 +16,6 @@ constexpr int kSlabRows = 32;      // rows of W per CTA in the transposed produc
 
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-// Sum of squares of a vector by one warp: lanes strided, then a butterfly -- every warp that calls this on the same
-// vector gets the same bits.
-__device__ __forceinline__ float warp_sumsq(const float* __restrict__ v, int len, int lane) {
-    float acc = 0.0f;
-    for (int i = lane; i < len; i += 32) acc = fmaf(v[i], v[i], acc);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    return acc;
-}
 __device__ __forceinline__ float inv_norm(float sumsq) {
     const float nrm = sqrtf(sumsq);
     return (nrm > 0.0f && isfinite(nrm)) ? 1.0f / nrm : 0.0f;
@@ -84,20 +75,34 @@ __global__ void __launch_bounds__(256) gemv_cols_kernel(const float* __restrict_
     reinterpret_cast<float4*>(partial + (size_t)slab * n)[c4] = acc;
 }
 
-// p[k] = (sum over slabs, ascending, of partial[slab][k]) / |y|; the first warp of every CTA forms |y|^2.
+// p[k] = (sum over slabs of partial[slab][k]) / |y|.  A CTA owns 32 columns; warp w adds the slabs w, w + 8, ... of
+// those columns (128-byte rows of the partial sums), the eight sums meet in shared memory in the order of w.  While
+// the other warps start on the slabs, every warp also takes an eighth of |y|^2 (lanes strided, fixed order).
 __global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ partial, int slabs, int n,
                                                      const float* __restrict__ y, int m, float* __restrict__ p) {
-    __shared__ float s_inv;
-    if (threadIdx.x < 32) {
-        const float ss = warp_sumsq(y, m, threadIdx.x);
-        if (threadIdx.x == 0) s_inv = inv_norm(ss);
-    }
-    __syncthreads();
-    const int k = blockIdx.x * 256 + threadIdx.x;
-    if (k >= n) return;
+    __shared__ float s_part[8][32];
+    __shared__ float s_sq[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int k = blockIdx.x * 32 + lane;
     float acc = 0.0f;
-    for (int s = 0; s < slabs; ++s) acc += partial[(size_t)s * n + k];
-    p[k] = acc * s_inv;
+    if (k < n)
+        for (int s = warp; s < slabs; s += 8) acc += partial[(size_t)s * n + k];
+    s_part[warp][lane] = acc;
+    float sq = 0.0f;
+    for (int i = warp * 32 + lane; i < m; i += 256) sq = fmaf(y[i], y[i], sq);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if (lane == 0) s_sq[warp] = sq;
+    __syncthreads();
+    if (warp == 0 && k < n) {
+        float total = 0.0f, ss = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            total += s_part[w][lane];
+            ss += s_sq[w];
+        }
+        p[k] = total * inv_norm(ss);
+    }
 }
 
 // fp32 -> nearest fp8 e4m3 value (ties to even, saturating), returned as fp32; bits optionally kept.
@@ -110,17 +115,37 @@ __device__ __forceinline__ float round_e4m3(float x, unsigned char* bits) {
 }
 
 // Rank j is done: U[:, j] = y / |y|, V[j, :] = p / |p| (cast to fp8 values when asked), sigma[j] = |p| where
-// p = W^T (y / |y|).  Every CTA forms the two norms itself.  A vanished y or p gives a zero triple.
+// p = W^T (y / |y|).  Every CTA forms the two norms itself (same order in every CTA, same bits).  A vanished y or p gives a zero triple.
 __global__ void __launch_bounds__(256) finish_rank_kernel(const float* __restrict__ y, const float* __restrict__ p,
                                                           int m, int n, int r, int j, int cast, float* __restrict__ U,
                                                           float* __restrict__ sigma, float* __restrict__ V,
                                                           float* __restrict__ u1, float* __restrict__ v1) {
+    __shared__ float s_sq[2][8];
     __shared__ float s_ny, s_np;
-    if (threadIdx.x < 32) {
-        const float a = warp_sumsq(y, m, threadIdx.x), b = warp_sumsq(p, n, threadIdx.x);
+    {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        float a = 0.0f, b = 0.0f;
+        for (int i = warp * 32 + lane; i < m; i += 256) a = fmaf(y[i], y[i], a);
+        for (int i = warp * 32 + lane; i < n; i += 256) b = fmaf(p[i], p[i], b);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, o);
+            b += __shfl_xor_sync(0xffffffffu, b, o);
+        }
+        if (lane == 0) {
+            s_sq[0][warp] = a;
+            s_sq[1][warp] = b;
+        }
+        __syncthreads();
         if (threadIdx.x == 0) {
-            s_ny = a;
-            s_np = b;
+            float sa = 0.0f, sb = 0.0f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                sa += s_sq[0][w];
+                sb += s_sq[1][w];
+            }
+            s_ny = sa;
+            s_np = sb;
         }
     }
     __syncthreads();
@@ -187,7 +212,7 @@ cudaError_t run_r1svd(float* w, int m, int n, int r, int it, const float* sketch
                       float* V, const R1Workspace& ws, cudaStream_t s) {
     const dim3 g_rows((m + kGemvThreads / 32 - 1) / (kGemvThreads / 32));
     const dim3 g_cols((n / 4 + 255) / 256, ws.slabs);
-    const dim3 g_sum((n + 255) / 256);
+    const dim3 g_sum((n + 31) / 32);
     const dim3 g_fin((max(m, n) + 255) / 256);
     const dim3 g_def(m, (n / 4 + 255) / 256);
     auto cols = [&]() {  // p = W^T y / |y|
