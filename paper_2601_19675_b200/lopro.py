@@ -26,7 +26,9 @@ SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packe
            "lopro_linear_fwd_path", "lopro_host_staging_bytes", "lopro_linear_fwd_host", "lopro_linear_fwd_noalloc",
            "lopro_configure", "lopro_selftest_wait", "lopro_group_workspace_bytes", "lopro_linear_fwd_group_path",
            "lopro_linear_fwd_group", "lopro_pack_lr8", "lopro_unpack_lr8", "lopro_r1svd_workspace_bytes", "lopro_r1svd",
-           "lopro_residual_rotate", "lopro_rtn_quantize", "lopro_quantize_workspace_bytes", "lopro_quantize_layer"]
+           "lopro_residual_rotate", "lopro_rtn_quantize", "lopro_quantize_workspace_bytes", "lopro_quantize_layer",
+           "lopro_block_add_rmsnorm", "lopro_block_rope_append", "lopro_block_attention_workspace_bytes",
+           "lopro_block_attention_decode", "lopro_block_silu_mul"]
 
 
 class Desc(ctypes.Structure):
@@ -112,6 +114,17 @@ def lib():
         L.lopro_quantize_workspace_bytes.argtypes = [dp]
         L.lopro_quantize_layer.restype = ctypes.c_int
         L.lopro_quantize_layer.argtypes = [dp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        f32 = ctypes.c_float
+        L.lopro_block_add_rmsnorm.restype = ctypes.c_int
+        L.lopro_block_add_rmsnorm.argtypes = [vp, i64, vp, i64, vp, f32, vp, i64, i32, i32, vp]
+        L.lopro_block_rope_append.restype = ctypes.c_int
+        L.lopro_block_rope_append.argtypes = [vp, i64, vp, i64, vp, i64, vp, vp, vp, i32, i32, i32, i32, f32, vp, vp]
+        L.lopro_block_attention_workspace_bytes.restype = sz
+        L.lopro_block_attention_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        L.lopro_block_attention_decode.restype = ctypes.c_int
+        L.lopro_block_attention_decode.argtypes = [vp, i64, vp, vp, vp, vp, i64, i32, i32, i32, i32, f32, vp, sz, vp, vp]
+        L.lopro_block_silu_mul.restype = ctypes.c_int
+        L.lopro_block_silu_mul.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, vp]
         _lib = L
     return _lib
 
@@ -311,6 +324,52 @@ def quantize_layer(desc, W, perm, sketches=None, it=8, s=None, workspace=None):
                                     _ptr(out["codes"]), _ptr(out["scales"]), _ptr(out["zeros"]), _ptr(lr[0]), _ptr(lr[1]),
                                     _ptr(lr[2]), _ptr(lr[3]), _ptr(workspace), workspace.numel(), _stream())
     _check(st, "lopro_quantize_layer")
+    return out
+
+
+def block_add_rmsnorm(h, y, w, eps, out=None):
+    """lopro_block_add_rmsnorm: h (bf16 [T][d], updated in place when y is given), y or None, w bf16 [d] -> out."""
+    T, d = h.shape
+    if out is None:
+        out = torch.empty((T, d), dtype=torch.bfloat16, device=h.device)
+    st = lib().lopro_block_add_rmsnorm(_ptr(h), h.stride(0), _ptr(y), 0 if y is None else y.stride(0), _ptr(_dev(w, 2)), eps,
+                                       _ptr(out), out.stride(0), T, d, _stream())
+    _check(st, "lopro_block_add_rmsnorm")
+    return out
+
+
+def block_rope_append(q, k, v, pos, k_cache, v_cache, theta, status):
+    """lopro_block_rope_append: q rotated in place; rotated k and v stored at entry pos[t] of the caches
+    [T][heads][ctx_max][head_dim]."""
+    T, n_heads, ctx_max, head_dim = k_cache.shape
+    st = lib().lopro_block_rope_append(_ptr(q), q.stride(0), _ptr(k), k.stride(0), _ptr(v), v.stride(0), _ptr(_dev(pos, 4)),
+                                       _ptr(_dev(k_cache, 2)), _ptr(_dev(v_cache, 2)), T, n_heads, head_dim, ctx_max, theta,
+                                       _ptr(status), _stream())
+    _check(st, "lopro_block_rope_append")
+
+
+def block_attention_workspace_bytes(T, n_heads, head_dim, ctx_max):
+    return lib().lopro_block_attention_workspace_bytes(T, n_heads, head_dim, ctx_max)
+
+
+def block_attention_decode(q, k_cache, v_cache, ctx, scale, workspace, status, out=None):
+    """lopro_block_attention_decode: q bf16 [T][heads * head_dim] against the caches; ctx int32 [T] valid entries."""
+    T, n_heads, ctx_max, head_dim = k_cache.shape
+    if out is None:
+        out = torch.empty((T, n_heads * head_dim), dtype=torch.bfloat16, device=q.device)
+    st = lib().lopro_block_attention_decode(_ptr(q), q.stride(0), _ptr(_dev(k_cache, 2)), _ptr(_dev(v_cache, 2)),
+                                            _ptr(_dev(ctx, 4)), _ptr(out), out.stride(0), T, n_heads, head_dim, ctx_max, scale,
+                                            _ptr(workspace), workspace.numel(), _ptr(status), _stream())
+    _check(st, "lopro_block_attention_decode")
+    return out
+
+
+def block_silu_mul(gate, up, out=None):
+    T, d = gate.shape
+    if out is None:
+        out = torch.empty((T, d), dtype=torch.bfloat16, device=gate.device)
+    st = lib().lopro_block_silu_mul(_ptr(gate), gate.stride(0), _ptr(up), up.stride(0), _ptr(out), out.stride(0), T, d, _stream())
+    _check(st, "lopro_block_silu_mul")
     return out
 
 
