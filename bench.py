@@ -45,7 +45,12 @@ WORKLOADS = {
     # attention, norms and activations are not part of the method and are not run
     "cfg5_T1": ("cfg5", 1, 224),
     "cfg5_T32": ("cfg5", 32, 224),
+    # the same stack as a whole decode step: the linears chained through residual + RMS norm, rotary embedding, attention of
+    # the new token over a 2048-token key/value cache per sequence, SiLU gating (plain kernels of this library)
+    "cfg5_T1_block": ("cfg5", 1, 224),
+    "cfg5_T32_block": ("cfg5", 32, 224),
 }
+STACK_HEADS, STACK_HEAD_DIM, STACK_CONTEXT = 32, 128, 2048
 # linears of one layer of the stack: name, d_in, d_out (hidden 4096, MLP 11008)
 STACK_LINEARS = [("q", 4096, 4096), ("k", 4096, 4096), ("v", 4096, 4096), ("o", 4096, 4096),
                  ("gate", 4096, 11008), ("up", 4096, 11008), ("down", 11008, 4096)]
@@ -55,6 +60,12 @@ STACK_QUANT = dict(bits=4, group_size=128, block_size=128, identity_cols=128, ra
 
 def stack_shape(n, m):
     return dict(d_in=n, d_out=m, **STACK_QUANT)
+
+
+def block_glue_bytes(T):
+    """HBM bytes of the decoder-block operations of one decode step: the key/value cache (keys and values of the
+    context plus the new token, bf16) dominates; the activation rows between the kernels stay in L2."""
+    return STACK_LAYERS * T * STACK_HEADS * (STACK_CONTEXT + 1) * STACK_HEAD_DIM * 2 * 2
 
 
 def stack_bytes(T):
@@ -262,6 +273,14 @@ def run_reference(args):
 def workload_config(name):
     from paper_2601_19675_b200 import synth
     cfg, T, ring = WORKLOADS[name]
+    if cfg == "cfg5" and name.endswith("_block"):
+        return dict(workload=f"{name}: one decode step of a 32-layer decoder stack (hidden 4096, MLP 11008, 32 heads x 128; the 224 "
+                             f"linears LoPRo 4-bit g128 block 128 rank 32), batch {T}, one new token per sequence over a "
+                             f"{STACK_CONTEXT}-token bf16 key/value cache; norms, rotary embedding, attention and gating by this "
+                             "library's plain kernels; no embedding, final norm or vocabulary projection",
+                    tokens=T, ring_layers=ring,
+                    l2="inputs larger than L2: one step reads %.0f MB of packed weights and %.0f MB of key/value cache"
+                       % (stack_bytes(T) / 1e6, block_glue_bytes(T) / 1e6))
     if cfg == "cfg5":
         return dict(workload=f"{name}: the 224 LoPRo linears of a 32-layer decoder stack (hidden 4096, MLP 11008; 4-bit g128 "
                              f"block 128 rank 32), batch {T}, one token per sequence; attention/norm/activation glue not run",
@@ -363,6 +382,10 @@ class Workload:
                     part = [L7[k] for k in idx]
                     self.calls.append(([g[0] for g in part], [g[1] for g in part], part[0][2], [g[3] for g in part]))
             self.x_dev, self.x_host_bits, self.y_last = xs[4096], self.x_bits[4096], self.calls[-1][3][-1]
+            self.block = name.endswith("_block")
+            self.ws_holder = [None]
+            if self.block:
+                self.build_block(linears, rank)
             self.forwards = len(linears)
             self.tokens_per_pass = T
             self.bytes_per_pass = stack_bytes(T)
@@ -370,9 +393,13 @@ class Workload:
             self.h2d, self.d2h = T * 4096 * 2, T * self.y_last.shape[1] * 2
             ws_bytes = max(lopro.group_workspace_bytes(c[0], T) for c in self.calls)
             self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+            self.ws_holder[0] = self.ws
             self.paths = sorted({lopro.PATH_NAMES.get(lopro.linear_fwd_path(d, T)[0], "?") for d, _, _, _ in linears})
             self.launches_per_pass = sum(lopro.linear_fwd_group_path(c[0], T)[1] if len(c[0]) > 1
                                          else lopro.linear_fwd_path(c[0][0], T)[1] for c in self.calls)
+            if self.block:
+                self.bytes_per_pass += block_glue_bytes(T)
+                self.launches_per_pass += 6 * STACK_LAYERS      # 2 norms, rotary + append, attention (2), gating
             self.c = None
             return
         c = synth.CONFIGS[cfg]
@@ -417,8 +444,59 @@ class Workload:
         self.paths = [lopro.PATH_NAMES.get(path, "?")]
         self.launches_per_pass = per_forward * ring
 
+    def build_block(self, linears, rank):
+        """Buffers and call list of a whole decode step: per layer norm -> (q, k, v) -> rotary + cache append -> attention
+        -> o -> residual + norm -> (gate, up) -> gating -> down; the residual of `down` is added by the next layer's norm."""
+        torch, lopro, dev, T = self.torch, self.lopro, self.dev, self.T
+        from paper_2601_19675_b200 import synth
+        H, hd, C = STACK_HEADS, STACK_HEAD_DIM, STACK_CONTEXT + 1
+        bf = torch.bfloat16
+        buf = lambda d: torch.empty((T, d), dtype=bf, device=dev)
+        self.h0, self.h, self.xn = self.x_dev, buf(4096), buf(4096)
+        q, k, v, attn, o = buf(4096), buf(4096), buf(4096), buf(4096), buf(4096)
+        gate, up, act, down = buf(11008), buf(11008), buf(11008), buf(4096)
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1234 + rank)
+        caches = []
+        for _ in range(STACK_LAYERS):           # random keys and values of the 2048-token context, one cache per layer
+            kc = torch.empty((T, H, C, hd), dtype=bf, device=dev).normal_(generator=gen)
+            vc = torch.empty((T, H, C, hd), dtype=bf, device=dev).normal_(generator=gen)
+            caches.append((kc, vc))
+        norm_w = torch.from_numpy(synth.f32_to_bf16_bits(
+            1.0 + 0.1 * synth.weights(2 * STACK_LAYERS, 4096, seed=77 + rank, std=1.0)).view(np.int16)).to(dev).view(bf)
+        pos = torch.full((T,), STACK_CONTEXT, dtype=torch.int32, device=dev)
+        ctx = torch.full((T,), C, dtype=torch.int32, device=dev)
+        self.block_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        attn_ws = torch.empty(lopro.block_attention_workspace_bytes(T, H, hd, C), dtype=torch.uint8, device=dev)
+        scale = 1.0 / float(np.sqrt(hd))
+        ws, st = self.ws_holder, self.block_status
+        steps = [lambda: self.h.copy_(self.h0)]
+        for li in range(STACK_LAYERS):
+            L7 = linears[li * 7:(li + 1) * 7]
+            ds, bl = [g[0] for g in L7], [g[1] for g in L7]
+            kc, vc = caches[li]
+            w1, w2 = norm_w[2 * li], norm_w[2 * li + 1]
+            prev = down if li else None
+            steps += [
+                lambda prev=prev, w1=w1: lopro.block_add_rmsnorm(self.h, prev, w1, 1e-5, out=self.xn),
+                lambda ds=ds, bl=bl: lopro.linear_fwd_group(ds[0:3], bl[0:3], self.xn, lopro.OUT_BF16, workspace=ws[0], ys=[q, k, v]),
+                lambda kc=kc, vc=vc: lopro.block_rope_append(q, k, v, pos, kc, vc, 10000.0, st),
+                lambda kc=kc, vc=vc: lopro.block_attention_decode(q, kc, vc, ctx, scale, attn_ws, st, out=attn),
+                lambda ds=ds, bl=bl: lopro.linear_fwd(ds[3], bl[3], attn, lopro.OUT_BF16, workspace=ws[0], y=o),
+                lambda w2=w2: lopro.block_add_rmsnorm(self.h, o, w2, 1e-5, out=self.xn),
+                lambda ds=ds, bl=bl: lopro.linear_fwd_group(ds[4:6], bl[4:6], self.xn, lopro.OUT_BF16, workspace=ws[0], ys=[gate, up]),
+                lambda: lopro.block_silu_mul(gate, up, out=act),
+                lambda ds=ds, bl=bl: lopro.linear_fwd(ds[6], bl[6], act, lopro.OUT_BF16, workspace=ws[0], y=down),
+            ]
+        self.block_steps = steps
+        self.y_last = down
+
     def one_pass(self):
         lopro = self.lopro
+        if getattr(self, "block", False):
+            for f in self.block_steps:
+                f()
+            return
         for ds, blobs, x, ys in self.calls:
             if len(ds) == 1:
                 lopro.linear_fwd(ds[0], blobs[0], x, lopro.OUT_BF16, workspace=self.ws, y=ys[0])
@@ -429,6 +507,15 @@ class Workload:
         """Untimed: every forward of the pass on its own, the device status word read after each of them (a forward
         resets the word when it starts, so reading it once at the end would report the last forward only)."""
         lopro, torch = self.lopro, self.torch
+        if getattr(self, "block", False):
+            for k, f in enumerate(self.block_steps):
+                f()
+                torch.cuda.current_stream().synchronize()
+                status = lopro.workspace_status(self.ws)
+                assert status == lopro.OK, f"device status {status} after step {k} of {self.name}"
+                assert int(self.block_status.item()) == lopro.OK, f"block status after step {k} of {self.name}"
+            assert torch.isfinite(self.y_last.float()).all() and torch.isfinite(self.h.float()).all()
+            return
         for k, (ds, blobs, x, ys) in enumerate(self.calls):
             if len(ds) == 1:
                 lopro.linear_fwd(ds[0], blobs[0], x, lopro.OUT_BF16, workspace=self.ws, y=ys[0])
@@ -540,6 +627,10 @@ def measure(args, name, steps, warmup, rank, world, local, dev, dist, with_e2e=T
                          "prefill": "prefill_kernel", "rowblock": "rowblock_kernel"}.get(n, n) for n in w.paths)
     note = ("duration = step time / layer forwards (includes the prologue kernels of each forward): an upper bound on the "
             "product kernel's own duration, a lower bound on `achieved`")
+    if getattr(w, "block", False):
+        kernel += " + attention_split_kernel"
+        note = ("whole decode step: bytes = packed weights + key/value cache, duration = step time / 224 linears (every kernel of "
+                "the step included)")
     if w.T <= 64:
         ach = w.bytes_per_pass / (ms_per_pass * 1e-3) / 1e9
         roofline = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
@@ -570,7 +661,7 @@ def measure(args, name, steps, warmup, rank, world, local, dev, dist, with_e2e=T
 
 # workloads reported beside the bench line (driver-run evidence for every regime), with the steps each gets
 EXTRA_WORKLOADS = [("cfg2_T1", 5), ("cfg2_T32", 5), ("cfg4_T16", 5), ("cfg5_T1", 5), ("cfg5_T32", 5), ("cfg3_T2048", 5),
-                   ("cfg4_T4096", 4)]
+                   ("cfg4_T4096", 4), ("cfg5_T1_block", 5), ("cfg5_T32_block", 4)]
 
 
 def measure_offline(dev, peaks, reps=3):
