@@ -35,7 +35,7 @@ LOPRO_API lopro_status lopro_block_rope_append(uint16_t* q, int64_t ldq, const u
                                                void* status_word, void* stream);
 
 /* out[t, h] = sum_j softmax_j(q[t, h] . K[t, h, j] * scale) V[t, h, j] over j < ctx[t] (1 <= ctx[t] <= ctx_max, else
- * LOPRO_ERR_INVALID_DATA in *status_word and zeros).  The keys are split into pieces of 256; a second launch merges the
+ * LOPRO_ERR_INVALID_DATA in *status_word and zeros).  The keys are split into pieces of 256 (128 for small batches); a second launch merges the
  * pieces' partial soft-max sums.  head_dim = 128.  workspace: lopro_block_attention_workspace_bytes(...) bytes of
  * device memory, 256-byte aligned.  out [T][n_heads * head_dim] (ldo). */
 LOPRO_API size_t lopro_block_attention_workspace_bytes(int32_t T, int32_t n_heads, int32_t head_dim, int32_t ctx_max);

@@ -11,7 +11,7 @@
 
 namespace {
 
-constexpr int kSplitKeys = 256;   // keys per attention CTA
+constexpr int kSplitKeys = 256;   // keys per attention CTA (128 when that is needed to fill the GPU)
 constexpr int kHeadDim = 128;     // the attention kernels are written for this head size
 constexpr int kPartial = kHeadDim + 2;  // per (token, head, split): running max, sum of weights, weighted values
 
@@ -92,19 +92,19 @@ __global__ void rope_append_kernel(__nv_bfloat16* __restrict__ q, int64_t ldq, c
     *reinterpret_cast<__nv_bfloat162*>(v_cache + entry) = *reinterpret_cast<const __nv_bfloat162*>(v + (size_t)t * ldv + col);
 }
 
-// grid (n_heads, T, splits), 128 threads.  A CTA takes keys [256 z, 256 z + 256) of one (sequence, head):
+// grid (n_heads, T, splits), 128 threads.  A CTA takes split_keys (256 or 128) consecutive keys of one (sequence, head):
 // scores with one key per thread (its 256-byte row in 16-byte loads), soft-max weights of the piece against the
 // piece's own maximum, then the weighted values with two dimensions per thread and the keys split by parity.
 __global__ void __launch_bounds__(128) attention_split_kernel(const __nv_bfloat16* __restrict__ q, int64_t ldq,
                                                               const __nv_bfloat16* __restrict__ k_cache,
                                                               const __nv_bfloat16* __restrict__ v_cache,
                                                               const int32_t* __restrict__ ctx, int n_heads, int ctx_max,
-                                                              int splits, float scale, float* __restrict__ partial,
-                                                              int* status) {
+                                                              int splits, int split_keys, float scale,
+                                                              float* __restrict__ partial, int* status) {
     __shared__ __align__(16) float qs[kHeadDim];
     __shared__ float ps[kSplitKeys];
     __shared__ float red[4];
-    __shared__ float2 half_acc[64];
+    __shared__ float group_acc[8][kHeadDim];
     const int hd = blockIdx.x, t = blockIdx.y, z = blockIdx.z, tid = threadIdx.x;
     float* out = partial + (((size_t)t * n_heads + hd) * splits + z) * kPartial;
     const int n = ctx[t];
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(128) attention_split_kernel(const __nv_bfloat1
         if (tid == 0) out[1] = 0.0f;  // an empty piece
         return;
     }
-    const int j0 = z * kSplitKeys, cnt = min(kSplitKeys, n - j0);
+    const int j0 = z * split_keys, cnt = min(split_keys, n - j0);
     if (cnt <= 0) {
         if (tid == 0) out[1] = 0.0f;
         return;
@@ -147,21 +147,33 @@ __global__ void __launch_bounds__(128) attention_split_kernel(const __nv_bfloat1
         sum += p;
     }
     sum = block_sum(sum, red);  // also orders the writes of ps before the reads below
-    const int pair = tid & 63, par = tid >> 6;
-    float2 acc = make_float2(0.0f, 0.0f);
-    const __nv_bfloat162* vr = reinterpret_cast<const __nv_bfloat162*>(v_cache + (base + j0) * kHeadDim) + pair;
-#pragma unroll 4
-    for (int j = par; j < cnt; j += 2) {
-        const float2 f = __bfloat1622float2(vr[(size_t)j * (kHeadDim / 2)]);
+    // weighted values: sixteen threads cover a 256-byte row with 16-byte loads, the eight groups of sixteen take the
+    // keys j = group, group + 8, ...; the groups' sums meet in shared memory in the order of the groups
+    const int piece = tid & 15, group = tid >> 4;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+    const uint4* vr = reinterpret_cast<const uint4*>(v_cache + (base + j0) * kHeadDim) + piece;
+#pragma unroll 8
+    for (int j = group; j < cnt; j += 8) {
+        const uint4 u = __ldg(vr + (size_t)j * (kHeadDim / 8));
+        const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&u);
         const float p = ps[j];
-        acc.x = fmaf(p, f.x, acc.x);
-        acc.y = fmaf(p, f.y, acc.y);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(b[e]);
+            acc[2 * e] = fmaf(p, f.x, acc[2 * e]);
+            acc[2 * e + 1] = fmaf(p, f.y, acc[2 * e + 1]);
+        }
     }
-    if (par == 1) half_acc[pair] = acc;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) group_acc[group][8 * piece + e] = acc[e];
     __syncthreads();
-    if (par == 0) {
-        out[2 + 2 * pair] = acc.x + half_acc[pair].x;
-        out[2 + 2 * pair + 1] = acc.y + half_acc[pair].y;
+    {
+        float total = 0.0f;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) total += group_acc[g][tid];
+        out[2 + tid] = total;
     }
     if (tid == 0) {
         out[0] = mx;
@@ -246,7 +258,7 @@ lopro_status lopro_block_rope_append(uint16_t* q, int64_t ldq, const uint16_t* k
 
 size_t lopro_block_attention_workspace_bytes(int32_t T, int32_t n_heads, int32_t head_dim, int32_t ctx_max) {
     if (T < 0 || n_heads < 1 || head_dim != kHeadDim || ctx_max < 1) return 0;
-    const size_t splits = ((size_t)ctx_max + kSplitKeys - 1) / kSplitKeys;
+    const size_t splits = ((size_t)ctx_max + kSplitKeys / 2 - 1) / (kSplitKeys / 2);  // the finer of the two splits
     return ((size_t)T * n_heads * splits * kPartial * sizeof(float) + 255) / 256 * 256 + 256;
 }
 
@@ -258,7 +270,9 @@ lopro_status lopro_block_attention_decode(const uint16_t* q, int64_t ldq, const 
     if (head_dim != kHeadDim) return LOPRO_ERR_UNSUPPORTED;
     if (T == 0) return LOPRO_OK;
     const int64_t width = (int64_t)n_heads * head_dim;
-    const int splits = (ctx_max + kSplitKeys - 1) / kSplitKeys;
+    // pieces of 256 keys, or of 128 when there would be too few CTAs for the GPU otherwise
+    const int split_keys = (int64_t)T * n_heads * ((ctx_max + kSplitKeys - 1) / kSplitKeys) < 1024 ? kSplitKeys / 2 : kSplitKeys;
+    const int splits = (ctx_max + split_keys - 1) / split_keys;
     if (!q || !k_cache || !v_cache || !ctx || !out || !workspace || !status_word || ldq < width || ldo < width || T > 65535 ||
         splits > 65535)
         return LOPRO_ERR_INVALID_ARG;
@@ -268,7 +282,7 @@ lopro_status lopro_block_attention_decode(const uint16_t* q, int64_t ldq, const 
     float* partial = reinterpret_cast<float*>(workspace);
     attention_split_kernel<<<dim3(n_heads, T, splits), 128, 0, s>>>(
         reinterpret_cast<const __nv_bfloat16*>(q), ldq, reinterpret_cast<const __nv_bfloat16*>(k_cache),
-        reinterpret_cast<const __nv_bfloat16*>(v_cache), ctx, n_heads, ctx_max, splits, scale, partial, (int*)status_word);
+        reinterpret_cast<const __nv_bfloat16*>(v_cache), ctx, n_heads, ctx_max, splits, split_keys, scale, partial, (int*)status_word);
     attention_merge_kernel<<<dim3(n_heads, T), 128, 0, s>>>(partial, n_heads, splits, reinterpret_cast<__nv_bfloat16*>(out), ldo);
     return cudaGetLastError() == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }
