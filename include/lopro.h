@@ -252,7 +252,7 @@ LOPRO_API int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32
  *   n_layers >= 1; descs[i], packed[i], y[i], ldy[i] per layer (host arrays of n_layers entries); all layers have
  *   the same d_in; x, out_dtype, T as for lopro_linear_fwd; workspace of lopro_group_workspace_bytes(...) bytes,
  *   256-byte aligned.  The status word of the group is the first word of the workspace.
- * When the layers differ in nothing but d_out and their data, are in LOPRO_LAYOUT_FRAGMENT, n_layers <= 4, T <= 32 and
+ * When the layers differ in nothing but d_out and their data, are in LOPRO_LAYOUT_FRAGMENT, n_layers <= 8, T <= 32 and
  * each would run as prologue + small-batch kernel of the same kind (all per-row-group, or all persistent: the
  * persistent CTAs are then shared out in proportion to the layers' rows), the group runs as TWO launches: one
  * prologue that writes every layer's rotated activations and B_i x, and one product launch over the row tiles of
@@ -310,6 +310,30 @@ LOPRO_API lopro_status lopro_linear_fwd_noalloc(const lopro_desc* desc, const vo
  * short limit (4096 polls), and on expiry stores LOPRO_ERR_TIMEOUT in *status_word (device memory, 4 bytes,
  * 4-byte aligned; the kernel first stores LOPRO_OK there).  Asynchronous: read the word after synchronising. */
 LOPRO_API lopro_status lopro_selftest_wait(void* status_word, void* stream);
+
+/* Forward of the EXPERTS of a mixture-of-experts layer (the paper quantizes Mixtral-8x7B expert by expert and lists
+ * MoE models among its evaluations): n_experts layers of one shape (`desc`), each with its own packed record, and a
+ * batch of token rows already grouped by expert, as a router's sort leaves them: expert e owns rows
+ * [row_offsets[e], row_offsets[e+1]) of x and of y (row_offsets: HOST array of n_experts + 1 non-decreasing entries,
+ * row_offsets[0] = 0; an expert without rows is skipped).  y[t] = A_e (B_e x[t]) + W^_e (Q^T P_e^T x[t]) for the rows
+ * t of expert e (Eq. 8 per expert).
+ *   x [rows][d_in] bf16 (ldx), y [rows][d_out] (ldy, out_dtype); workspace of
+ *   lopro_experts_workspace_bytes(desc, n_experts, max_rows) bytes, max_rows >= the largest row count of an expert,
+ *   256-byte aligned.
+ * When no expert has more than 32 rows and the layer runs through the small-batch kernels (LOPRO_LAYOUT_FRAGMENT,
+ * folded fp16 record), every 8 experts with rows run as TWO launches: one prologue (each expert its own permutation,
+ * B and rows) and one product launch over the row tiles of all of them, both shaped for the largest row count.
+ * Otherwise the experts run one after the other.  Status words: the first word of the workspace for the first 8
+ * experts with rows, the first word of the k-th such expert's region (workspace_bytes / n_experts each) for the
+ * next 8, and so on; in the one-after-the-other case every expert's region starts with its own.
+ * lopro_linear_fwd_experts_path returns 2 / 1 for the two cases (0 on bad arguments) and the number of launches. */
+LOPRO_API size_t lopro_experts_workspace_bytes(const lopro_desc* desc, int32_t n_experts, int32_t max_rows);
+LOPRO_API int32_t lopro_linear_fwd_experts_path(const lopro_desc* desc, int32_t n_experts, const int32_t* row_offsets,
+                                                int32_t* launches);
+LOPRO_API lopro_status lopro_linear_fwd_experts(const lopro_desc* desc, int32_t n_experts, const void* const* packed,
+                                                const int32_t* row_offsets, const uint16_t* x_bf16, int64_t ldx, void* y,
+                                                int64_t ldy, int32_t out_dtype, void* workspace, size_t workspace_bytes,
+                                                void* stream);
 
 /* ---------------------------------------------------------------------------------------------------
  * Offline side of the method on the GPU (Algorithm 1 without its calibration inputs): the step BEFORE the forward

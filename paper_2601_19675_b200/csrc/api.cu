@@ -637,6 +637,143 @@ lopro_status lopro_linear_fwd_group(int32_t n_layers, const lopro_desc* const* d
     return e == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }
 
+// ---- experts of a mixture layer: the same layer shape, each expert its own rows of x and y -----------------------
+
+static bool experts_share_launches(const lopro_desc& d, int max_rows) {
+    if (max_rows < 1 || max_rows > kDecodeMaxT) return false;
+    if (d.layout != LOPRO_LAYOUT_FRAGMENT || d.lowrank_format != LOPRO_LOWRANK_FOLDED_F16) return false;
+    if (!prologue_supported(d, max_rows)) return false;
+    return use_tall(d, max_rows) || stream_supported(d, max_rows);
+}
+
+static lopro_status check_expert_rows(int32_t n_experts, const int32_t* row_offsets, int* max_rows, int* active) {
+    if (n_experts < 1 || !row_offsets || row_offsets[0] != 0) return LOPRO_ERR_INVALID_ARG;
+    int mx = 0, act = 0;
+    for (int e = 0; e < n_experts; ++e) {
+        const int cnt = row_offsets[e + 1] - row_offsets[e];
+        if (cnt < 0) return LOPRO_ERR_INVALID_ARG;
+        if (cnt > mx) mx = cnt;
+        if (cnt > 0) ++act;
+    }
+    *max_rows = mx;
+    *active = act;
+    return LOPRO_OK;
+}
+
+size_t lopro_experts_workspace_bytes(const lopro_desc* desc, int32_t n_experts, int32_t max_rows) {
+    if (!desc || n_experts < 1 || max_rows < 0 || check_desc(*desc) != LOPRO_OK) return 0;
+    const size_t region = group_region_bytes(*desc, max_rows < 1 ? 1 : max_rows);
+    return region == 0 ? 0 : region * (size_t)n_experts;
+}
+
+int32_t lopro_linear_fwd_experts_path(const lopro_desc* desc, int32_t n_experts, const int32_t* row_offsets, int32_t* launches) {
+    int max_rows = 0, active = 0;
+    if (!desc || check_desc(*desc) != LOPRO_OK || check_expert_rows(n_experts, row_offsets, &max_rows, &active) != LOPRO_OK)
+        return 0;
+    if (active == 0) {
+        if (launches) *launches = 0;
+        return 1;
+    }
+    if (experts_share_launches(*desc, max_rows)) {
+        if (launches) *launches = 2 * ((active + kMaxSiblings - 1) / kMaxSiblings);
+        return 2;
+    }
+    int32_t total = 0;
+    for (int e = 0; e < n_experts; ++e) {
+        const int cnt = row_offsets[e + 1] - row_offsets[e];
+        int32_t one = 0;
+        if (cnt > 0 && lopro_linear_fwd_path(desc, cnt, &one) == 0) return 0;
+        total += cnt > 0 ? one : 0;
+    }
+    if (launches) *launches = total;
+    return 1;
+}
+
+lopro_status lopro_linear_fwd_experts(const lopro_desc* desc, int32_t n_experts, const void* const* packed,
+                                      const int32_t* row_offsets, const uint16_t* x_bf16, int64_t ldx, void* y, int64_t ldy,
+                                      int32_t out_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!desc || !packed) return LOPRO_ERR_INVALID_ARG;
+    if (out_dtype != LOPRO_OUT_BF16 && out_dtype != LOPRO_OUT_F32) return LOPRO_ERR_INVALID_ARG;
+    lopro_status st = check_desc(*desc);
+    if (st != LOPRO_OK) return st;
+    const lopro_desc& d = *desc;
+    int max_rows = 0, active = 0;
+    st = check_expert_rows(n_experts, row_offsets, &max_rows, &active);
+    if (st != LOPRO_OK) return st;
+    if (active == 0) return LOPRO_OK;
+    const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;
+    if (!x_bf16 || !y || !workspace || ldx < d.d_in || (ldx % 8) || ldy < d.d_out || !aligned(x_bf16, 16) ||
+        !aligned(y, esz) || !aligned(workspace, 256))
+        return LOPRO_ERR_INVALID_ARG;
+    if (workspace_bytes < lopro_experts_workspace_bytes(desc, n_experts, max_rows)) return LOPRO_ERR_BUFFER_TOO_SMALL;
+    for (int e = 0; e < n_experts; ++e)
+        if (row_offsets[e + 1] > row_offsets[e] && (!packed[e] || !aligned(packed[e], 256))) return LOPRO_ERR_INVALID_ARG;
+    const size_t region = group_region_bytes(d, max_rows);
+    uint8_t* ws = (uint8_t*)workspace;
+    const __nv_bfloat16* x = (const __nv_bfloat16*)x_bf16;
+    auto rows_of_y = [&](int row) { return (void*)((uint8_t*)y + (size_t)row * (size_t)ldy * esz); };
+    if (!experts_share_launches(d, max_rows)) {
+        // expert by expert, each in its own region of the workspace
+        for (int e = 0; e < n_experts; ++e) {
+            const int r0 = row_offsets[e], cnt = row_offsets[e + 1] - r0;
+            if (cnt == 0) continue;
+            st = lopro_linear_fwd(desc, packed[e], x_bf16 + (size_t)r0 * ldx, ldx, rows_of_y(r0), ldy, out_dtype, cnt,
+                                  ws + (size_t)e * region, region, stream);
+            if (st != LOPRO_OK) return st;
+        }
+        return LOPRO_OK;
+    }
+    // up to kMaxSiblings experts per pair of launches: one prologue (every expert its own permutation, B and rows of
+    // x), one product launch over the row tiles of all of them; the launches are shaped for the largest row count
+    WorkspaceLayout W;
+    st = workspace_layout(d, max_rows, &W);
+    if (st != LOPRO_OK) return st;
+    BlobLayout L;
+    st = blob_layout(d, &L);
+    if (st != LOPRO_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    int e = 0;
+    while (e < n_experts) {
+        int ids[kMaxSiblings], n = 0;
+        for (; e < n_experts && n < kMaxSiblings; ++e)
+            if (row_offsets[e + 1] > row_offsets[e]) ids[n++] = e;
+        if (n == 0) break;
+        PrologueSiblings ps = {};
+        StreamSiblingArgs ss = {};
+        ps.n = ss.n = n - 1;
+        ps.own_rows = ss.own_rows = 1;
+        for (int i = 0; i < n; ++i) {
+            const int r0 = row_offsets[ids[i]], cnt = row_offsets[ids[i] + 1] - r0;
+            const uint8_t* blob = (const uint8_t*)packed[ids[i]];
+            uint8_t* wsi = ws + (size_t)ids[i] * region;
+            ps.x_of[i] = x + (size_t)r0 * ldx;
+            ps.T_of[i] = ss.T_of[i] = cnt;
+            if (i == 0) continue;
+            ps.perm[i - 1] = (const int32_t*)(blob + L.off[LOPRO_SEC_PERM]);
+            ps.B[i - 1] = (const __half*)(blob + L.off[LOPRO_SEC_B]);
+            ps.act[i - 1] = wsi + W.off_xrot;
+            ps.t[i - 1] = (__half*)(wsi + W.off_t);
+            ss.blob[i - 1] = blob;
+            ss.L[i - 1] = L;
+            ss.ws[i - 1] = wsi;
+            ss.y[i - 1] = rows_of_y(r0);
+            ss.ldy[i - 1] = ldy;
+            ss.d_out[i - 1] = d.d_out;
+        }
+        const uint8_t* blob0 = (const uint8_t*)packed[ids[0]];
+        uint8_t* ws0 = ws + (size_t)ids[0] * region;
+        if (launch_prologue(d, (const int32_t*)(blob0 + L.off[LOPRO_SEC_PERM]), (const __half*)(blob0 + L.off[LOPRO_SEC_B]),
+                            L.r_pad, ps.x_of[0], ldx, ws0 + W.off_xrot, (__half*)(ws0 + W.off_t), W.t_pad,
+                            (int*)(ws0 + W.off_status), max_rows, s, nullptr, &ps) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
+        void* y0 = rows_of_y(row_offsets[ids[0]]);
+        const cudaError_t err = use_tall(d, max_rows) ? launch_tall(d, blob0, L, ws0, W, y0, ldy, out_dtype, max_rows, s, 0, &ss)
+                                                      : launch_stream(d, blob0, L, ws0, W, y0, ldy, out_dtype, max_rows, s, 0, &ss);
+        if (err != cudaSuccess) return LOPRO_ERR_CUDA;
+    }
+    return LOPRO_OK;
+}
+
 size_t lopro_host_staging_bytes(const lopro_desc* desc, int32_t T, int32_t out_dtype) {
     if (!desc || check_desc(*desc) != LOPRO_OK || T < 0) return 0;
     const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;

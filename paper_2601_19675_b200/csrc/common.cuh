@@ -139,13 +139,18 @@ cudaError_t launch_rotate(const lopro_desc& d, const int32_t* perm, const __nv_b
 // Small-batch prologue: rotation, 64-column sums and t = B x in one launch.
 bool prologue_supported(const lopro_desc& d, int T);
 // Sibling layers of a grouped forward: they read the same x and differ only in their rows (d_out) and data.
-constexpr int kMaxSiblings = 4;
+constexpr int kMaxSiblings = 8;
 struct PrologueSiblings {  // siblings 1 .. n of a grouped prologue (sibling 0 travels in the ordinary arguments)
     int n;
     const int32_t* perm[kMaxSiblings - 1];
     const __half* B[kMaxSiblings - 1];
     unsigned char* act[kMaxSiblings - 1];
     __half* t[kMaxSiblings - 1];
+    // own_rows != 0 (experts of a mixture layer): sibling z = 0 .. n reads its own rows x_of[z] and has T_of[z] of
+    // them; the launch is shaped for the largest count and the siblings with fewer rows leave the rest idle
+    int own_rows;
+    const __nv_bfloat16* x_of[kMaxSiblings];
+    int T_of[kMaxSiblings];
 };
 // FP8 low-rank record: t = Sigma (V (x / s)) instead of t = B x (V null: folded fp16 format).
 struct Lr8Args {
@@ -185,6 +190,10 @@ struct StreamSiblingArgs {
     void* y[kMaxSiblings - 1];
     int64_t ldy[kMaxSiblings - 1];
     int d_out[kMaxSiblings - 1];
+    // own_rows != 0: token counts per sibling, T_of[0] for the layer of the ordinary arguments (whose T then only
+    // shapes the launch: the largest of the counts)
+    int own_rows;
+    int T_of[kMaxSiblings];
 };
 cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0 = 0,

@@ -351,15 +351,17 @@ constexpr int kPrologueMaxSmem = 200 * 1024;  // one row of x: d_in <= 102400
 // wait, everything is loaded after it.
 template <bool STAGED>
 __global__ void __launch_bounds__(256)
-prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm0,
+prologue_kernel(const __nv_bfloat16* __restrict__ x0, int64_t ldx, const int32_t* __restrict__ perm0,
                 const __half* __restrict__ B0, unsigned char* __restrict__ act_image0, __half* __restrict__ t0,
-                int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T,
+                int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T_grid,
                 int tpr, const ImageOut img, const PrologueSiblings sibs, const Lr8Args lr8) {
     // sibling layers (grid z): the same x, each layer its own permutation, B and outputs
     const int32_t* __restrict__ perm = perm0;
     const __half* __restrict__ B = B0;
     unsigned char* __restrict__ act_image = act_image0;
     __half* __restrict__ t = t0;
+    const __nv_bfloat16* __restrict__ x = x0;
+    int T = T_grid;  // T_grid shapes the grid; T is the number of token rows of this CTA's layer
 #pragma unroll
     for (int i = 0; i < kMaxSiblings - 1; ++i)
         if ((int)blockIdx.z == i + 1) {
@@ -368,12 +370,20 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t*
             act_image = sibs.act[i];
             t = sibs.t[i];
         }
+    if (sibs.own_rows) {
+#pragma unroll
+        for (int i = 0; i < kMaxSiblings; ++i)
+            if ((int)blockIdx.z == i) {
+                x = sibs.x_of[i];
+                T = sibs.T_of[i];
+            }
+    }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nchunks = (n + 255) >> 8;
     const int tok0 = blockIdx.y * 8;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    const int live = T < 8 ? T : 8;
+    const int live = T_grid < 8 ? T_grid : 8;
     // the row CTAs come first in the grid, the rotation CTAs last
     const int nrow = (int)gridDim.x - (STAGED ? live * ((nchunks + 7) >> 3) : nchunks);
     if ((int)blockIdx.x < nrow) {

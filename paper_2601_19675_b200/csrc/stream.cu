@@ -65,6 +65,7 @@ struct StreamSiblings {
     void* y[kMaxSiblings - 1];
     int64_t ldy[kMaxSiblings - 1];
     int m[kMaxSiblings - 1];
+    int T[kMaxSiblings - 1];  // token rows of the sibling (experts of a mixture layer differ; otherwise all alike)
 };
 
 // The layer a CTA works on: patches the per-layer fields of the parameters, returns the CTA's index within the layer.
@@ -82,6 +83,7 @@ __device__ __forceinline__ int select_sibling(StreamParams& p, const StreamSibli
             p.y = sibs.y[i];
             p.ldy = sibs.ldy[i];
             p.m = sibs.m[i];
+            p.T = sibs.T[i];
         }
     return bx;
 }
@@ -673,6 +675,7 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
     StreamSiblings sibs = {};
     if (more != nullptr) {
         sibs.n = more->n;
+        if (more->own_rows) p.T = more->T_of[0];
         for (int i = 0; i < more->n; ++i) {
             const uint8_t* b = more->blob[i];
             const BlobLayout& Li = more->L[i];
@@ -686,6 +689,7 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
             sibs.y[i] = more->y[i];
             sibs.ldy[i] = more->ldy[i];
             sibs.m[i] = more->d_out[i];
+            sibs.T[i] = more->own_rows ? more->T_of[i + 1] : T;
             grid += (more->d_out[i] + rows_per_cta - 1) / rows_per_cta;
         }
     }

@@ -73,6 +73,7 @@ struct TallSiblings {
     void* y[kMaxSiblings - 1];
     int64_t ldy[kMaxSiblings - 1];
     int m[kMaxSiblings - 1];
+    int T[kMaxSiblings - 1];  // token rows of the sibling
 };
 
 // The layer a CTA works on: patches the per-layer fields, returns the CTA's index among the layer's CTAs and
@@ -92,6 +93,7 @@ __device__ __forceinline__ int2 select_sibling(TallParams& p, const TallSiblings
             p.y = sibs.y[i];
             p.ldy = sibs.ldy[i];
             p.m = sibs.m[i];
+            p.T = sibs.T[i];
         }
     return make_int2((int)blockIdx.x - first, end - first);
 }
@@ -539,7 +541,9 @@ cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayo
             sibs.y[i] = more->y[i];
             sibs.ldy[i] = more->ldy[i];
             sibs.m[i] = more->d_out[i];
+            sibs.T[i] = more->own_rows ? more->T_of[i + 1] : T;
         }
+        if (more->own_rows) p.T = more->T_of[0];
     }
     switch (d.bits) {
         case 2: return launch_tall_bits<2>(p, sibs, pl.nt, pl.grid, pl.smem_bytes, s);

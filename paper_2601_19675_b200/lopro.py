@@ -28,7 +28,8 @@ SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packe
            "lopro_linear_fwd_group", "lopro_pack_lr8", "lopro_unpack_lr8", "lopro_r1svd_workspace_bytes", "lopro_r1svd",
            "lopro_residual_rotate", "lopro_rtn_quantize", "lopro_quantize_workspace_bytes", "lopro_quantize_layer",
            "lopro_block_add_rmsnorm", "lopro_block_rope_append", "lopro_block_attention_workspace_bytes",
-           "lopro_block_attention_decode", "lopro_block_silu_mul"]
+           "lopro_block_attention_decode", "lopro_block_silu_mul", "lopro_experts_workspace_bytes",
+           "lopro_linear_fwd_experts_path", "lopro_linear_fwd_experts"]
 
 
 class Desc(ctypes.Structure):
@@ -115,6 +116,12 @@ def lib():
         L.lopro_quantize_layer.restype = ctypes.c_int
         L.lopro_quantize_layer.argtypes = [dp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         f32 = ctypes.c_float
+        L.lopro_experts_workspace_bytes.restype = sz
+        L.lopro_experts_workspace_bytes.argtypes = [dp, i32, i32]
+        L.lopro_linear_fwd_experts_path.restype = i32
+        L.lopro_linear_fwd_experts_path.argtypes = [dp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.lopro_linear_fwd_experts.restype = ctypes.c_int
+        L.lopro_linear_fwd_experts.argtypes = [dp, i32, ctypes.POINTER(vp), ctypes.POINTER(i32), vp, i64, vp, i64, i32, vp, sz, vp]
         L.lopro_block_add_rmsnorm.restype = ctypes.c_int
         L.lopro_block_add_rmsnorm.argtypes = [vp, i64, vp, i64, vp, f32, vp, i64, i32, i32, vp]
         L.lopro_block_rope_append.restype = ctypes.c_int
@@ -371,6 +378,37 @@ def block_silu_mul(gate, up, out=None):
     st = lib().lopro_block_silu_mul(_ptr(gate), gate.stride(0), _ptr(up), up.stride(0), _ptr(out), out.stride(0), T, d, _stream())
     _check(st, "lopro_block_silu_mul")
     return out
+
+
+def experts_workspace_bytes(desc, n_experts, max_rows):
+    return lib().lopro_experts_workspace_bytes(ctypes.byref(desc), n_experts, max_rows)
+
+
+def _offsets(row_offsets):
+    return (ctypes.c_int32 * len(row_offsets))(*[int(v) for v in row_offsets])
+
+
+def linear_fwd_experts_path(desc, row_offsets):
+    """(path, launches) of lopro_linear_fwd_experts: 2 = shared launches, 1 = expert by expert."""
+    launches = ctypes.c_int32(0)
+    path = lib().lopro_linear_fwd_experts_path(ctypes.byref(desc), len(row_offsets) - 1, _offsets(row_offsets), ctypes.byref(launches))
+    return path, launches.value
+
+
+def linear_fwd_experts(desc, blobs, row_offsets, x, out_dtype=OUT_BF16, workspace=None, y=None):
+    """lopro_linear_fwd_experts: x bf16 [rows][d_in] grouped by expert (host list row_offsets of len(blobs) + 1 entries)."""
+    n = len(blobs)
+    rows = x.shape[0]
+    max_rows = max([row_offsets[e + 1] - row_offsets[e] for e in range(n)] + [1])
+    if workspace is None:
+        workspace = torch.zeros(max(experts_workspace_bytes(desc, n, max_rows), 256), dtype=torch.uint8, device=x.device)
+    if y is None:
+        y = torch.empty((rows, desc.d_out), dtype=torch.float32 if out_dtype == OUT_F32 else torch.bfloat16, device=x.device)
+    ptrs = (ctypes.c_void_p * n)(*[b.data_ptr() for b in blobs])
+    st = lib().lopro_linear_fwd_experts(ctypes.byref(desc), n, ptrs, _offsets(row_offsets), _ptr(x), x.stride(0), _ptr(y),
+                                        y.stride(0), out_dtype, _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "lopro_linear_fwd_experts")
+    return y
 
 
 def unpack_lr8(desc, packed):
