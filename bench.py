@@ -709,6 +709,67 @@ def measure_offline(dev, peaks, reps=3):
     return out
 
 
+def measure_experts(dev, peaks, reps=20):
+    """The experts of a mixture layer at decode: 8 experts 4096 -> 14336 (2-bit g64, block 256, rank 16), 16 tokens routed
+    to 2 experts each = 32 rows, 4 per expert; a ring of 3 distinct expert sets (each larger than L2); the grouped call
+    against one call per expert."""
+    import torch
+    from paper_2601_19675_b200 import lopro, synth
+    n, m, E, sets, per = 4096, 14336, 8, 3, 4
+    d = lopro.make_desc(n, m, 2, 64, 256, 256, 16, lopro.LAYOUT_FRAGMENT)
+    base = synth.random_layer(n, m, 2, 64, 16, seed=5)
+
+    def dev16(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev)
+
+    codes0 = torch.from_numpy(base["codes"]).to(dev)
+    sc, zr, pm, A, B = dev16(base["scales"]), dev16(base["zeros"]), torch.from_numpy(base["perm"]).to(dev), dev16(base["A"]), dev16(base["B"])
+    blobs = [[lopro.pack(d, torch.roll(codes0, shifts=(7 * (s * E + e), 3 * (s * E + e)), dims=(0, 1)), sc, zr, pm, A, B)
+              for e in range(E)] for s in range(sets)]
+    del codes0
+    offs = [per * e for e in range(E + 1)]
+    x = dev16(synth.activations(per * E, n, seed=6)).view(torch.bfloat16)
+    y = torch.empty((per * E, m), dtype=torch.bfloat16, device=dev)
+    ws = torch.zeros(lopro.experts_workspace_bytes(d, E, per), dtype=torch.uint8, device=dev)
+    c = dict(d_out=m, d_in=n, bits=2, group_size=64, rank=16)
+    nbytes = E * algorithmic_bytes(c, per)
+
+    def grouped():
+        for s in range(sets):
+            lopro.linear_fwd_experts(d, blobs[s], offs, x, lopro.OUT_BF16, workspace=ws, y=y)
+
+    def one_by_one():
+        for s in range(sets):
+            for e in range(E):
+                lopro.linear_fwd(d, blobs[s][e], x[offs[e]:offs[e + 1]], lopro.OUT_BF16, workspace=ws, y=y[offs[e]:offs[e + 1]])
+
+    out = {}
+    for name, fn in (("grouped", grouped), ("one_call_per_expert", one_by_one)):
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            fn()
+            stream.synchronize()
+            assert lopro.workspace_status(ws) == lopro.OK
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                fn()
+            for _ in range(3):
+                graph.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(reps):
+                graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (reps * sets)
+        out[name] = dict(us_per_layer=us, achieved_gbs=nbytes / (us * 1e-6) / 1e9,
+                         frac_of_measured_hbm=nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                         launches_per_layer=lopro.linear_fwd_experts_path(d, offs)[1] if name == "grouped" else 2 * E)
+    out["workload"] = ("8 experts 4096 -> 14336, 2-bit g64 block 256 rank 16, 4 rows per expert (16 tokens, 2 experts each); "
+                       "%d bytes per layer forward; ring of %d expert sets" % (nbytes, sets))
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -725,7 +786,7 @@ def main():
     ap.add_argument("--lowrank", default="f16", choices=["f16", "fp8"],
                     help="storage of the rank-r term of single-layer workloads: folded fp16 A, B or the fp8 record U, V, Sigma, s")
     ap.add_argument("--offline", action="store_true",
-                    help="only the offline side (quantization of a layer on the GPU), as one JSON line of its own")
+                    help="only the offline side (quantization of a layer on the GPU) and the mixture-layer experts, as one JSON line of their own")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -754,7 +815,8 @@ def main():
 
     if args.offline:
         if rank == 0:
-            print(json.dumps(dict(offline=measure_offline(dev, measured_peaks()), n_gpus=1, data="synthetic", dtype="f32")))
+            print(json.dumps(dict(offline=measure_offline(dev, measured_peaks()), experts=measure_experts(dev, measured_peaks()),
+                                  n_gpus=1, data="synthetic", dtype="f32")))
         if world > 1:
             dist.destroy_process_group()
         return 0
@@ -783,6 +845,7 @@ def main():
         line["workloads"] = table
         if rank == 0:
             line["offline"] = measure_offline(dev, measured_peaks())
+            line["experts"] = measure_experts(dev, measured_peaks())
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
