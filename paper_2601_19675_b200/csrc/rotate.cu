@@ -6,6 +6,7 @@
 #include "common.cuh"
 #include "ptx.cuh"
 #include "rotate_body.cuh"
+#include "rotate_mma.cuh"
 
 namespace lopro {
 
@@ -503,8 +504,40 @@ cudaError_t launch_rotate_e(const lopro_desc& d, const int32_t* perm, const __nv
 
 }  // namespace
 
+namespace {
+
+template <int TOK>
+__global__ void __launch_bounds__(256, 2)
+rotate_mma_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
+                  __nv_bfloat16* __restrict__ xrot, int64_t ldo, int* __restrict__ status, int n, int b_i, int b_h,
+                  float inv_sqrt_bh, int T) {
+    extern __shared__ __align__(16) unsigned char rot_smem[];
+    rotate_mma_body<TOK>(rot_smem, (int)blockIdx.x, x, ldx, perm, xrot, ldo, status, n, b_i, b_h, inv_sqrt_bh, T);
+}
+
+template <int TOK>
+cudaError_t launch_rotate_mma(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
+                              __nv_bfloat16* xrot, int64_t ldo, int* status, int T, cudaStream_t s) {
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(rotate_mma_kernel<TOK>, kRotMmaMaxSmem, &attr_done);
+    if (e != cudaSuccess) return e;
+    const float inv = (float)(1.0 / sqrt((double)d.block_size));
+    rotate_mma_kernel<TOK><<<(T + TOK - 1) / TOK, 256, rotate_mma_smem_bytes(TOK, d.d_in), s>>>(
+        x, ldx, perm, xrot, ldo, status, d.d_in, d.identity_cols, d.block_size, inv, T);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
 cudaError_t launch_rotate(const lopro_desc& d, const int32_t* perm, const __nv_bfloat16* x, int64_t ldx,
                           __nv_bfloat16* xrot, int64_t ldo, float* s64, int* status, int T, cudaStream_t s) {
+    // many rows and no column sums wanted: the tensor-core form of the recursion, eight (or four) rows per CTA
+    if (s64 == nullptr && T >= 16 && rotate_mma_shape_ok(d) && (reinterpret_cast<uintptr_t>(perm) % 16) == 0) {
+        if (rotate_mma_smem_bytes(8, d.d_in) <= (size_t)kRotMmaMaxSmem / 2)
+            return launch_rotate_mma<8>(d, perm, x, ldx, xrot, ldo, status, T, s);
+        if (rotate_mma_smem_bytes(4, d.d_in) <= (size_t)kRotMmaMaxSmem)
+            return launch_rotate_mma<4>(d, perm, x, ldx, xrot, ldo, status, T, s);
+    }
     if (d.block_size <= 256) return launch_rotate_e<8>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
     if (d.block_size == 512) return launch_rotate_e<16>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);
     return launch_rotate_e<32>(d, perm, x, ldx, xrot, ldo, s64, status, T, s);

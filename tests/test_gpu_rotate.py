@@ -49,6 +49,20 @@ def test_rotate_matches_oracle_within_one_bf16_ulp(n, b_i, b_h, T):
     assert np.array_equal(got[:, :b_i], ref[:, :b_i])
 
 
+@pytest.mark.parametrize("n,b_i,b_h,T", [
+    (4096, 128, 128, 16), (4096, 128, 128, 2048), (8192, 256, 256, 77), (11008, 128, 128, 21), (1024, 0, 16, 19),
+    (2048, 32, 32, 40), (4096, 64, 64, 257), (512, 512, 64, 17), (1024, 16, 16, 30), (12288, 0, 256, 18), (14336, 256, 128, 16),
+])
+def test_rotate_many_rows_tensor_core_form(n, b_i, b_h, T):
+    # 16 rows and more, b_H in 16..256, b_I a multiple of 16: the first four levels of the recursion as a product with
+    # H_16 on the tensor cores (fp32 accumulation of sixteen +-x terms), the rest as fp32 add / subtract
+    got, exact, _, _ = _run(n, b_i, b_h, T, seed=n + b_h + T, outlier_frac=0.01)
+    ref = o.round_bf16(exact)
+    assert np.all(np.abs(got - exact) <= 0.5001 * _ulp_bf16(exact) + 1e-6 * np.abs(exact).max())
+    assert np.mean(got == ref) > 0.995
+    assert np.array_equal(got[:, :b_i], ref[:, :b_i])
+
+
 def test_pure_permutation_is_bit_exact_and_strided_rows_work():
     n, T = 4096, 9
     got, exact, x_bits, perm = _run(n, n, 128, T, seed=11, ldx=n + 64)
@@ -56,6 +70,9 @@ def test_pure_permutation_is_bit_exact_and_strided_rows_work():
     got2, exact2, _, _ = _run(n, 128, 128, T, seed=11, ldx=n + 64)
     got3, _, _, _ = _run(n, 128, 128, T, seed=11)
     assert np.array_equal(got2, got3)
+    got4, _, _, _ = _run(n, 128, 128, 37, seed=12, ldx=n + 64)          # many rows: the other kernel, strided as well
+    got5, _, _, _ = _run(n, 128, 128, 37, seed=12)
+    assert np.array_equal(got4, got5)
 
 
 def test_rotation_preserves_norm_and_is_an_involution_on_the_device():
