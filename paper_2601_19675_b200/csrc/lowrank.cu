@@ -10,6 +10,7 @@
 #include "common.cuh"
 #include "ptx.cuh"
 #include "rotate_body.cuh"
+#include "rotate_mma.cuh"
 
 namespace lopro {
 
@@ -141,15 +142,29 @@ __global__ void __launch_bounds__(kLrThreads, NJ <= 8 ? 3 : 2)
 rotate_lowrank_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, const int32_t* __restrict__ perm,
                       __nv_bfloat16* __restrict__ xrot, int64_t ldo, float* __restrict__ s64, int s64_ld,
                       int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int T, int n_rot,
-                      const __half* __restrict__ B, float* __restrict__ partial, int r_pad, int lr_gx, int slice_cols) {
+                      const __half* __restrict__ B, float* __restrict__ partial, int r_pad, int lr_gx, int slice_cols,
+                      int mma_form, int rows_per_cta) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if ((int)blockIdx.x < n_rot) {
-        rotate_body<8, 4, true>(smem_raw, (int)blockIdx.x, x, ldx, perm, xrot, ldo, s64, s64_ld, status, n, b_i, b_h,
-                                inv_sqrt_bh, T);
+    // The two kinds of CTA are dealt out evenly over the grid (rot_before(i) = rotation CTAs among the first i), so
+    // that every wave of resident CTAs holds both: their memory and arithmetic phases then overlap instead of all
+    // rotation CTAs loading at once and all of them computing at once.
+    const unsigned total = gridDim.x, i = blockIdx.x;
+    const int rot_before = (int)(((unsigned long long)i * (unsigned)n_rot) / total);
+    const int rot_through = (int)(((unsigned long long)(i + 1) * (unsigned)n_rot) / total);
+    if (rot_through > rot_before) {
+        const int rb = rot_before;
+        // (no 64-column sums: the tensor-core product that follows dequantizes the weights and needs none)
+        if (rows_per_cta == 8)
+            rotate_mma_body<8>(smem_raw, rb, x, ldx, perm, xrot, ldo, status, n, b_i, b_h, inv_sqrt_bh, T);
+        else if (mma_form)
+            rotate_mma_body<4>(smem_raw, rb, x, ldx, perm, xrot, ldo, status, n, b_i, b_h, inv_sqrt_bh, T);
+        else
+            rotate_body<8, 4, true>(smem_raw, rb, x, ldx, perm, xrot, ldo, s64, s64_ld, status, n, b_i, b_h,
+                                    inv_sqrt_bh, T);
     } else {
-        const int b = (int)blockIdx.x - n_rot;
+        const int b = (int)i - rot_before;
         lowrank_body<NJ>(smem_raw, b % lr_gx, b / lr_gx, B, x, ldx, partial, n, r_pad, T, 0, slice_cols);
     }
 }
@@ -230,8 +245,14 @@ cudaError_t launch_rotate_lowrank_nj(const lopro_desc& d, const int32_t* perm, c
                                      float* partial, int T, cudaStream_t s) {
     const int slices = lowrank_mma_slices(d, T);
     const int slice_cols = d.d_in / slices;
-    const int n_rot = (T + 3) / 4, lr_gx = (T + kLrTokens - 1) / kLrTokens;
-    const size_t smem_rot = (size_t)d.d_in * 8, smem_lr = (size_t)(kLrTokens + 2 * NJ * 8) * kLrStride * 2;
+    // rotation CTAs: the tensor-core form of the recursion with 8 rows per CTA where that leaves room for three CTAs
+    // per SM, with 4 rows otherwise; the register-and-shuffle form where the block size or prefix rules it out
+    const bool mma_form = rotate_mma_shape_ok(d) && (reinterpret_cast<uintptr_t>(perm) % 16) == 0 &&
+                          rotate_mma_smem_bytes(4, d.d_in) <= 160 * 1024;
+    const int rows_per_cta = mma_form && rotate_mma_smem_bytes(8, d.d_in) <= 74 * 1024 ? 8 : 4;
+    const int n_rot = (T + rows_per_cta - 1) / rows_per_cta, lr_gx = (T + kLrTokens - 1) / kLrTokens;
+    const size_t smem_rot = mma_form ? rotate_mma_smem_bytes(rows_per_cta, d.d_in) : (size_t)d.d_in * 8;
+    const size_t smem_lr = (size_t)(kLrTokens + 2 * NJ * 8) * kLrStride * 2;
     const size_t smem = smem_rot > smem_lr ? smem_rot : smem_lr;
     static unsigned long long attr_done = 0;
     cudaError_t e = ensure_dynamic_smem(rotate_lowrank_kernel<NJ>, 160 * 1024, &attr_done);
@@ -248,7 +269,8 @@ cudaError_t launch_rotate_lowrank_nj(const lopro_desc& d, const int32_t* perm, c
     cfg.numAttrs = 1;
     const float inv = (float)(1.0 / sqrt((double)d.block_size));
     return cudaLaunchKernelEx(&cfg, rotate_lowrank_kernel<NJ>, x, ldx, perm, xrot, ldo, s64, s64_stride(d.d_in), status,
-                              d.d_in, d.identity_cols, d.block_size, inv, T, n_rot, B, partial, r_pad, lr_gx, slice_cols);
+                              d.d_in, d.identity_cols, d.block_size, inv, T, n_rot, B, partial, r_pad, lr_gx, slice_cols,
+                              mma_form ? 1 : 0, rows_per_cta);
 }
 
 }  // namespace

@@ -36,17 +36,18 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 }
 
 // The lane's four gathered entries of the 16-tile that starts at column k0, as two bf16 pairs.  xrow_s: shared-space
-// address of the lane's staged row; off_s: shared-space address of the CTA's table of BYTE offsets 2 * perm[k]
-// (clamped to the row when it was built, so that a perm that is no permutation cannot reach foreign memory).
+// address of the lane's staged row; off_s: shared-space address of the CTA's table of 16-bit column indices perm[k]
+// (d_in <= 32768; clamped to the row when it was built, so that a perm that is no permutation cannot reach foreign
+// memory).
 __device__ __forceinline__ void gather_tile(uint32_t xrow_s, uint32_t off_s, int k0, int t, uint32_t& a0, uint32_t& a2) {
-    uint32_t p0, p1, p2, p3;
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(p0), "=r"(p1) : "r"(off_s + 4u * (uint32_t)(k0 + 2 * t)));
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(p2), "=r"(p3) : "r"(off_s + 4u * (uint32_t)(k0 + 8 + 2 * t)));
+    uint32_t w0, w1;  // two 16-bit column indices each
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w0) : "r"(off_s + 2u * (uint32_t)(k0 + 2 * t)));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w1) : "r"(off_s + 2u * (uint32_t)(k0 + 8 + 2 * t)));
     unsigned short v0, v1, v2, v3;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v0) : "r"(xrow_s + p0));
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v1) : "r"(xrow_s + p1));
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v2) : "r"(xrow_s + p2));
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v3) : "r"(xrow_s + p3));
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v0) : "r"(xrow_s + 2u * (w0 & 0xFFFFu)));
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v1) : "r"(xrow_s + 2u * (w0 >> 16)));
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v2) : "r"(xrow_s + 2u * (w1 & 0xFFFFu)));
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v3) : "r"(xrow_s + 2u * (w1 >> 16)));
     asm("mov.b32 %0, {%1,%2};" : "=r"(a0) : "h"(v0), "h"(v1));
     asm("mov.b32 %0, {%1,%2};" : "=r"(a2) : "h"(v2), "h"(v3));
 }
@@ -97,7 +98,7 @@ __device__ __forceinline__ void rotate_block_mma(uint32_t xrow, uint32_t perm,
 constexpr int kRotMmaPad = 8;  // bf16 entries between the staged rows
 constexpr int kRotMmaMaxSmem = 200 * 1024;
 __host__ __device__ inline size_t rotate_mma_smem_bytes(int tok, int n) {
-    return (size_t)tok * (size_t)(n + kRotMmaPad) * 2 + (size_t)n * 4;  // the rows, then a copy of perm
+    return (size_t)tok * (size_t)(n + kRotMmaPad) * 2 + (size_t)n * 2;  // the rows, then perm as 16-bit indices
 }
 
 template <int TOK>
@@ -120,17 +121,15 @@ __device__ __forceinline__ void rotate_mma_body(unsigned char* smem_raw, int blo
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * (uint32_t)c), "l"(src + 8 * c) : "memory");
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
-    // byte offsets 2 * min(perm[k], n - 1) of the gather, one table per CTA
-    uint32_t* off_tab = reinterpret_cast<uint32_t*>(xs + (size_t)TOK * stride);
+    // the gather's column indices min(perm[k], n - 1) as 16-bit numbers, one table per CTA
+    unsigned short* off_tab = xs + (size_t)TOK * stride;
     for (int c = tid; c < (n >> 2); c += 256) {
         const int4 p4 = __ldg(reinterpret_cast<const int4*>(perm) + c);
         const uint32_t last = (uint32_t)n - 1u;
-        uint4 o4;
-        o4.x = 2u * min((uint32_t)p4.x, last);
-        o4.y = 2u * min((uint32_t)p4.y, last);
-        o4.z = 2u * min((uint32_t)p4.z, last);
-        o4.w = 2u * min((uint32_t)p4.w, last);
-        reinterpret_cast<uint4*>(off_tab)[c] = o4;
+        uint2 o2;
+        o2.x = min((uint32_t)p4.x, last) | (min((uint32_t)p4.y, last) << 16);
+        o2.y = min((uint32_t)p4.z, last) | (min((uint32_t)p4.w, last) << 16);
+        reinterpret_cast<uint2*>(off_tab)[c] = o2;
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
