@@ -516,6 +516,72 @@ def e4m3_bits_to_f64(b):
     return sign * np.where(exp == 0, man * 2.0 ** -9, (1.0 + man / 8.0) * 2.0 ** (exp - 7.0))
 
 
+# --------------------------------------------------------------------------
+# vector-quantized residual (the LoPRo_v variant, Appendix "implementation details")
+# --------------------------------------------------------------------------
+# Reading (the paper names a randomly initialised codebook, 4-D at 2 bits, 2-D at 3 bits, no block-wise scaling, no
+# learned codebooks, and leaves every format detail to the vector quantizer it calls): the rotated residual R' is cut
+# into groups of cb_rows rows x cb_cols columns; a group has ONE codebook of 2^(dim * q) centroids of dimension dim;
+# a centroid stands for dim consecutive (rotated) columns of one row; no scale.  With 4-D / 8-bit indices, bf16
+# centroids and groups of 512 x 256 the codebook costs 256 * 4 * 16 / (512 * 256) = 0.125 bit per weight -- the
+# figure the results table implies (2.17 = 2 + 0.125 + the 0.05 of the rank-16 factors).
+
+
+def vq_dequant(idx, codebooks, dim, cb_rows, cb_cols):
+    """W^[i, dim v + e] = C[i // cb_rows][(dim v) // cb_cols][idx[i, v]][e].
+    idx [m][n / dim] integer; codebooks [ceil(m / cb_rows)][n / cb_cols][K][dim] fp64."""
+    idx = np.asarray(idx)
+    m, nv = idx.shape
+    out = np.empty((m, nv * dim))
+    for i in range(m):
+        for v in range(nv):
+            out[i, dim * v:dim * (v + 1)] = codebooks[i // cb_rows][(dim * v) // cb_cols][idx[i, v]]
+    return out
+
+
+def vq_quantize(rp, dim, index_bits, cb_rows, cb_cols, picks):
+    """Vector quantization of R' with a randomly initialised codebook: the centroids of a group are 2^index_bits of the
+    group's own vectors -- `picks` [row groups][column groups][2^index_bits] indexes the group's vectors in row-major
+    order (row within the group, then vector within the row) and is passed in, so that the routine draws nothing --
+    rounded to bf16; every vector takes the nearest centroid in the Euclidean norm (the loss of Eq. "rotate loss"
+    with H' = I), ties to the lower index.  Returns (idx uint16 [m][n / dim], codebooks fp64 holding bf16 values)."""
+    rp = np.asarray(rp, dtype=np.float64)
+    m, n = rp.shape
+    if n % cb_cols or cb_cols % dim:
+        raise ValueError("codebook columns must divide n and hold whole vectors")
+    k = 2 ** index_bits
+    n_rg, n_cg, vpg = -(-m // cb_rows), n // cb_cols, cb_cols // dim
+    idx = np.zeros((m, n // dim), dtype=np.uint16)
+    books = np.zeros((n_rg, n_cg, k, dim))
+    for rg in range(n_rg):
+        r0, r1 = rg * cb_rows, min(m, (rg + 1) * cb_rows)
+        for cg in range(n_cg):
+            vecs = rp[r0:r1, cg * cb_cols:(cg + 1) * cb_cols].reshape(-1, dim)        # row-major: (row, vector)
+            cb = round_bf16(vecs[np.asarray(picks[rg][cg]) % vecs.shape[0]])
+            d2 = ((vecs[:, None, :] - cb[None, :, :]) ** 2).sum(axis=2)
+            idx[r0:r1, cg * vpg:(cg + 1) * vpg] = np.argmin(d2, axis=1).reshape(r1 - r0, vpg)
+            books[rg, cg] = cb
+    return idx, books
+
+
+def forward_exact_vq(x, idx, codebooks, perm, a, b, dim, cb_rows, cb_cols, b_i, b_h):
+    """Eq. 8 with the vector-quantized residual: y = x B^T A^T + rotate(x) W^_vq^T, fp64, no rounding."""
+    x = np.asarray(x, dtype=np.float64)
+    w_hat = vq_dequant(idx, codebooks, dim, cb_rows, cb_cols)
+    y = rotate(x, perm, b_i, b_h) @ w_hat.T
+    a, b = np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64)
+    if a.shape[1]:
+        y = y + (x @ b.T) @ a.T
+    return y
+
+
+def vq_average_bits(m, n, dim, index_bits, d_c, cb_rows, cb_cols, r, d_r):
+    """Average bits per weight of the vector-quantized record: index bits per weight, the codebooks (d_c bits per
+    centroid entry), and the rank-r factors with d_r bits per entry (the last term of Eq. 13)."""
+    n_books = -(-m // cb_rows) * (n // cb_cols)
+    return index_bits / dim + n_books * (2 ** index_bits) * dim * d_c / (m * n) + r * d_r * (m + n) / (m * n)
+
+
 def max_rel_err(y, y_ref):
     """Element-wise error relative to max(|y_ref[t, i]|, rms_i y_ref[t, :]): the
     'max relative error' of the acceptance gates, floored at the row RMS so that
