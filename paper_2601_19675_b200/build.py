@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblopro.so")
-SOURCES = ["api.cu", "pack.cu", "rotate.cu", "decode.cu", "stream.cu", "tall.cu", "noalloc.cu", "prefill.cu", "lowrank.cu", "rowblock.cu", "quantize.cu", "block.cu"]
+SOURCES = ["api.cu", "pack.cu", "rotate.cu", "decode.cu", "stream.cu", "tall.cu", "noalloc.cu", "prefill.cu", "lowrank.cu", "rowblock.cu", "quantize.cu", "block.cu", "vq.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -1,0 +1,370 @@
+// Vector-quantized residual (the vector variant of the method: a codebook of 256 four-dimensional centroids per group
+// of cb_rows x cb_cols rotated weights, one 8-bit index per four consecutive columns): packed record and forward.
+// The forward is Eq. 8 with W^ looked up instead of dequantized: rotation and t = B x by the library's kernels, then
+// one product kernel per group of up to 32 tokens.
+#include "lopro_vq.h"
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <cstring>
+
+namespace lopro {
+
+namespace {
+
+constexpr uint32_t kVqMagic = 0x5156504Cu;  // "LPVQ"
+constexpr int kVqHeader = 256;
+constexpr int kVqRowsPerCta = 64;           // four warps, sixteen rows each
+constexpr int kVqBookBytes = 256 * 4 * 2;   // one codebook
+
+inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+struct VqLayout {
+    size_t off_idx, off_books, off_perm, off_a, off_b, off_bitmap, total;
+    int r_pad, n_rg, n_cg;
+};
+
+lopro_status vq_check(const lopro_vq_desc* d) {
+    if (!d) return LOPRO_ERR_INVALID_ARG;
+    if (d->d_in <= 0 || d->d_out <= 0 || d->cb_rows <= 0 || d->cb_cols <= 0) return LOPRO_ERR_INVALID_ARG;
+    if (d->block_size < 2 || d->block_size > 1024 || (d->block_size & (d->block_size - 1))) return LOPRO_ERR_INVALID_ARG;
+    if (d->identity_cols < 0 || d->identity_cols > d->d_in || (d->d_in - d->identity_cols) % d->block_size)
+        return LOPRO_ERR_INVALID_ARG;
+    if (d->rank < 0 || d->rank > 512 || d->d_in % d->cb_cols) return LOPRO_ERR_INVALID_ARG;
+    if (d->d_in % 64 || d->d_out % kVqRowsPerCta || d->cb_rows % kVqRowsPerCta || d->cb_cols % 64) return LOPRO_ERR_UNSUPPORTED;
+    if (d->d_in > 32768 || d->d_out > (1 << 20)) return LOPRO_ERR_UNSUPPORTED;
+    if ((size_t)(d->d_in / d->cb_cols) * kVqBookBytes > 160 * 1024) return LOPRO_ERR_UNSUPPORTED;  // a row group's books in shared memory
+    return LOPRO_OK;
+}
+
+VqLayout vq_layout(const lopro_vq_desc& d) {
+    VqLayout L;
+    const size_t m = d.d_out, n = d.d_in;
+    L.r_pad = round_up_int(d.rank, 16);
+    L.n_rg = (d.d_out + d.cb_rows - 1) / d.cb_rows;
+    L.n_cg = d.d_in / d.cb_cols;
+    size_t off = kVqHeader;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off += round_up_size(bytes, 256);
+        return at;
+    };
+    L.off_idx = take(m * (n / 4));
+    L.off_books = take((size_t)L.n_rg * L.n_cg * kVqBookBytes);
+    L.off_perm = take(n * 4);
+    L.off_a = take(m * (size_t)L.r_pad * 2);
+    L.off_b = take((size_t)L.r_pad * n * 2);
+    L.off_bitmap = take((n + 31) / 32 * 4);  // scratch of the permutation check
+    L.total = off;
+    return L;
+}
+
+// The rotation and the low-rank down-projection are those of the scalar forward: they see this descriptor.
+lopro_desc as_scalar_desc(const lopro_vq_desc& d) {
+    lopro_desc s = {};
+    s.d_in = d.d_in;
+    s.d_out = d.d_out;
+    s.bits = 4;
+    s.group_size = 64;
+    s.block_size = d.block_size;
+    s.identity_cols = d.identity_cols;
+    s.rank = d.rank;
+    s.layout = LOPRO_LAYOUT_FRAGMENT;
+    s.lowrank_format = LOPRO_LOWRANK_FOLDED_F16;
+    return s;
+}
+
+struct VqWorkspace {
+    size_t off_status, off_xrot, off_t, off_part, total;
+    int r_pad;
+};
+
+VqWorkspace vq_workspace(const lopro_vq_desc& d, int T) {
+    VqWorkspace W;
+    W.r_pad = round_up_int(d.rank, 16);
+    size_t off = 0;
+    W.off_status = off;
+    off += 256;
+    W.off_xrot = off;
+    off += round_up_size((size_t)T * d.d_in * 2, 256);
+    W.off_t = off;
+    off += round_up_size((size_t)T * (W.r_pad > 0 ? W.r_pad : 16) * 2, 256);
+    W.off_part = off;
+    off += d.rank > 0 && T > kDecodeMaxT ? round_up_size(lowrank_mma_scratch_bytes(as_scalar_desc(d), T), 256) : 0;
+    W.total = off;
+    return W;
+}
+
+__global__ void vq_perm_check_kernel(const int32_t* __restrict__ perm, int n, uint32_t* __restrict__ bitmap, int* flag) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int p = perm[i];
+    if ((unsigned)p >= (unsigned)n) {
+        *flag = 1;
+        return;
+    }
+    const uint32_t bit = 1u << (p & 31);
+    if (atomicOr(bitmap + (p >> 5), bit) & bit) *flag = 1;
+}
+
+__global__ void vq_identity_perm_kernel(int32_t* __restrict__ perm, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) perm[i] = i;
+}
+
+// rows of a factor matrix into rows padded to r_pad (zeros beyond r)
+__global__ void vq_copy_padded_kernel(const __half* __restrict__ src, int rows, int cols, int cols_pad, __half* __restrict__ dst) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)rows * cols_pad) return;
+    const int r = (int)(i / cols_pad), c = (int)(i % cols_pad);
+    dst[i] = c < cols ? src[(size_t)r * cols + c] : __float2half(0.0f);
+}
+
+struct VqParams {
+    const uint8_t* idx;          // [m][n / 4]
+    const unsigned char* books;  // [n_rg][n_cg][256][4] bf16
+    const __half* A;             // [m][r_pad]
+    const __nv_bfloat16* xrot;   // [T][n] rotated activations of this launch's tokens
+    const __half* t;             // [T][r_pad]
+    void* y;
+    int64_t ldy;
+    int out_f32, m, n, T, r_pad, cb_rows, cb_cols, n_cg;
+};
+
+
+// grid = m / 64, 128 threads: warp w owns rows 64 b + 16 w .. + 15 over all of K.  The codebooks of the CTA's row group
+// sit in shared memory.  K is walked in super-tiles of 64 columns = 16 vectors per row: lane 4 g + t takes the
+// vectors 4 t .. 4 t + 3 of rows g and g + 8 (one 32-bit word of indices per row), and product s of the four
+// m16n8k16 products of a super-tile uses vector 4 t + s, i.e. the lane's k-slots {2t, 2t+1, 2t+8, 2t+9} stand for
+// the columns 16 t + 4 s .. + 3.  The activation fragments follow the same assignment (32 contiguous bytes of a
+// token's rotated row per lane and super-tile), so both operands agree on which column a k-slot means.
+template <int NT>
+__global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
+    extern __shared__ __align__(16) unsigned char vq_smem[];  // [n_cg][256][4] bf16
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const int row0 = blockIdx.x * kVqRowsPerCta + warp * 16;
+    const int rg = (blockIdx.x * kVqRowsPerCta) / p.cb_rows;
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(p.books + (size_t)rg * p.n_cg * kVqBookBytes);
+        uint4* dst = reinterpret_cast<uint4*>(vq_smem);
+        for (int i = tid; i < p.n_cg * (kVqBookBytes / 16); i += 128) dst[i] = __ldg(src + i);
+    }
+    __syncthreads();
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[nt][e] = 0.0f;
+    const uint32_t* idx_lo = reinterpret_cast<const uint32_t*>(p.idx + (size_t)(row0 + g) * (p.n / 4)) + t;
+    const uint32_t* idx_hi = reinterpret_cast<const uint32_t*>(p.idx + (size_t)(row0 + g + 8) * (p.n / 4)) + t;
+    const uint32_t books_s = (uint32_t)__cvta_generic_to_shared(vq_smem);
+    const int n_super = p.n >> 6, per_book = p.cb_cols >> 6;
+    uint32_t w_lo = __ldg(idx_lo), w_hi = __ldg(idx_hi);
+    for (int S = 0; S < n_super; ++S) {
+        const uint32_t cur_lo = w_lo, cur_hi = w_hi;
+        if (S + 1 < n_super) {  // the next super-tile's indices are in flight during this one's products
+            w_lo = __ldg(idx_lo + 4 * (S + 1));
+            w_hi = __ldg(idx_hi + 4 * (S + 1));
+        }
+        // activations: 32 bytes (columns 64 S + 16 t .. + 15) of token 8 nt + g
+        uint4 xa[NT], xb[NT];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int tok = nt * 8 + g;
+            if (tok < p.T) {
+                const uint4* xr = reinterpret_cast<const uint4*>(p.xrot + (size_t)tok * p.n + 64 * S + 16 * t);
+                xa[nt] = __ldg(xr);
+                xb[nt] = __ldg(xr + 1);
+            } else {
+                xa[nt] = make_uint4(0, 0, 0, 0);
+                xb[nt] = make_uint4(0, 0, 0, 0);
+            }
+        }
+        const uint32_t book = books_s + (uint32_t)((S / per_book) * kVqBookBytes);
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            uint32_t a[4];
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[0]), "=r"(a[2]) : "r"(book + 8u * ((cur_lo >> (8 * s)) & 255u)));
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[1]), "=r"(a[3]) : "r"(book + 8u * ((cur_hi >> (8 * s)) & 255u)));
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const uint4& v = s < 2 ? xa[nt] : xb[nt];
+                const uint32_t b0 = (s & 1) ? v.z : v.x, b1 = (s & 1) ? v.w : v.y;
+                mma_bf16(acc[nt], a, b0, b1);
+            }
+        }
+    }
+    // low-rank term and store: the lane holds rows g, g + 8 and tokens 8 nt + 2 t, + 1
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int row = row0 + g + 8 * (e >> 1), tok = nt * 8 + 2 * t + (e & 1);
+            if (tok >= p.T) continue;
+            float v = acc[nt][e];
+            if (p.r_pad > 0) {
+                const uint4* ar = reinterpret_cast<const uint4*>(p.A + (size_t)row * p.r_pad);
+                const uint4* tr = reinterpret_cast<const uint4*>(p.t + (size_t)tok * p.r_pad);
+                float lr = 0.0f;
+                for (int j = 0; j < p.r_pad / 8; ++j) {
+                    const uint4 av = __ldg(ar + j), tv = __ldg(tr + j);
+                    const __half2* ah = reinterpret_cast<const __half2*>(&av);
+                    const __half2* th = reinterpret_cast<const __half2*>(&tv);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 fa = __half22float2(ah[q]), ft = __half22float2(th[q]);
+                        lr = fmaf(fa.x, ft.x, lr);
+                        lr = fmaf(fa.y, ft.y, lr);
+                    }
+                }
+                v += lr;
+            }
+            if (p.out_f32) reinterpret_cast<float*>(p.y)[(size_t)tok * p.ldy + row] = v;
+            else reinterpret_cast<__nv_bfloat16*>(p.y)[(size_t)tok * p.ldy + row] = __float2bfloat16_rn(v);
+        }
+}
+
+template <int NT>
+cudaError_t launch_vq_decode(const VqParams& p, cudaStream_t s) {
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(vq_decode_kernel<NT>, 160 * 1024, &attr_done);
+    if (e != cudaSuccess) return e;
+    vq_decode_kernel<NT><<<p.m / kVqRowsPerCta, 128, (size_t)p.n_cg * kVqBookBytes, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+}  // namespace lopro
+
+using namespace lopro;
+
+extern "C" {
+
+size_t lopro_vq_packed_bytes(const lopro_vq_desc* desc) {
+    if (vq_check(desc) != LOPRO_OK) return 0;
+    return vq_layout(*desc).total;
+}
+
+size_t lopro_vq_workspace_bytes(const lopro_vq_desc* desc, int32_t T) {
+    if (vq_check(desc) != LOPRO_OK || T < 0) return 0;
+    return vq_workspace(*desc, T < 1 ? 1 : T).total;
+}
+
+lopro_status lopro_vq_pack(const lopro_vq_desc* desc, const uint8_t* idx, const uint16_t* codebooks_bf16, const int32_t* perm,
+                           const uint16_t* A_f16, const uint16_t* B_f16, void* packed, size_t packed_bytes, void* stream) {
+    lopro_status st = vq_check(desc);
+    if (st != LOPRO_OK) return st;
+    const lopro_vq_desc& d = *desc;
+    if (!idx || !codebooks_bf16 || !perm || !packed || (d.rank > 0 && (!A_f16 || !B_f16))) return LOPRO_ERR_INVALID_ARG;
+    if (!aligned_to(packed, 256)) return LOPRO_ERR_INVALID_ARG;
+    const VqLayout L = vq_layout(d);
+    if (packed_bytes < L.total) return LOPRO_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t* blob = (uint8_t*)packed;
+    const size_t m = d.d_out, n = d.d_in;
+    // header: magic, the descriptor, and a word the permutation check raises
+    uint32_t header[kVqHeader / 4] = {};
+    header[0] = kVqMagic;
+    memcpy(header + 1, &d, sizeof(d));
+    if (cudaMemcpyAsync(blob, header, kVqHeader, cudaMemcpyHostToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (cudaMemcpyAsync(blob + L.off_idx, idx, m * (n / 4), cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (cudaMemcpyAsync(blob + L.off_books, codebooks_bf16, (size_t)L.n_rg * L.n_cg * kVqBookBytes, cudaMemcpyDeviceToDevice, s) !=
+        cudaSuccess)
+        return LOPRO_ERR_CUDA;
+    if (cudaMemcpyAsync(blob + L.off_perm, perm, n * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (d.rank > 0) {
+        const size_t na = m * (size_t)L.r_pad, nb = (size_t)L.r_pad * n;
+        vq_copy_padded_kernel<<<(unsigned)((na + 255) / 256), 256, 0, s>>>((const __half*)A_f16, (int)m, d.rank, L.r_pad,
+                                                                          (__half*)(blob + L.off_a));
+        // B [r][n] -> [r_pad][n]: whole rows, then zero rows
+        if (cudaMemcpyAsync(blob + L.off_b, B_f16, (size_t)d.rank * n * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
+        if (L.r_pad > d.rank &&
+            cudaMemsetAsync(blob + L.off_b + (size_t)d.rank * n * 2, 0, (size_t)(L.r_pad - d.rank) * n * 2, s) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
+        (void)nb;
+    }
+    if (cudaMemsetAsync(blob + L.off_bitmap, 0, (n + 31) / 32 * 4, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    int* flag = (int*)(blob + 128);  // inside the header, zero so far
+    vq_perm_check_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const int32_t*)(blob + L.off_perm), (int)n,
+                                                                     (uint32_t*)(blob + L.off_bitmap), flag);
+    if (cudaGetLastError() != cudaSuccess) return LOPRO_ERR_CUDA;
+    int bad = 0;
+    if (cudaMemcpyAsync(&bad, flag, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (bad) {
+        // a caller that ignores the verdict and runs a forward on the record must still read in bounds: the identity
+        // takes the place of the rejected index vector
+        vq_identity_perm_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>((int32_t*)(blob + L.off_perm), (int)n);
+        return LOPRO_ERR_INVALID_DATA;
+    }
+    return LOPRO_OK;
+}
+
+lopro_status lopro_vq_linear_fwd(const lopro_vq_desc* desc, const void* packed, const uint16_t* x_bf16, int64_t ldx, void* y,
+                                 int64_t ldy, int32_t out_dtype, int32_t T, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+    lopro_status st = vq_check(desc);
+    if (st != LOPRO_OK) return st;
+    const lopro_vq_desc& d = *desc;
+    if (T < 0 || (out_dtype != LOPRO_OUT_BF16 && out_dtype != LOPRO_OUT_F32)) return LOPRO_ERR_INVALID_ARG;
+    if (T == 0) return LOPRO_OK;
+    if (!packed || !x_bf16 || !y || !workspace) return LOPRO_ERR_INVALID_ARG;
+    if (ldx < d.d_in || (ldx % 8) || ldy < d.d_out) return LOPRO_ERR_INVALID_ARG;
+    if (!aligned_to(packed, 256) || !aligned_to(workspace, 256) || !aligned_to(x_bf16, 16) ||
+        !aligned_to(y, out_dtype == LOPRO_OUT_F32 ? 4 : 2))
+        return LOPRO_ERR_INVALID_ARG;
+    const VqWorkspace W = vq_workspace(d, T);
+    if (workspace_bytes < W.total) return LOPRO_ERR_BUFFER_TOO_SMALL;
+    const VqLayout L = vq_layout(d);
+    const lopro_desc sd = as_scalar_desc(d);
+    cudaStream_t s = (cudaStream_t)stream;
+    const uint8_t* blob = (const uint8_t*)packed;
+    uint8_t* ws = (uint8_t*)workspace;
+    __nv_bfloat16* xrot = (__nv_bfloat16*)(ws + W.off_xrot);
+    __half* tbuf = (__half*)(ws + W.off_t);
+    int* status = (int*)(ws + W.off_status);
+    // the rotation kernels that write no column sums do not reset the status word themselves in every form: clear it here
+    if (cudaMemsetAsync(status, 0, 4, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    if (launch_rotate(sd, (const int32_t*)(blob + L.off_perm), (const __nv_bfloat16*)x_bf16, ldx, xrot, d.d_in, nullptr,
+                      status, T, s) != cudaSuccess)
+        return LOPRO_ERR_CUDA;
+    if (d.rank > 0) {
+        const __half* B = (const __half*)(blob + L.off_b);
+        const cudaError_t e = T > kDecodeMaxT
+                                  ? launch_lowrank_down_mma(sd, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx,
+                                                            (float*)(ws + W.off_part), tbuf, T, s)
+                                  : launch_lowrank_down(sd, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, tbuf, T, s);
+        if (e != cudaSuccess) return LOPRO_ERR_CUDA;
+    }
+    const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;
+    for (int t0 = 0; t0 < T; t0 += kDecodeMaxT) {
+        const int tc = T - t0 < kDecodeMaxT ? T - t0 : kDecodeMaxT;
+        VqParams p;
+        p.idx = blob + L.off_idx;
+        p.books = blob + L.off_books;
+        p.A = (const __half*)(blob + L.off_a);
+        p.xrot = xrot + (size_t)t0 * d.d_in;
+        p.t = tbuf + (size_t)t0 * L.r_pad;
+        p.y = (uint8_t*)y + (size_t)t0 * ldy * esz;
+        p.ldy = ldy;
+        p.out_f32 = out_dtype == LOPRO_OUT_F32;
+        p.m = d.d_out;
+        p.n = d.d_in;
+        p.T = tc;
+        p.r_pad = d.rank > 0 ? L.r_pad : 0;
+        p.cb_rows = d.cb_rows;
+        p.cb_cols = d.cb_cols;
+        p.n_cg = L.n_cg;
+        const cudaError_t e = tc <= 8 ? launch_vq_decode<1>(p, s) : (tc <= 16 ? launch_vq_decode<2>(p, s) : launch_vq_decode<4>(p, s));
+        if (e != cudaSuccess) return LOPRO_ERR_CUDA;
+    }
+    return LOPRO_OK;
+}
+
+}  // extern "C"

@@ -29,7 +29,8 @@ SYMBOLS = ["lopro_version", "lopro_status_str", "lopro_check_desc", "lopro_packe
            "lopro_residual_rotate", "lopro_rtn_quantize", "lopro_quantize_workspace_bytes", "lopro_quantize_layer",
            "lopro_block_add_rmsnorm", "lopro_block_rope_append", "lopro_block_attention_workspace_bytes",
            "lopro_block_attention_decode", "lopro_block_silu_mul", "lopro_experts_workspace_bytes",
-           "lopro_linear_fwd_experts_path", "lopro_linear_fwd_experts"]
+           "lopro_linear_fwd_experts_path", "lopro_linear_fwd_experts", "lopro_vq_packed_bytes", "lopro_vq_workspace_bytes",
+           "lopro_vq_pack", "lopro_vq_linear_fwd"]
 
 
 class Desc(ctypes.Structure):
@@ -48,6 +49,12 @@ class LoproError(RuntimeError):
 
 
 _lib = None
+
+
+class VqDesc(ctypes.Structure):
+    """lopro_vq_desc: the vector-quantized record (4-D centroids, 8-bit indices)."""
+    _fields_ = [("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32), ("cb_rows", ctypes.c_int32), ("cb_cols", ctypes.c_int32),
+                ("block_size", ctypes.c_int32), ("identity_cols", ctypes.c_int32), ("rank", ctypes.c_int32)]
 
 
 def lib():
@@ -116,6 +123,15 @@ def lib():
         L.lopro_quantize_layer.restype = ctypes.c_int
         L.lopro_quantize_layer.argtypes = [dp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         f32 = ctypes.c_float
+        vdp = ctypes.POINTER(VqDesc)
+        L.lopro_vq_packed_bytes.restype = sz
+        L.lopro_vq_packed_bytes.argtypes = [vdp]
+        L.lopro_vq_workspace_bytes.restype = sz
+        L.lopro_vq_workspace_bytes.argtypes = [vdp, i32]
+        L.lopro_vq_pack.restype = ctypes.c_int
+        L.lopro_vq_pack.argtypes = [vdp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.lopro_vq_linear_fwd.restype = ctypes.c_int
+        L.lopro_vq_linear_fwd.argtypes = [vdp, vp, vp, i64, vp, i64, i32, i32, vp, sz, vp]
         L.lopro_experts_workspace_bytes.restype = sz
         L.lopro_experts_workspace_bytes.argtypes = [dp, i32, i32]
         L.lopro_linear_fwd_experts_path.restype = i32
@@ -408,6 +424,46 @@ def linear_fwd_experts(desc, blobs, row_offsets, x, out_dtype=OUT_BF16, workspac
     st = lib().lopro_linear_fwd_experts(ctypes.byref(desc), n, ptrs, _offsets(row_offsets), _ptr(x), x.stride(0), _ptr(y),
                                         y.stride(0), out_dtype, _ptr(workspace), workspace.numel(), _stream())
     _check(st, "lopro_linear_fwd_experts")
+    return y
+
+
+def make_vq_desc(d_in, d_out, cb_rows, cb_cols, block_size, identity_cols=None, rank=0):
+    return VqDesc(d_in, d_out, cb_rows, cb_cols, block_size, block_size if identity_cols is None else identity_cols, rank)
+
+
+def vq_packed_bytes(desc):
+    return lib().lopro_vq_packed_bytes(ctypes.byref(desc))
+
+
+def vq_workspace_bytes(desc, T):
+    return lib().lopro_vq_workspace_bytes(ctypes.byref(desc), T)
+
+
+def vq_pack(desc, idx, codebooks_bf16, perm, A_f16=None, B_f16=None):
+    """lopro_vq_pack: idx uint8 [m][n/4], codebooks int16 bf16 bits [row groups][column groups][256][4], perm int32 [n],
+    A, B int16 fp16 bits (None with rank 0) -> packed device bytes."""
+    nbytes = vq_packed_bytes(desc)
+    if nbytes == 0:
+        raise LoproError(ERR_UNSUPPORTED, "lopro_vq_packed_bytes")
+    out = torch.empty(nbytes, dtype=torch.uint8, device=idx.device)
+    st = lib().lopro_vq_pack(ctypes.byref(desc), _ptr(_dev(idx, 1)), _ptr(_dev(codebooks_bf16, 2)), _ptr(_dev(perm, 4)),
+                             _ptr(None if A_f16 is None else _dev(A_f16, 2)), _ptr(None if B_f16 is None else _dev(B_f16, 2)),
+                             _ptr(out), out.numel(), _stream())
+    _check(st, "lopro_vq_pack")
+    return out
+
+
+def vq_linear_fwd(desc, packed, x, out_dtype=OUT_BF16, workspace=None, y=None):
+    """lopro_vq_linear_fwd: x bf16 [T][n] device -> y [T][m]."""
+    T = x.shape[0]
+    if workspace is None:
+        workspace = torch.zeros(max(vq_workspace_bytes(desc, T), 256), dtype=torch.uint8, device=x.device)
+    if y is None:
+        y = torch.empty((T, desc.d_out), dtype=torch.float32 if out_dtype == OUT_F32 else torch.bfloat16, device=x.device)
+    st = lib().lopro_vq_linear_fwd(ctypes.byref(desc), _ptr(packed), _ptr(x), x.stride(0) if T > 1 else max(x.stride(0), desc.d_in),
+                                   _ptr(y), y.stride(0) if T > 1 else max(y.stride(0), desc.d_out), out_dtype, T, _ptr(workspace),
+                                   workspace.numel(), _stream())
+    _check(st, "lopro_vq_linear_fwd")
     return y
 
 

@@ -17,7 +17,8 @@ def _built():
 
 
 def _declared_symbols():
-    text = open(os.path.join(ROOT, "include", "lopro.h")).read() + open(os.path.join(ROOT, "include", "lopro_block.h")).read()
+    text = open(os.path.join(ROOT, "include", "lopro.h")).read() + open(os.path.join(ROOT, "include", "lopro_block.h")).read() + \
+        open(os.path.join(ROOT, "include", "lopro_vq.h")).read()
     return sorted(set(re.findall(r"LOPRO_API[^;(]*?\b(lopro_\w+)\s*\(", text)))
 
 
