@@ -770,6 +770,59 @@ def measure_experts(dev, peaks, reps=20):
     return out
 
 
+def measure_vq(dev, peaks, reps=20):
+    """The vector-quantized variant at decode: 8192 -> 28672 (the shape of configuration 4), 4-D centroids with 8-bit indices
+    (2 bits per weight), codebooks of 512 x 256, block 256, rank 16; a ring of 3 distinct records (198 MB), 1 and 16 tokens."""
+    import torch
+    from paper_2601_19675_b200 import lopro, synth
+    n, m, cr, cc, b, r, ring = 8192, 28672, 512, 256, 256, 16, 3
+    d = lopro.make_vq_desc(n, m, cr, cc, b, rank=r)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4321)
+    a_bits, b_bits = synth.factors(m, n, r, seed=9)
+
+    def dev16(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev)
+
+    perm = torch.from_numpy(synth.permutation(n, seed=9)).to(dev)
+    blobs = []
+    for _ in range(ring):
+        idx = torch.randint(0, 256, (m, n // 4), dtype=torch.uint8, device=dev, generator=gen)
+        books = (torch.randn((m // cr, n // cc, 256, 4), device=dev, generator=gen) * 0.02).to(torch.bfloat16).view(torch.int16)
+        blobs.append(lopro.vq_pack(d, idx, books, perm, dev16(a_bits), dev16(b_bits)))
+    del idx, books
+    out = {}
+    for T in (1, 16):
+        x = dev16(synth.activations(T, n, seed=10)).view(torch.bfloat16)
+        y = torch.empty((T, m), dtype=torch.bfloat16, device=dev)
+        ws = torch.zeros(lopro.vq_workspace_bytes(d, T), dtype=torch.uint8, device=dev)
+        nbytes = m * (n // 4) + (m // cr) * (n // cc) * 2048 + (m * r + r * n) * 2 + n * 4 + T * (n + m) * 2
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            for blob in blobs:
+                lopro.vq_linear_fwd(d, blob, x, lopro.OUT_BF16, workspace=ws, y=y)
+            stream.synchronize()
+            assert lopro.workspace_status(ws) == lopro.OK and bool(torch.isfinite(y.float()).all())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for blob in blobs:
+                    lopro.vq_linear_fwd(d, blob, x, lopro.OUT_BF16, workspace=ws, y=y)
+            for _ in range(3):
+                graph.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(reps):
+                graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (reps * ring)
+        out[f"T{T}"] = dict(us_per_layer=us, tokens_per_s=T / (us * 1e-6), algorithmic_bytes=nbytes,
+                            achieved_gbs=nbytes / (us * 1e-6) / 1e9, frac_of_measured_hbm=nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                            gpu_launches_per_layer=3)
+    out["workload"] = "vector-quantized record 8192 -> 28672: 8-bit indices of 4-D centroids, codebooks of 512 x 256, block 256, rank 16"
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -815,7 +868,7 @@ def main():
 
     if args.offline:
         if rank == 0:
-            print(json.dumps(dict(offline=measure_offline(dev, measured_peaks()), experts=measure_experts(dev, measured_peaks()),
+            print(json.dumps(dict(offline=measure_offline(dev, measured_peaks()), experts=measure_experts(dev, measured_peaks()), vq=measure_vq(dev, measured_peaks()),
                                   n_gpus=1, data="synthetic", dtype="f32")))
         if world > 1:
             dist.destroy_process_group()
@@ -846,6 +899,7 @@ def main():
         if rank == 0:
             line["offline"] = measure_offline(dev, measured_peaks())
             line["experts"] = measure_experts(dev, measured_peaks())
+            line["vq"] = measure_vq(dev, measured_peaks())
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

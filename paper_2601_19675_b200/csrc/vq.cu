@@ -20,6 +20,7 @@ constexpr uint32_t kVqMagic = 0x5156504Cu;  // "LPVQ"
 constexpr int kVqHeader = 256;
 constexpr int kVqRowsPerCta = 64;           // four warps, sixteen rows each
 constexpr int kVqBookBytes = 256 * 4 * 2;   // one codebook
+constexpr int kVqSection = 8;               // codebooks per shared-memory buffer
 
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -37,7 +38,6 @@ lopro_status vq_check(const lopro_vq_desc* d) {
     if (d->rank < 0 || d->rank > 512 || d->d_in % d->cb_cols) return LOPRO_ERR_INVALID_ARG;
     if (d->d_in % 64 || d->d_out % kVqRowsPerCta || d->cb_rows % kVqRowsPerCta || d->cb_cols % 64) return LOPRO_ERR_UNSUPPORTED;
     if (d->d_in > 32768 || d->d_out > (1 << 20)) return LOPRO_ERR_UNSUPPORTED;
-    if ((size_t)(d->d_in / d->cb_cols) * kVqBookBytes > 160 * 1024) return LOPRO_ERR_UNSUPPORTED;  // a row group's books in shared memory
     return LOPRO_OK;
 }
 
@@ -124,6 +124,54 @@ __global__ void vq_copy_padded_kernel(const __half* __restrict__ src, int rows, 
     dst[i] = c < cols ? src[(size_t)r * cols + c] : __float2half(0.0f);
 }
 
+// t[tok][j] = sum_k B[j][k] x[tok][k] for one row j of B and up to 8 tokens per CTA (grid: r_pad x token groups):
+// 16-byte loads strided over the row, fp32 sums, one rounding to fp16.
+__global__ void __launch_bounds__(256) vq_lowrank_down_kernel(const __half* __restrict__ B, const __nv_bfloat16* __restrict__ x,
+                                                              int64_t ldx, __half* __restrict__ t, int n, int r_pad, int T) {
+    __shared__ float part[8][8];
+    const int j = blockIdx.x, tok0 = blockIdx.y * 8, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nt = min(8, T - tok0);
+    float acc[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) acc[q] = 0.0f;
+    for (int c = tid; c < (n >> 3); c += 256) {
+        const uint4 bv = __ldg(reinterpret_cast<const uint4*>(B + (size_t)j * n) + c);
+        const __half2* bh = reinterpret_cast<const __half2*>(&bv);
+        float bf[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __half22float2(bh[e]);
+            bf[2 * e] = f.x;
+            bf[2 * e + 1] = f.y;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            if (q < nt) {
+                const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)(tok0 + q) * ldx) + c);
+                const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xv);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __bfloat1622float2(xh[e]);
+                    acc[q] = fmaf(bf[2 * e], f.x, acc[q]);
+                    acc[q] = fmaf(bf[2 * e + 1], f.y, acc[q]);
+                }
+            }
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], o);
+        if (lane == 0) part[warp][q] = acc[q];
+    }
+    __syncthreads();
+    if (tid < nt) {
+        float v = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += part[w][tid];
+        t[(size_t)(tok0 + tid) * r_pad + j] = __float2half_rn(v);
+    }
+}
+
 struct VqParams {
     const uint8_t* idx;          // [m][n / 4]
     const unsigned char* books;  // [n_rg][n_cg][256][4] bf16
@@ -144,16 +192,24 @@ struct VqParams {
 // token's rotated row per lane and super-tile), so both operands agree on which column a k-slot means.
 template <int NT>
 __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
-    extern __shared__ __align__(16) unsigned char vq_smem[];  // [n_cg][256][4] bf16
+    extern __shared__ __align__(16) unsigned char vq_smem[];  // two sections of kVqSection codebooks
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int row0 = blockIdx.x * kVqRowsPerCta + warp * 16;
     const int rg = (blockIdx.x * kVqRowsPerCta) / p.cb_rows;
-    {
-        const uint4* src = reinterpret_cast<const uint4*>(p.books + (size_t)rg * p.n_cg * kVqBookBytes);
-        uint4* dst = reinterpret_cast<uint4*>(vq_smem);
-        for (int i = tid; i < p.n_cg * (kVqBookBytes / 16); i += 128) dst[i] = __ldg(src + i);
-    }
-    __syncthreads();
+    // The row group's codebooks pass through shared memory in sections of kVqSection books, the next section copied
+    // asynchronously while the warps work on the present one (a CTA then holds 32 KB instead of all its books, and
+    // every CTA of a large layer is resident at once).
+    const unsigned char* books_g = p.books + (size_t)rg * p.n_cg * kVqBookBytes;
+    const int n_sections = (p.n_cg + kVqSection - 1) / kVqSection;
+    auto copy_section = [&](int sec) {
+        const int first = sec * kVqSection, cnt = min(kVqSection, p.n_cg - first);
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(vq_smem) + (uint32_t)((sec & 1) * kVqSection * kVqBookBytes);
+        const unsigned char* src = books_g + (size_t)first * kVqBookBytes;
+        for (int i = tid; i < cnt * (kVqBookBytes / 16); i += 128)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * (uint32_t)i), "l"(src + 16 * (size_t)i) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    copy_section(0);
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
@@ -161,42 +217,84 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
         for (int e = 0; e < 4; ++e) acc[nt][e] = 0.0f;
     const uint32_t* idx_lo = reinterpret_cast<const uint32_t*>(p.idx + (size_t)(row0 + g) * (p.n / 4)) + t;
     const uint32_t* idx_hi = reinterpret_cast<const uint32_t*>(p.idx + (size_t)(row0 + g + 8) * (p.n / 4)) + t;
-    const uint32_t books_s = (uint32_t)__cvta_generic_to_shared(vq_smem);
     const int n_super = p.n >> 6, per_book = p.cb_cols >> 6;
-    uint32_t w_lo = __ldg(idx_lo), w_hi = __ldg(idx_hi);
-    for (int S = 0; S < n_super; ++S) {
-        const uint32_t cur_lo = w_lo, cur_hi = w_hi;
-        if (S + 1 < n_super) {  // the next super-tile's indices are in flight during this one's products
-            w_lo = __ldg(idx_lo + 4 * (S + 1));
-            w_hi = __ldg(idx_hi + 4 * (S + 1));
-        }
-        // activations: 32 bytes (columns 64 S + 16 t .. + 15) of token 8 nt + g
+    // Everything a super-tile needs from global memory -- one word of indices per row and 32 bytes of every token's
+    // rotated row -- is requested one super-tile ahead and kept in registers meanwhile (two register stages).
+    struct Stage {
+        uint32_t w_lo, w_hi;
         uint4 xa[NT], xb[NT];
+    };
+    const uint4* xptr[NT];
+    bool live[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int tok = nt * 8 + g;
+        live[nt] = tok < p.T;
+        xptr[nt] = reinterpret_cast<const uint4*>(p.xrot + (size_t)(live[nt] ? tok : 0) * p.n + 16 * t);
+    }
+    auto fetch = [&](Stage& st, int S) {
+        st.w_lo = __ldg(idx_lo + 4 * S);
+        st.w_hi = __ldg(idx_hi + 4 * S);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            const int tok = nt * 8 + g;
-            if (tok < p.T) {
-                const uint4* xr = reinterpret_cast<const uint4*>(p.xrot + (size_t)tok * p.n + 64 * S + 16 * t);
-                xa[nt] = __ldg(xr);
-                xb[nt] = __ldg(xr + 1);
-            } else {
-                xa[nt] = make_uint4(0, 0, 0, 0);
-                xb[nt] = make_uint4(0, 0, 0, 0);
-            }
+            st.xa[nt] = live[nt] ? __ldg(xptr[nt] + 8 * S) : make_uint4(0, 0, 0, 0);
+            st.xb[nt] = live[nt] ? __ldg(xptr[nt] + 8 * S + 1) : make_uint4(0, 0, 0, 0);
         }
-        const uint32_t book = books_s + (uint32_t)((S / per_book) * kVqBookBytes);
+    };
+    uint32_t book = 0;  // byte offset of the present codebook in the shared-memory buffers
+    int in_book = 0;    // super-tiles of it already done
+    auto consume = [&](const Stage& st) {
+        // all eight centroids first (plain shared-memory loads, free to be scheduled together), then the products
+        const unsigned char* bk = vq_smem + book;
+        uint32_t a[4][4];
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
-            uint32_t a[4];
-            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[0]), "=r"(a[2]) : "r"(book + 8u * ((cur_lo >> (8 * s)) & 255u)));
-            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[1]), "=r"(a[3]) : "r"(book + 8u * ((cur_hi >> (8 * s)) & 255u)));
+            const uint2 lo = *reinterpret_cast<const uint2*>(bk + 8u * ((st.w_lo >> (8 * s)) & 255u));
+            const uint2 hi = *reinterpret_cast<const uint2*>(bk + 8u * ((st.w_hi >> (8 * s)) & 255u));
+            a[s][0] = lo.x;
+            a[s][2] = lo.y;
+            a[s][1] = hi.x;
+            a[s][3] = hi.y;
+        }
+#pragma unroll
+        for (int s = 0; s < 4; ++s)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                const uint4& v = s < 2 ? xa[nt] : xb[nt];
+                const uint4& v = s < 2 ? st.xa[nt] : st.xb[nt];
                 const uint32_t b0 = (s & 1) ? v.z : v.x, b1 = (s & 1) ? v.w : v.y;
-                mma_bf16(acc[nt], a, b0, b1);
+                mma_bf16(acc[nt], a[s], b0, b1);
             }
+        if (++in_book == per_book) {
+            in_book = 0;
+            book += kVqBookBytes;
         }
+    };
+    Stage stA, stB;
+    const int per_section = per_book * kVqSection;  // super-tiles per section of codebooks
+    int S = 0;
+    for (int sec = 0; sec < n_sections; ++sec) {
+        const int S_end = min(n_super, (sec + 1) * per_section);
+        fetch(stA, S);  // (in flight while the section's codebooks land)
+        if (sec + 1 < n_sections) {
+            copy_section(sec + 1);  // into the buffer whose last reader passed the barrier at the end of section sec - 1
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncthreads();  // section sec has landed for every warp
+        book = (uint32_t)((sec & 1) * kVqSection * kVqBookBytes);
+        in_book = 0;
+        for (; S + 1 < S_end; S += 2) {
+            fetch(stB, S + 1);
+            consume(stA);
+            if (S + 2 < S_end) fetch(stA, S + 2);
+            consume(stB);
+        }
+        if (S < S_end) {  // an odd super-tile at the end of the section: stage A holds it
+            consume(stA);
+            ++S;
+        }
+        __syncthreads();  // every warp is done with section sec before its buffer is overwritten
     }
     // low-rank term and store: the lane holds rows g, g + 8 and tokens 8 nt + 2 t, + 1
 #pragma unroll
@@ -230,10 +328,7 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
 
 template <int NT>
 cudaError_t launch_vq_decode(const VqParams& p, cudaStream_t s) {
-    static unsigned long long attr_done = 0;
-    cudaError_t e = ensure_dynamic_smem(vq_decode_kernel<NT>, 160 * 1024, &attr_done);
-    if (e != cudaSuccess) return e;
-    vq_decode_kernel<NT><<<p.m / kVqRowsPerCta, 128, (size_t)p.n_cg * kVqBookBytes, s>>>(p);
+    vq_decode_kernel<NT><<<p.m / kVqRowsPerCta, 128, 2 * kVqSection * kVqBookBytes, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -336,10 +431,14 @@ lopro_status lopro_vq_linear_fwd(const lopro_vq_desc* desc, const void* packed, 
         return LOPRO_ERR_CUDA;
     if (d.rank > 0) {
         const __half* B = (const __half*)(blob + L.off_b);
-        const cudaError_t e = T > kDecodeMaxT
-                                  ? launch_lowrank_down_mma(sd, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx,
-                                                            (float*)(ws + W.off_part), tbuf, T, s)
-                                  : launch_lowrank_down(sd, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, tbuf, T, s);
+        cudaError_t e;
+        if (T > kDecodeMaxT) {
+            e = launch_lowrank_down_mma(sd, B, L.r_pad, (const __nv_bfloat16*)x_bf16, ldx, (float*)(ws + W.off_part), tbuf, T, s);
+        } else {
+            vq_lowrank_down_kernel<<<dim3(L.r_pad, (T + 7) / 8), 256, 0, s>>>(B, (const __nv_bfloat16*)x_bf16, ldx, tbuf, d.d_in,
+                                                                            L.r_pad, T);
+            e = cudaGetLastError();
+        }
         if (e != cudaSuccess) return LOPRO_ERR_CUDA;
     }
     const size_t esz = out_dtype == LOPRO_OUT_F32 ? 4 : 2;
