@@ -190,12 +190,16 @@ struct VqParams {
 // m16n8k16 products of a super-tile uses vector 4 t + s, i.e. the lane's k-slots {2t, 2t+1, 2t+8, 2t+9} stand for
 // the columns 16 t + 4 s .. + 3.  The activation fragments follow the same assignment (32 contiguous bytes of a
 // token's rotated row per lane and super-tile), so both operands agree on which column a k-slot means.
-template <int NT>
+// KS = 4: the four warps share ONE 16-row tile and take every fourth super-tile each (grid = m / 16; four times the
+// warps per SM for the same registers per warp, which is what hides the lookup latency); their sums meet in shared
+// memory at the end.  KS = 1: a warp per tile over all of K (grid = m / 64).
+template <int NT, int KS>
 __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
     extern __shared__ __align__(16) unsigned char vq_smem[];  // two sections of kVqSection codebooks
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-    const int row0 = blockIdx.x * kVqRowsPerCta + warp * 16;
-    const int rg = (blockIdx.x * kVqRowsPerCta) / p.cb_rows;
+    const int row0 = KS == 1 ? blockIdx.x * kVqRowsPerCta + warp * 16 : blockIdx.x * 16;
+    const int kq = KS == 1 ? 0 : warp;  // this warp's share of K: super-tiles S = kq (mod KS)
+    const int rg = row0 / p.cb_rows;
     // The row group's codebooks pass through shared memory in sections of kVqSection books, the next section copied
     // asynchronously while the warps work on the present one (a CTA then holds 32 KB instead of all its books, and
     // every CTA of a large layer is resident at once).
@@ -241,20 +245,22 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
             st.xb[nt] = live[nt] ? __ldg(xptr[nt] + 8 * S + 1) : make_uint4(0, 0, 0, 0);
         }
     };
+    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(vq_smem);
     uint32_t book = 0;  // byte offset of the present codebook in the shared-memory buffers
     int in_book = 0;    // super-tiles of it already done
     auto consume = [&](const Stage& st) {
-        // all eight centroids first (plain shared-memory loads, free to be scheduled together), then the products
-        const unsigned char* bk = vq_smem + book;
+        while (in_book >= per_book) {  // the codebook of this super-tile
+            in_book -= per_book;
+            book += kVqBookBytes;
+        }
+        // all eight centroids first (32-bit shared-space addresses; the loads keep their place before the products),
+        // then the products
+        const uint32_t bk = smem_s + book;
         uint32_t a[4][4];
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
-            const uint2 lo = *reinterpret_cast<const uint2*>(bk + 8u * ((st.w_lo >> (8 * s)) & 255u));
-            const uint2 hi = *reinterpret_cast<const uint2*>(bk + 8u * ((st.w_hi >> (8 * s)) & 255u));
-            a[s][0] = lo.x;
-            a[s][2] = lo.y;
-            a[s][1] = hi.x;
-            a[s][3] = hi.y;
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[s][0]), "=r"(a[s][2]) : "r"(bk + 8u * ((st.w_lo >> (8 * s)) & 255u)));
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[s][1]), "=r"(a[s][3]) : "r"(bk + 8u * ((st.w_hi >> (8 * s)) & 255u)));
         }
 #pragma unroll
         for (int s = 0; s < 4; ++s)
@@ -264,17 +270,14 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
                 const uint32_t b0 = (s & 1) ? v.z : v.x, b1 = (s & 1) ? v.w : v.y;
                 mma_bf16(acc[nt], a[s], b0, b1);
             }
-        if (++in_book == per_book) {
-            in_book = 0;
-            book += kVqBookBytes;
-        }
+        in_book += KS;
     };
     Stage stA, stB;
     const int per_section = per_book * kVqSection;  // super-tiles per section of codebooks
-    int S = 0;
     for (int sec = 0; sec < n_sections; ++sec) {
         const int S_end = min(n_super, (sec + 1) * per_section);
-        fetch(stA, S);  // (in flight while the section's codebooks land)
+        int S = sec * per_section + kq;
+        if (S < S_end) fetch(stA, S);  // (in flight while the section's codebooks land)
         if (sec + 1 < n_sections) {
             copy_section(sec + 1);  // into the buffer whose last reader passed the barrier at the end of section sec - 1
             asm volatile("cp.async.wait_group 1;" ::: "memory");
@@ -283,24 +286,44 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
         }
         __syncthreads();  // section sec has landed for every warp
         book = (uint32_t)((sec & 1) * kVqSection * kVqBookBytes);
-        in_book = 0;
-        for (; S + 1 < S_end; S += 2) {
-            fetch(stB, S + 1);
+        in_book = kq;
+        for (; S + KS < S_end; S += 2 * KS) {
+            fetch(stB, S + KS);
             consume(stA);
-            if (S + 2 < S_end) fetch(stA, S + 2);
+            if (S + 2 * KS < S_end) fetch(stA, S + 2 * KS);
             consume(stB);
         }
-        if (S < S_end) {  // an odd super-tile at the end of the section: stage A holds it
-            consume(stA);
-            ++S;
-        }
+        if (S < S_end) consume(stA);  // an odd one at the end of the section: stage A holds it
         __syncthreads();  // every warp is done with section sec before its buffer is overwritten
+    }
+    if (KS > 1) {
+        // the four shares of K meet in shared memory (the codebook buffers are free after the last barrier); warp w then
+        // finishes token tile w
+        float* part = reinterpret_cast<float*>(vq_smem);  // [KS][NT][4][32]
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) part[((warp * NT + nt) * 4 + e) * 32 + lane] = acc[nt][e];
+        __syncthreads();
+        if (warp >= NT) return;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+            if (nt == warp) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float v = 0.0f;
+#pragma unroll
+                    for (int w = 0; w < KS; ++w) v += part[((w * NT + nt) * 4 + e) * 32 + lane];
+                    acc[nt][e] = v;
+                }
+            }
     }
     // low-rank term and store: the lane holds rows g, g + 8 and tokens 8 nt + 2 t, + 1
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
+            if (KS > 1 && nt != warp) continue;
             const int row = row0 + g + 8 * (e >> 1), tok = nt * 8 + 2 * t + (e & 1);
             if (tok >= p.T) continue;
             float v = acc[nt][e];
@@ -328,7 +351,7 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
 
 template <int NT>
 cudaError_t launch_vq_decode(const VqParams& p, cudaStream_t s) {
-    vq_decode_kernel<NT><<<p.m / kVqRowsPerCta, 128, 2 * kVqSection * kVqBookBytes, s>>>(p);
+    vq_decode_kernel<NT, 4><<<p.m / 16, 128, 2 * kVqSection * kVqBookBytes, s>>>(p);
     return cudaGetLastError();
 }
 
