@@ -552,6 +552,9 @@ def measure(args, name, steps, warmup, rank, world, local, dev, dist, with_e2e=T
     import torch
     from paper_2601_19675_b200 import lopro
     w = Workload(args, name, rank, dev)
+    # the stack alternates single-layer and grouped forwards: one set of kernel variants for both (see the switch's
+    # description in lopro.h); every other workload launches single layers only and keeps the default
+    lopro.configure(lopro.OPT_ONE_KERNEL_SET, 1 if w.cfg == "cfg5" else 0)
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):
         w.verify_pass()
@@ -656,6 +659,9 @@ def measure(args, name, steps, warmup, rank, world, local, dev, dist, with_e2e=T
                           d2h_bytes_per_step=w.d2h, steps=e2e_steps,
                           note="one pass per step through the host-buffer entry point (pinned host x in, host y out)")
     rec["_workload"] = w
+    if w.cfg == "cfg5":
+        rec["config"]["one_kernel_set"] = 1
+        lopro.configure(lopro.OPT_ONE_KERNEL_SET, 0)
     return rec
 
 

@@ -350,19 +350,13 @@ constexpr int kPrologueMaxSmem = 200 * 1024;  // one row of x: d_in <= 102400
 //    (8 / tpr CTAs per row): the low-rank intermediate "Y = V X".
 // Launched with programmatic stream serialization: perm and B (layer data) are pulled into L2 before the
 // wait, everything is loaded after it.
-template <bool STAGED>
-__global__ void __launch_bounds__(256)
-prologue_kernel(const __nv_bfloat16* __restrict__ x0, int64_t ldx, const int32_t* __restrict__ perm0,
-                const __half* __restrict__ B0, unsigned char* __restrict__ act_image0, __half* __restrict__ t0,
-                int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T_grid,
-                int tpr, const ImageOut img, const PrologueSiblings sibs, const Lr8Args lr8) {
-    // sibling layers (grid z): the same x, each layer its own permutation, B and outputs
-    const int32_t* __restrict__ perm = perm0;
-    const __half* __restrict__ B = B0;
-    unsigned char* __restrict__ act_image = act_image0;
-    __half* __restrict__ t = t0;
-    const __nv_bfloat16* __restrict__ x = x0;
-    int T = T_grid;  // T_grid shapes the grid; T is the number of token rows of this CTA's layer
+// A launch for a single layer carries no sibling table (several hundred bytes of kernel parameters less).
+struct NoPrologueSiblings {};
+__device__ __forceinline__ void select_prologue_sibling(const NoPrologueSiblings&, const int32_t*&, const __half*&,
+                                                        unsigned char*&, __half*&, const __nv_bfloat16*&, int&) {}
+__device__ __forceinline__ void select_prologue_sibling(const PrologueSiblings& sibs, const int32_t*& perm, const __half*& B,
+                                                        unsigned char*& act_image, __half*& t, const __nv_bfloat16*& x,
+                                                        int& T) {
 #pragma unroll
     for (int i = 0; i < kMaxSiblings - 1; ++i)
         if ((int)blockIdx.z == i + 1) {
@@ -379,6 +373,22 @@ prologue_kernel(const __nv_bfloat16* __restrict__ x0, int64_t ldx, const int32_t
                 T = sibs.T_of[i];
             }
     }
+}
+
+template <bool STAGED, typename SIBS>
+__global__ void __launch_bounds__(256)
+prologue_kernel(const __nv_bfloat16* __restrict__ x0, int64_t ldx, const int32_t* __restrict__ perm0,
+                const __half* __restrict__ B0, unsigned char* __restrict__ act_image0, __half* __restrict__ t0,
+                int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T_grid,
+                int tpr, const ImageOut img, const SIBS sibs, const Lr8Args lr8) {
+    // sibling layers (grid z): the same x (or each its own rows), each layer its own permutation, B and outputs
+    const int32_t* perm = perm0;
+    const __half* B = B0;
+    unsigned char* act_image = act_image0;
+    __half* t = t0;
+    const __nv_bfloat16* x = x0;
+    int T = T_grid;  // T_grid shapes the grid; T is the number of token rows of this CTA's layer
+    select_prologue_sibling(sibs, perm, B, act_image, t, x, T);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nchunks = (n + 255) >> 8;
     const int tok0 = blockIdx.y * 8;
@@ -576,7 +586,11 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
     const int rot_ctas = staged ? live * ((nchunks + 7) / 8) : nchunks;
     if (staged && (size_t)d.d_in * 2 > 48 * 1024) {  // a row of x beyond the default limit
         static unsigned long long attr_done = 0;
-        cudaError_t e = ensure_dynamic_smem(prologue_kernel<true>, kPrologueMaxSmem, &attr_done);
+        cudaError_t e = ensure_dynamic_smem(prologue_kernel<true, PrologueSiblings>, kPrologueMaxSmem, &attr_done);
+        if (e == cudaSuccess) {
+            static unsigned long long attr_done2 = 0;
+            e = ensure_dynamic_smem(prologue_kernel<true, NoPrologueSiblings>, kPrologueMaxSmem, &attr_done2);
+        }
         if (e != cudaSuccess) return e;
     }
     cfg.gridDim = dim3(row_ctas + rot_ctas, (T + 7) / 8, 1 + sibs.n);
@@ -589,9 +603,16 @@ cudaError_t launch_prologue(const lopro_desc& d, const int32_t* perm, const __ha
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     const int rp = d.rank > 0 ? r_pad : 0;
-    return staged ? cudaLaunchKernelEx(&cfg, prologue_kernel<true>, x, ldx, perm, B, act_image, t, status, d.d_in,
+    if (sibs.n == 0 && !sibs.own_rows && option(LOPRO_OPT_ONE_KERNEL_SET) != 1) {
+        const NoPrologueSiblings none;
+        return staged ? cudaLaunchKernelEx(&cfg, prologue_kernel<true, NoPrologueSiblings>, x, ldx, perm, B, act_image, t, status,
+                                           d.d_in, d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, none, lr8)
+                      : cudaLaunchKernelEx(&cfg, prologue_kernel<false, NoPrologueSiblings>, x, ldx, perm, B, act_image, t, status,
+                                           d.d_in, d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, none, lr8);
+    }
+    return staged ? cudaLaunchKernelEx(&cfg, prologue_kernel<true, PrologueSiblings>, x, ldx, perm, B, act_image, t, status, d.d_in,
                                        d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, sibs, lr8)
-                  : cudaLaunchKernelEx(&cfg, prologue_kernel<false>, x, ldx, perm, B, act_image, t, status, d.d_in,
+                  : cudaLaunchKernelEx(&cfg, prologue_kernel<false, PrologueSiblings>, x, ldx, perm, B, act_image, t, status, d.d_in,
                                        d.identity_cols, d.block_size, inv, rp, t_pad, T, tpr, img, sibs, lr8);
 }
 

@@ -68,6 +68,11 @@ struct StreamSiblings {
     int T[kMaxSiblings - 1];  // token rows of the sibling (experts of a mixture layer differ; otherwise all alike)
 };
 
+// A launch of a single layer carries no table at all (the table is several hundred bytes of kernel parameters, and
+// their mere presence was measured at 0.15 us per launch of the smallest layers).
+struct NoSiblings {};
+__device__ __forceinline__ int select_sibling(StreamParams&, const NoSiblings&) { return (int)blockIdx.x; }
+
 // The layer a CTA works on: patches the per-layer fields of the parameters, returns the CTA's index within the layer.
 __device__ __forceinline__ int select_sibling(StreamParams& p, const StreamSiblings& sibs) {
     int bx = (int)blockIdx.x;
@@ -88,9 +93,9 @@ __device__ __forceinline__ int select_sibling(StreamParams& p, const StreamSibli
     return bx;
 }
 
-template <int BITS, int NT, int RT>
+template <int BITS, int NT, int RT, typename SIBS>
 __global__ void __launch_bounds__(kThreads, 1)
-stream_kernel(const StreamParams p_in, const StreamSiblings sibs) {
+stream_kernel(const StreamParams p_in, const SIBS sibs) {
     StreamParams p = p_in;
     const int bx = select_sibling(p, sibs);
     extern __shared__ __align__(128) unsigned char smem[];
@@ -353,9 +358,9 @@ constexpr int kWideThreads = kWideWarps * 32;
 constexpr int kRedTok = 36;                 // floats between tokens
 constexpr int kRedStep = 8 * kRedTok + 8;   // floats between steps
 
-template <int BITS>
+template <int BITS, typename SIBS>
 __global__ void __launch_bounds__(kWideThreads, 1)
-stream_wide_kernel(const StreamParams p_in, const StreamSiblings sibs) {
+stream_wide_kernel(const StreamParams p_in, const SIBS sibs) {
     StreamParams p = p_in;
     const int bx = select_sibling(p, sibs);
     extern __shared__ __align__(128) unsigned char smem[];
@@ -518,10 +523,10 @@ stream_wide_kernel(const StreamParams p_in, const StreamSiblings sibs) {
     }
 }
 
-template <int BITS>
-cudaError_t launch_stream_wide(const StreamParams& p, const StreamSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
+template <int BITS, typename SIBS>
+cudaError_t launch_stream_wide_s(const StreamParams& p, const SIBS& sibs, int grid, int smem_bytes, cudaStream_t s) {
     static unsigned long long attr_done = 0;
-    cudaError_t e = ensure_dynamic_smem(stream_wide_kernel<BITS>, kStreamMaxSmem, &attr_done);
+    cudaError_t e = ensure_dynamic_smem(stream_wide_kernel<BITS, SIBS>, kStreamMaxSmem, &attr_done);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -533,13 +538,19 @@ cudaError_t launch_stream_wide(const StreamParams& p, const StreamSiblings& sibs
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, stream_wide_kernel<BITS>, p, sibs);
+    return cudaLaunchKernelEx(&cfg, stream_wide_kernel<BITS, SIBS>, p, sibs);
 }
 
-template <int BITS, int NT, int RT>
-cudaError_t launch_stream_k(const StreamParams& p, const StreamSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
+template <int BITS>
+cudaError_t launch_stream_wide(const StreamParams& p, const StreamSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
+    return sibs.n == 0 && option(LOPRO_OPT_ONE_KERNEL_SET) != 1 ? launch_stream_wide_s<BITS, NoSiblings>(p, NoSiblings{}, grid, smem_bytes, s)
+                       : launch_stream_wide_s<BITS, StreamSiblings>(p, sibs, grid, smem_bytes, s);
+}
+
+template <int BITS, int NT, int RT, typename SIBS>
+cudaError_t launch_stream_ks(const StreamParams& p, const SIBS& sibs, int grid, int smem_bytes, cudaStream_t s) {
     static unsigned long long attr_done = 0;
-    cudaError_t e = ensure_dynamic_smem(stream_kernel<BITS, NT, RT>, kStreamMaxSmem, &attr_done);
+    cudaError_t e = ensure_dynamic_smem(stream_kernel<BITS, NT, RT, SIBS>, kStreamMaxSmem, &attr_done);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -551,7 +562,13 @@ cudaError_t launch_stream_k(const StreamParams& p, const StreamSiblings& sibs, i
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, stream_kernel<BITS, NT, RT>, p, sibs);
+    return cudaLaunchKernelEx(&cfg, stream_kernel<BITS, NT, RT, SIBS>, p, sibs);
+}
+
+template <int BITS, int NT, int RT>
+cudaError_t launch_stream_k(const StreamParams& p, const StreamSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
+    return sibs.n == 0 && option(LOPRO_OPT_ONE_KERNEL_SET) != 1 ? launch_stream_ks<BITS, NT, RT, NoSiblings>(p, NoSiblings{}, grid, smem_bytes, s)
+                       : launch_stream_ks<BITS, NT, RT, StreamSiblings>(p, sibs, grid, smem_bytes, s);
 }
 
 template <int BITS>

@@ -76,6 +76,12 @@ struct TallSiblings {
     int T[kMaxSiblings - 1];  // token rows of the sibling
 };
 
+// A launch of a single layer carries no table (several hundred bytes of kernel parameters less).
+struct NoTallSiblings {};
+__device__ __forceinline__ int2 select_sibling(TallParams&, const NoTallSiblings&) {
+    return make_int2((int)blockIdx.x, (int)gridDim.x);
+}
+
 // The layer a CTA works on: patches the per-layer fields, returns the CTA's index among the layer's CTAs and
 // their number.
 __device__ __forceinline__ int2 select_sibling(TallParams& p, const TallSiblings& sibs) {
@@ -183,9 +189,9 @@ __device__ __forceinline__ void consume_stage(const unsigned char* stage, uint32
     }
 }
 
-template <int BITS, int NT>
+template <int BITS, int NT, typename SIBS>
 __global__ void __launch_bounds__(kThreads, 1)
-tall_kernel(const TallParams p_in, const TallSiblings sibs) {
+tall_kernel(const TallParams p_in, const SIBS sibs) {
     TallParams p = p_in;
     const int2 cta = select_sibling(p, sibs);  // x: index among the layer's CTAs, y: their number
     extern __shared__ __align__(128) unsigned char smem[];
@@ -446,10 +452,10 @@ bool plan_tall(const lopro_desc& d, int T, TallPlan* pl) {
     return true;
 }
 
-template <int BITS, int NT>
-cudaError_t launch_tall_k(const TallParams& p, const TallSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
+template <int BITS, int NT, typename SIBS>
+cudaError_t launch_tall_ks(const TallParams& p, const SIBS& sibs, int grid, int smem_bytes, cudaStream_t s) {
     static unsigned long long attr_done = 0;
-    cudaError_t e = ensure_dynamic_smem(tall_kernel<BITS, NT>, kStreamMaxSmem, &attr_done);
+    cudaError_t e = ensure_dynamic_smem(tall_kernel<BITS, NT, SIBS>, kStreamMaxSmem, &attr_done);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -461,7 +467,13 @@ cudaError_t launch_tall_k(const TallParams& p, const TallSiblings& sibs, int gri
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tall_kernel<BITS, NT>, p, sibs);
+    return cudaLaunchKernelEx(&cfg, tall_kernel<BITS, NT, SIBS>, p, sibs);
+}
+
+template <int BITS, int NT>
+cudaError_t launch_tall_k(const TallParams& p, const TallSiblings& sibs, int grid, int smem_bytes, cudaStream_t s) {
+    return sibs.n == 0 && option(LOPRO_OPT_ONE_KERNEL_SET) != 1 ? launch_tall_ks<BITS, NT, NoTallSiblings>(p, NoTallSiblings{}, grid, smem_bytes, s)
+                       : launch_tall_ks<BITS, NT, TallSiblings>(p, sibs, grid, smem_bytes, s);
 }
 
 template <int BITS>

@@ -152,7 +152,7 @@ def lib():
     return _lib
 
 
-OPT_NO_WIDE, OPT_NO_TALL, OPT_NO_CHUNKS, OPT_NO_TCGEN05, OPT_PREFILL_PAIRS = range(5)
+OPT_NO_WIDE, OPT_NO_TALL, OPT_NO_CHUNKS, OPT_NO_TCGEN05, OPT_PREFILL_PAIRS, OPT_ONE_KERNEL_SET = range(6)
 
 
 def configure(option, value):
