@@ -20,7 +20,9 @@ constexpr uint32_t kVqMagic = 0x5156504Cu;  // "LPVQ"
 constexpr int kVqHeader = 256;
 constexpr int kVqRowsPerCta = 64;           // four warps, sixteen rows each
 constexpr int kVqBookBytes = 256 * 4 * 2;   // one codebook
-constexpr int kVqSection = 8;               // codebooks per shared-memory buffer
+// codebooks per shared-memory buffer (two buffers): 6 with one token tile (24 KB, seven CTAs per SM, so that two waves
+// hold the grid of a 28672-row layer), 8 otherwise (the registers of the wider variants allow five CTAs per SM anyway)
+constexpr int kVqSectionMax = 8;
 
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -180,7 +182,7 @@ struct VqParams {
     const __half* t;             // [T][r_pad]
     void* y;
     int64_t ldy;
-    int out_f32, m, n, T, r_pad, cb_rows, cb_cols, n_cg;
+    int out_f32, m, n, T, r_pad, cb_rows, cb_cols, n_cg, section;
 };
 
 
@@ -195,19 +197,19 @@ struct VqParams {
 // memory at the end.  KS = 1: a warp per tile over all of K (grid = m / 64).
 template <int NT, int KS>
 __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
-    extern __shared__ __align__(16) unsigned char vq_smem[];  // two sections of kVqSection codebooks
+    extern __shared__ __align__(16) unsigned char vq_smem[];  // two sections of p.section codebooks
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int row0 = KS == 1 ? blockIdx.x * kVqRowsPerCta + warp * 16 : blockIdx.x * 16;
     const int kq = KS == 1 ? 0 : warp;  // this warp's share of K: super-tiles S = kq (mod KS)
     const int rg = row0 / p.cb_rows;
-    // The row group's codebooks pass through shared memory in sections of kVqSection books, the next section copied
+    // The row group's codebooks pass through shared memory in sections of p.section books, the next section copied
     // asynchronously while the warps work on the present one (a CTA then holds 32 KB instead of all its books, and
     // every CTA of a large layer is resident at once).
     const unsigned char* books_g = p.books + (size_t)rg * p.n_cg * kVqBookBytes;
-    const int n_sections = (p.n_cg + kVqSection - 1) / kVqSection;
+    const int n_sections = (p.n_cg + p.section - 1) / p.section;
     auto copy_section = [&](int sec) {
-        const int first = sec * kVqSection, cnt = min(kVqSection, p.n_cg - first);
-        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(vq_smem) + (uint32_t)((sec & 1) * kVqSection * kVqBookBytes);
+        const int first = sec * p.section, cnt = min(p.section, p.n_cg - first);
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(vq_smem) + (uint32_t)((sec & 1) * p.section * kVqBookBytes);
         const unsigned char* src = books_g + (size_t)first * kVqBookBytes;
         for (int i = tid; i < cnt * (kVqBookBytes / 16); i += 128)
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * (uint32_t)i), "l"(src + 16 * (size_t)i) : "memory");
@@ -273,7 +275,7 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
         in_book += KS;
     };
     Stage stA, stB;
-    const int per_section = per_book * kVqSection;  // super-tiles per section of codebooks
+    const int per_section = per_book * p.section;  // super-tiles per section of codebooks
     for (int sec = 0; sec < n_sections; ++sec) {
         const int S_end = min(n_super, (sec + 1) * per_section);
         int S = sec * per_section + kq;
@@ -285,7 +287,7 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
         __syncthreads();  // section sec has landed for every warp
-        book = (uint32_t)((sec & 1) * kVqSection * kVqBookBytes);
+        book = (uint32_t)((sec & 1) * p.section * kVqBookBytes);
         in_book = kq;
         for (; S + KS < S_end; S += 2 * KS) {
             fetch(stB, S + KS);
@@ -351,7 +353,7 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
 
 template <int NT>
 cudaError_t launch_vq_decode(const VqParams& p, cudaStream_t s) {
-    vq_decode_kernel<NT, 4><<<p.m / 16, 128, 2 * kVqSection * kVqBookBytes, s>>>(p);
+    vq_decode_kernel<NT, 4><<<p.m / 16, 128, 2 * p.section * kVqBookBytes, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -483,6 +485,7 @@ lopro_status lopro_vq_linear_fwd(const lopro_vq_desc* desc, const void* packed, 
         p.cb_rows = d.cb_rows;
         p.cb_cols = d.cb_cols;
         p.n_cg = L.n_cg;
+        p.section = tc <= 8 ? 6 : kVqSectionMax;
         const cudaError_t e = tc <= 8 ? launch_vq_decode<1>(p, s) : (tc <= 16 ? launch_vq_decode<2>(p, s) : launch_vq_decode<4>(p, s));
         if (e != cudaSuccess) return LOPRO_ERR_CUDA;
     }
