@@ -357,21 +357,17 @@ __device__ __forceinline__ void select_prologue_sibling(const NoPrologueSiblings
 __device__ __forceinline__ void select_prologue_sibling(const PrologueSiblings& sibs, const int32_t*& perm, const __half*& B,
                                                         unsigned char*& act_image, __half*& t, const __nv_bfloat16*& x,
                                                         int& T) {
-#pragma unroll
-    for (int i = 0; i < kMaxSiblings - 1; ++i)
-        if ((int)blockIdx.z == i + 1) {
-            perm = sibs.perm[i];
-            B = sibs.B[i];
-            act_image = sibs.act[i];
-            t = sibs.t[i];
-        }
+    // (a __grid_constant__ parameter: one constant-bank load per field at a computed index)
+    const int z = (int)blockIdx.z;
+    if (z > 0) {
+        perm = sibs.perm[z - 1];
+        B = sibs.B[z - 1];
+        act_image = sibs.act[z - 1];
+        t = sibs.t[z - 1];
+    }
     if (sibs.own_rows) {
-#pragma unroll
-        for (int i = 0; i < kMaxSiblings; ++i)
-            if ((int)blockIdx.z == i) {
-                x = sibs.x_of[i];
-                T = sibs.T_of[i];
-            }
+        x = sibs.x_of[z];
+        T = sibs.T_of[z];
     }
 }
 
@@ -380,7 +376,7 @@ __global__ void __launch_bounds__(256)
 prologue_kernel(const __nv_bfloat16* __restrict__ x0, int64_t ldx, const int32_t* __restrict__ perm0,
                 const __half* __restrict__ B0, unsigned char* __restrict__ act_image0, __half* __restrict__ t0,
                 int* __restrict__ status, int n, int b_i, int b_h, float inv_sqrt_bh, int r_pad, int t_pad, int T_grid,
-                int tpr, const ImageOut img, const SIBS sibs, const Lr8Args lr8) {
+                int tpr, const ImageOut img, const __grid_constant__ SIBS sibs, const Lr8Args lr8) {
     // sibling layers (grid z): the same x (or each its own rows), each layer its own permutation, B and outputs
     const int32_t* perm = perm0;
     const __half* B = B0;

@@ -74,28 +74,29 @@ struct NoSiblings {};
 __device__ __forceinline__ int select_sibling(StreamParams&, const NoSiblings&) { return (int)blockIdx.x; }
 
 // The layer a CTA works on: patches the per-layer fields of the parameters, returns the CTA's index within the layer.
+// (The table is a __grid_constant__ parameter: its arrays are read from the constant bank with a computed index,
+// one load per field, instead of a chain of selects over every entry.)
 __device__ __forceinline__ int select_sibling(StreamParams& p, const StreamSiblings& sibs) {
-    int bx = (int)blockIdx.x;
+    int idx = -1;
 #pragma unroll
-    for (int i = kMaxSiblings - 2; i >= 0; --i)
-        if (i < sibs.n && (int)blockIdx.x >= sibs.cta0[i] && bx == (int)blockIdx.x) {
-            bx = (int)blockIdx.x - sibs.cta0[i];
-            p.codes = sibs.codes[i];
-            p.sz = sibs.sz[i];
-            p.A = sibs.A[i];
-            p.act = sibs.act[i];
-            p.t = sibs.t[i];
-            p.y = sibs.y[i];
-            p.ldy = sibs.ldy[i];
-            p.m = sibs.m[i];
-            p.T = sibs.T[i];
-        }
-    return bx;
+    for (int i = 0; i < kMaxSiblings - 1; ++i)
+        if (i < sibs.n && (int)blockIdx.x >= sibs.cta0[i]) idx = i;
+    if (idx < 0) return (int)blockIdx.x;
+    p.codes = sibs.codes[idx];
+    p.sz = sibs.sz[idx];
+    p.A = sibs.A[idx];
+    p.act = sibs.act[idx];
+    p.t = sibs.t[idx];
+    p.y = sibs.y[idx];
+    p.ldy = sibs.ldy[idx];
+    p.m = sibs.m[idx];
+    p.T = sibs.T[idx];
+    return (int)blockIdx.x - sibs.cta0[idx];
 }
 
 template <int BITS, int NT, int RT, typename SIBS>
 __global__ void __launch_bounds__(kThreads, 1)
-stream_kernel(const StreamParams p_in, const SIBS sibs) {
+stream_kernel(const StreamParams p_in, const __grid_constant__ SIBS sibs) {
     StreamParams p = p_in;
     const int bx = select_sibling(p, sibs);
     extern __shared__ __align__(128) unsigned char smem[];
@@ -360,7 +361,7 @@ constexpr int kRedStep = 8 * kRedTok + 8;   // floats between steps
 
 template <int BITS, typename SIBS>
 __global__ void __launch_bounds__(kWideThreads, 1)
-stream_wide_kernel(const StreamParams p_in, const SIBS sibs) {
+stream_wide_kernel(const StreamParams p_in, const __grid_constant__ SIBS sibs) {
     StreamParams p = p_in;
     const int bx = select_sibling(p, sibs);
     extern __shared__ __align__(128) unsigned char smem[];

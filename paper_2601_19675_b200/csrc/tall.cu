@@ -85,22 +85,22 @@ __device__ __forceinline__ int2 select_sibling(TallParams&, const NoTallSiblings
 // The layer a CTA works on: patches the per-layer fields, returns the CTA's index among the layer's CTAs and
 // their number.
 __device__ __forceinline__ int2 select_sibling(TallParams& p, const TallSiblings& sibs) {
-    int first = 0, end = sibs.n > 0 ? sibs.cta0[0] : (int)gridDim.x;
+    int idx = -1;
 #pragma unroll
     for (int i = 0; i < kMaxSiblings - 1; ++i)
-        if (i < sibs.n && (int)blockIdx.x >= sibs.cta0[i]) {
-            first = sibs.cta0[i];
-            end = i + 1 < sibs.n ? sibs.cta0[i + 1] : (int)gridDim.x;
-            p.codes = sibs.codes[i];
-            p.sz = sibs.sz[i];
-            p.A = sibs.A[i];
-            p.act = sibs.act[i];
-            p.t = sibs.t[i];
-            p.y = sibs.y[i];
-            p.ldy = sibs.ldy[i];
-            p.m = sibs.m[i];
-            p.T = sibs.T[i];
-        }
+        if (i < sibs.n && (int)blockIdx.x >= sibs.cta0[i]) idx = i;
+    if (idx < 0) return make_int2((int)blockIdx.x, sibs.n > 0 ? sibs.cta0[0] : (int)gridDim.x);
+    // (a __grid_constant__ parameter: one constant-bank load per field at a computed index)
+    const int first = sibs.cta0[idx], end = idx + 1 < sibs.n ? sibs.cta0[idx + 1] : (int)gridDim.x;
+    p.codes = sibs.codes[idx];
+    p.sz = sibs.sz[idx];
+    p.A = sibs.A[idx];
+    p.act = sibs.act[idx];
+    p.t = sibs.t[idx];
+    p.y = sibs.y[idx];
+    p.ldy = sibs.ldy[idx];
+    p.m = sibs.m[idx];
+    p.T = sibs.T[idx];
     return make_int2((int)blockIdx.x - first, end - first);
 }
 
@@ -191,7 +191,7 @@ __device__ __forceinline__ void consume_stage(const unsigned char* stage, uint32
 
 template <int BITS, int NT, typename SIBS>
 __global__ void __launch_bounds__(kThreads, 1)
-tall_kernel(const TallParams p_in, const SIBS sibs) {
+tall_kernel(const TallParams p_in, const __grid_constant__ SIBS sibs) {
     TallParams p = p_in;
     const int2 cta = select_sibling(p, sibs);  // x: index among the layer's CTAs, y: their number
     extern __shared__ __align__(128) unsigned char smem[];
