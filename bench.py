@@ -829,6 +829,45 @@ def measure_vq(dev, peaks, reps=20):
     return out
 
 
+def measure_rotate(dev, peaks, reps=5):
+    """The activation-side transform alone (permutation gather + partial block rotation, lopro_rotate) on prefill batches:
+    read x once, write the rotated rows once.  Distinct inputs per launch (more than L2 in total)."""
+    import torch
+    from paper_2601_19675_b200 import lopro, synth
+    out = {}
+    for (n, T, b) in ((4096, 2048, 128), (8192, 4096, 256)):
+        d = lopro.make_desc(n, 256, 4, 128, b, b, 0, lopro.LAYOUT_FRAGMENT)
+        perm = torch.from_numpy(synth.permutation(n, seed=1)).to(dev)
+        k = max(8, int(300e6 / (T * n * 2)))
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(99)
+        xs = [torch.randn((T, n), device=dev, generator=gen).to(torch.bfloat16) for _ in range(k)]
+        outs = [torch.empty((T, n), dtype=torch.bfloat16, device=dev) for _ in range(min(k, 8))]
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            for i, x in enumerate(xs):
+                lopro.rotate(d, perm, x, out=outs[i % len(outs)])
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for i, x in enumerate(xs):
+                    lopro.rotate(d, perm, x, out=outs[i % len(outs)])
+            graph.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(reps):
+                graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (reps * k)
+        nbytes = 2 * T * n * 2 + n * 4
+        out[f"rotate_{T}x{n}_b{b}"] = dict(us=us, algorithmic_bytes=nbytes, achieved_gbs=nbytes / (us * 1e-6) / 1e9,
+                                           frac_of_measured_hbm=nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"])
+        del xs, outs
+        torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -874,7 +913,7 @@ def main():
 
     if args.offline:
         if rank == 0:
-            print(json.dumps(dict(offline=measure_offline(dev, measured_peaks()), experts=measure_experts(dev, measured_peaks()), vq=measure_vq(dev, measured_peaks()),
+            print(json.dumps(dict(offline=measure_offline(dev, measured_peaks()), experts=measure_experts(dev, measured_peaks()), vq=measure_vq(dev, measured_peaks()), rotate=measure_rotate(dev, measured_peaks()),
                                   n_gpus=1, data="synthetic", dtype="f32")))
         if world > 1:
             dist.destroy_process_group()
@@ -906,6 +945,7 @@ def main():
             line["offline"] = measure_offline(dev, measured_peaks())
             line["experts"] = measure_experts(dev, measured_peaks())
             line["vq"] = measure_vq(dev, measured_peaks())
+            line["rotate"] = measure_rotate(dev, measured_peaks())
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
