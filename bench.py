@@ -87,10 +87,11 @@ def time_oracle_stack(T, budget_s):
     return dict(value=T / total, cores=cores, sample="oracle.forward_exact (fp64 numpy) on sampled rows of the three "
                 "linear shapes (" + "; ".join(desc) + f"), {T} tokens, scaled linearly to 32 layers x 7 linears")
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
-# capture summarised in profiles/; valid for the kernel as committed with that summary, null otherwise.
-NCU_TRAFFIC = {("cfg2_T8", "stream_wide_kernel"): 9295872, ("cfg2_T32", "stream_kernel"): 9488896,
-               ("cfg4_T16", "tall_kernel"): 83944448, ("cfg3_T2048", "prefill_kernel"): 53353984}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from ncu captures of
+# the kernels as committed (profiles/: the commands; counters re-read after the last change of each kernel, as ncu
+# prints them, i.e. to 10 kB); null for workloads without a capture.
+NCU_TRAFFIC = {("cfg2_T8", "stream_wide_kernel"): 9290000, ("cfg2_T32", "stream_kernel"): 9490000,
+               ("cfg4_T16", "tall_kernel"): 82610000, ("cfg3_T2048", "prefill_kernel"): 55460000}
 METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
 
