@@ -120,7 +120,8 @@ enum {
     LOPRO_OPT_NO_TALL = 1,       /* 1: never the persistent streaming kernel for layers with many rows         */
     LOPRO_OPT_NO_CHUNKS = 2,     /* 1: token counts above 32 always take the tensor-core (prefill) kernel      */
     LOPRO_OPT_NO_TCGEN05 = 3,    /* 1: never the tcgen05 prefill kernel (general register-ring product)        */
-    LOPRO_OPT_PREFILL_PAIRS = 4, /* >= 0: number of two-block row tiles of the prefill grid; -1: chosen by it  */
+    LOPRO_OPT_PREFILL_PAIRS = 4, /* >= 0: number of two-block row tiles of the prefill grid (of 512-token chunks
+                                     where two CTAs share a tile); -1: chosen by the library                   */
     LOPRO_OPT_ONE_KERNEL_SET = 5, /* 1: single-layer forwards launch the same kernel variants as grouped ones
                                       (lopro_linear_fwd_group / _experts), which carry a table of sibling layers in
                                       their parameters.  By default a single-layer forward launches variants without
@@ -128,7 +129,8 @@ enum {
                                       alternates single and grouped forwards -- a decoder stack -- then alternates
                                       between two copies of every kernel, which costs more than the table does
                                       (measured: 4 % of a 224-layer decode step).  Such callers set this switch. */
-    LOPRO_OPT_COUNT = 6
+    LOPRO_OPT_NO_CTA_PAIRS = 6,  /* 1: the prefill kernel never pairs two CTAs on a tile (tcgen05 cta_group::2)   */
+    LOPRO_OPT_COUNT = 7
 };
 /* Sets one switch for the whole process (not thread-safe against forwards running on other host threads).
  * Returns LOPRO_ERR_INVALID_ARG for an unknown option. */

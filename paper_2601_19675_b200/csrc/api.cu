@@ -123,7 +123,7 @@ void read_options_once() {
     if (__atomic_compare_exchange_n(&g_options_ready, &expected, 1, false, __ATOMIC_ACQ_REL, __ATOMIC_ACQUIRE)) {
         static const char* const names[LOPRO_OPT_COUNT] = {"LOPRO_NO_WIDE", "LOPRO_NO_TALL", "LOPRO_NO_CHUNKS",
                                                            "LOPRO_NO_TCGEN05", "LOPRO_PREFILL_PAIRS",
-                                                           "LOPRO_ONE_KERNEL_SET"};
+                                                           "LOPRO_ONE_KERNEL_SET", "LOPRO_NO_CTA_PAIRS"};
         for (int i = 0; i < LOPRO_OPT_COUNT; ++i) {
             const char* e = getenv(names[i]);
             g_options[i] = e ? atoi(e) : (i == LOPRO_OPT_PREFILL_PAIRS ? -1 : 0);

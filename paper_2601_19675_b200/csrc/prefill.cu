@@ -329,6 +329,313 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// The same GEMM with the two CTAs of a cluster on one tile (tcgen05 cta_group::2): 256 weight rows (128 per CTA)
+// x 512 or 256 tokens (two accumulators or one, N = 256 each) x 64 columns of K per stage.  Every dequantized weight
+// tile now meets 512 tokens instead of 256 -- half the conversion work per multiply-add -- while each CTA still
+// streams the activations of only 256 tokens per stage (its half of each accumulator's B operand).
+//   * both CTAs: 16 dequant warps (two per 16-row tile, taking turns by pairs of stages), a loader thread (its own
+//     halves of the activation tiles; its own 128 rows of A in the low-rank stages), 4 epilogue warps (own 128 rows);
+//   * the pair's first CTA alone: the MMA issuers, one thread per accumulator.  All "full" barriers are the first
+//     CTA's (the second CTA's warps arrive on them through the cluster's shared-memory window, its TMA copies count
+//     their bytes there); the "empty" and "accumulator ready" barriers exist in both CTAs and take the commits of
+//     the first CTA's issuers by multicast.
+// A wait that runs out stops all further waits of both CTAs; both still reach the final cluster barrier, free the
+// tensor memory and return.
+constexpr int kPairABytes = kABlock;                 // 16 KB: 128 rows of one stage
+constexpr int kPairBHalf = 128 * 128;                // 16 KB: this CTA's 128 tokens of one accumulator's stage
+constexpr int kPairBBytes = 2 * kPairBHalf;          // 32 KB: both accumulators
+constexpr int kPairAStages = 4;
+constexpr int kPairBStages = 5;
+constexpr int kPairSmemBytes = kPairAStages * kPairABytes + kPairBStages * kPairBBytes + 1024;
+constexpr int kPairMinT = 512;           // smaller batches keep one CTA per tile (finer tiles fill the machine better)
+constexpr double kHalfTileCost = 0.6;  // duration of a 256-token tile relative to a 512-token tile (scheduling estimate)
+
+struct PairParams {
+    const uint32_t* codes;
+    const uint32_t* sz;
+    int* status;
+    void* y;
+    int64_t ldy;
+    int out_f32;
+    int y_vec;
+    int m, n, T;
+    int nsteps, gshift, ng, r_pad;
+    int row_tiles;    // tiles of 256 rows
+    int full_units;   // token chunks of 512 (two accumulators), listed first in the grid
+    int half_units;   // token chunks of 256 that follow them
+    int lr_stages;
+};
+
+template <int BITS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a,
+                    const __grid_constant__ CUtensorMap map_t) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * kPairAStages + 2 * kPairBStages + 1];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_timeout;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = cluster_cta_rank();  // 0: the CTA that issues the MMAs
+    const int tile = (int)(blockIdx.x >> 1);
+    const int n_full = p.row_tiles * p.full_units;
+    const bool is_full = tile < n_full;
+    const int n_acc = is_full ? 2 : 1;
+    const int rest = tile - n_full;
+    const int tile_x = (is_full ? tile : rest) % p.row_tiles;
+    const int tile_y = (is_full ? tile : rest) / p.row_tiles;
+    const int row_base = tile_x * 2 * kTileM + (int)rank * kTileM;  // this CTA's 128 rows
+    const int tok_base = is_full ? tile_y * 512 : p.full_units * 512 + tile_y * 256;
+    const int total = p.nsteps + p.lr_stages;
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - raw);
+    const uint32_t b_ring = base + kPairAStages * kPairABytes;
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_a = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto empty_a = [&](int s) { return bar0 + 8u * (uint32_t)(kPairAStages + s); };
+    auto full_b = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kPairAStages + s); };
+    auto empty_b = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kPairAStages + kPairBStages + s); };
+    const uint32_t acc_ready = bar0 + 8u * (uint32_t)(2 * kPairAStages + 2 * kPairBStages);
+    const uint32_t peer_timeout = map_to_cta(smem_u32(&s_timeout), rank ^ 1u);
+    auto time_out = [&]() {
+        s_timeout = 1;
+        st_cluster_u32(peer_timeout, 1u);
+        atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
+    };
+    auto timed_out = [&]() { return *reinterpret_cast<volatile int*>(&s_timeout) != 0; };
+    auto warp_wait = [&](uint32_t bar, uint32_t parity) {
+        if (lane == 0 && !timed_out() && !mbar_wait_cluster(bar, parity, kPrefillSpin)) time_out();
+        __syncwarp();
+    };
+    const uint32_t tmem_cols = n_acc == 2 ? 512u : 256u;
+
+    if (tid == 0) {
+        for (int s = 0; s < kPairAStages; ++s) {
+            mbar_init(full_a(s), kDequantWarps + 1);  // eight dequant warps of each CTA, and the first CTA's loader
+            mbar_init(empty_a(s), n_acc);
+        }
+        for (int s = 0; s < kPairBStages; ++s) {
+            mbar_init(full_b(s), 1);
+            mbar_init(empty_b(s), n_acc);
+        }
+        mbar_init(acc_ready, n_acc);
+        s_timeout = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kDequantWarps + 1) tmem_alloc_pair(smem_u32(&s_tmem_base), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the other CTA's barriers are initialised before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+
+    if (warp < kDequantWarps) {
+        // ---------------- dequant warps: warps w and w + 8 share tile w; group g = w >> 3 converts the stages
+        // 4 v + 2 g and 4 v + 2 g + 1 of visit v ----------------
+        static_assert(kPairAStages == 4, "the visit schedule assumes four weight slots");
+        const int gq = lane >> 2, tg = lane & 3;
+        const int g = warp >> 3;
+        const int rt = row_base / 16 + (warp & 7);
+        const bool valid = rt * 16 < p.m;
+        uint32_t wbuf[2][2][BITS];
+        uint32_t szbuf[2][2][2];
+        const uint32_t* wbase = p.codes + ((size_t)rt * p.nsteps * 32 + lane) * BITS;
+        const uint32_t* szbase = p.sz + (size_t)rt * p.ng * 16 + gq;
+        auto load_visit = [&](int buf, int v) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int s = 4 * v + 2 * g + j;
+                if (valid && s < p.nsteps) {
+#pragma unroll
+                    for (int q = 0; q < BITS; ++q) wbuf[buf][j][q] = __ldg(wbase + (size_t)s * 32 * BITS + q);
+                    const uint32_t* z = szbase + (size_t)(s >> p.gshift) * 16;
+                    szbuf[buf][j][0] = __ldg(z);
+                    szbuf[buf][j][1] = __ldg(z + 8);
+                }
+            }
+        };
+        load_visit(0, 0);
+        load_visit(1, 1);
+        uint32_t off[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) off[c] = (uint32_t)(((warp & 7) * 16 + gq) * 128 + ((c ^ gq) << 4) + tg * 4);
+        auto convert = [&](const uint32_t (&w)[BITS], uint32_t sz_lo, uint32_t sz_hi, unsigned char* a_tile) {
+            uint32_t a[16];
+            expand_codes<BITS>(a, w);
+            const float2 f_lo = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
+            const float2 f_hi = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
+            const float sc[2] = {f_lo.x, f_hi.x};
+            const float zs[2] = {128.0f + f_lo.y, 128.0f + f_hi.y};  // exact in fp32
+#pragma unroll
+            for (int pi = 0; pi < 16; ++pi) {
+                const int j = pi >> 2, rho = pi & 3, hi8 = rho & 1;
+                const uint32_t av = a[pi];
+                const float lo_f = __uint_as_float(av << 16), hi_f = __uint_as_float(av & 0xFFFF0000u);
+                // (128 + c) - (128 + z) is exact, so s (c - z) is rounded once to fp32, once to bf16
+                const __nv_bfloat162 wv = __floats2bfloat162_rn((lo_f - zs[hi8]) * sc[hi8], (hi_f - zs[hi8]) * sc[hi8]);
+                *reinterpret_cast<__nv_bfloat162*>(a_tile + off[2 * j + (rho >> 1)] + hi8 * 1024) = wv;
+            }
+        };
+        const uint32_t full_a0 = map_to_cta(full_a(0), 0u);  // the first CTA's barriers, 8 bytes apart
+        const int n_visits = total > 2 * g ? (total - 2 * g + 3) / 4 : 0;
+        for (int v0 = 0; v0 < n_visits; v0 += 2) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int v = v0 + u;
+                if (v < n_visits) {
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const int s = 4 * v + 2 * g + j;
+                        if (s < total) {
+                            const int slot = s & 3, use = s >> 2;
+                            if (use >= 1) warp_wait(empty_a(slot), (uint32_t)(use - 1) & 1u);
+                            if (valid && s < p.nsteps) convert(wbuf[u][j], szbuf[u][j][0], szbuf[u][j][1], base_ptr + slot * kPairABytes);
+                        }
+                    }
+                    load_visit(u, v + 2);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int s0 = 4 * v + 2 * g;
+                        mbar_arrive_cluster(full_a0 + 8u * (uint32_t)(s0 & 3));
+                        if (s0 + 1 < total) mbar_arrive_cluster(full_a0 + 8u * (uint32_t)((s0 + 1) & 3));
+                    }
+                }
+            }
+        }
+    } else if (warp == kDequantWarps) {
+        // ---------------- loader: this CTA's halves of the activation tiles; its rows of A in the low-rank stages ----------------
+        if (lane == 0) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            const uint32_t full_a0 = map_to_cta(full_a(0), 0u), full_b0 = map_to_cta(full_b(0), 0u);
+            const uint32_t b_bytes = (uint32_t)(2 * n_acc * kPairBHalf);  // both CTAs' copies of a stage
+            int sa = 0, sb = 0;
+            uint32_t pa = 1, pb = 1;  // parity of the previous use's "empty" phase
+            for (int s = 0; s < total; ++s) {
+                if (s >= kPairAStages && !timed_out() && !mbar_wait_cluster(empty_a(sa), pa, kPrefillSpin)) time_out();
+                if (s >= kPairBStages && !timed_out() && !mbar_wait_cluster(empty_b(sb), pb, kPrefillSpin)) time_out();
+                const uint32_t a_tile = base + sa * kPairABytes, b_tile = b_ring + sb * kPairBBytes;
+                const uint32_t fb = full_b0 + 8u * (uint32_t)sb, fa = full_a0 + 8u * (uint32_t)sa;
+                if (rank == 0) mbar_expect_tx(full_b(sb), b_bytes);
+                const CUtensorMap* bmap = s < p.nsteps ? &map_x : &map_t;
+                const int kcol = (s < p.nsteps ? s : s - p.nsteps) * kStageK;
+                for (int acc = 0; acc < n_acc; ++acc)
+                    tma_load_2d_pair(b_tile + acc * kPairBHalf, bmap, kcol, tok_base + acc * 256 + (int)rank * 128, fb);
+                if (s < p.nsteps) {
+                    if (rank == 0) mbar_arrive(full_a(sa));
+                } else {
+                    if (rank == 0) mbar_expect_tx(full_a(sa), (uint32_t)(2 * kPairABytes));
+                    tma_load_2d_pair(a_tile, &map_a, kcol, row_base, fa);
+                }
+                if (++sa == kPairAStages) {
+                    sa = 0;
+                    pa ^= 1u;
+                }
+                if (++sb == kPairBStages) {
+                    sb = 0;
+                    pb ^= 1u;
+                }
+            }
+        }
+    } else if ((warp == kDequantWarps + 1 || warp == kDequantWarps + 2) && rank == 0) {
+        // ---------------- MMA issuers (first CTA): one thread per accumulator ----------------
+        const int acc = warp - (kDequantWarps + 1);
+        if (lane == 0 && acc < n_acc) {
+            const uint32_t idesc_w = make_idesc_pair(256, 1u), idesc_lr = make_idesc_pair(256, 0u);
+            const uint32_t d = tmem + (uint32_t)(acc * 256);
+            int sa = 0, sb = 0;
+            uint32_t pa = 0, pb = 0;
+            for (int s = 0; s < total; ++s) {
+                if (!timed_out() && !(mbar_wait_cluster(full_a(sa), pa, kPrefillSpin) && mbar_wait_cluster(full_b(sb), pb, kPrefillSpin)))
+                    time_out();
+                tc_fence_after();
+                const uint64_t da = make_desc_sw128(base + sa * kPairABytes);
+                const uint64_t db = make_desc_sw128(b_ring + sb * kPairBBytes + acc * kPairBHalf);
+                const bool lowrank = s >= p.nsteps;
+                const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
+                const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
+                for (int k = 0; k < ksub; ++k)
+                    umma_f16_pair(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (s > 0 || k > 0) ? 1u : 0u);
+                umma_commit_pair(empty_a(sa));
+                umma_commit_pair(empty_b(sb));
+                if (++sa == kPairAStages) {
+                    sa = 0;
+                    pa ^= 1u;
+                }
+                if (++sb == kPairBStages) {
+                    sb = 0;
+                    pb ^= 1u;
+                }
+            }
+            umma_commit_pair(acc_ready);
+        }
+    }
+
+    if (warp >= kDequantWarps) {
+        // ---------------- epilogue: this CTA's 128 rows of every accumulator ----------------
+        __syncwarp();
+        if (lane == 0 && !timed_out() && !mbar_wait_cluster(acc_ready, 0, kPrefillSpin)) time_out();
+        __syncwarp();
+        tc_fence_after();
+        const int lane_base = (warp & 3) * 32;
+        const int row = row_base + lane_base + lane;
+        for (int acc = 0; acc < n_acc; ++acc) {
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                if (tok_base + acc * 256 + c0 >= p.T) break;  // uniform over the warp
+                uint32_t v[32];
+                const uint32_t taddr = tmem + ((uint32_t)lane_base << 16) + (uint32_t)(acc * 256 + c0);
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                      "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                      "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                      "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                    : "r"(taddr)
+                    : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const int tok0 = tok_base + acc * 256 + c0;
+                if (p.y_vec) {
+                    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(base_ptr + (warp - kDequantWarps) * 2048);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) stg[i * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int piece = q * 32 + lane, ti = piece >> 2, r8 = (piece & 3) * 8;
+                        const int tok = tok0 + ti, prow = row_base + lane_base + r8;
+                        if (tok < p.T && prow < p.m)
+                            *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.y) + (size_t)tok * p.ldy + prow) =
+                                *reinterpret_cast<const uint4*>(stg + ti * 32 + r8);
+                    }
+                } else if (row < p.m) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int tok = tok0 + i;
+                        if (tok < p.T) {
+                            const size_t o = (size_t)tok * p.ldy + row;
+                            if (p.out_f32) reinterpret_cast<float*>(p.y)[o] = __uint_as_float(v[i]);
+                            else reinterpret_cast<__nv_bfloat16*>(p.y)[o] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                        }
+                    }
+                }
+            }
+        }
+    }
+    // neither CTA leaves, or frees tensor memory, while the other may still read its shared memory, arrive on its
+    // barriers or read the accumulators
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == kDequantWarps + 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem, tmem_cols);
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -379,6 +686,83 @@ cudaError_t launch_prefill_bits(const PrefillParams& p, const CUtensorMap& mx, c
     return cudaLaunchKernelEx(&cfg, prefill_kernel<BITS>, p, mx, ma, mt);
 }
 
+// CTA pairs that can be resident at once (each CTA fills a multiprocessor); cached per device, 0 if the query fails
+template <int BITS>
+int pair_slots() {
+    static int cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    int v = __atomic_load_n(&cached[dev & 63], __ATOMIC_ACQUIRE);
+    if (v != 0) return v > 0 ? v : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * 1024);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kPairSmemBytes;
+    int n = 0;
+    const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, prefill_pair_kernel<BITS>, &cfg);
+    v = (e == cudaSuccess && n > 0) ? n : -1;
+    if (e != cudaSuccess) (void)cudaGetLastError();
+    __atomic_store_n(&cached[dev & 63], v, __ATOMIC_RELEASE);
+    return v > 0 ? v : 0;
+}
+
+template <int BITS>
+cudaError_t launch_pair_bits(PairParams p, const CUtensorMap& mx, const CUtensorMap& ma, const CUtensorMap& mt, int chunks256,
+                             cudaStream_t s) {
+    static unsigned long long attr_done = 0;
+    cudaError_t e = ensure_dynamic_smem(prefill_pair_kernel<BITS>, kPairSmemBytes, &attr_done);
+    if (e != cudaSuccess) return e;
+    // Token chunks: full_units of 512 tokens first, then half_units of 256; the mix that minimises the makespan of a
+    // greedy schedule over the resident pairs (the cheaper tiles fill the last wave).
+    int slots = pair_slots<BITS>();
+    if (slots <= 0) slots = sm_count() / 2;
+    if (slots > 256) slots = 256;
+    int best_full = chunks256 / 2;
+    if ((long long)p.row_tiles * chunks256 <= 20000) {
+        double best_cost = 1e30;
+        for (int full = chunks256 / 2; full >= 0; --full) {
+            const int half = chunks256 - 2 * full;
+            double finish[256];
+            for (int i = 0; i < slots; ++i) finish[i] = 0.0;
+            auto place = [&](long long count, double dur) {
+                for (long long c = 0; c < count; ++c) {
+                    int best = 0;
+                    for (int i = 1; i < slots; ++i)
+                        if (finish[i] < finish[best]) best = i;
+                    finish[best] += dur;
+                }
+            };
+            place((long long)p.row_tiles * full, 1.0);
+            place((long long)p.row_tiles * half, kHalfTileCost);
+            double cost = 0.0;
+            for (int i = 0; i < slots; ++i) cost = finish[i] > cost ? finish[i] : cost;
+            if (cost < best_cost - 1e-9) {
+                best_cost = cost;
+                best_full = full;
+            }
+        }
+    }
+    {
+        const int forced = option(LOPRO_OPT_PREFILL_PAIRS);  // overrides the number of 512-token chunks (tuning only)
+        if (forced >= 0 && forced <= chunks256 / 2) best_full = forced;
+    }
+    p.full_units = best_full;
+    p.half_units = chunks256 - 2 * best_full;
+    const long long n_ctas = 2LL * p.row_tiles * (p.full_units + p.half_units);
+    if (n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kPairSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BITS>, p, mx, ma, mt);
+}
+
 }  // namespace
 
 bool prefill_supported(const lopro_desc& d, int T) {
@@ -407,6 +791,44 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     p.r_pad = d.rank > 0 ? L.r_pad : 0;
     p.tile_n = T <= 64 ? 64 : (T <= 128 ? 128 : 256);
     p.lr_stages = (p.r_pad + kStageK - 1) / kStageK;
+    if (T >= kPairMinT && option(LOPRO_OPT_NO_CTA_PAIRS) != 1) {
+        // large batches: two CTAs per tile (each loads boxes of 128 tokens)
+        PairParams q;
+        q.codes = p.codes;
+        q.sz = p.sz;
+        q.status = p.status;
+        q.y = y;
+        q.ldy = ldy;
+        q.out_f32 = p.out_f32;
+        q.y_vec = p.y_vec;
+        q.m = p.m;
+        q.n = p.n;
+        q.T = T;
+        q.nsteps = p.nsteps;
+        q.gshift = p.gshift;
+        q.ng = p.ng;
+        q.r_pad = p.r_pad;
+        q.lr_stages = p.lr_stages;
+        q.row_tiles = (d.d_out + 2 * kTileM - 1) / (2 * kTileM);
+        q.full_units = q.half_units = 0;
+        CUtensorMap qx, qa, qt;
+        if (!make_map(&qx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ws + W.off_xrot, (uint64_t)d.d_in, (uint64_t)T, 128u))
+            return cudaErrorInvalidValue;
+        qa = qx;
+        qt = qx;
+        if (q.r_pad > 0) {
+            if (!make_map(&qa, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, blob + L.off[LOPRO_SEC_A], (uint64_t)q.r_pad, (uint64_t)d.d_out,
+                          (uint32_t)kTileM) ||
+                !make_map(&qt, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ws + W.off_t, (uint64_t)q.r_pad, (uint64_t)T, 128u))
+                return cudaErrorInvalidValue;
+        }
+        const int chunks256 = (T + 255) / 256;
+        switch (d.bits) {
+            case 2: return launch_pair_bits<2>(q, qx, qa, qt, chunks256, s);
+            case 3: return launch_pair_bits<3>(q, qx, qa, qt, chunks256, s);
+            default: return launch_pair_bits<4>(q, qx, qa, qt, chunks256, s);
+        }
+    }
     CUtensorMap mx, ma, mt;
     if (!make_map(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ws + W.off_xrot, (uint64_t)d.d_in, (uint64_t)T, (uint32_t)p.tile_n))
         return cudaErrorInvalidValue;

@@ -152,7 +152,7 @@ def lib():
     return _lib
 
 
-OPT_NO_WIDE, OPT_NO_TALL, OPT_NO_CHUNKS, OPT_NO_TCGEN05, OPT_PREFILL_PAIRS, OPT_ONE_KERNEL_SET = range(6)
+OPT_NO_WIDE, OPT_NO_TALL, OPT_NO_CHUNKS, OPT_NO_TCGEN05, OPT_PREFILL_PAIRS, OPT_ONE_KERNEL_SET, OPT_NO_CTA_PAIRS = range(7)
 
 
 def configure(option, value):

@@ -162,6 +162,35 @@ def test_shapes_in_the_parameter_domain(n, m, bits, g, b_i, b_h, r, T):
     _check_forward(layer, d, synth.activations(T, n, seed=7, outlier_frac=0.01))
 
 
+@pytest.mark.parametrize("n,m,bits,g,r,T", [
+    (512, 320, 3, 64, 17, 512),      # one 512-token chunk; second row tile ragged (its second CTA has no rows at all)
+    (1024, 256, 4, 128, 64, 600),    # 512 + 88 tokens
+    (768, 144, 2, 64, 0, 777),       # no low-rank stages; 144 rows in a tile of 256
+    (1024, 512, 4, 64, 128, 1030),   # two low-rank stages; last chunk holds 6 tokens
+    (2048, 384, 3, 128, 40, 512),    # rank padded inside a stage
+])
+def test_large_batches_pair_two_ctas_on_a_tile(n, m, bits, g, r, T):
+    """512 tokens and more: the prefill kernel puts the two CTAs of a cluster on one tile of 256 rows x 512 or 256
+    tokens.  Every mix of 512- and 256-token chunks is run, and the kernel with one CTA per tile on the same inputs."""
+    layer = random_layer_np(n, m, bits, g, r, seed=n + m + T)
+    d = lopro.make_desc(n, m, bits, g, 128, identity_cols=128, rank=r)
+    x_bits = synth.activations(T, n, seed=T, outlier_frac=0.01)
+    assert lopro.linear_fwd_path(d, T)[0] == lopro.PATH_PREFILL
+    chunks = (T + 255) // 256
+    for full in [-1] + list(range(chunks // 2 + 1)):
+        with lopro.configured(lopro.OPT_PREFILL_PAIRS, full):
+            _check_forward_once(layer, d, x_bits, None, GATE_A, GATE_B)
+    blob = _pack(layer, d)
+    x = bf16_bits_to_device(x_bits)
+    y_pair = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
+    with lopro.configured(lopro.OPT_NO_CTA_PAIRS, 1):
+        _check_forward_once(layer, d, x_bits, None, GATE_A, GATE_B)
+        y_single = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
+    # the same products summed in the same K order by both kernels
+    scale = y_single.abs().max().item()
+    assert (y_pair - y_single).abs().max().item() <= 1e-5 * scale
+
+
 @pytest.mark.parametrize("bits,g", [(4, 128), (3, 64), (2, 64)])
 @pytest.mark.parametrize("T", [1, 2, 5, 8])
 @pytest.mark.parametrize("n,m,r,b", [(2048, 144, 17, 128), (4096, 528, 32, 256), (4096, 64, 0, 64)])
