@@ -99,8 +99,14 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
         atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
     };
     // one lane polls, the warp follows (bar.warp.sync orders the other lanes' accesses after the wait)
+    // A wait on a phase that is already complete costs one shared-memory round trip; the time-out flag (another
+    // round trip) is read only when the first poll fails.
+    auto wait_phase = [&](uint32_t bar, uint32_t parity) {
+        if (mbar_try_wait(bar, parity)) return;
+        if (!*reinterpret_cast<volatile int*>(&s_timeout) && !mbar_wait(bar, parity, kPrefillSpin)) time_out();
+    };
     auto warp_wait = [&](uint32_t bar, uint32_t parity) {
-        if (lane == 0 && !s_timeout && !mbar_wait(bar, parity, kPrefillSpin)) time_out();
+        if (lane == 0) wait_phase(bar, parity);
         __syncwarp();
     };
     const uint32_t tmem_cols = n_acc == 2 ? 512u : 256u;
@@ -196,7 +202,6 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                                 convert(wbuf[u][j], szbuf[u][j][0], szbuf[u][j][1], blk_ptr + slot * kABytes);
                         }
                     }
-                    load_visit(u, v + 2);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
                     __syncwarp();
                     if (lane == 0) {
@@ -204,6 +209,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                         mbar_arrive(full_a(s0 & 3));
                         if (s0 + 1 < total) mbar_arrive(full_a((s0 + 1) & 3));
                     }
+                    // after the fence and the releasing arrivals, which would wait for these loads to land
+                    load_visit(u, v + 2);
                 }
             }
         }
@@ -216,8 +223,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
             const uint32_t b_bytes = (uint32_t)(p.tile_n * 128);
             for (int s = 0; s < total; ++s) {
                 const int sa = s % kAStages, sb = s % kBStages;
-                if (s >= kAStages && !s_timeout && !mbar_wait(empty_a(sa), (uint32_t)((s / kAStages) - 1) & 1u, kPrefillSpin)) time_out();
-                if (s >= kBStages && !s_timeout && !mbar_wait(empty_b(sb), (uint32_t)((s / kBStages) - 1) & 1u, kPrefillSpin)) time_out();
+                if (s >= kAStages) wait_phase(empty_a(sa), (uint32_t)((s / kAStages) - 1) & 1u);
+                if (s >= kBStages) wait_phase(empty_b(sb), (uint32_t)((s / kBStages) - 1) & 1u);
                 const uint32_t a_tile = base + sa * kABytes, b_tile = b_ring + sb * kBBytes;
                 mbar_expect_tx(full_b(sb), b_bytes);
                 if (s < p.nsteps) {
@@ -242,20 +249,19 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
         if (lane == 0 && acc < n_acc) {
             const uint32_t idesc_w = make_idesc(p.tile_n, 1u), idesc_lr = make_idesc(p.tile_n, 0u);
             const uint32_t d = tmem + (uint32_t)(acc * 256);
+            // The next stage's barriers are polled (without suspending) before this stage's MMAs are issued, so
+            // that the answers arrive while the MMAs queue up: every barrier operation is a shared-memory round
+            // trip behind the dequant warps' traffic, and the tensor pipe idles while this thread waits.
             int sa = 0, sb = 0;
             uint32_t pa = 0, pb = 0;
+            bool ready_a = mbar_test_wait(full_a(0), 0u), ready_b = mbar_test_wait(full_b(0), 0u);
             for (int s = 0; s < total; ++s) {
-                if (!s_timeout && !(mbar_wait(full_a(sa), pa, kPrefillSpin) && mbar_wait(full_b(sb), pb, kPrefillSpin))) time_out();
+                if (!ready_a) wait_phase(full_a(sa), pa);
+                if (!ready_b) wait_phase(full_b(sb), pb);
                 tc_fence_after();
                 const uint64_t da = make_desc_sw128(base + sa * kABytes + acc * kABlock);
                 const uint64_t db = make_desc_sw128(b_ring + sb * kBBytes);
-                const bool lowrank = s >= p.nsteps;
-                const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
-                const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
-                for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
-                    umma_f16(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (s > 0 || k > 0) ? 1u : 0u);
-                umma_commit(empty_a(sa));  // the slots may be refilled once these MMAs have read them
-                umma_commit(empty_b(sb));
+                const uint32_t commit_a = empty_a(sa), commit_b = empty_b(sb);
                 if (++sa == kAStages) {
                     sa = 0;
                     pa ^= 1u;
@@ -264,6 +270,17 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                     sb = 0;
                     pb ^= 1u;
                 }
+                if (s + 1 < total) {
+                    ready_a = mbar_test_wait(full_a(sa), pa);
+                    ready_b = mbar_test_wait(full_b(sb), pb);
+                }
+                const bool lowrank = s >= p.nsteps;
+                const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
+                const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
+                for (int k = 0; k < ksub; ++k)  // 16 columns = 32 bytes = 2 descriptor address units
+                    umma_f16(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (s > 0 || k > 0) ? 1u : 0u);
+                umma_commit(commit_a);  // the slots may be refilled once these MMAs have read them
+                umma_commit(commit_b);
             }
             umma_commit(acc_ready);
         }
@@ -272,7 +289,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
     if (warp >= kDequantWarps) {
         // ---------------- epilogue: TMEM -> registers -> y[token][row] ----------------
         __syncwarp();
-        if (lane == 0 && !mbar_wait(acc_ready, 0, kPrefillSpin)) time_out();
+        if (lane == 0) wait_phase(acc_ready, 0u);
         __syncwarp();
         tc_fence_after();
         const int lane_base = (warp & 3) * 32;  // a warp may read the 32 TMEM lanes of its quarter
@@ -345,8 +362,14 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap map_x,
 constexpr int kPairABytes = kABlock;                 // 16 KB: 128 rows of one stage
 constexpr int kPairBHalf = 128 * 128;                // 16 KB: this CTA's 128 tokens of one accumulator's stage
 constexpr int kPairBBytes = 2 * kPairBHalf;          // 32 KB: both accumulators
-constexpr int kPairAStages = 4;
-constexpr int kPairBStages = 5;
+#ifndef LOPRO_PAIR_A_STAGES
+#define LOPRO_PAIR_A_STAGES 8
+#endif
+#ifndef LOPRO_PAIR_B_STAGES
+#define LOPRO_PAIR_B_STAGES 3
+#endif
+constexpr int kPairAStages = LOPRO_PAIR_A_STAGES;  // even: a visit fills two neighbouring slots
+constexpr int kPairBStages = LOPRO_PAIR_B_STAGES;
 constexpr int kPairSmemBytes = kPairAStages * kPairABytes + kPairBStages * kPairBBytes + 1024;
 constexpr int kPairMinT = 512;           // smaller batches keep one CTA per tile (finer tiles fill the machine better)
 constexpr double kHalfTileCost = 0.6;  // duration of a 256-token tile relative to a 512-token tile (scheduling estimate)
@@ -405,8 +428,14 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
         atomicExch(p.status, (int)LOPRO_ERR_TIMEOUT);
     };
     auto timed_out = [&]() { return *reinterpret_cast<volatile int*>(&s_timeout) != 0; };
+    // A wait on a phase that is already complete costs one shared-memory round trip; the time-out flag (another
+    // round trip) is read only when the first poll fails.
+    auto wait_phase = [&](uint32_t bar, uint32_t parity) {
+        if (mbar_try_wait(bar, parity)) return;
+        if (!timed_out() && !mbar_wait(bar, parity, kPrefillSpin)) time_out();
+    };
     auto warp_wait = [&](uint32_t bar, uint32_t parity) {
-        if (lane == 0 && !timed_out() && !mbar_wait_cluster(bar, parity, kPrefillSpin)) time_out();
+        if (lane == 0) wait_phase(bar, parity);
         __syncwarp();
     };
     const uint32_t tmem_cols = n_acc == 2 ? 512u : 256u;
@@ -434,7 +463,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
     if (warp < kDequantWarps) {
         // ---------------- dequant warps: warps w and w + 8 share tile w; group g = w >> 3 converts the stages
         // 4 v + 2 g and 4 v + 2 g + 1 of visit v ----------------
-        static_assert(kPairAStages == 4, "the visit schedule assumes four weight slots");
+        static_assert(kPairAStages % 2 == 0 && kPairAStages >= 4, "a visit fills two neighbouring weight slots");
         const int gq = lane >> 2, tg = lane & 3;
         const int g = warp >> 3;
         const int rt = row_base / 16 + (warp & 7);
@@ -489,19 +518,20 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                     for (int j = 0; j < 2; ++j) {
                         const int s = 4 * v + 2 * g + j;
                         if (s < total) {
-                            const int slot = s & 3, use = s >> 2;
+                            const int slot = s % kPairAStages, use = s / kPairAStages;
                             if (use >= 1) warp_wait(empty_a(slot), (uint32_t)(use - 1) & 1u);
                             if (valid && s < p.nsteps) convert(wbuf[u][j], szbuf[u][j][0], szbuf[u][j][1], base_ptr + slot * kPairABytes);
                         }
                     }
-                    load_visit(u, v + 2);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
                     __syncwarp();
                     if (lane == 0) {
                         const int s0 = 4 * v + 2 * g;
-                        mbar_arrive_cluster(full_a0 + 8u * (uint32_t)(s0 & 3));
-                        if (s0 + 1 < total) mbar_arrive_cluster(full_a0 + 8u * (uint32_t)((s0 + 1) & 3));
+                        mbar_arrive_cluster(full_a0 + 8u * (uint32_t)(s0 % kPairAStages));
+                        if (s0 + 1 < total) mbar_arrive_cluster(full_a0 + 8u * (uint32_t)(s0 % kPairAStages + 1));
                     }
+                    // after the fence and the releasing arrivals, which would wait for these loads to land
+                    load_visit(u, v + 2);
                 }
             }
         }
@@ -514,8 +544,14 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
             int sa = 0, sb = 0;
             uint32_t pa = 1, pb = 1;  // parity of the previous use's "empty" phase
             for (int s = 0; s < total; ++s) {
-                if (s >= kPairAStages && !timed_out() && !mbar_wait_cluster(empty_a(sa), pa, kPrefillSpin)) time_out();
-                if (s >= kPairBStages && !timed_out() && !mbar_wait_cluster(empty_b(sb), pb, kPrefillSpin)) time_out();
+                // Weight stages: the first CTA's loader is one of the arrivals of full_a (so that the low-rank stages
+                // can count their A tiles there); it may arrive for this use of the slot once the previous use's
+                // phase is complete, which does not wait for the MMAs.  Low-rank stages write the slot: empty_a.
+                if (s >= kPairAStages) {
+                    if (s >= p.nsteps) wait_phase(empty_a(sa), pa);
+                    else if (rank == 0) wait_phase(full_a(sa), pa);
+                }
+                if (s >= kPairBStages) wait_phase(empty_b(sb), pb);
                 const uint32_t a_tile = base + sa * kPairABytes, b_tile = b_ring + sb * kPairBBytes;
                 const uint32_t fb = full_b0 + 8u * (uint32_t)sb, fa = full_a0 + 8u * (uint32_t)sa;
                 if (rank == 0) mbar_expect_tx(full_b(sb), b_bytes);
@@ -545,21 +581,20 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
         if (lane == 0 && acc < n_acc) {
             const uint32_t idesc_w = make_idesc_pair(256, 1u), idesc_lr = make_idesc_pair(256, 0u);
             const uint32_t d = tmem + (uint32_t)(acc * 256);
+            // The thread's time per stage bounds the kernel (the tensor pipe idles while it waits), and every
+            // barrier operation is a shared-memory round trip behind the dequant warps' traffic.  So the next
+            // stage's barriers are polled (without suspending) before this stage's MMAs are issued: the answers
+            // arrive while the MMAs queue up, and a stage whose tiles were ready by then waits for nothing.
             int sa = 0, sb = 0;
             uint32_t pa = 0, pb = 0;
+            bool ready_a = mbar_test_wait(full_a(0), 0u), ready_b = mbar_test_wait(full_b(0), 0u);
             for (int s = 0; s < total; ++s) {
-                if (!timed_out() && !(mbar_wait_cluster(full_a(sa), pa, kPrefillSpin) && mbar_wait_cluster(full_b(sb), pb, kPrefillSpin)))
-                    time_out();
+                if (!ready_a) wait_phase(full_a(sa), pa);
+                if (!ready_b) wait_phase(full_b(sb), pb);
                 tc_fence_after();
                 const uint64_t da = make_desc_sw128(base + sa * kPairABytes);
                 const uint64_t db = make_desc_sw128(b_ring + sb * kPairBBytes + acc * kPairBHalf);
-                const bool lowrank = s >= p.nsteps;
-                const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
-                const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
-                for (int k = 0; k < ksub; ++k)
-                    umma_f16_pair(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (s > 0 || k > 0) ? 1u : 0u);
-                umma_commit_pair(empty_a(sa));
-                umma_commit_pair(empty_b(sb));
+                const uint32_t commit_a = empty_a(sa), commit_b = empty_b(sb);
                 if (++sa == kPairAStages) {
                     sa = 0;
                     pa ^= 1u;
@@ -568,6 +603,17 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                     sb = 0;
                     pb ^= 1u;
                 }
+                if (s + 1 < total) {
+                    ready_a = mbar_test_wait(full_a(sa), pa);
+                    ready_b = mbar_test_wait(full_b(sb), pb);
+                }
+                const bool lowrank = s >= p.nsteps;
+                const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
+                const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
+                for (int k = 0; k < ksub; ++k)
+                    umma_f16_pair(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (s > 0 || k > 0) ? 1u : 0u);
+                umma_commit_pair(commit_a);
+                umma_commit_pair(commit_b);
             }
             umma_commit_pair(acc_ready);
         }
@@ -576,7 +622,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
     if (warp >= kDequantWarps) {
         // ---------------- epilogue: this CTA's 128 rows of every accumulator ----------------
         __syncwarp();
-        if (lane == 0 && !timed_out() && !mbar_wait_cluster(acc_ready, 0, kPrefillSpin)) time_out();
+        if (lane == 0) wait_phase(acc_ready, 0u);
         __syncwarp();
         tc_fence_after();
         const int lane_base = (warp & 3) * 32;
