@@ -370,6 +370,7 @@ constexpr int kPairBBytes = 2 * kPairBHalf;          // 32 KB: both accumulators
 #endif
 constexpr int kPairAStages = LOPRO_PAIR_A_STAGES;  // even: a visit fills two neighbouring slots
 constexpr int kPairBStages = LOPRO_PAIR_B_STAGES;
+static_assert(kPairBStages <= kPairAStages, "one 'empty' barrier per weight slot serves both rings");
 constexpr int kPairSmemBytes = kPairAStages * kPairABytes + kPairBStages * kPairBBytes + 1024;
 constexpr int kPairMinT = 512;           // smaller batches keep one CTA per tile (finer tiles fill the machine better)
 constexpr double kHalfTileCost = 0.6;  // duration of a 256-token tile relative to a 512-token tile (scheduling estimate)
@@ -395,7 +396,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a,
                     const __grid_constant__ CUtensorMap map_t) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * kPairAStages + 2 * kPairBStages + 1];
+    __shared__ __align__(8) uint64_t bars[2 * kPairAStages + kPairBStages + 1];  // full_a, empty, full_b, accumulators ready
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_timeout;
 
@@ -419,8 +420,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
     auto full_a = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto empty_a = [&](int s) { return bar0 + 8u * (uint32_t)(kPairAStages + s); };
     auto full_b = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kPairAStages + s); };
-    auto empty_b = [&](int s) { return bar0 + 8u * (uint32_t)(2 * kPairAStages + kPairBStages + s); };
-    const uint32_t acc_ready = bar0 + 8u * (uint32_t)(2 * kPairAStages + 2 * kPairBStages);
+    const uint32_t acc_ready = bar0 + 8u * (uint32_t)(2 * kPairAStages + kPairBStages);
     const uint32_t peer_timeout = map_to_cta(smem_u32(&s_timeout), rank ^ 1u);
     auto time_out = [&]() {
         s_timeout = 1;
@@ -445,10 +445,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
             mbar_init(full_a(s), kDequantWarps + 1);  // eight dequant warps of each CTA, and the first CTA's loader
             mbar_init(empty_a(s), n_acc);
         }
-        for (int s = 0; s < kPairBStages; ++s) {
-            mbar_init(full_b(s), 1);
-            mbar_init(empty_b(s), n_acc);
-        }
+        for (int s = 0; s < kPairBStages; ++s) mbar_init(full_b(s), 1);
         mbar_init(acc_ready, n_acc);
         s_timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -551,7 +548,9 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                     if (s >= p.nsteps) wait_phase(empty_a(sa), pa);
                     else if (rank == 0) wait_phase(full_a(sa), pa);
                 }
-                if (s >= kPairBStages) wait_phase(empty_b(sb), pb);
+                // the commit that frees weight slot (s - kPairBStages) % kPairAStages frees this activation slot too
+                if (s >= kPairBStages)
+                    wait_phase(empty_a((s - kPairBStages) % kPairAStages), (uint32_t)((s - kPairBStages) / kPairAStages) & 1u);
                 const uint32_t a_tile = base + sa * kPairABytes, b_tile = b_ring + sb * kPairBBytes;
                 const uint32_t fb = full_b0 + 8u * (uint32_t)sb, fa = full_a0 + 8u * (uint32_t)sa;
                 if (rank == 0) mbar_expect_tx(full_b(sb), b_bytes);
@@ -594,7 +593,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                 tc_fence_after();
                 const uint64_t da = make_desc_sw128(base + sa * kPairABytes);
                 const uint64_t db = make_desc_sw128(b_ring + sb * kPairBBytes + acc * kPairBHalf);
-                const uint32_t commit_a = empty_a(sa), commit_b = empty_b(sb);
+                const uint32_t commit_a = empty_a(sa);
                 if (++sa == kPairAStages) {
                     sa = 0;
                     pa ^= 1u;
@@ -612,8 +611,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                 const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
                 for (int k = 0; k < ksub; ++k)
                     umma_f16_pair(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (s > 0 || k > 0) ? 1u : 0u);
-                umma_commit_pair(commit_a);
-                umma_commit_pair(commit_b);
+                umma_commit_pair(commit_a);  // one commit per stage: the stage's weight and activation slots
             }
             umma_commit_pair(acc_ready);
         }
