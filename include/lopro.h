@@ -120,8 +120,9 @@ enum {
     LOPRO_OPT_NO_TALL = 1,       /* 1: never the persistent streaming kernel for layers with many rows         */
     LOPRO_OPT_NO_CHUNKS = 2,     /* 1: token counts above 32 always take the tensor-core (prefill) kernel      */
     LOPRO_OPT_NO_TCGEN05 = 3,    /* 1: never the tcgen05 prefill kernel (general register-ring product)        */
-    LOPRO_OPT_PREFILL_PAIRS = 4, /* >= 0: number of two-block row tiles of the prefill grid (of 512-token chunks
-                                     where two CTAs share a tile); -1: chosen by the library                   */
+    LOPRO_OPT_PREFILL_PAIRS = 4, /* >= 0: number of two-block row tiles of the prefill grid; where two CTAs share a
+                                     tile (512 tokens and more): number of K parts of the last wave's tiles, 0 or 1
+                                     = none, at most 4; -1: chosen by the library                              */
     LOPRO_OPT_ONE_KERNEL_SET = 5, /* 1: single-layer forwards launch the same kernel variants as grouped ones
                                       (lopro_linear_fwd_group / _experts), which carry a table of sibling layers in
                                       their parameters.  By default a single-layer forward launches variants without

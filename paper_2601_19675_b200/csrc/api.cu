@@ -74,6 +74,8 @@ lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
     off += round_up_size((size_t)t_pad * (r_pad > 0 ? r_pad : 16) * 2, 256);
     W->off_lrpart = off;
     if (T > kDecodeMaxT && d.rank > 0) off += round_up_size(lowrank_mma_scratch_bytes(d, T), 256);
+    W->off_kparts = off;
+    off += round_up_size(prefill_kparts_bytes(d, T), 256);
     // operand image of the tcgen05 small-batch kernel (row-block layout)
     W->np = T <= 16 ? 16 : 32;
     W->n_tgroups = T <= 16 ? 1 : (T + 31) / 32;
@@ -387,6 +389,10 @@ int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launch
                             : 1 + (desc->rank > 0 ? (T > kDecodeMaxT ? 2 : 1) : 0);
         path = prefill_supported(*desc, T) ? LOPRO_PATH_PREFILL : LOPRO_PATH_GENERAL;
         n = pre + 1;
+        if (path == LOPRO_PATH_PREFILL && option(LOPRO_OPT_NO_CTA_PAIRS) != 1) {
+            const PairPlan plan = pair_plan(*desc, T);
+            if (plan.use && plan.split_tiles > 0) ++n;  // the sum of the K parts of the last wave's tiles
+        }
     }
     if (launches) *launches = n;
     return path;

@@ -74,7 +74,7 @@ inline size_t round_up_size(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // activations, low-rank intermediate (fp16, general path), per-chunk partial sums of the low-rank
 // intermediate (fp32, small-batch path).
 struct WorkspaceLayout {
-    size_t off_status, off_xrot, off_s64, off_t, off_lrpart, total;
+    size_t off_status, off_xrot, off_s64, off_t, off_lrpart, off_kparts, total;
     int t_pad;  // tokens padded to a multiple of 8
     // row-block layout only: the operand image of the tcgen05 small-batch kernel (see ImageOut)
     size_t off_counters, off_ximg, off_sums, off_timg, off_partial;
@@ -216,6 +216,13 @@ cudaError_t launch_rotate_lowrank(const lopro_desc& d, const int32_t* perm, cons
                                   float* partial, __half* t, int T, cudaStream_t s);
 // Prefill forward (T > 32) on tcgen05 / TMEM, after launch_rotate and launch_lowrank_down.
 bool prefill_supported(const lopro_desc& d, int T);
+// Tiling of the prefill kernel that puts two CTAs on a tile (large batches): n_tiles tiles of 256 rows x 512 tokens, the
+// last split_tiles of them cut along K into k_parts units whose fp32 partial sums meet in the workspace.
+struct PairPlan {
+    int use, row_tiles, n_tiles, split_tiles, k_parts;
+};
+PairPlan pair_plan(const lopro_desc& d, int T);
+size_t prefill_kparts_bytes(const lopro_desc& d, int T);
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                            const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
 

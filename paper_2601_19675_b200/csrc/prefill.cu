@@ -372,8 +372,8 @@ constexpr int kPairAStages = LOPRO_PAIR_A_STAGES;  // even: a visit fills two ne
 constexpr int kPairBStages = LOPRO_PAIR_B_STAGES;
 static_assert(kPairBStages <= kPairAStages, "one 'empty' barrier per weight slot serves both rings");
 constexpr int kPairSmemBytes = kPairAStages * kPairABytes + kPairBStages * kPairBBytes + 1024;
-constexpr int kPairMinT = 512;           // smaller batches keep one CTA per tile (finer tiles fill the machine better)
-constexpr double kHalfTileCost = 0.6;  // duration of a 256-token tile relative to a 512-token tile (scheduling estimate)
+constexpr int kPairMinT = 512;   // smaller batches keep one CTA per tile (finer tiles fill the machine better)
+constexpr int kMaxKParts = 4;    // K parts of a tile of the last wave
 
 struct PairParams {
     const uint32_t* codes;
@@ -386,8 +386,9 @@ struct PairParams {
     int m, n, T;
     int nsteps, gshift, ng, r_pad;
     int row_tiles;    // tiles of 256 rows
-    int full_units;   // token chunks of 512 (two accumulators), listed first in the grid
-    int half_units;   // token chunks of 256 that follow them
+    int split_first;  // tiles from this index on are split along K into k_parts units each (the last wave)
+    int k_parts;
+    float* kparts;    // their fp32 partial sums, [unit][512 tokens][256 rows]
     int lr_stages;
 };
 
@@ -402,16 +403,21 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = cluster_cta_rank();  // 0: the CTA that issues the MMAs
-    const int tile = (int)(blockIdx.x >> 1);
-    const int n_full = p.row_tiles * p.full_units;
-    const bool is_full = tile < n_full;
-    const int n_acc = is_full ? 2 : 1;
-    const int rest = tile - n_full;
-    const int tile_x = (is_full ? tile : rest) % p.row_tiles;
-    const int tile_y = (is_full ? tile : rest) / p.row_tiles;
+    // Units in grid order: whole tiles first, then the tiles of the last wave cut along K into k_parts units, which
+    // leave fp32 partial sums for prefill_kparts_kernel (so that the last wave fills the machine too).
+    const int unit = (int)(blockIdx.x >> 1);
+    const bool whole = unit < p.split_first;
+    const int tile = whole ? unit : p.split_first + (unit - p.split_first) / p.k_parts;
+    const int part = whole ? 0 : (unit - p.split_first) % p.k_parts;
+    const int parts = whole ? 1 : p.k_parts;
+    const int tile_x = tile % p.row_tiles, tile_y = tile / p.row_tiles;
     const int row_base = tile_x * 2 * kTileM + (int)rank * kTileM;  // this CTA's 128 rows
-    const int tok_base = is_full ? tile_y * 512 : p.full_units * 512 + tile_y * 256;
-    const int total = p.nsteps + p.lr_stages;
+    const int tok_base = tile_y * 512;
+    const int n_acc = p.T - tok_base > 256 ? 2 : 1;
+    // the unit's stages [s_begin, s_begin + total) of the layer's nsteps weight stages and lr_stages low-rank stages
+    const int all_stages = p.nsteps + p.lr_stages;
+    const int s_begin = (all_stages * part / parts) & ~1;
+    const int total = (part == parts - 1 ? all_stages : ((all_stages * (part + 1) / parts) & ~1)) - s_begin;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - raw);
@@ -472,8 +478,8 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
         auto load_visit = [&](int buf, int v) {
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
-                const int s = 4 * v + 2 * g + j;
-                if (valid && s < p.nsteps) {
+                const int i = 4 * v + 2 * g + j, s = s_begin + i;
+                if (valid && i < total && s < p.nsteps) {
 #pragma unroll
                     for (int q = 0; q < BITS; ++q) wbuf[buf][j][q] = __ldg(wbase + (size_t)s * 32 * BITS + q);
                     const uint32_t* z = szbase + (size_t)(s >> p.gshift) * 16;
@@ -513,11 +519,12 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                 if (v < n_visits) {
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
-                        const int s = 4 * v + 2 * g + j;
-                        if (s < total) {
-                            const int slot = s % kPairAStages, use = s / kPairAStages;
+                        const int i = 4 * v + 2 * g + j;
+                        if (i < total) {
+                            const int slot = i % kPairAStages, use = i / kPairAStages;
                             if (use >= 1) warp_wait(empty_a(slot), (uint32_t)(use - 1) & 1u);
-                            if (valid && s < p.nsteps) convert(wbuf[u][j], szbuf[u][j][0], szbuf[u][j][1], base_ptr + slot * kPairABytes);
+                            if (valid && s_begin + i < p.nsteps)
+                                convert(wbuf[u][j], szbuf[u][j][0], szbuf[u][j][1], base_ptr + slot * kPairABytes);
                         }
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy (MMA)
@@ -540,17 +547,18 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
             const uint32_t b_bytes = (uint32_t)(2 * n_acc * kPairBHalf);  // both CTAs' copies of a stage
             int sa = 0, sb = 0;
             uint32_t pa = 1, pb = 1;  // parity of the previous use's "empty" phase
-            for (int s = 0; s < total; ++s) {
+            for (int i = 0; i < total; ++i) {
+                const int s = s_begin + i;  // stage of the layer; i counts the unit's stages (rings, parities)
                 // Weight stages: the first CTA's loader is one of the arrivals of full_a (so that the low-rank stages
                 // can count their A tiles there); it may arrive for this use of the slot once the previous use's
                 // phase is complete, which does not wait for the MMAs.  Low-rank stages write the slot: empty_a.
-                if (s >= kPairAStages) {
+                if (i >= kPairAStages) {
                     if (s >= p.nsteps) wait_phase(empty_a(sa), pa);
                     else if (rank == 0) wait_phase(full_a(sa), pa);
                 }
-                // the commit that frees weight slot (s - kPairBStages) % kPairAStages frees this activation slot too
-                if (s >= kPairBStages)
-                    wait_phase(empty_a((s - kPairBStages) % kPairAStages), (uint32_t)((s - kPairBStages) / kPairAStages) & 1u);
+                // the commit that frees weight slot (i - kPairBStages) % kPairAStages frees this activation slot too
+                if (i >= kPairBStages)
+                    wait_phase(empty_a((i - kPairBStages) % kPairAStages), (uint32_t)((i - kPairBStages) / kPairAStages) & 1u);
                 const uint32_t a_tile = base + sa * kPairABytes, b_tile = b_ring + sb * kPairBBytes;
                 const uint32_t fb = full_b0 + 8u * (uint32_t)sb, fa = full_a0 + 8u * (uint32_t)sa;
                 if (rank == 0) mbar_expect_tx(full_b(sb), b_bytes);
@@ -587,7 +595,8 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
             int sa = 0, sb = 0;
             uint32_t pa = 0, pb = 0;
             bool ready_a = mbar_test_wait(full_a(0), 0u), ready_b = mbar_test_wait(full_b(0), 0u);
-            for (int s = 0; s < total; ++s) {
+            for (int i = 0; i < total; ++i) {
+                const int s = s_begin + i;
                 if (!ready_a) wait_phase(full_a(sa), pa);
                 if (!ready_b) wait_phase(full_b(sb), pb);
                 tc_fence_after();
@@ -602,7 +611,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                     sb = 0;
                     pb ^= 1u;
                 }
-                if (s + 1 < total) {
+                if (i + 1 < total) {
                     ready_a = mbar_test_wait(full_a(sa), pa);
                     ready_b = mbar_test_wait(full_b(sb), pb);
                 }
@@ -610,7 +619,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                 const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
                 const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
                 for (int k = 0; k < ksub; ++k)
-                    umma_f16_pair(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (s > 0 || k > 0) ? 1u : 0u);
+                    umma_f16_pair(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
                 umma_commit_pair(commit_a);  // one commit per stage: the stage's weight and activation slots
             }
             umma_commit_pair(acc_ready);
@@ -641,7 +650,14 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                     : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const int tok0 = tok_base + acc * 256 + c0;
-                if (p.y_vec) {
+                if (!whole) {
+                    // fp32 partial sums of this K part: [unit][token of the tile][row of the tile]
+                    float* dst = p.kparts + ((size_t)(unit - p.split_first) * 512 + (size_t)(acc * 256 + c0)) * 256 +
+                                 (int)rank * kTileM + lane_base + lane;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (tok0 + i < p.T) dst[(size_t)i * 256] = __uint_as_float(v[i]);
+                } else if (p.y_vec) {
                     __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(base_ptr + (warp - kDequantWarps) * 2048);
                     __syncwarp();
 #pragma unroll
@@ -730,69 +746,43 @@ cudaError_t launch_prefill_bits(const PrefillParams& p, const CUtensorMap& mx, c
     return cudaLaunchKernelEx(&cfg, prefill_kernel<BITS>, p, mx, ma, mt);
 }
 
-// CTA pairs that can be resident at once (each CTA fills a multiprocessor); cached per device, 0 if the query fails
-template <int BITS>
-int pair_slots() {
-    static int cached[64];
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    int v = __atomic_load_n(&cached[dev & 63], __ATOMIC_ACQUIRE);
-    if (v != 0) return v > 0 ? v : 0;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * 1024);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kPairSmemBytes;
-    int n = 0;
-    const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, prefill_pair_kernel<BITS>, &cfg);
-    v = (e == cudaSuccess && n > 0) ? n : -1;
-    if (e != cudaSuccess) (void)cudaGetLastError();
-    __atomic_store_n(&cached[dev & 63], v, __ATOMIC_RELEASE);
-    return v > 0 ? v : 0;
+// The partial sums of the units cut along K, added in a fixed order: y[token][row] = sum over parts.  One thread per
+// token and four rows.
+__global__ void __launch_bounds__(256)
+prefill_kparts_kernel(const float* __restrict__ kparts, void* __restrict__ y, int64_t ldy, int out_f32, int m, int T,
+                      int row_tiles, int first_tile, int k_parts) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int split_tile = (int)blockIdx.x >> 7;                 // 128 blocks of 4 tokens x 256 rows per tile
+    const int tok_l = (((int)blockIdx.x & 127) << 2) + ((int)threadIdx.x >> 6);
+    const int row_l = ((int)threadIdx.x & 63) << 2;
+    const int tile = first_tile + split_tile;
+    const int tok = (tile / row_tiles) * 512 + tok_l, row = (tile % row_tiles) * 256 + row_l;
+    if (tok >= T || row >= m) return;
+    const float* src = kparts + (((size_t)split_tile * k_parts) * 512 + tok_l) * 256 + row_l;
+    float4 acc = *reinterpret_cast<const float4*>(src);
+    for (int part = 1; part < k_parts; ++part) {
+        const float4 v = *reinterpret_cast<const float4*>(src + (size_t)part * 512 * 256);
+        acc.x += v.x;
+        acc.y += v.y;
+        acc.z += v.z;
+        acc.w += v.w;
+    }
+    const float r[4] = {acc.x, acc.y, acc.z, acc.w};
+    const size_t o = (size_t)tok * ldy + row;
+    for (int e = 0; e < 4; ++e)
+        if (row + e < m) {  // d_out is a multiple of 64 today; the check keeps the kernel right for any m
+            if (out_f32) reinterpret_cast<float*>(y)[o + e] = r[e];
+            else reinterpret_cast<__nv_bfloat16*>(y)[o + e] = __float2bfloat16_rn(r[e]);
+        }
 }
 
 template <int BITS>
-cudaError_t launch_pair_bits(PairParams p, const CUtensorMap& mx, const CUtensorMap& ma, const CUtensorMap& mt, int chunks256,
-                             cudaStream_t s) {
+cudaError_t launch_pair_bits(PairParams p, const CUtensorMap& mx, const CUtensorMap& ma, const CUtensorMap& mt,
+                             const PairPlan& plan, cudaStream_t s) {
     static unsigned long long attr_done = 0;
     cudaError_t e = ensure_dynamic_smem(prefill_pair_kernel<BITS>, kPairSmemBytes, &attr_done);
     if (e != cudaSuccess) return e;
-    // Token chunks: full_units of 512 tokens first, then half_units of 256; the mix that minimises the makespan of a
-    // greedy schedule over the resident pairs (the cheaper tiles fill the last wave).
-    int slots = pair_slots<BITS>();
-    if (slots <= 0) slots = sm_count() / 2;
-    if (slots > 256) slots = 256;
-    int best_full = chunks256 / 2;
-    if ((long long)p.row_tiles * chunks256 <= 20000) {
-        double best_cost = 1e30;
-        for (int full = chunks256 / 2; full >= 0; --full) {
-            const int half = chunks256 - 2 * full;
-            double finish[256];
-            for (int i = 0; i < slots; ++i) finish[i] = 0.0;
-            auto place = [&](long long count, double dur) {
-                for (long long c = 0; c < count; ++c) {
-                    int best = 0;
-                    for (int i = 1; i < slots; ++i)
-                        if (finish[i] < finish[best]) best = i;
-                    finish[best] += dur;
-                }
-            };
-            place((long long)p.row_tiles * full, 1.0);
-            place((long long)p.row_tiles * half, kHalfTileCost);
-            double cost = 0.0;
-            for (int i = 0; i < slots; ++i) cost = finish[i] > cost ? finish[i] : cost;
-            if (cost < best_cost - 1e-9) {
-                best_cost = cost;
-                best_full = full;
-            }
-        }
-    }
-    {
-        const int forced = option(LOPRO_OPT_PREFILL_PAIRS);  // overrides the number of 512-token chunks (tuning only)
-        if (forced >= 0 && forced <= chunks256 / 2) best_full = forced;
-    }
-    p.full_units = best_full;
-    p.half_units = chunks256 - 2 * best_full;
-    const long long n_ctas = 2LL * p.row_tiles * (p.full_units + p.half_units);
+    const long long n_ctas = 2LL * (plan.n_tiles - plan.split_tiles + (long long)plan.split_tiles * plan.k_parts);
     if (n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)n_ctas);
@@ -804,7 +794,13 @@ cudaError_t launch_pair_bits(PairParams p, const CUtensorMap& mx, const CUtensor
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BITS>, p, mx, ma, mt);
+    e = cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BITS>, p, mx, ma, mt);
+    if (e != cudaSuccess || plan.split_tiles == 0) return e;
+    cfg.gridDim = dim3((unsigned)plan.split_tiles * 128u);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    return cudaLaunchKernelEx(&cfg, prefill_kparts_kernel, (const float*)p.kparts, p.y, p.ldy, p.out_f32, p.m, p.T, p.row_tiles,
+                              plan.n_tiles - plan.split_tiles, plan.k_parts);
 }
 
 }  // namespace
@@ -812,6 +808,49 @@ cudaError_t launch_pair_bits(PairParams p, const CUtensorMap& mx, const CUtensor
 bool prefill_supported(const lopro_desc& d, int T) {
     const int off = option(LOPRO_OPT_NO_TCGEN05) == 1 ? 1 : 0;  // tuning / A-B comparison only
     return off == 0 && T > kDecodeMaxT && encode_tiled_fn() != nullptr && (d.d_in % 64) == 0;
+}
+
+// Tiling of the two-CTA kernel: tiles of 256 rows x 512 tokens over the CTA pairs the device holds at once (one CTA
+// fills a multiprocessor).  The tiles of the last, partial wave are cut along K into as many parts as fill the idle
+// pairs (at most kMaxKParts, at least eight stages each), so that the wave ends early instead of running a full
+// tile's length on a few pairs.
+PairPlan pair_plan(const lopro_desc& d, int T) {
+    PairPlan plan = {};
+    if (T < kPairMinT) return plan;
+    plan.use = 1;
+    plan.row_tiles = (d.d_out + 2 * kTileM - 1) / (2 * kTileM);
+    const long long n_tiles = (long long)plan.row_tiles * ((T + 511) / 512);
+    if (n_tiles > 0x3fffffffLL) {
+        plan.use = 0;
+        return plan;
+    }
+    plan.n_tiles = (int)n_tiles;
+    const int slots = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
+    const int rem = plan.n_tiles % slots;
+    const int stages = d.d_in / kStageK + (round_up_int(d.rank, 16) + kStageK - 1) / kStageK;
+    int parts = rem > 0 ? slots / rem : 1;
+    if (parts > kMaxKParts) parts = kMaxKParts;
+    if (parts > stages / 8) parts = stages / 8;
+    const int forced = option(LOPRO_OPT_PREFILL_PAIRS);  // tuning and tests: K parts of the last wave, 0 or 1 = none
+    if (forced >= 0 && rem > 0) parts = forced < kMaxKParts ? forced : kMaxKParts;
+    if (parts > stages / 2) parts = stages / 2;  // every part holds at least two stages
+    if (parts >= 2) {
+        plan.split_tiles = rem;
+        plan.k_parts = parts;
+    } else {
+        plan.split_tiles = 0;
+        plan.k_parts = 1;
+    }
+    return plan;
+}
+
+// fp32 partial sums of the tiles cut along K; sized for the most parts the plan may use, whatever the switches say
+size_t prefill_kparts_bytes(const lopro_desc& d, int T) {
+    const PairPlan plan = pair_plan(d, T);
+    if (!plan.use) return 0;
+    const int slots = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
+    const int rem = plan.n_tiles % slots;
+    return (size_t)rem * kMaxKParts * 512 * 256 * sizeof(float);
 }
 
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
@@ -835,7 +874,8 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     p.r_pad = d.rank > 0 ? L.r_pad : 0;
     p.tile_n = T <= 64 ? 64 : (T <= 128 ? 128 : 256);
     p.lr_stages = (p.r_pad + kStageK - 1) / kStageK;
-    if (T >= kPairMinT && option(LOPRO_OPT_NO_CTA_PAIRS) != 1) {
+    const PairPlan plan = pair_plan(d, T);
+    if (plan.use && option(LOPRO_OPT_NO_CTA_PAIRS) != 1) {
         // large batches: two CTAs per tile (each loads boxes of 128 tokens)
         PairParams q;
         q.codes = p.codes;
@@ -853,8 +893,10 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
         q.ng = p.ng;
         q.r_pad = p.r_pad;
         q.lr_stages = p.lr_stages;
-        q.row_tiles = (d.d_out + 2 * kTileM - 1) / (2 * kTileM);
-        q.full_units = q.half_units = 0;
+        q.row_tiles = plan.row_tiles;
+        q.split_first = plan.n_tiles - plan.split_tiles;
+        q.k_parts = plan.k_parts;
+        q.kparts = reinterpret_cast<float*>(const_cast<uint8_t*>(ws) + W.off_kparts);
         CUtensorMap qx, qa, qt;
         if (!make_map(&qx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ws + W.off_xrot, (uint64_t)d.d_in, (uint64_t)T, 128u))
             return cudaErrorInvalidValue;
@@ -866,11 +908,10 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
                 !make_map(&qt, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ws + W.off_t, (uint64_t)q.r_pad, (uint64_t)T, 128u))
                 return cudaErrorInvalidValue;
         }
-        const int chunks256 = (T + 255) / 256;
         switch (d.bits) {
-            case 2: return launch_pair_bits<2>(q, qx, qa, qt, chunks256, s);
-            case 3: return launch_pair_bits<3>(q, qx, qa, qt, chunks256, s);
-            default: return launch_pair_bits<4>(q, qx, qa, qt, chunks256, s);
+            case 2: return launch_pair_bits<2>(q, qx, qa, qt, plan, s);
+            case 3: return launch_pair_bits<3>(q, qx, qa, qt, plan, s);
+            default: return launch_pair_bits<4>(q, qx, qa, qt, plan, s);
         }
     }
     CUtensorMap mx, ma, mt;

@@ -170,16 +170,19 @@ def test_shapes_in_the_parameter_domain(n, m, bits, g, b_i, b_h, r, T):
     (2048, 384, 3, 128, 40, 512),    # rank padded inside a stage
 ])
 def test_large_batches_pair_two_ctas_on_a_tile(n, m, bits, g, r, T):
-    """512 tokens and more: the prefill kernel puts the two CTAs of a cluster on one tile of 256 rows x 512 or 256
-    tokens.  Every mix of 512- and 256-token chunks is run, and the kernel with one CTA per tile on the same inputs."""
+    """512 tokens and more: the prefill kernel puts the two CTAs of a cluster on one tile of 256 rows x 512 tokens and
+    cuts the tiles of the last wave along K (their partial sums are added by a second kernel).  Run with the library's
+    choice of K parts, with none, and with 2, 3 and 4; and with one CTA per tile on the same inputs."""
     layer = random_layer_np(n, m, bits, g, r, seed=n + m + T)
     d = lopro.make_desc(n, m, bits, g, 128, identity_cols=128, rank=r)
     x_bits = synth.activations(T, n, seed=T, outlier_frac=0.01)
     assert lopro.linear_fwd_path(d, T)[0] == lopro.PATH_PREFILL
-    chunks = (T + 255) // 256
-    for full in [-1] + list(range(chunks // 2 + 1)):
-        with lopro.configured(lopro.OPT_PREFILL_PAIRS, full):
+    launches = set()
+    for parts in (-1, 0, 2, 3, 4):
+        with lopro.configured(lopro.OPT_PREFILL_PAIRS, parts):
+            launches.add(lopro.linear_fwd_path(d, T)[1])
             _check_forward_once(layer, d, x_bits, None, GATE_A, GATE_B)
+    assert len(launches) == 2                       # with and without the kernel that adds the K parts
     blob = _pack(layer, d)
     x = bf16_bits_to_device(x_bits)
     y_pair = lopro.linear_fwd(d, blob, x, lopro.OUT_F32)
