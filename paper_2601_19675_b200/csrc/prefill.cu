@@ -440,8 +440,19 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
         if (mbar_try_wait(bar, parity)) return;
         if (!timed_out() && !mbar_wait(bar, parity, kPrefillSpin)) time_out();
     };
+    // Waits of the warps that run ahead of the MMAs or behind them: a failed poll sleeps before the next one.  Every
+    // poll is a shared-memory operation, and the MMA-issuing threads' own barrier operations queue behind them.
+    auto wait_relaxed = [&](uint32_t bar, uint32_t parity, unsigned sleep_ns) {
+        if (mbar_try_wait(bar, parity)) return;
+        if (timed_out()) return;
+        for (uint32_t it = 0; it < kPrefillSpin; ++it) {
+            __nanosleep(sleep_ns);
+            if (mbar_try_wait(bar, parity)) return;
+        }
+        time_out();
+    };
     auto warp_wait = [&](uint32_t bar, uint32_t parity) {
-        if (lane == 0) wait_phase(bar, parity);
+        if (lane == 0) wait_relaxed(bar, parity, 128u);
         __syncwarp();
     };
     const uint32_t tmem_cols = n_acc == 2 ? 512u : 256u;
@@ -553,12 +564,12 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                 // can count their A tiles there); it may arrive for this use of the slot once the previous use's
                 // phase is complete, which does not wait for the MMAs.  Low-rank stages write the slot: empty_a.
                 if (i >= kPairAStages) {
-                    if (s >= p.nsteps) wait_phase(empty_a(sa), pa);
-                    else if (rank == 0) wait_phase(full_a(sa), pa);
+                    if (s >= p.nsteps) wait_relaxed(empty_a(sa), pa, 64u);
+                    else if (rank == 0) wait_relaxed(full_a(sa), pa, 64u);
                 }
                 // the commit that frees weight slot (i - kPairBStages) % kPairAStages frees this activation slot too
                 if (i >= kPairBStages)
-                    wait_phase(empty_a((i - kPairBStages) % kPairAStages), (uint32_t)((i - kPairBStages) / kPairAStages) & 1u);
+                    wait_relaxed(empty_a((i - kPairBStages) % kPairAStages), (uint32_t)((i - kPairBStages) / kPairAStages) & 1u, 64u);
                 const uint32_t a_tile = base + sa * kPairABytes, b_tile = b_ring + sb * kPairBBytes;
                 const uint32_t fb = full_b0 + 8u * (uint32_t)sb, fa = full_a0 + 8u * (uint32_t)sa;
                 if (rank == 0) mbar_expect_tx(full_b(sb), b_bytes);
@@ -588,10 +599,10 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
         if (lane == 0 && acc < n_acc) {
             const uint32_t idesc_w = make_idesc_pair(256, 1u), idesc_lr = make_idesc_pair(256, 0u);
             const uint32_t d = tmem + (uint32_t)(acc * 256);
-            // The thread's time per stage bounds the kernel (the tensor pipe idles while it waits), and every
-            // barrier operation is a shared-memory round trip behind the dequant warps' traffic.  So the next
-            // stage's barriers are polled (without suspending) before this stage's MMAs are issued: the answers
-            // arrive while the MMAs queue up, and a stage whose tiles were ready by then waits for nothing.
+            // The thread's time per stage bounds the kernel: the tensor pipe holds a few MMAs in its queue and idles
+            // once the thread falls behind, and every barrier operation is a shared-memory round trip behind the
+            // dequant warps' traffic.  So the next stage's barriers are polled (without suspending) right after
+            // this stage's MMAs and commit are queued, and a stage whose tiles were ready by then waits for nothing.
             int sa = 0, sb = 0;
             uint32_t pa = 0, pb = 0;
             bool ready_a = mbar_test_wait(full_a(0), 0u), ready_b = mbar_test_wait(full_b(0), 0u);
@@ -611,16 +622,16 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                     sb = 0;
                     pb ^= 1u;
                 }
-                if (i + 1 < total) {
-                    ready_a = mbar_test_wait(full_a(sa), pa);
-                    ready_b = mbar_test_wait(full_b(sb), pb);
-                }
                 const bool lowrank = s >= p.nsteps;
                 const int ksub = lowrank ? min(4, (p.r_pad - (s - p.nsteps) * kStageK) / 16) : 4;
                 const uint32_t idesc = lowrank ? idesc_lr : idesc_w;
                 for (int k = 0; k < ksub; ++k)
                     umma_f16_pair(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
                 umma_commit_pair(commit_a);  // one commit per stage: the stage's weight and activation slots
+                if (i + 1 < total) {  // answered while the tensor pipe works through the MMAs just queued
+                    ready_a = mbar_test_wait(full_a(sa), pa);
+                    ready_b = mbar_test_wait(full_b(sb), pb);
+                }
             }
             umma_commit_pair(acc_ready);
         }
@@ -629,7 +640,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
     if (warp >= kDequantWarps) {
         // ---------------- epilogue: this CTA's 128 rows of every accumulator ----------------
         __syncwarp();
-        if (lane == 0) wait_phase(acc_ready, 0u);
+        if (lane == 0) wait_relaxed(acc_ready, 0u, 512u);
         __syncwarp();
         tc_fence_after();
         const int lane_base = (warp & 3) * 32;
