@@ -91,7 +91,7 @@ def time_oracle_stack(T, budget_s):
 # the kernels as committed (profiles/: the commands; counters re-read after the last change of each kernel, as ncu
 # prints them, i.e. to 10 kB); null for workloads without a capture.
 NCU_TRAFFIC = {("cfg2_T8", "stream_wide_kernel"): 9290000, ("cfg2_T32", "stream_kernel"): 9490000,
-               ("cfg4_T16", "tall_kernel"): 82610000, ("cfg3_T2048", "prefill_kernel"): 55460000}
+               ("cfg4_T16", "tall_kernel"): 82610000, ("cfg3_T2048", "prefill_pair_kernel"): 61700000}
 METRIC = "quantized-linear fwd tokens/s"
 UNIT = "tokens/s"
 
@@ -628,7 +628,8 @@ def measure(args, name, steps, warmup, rank, world, local, dev, dist, with_e2e=T
     value = w.tokens_per_pass * passes * world / (ms_per_step * 1e-3)
     per_forward_s = ms_per_pass * 1e-3 / w.forwards
     kernel = " + ".join({"stream": "stream_kernel", "wide": "stream_wide_kernel", "tall": "tall_kernel", "general": "decode_kernel",
-                         "prefill": "prefill_kernel", "rowblock": "rowblock_kernel"}.get(n, n) for n in w.paths)
+                         "prefill": "prefill_pair_kernel" if w.T >= 512 else "prefill_kernel",
+                         "rowblock": "rowblock_kernel"}.get(n, n) for n in w.paths)
     note = ("duration = step time / layer forwards (includes the prologue kernels of each forward): an upper bound on the "
             "product kernel's own duration, a lower bound on `achieved`")
     if getattr(w, "block", False):
