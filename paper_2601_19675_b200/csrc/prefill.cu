@@ -844,6 +844,7 @@ PairPlan pair_plan(const lopro_desc& d, int T) {
     if (parts > stages / 8) parts = stages / 8;
     const int forced = option(LOPRO_OPT_PREFILL_PAIRS);  // tuning and tests: K parts of the last wave, 0 or 1 = none
     if (forced >= 0 && rem > 0) parts = forced < kMaxKParts ? forced : kMaxKParts;
+    if (rem > 0 && parts > slots / rem) parts = slots / rem;  // the units of the last wave fit the resident pairs
     if (parts > stages / 2) parts = stages / 2;  // every part holds at least two stages
     if (parts >= 2) {
         plan.split_tiles = rem;
@@ -855,13 +856,14 @@ PairPlan pair_plan(const lopro_desc& d, int T) {
     return plan;
 }
 
-// fp32 partial sums of the tiles cut along K; sized for the most parts the plan may use, whatever the switches say
+// fp32 partial sums of the tiles cut along K: room for the most units any plan may use (one per resident pair, four
+// per tile), whatever the switches say -- a bound that does not decrease as T grows, unlike the plan's own count
 size_t prefill_kparts_bytes(const lopro_desc& d, int T) {
     const PairPlan plan = pair_plan(d, T);
     if (!plan.use) return 0;
-    const int slots = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
-    const int rem = plan.n_tiles % slots;
-    return (size_t)rem * kMaxKParts * 512 * 256 * sizeof(float);
+    const long long slots = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
+    const long long by_tiles = (long long)plan.n_tiles * kMaxKParts;
+    return (size_t)(by_tiles < slots ? by_tiles : slots) * 512 * 256 * sizeof(float);
 }
 
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
