@@ -637,16 +637,19 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
         }
     }
 
-    if (warp >= kDequantWarps) {
-        // ---------------- epilogue: this CTA's 128 rows of every accumulator ----------------
+    {
+        // ---------------- epilogue: this CTA's 128 rows of every accumulator, by all twenty warps ----------------
+        // A warp may read the 32 tensor-memory lanes of its quarter (warp & 3); the five warps of a quarter take the
+        // accumulators' 32-column pieces in turn, so the tensor pipe idles a fifth as long as with four warps.
         __syncwarp();
-        if (lane == 0) wait_relaxed(acc_ready, 0u, 512u);
+        if (lane == 0) wait_relaxed(acc_ready, 0u, warp < kDequantWarps ? 256u : 512u);
         __syncwarp();
         tc_fence_after();
         const int lane_base = (warp & 3) * 32;
         const int row = row_base + lane_base + lane;
-        for (int acc = 0; acc < n_acc; ++acc) {
-            for (int c0 = 0; c0 < 256; c0 += 32) {
+        for (int piece32 = warp >> 2; piece32 < n_acc * 8; piece32 += (kDequantWarps + 4) / 4) {
+            {
+                const int acc = piece32 >> 3, c0 = (piece32 & 7) * 32;
                 if (tok_base + acc * 256 + c0 >= p.T) break;  // uniform over the warp
                 uint32_t v[32];
                 const uint32_t taddr = tmem + ((uint32_t)lane_base << 16) + (uint32_t)(acc * 256 + c0);
@@ -669,7 +672,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                     for (int i = 0; i < 32; ++i)
                         if (tok0 + i < p.T) dst[(size_t)i * 256] = __uint_as_float(v[i]);
                 } else if (p.y_vec) {
-                    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(base_ptr + (warp - kDequantWarps) * 2048);
+                    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(base_ptr + warp * 2048);
                     __syncwarp();
 #pragma unroll
                     for (int i = 0; i < 32; ++i) stg[i * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[i]));
