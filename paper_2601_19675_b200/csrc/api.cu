@@ -337,9 +337,9 @@ static bool use_tall(const lopro_desc& d, int T) {
 // the small-batch kernels when that costs less than the tensor-core path: a prefill CTA walks all of K for its
 // 128 or 256 rows whatever the token count, and a layer with few rows fills few SMs.  Both sides are estimated from
 // timings on B200 (microseconds, beyond a common 8 for the first launches): a chunk 3 + 0.45e-6 d_out d_in (10.9 for
-// 4096 x 4096, 23.4 for 4096 x 11008 either way round), the prefill kernel 0.017 d_in per wave of CTAs (74 in all
-// for d_in = 4096, 205 for 11008, flat from 33 to 256 tokens).  LOPRO_OPT_NO_CHUNKS turns this off (A/B runs, tests
-// of the prefill kernel on small layers).
+// 4096 x 4096, 23.4 for 4096 x 11008 either way round), the tensor-core product by prefill_estimate_us plus 0.0015 d_in
+// for the longer launches in front of it (4096 x 4096: chunks up to 64 tokens, 25.0 against 29.8; 11008 -> 4096: up to
+// 96, 77 against 84).  LOPRO_OPT_NO_CHUNKS turns this off (A/B runs, tests of the prefill kernels on small layers).
 static int small_batch_chunks(const lopro_desc& d, int T) {
     if (T <= kDecodeMaxT) return 0;
     if (d.lowrank_format == LOPRO_LOWRANK_FP8)  // served by the small-batch kernels only: always chunks
@@ -348,9 +348,7 @@ static int small_batch_chunks(const lopro_desc& d, int T) {
     if (!prefill_supported(d, T)) return 0;  // keep the general path's behaviour where there is no prefill kernel
     const int chunks = (T + kDecodeMaxT - 1) / kDecodeMaxT;
     const double chunk_us = 3.0 + 0.45e-6 * (double)d.d_out * (double)d.d_in;
-    const int ctas = ((d.d_out + 255) / 256) * ((T + 255) / 256);  // two 128-row blocks per CTA
-    const int sms = sm_count();
-    const double prefill_us = 0.017 * (double)d.d_in * (double)((ctas + sms - 1) / sms);
+    const double prefill_us = prefill_estimate_us(d, T, nullptr) + 0.0015 * (double)d.d_in;  // + its longer launches in front
     if ((double)chunks * chunk_us >= prefill_us) return 0;
     if (!prologue_supported(d, kDecodeMaxT) || !stream_supported(d, kDecodeMaxT)) return 0;
     return chunks;
@@ -389,9 +387,10 @@ int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launch
                             : 1 + (desc->rank > 0 ? (T > kDecodeMaxT ? 2 : 1) : 0);
         path = prefill_supported(*desc, T) ? LOPRO_PATH_PREFILL : LOPRO_PATH_GENERAL;
         n = pre + 1;
-        if (path == LOPRO_PATH_PREFILL && option(LOPRO_OPT_NO_CTA_PAIRS) != 1) {
-            const PairPlan plan = pair_plan(*desc, T);
-            if (plan.use && plan.split_tiles > 0) ++n;  // the sum of the K parts of the last wave's tiles
+        if (path == LOPRO_PATH_PREFILL) {
+            bool use_pairs = false;
+            (void)prefill_estimate_us(*desc, T, &use_pairs);
+            if (use_pairs && pair_plan(*desc, T).split_tiles > 0) ++n;  // the sum of the K parts of the last wave's tiles
         }
     }
     if (launches) *launches = n;

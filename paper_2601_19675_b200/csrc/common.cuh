@@ -223,6 +223,8 @@ struct PairPlan {
 };
 PairPlan pair_plan(const lopro_desc& d, int T);
 size_t prefill_kparts_bytes(const lopro_desc& d, int T);
+// Estimated duration (microseconds) of the tensor-core product for T > 32 tokens and whether it runs two CTAs per tile
+double prefill_estimate_us(const lopro_desc& d, int T, bool* use_pairs);
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                            const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
 

@@ -372,7 +372,10 @@ constexpr int kPairAStages = LOPRO_PAIR_A_STAGES;  // even: a visit fills two ne
 constexpr int kPairBStages = LOPRO_PAIR_B_STAGES;
 static_assert(kPairBStages <= kPairAStages, "one 'empty' barrier per weight slot serves both rings");
 constexpr int kPairSmemBytes = kPairAStages * kPairABytes + kPairBStages * kPairBBytes + 1024;
-constexpr int kPairMinT = 512;   // smaller batches keep one CTA per tile (finer tiles fill the machine better)
+#ifndef LOPRO_PAIR_MIN_T
+#define LOPRO_PAIR_MIN_T 512
+#endif
+constexpr int kPairMinT = LOPRO_PAIR_MIN_T;   // from here on always two CTAs per tile; below, by prefill_estimate_us
 constexpr int kMaxKParts = 4;    // K parts of a tile of the last wave
 
 struct PairParams {
@@ -388,7 +391,8 @@ struct PairParams {
     int row_tiles;    // tiles of 256 rows
     int split_first;  // tiles from this index on are split along K into k_parts units each (the last wave)
     int k_parts;
-    float* kparts;    // their fp32 partial sums, [unit][512 tokens][256 rows]
+    float* kparts;    // their fp32 partial sums, [unit][kp_tokens][256 rows]
+    int kp_tokens;    // token rows per unit there: min(512, T rounded up to 32)
     int lr_stages;
 };
 
@@ -666,7 +670,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                 const int tok0 = tok_base + acc * 256 + c0;
                 if (!whole) {
                     // fp32 partial sums of this K part: [unit][token of the tile][row of the tile]
-                    float* dst = p.kparts + ((size_t)(unit - p.split_first) * 512 + (size_t)(acc * 256 + c0)) * 256 +
+                    float* dst = p.kparts + ((size_t)(unit - p.split_first) * p.kp_tokens + (size_t)(acc * 256 + c0)) * 256 +
                                  (int)rank * kTileM + lane_base + lane;
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
@@ -764,18 +768,19 @@ cudaError_t launch_prefill_bits(const PrefillParams& p, const CUtensorMap& mx, c
 // token and four rows.
 __global__ void __launch_bounds__(256)
 prefill_kparts_kernel(const float* __restrict__ kparts, void* __restrict__ y, int64_t ldy, int out_f32, int m, int T,
-                      int row_tiles, int first_tile, int k_parts) {
+                      int row_tiles, int first_tile, int k_parts, int kp_tokens) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int split_tile = (int)blockIdx.x >> 7;                 // 128 blocks of 4 tokens x 256 rows per tile
-    const int tok_l = (((int)blockIdx.x & 127) << 2) + ((int)threadIdx.x >> 6);
+    const int blocks_per_tile = kp_tokens >> 2;                  // blocks of 4 tokens x 256 rows
+    const int split_tile = (int)blockIdx.x / blocks_per_tile;
+    const int tok_l = (((int)blockIdx.x % blocks_per_tile) << 2) + ((int)threadIdx.x >> 6);
     const int row_l = ((int)threadIdx.x & 63) << 2;
     const int tile = first_tile + split_tile;
     const int tok = (tile / row_tiles) * 512 + tok_l, row = (tile % row_tiles) * 256 + row_l;
     if (tok >= T || row >= m) return;
-    const float* src = kparts + (((size_t)split_tile * k_parts) * 512 + tok_l) * 256 + row_l;
+    const float* src = kparts + (((size_t)split_tile * k_parts) * kp_tokens + tok_l) * 256 + row_l;
     float4 acc = *reinterpret_cast<const float4*>(src);
     for (int part = 1; part < k_parts; ++part) {
-        const float4 v = *reinterpret_cast<const float4*>(src + (size_t)part * 512 * 256);
+        const float4 v = *reinterpret_cast<const float4*>(src + (size_t)part * kp_tokens * 256);
         acc.x += v.x;
         acc.y += v.y;
         acc.z += v.z;
@@ -810,11 +815,11 @@ cudaError_t launch_pair_bits(PairParams p, const CUtensorMap& mx, const CUtensor
     cfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BITS>, p, mx, ma, mt);
     if (e != cudaSuccess || plan.split_tiles == 0) return e;
-    cfg.gridDim = dim3((unsigned)plan.split_tiles * 128u);
+    cfg.gridDim = dim3((unsigned)plan.split_tiles * (unsigned)(p.kp_tokens / 4));
     cfg.blockDim = dim3(256);
     cfg.dynamicSmemBytes = 0;
     return cudaLaunchKernelEx(&cfg, prefill_kparts_kernel, (const float*)p.kparts, p.y, p.ldy, p.out_f32, p.m, p.T, p.row_tiles,
-                              plan.n_tiles - plan.split_tiles, plan.k_parts);
+                              plan.n_tiles - plan.split_tiles, plan.k_parts, p.kp_tokens);
 }
 
 }  // namespace
@@ -830,7 +835,7 @@ bool prefill_supported(const lopro_desc& d, int T) {
 // tile's length on a few pairs.
 PairPlan pair_plan(const lopro_desc& d, int T) {
     PairPlan plan = {};
-    if (T < kPairMinT) return plan;
+    if (T <= kDecodeMaxT) return plan;
     plan.use = 1;
     plan.row_tiles = (d.d_out + 2 * kTileM - 1) / (2 * kTileM);
     const long long n_tiles = (long long)plan.row_tiles * ((T + 511) / 512);
@@ -861,12 +866,45 @@ PairPlan pair_plan(const lopro_desc& d, int T) {
 
 // fp32 partial sums of the tiles cut along K: room for the most units any plan may use (one per resident pair, four
 // per tile), whatever the switches say -- a bound that does not decrease as T grows, unlike the plan's own count
+static int kparts_tokens(int T) { return T >= 512 ? 512 : round_up_int(T, 32); }
 size_t prefill_kparts_bytes(const lopro_desc& d, int T) {
     const PairPlan plan = pair_plan(d, T);
     if (!plan.use) return 0;
     const long long slots = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
     const long long by_tiles = (long long)plan.n_tiles * kMaxKParts;
-    return (size_t)(by_tiles < slots ? by_tiles : slots) * 512 * 256 * sizeof(float);
+    return (size_t)(by_tiles < slots ? by_tiles : slots) * kparts_tokens(T) * 256 * sizeof(float);
+}
+
+// Which of the two tensor-core kernels serves T tokens, and an estimate of its duration in microseconds (beyond the
+// launches in front of it), from timings on B200 per 64-column stage of one CTA: two CTAs on a tile 0.95 (two
+// accumulators) or 0.80 (one, T <= 256), one CTA per tile 0.78 (one 128-row block) or 1.03 (two); a tile cut along K
+// costs its share plus 9 (start-up of the shorter units and the kernel that adds them).  From 512 tokens on the
+// two-CTA kernel always; below, whichever is estimated faster: few row tiles favour the two-CTA kernel (its K parts
+// fill the machine), many row tiles and at most 256 tokens the other (twice the rows per CTA for the same conversion).
+double prefill_estimate_us(const lopro_desc& d, int T, bool* use_pairs) {
+    const int stages = d.d_in / kStageK + (round_up_int(d.rank, 16) + kStageK - 1) / kStageK;
+    // one CTA per tile
+    const int tile_n = T <= 64 ? 64 : (T <= 128 ? 128 : 256);
+    const int units = (T + tile_n - 1) / tile_n, m_tiles = (d.d_out + kTileM - 1) / kTileM;
+    const int n_sm = sm_count() > 0 ? sm_count() : 1;
+    const long long two_block = (long long)(m_tiles / 2) * units, one_block = (long long)(m_tiles % 2) * units;
+    const long long waves2 = (two_block + n_sm - 1) / n_sm, all_single_waves = ((long long)m_tiles * units + n_sm - 1) / n_sm;
+    double single_us = (double)stages * 0.78 * (double)all_single_waves;
+    const double mixed_us = (double)stages * (1.03 * (double)waves2 + (one_block > 0 && two_block % n_sm == 0 ? 0.78 : 0.0));
+    if (two_block > 0 && mixed_us < single_us) single_us = mixed_us;
+    single_us += 4.0;  // start-up and read-out of a CTA
+    // two CTAs per tile
+    const PairPlan plan = pair_plan(d, T);
+    double pair_us = 1e30;
+    if (plan.use && option(LOPRO_OPT_NO_CTA_PAIRS) != 1) {
+        const int slots = n_sm / 2 > 0 ? n_sm / 2 : 1;
+        const double tile_us = (double)stages * (T > 256 ? 0.95 : 0.80) + 4.0;
+        const int whole_waves = (plan.n_tiles - plan.split_tiles + slots - 1) / slots;
+        pair_us = tile_us * (double)whole_waves + (plan.split_tiles > 0 ? tile_us / (double)plan.k_parts + 9.0 : 0.0);
+    }
+    const bool pairs = T >= kPairMinT ? pair_us < 1e29 : (T > 256 ? pair_us <= single_us * 1.05 : pair_us < single_us);
+    if (use_pairs) *use_pairs = pairs;
+    return pairs ? pair_us : single_us;
 }
 
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
@@ -891,8 +929,10 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     p.tile_n = T <= 64 ? 64 : (T <= 128 ? 128 : 256);
     p.lr_stages = (p.r_pad + kStageK - 1) / kStageK;
     const PairPlan plan = pair_plan(d, T);
-    if (plan.use && option(LOPRO_OPT_NO_CTA_PAIRS) != 1) {
-        // large batches: two CTAs per tile (each loads boxes of 128 tokens)
+    bool use_pairs = false;
+    (void)prefill_estimate_us(d, T, &use_pairs);
+    if (use_pairs) {
+        // two CTAs per tile (each loads boxes of 128 tokens)
         PairParams q;
         q.codes = p.codes;
         q.sz = p.sz;
@@ -913,6 +953,7 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
         q.split_first = plan.n_tiles - plan.split_tiles;
         q.k_parts = plan.k_parts;
         q.kparts = reinterpret_cast<float*>(const_cast<uint8_t*>(ws) + W.off_kparts);
+        q.kp_tokens = kparts_tokens(T);
         CUtensorMap qx, qa, qt;
         if (!make_map(&qx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ws + W.off_xrot, (uint64_t)d.d_in, (uint64_t)T, 128u))
             return cudaErrorInvalidValue;
@@ -948,25 +989,27 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     const int units = (T + p.tile_n - 1) / p.tile_n;
     const int m_tiles = (d.d_out + kTileM - 1) / kTileM;
     int best_pairs = m_tiles / 2;
-    const int n_sm = sm_count() < 256 ? sm_count() : 256;
-    if ((long long)m_tiles * units <= 20000) {
+    const int n_sm = sm_count() > 0 ? sm_count() : 1;
+    {
+        // Makespan of the greedy schedule in closed form (the search runs on the host at every launch): the two-block
+        // CTAs leave the SMs on at most two levels, and the one-block CTAs then fill the lower level a round at a time.
+        auto makespan = [&](long long n_pairs, long long n_singles) {
+            const long long q = n_pairs / n_sm, rem = n_pairs % n_sm;
+            double level[2] = {(double)q * kPairCost, (double)(q + 1) * kPairCost};
+            long long count[2] = {n_sm - rem, rem};
+            double span = n_pairs > 0 ? (rem > 0 ? level[1] : level[0]) : 0.0;
+            while (n_singles > 0) {
+                const int g = (count[1] == 0 || level[0] <= level[1]) ? 0 : 1;
+                level[g] += 1.0;
+                if (level[g] > span) span = level[g];
+                n_singles -= count[g];
+            }
+            return span;
+        };
         double best_cost = 1e30;
-        for (int pairs = m_tiles / 2; pairs >= 0; --pairs) {
-            const int singles = m_tiles - 2 * pairs;
-            double finish[256];
-            for (int i = 0; i < n_sm; ++i) finish[i] = 0.0;
-            auto place = [&](long long count, double dur) {
-                for (long long c = 0; c < count; ++c) {
-                    int best = 0;
-                    for (int i = 1; i < n_sm; ++i)
-                        if (finish[i] < finish[best]) best = i;
-                    finish[best] += dur;
-                }
-            };
-            place((long long)pairs * units, kPairCost);
-            place((long long)singles * units, 1.0);
-            double cost = 0.0;
-            for (int i = 0; i < n_sm; ++i) cost = finish[i] > cost ? finish[i] : cost;
+        // (many waves: the mix hardly matters, and the search is not worth its host time)
+        for (int pairs = m_tiles / 2; pairs >= ((long long)m_tiles * units <= 20000 ? 0 : m_tiles / 2); --pairs) {
+            const double cost = makespan((long long)pairs * units, (long long)(m_tiles - 2 * pairs) * units);
             if (cost < best_cost - 1e-9) {
                 best_cost = cost;
                 best_pairs = pairs;

@@ -168,6 +168,9 @@ def test_shapes_in_the_parameter_domain(n, m, bits, g, b_i, b_h, r, T):
     (768, 144, 2, 64, 0, 777),       # no low-rank stages; 144 rows in a tile of 256
     (1024, 512, 4, 64, 128, 1030),   # two low-rank stages; last chunk holds 6 tokens
     (2048, 384, 3, 128, 40, 512),    # rank padded inside a stage
+    (1024, 256, 4, 128, 16, 40),     # below 512 tokens the two-CTA kernel serves layers with few row tiles:
+    (768, 144, 2, 64, 17, 130),      # one accumulator, token boxes that reach past the batch,
+    (2048, 384, 3, 64, 64, 300),     # two accumulators with a ragged second one
 ])
 def test_large_batches_pair_two_ctas_on_a_tile(n, m, bits, g, r, T):
     """512 tokens and more: the prefill kernel puts the two CTAs of a cluster on one tile of 256 rows x 512 tokens and
@@ -176,6 +179,11 @@ def test_large_batches_pair_two_ctas_on_a_tile(n, m, bits, g, r, T):
     layer = random_layer_np(n, m, bits, g, r, seed=n + m + T)
     d = lopro.make_desc(n, m, bits, g, 128, identity_cols=128, rank=r)
     x_bits = synth.activations(T, n, seed=T, outlier_frac=0.01)
+    with lopro.configured(lopro.OPT_NO_CHUNKS, 1):
+        _pair_kernel_cases(layer, d, x_bits, T)
+
+
+def _pair_kernel_cases(layer, d, x_bits, T):
     assert lopro.linear_fwd_path(d, T)[0] == lopro.PATH_PREFILL
     launches = set()
     for parts in (-1, 0, 2, 3, 4):
@@ -249,10 +257,10 @@ def test_groups_as_long_as_or_longer_than_a_stage(g, T, m):
 
 @pytest.mark.parametrize("T,n,m,path", [(33, 1024, 4096, "stream"), (96, 1024, 4096, "stream"), (128, 1024, 4096, "prefill"),
                                         (64, 1024, 11008, "tall"), (65, 1024, 11008, "prefill"),
-                                        (192, 4096, 4096, "stream"), (193, 4096, 4096, "prefill")])
+                                        (64, 4096, 4096, "stream"), (65, 4096, 4096, "prefill")])
 def test_token_counts_above_32_run_as_chunks_where_that_is_estimated_faster(T, n, m, path):
     # one prologue, then chunks of 32 tokens through the small-batch kernels (a ragged last chunk) while
-    # chunks x (3 + 0.45e-6 m n) us stays below the estimate for the tensor-core kernel, 0.017 n us per wave
+    # chunks x (3 + 0.45e-6 m n) us stays below the estimate for the tensor-core kernels (per 64-column stage and wave)
     d = lopro.make_desc(n, m, 4, 128, 128, identity_cols=128, rank=16)
     got, launches = lopro.linear_fwd_path(d, T)
     assert lopro.PATH_NAMES[got] == path
