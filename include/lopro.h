@@ -94,7 +94,9 @@ typedef struct {
  *   FP8: the record Algorithm 1 saves, (U, V, Sigma, s): U [m][r] and V [r][n] in fp8 e4m3 (Sec. 3.3 casts the unit
  *   vectors of every R1SVD step to fp8), Sigma [r] and the activation scale s [n] in fp16;
  *   y_lr = U (Sigma (V (x / s))).  Half the bytes per factor entry (Appendix A.2: about 0.05 bit per weight at r = 16).
- *   Served by the small-batch kernels of LOPRO_LAYOUT_FRAGMENT (any T: more than 32 tokens run as chunks of 32). */
+ *   Served by the small-batch kernels of LOPRO_LAYOUT_FRAGMENT; with more than 32 tokens either as chunks of 32 through
+ *   them or, where the tensor-core path is estimated faster, by that path after the record has been folded into fp16
+ *   factors in the workspace (A = fp16(U Sigma), B = fp16(V / s): one more rounding per factor entry, one more launch). */
 enum { LOPRO_LOWRANK_FOLDED_F16 = 0, LOPRO_LOWRANK_FP8 = 1 };
 
 /* Sections of the packed blob, for lopro_packed_section. */
@@ -238,9 +240,10 @@ LOPRO_API lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* pack
  *   LOPRO_PATH_WIDE     the same with the 32-warp variant of the streaming kernel (T <= 8, all of K in the ring)
  *   LOPRO_PATH_TALL     the same with the persistent streaming kernel for layers with many output rows
  *   LOPRO_PATH_GENERAL  rotation, B x, register-ring product (any shape the descriptor allows)
- *   LOPRO_PATH_PREFILL  rotation, B x (2 launches), tcgen05 product, T > 32
+ *   LOPRO_PATH_PREFILL  rotation, B x (2 launches), tcgen05 product (one CTA per tile, or two with a launch more
+ *                       where the last wave's tiles are cut along K), T > 32
  * For T a little above 32, where the library estimates it to be faster than the tensor-core path (layers with
- * few output rows; e.g. up to 192 tokens for 4096 x 4096), the forward runs as chunks of 32 tokens through the
+ * few output rows; e.g. up to 64 tokens for 4096 x 4096), the forward runs as chunks of 32 tokens through the
  * small-batch kernels: STREAM or TALL with one prologue launch and one launch per chunk.
  * Returns the path (> 0) and stores the number of kernel launches in *launches (may be NULL), or
  * returns 0 for a bad descriptor or T < 1. */

@@ -76,6 +76,14 @@ lopro_status workspace_layout(const lopro_desc& d, int T, WorkspaceLayout* W) {
     if (T > kDecodeMaxT && d.rank > 0) off += round_up_size(lowrank_mma_scratch_bytes(d, T), 256);
     W->off_kparts = off;
     off += round_up_size(prefill_kparts_bytes(d, T), 256);
+    // FP8 low-rank record on the tensor-core path: the fp16 factors it is folded into
+    W->off_fold_a = W->off_fold_b = off;
+    if (d.lowrank_format == LOPRO_LOWRANK_FP8 && T > kDecodeMaxT) {
+        W->off_fold_a = off;
+        off += round_up_size((size_t)d.d_out * r_pad * 2, 256);
+        W->off_fold_b = off;
+        off += round_up_size((size_t)r_pad * d.d_in * 2, 256);
+    }
     // operand image of the tcgen05 small-batch kernel (row-block layout)
     W->np = T <= 16 ? 16 : 32;
     W->n_tgroups = T <= 16 ? 1 : (T + 31) / 32;
@@ -342,7 +350,8 @@ static bool use_tall(const lopro_desc& d, int T) {
 // 96, 77 against 84).  LOPRO_OPT_NO_CHUNKS turns this off (A/B runs, tests of the prefill kernels on small layers).
 static int small_batch_chunks(const lopro_desc& d, int T) {
     if (T <= kDecodeMaxT) return 0;
-    if (d.lowrank_format == LOPRO_LOWRANK_FP8)  // served by the small-batch kernels only: always chunks
+    // the FP8 low-rank record has no general path: chunks wherever the tensor-core kernels cannot take the layer
+    if (d.lowrank_format == LOPRO_LOWRANK_FP8 && !prefill_supported(d, T))
         return (prologue_supported(d, kDecodeMaxT) && stream_supported(d, kDecodeMaxT)) ? (T + kDecodeMaxT - 1) / kDecodeMaxT : 0;
     if (option(LOPRO_OPT_NO_CHUNKS) == 1) return 0;
     if (!prefill_supported(d, T)) return 0;  // keep the general path's behaviour where there is no prefill kernel
@@ -387,6 +396,7 @@ int32_t lopro_linear_fwd_path(const lopro_desc* desc, int32_t T, int32_t* launch
                             : 1 + (desc->rank > 0 ? (T > kDecodeMaxT ? 2 : 1) : 0);
         path = prefill_supported(*desc, T) ? LOPRO_PATH_PREFILL : LOPRO_PATH_GENERAL;
         n = pre + 1;
+        if (desc->lowrank_format == LOPRO_LOWRANK_FP8) ++n;  // the record folded into fp16 factors
         if (path == LOPRO_PATH_PREFILL) {
             bool use_pairs = false;
             (void)prefill_estimate_us(*desc, T, &use_pairs);
@@ -484,6 +494,18 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
         if (e != cudaSuccess) return LOPRO_ERR_CUDA;
         return LOPRO_OK;
     }
+    const void* a_f16 = nullptr;  // the up factor where it is not the blob's section
+    if (desc->lowrank_format == LOPRO_LOWRANK_FP8) {
+        // More than 32 tokens on the tensor-core path (small_batch_chunks has sent every other case to the small-batch
+        // kernels): the record is folded into fp16 factors in the workspace, A = U Sigma and B = V / s, one rounding each.
+        if (!(T > kDecodeMaxT && prefill_supported(*desc, T))) return LOPRO_ERR_UNSUPPORTED;
+        __half* fa = (__half*)(ws + W.off_fold_a);
+        __half* fb = (__half*)(ws + W.off_fold_b);
+        if (launch_lr8_fold(*desc, L.r_pad, blob + L.off[LOPRO_SEC_A], lr8.V, lr8.sigma, lr8.svec, fa, fb, s) != cudaSuccess)
+            return LOPRO_ERR_CUDA;
+        B = fb;
+        a_f16 = fa;
+    }
     if (T > kDecodeMaxT && rotate_lowrank_supported(*desc, T)) {
         // many tokens: rotation and B x side by side in one grid, then the sum over K slices
         if (launch_rotate_lowrank(*desc, perm, (const __nv_bfloat16*)x_bf16, ldx, xrot, desc->d_in, s64, status, B, L.r_pad,
@@ -503,7 +525,7 @@ lopro_status lopro_linear_fwd(const lopro_desc* desc, const void* packed, const 
     }
     }
     if (prefill_supported(*desc, T)) {
-        if (launch_prefill(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+        if (launch_prefill(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s, a_f16) != cudaSuccess) return LOPRO_ERR_CUDA;
         return LOPRO_OK;
     }
     if (launch_decode(*desc, blob, L, ws, W, y, ldy, out_dtype, T, s) != cudaSuccess) return LOPRO_ERR_CUDA;

@@ -74,7 +74,7 @@ inline size_t round_up_size(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // activations, low-rank intermediate (fp16, general path), per-chunk partial sums of the low-rank
 // intermediate (fp32, small-batch path).
 struct WorkspaceLayout {
-    size_t off_status, off_xrot, off_s64, off_t, off_lrpart, off_kparts, total;
+    size_t off_status, off_xrot, off_s64, off_t, off_lrpart, off_kparts, off_fold_a, off_fold_b, total;
     int t_pad;  // tokens padded to a multiple of 8
     // row-block layout only: the operand image of the tcgen05 small-batch kernel (see ImageOut)
     size_t off_counters, off_ximg, off_sums, off_timg, off_partial;
@@ -225,8 +225,12 @@ PairPlan pair_plan(const lopro_desc& d, int T);
 size_t prefill_kparts_bytes(const lopro_desc& d, int T);
 // Estimated duration (microseconds) of the tensor-core product for T > 32 tokens and whether it runs two CTAs per tile
 double prefill_estimate_us(const lopro_desc& d, int T, bool* use_pairs);
+// FP8 low-rank record -> fp16 factors A = U Sigma [m][r_pad], B = V / s [r_pad][n] in the workspace (tensor-core path)
+cudaError_t launch_lr8_fold(const lopro_desc& d, int r_pad, const uint8_t* U, const uint8_t* V, const __half* sigma,
+                            const __half* svec, __half* A, __half* B, cudaStream_t s);
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s);
+                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s,
+                           const void* a_f16 = nullptr);  // a_f16: the up factor where it is not the blob's section
 
 // ---- fragment layout ----------------------------------------------------------------------
 // Codes are stored per tile of 16 rows x 64 columns as [32 lanes][q words].  Lane l = 4 gq + tg

@@ -275,6 +275,44 @@ cudaError_t launch_rotate_lowrank_nj(const lopro_desc& d, const int32_t* perm, c
 
 }  // namespace
 
+namespace {
+
+// The FP8 low-rank record folded for the tensor-core path: A[i][j] = fp16(U[i][j] sigma[j]) (the product of a 4-bit and an
+// 11-bit significand is exact in fp32: one rounding), B[j][k] = fp16(V[j][k] / s[k]) (IEEE single division, then one
+// rounding).  Two entries per thread; r_pad and n are even.
+__global__ void __launch_bounds__(256)
+lr8_fold_kernel(const uint8_t* __restrict__ U, const uint8_t* __restrict__ V, const __half* __restrict__ sigma,
+                const __half* __restrict__ svec, __half* __restrict__ A, __half* __restrict__ B, size_t pairs_a, int r_pad,
+                size_t pairs_b, int n) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < pairs_a) {
+        const uint32_t h2 = e4m3x2_to_f16x2(reinterpret_cast<const uint16_t*>(U)[i]);
+        const float2 u = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+        const int j = (int)((2 * i) % (size_t)r_pad);
+        reinterpret_cast<__half2*>(A)[i] = __floats2half2_rn(u.x * __half2float(sigma[j]), u.y * __half2float(sigma[j + 1]));
+    } else if (i - pairs_a < pairs_b) {
+        const size_t b = i - pairs_a;
+        const uint32_t h2 = e4m3x2_to_f16x2(reinterpret_cast<const uint16_t*>(V)[b]);
+        const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+        const int k = (int)((2 * b) % (size_t)n);
+        reinterpret_cast<__half2*>(B)[b] =
+            __floats2half2_rn(__fdiv_rn(v.x, __half2float(svec[k])), __fdiv_rn(v.y, __half2float(svec[k + 1])));
+    }
+}
+
+}  // namespace
+
+// A plain launch (not a programmatic one): the buffers it writes may still be read by the tensor-core kernel of the
+// previous forward on this stream.
+cudaError_t launch_lr8_fold(const lopro_desc& d, int r_pad, const uint8_t* U, const uint8_t* V, const __half* sigma,
+                            const __half* svec, __half* A, __half* B, cudaStream_t s) {
+    const size_t pairs_a = (size_t)d.d_out * r_pad / 2, pairs_b = (size_t)r_pad * d.d_in / 2;
+    const size_t blocks = (pairs_a + pairs_b + 255) / 256;
+    if (blocks > 0x7fffffffull) return cudaErrorInvalidValue;
+    lr8_fold_kernel<<<(unsigned)blocks, 256, 0, s>>>(U, V, sigma, svec, A, B, pairs_a, r_pad, pairs_b, d.d_in);
+    return cudaGetLastError();
+}
+
 bool rotate_lowrank_supported(const lopro_desc& d, int T) {
     const int r_pad = round_up_int(d.rank, 16);
     return d.rank > 0 && r_pad <= kLrMaxRank && T >= 256 && d.block_size <= 256 && d.identity_cols % 64 == 0 &&

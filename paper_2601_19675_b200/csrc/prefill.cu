@@ -908,7 +908,9 @@ double prefill_estimate_us(const lopro_desc& d, int T, bool* use_pairs) {
 }
 
 cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
-                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s) {
+                           const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s,
+                           const void* a_f16) {
+    const void* const a_src = a_f16 != nullptr ? a_f16 : (const void*)(blob + L.off[LOPRO_SEC_A]);
     PrefillParams p;
     p.codes = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_CODES]);
     p.sz = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_SCALEZERO]);
@@ -960,7 +962,7 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
         qa = qx;
         qt = qx;
         if (q.r_pad > 0) {
-            if (!make_map(&qa, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, blob + L.off[LOPRO_SEC_A], (uint64_t)q.r_pad, (uint64_t)d.d_out,
+            if (!make_map(&qa, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, a_src, (uint64_t)q.r_pad, (uint64_t)d.d_out,
                           (uint32_t)kTileM) ||
                 !make_map(&qt, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ws + W.off_t, (uint64_t)q.r_pad, (uint64_t)T, 128u))
                 return cudaErrorInvalidValue;
@@ -977,7 +979,7 @@ cudaError_t launch_prefill(const lopro_desc& d, const uint8_t* blob, const BlobL
     ma = mx;
     mt = mx;
     if (p.r_pad > 0) {
-        if (!make_map(&ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, blob + L.off[LOPRO_SEC_A], (uint64_t)p.r_pad, (uint64_t)d.d_out,
+        if (!make_map(&ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, a_src, (uint64_t)p.r_pad, (uint64_t)d.d_out,
                       (uint32_t)kTileM) ||
             !make_map(&mt, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, ws + W.off_t, (uint64_t)p.r_pad, (uint64_t)T, (uint32_t)p.tile_n))
             return cudaErrorInvalidValue;

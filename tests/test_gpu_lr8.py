@@ -7,6 +7,7 @@ import torch
 from oracle import lopro_oracle as o
 from paper_2601_19675_b200 import lopro, synth
 from tests._layers import bf16_bits_to_device, device_bf16_to_f64, random_layer_np
+from tests.test_gpu_forward import _gate_b_with_ties
 
 pytestmark = pytest.mark.gpu
 
@@ -30,6 +31,33 @@ def _oracle_args(layer, rec, d, rows=None):
                 v=o.e4m3_bits_to_f64(rec["V"]), s=o.f16_bits_to_f64(rec["s"]), g=d.group_size, b_i=d.identity_cols, b_h=d.block_size)
 
 
+def _gate_b_with_t_ties(x64, folded, mirrored, got_f32):
+    """Gate B when an entry of t = B x sits on an fp16 rounding boundary.  The kernel adds the products of a row of B
+    in fp32 (tile by tile), the oracle in fp64; an entry of the exact t within the fp32 summation error of the midpoint
+    of two fp16 values (here: 64 * 2^-24 * sum_k |B[j,k] x[k]|) may round to either side, which moves the token's
+    outputs by (other - chosen) * A[:, j] -- visible where the rank-r term dominates y.  Everything here comes from the
+    oracle; a flip is kept only if it lowers the token's error (greedy witness search, as for the bf16 ties of the
+    rotated activations)."""
+    a, b = folded["a"], folded["b"]
+    t_exact = x64 @ b.T
+    slack = 64.0 * 2.0 ** -24 * (np.abs(x64) @ np.abs(b).T)
+    chosen = o.round_f16(t_exact)
+    step = np.maximum(np.abs(chosen), 2.0 ** -14) * 2.0 ** -10
+    other = np.where(t_exact > chosen, o.round_f16(chosen + step), np.where(t_exact < chosen, o.round_f16(chosen - step), chosen))
+    near = (other != chosen) & (np.abs(t_exact - 0.5 * (chosen + other)) <= slack)
+    worst = 0.0
+    for tok in range(x64.shape[0]):
+        y = mirrored[tok].copy()
+        best = o.max_rel_err(got_f32[tok:tok + 1], y[None, :])
+        for j in np.flatnonzero(near[tok]):
+            y_alt = y + (other[tok, j] - chosen[tok, j]) * a[:, j]
+            e = o.max_rel_err(got_f32[tok:tok + 1], y_alt[None, :])
+            if e < best:
+                y, best = y_alt, e
+        worst = max(worst, best)
+    return worst
+
+
 def _check(d, layer, rec, x_bits, rows=None):
     blob = _pack(d, layer, rec)
     x = bf16_bits_to_device(x_bits)
@@ -42,12 +70,26 @@ def _check(d, layer, rec, x_bits, rows=None):
     args = _oracle_args(layer, rec, d, rows)
     x64 = o.bf16_bits_to_f64(x_bits)
     exact = o.forward_exact_unfolded(x64, **args)
-    mirrored = o.forward_mirrored_unfolded(x64, **args, round_t="f16", out="f32")
+    if lopro.linear_fwd_path(d, T)[0] == lopro.PATH_PREFILL:
+        # tensor-core path: the record is folded into fp16 factors first, A = U Sigma and B = V / s (one rounding each),
+        # and the dequantized weights are rounded to bf16
+        folded = {k: args[k] for k in ("codes", "scales", "zeros", "perm", "g", "b_i", "b_h")}
+        folded.update(a=o.round_f16(args["u"] * args["sigma"][None, :]), b=o.round_f16(args["v"] / args["s"][None, :]))
+        mirrored = o.forward_mirrored(x64, **folded, round_w=True, round_t="f16", out="f32")
+    else:
+        folded = None
+        mirrored = o.forward_mirrored_unfolded(x64, **args, round_t="f16", out="f32")
     got_bf, got_f32 = device_bf16_to_f64(y_bf), y_f32.cpu().numpy().astype(np.float64)
     if rows is not None:
         got_bf, got_f32 = got_bf[:, rows], got_f32[:, rows]
     assert o.max_rel_err(got_bf, exact) <= 2e-2
-    assert o.max_rel_err(got_f32, mirrored) <= 1e-3
+    err_b = o.max_rel_err(got_f32, mirrored)
+    if err_b > 1e-3 and folded is not None:
+        # a rotated entry within rounding distance of a bf16 tie may go to either side (see test_gpu_forward)
+        err_b = _gate_b_with_ties(x64, folded, True, mirrored, got_f32)
+    if err_b > 1e-3 and folded is not None:
+        err_b = _gate_b_with_t_ties(x64, folded, mirrored, got_f32)
+    assert err_b <= 1e-3
     # the low-rank branch is not negligible in these layers: dropping it would fail the gate
     no_lr = dict(args, sigma=np.zeros_like(args["sigma"]))
     assert o.max_rel_err(o.forward_exact_unfolded(x64, **no_lr), exact) > 5e-2
@@ -126,11 +168,28 @@ def test_forward_with_the_fp8_record(T, bits, g, r, m):
     rec["sigma"] = synth.f32_to_f16_bits(np.float32(40.0) * o.f16_bits_to_f64(rec["sigma"]).astype(np.float32))
     d = lopro.make_desc(n, m, bits, g, 128, rank=r, lowrank_format=lopro.LOWRANK_FP8)
     path, launches = lopro.linear_fwd_path(d, T)
-    assert path in (lopro.PATH_WIDE, lopro.PATH_STREAM, lopro.PATH_TALL)
-    if T > 32:
+    assert path in (lopro.PATH_WIDE, lopro.PATH_STREAM, lopro.PATH_TALL) or (T > 32 and path == lopro.PATH_PREFILL)
+    if T > 32 and path != lopro.PATH_PREFILL:
         assert launches == 1 + (T + 31) // 32
     rows = None if m * n <= 1 << 21 else np.arange(0, m, 5)
     _check(d, layer, rec, synth.activations(T, n, seed=T + 1, outlier_frac=0.01), rows=rows)
+
+
+@pytest.mark.parametrize("n,m,bits,g,r,T", [(1024, 256, 4, 128, 16, 300), (2048, 400, 3, 64, 33, 130), (1024, 384, 2, 64, 128, 700)])
+def test_many_tokens_with_the_fp8_record_run_on_the_tensor_core_kernels(n, m, bits, g, r, T):
+    # the record is folded into fp16 factors in the workspace (one more launch), then the same kernels as for a folded layer
+    layer = random_layer_np(n, m, bits, g, 0, seed=T + bits)
+    rec = synth.lowrank_record(m, n, r, seed=T + r)
+    rec["sigma"] = synth.f32_to_f16_bits(np.float32(40.0) * o.f16_bits_to_f64(rec["sigma"]).astype(np.float32))
+    d = lopro.make_desc(n, m, bits, g, 128, rank=r, lowrank_format=lopro.LOWRANK_FP8)
+    x_bits = synth.activations(T, n, seed=T + 1, outlier_frac=0.01)
+    with lopro.configured(lopro.OPT_NO_CHUNKS, 1):
+        assert lopro.linear_fwd_path(d, T)[0] == lopro.PATH_PREFILL
+        _check(d, layer, rec, x_bits)
+        with lopro.configured(lopro.OPT_NO_CTA_PAIRS, 1):
+            _check(d, layer, rec, x_bits)
+    # the library's own choice (chunks of 32 tokens or the tensor-core kernels) agrees with the oracle as well
+    _check(d, layer, rec, x_bits)
 
 
 def test_large_layer_with_the_fp8_record_and_its_byte_saving():
