@@ -336,9 +336,16 @@ lopro_status lopro_rotate(const lopro_desc* desc, const int32_t* perm, const uin
 }
 
 // LOPRO_OPT_NO_TALL keeps the persistent kernel for tall layers off (A/B comparison and tests of the other kernel).
-static bool use_tall(const lopro_desc& d, int T) {
+static bool use_tall(const lopro_desc& d, int T, long long total_rows = 0) {
     if (option(LOPRO_OPT_NO_TALL) == 1) return false;
-    return tall_supported(d, T);
+    return tall_supported(d, T, total_rows);
+}
+// Sibling layers that share their launches: the persistent kernel when their rows together make more than one wave of
+// the per-group kernel (three 4096-row projections do, each alone does not).
+static bool group_uses_tall(int32_t n, const lopro_desc* const* descs, int32_t T) {
+    long long rows = 0;
+    for (int i = 0; i < n; ++i) rows += descs[i]->d_out;
+    return use_tall(*descs[0], T, rows);
 }
 
 // Token counts a little above the small-batch range run as ONE prologue plus chunks of kDecodeMaxT tokens through
@@ -552,10 +559,11 @@ static bool group_shares_launches(int32_t n, const lopro_desc* const* descs, int
             d.lowrank_format != LOPRO_LOWRANK_FOLDED_F16)
             return false;
         if (!prologue_supported(d, T)) return false;
-        // all siblings through the persistent kernel or all through the per-group kernel
-        if (use_tall(d, T) != use_tall(d0, T)) return false;
-        if (!use_tall(d, T) && !stream_supported(d, T)) return false;
     }
+    // all siblings through the persistent kernel (by their rows together) or all through the per-group kernel
+    if (!group_uses_tall(n, descs, T))
+        for (int i = 0; i < n; ++i)
+            if (!stream_supported(*descs[i], T)) return false;
     return true;
 }
 
@@ -660,8 +668,9 @@ lopro_status lopro_linear_fwd_group(int32_t n_layers, const lopro_desc* const* d
                         L[0].r_pad, (const __nv_bfloat16*)x_bf16, ldx, ws + W.off_xrot, (__half*)(ws + W.off_t), W.t_pad,
                         (int*)(ws + W.off_status), T, s, nullptr, &ps) != cudaSuccess)
         return LOPRO_ERR_CUDA;
-    const cudaError_t e = use_tall(d0, T) ? launch_tall(d0, blob0, L[0], ws, W, y[0], ldy[0], out_dtype, T, s, 0, &ss)
-                                          : launch_stream(d0, blob0, L[0], ws, W, y[0], ldy[0], out_dtype, T, s, 0, &ss);
+    const cudaError_t e = group_uses_tall(n_layers, descs, T)
+                              ? launch_tall(d0, blob0, L[0], ws, W, y[0], ldy[0], out_dtype, T, s, 0, &ss)
+                              : launch_stream(d0, blob0, L[0], ws, W, y[0], ldy[0], out_dtype, T, s, 0, &ss);
     return e == cudaSuccess ? LOPRO_OK : LOPRO_ERR_CUDA;
 }
 

@@ -200,7 +200,7 @@ cudaError_t launch_stream(const lopro_desc& d, const uint8_t* blob, const BlobLa
                           const StreamSiblingArgs* more = nullptr);
 
 // Small-batch forward for tall layers after launch_prologue: persistent CTAs, one ring across tile groups.
-bool tall_supported(const lopro_desc& d, int T);
+bool tall_supported(const lopro_desc& d, int T, long long total_rows = 0);  // total_rows: of all siblings sharing the launch
 cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                         const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0 = 0,
                         const StreamSiblingArgs* more = nullptr);

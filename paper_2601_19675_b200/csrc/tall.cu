@@ -420,11 +420,15 @@ struct TallPlan {
     int off_a, a_bytes, off_t, off_red, off_ring, stage_bytes, off_stage_sz, off_stage_x, smem_bytes;
 };
 
-bool plan_tall(const lopro_desc& d, int T, TallPlan* pl) {
+// total_rows: rows of the layer, or of all the sibling layers that share the launch
+bool plan_tall(const lopro_desc& d, int T, TallPlan* pl, long long total_rows = 0) {
     if (T < 1 || T > kDecodeMaxT) return false;
     const int n_sm = sm_count();
-    const int tiles = d.d_out / 16;
-    if (tiles <= 2 * n_sm) return false;  // one wave of the per-group kernel holds the layer
+    const long long tiles = (total_rows > 0 ? total_rows : (long long)d.d_out) / 16;
+    // Up to two 16-row tiles per SM one wave of the per-group kernel holds the layer and is faster (4096 rows at 1 and 8
+    // tokens: 5.7 and 6.2 us against 7.4 and 8.4); with more than 16 tokens the persistent kernel wins from one tile
+    // per SM on (4096 rows 12.8 -> 12.5 us, 11008 -> 4096 27.6 -> 25.6).
+    if (tiles <= (T > 16 ? 1LL : 2LL) * n_sm) return false;
     const int r_pad = d.rank > 0 ? round_up_int(d.rank, 16) : 0;
     pl->nt = T <= 8 ? 1 : (T <= 16 ? 2 : 4);
     const int ktok = pl->nt * 8;
@@ -485,16 +489,19 @@ cudaError_t launch_tall_bits(const TallParams& p, const TallSiblings& sibs, int 
 
 }  // namespace
 
-bool tall_supported(const lopro_desc& d, int T) {
+bool tall_supported(const lopro_desc& d, int T, long long total_rows) {
     TallPlan pl;
-    return plan_tall(d, T, &pl);
+    return plan_tall(d, T, &pl, total_rows);
 }
 
 cudaError_t launch_tall(const lopro_desc& d, const uint8_t* blob, const BlobLayout& L, const uint8_t* ws,
                         const WorkspaceLayout& W, void* y, int64_t ldy, int out_dtype, int T, cudaStream_t s, int t0,
                         const StreamSiblingArgs* more) {
     TallPlan pl;
-    if (!plan_tall(d, T, &pl)) return cudaErrorInvalidValue;
+    long long total_rows = d.d_out;
+    if (more != nullptr)
+        for (int i = 0; i < more->n; ++i) total_rows += more->d_out[i];
+    if (!plan_tall(d, T, &pl, total_rows)) return cudaErrorInvalidValue;
     TallParams p;
     p.codes = blob + L.off[LOPRO_SEC_CODES];
     p.sz = reinterpret_cast<const uint32_t*>(blob + L.off[LOPRO_SEC_SCALEZERO]);

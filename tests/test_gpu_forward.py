@@ -255,9 +255,10 @@ def test_groups_as_long_as_or_longer_than_a_stage(g, T, m):
     _check_forward(layer, d, synth.activations(T, n, seed=T + g))
 
 
-@pytest.mark.parametrize("T,n,m,path", [(33, 1024, 4096, "stream"), (96, 1024, 4096, "stream"), (128, 1024, 4096, "prefill"),
+@pytest.mark.parametrize("T,n,m,path", [(33, 1024, 4096, "tall"), (96, 1024, 4096, "tall"), (128, 1024, 4096, "prefill"),
                                         (64, 1024, 11008, "tall"), (65, 1024, 11008, "prefill"),
-                                        (64, 4096, 4096, "stream"), (65, 4096, 4096, "prefill")])
+                                        (64, 4096, 4096, "tall"), (65, 4096, 4096, "prefill"),
+                                        (40, 2048, 2048, "stream")])
 def test_token_counts_above_32_run_as_chunks_where_that_is_estimated_faster(T, n, m, path):
     # one prologue, then chunks of 32 tokens through the small-batch kernels (a ragged last chunk) while
     # chunks x (3 + 0.45e-6 m n) us stays below the estimate for the tensor-core kernels (per 64-column stage and wave)
