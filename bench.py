@@ -784,7 +784,19 @@ def measure_vq(dev, peaks, reps=20):
     import torch
     from paper_2601_19675_b200 import lopro, synth
     n, m, cr, cc, b, r, ring = 8192, 28672, 512, 256, 256, 16, 3
-    d = lopro.make_vq_desc(n, m, cr, cc, b, rank=r)
+    out = {}
+    for dim in (4, 2):
+        _measure_vq_dim(dev, peaks, reps, out, n, m, cr, cc, b, r, ring, dim)
+    out["workload"] = ("vector-quantized record 8192 -> 28672: 8-bit indices of 4-D centroids (T1, T16) or 6-bit indices of 2-D "
+                       "centroids (dim2_T1, dim2_T16), codebooks of 512 x 256, block 256, rank 16")
+    return out
+
+
+def _measure_vq_dim(dev, peaks, reps, out, n, m, cr, cc, b, r, ring, dim):
+    import torch
+    from paper_2601_19675_b200 import lopro, synth
+    k = 256 if dim == 4 else 64
+    d = lopro.make_vq_desc(n, m, cr, cc, b, rank=r, dim=dim)
     gen = torch.Generator(device=dev)
     gen.manual_seed(4321)
     a_bits, b_bits = synth.factors(m, n, r, seed=9)
@@ -795,16 +807,16 @@ def measure_vq(dev, peaks, reps=20):
     perm = torch.from_numpy(synth.permutation(n, seed=9)).to(dev)
     blobs = []
     for _ in range(ring):
-        idx = torch.randint(0, 256, (m, n // 4), dtype=torch.uint8, device=dev, generator=gen)
-        books = (torch.randn((m // cr, n // cc, 256, 4), device=dev, generator=gen) * 0.02).to(torch.bfloat16).view(torch.int16)
+        idx = torch.randint(0, k, (m, n // dim), dtype=torch.uint8, device=dev, generator=gen)
+        books = (torch.randn((m // cr, n // cc, k, dim), device=dev, generator=gen) * 0.02).to(torch.bfloat16).view(torch.int16)
         blobs.append(lopro.vq_pack(d, idx, books, perm, dev16(a_bits), dev16(b_bits)))
     del idx, books
-    out = {}
     for T in (1, 16):
         x = dev16(synth.activations(T, n, seed=10)).view(torch.bfloat16)
         y = torch.empty((T, m), dtype=torch.bfloat16, device=dev)
         ws = torch.zeros(lopro.vq_workspace_bytes(d, T), dtype=torch.uint8, device=dev)
-        nbytes = m * (n // 4) + (m // cr) * (n // cc) * 2048 + (m * r + r * n) * 2 + n * 4 + T * (n + m) * 2
+        idx_bytes = m * (n // 4) if dim == 4 else m * (n // 8 * 3)
+        nbytes = idx_bytes + (m // cr) * (n // cc) * k * dim * 2 + (m * r + r * n) * 2 + n * 4 + T * (n + m) * 2
         stream = torch.cuda.Stream(device=dev)
         with torch.cuda.stream(stream):
             for blob in blobs:
@@ -824,11 +836,9 @@ def measure_vq(dev, peaks, reps=20):
             e1.record(stream)
             stream.synchronize()
         us = e0.elapsed_time(e1) * 1e3 / (reps * ring)
-        out[f"T{T}"] = dict(us_per_layer=us, tokens_per_s=T / (us * 1e-6), algorithmic_bytes=nbytes,
+        out[f"T{T}" if dim == 4 else f"dim2_T{T}"] = dict(us_per_layer=us, tokens_per_s=T / (us * 1e-6), algorithmic_bytes=nbytes,
                             achieved_gbs=nbytes / (us * 1e-6) / 1e9, frac_of_measured_hbm=nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
                             gpu_launches_per_layer=3)
-    out["workload"] = "vector-quantized record 8192 -> 28672: 8-bit indices of 4-D centroids, codebooks of 512 x 256, block 256, rank 16"
-    return out
 
 
 def measure_rotate(dev, peaks, reps=5):

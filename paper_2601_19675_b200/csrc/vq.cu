@@ -1,5 +1,6 @@
 // Vector-quantized residual (the vector variant of the method: a codebook of 256 four-dimensional centroids per group
-// of cb_rows x cb_cols rotated weights, one 8-bit index per four consecutive columns): packed record and forward.
+// of cb_rows x cb_cols rotated weights, one 8-bit index per four consecutive columns; or 64 two-dimensional centroids,
+// one 6-bit index per two columns, the 3-bit form): packed record and forward.
 // The forward is Eq. 8 with W^ looked up instead of dequantized: rotation and t = B x by the library's kernels, then
 // one product kernel per group of up to 32 tokens.
 #include "lopro_vq.h"
@@ -19,7 +20,12 @@ namespace {
 constexpr uint32_t kVqMagic = 0x5156504Cu;  // "LPVQ"
 constexpr int kVqHeader = 256;
 constexpr int kVqRowsPerCta = 64;           // four warps, sixteen rows each
-constexpr int kVqBookBytes = 256 * 4 * 2;   // one codebook
+constexpr int kVqBookBytes = 256 * 4 * 2;   // one codebook of 256 four-dimensional centroids
+constexpr int kVqBook2Bytes = 64 * 2 * 2;   // one codebook of 64 two-dimensional centroids
+inline int vq_dim(const lopro_vq_desc& d) { return d.dim == 0 ? 4 : d.dim; }
+inline int vq_book_bytes(int dim) { return dim == 4 ? kVqBookBytes : kVqBook2Bytes; }
+// bytes of a row's indices: one byte per four columns, or 6 bits per two columns
+inline size_t vq_idx_row_bytes(size_t n, int dim) { return dim == 4 ? n / 4 : n / 8 * 3; }
 // codebooks per shared-memory buffer (two buffers): 6 with one token tile (24 KB, seven CTAs per SM, so that two waves
 // hold the grid of a 28672-row layer), 8 otherwise (the registers of the wider variants allow five CTAs per SM anyway)
 constexpr int kVqSectionMax = 8;
@@ -38,6 +44,7 @@ lopro_status vq_check(const lopro_vq_desc* d) {
     if (d->identity_cols < 0 || d->identity_cols > d->d_in || (d->d_in - d->identity_cols) % d->block_size)
         return LOPRO_ERR_INVALID_ARG;
     if (d->rank < 0 || d->rank > 512 || d->d_in % d->cb_cols) return LOPRO_ERR_INVALID_ARG;
+    if (d->dim != 0 && d->dim != 2 && d->dim != 4) return LOPRO_ERR_INVALID_ARG;
     if (d->d_in % 64 || d->d_out % kVqRowsPerCta || d->cb_rows % kVqRowsPerCta || d->cb_cols % 64) return LOPRO_ERR_UNSUPPORTED;
     if (d->d_in > 32768 || d->d_out > (1 << 20)) return LOPRO_ERR_UNSUPPORTED;
     return LOPRO_OK;
@@ -55,8 +62,8 @@ VqLayout vq_layout(const lopro_vq_desc& d) {
         off += round_up_size(bytes, 256);
         return at;
     };
-    L.off_idx = take(m * (n / 4));
-    L.off_books = take((size_t)L.n_rg * L.n_cg * kVqBookBytes);
+    L.off_idx = take(m * vq_idx_row_bytes(n, vq_dim(d)));
+    L.off_books = take((size_t)L.n_rg * L.n_cg * vq_book_bytes(vq_dim(d)));
     L.off_perm = take(n * 4);
     L.off_a = take(m * (size_t)L.r_pad * 2);
     L.off_b = take((size_t)L.r_pad * n * 2);
@@ -111,6 +118,19 @@ __global__ void vq_perm_check_kernel(const int32_t* __restrict__ perm, int n, ui
     }
     const uint32_t bit = 1u << (p & 31);
     if (atomicOr(bitmap + (p >> 5), bit) & bit) *flag = 1;
+}
+
+// 6-bit indices, one per byte -> the packed bit stream: four indices (24 bits) per thread; an index of 64 or more
+// raises the flag and is reduced modulo 64
+__global__ void vq_pack6_kernel(const uint8_t* __restrict__ idx, size_t quads, uint8_t* __restrict__ out, int* flag) {
+    const size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= quads) return;
+    const uchar4 v = reinterpret_cast<const uchar4*>(idx)[q];
+    if ((v.x | v.y | v.z | v.w) & 0xC0) *flag = 1;
+    const uint32_t w = (v.x & 63u) | ((v.y & 63u) << 6) | ((v.z & 63u) << 12) | ((v.w & 63u) << 18);
+    out[3 * q] = (uint8_t)w;
+    out[3 * q + 1] = (uint8_t)(w >> 8);
+    out[3 * q + 2] = (uint8_t)(w >> 16);
 }
 
 __global__ void vq_identity_perm_kernel(int32_t* __restrict__ perm, int n) {
@@ -175,8 +195,8 @@ __global__ void __launch_bounds__(256) vq_lowrank_down_kernel(const __half* __re
 }
 
 struct VqParams {
-    const uint8_t* idx;          // [m][n / 4]
-    const unsigned char* books;  // [n_rg][n_cg][256][4] bf16
+    const uint8_t* idx;          // [m][n / 4] bytes, or [m] rows of n / 2 six-bit indices
+    const unsigned char* books;  // [n_rg][n_cg][256][4] or [n_rg][n_cg][64][2] bf16
     const __half* A;             // [m][r_pad]
     const __nv_bfloat16* xrot;   // [T][n] rotated activations of this launch's tokens
     const __half* t;             // [T][r_pad]
@@ -195,8 +215,12 @@ struct VqParams {
 // KS = 4: the four warps share ONE 16-row tile and take every fourth super-tile each (grid = m / 16; four times the
 // warps per SM for the same registers per warp, which is what hides the lookup latency); their sums meet in shared
 // memory at the end.  KS = 1: a warp per tile over all of K (grid = m / 64).
-template <int NT, int KS>
+// DIM = 2 (64 two-dimensional centroids, 6-bit indices): the lane's 16 columns of a super-tile are eight vectors, 48 bits
+// of the row's index stream starting at bit 48 t -- two 32-bit words from the 4-byte boundary below, shifted by 16 bits
+// for odd t --, and product s uses the vectors 2 s (k-slots 2t, 2t+1) and 2 s + 1 (k-slots 2t+8, 2t+9).
+template <int NT, int KS, int DIM>
 __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
+    constexpr int kBook = DIM == 4 ? kVqBookBytes : kVqBook2Bytes;
     extern __shared__ __align__(16) unsigned char vq_smem[];  // two sections of p.section codebooks
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int row0 = KS == 1 ? blockIdx.x * kVqRowsPerCta + warp * 16 : blockIdx.x * 16;
@@ -205,13 +229,13 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
     // The row group's codebooks pass through shared memory in sections of p.section books, the next section copied
     // asynchronously while the warps work on the present one (a CTA then holds 32 KB instead of all its books, and
     // every CTA of a large layer is resident at once).
-    const unsigned char* books_g = p.books + (size_t)rg * p.n_cg * kVqBookBytes;
+    const unsigned char* books_g = p.books + (size_t)rg * p.n_cg * kBook;
     const int n_sections = (p.n_cg + p.section - 1) / p.section;
     auto copy_section = [&](int sec) {
         const int first = sec * p.section, cnt = min(p.section, p.n_cg - first);
-        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(vq_smem) + (uint32_t)((sec & 1) * p.section * kVqBookBytes);
-        const unsigned char* src = books_g + (size_t)first * kVqBookBytes;
-        for (int i = tid; i < cnt * (kVqBookBytes / 16); i += 128)
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(vq_smem) + (uint32_t)((sec & 1) * p.section * kBook);
+        const unsigned char* src = books_g + (size_t)first * kBook;
+        for (int i = tid; i < cnt * (kBook / 16); i += 128)
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * (uint32_t)i), "l"(src + 16 * (size_t)i) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -221,13 +245,18 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[nt][e] = 0.0f;
-    const uint32_t* idx_lo = reinterpret_cast<const uint32_t*>(p.idx + (size_t)(row0 + g) * (p.n / 4)) + t;
-    const uint32_t* idx_hi = reinterpret_cast<const uint32_t*>(p.idx + (size_t)(row0 + g + 8) * (p.n / 4)) + t;
+    // DIM 4: word t of the super-tile's four index words; DIM 2: the word that holds bit 48 t of its six
+    const size_t row_bytes = DIM == 4 ? (size_t)(p.n / 4) : (size_t)(p.n / 8 * 3);
+    const int word0 = DIM == 4 ? t : (6 * t) >> 2;
+    constexpr int kWordsPerSuper = DIM == 4 ? 4 : 6;
+    const uint32_t* idx_lo = reinterpret_cast<const uint32_t*>(p.idx + (size_t)(row0 + g) * row_bytes) + word0;
+    const uint32_t* idx_hi = reinterpret_cast<const uint32_t*>(p.idx + (size_t)(row0 + g + 8) * row_bytes) + word0;
     const int n_super = p.n >> 6, per_book = p.cb_cols >> 6;
     // Everything a super-tile needs from global memory -- one word of indices per row and 32 bytes of every token's
     // rotated row -- is requested one super-tile ahead and kept in registers meanwhile (two register stages).
     struct Stage {
         uint32_t w_lo, w_hi;
+        uint32_t w_lo2, w_hi2;  // DIM 2: the second word of the lane's 48 bits
         uint4 xa[NT], xb[NT];
     };
     const uint4* xptr[NT];
@@ -239,8 +268,12 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
         xptr[nt] = reinterpret_cast<const uint4*>(p.xrot + (size_t)(live[nt] ? tok : 0) * p.n + 16 * t);
     }
     auto fetch = [&](Stage& st, int S) {
-        st.w_lo = __ldg(idx_lo + 4 * S);
-        st.w_hi = __ldg(idx_hi + 4 * S);
+        st.w_lo = __ldg(idx_lo + kWordsPerSuper * S);
+        st.w_hi = __ldg(idx_hi + kWordsPerSuper * S);
+        if (DIM == 2) {
+            st.w_lo2 = __ldg(idx_lo + kWordsPerSuper * S + 1);
+            st.w_hi2 = __ldg(idx_hi + kWordsPerSuper * S + 1);
+        }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             st.xa[nt] = live[nt] ? __ldg(xptr[nt] + 8 * S) : make_uint4(0, 0, 0, 0);
@@ -253,16 +286,29 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
     auto consume = [&](const Stage& st) {
         while (in_book >= per_book) {  // the codebook of this super-tile
             in_book -= per_book;
-            book += kVqBookBytes;
+            book += kBook;
         }
         // all eight centroids first (32-bit shared-space addresses; the loads keep their place before the products),
         // then the products
         const uint32_t bk = smem_s + book;
         uint32_t a[4][4];
+        if (DIM == 4) {
 #pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[s][0]), "=r"(a[s][2]) : "r"(bk + 8u * ((st.w_lo >> (8 * s)) & 255u)));
-            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[s][1]), "=r"(a[s][3]) : "r"(bk + 8u * ((st.w_hi >> (8 * s)) & 255u)));
+            for (int s = 0; s < 4; ++s) {
+                asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[s][0]), "=r"(a[s][2]) : "r"(bk + 8u * ((st.w_lo >> (8 * s)) & 255u)));
+                asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(a[s][1]), "=r"(a[s][3]) : "r"(bk + 8u * ((st.w_hi >> (8 * s)) & 255u)));
+            }
+        } else {
+            const int sh = (t & 1) * 16;
+            const unsigned long long v_lo = (((unsigned long long)st.w_lo2 << 32) | st.w_lo) >> sh;
+            const unsigned long long v_hi = (((unsigned long long)st.w_hi2 << 32) | st.w_hi) >> sh;
+#pragma unroll
+            for (int s = 0; s < 4; ++s) {
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(a[s][0]) : "r"(bk + 4u * ((uint32_t)(v_lo >> (12 * s)) & 63u)));
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(a[s][2]) : "r"(bk + 4u * ((uint32_t)(v_lo >> (12 * s + 6)) & 63u)));
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(a[s][1]) : "r"(bk + 4u * ((uint32_t)(v_hi >> (12 * s)) & 63u)));
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(a[s][3]) : "r"(bk + 4u * ((uint32_t)(v_hi >> (12 * s + 6)) & 63u)));
+            }
         }
 #pragma unroll
         for (int s = 0; s < 4; ++s)
@@ -287,7 +333,7 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
         __syncthreads();  // section sec has landed for every warp
-        book = (uint32_t)((sec & 1) * p.section * kVqBookBytes);
+        book = (uint32_t)((sec & 1) * p.section * kBook);
         in_book = kq;
         for (; S + KS < S_end; S += 2 * KS) {
             fetch(stB, S + KS);
@@ -352,8 +398,12 @@ __global__ void __launch_bounds__(128) vq_decode_kernel(const VqParams p) {
 }
 
 template <int NT>
-cudaError_t launch_vq_decode(const VqParams& p, cudaStream_t s) {
-    vq_decode_kernel<NT, 4><<<p.m / 16, 128, 2 * p.section * kVqBookBytes, s>>>(p);
+cudaError_t launch_vq_decode(const VqParams& p, int dim, cudaStream_t s) {
+    // two sections of codebooks; at the end the same memory holds the four warps' partial sums [4][NT][4][32] fp32
+    size_t smem = (size_t)2 * p.section * vq_book_bytes(dim);
+    if (smem < (size_t)4 * NT * 4 * 32 * 4) smem = (size_t)4 * NT * 4 * 32 * 4;
+    if (dim == 4) vq_decode_kernel<NT, 4, 4><<<p.m / 16, 128, smem, s>>>(p);
+    else vq_decode_kernel<NT, 4, 2><<<p.m / 16, 128, smem, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -392,9 +442,18 @@ lopro_status lopro_vq_pack(const lopro_vq_desc* desc, const uint8_t* idx, const 
     header[0] = kVqMagic;
     memcpy(header + 1, &d, sizeof(d));
     if (cudaMemcpyAsync(blob, header, kVqHeader, cudaMemcpyHostToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
-    if (cudaMemcpyAsync(blob + L.off_idx, idx, m * (n / 4), cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
-    if (cudaMemcpyAsync(blob + L.off_books, codebooks_bf16, (size_t)L.n_rg * L.n_cg * kVqBookBytes, cudaMemcpyDeviceToDevice, s) !=
-        cudaSuccess)
+    const int dim = vq_dim(d);
+    int* flag = (int*)(blob + 128);  // inside the header, zero so far
+    if (dim == 4) {
+        if (cudaMemcpyAsync(blob + L.off_idx, idx, m * (n / 4), cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
+    } else {
+        if (!aligned_to(idx, 4)) return LOPRO_ERR_INVALID_ARG;
+        const size_t quads = m * (n / 2) / 4;  // n is a multiple of 64: whole quads per row
+        vq_pack6_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, s>>>(idx, quads, blob + L.off_idx, flag);
+        if (cudaGetLastError() != cudaSuccess) return LOPRO_ERR_CUDA;
+    }
+    if (cudaMemcpyAsync(blob + L.off_books, codebooks_bf16, (size_t)L.n_rg * L.n_cg * vq_book_bytes(dim), cudaMemcpyDeviceToDevice,
+                        s) != cudaSuccess)
         return LOPRO_ERR_CUDA;
     if (cudaMemcpyAsync(blob + L.off_perm, perm, n * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LOPRO_ERR_CUDA;
     if (d.rank > 0) {
@@ -410,7 +469,6 @@ lopro_status lopro_vq_pack(const lopro_vq_desc* desc, const uint8_t* idx, const 
         (void)nb;
     }
     if (cudaMemsetAsync(blob + L.off_bitmap, 0, (n + 31) / 32 * 4, s) != cudaSuccess) return LOPRO_ERR_CUDA;
-    int* flag = (int*)(blob + 128);  // inside the header, zero so far
     vq_perm_check_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const int32_t*)(blob + L.off_perm), (int)n,
                                                                      (uint32_t*)(blob + L.off_bitmap), flag);
     if (cudaGetLastError() != cudaSuccess) return LOPRO_ERR_CUDA;
@@ -485,8 +543,11 @@ lopro_status lopro_vq_linear_fwd(const lopro_vq_desc* desc, const void* packed, 
         p.cb_rows = d.cb_rows;
         p.cb_cols = d.cb_cols;
         p.n_cg = L.n_cg;
-        p.section = tc <= 8 ? 6 : kVqSectionMax;
-        const cudaError_t e = tc <= 8 ? launch_vq_decode<1>(p, s) : (tc <= 16 ? launch_vq_decode<2>(p, s) : launch_vq_decode<4>(p, s));
+        const int dim = vq_dim(d);
+        // dim 2: the books are an eighth the size -- 32 per section hold the row group's books of most layers at once
+        p.section = dim == 4 ? (tc <= 8 ? 6 : kVqSectionMax) : (L.n_cg < 32 ? L.n_cg : 32);
+        const cudaError_t e = tc <= 8 ? launch_vq_decode<1>(p, dim, s)
+                                      : (tc <= 16 ? launch_vq_decode<2>(p, dim, s) : launch_vq_decode<4>(p, dim, s));
         if (e != cudaSuccess) return LOPRO_ERR_CUDA;
     }
     return LOPRO_OK;

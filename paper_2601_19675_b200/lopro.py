@@ -52,9 +52,10 @@ _lib = None
 
 
 class VqDesc(ctypes.Structure):
-    """lopro_vq_desc: the vector-quantized record (4-D centroids, 8-bit indices)."""
+    """lopro_vq_desc: the vector-quantized record (4-D centroids with 8-bit indices, or 2-D with 6-bit indices)."""
     _fields_ = [("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32), ("cb_rows", ctypes.c_int32), ("cb_cols", ctypes.c_int32),
-                ("block_size", ctypes.c_int32), ("identity_cols", ctypes.c_int32), ("rank", ctypes.c_int32)]
+                ("block_size", ctypes.c_int32), ("identity_cols", ctypes.c_int32), ("rank", ctypes.c_int32),
+                ("dim", ctypes.c_int32)]
 
 
 def lib():
@@ -427,8 +428,8 @@ def linear_fwd_experts(desc, blobs, row_offsets, x, out_dtype=OUT_BF16, workspac
     return y
 
 
-def make_vq_desc(d_in, d_out, cb_rows, cb_cols, block_size, identity_cols=None, rank=0):
-    return VqDesc(d_in, d_out, cb_rows, cb_cols, block_size, block_size if identity_cols is None else identity_cols, rank)
+def make_vq_desc(d_in, d_out, cb_rows, cb_cols, block_size, identity_cols=None, rank=0, dim=4):
+    return VqDesc(d_in, d_out, cb_rows, cb_cols, block_size, block_size if identity_cols is None else identity_cols, rank, dim)
 
 
 def vq_packed_bytes(desc):
@@ -440,7 +441,7 @@ def vq_workspace_bytes(desc, T):
 
 
 def vq_pack(desc, idx, codebooks_bf16, perm, A_f16=None, B_f16=None):
-    """lopro_vq_pack: idx uint8 [m][n/4], codebooks int16 bf16 bits [row groups][column groups][256][4], perm int32 [n],
+    """lopro_vq_pack: idx uint8 [m][n/dim], codebooks int16 bf16 bits [row groups][column groups][256 or 64][dim], perm int32 [n],
     A, B int16 fp16 bits (None with rank 0) -> packed device bytes."""
     nbytes = vq_packed_bytes(desc)
     if nbytes == 0:

@@ -78,3 +78,21 @@ def test_vq_storage_matches_the_printed_average_bits():
     assert 0.0 <= bits - val <= 0.0081
     assert o.vq_average_bits(4096, 4096, 4, 8, 16, 512, 256, 0, 8) == 2.125
     assert abs(o.vq_average_bits(4096, 4096, 4, 8, 16, 512, 256, 16, 8) - (2.125 + 2 * 16 * 8 / 4096)) < 1e-15
+    # the 3-bit form: 2-D centroids, 6-bit indices, 64 centroids per group of 512 x 256 -- 3 + 64 * 2 * 16 / 131072 bits
+    assert o.vq_average_bits(4096, 4096, 2, 6, 16, 512, 256, 0, 8) == 3.015625
+    assert abs(o.vq_average_bits(4096, 4096, 2, 6, 16, 512, 256, 16, 8) - (3.015625 + 2 * 16 * 8 / 4096)) < 1e-15
+
+
+def test_vq_quantize_with_two_dimensional_centroids_brute_force():
+    rng = np.random.default_rng(11)
+    m, n, dim, bits, cr, cc = 5, 12, 2, 6, 4, 6
+    rp = rng.standard_normal((m, n))
+    picks = [[rng.integers(0, 1000, size=2 ** bits) for _ in range(n // cc)] for _ in range(2)]
+    idx, books = o.vq_quantize(rp, dim, bits, cr, cc, picks)
+    assert idx.max() < 64 and books.shape == (2, 2, 64, 2)
+    for i in range(m):
+        for v in range(n // dim):
+            cb = books[i // cr][(dim * v) // cc]
+            d = [float(np.sum((rp[i, dim * v:dim * v + dim] - c) ** 2)) for c in cb]
+            assert idx[i, v] == int(np.argmin(d))
+
