@@ -376,3 +376,31 @@ def test_a_bounded_wait_that_runs_out_reports_a_timeout():
     y = lopro.linear_fwd(d, blob, torch.ones((4, n), dtype=torch.bfloat16, device="cuda"), workspace=ws)
     torch.cuda.synchronize()
     assert lopro.workspace_status(ws) == lopro.OK and torch.isfinite(y.float()).all()
+
+
+@pytest.mark.parametrize("n,m,bits,g,r,T", [
+    (4096, 4096, 4, 128, 32, 1), (4096, 4096, 4, 128, 32, 8), (2048, 272, 3, 64, 17, 32),     # small-batch kernels
+    (2048, 5008, 2, 64, 128, 16),                                                              # persistent kernel
+    (1024, 256, 4, 128, 16, 40), (1024, 4096, 4, 128, 16, 100),                               # chunks / tensor-core kernels
+    (1024, 512, 4, 64, 128, 300), (2048, 384, 3, 128, 40, 777),                               # K parts in the workspace
+])
+def test_nothing_is_written_outside_the_workspace_or_the_output(n, m, bits, g, r, T):
+    """Guard bytes behind the workspace (sized exactly by lopro_workspace_bytes) and behind every output row (ldy > m)
+    keep their pattern on every path; so does the packed layer (a forward only reads it)."""
+    layer = random_layer_np(n, m, bits, g, r, seed=n + T)
+    d = lopro.make_desc(n, m, bits, g, 128, identity_cols=128, rank=r)
+    blob = _pack(layer, d)
+    blob_before = blob.clone()
+    x = bf16_bits_to_device(synth.activations(T, n, seed=T))
+    need, guard, pad = lopro.workspace_bytes(d, T), 1 << 16, 24
+    for no_chunks in (0, 1):
+        with lopro.configured(lopro.OPT_NO_CHUNKS, no_chunks):
+            for out_dtype, tdt in ((lopro.OUT_BF16, torch.bfloat16), (lopro.OUT_F32, torch.float32)):
+                buf = torch.full((need + guard,), 0xA5, dtype=torch.uint8, device="cuda")
+                y = torch.full((T, m + pad), -7.0, dtype=tdt, device="cuda")
+                lopro.linear_fwd(d, blob, x, out_dtype, workspace=buf[:need], y=y[:, :m])
+                torch.cuda.synchronize()
+                assert lopro.workspace_status(buf) == lopro.OK
+                assert bool((buf[need:] == 0xA5).all())
+                assert bool((y[:, m:] == -7.0).all()) and bool(torch.isfinite(y[:, :m].float()).all())
+    assert torch.equal(blob, blob_before)
