@@ -561,7 +561,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
             const uint32_t full_a0 = map_to_cta(full_a(0), 0u), full_b0 = map_to_cta(full_b(0), 0u);
             const uint32_t b_bytes = (uint32_t)(2 * n_acc * kPairBHalf);  // both CTAs' copies of a stage
             int sa = 0, sb = 0;
-            uint32_t pa = 1, pb = 1;  // parity of the previous use's "empty" phase
+            uint32_t pa = 1;  // parity of the phase of the weight slot's previous use
             for (int i = 0; i < total; ++i) {
                 const int s = s_begin + i;  // stage of the layer; i counts the unit's stages (rings, parities)
                 // Weight stages: the first CTA's loader is one of the arrivals of full_a (so that the low-rank stages
@@ -591,10 +591,7 @@ prefill_pair_kernel(const PairParams p, const __grid_constant__ CUtensorMap map_
                     sa = 0;
                     pa ^= 1u;
                 }
-                if (++sb == kPairBStages) {
-                    sb = 0;
-                    pb ^= 1u;
-                }
+                if (++sb == kPairBStages) sb = 0;
             }
         }
     } else if ((warp == kDequantWarps + 1 || warp == kDequantWarps + 2) && rank == 0) {
