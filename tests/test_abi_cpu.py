@@ -84,8 +84,10 @@ def test_workspace_size_is_monotone_in_tokens():
     sizes = [lopro.workspace_bytes(d, t) for t in (0, 1, 7, 8, 9, 32, 33, 2048)]
     assert all(a <= b for a, b in zip(sizes, sizes[1:])) and sizes[0] > 0
     # every token count, on the shapes of the configurations (the prefill tiling's last wave shrinks and grows with T)
-    for n, m, bits, g, b, r in ((4096, 11008, 3, 64, 128, 64), (8192, 28672, 2, 64, 256, 128), (4096, 4096, 4, 128, 128, 32)):
+    for n, m, bits, g, b, r in ((4096, 11008, 3, 64, 128, 64), (8192, 28672, 2, 64, 256, 128), (4096, 4096, 4, 128, 128, 32),
+                                (32768, 1024, 4, 128, 256, 256), (4096, 4096, 4, 128, 128, 0), (8192, 8192, 2, 64, 256, 17)):
         dd = lopro.make_desc(n, m, bits, g, b, identity_cols=b, rank=r)
+        assert lopro.workspace_bytes(dd, 1) > 0
         prev = 0
         for t in range(0, 8193):
             cur = lopro.workspace_bytes(dd, t)
